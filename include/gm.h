@@ -1,0 +1,202 @@
+/*
+ * gm.h - C ABI of libgm: one speculative-decoding rollout step on one B200 (sm_100a).
+ *
+ * The step is the draft-then-verify cycle of the paper's Sec. 2.2: a recurrent one-layer MTP
+ * draft head (App. B.1 "MTP Architecture") proposes K tokens, the target decoder verifies all
+ * K+1 positions in one batched forward against a paged per-sequence KV cache, and speculative
+ * rejection sampling (Eq. 1) accepts a prefix and draws the final token from the corrected
+ * distribution norm(max(0, p - q)) or, on full acceptance, from p_{K+1}.
+ *
+ * Conventions
+ *  - Every pointer is a DEVICE pointer owned by the caller unless marked "host".  The library
+ *    owns only what gm_init allocates (workspaces, tensor maps, a status word) and frees it in
+ *    gm_destroy.  Nothing passed to a call is retained after the call's kernels are enqueued,
+ *    except the weight pointers given to gm_init, which must stay valid until gm_destroy.
+ *  - All work is enqueued on the CUDA stream given to gm_init.  Calls return after enqueueing;
+ *    gm_last_status is the only call that synchronises.
+ *  - Matrices are row-major bf16 [out_features, in_features].  Token ids, lengths, page ids are
+ *    int32.  Probabilities and debug dumps are fp32.
+ *  - Every call returns 0 or a negative GM_ERR_* code.  Arguments are validated on the host
+ *    before anything is launched.  Conditions only the device can see (a sequence that runs out
+ *    of pages, a page id outside the pool, a bounded wait that expired) set a sticky bit in the
+ *    device status word and the offending rows are skipped; gm_last_status reports it.
+ *
+ * Per-sequence state (struct gm_state).  The committed tokens are x[0..Len-1].  The target
+ * cache holds positions 0..Len-2 (kv_len = Len-1): the last committed token has not been fed to
+ * the target yet.  The head consumes pairs (H_{i-1}, x_i) - the target hidden state that
+ * produced token x_i and that token - and stores pair i at head-cache position i-1, so after
+ * the first draft application the head cache also holds positions 0..Len-2.  The pairs the head
+ * has not consumed yet are "pending": pending_n[b] of them (1 after a prefill, a+1 after a
+ * cycle that accepted a drafts), oldest first; pending_tok[b][pending_n[b]-1] is x[Len-1].
+ *
+ * KV pool layout: bf16 [layer][2 (K,V)][page][kv_head][16 slots][head_dim]; page_table[b][i] is
+ * the physical page of positions 16 i .. 16 i + 15 of sequence b.  Slots that were never
+ * written must hold finite values (zero-fill the pool once).
+ */
+#ifndef GM_H_
+#define GM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GM_OK                 0
+#define GM_ERR_INVALID_ARG   (-1)   /* null pointer, batch/k out of range, bad shape            */
+#define GM_ERR_UNSUPPORTED   (-2)   /* k > max_k, temperature <= 0, page_size != 16, vocab % 8  */
+#define GM_ERR_KV_CAPACITY   (-3)   /* a row's pages cannot hold kv_len + k + 1 (device-seen)   */
+#define GM_ERR_CUDA          (-4)   /* a CUDA runtime / driver call failed                      */
+#define GM_ERR_DEVICE_TIMEOUT (-5)  /* a bounded device-side wait expired (device-seen)         */
+#define GM_ERR_BAD_PAGE      (-6)   /* a page id outside the pool (device-seen)                 */
+#define GM_ERR_NO_EXTENSION  (-7)   /* not an sm_100 device                                     */
+
+#define GM_MAX_K 7
+#define GM_PAGE  16
+
+/* gm_config.flags */
+#define GM_FLAG_SIMPLE_GEMM 1       /* debug: route every GEMM through the plain mma.sync kernel */
+
+typedef struct gm_ctx gm_ctx;       /* opaque */
+
+typedef struct {
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  int32_t page_size;                /* must be 16                                        */
+  int32_t max_batch;                /* largest batch any call will use                   */
+  int32_t max_k;                    /* largest drafting depth, <= GM_MAX_K               */
+  int32_t max_pages_per_seq;        /* row length of both page tables                    */
+  int32_t num_pages;                /* physical pages in the target pool                 */
+  int32_t head_num_pages;           /* physical pages in the draft-head pool             */
+  float   rope_base;                /* rotary base (1e4)                                 */
+  float   rms_eps;                  /* RMSNorm epsilon (1e-6)                            */
+  int32_t flags;
+} gm_config;
+
+/* One decoder layer.  wqkv rows: all query heads, then all key heads, then all value heads.
+ * w_gate_up rows are interleaved: row 2i = gate_i, row 2i+1 = up_i.                       */
+typedef struct {
+  const void *ln1;                  /* [d]                                  */
+  const void *wqkv;                 /* [(n_q + 2 n_kv) head_dim, d]         */
+  const void *wo;                   /* [d, n_q head_dim]                    */
+  const void *ln2;                  /* [d]                                  */
+  const void *w_gate_up;            /* [2 d_ffn, d]                         */
+  const void *w_down;               /* [d, d_ffn]                           */
+} gm_layer_weights;
+
+/* Model weights (App. B.1: the head has neither embedding nor output projection and takes
+ * both from the backbone; its two inputs go through separate RMSNorms, are concatenated
+ * [embedding ; hidden] and projected by a bias-free linear layer).                       */
+typedef struct {
+  const void *embed;                /* [vocab, d]                           */
+  const void *lm_head;              /* [vocab, d]                           */
+  const void *final_norm;           /* [d]                                  */
+  const gm_layer_weights *layers;   /* HOST array [n_layers]                */
+  const void *head_enorm;           /* [d]   RMSNorm of the token embedding */
+  const void *head_hnorm;           /* [d]   RMSNorm of the hidden state    */
+  const void *head_proj;            /* [d, 2 d]                             */
+  const void *head_final_norm;      /* [d]                                  */
+  gm_layer_weights head_layer;
+} gm_weights;
+
+typedef struct {
+  int32_t  batch;                   /* B <= max_batch                                   */
+  int32_t *kv_len;                  /* [B]   entries in the target cache = Len - 1      */
+  int32_t *page_table;              /* [B, max_pages_per_seq]                           */
+  void    *kv_pool;                 /* bf16 [n_layers][2][num_pages][n_kv][16][hd]      */
+  int32_t *head_page_table;         /* [B, max_pages_per_seq]                           */
+  void    *head_kv_pool;            /* bf16 [1][2][head_num_pages][n_kv][16][hd]        */
+  int32_t *pending_n;               /* [B]   1 .. max_k+1                               */
+  int32_t *pending_tok;             /* [B, max_k+1]                                     */
+  void    *pending_hidden;          /* bf16 [B, max_k+1, d]                             */
+} gm_state;
+
+/* Create a context.  Validates the configuration, allocates workspaces sized for max_batch and
+ * max_k, encodes the weight tensor maps, builds the rotary table.  `cuda_stream` is a
+ * cudaStream_t (NULL = the default stream).  Fails with GM_ERR_NO_EXTENSION on a device that is
+ * not compute capability 10.x.                                                              */
+int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_stream);
+void gm_destroy(gm_ctx *ctx);
+
+/* Draft phase (App. E, restart equations).  Application 1 runs the head over the pending pairs,
+ * overwriting head-cache entries of the previous chain; applications 2..k feed the head its own
+ * output and the previous draft.  After each application q_j = softmax(logits / T) and d_j is
+ * drawn from q_j by the integer inverse CDF.
+ *   u24_draft  [B, k] 24-bit uniforms, or NULL to generate them from Philox4x32-10
+ *              (key = seed, counter = (slot >> 2, row, step lo, step hi), slot = j-1).
+ *   draft_tok  [B, k] out.   draft_logits bf16 [B, k, V] out.   dbg_q fp32 [B, k, V] out or NULL.
+ * Does not change kv_len / pending_*.                                                        */
+int gm_draft(gm_ctx *ctx, const gm_state *st, int k, float temperature,
+             const uint32_t *u24_draft, uint64_t seed, uint64_t step,
+             int32_t *draft_tok, void *draft_logits, float *dbg_q);
+
+/* Verify phase (Sec. 2.2, Eq. 2): target forward over [x[Len-1], d_1..d_k] at positions
+ * kv_len .. kv_len+k; appends their keys/values to the pages.
+ *   target_logits bf16 [B, k+1, V] out;  target_hidden bf16 [B, k+1, d] out (residual stream
+ *   before the final norm: the feature the head consumes).  Does not change kv_len.          */
+int gm_verify(gm_ctx *ctx, const gm_state *st, int k, const int32_t *draft_tok,
+              void *target_logits, void *target_hidden);
+
+/* Accept phase (Sec. 2.2, Eq. 1).  p_j = softmax(target_logits[j-1] / T), q_j likewise.
+ * d_j is accepted iff p_j(d_j) >= q_j(d_j) or fl32(u_j q_j(d_j)) < p_j(d_j), u_j = u24_j 2^-24;
+ * a = accepted prefix length; next_token is drawn from max(0, p_{a+1} - q_{a+1}) (a < k) or from
+ * p_{k+1} (a == k) through 64-bit integer weights: w[v] = trunc(r[v] 2^44) for r[v] > 0 else 0,
+ * W = sum w, t = (u24 W) >> 24, token = the first v whose inclusive prefix sum exceeds t.  If the
+ * residual quantises to nothing the draw is repeated on p_{a+1}.
+ *   u24_accept [B, k+1]: k accept uniforms then the final one; NULL = Philox slots 8+j-1 and 16.
+ *   accept_len [B] out (0..k), next_token [B] out.
+ *   dbg_p fp32 [B, k+1, V], dbg_q fp32 [B, k, V]: the probabilities the decisions used, or NULL.
+ *   commit_state != 0 (needs st and target_hidden): kv_len += a+1, pending_n = a+1,
+ *   pending_tok = d_1..d_a, next_token, pending_hidden = target_hidden rows 0..a.
+ *   With commit_state == 0, st and target_hidden may be NULL (sampler-only use).             */
+int gm_accept(gm_ctx *ctx, gm_state *st, int batch, int k, float temperature,
+              const void *target_logits, const void *draft_logits, const int32_t *draft_tok,
+              const uint32_t *u24_accept, uint64_t seed, uint64_t step,
+              int32_t *accept_len, int32_t *next_token,
+              float *dbg_p, float *dbg_q, const void *target_hidden, int commit_state);
+
+/* One whole cycle: gm_draft, gm_verify, gm_accept(commit_state = 1) on library-owned logit
+ * buffers, bit-for-bit the same as the three calls.  draft_tok [B, k] may be NULL.          */
+int gm_spec_step(gm_ctx *ctx, gm_state *st, int k, float temperature, uint64_t seed,
+                 uint64_t step, int32_t *accept_len, int32_t *next_token, int32_t *draft_tok);
+
+/* Draw one token per row from softmax(logits / T) by the integer inverse CDF (the draw of the
+ * draft phase as a stand-alone call).  logits bf16 [rows, V]; u24 [rows]; out_tok [rows];
+ * dbg_prob fp32 [rows, V] or NULL.                                                           */
+int gm_draw(gm_ctx *ctx, const void *logits, int rows, float temperature, const uint32_t *u24,
+            int32_t *out_tok, float *dbg_prob);
+
+/* Host-buffer form of the cycle: copies accept_len / next_token to HOST arrays and waits.   */
+int gm_spec_step_host(gm_ctx *ctx, gm_state *st, int k, float temperature, uint64_t seed,
+                      uint64_t step, int32_t *accept_len_host, int32_t *next_token_host);
+
+/* Dense projection out[M, N] = x[M, K] w[N, K]^T on the context's stream (bf16 in, fp32
+ * accumulate; the kernel every QKV / O / FFN / LM-head projection of the step uses).
+ *   out_fp32 != 0: out is fp32 [M, N]; else bf16 [M, N].  K % 64 == 0, N % 8 == 0, M >= 1.   */
+int gm_gemm(gm_ctx *ctx, const void *x, const void *w, void *out, int M, int N, int K,
+            int out_fp32);
+
+/* Kernel-class timing.  gm_profile(ctx, mask) makes later calls bracket every launch of the
+ * selected classes with CUDA events on the context's stream; gm_profile_read waits for the
+ * stream and returns the accumulated device time and launch count of one class since the
+ * last gm_profile call.                                                                     */
+#define GM_KC_GEMM       0
+#define GM_KC_ATTENTION  1
+#define GM_KC_ELEMENTWISE 2
+#define GM_KC_SAMPLER    3
+#define GM_KC_COUNT      4
+int gm_profile(gm_ctx *ctx, int class_mask);
+int gm_profile_read(gm_ctx *ctx, int kernel_class, double *total_ms, int64_t *launches);
+
+/* Number of kernels this library launched since gm_init (all calls).                        */
+int64_t gm_launch_count(gm_ctx *ctx);
+
+/* Waits for the stream and returns 0 or the GM_ERR_* of the first sticky device condition;
+ * clears the status word.                                                                   */
+int gm_last_status(gm_ctx *ctx);
+const char *gm_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GM_H_ */

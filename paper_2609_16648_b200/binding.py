@@ -1,0 +1,289 @@
+"""ctypes binding of libgm.so: the same entry points as include/gm.h, taking torch CUDA tensors.
+
+Argument marshalling only - every step of the path runs in the library's kernels.  PyTorch is used
+for device memory and streams.  Importing this module never falls back to a CPU path: if the
+shared library is missing or fails to load, `lib()` raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libgm.so")
+
+GM_OK = 0
+GM_ERR_INVALID_ARG, GM_ERR_UNSUPPORTED, GM_ERR_KV_CAPACITY, GM_ERR_CUDA = -1, -2, -3, -4
+GM_ERR_DEVICE_TIMEOUT, GM_ERR_BAD_PAGE, GM_ERR_NO_EXTENSION = -5, -6, -7
+GM_MAX_K, GM_PAGE = 7, 16
+GM_FLAG_SIMPLE_GEMM = 1
+GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER = 0, 1, 2, 3
+
+EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw",
+           "gm_spec_step_host", "gm_gemm", "gm_profile", "gm_profile_read", "gm_launch_count",
+           "gm_last_status", "gm_strerror"]
+
+
+class gm_config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn",
+                                          "vocab", "page_size", "max_batch", "max_k", "max_pages_per_seq",
+                                          "num_pages", "head_num_pages")] + \
+               [("rope_base", C.c_float), ("rms_eps", C.c_float), ("flags", C.c_int32)]
+
+
+class gm_layer_weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("ln1", "wqkv", "wo", "ln2", "w_gate_up", "w_down")]
+
+
+class gm_weights(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p),
+                ("layers", C.POINTER(gm_layer_weights)),
+                ("head_enorm", C.c_void_p), ("head_hnorm", C.c_void_p), ("head_proj", C.c_void_p),
+                ("head_final_norm", C.c_void_p), ("head_layer", gm_layer_weights)]
+
+
+class gm_state(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("kv_len", C.c_void_p), ("page_table", C.c_void_p), ("kv_pool", C.c_void_p),
+                ("head_page_table", C.c_void_p), ("head_kv_pool", C.c_void_p), ("pending_n", C.c_void_p),
+                ("pending_tok", C.c_void_p), ("pending_hidden", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libgm.so (built in-tree by paper_2609_16648_b200.build); raises if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2609_16648_b200.build` "
+                           "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, i32, u64, f32 = C.c_void_p, C.c_int, C.c_uint64, C.c_float
+    L.gm_init.argtypes = [C.POINTER(vp), C.POINTER(gm_config), C.POINTER(gm_weights), vp]
+    L.gm_destroy.argtypes = [vp]
+    L.gm_destroy.restype = None
+    L.gm_draft.argtypes = [vp, C.POINTER(gm_state), i32, f32, vp, u64, u64, vp, vp, vp]
+    L.gm_verify.argtypes = [vp, C.POINTER(gm_state), i32, vp, vp, vp]
+    L.gm_accept.argtypes = [vp, C.POINTER(gm_state), i32, i32, f32, vp, vp, vp, vp, u64, u64, vp, vp, vp, vp, vp, i32]
+    L.gm_spec_step.argtypes = [vp, C.POINTER(gm_state), i32, f32, u64, u64, vp, vp, vp]
+    L.gm_spec_step_host.argtypes = [vp, C.POINTER(gm_state), i32, f32, u64, u64, vp, vp]
+    L.gm_draw.argtypes = [vp, vp, i32, f32, vp, vp, vp]
+    L.gm_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
+    L.gm_profile.argtypes = [vp, i32]
+    L.gm_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    L.gm_launch_count.argtypes = [vp]
+    L.gm_launch_count.restype = C.c_int64
+    L.gm_last_status.argtypes = [vp]
+    L.gm_strerror.argtypes = [i32]
+    L.gm_strerror.restype = C.c_char_p
+    _lib = L
+    return L
+
+
+class GmError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {gm_strerror(code)} ({code})")
+
+
+def gm_strerror(code: int) -> str:
+    return lib().gm_strerror(code).decode()
+
+
+def _check(code: int, where: str):
+    if code != GM_OK:
+        raise GmError(code, where)
+
+
+def _p(t):
+    """Device pointer of a tensor (None -> NULL)."""
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "expected a contiguous CUDA tensor"
+    return C.c_void_p(t.data_ptr())
+
+
+# ---- weights ---------------------------------------------------------------------------------------------------
+
+def pack_layer(lw: dict, device) -> dict:
+    """Canonical per-projection matrices -> the library's fused layout (bf16 on `device`):
+    wqkv = [wq; wk; wv] stacked by rows, w_gate_up rows interleaved (2i = gate_i, 2i+1 = up_i)."""
+    bf = lambda a: torch.as_tensor(a).to(device=device, dtype=torch.bfloat16).contiguous()
+    wg, wu = torch.as_tensor(lw["wg"]), torch.as_tensor(lw["wu"])
+    return {
+        "ln1": bf(lw["ln1"]), "ln2": bf(lw["ln2"]),
+        "wqkv": bf(torch.cat([torch.as_tensor(lw["wq"]), torch.as_tensor(lw["wk"]), torch.as_tensor(lw["wv"])], 0)),
+        "wo": bf(lw["wo"]),
+        "w_gate_up": bf(torch.stack([wg, wu], 1).reshape(2 * wg.shape[0], wg.shape[1])),
+        "w_down": bf(lw["wd"]),
+    }
+
+
+def pack_weights(w: dict, device="cuda") -> dict:
+    bf = lambda a: torch.as_tensor(a).to(device=device, dtype=torch.bfloat16).contiguous()
+    return {
+        "embed": bf(w["embed"]), "lm_head": bf(w["lm_head"]), "final_norm": bf(w["final_norm"]),
+        "layers": [pack_layer(lw, device) for lw in w["layers"]],
+        "head": {"enorm": bf(w["head"]["enorm"]), "hnorm": bf(w["head"]["hnorm"]), "proj": bf(w["head"]["proj"]),
+                 "final_norm": bf(w["head"]["final_norm"]), "layer": pack_layer(w["head"]["layer"], device)},
+    }
+
+
+def random_packed_weights(cfg, device="cuda", seed=0, std=0.02) -> dict:
+    """Random weights generated directly on the device in the packed layout (large shapes)."""
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+
+    def rnd(*shape):
+        out = torch.empty(shape, device=device, dtype=torch.bfloat16)
+        rows = max(1, (1 << 26) // max(1, shape[-1]))
+        for r0 in range(0, shape[0], rows):          # in slabs, to bound the fp32 temporary
+            r1 = min(shape[0], r0 + rows)
+            out[r0:r1] = (torch.randn((r1 - r0,) + tuple(shape[1:]), device=device, generator=gen) * std).to(torch.bfloat16)
+        return out
+
+    ones = lambda n: torch.ones(n, device=device, dtype=torch.bfloat16)
+    d, f = cfg.d_model, cfg.d_ffn
+
+    def layer():
+        return {"ln1": ones(d), "ln2": ones(d), "wqkv": rnd(cfg.q_dim + 2 * cfg.kv_dim, d), "wo": rnd(d, cfg.q_dim),
+                "w_gate_up": rnd(2 * f, d), "w_down": rnd(d, f)}
+
+    return {"embed": rnd(cfg.vocab, d), "lm_head": rnd(cfg.vocab, d), "final_norm": ones(d),
+            "layers": [layer() for _ in range(cfg.n_layers)],
+            "head": {"enorm": ones(d), "hnorm": ones(d), "proj": rnd(d, 2 * d), "final_norm": ones(d),
+                     "layer": layer()}}
+
+
+def _layer_struct(lw: dict) -> gm_layer_weights:
+    return gm_layer_weights(*[lw[n].data_ptr() for n in ("ln1", "wqkv", "wo", "ln2", "w_gate_up", "w_down")])
+
+
+class Context:
+    """Owns a gm_ctx and keeps the weight tensors alive."""
+
+    def __init__(self, cfg, packed: dict, max_batch: int, max_k: int, max_pages_per_seq: int, num_pages: int,
+                 head_num_pages: int, flags: int = 0, stream=None):
+        self.cfg, self.packed = cfg, packed
+        self.max_batch, self.max_k, self.max_pages_per_seq = max_batch, max_k, max_pages_per_seq
+        self.num_pages, self.head_num_pages = num_pages, head_num_pages
+        self._layers = (gm_layer_weights * len(packed["layers"]))(*[_layer_struct(l) for l in packed["layers"]])
+        h = packed["head"]
+        self._w = gm_weights(packed["embed"].data_ptr(), packed["lm_head"].data_ptr(), packed["final_norm"].data_ptr(),
+                             self._layers, h["enorm"].data_ptr(), h["hnorm"].data_ptr(), h["proj"].data_ptr(),
+                             h["final_norm"].data_ptr(), _layer_struct(h["layer"]))
+        self._c = gm_config(len(packed["layers"]), cfg.d_model, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.d_ffn,
+                            cfg.vocab, cfg.page_size, max_batch, max_k, max_pages_per_seq, num_pages, head_num_pages,
+                            cfg.rope_base, cfg.rms_eps, flags)
+        self.stream = torch.cuda.current_stream() if stream is None else stream
+        self.handle = C.c_void_p()
+        _check(lib().gm_init(C.byref(self.handle), C.byref(self._c), C.byref(self._w),
+                             C.c_void_p(self.stream.cuda_stream)), "gm_init")
+
+    def close(self):
+        if self.handle:
+            lib().gm_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class State:
+    """Device tensors of struct gm_state."""
+
+    def __init__(self, ctx: Context, batch: int, page_table, head_page_table, device="cuda"):
+        cfg = ctx.cfg
+        i32 = dict(device=device, dtype=torch.int32)
+        self.batch = batch
+        self.kv_len = torch.zeros(batch, **i32)
+        self.page_table = torch.as_tensor(page_table).to(**i32).contiguous()
+        self.head_page_table = torch.as_tensor(head_page_table).to(**i32).contiguous()
+        assert self.page_table.shape == (batch, ctx.max_pages_per_seq) == self.head_page_table.shape
+        L = len(ctx.packed["layers"])
+        self.kv_pool = torch.zeros((L, 2, ctx.num_pages, cfg.n_kv_heads, 16, cfg.head_dim), device=device,
+                                   dtype=torch.bfloat16)
+        self.head_kv_pool = torch.zeros((1, 2, ctx.head_num_pages, cfg.n_kv_heads, 16, cfg.head_dim), device=device,
+                                        dtype=torch.bfloat16)
+        self.pending_n = torch.ones(batch, **i32)
+        self.pending_tok = torch.zeros((batch, ctx.max_k + 1), **i32)
+        self.pending_hidden = torch.zeros((batch, ctx.max_k + 1, cfg.d_model), device=device, dtype=torch.bfloat16)
+
+    def struct(self) -> gm_state:
+        return gm_state(self.batch, self.kv_len.data_ptr(), self.page_table.data_ptr(), self.kv_pool.data_ptr(),
+                        self.head_page_table.data_ptr(), self.head_kv_pool.data_ptr(), self.pending_n.data_ptr(),
+                        self.pending_tok.data_ptr(), self.pending_hidden.data_ptr())
+
+
+# ---- entry points (same names as the C ABI) ------------------------------------------------------------------------
+
+def gm_draft(ctx: Context, st: State, k: int, temperature: float, u24_draft, seed: int, step: int, draft_tok,
+             draft_logits, dbg_q=None):
+    s = st.struct()
+    _check(lib().gm_draft(ctx.handle, C.byref(s), k, temperature, _p(u24_draft), seed, step, _p(draft_tok),
+                          _p(draft_logits), _p(dbg_q)), "gm_draft")
+
+
+def gm_verify(ctx: Context, st: State, k: int, draft_tok, target_logits, target_hidden):
+    s = st.struct()
+    _check(lib().gm_verify(ctx.handle, C.byref(s), k, _p(draft_tok), _p(target_logits), _p(target_hidden)), "gm_verify")
+
+
+def gm_accept(ctx: Context, st, batch: int, k: int, temperature: float, target_logits, draft_logits, draft_tok,
+              u24_accept, seed: int, step: int, accept_len, next_token, dbg_p=None, dbg_q=None, target_hidden=None,
+              commit_state: bool = False):
+    s = st.struct() if st is not None else None
+    _check(lib().gm_accept(ctx.handle, C.byref(s) if s is not None else None, batch, k, temperature,
+                           _p(target_logits), _p(draft_logits), _p(draft_tok), _p(u24_accept), seed, step,
+                           _p(accept_len), _p(next_token), _p(dbg_p), _p(dbg_q), _p(target_hidden),
+                           1 if commit_state else 0), "gm_accept")
+
+
+def gm_spec_step(ctx: Context, st: State, k: int, temperature: float, seed: int, step: int, accept_len, next_token,
+                 draft_tok=None):
+    s = st.struct()
+    _check(lib().gm_spec_step(ctx.handle, C.byref(s), k, temperature, seed, step, _p(accept_len), _p(next_token),
+                              _p(draft_tok)), "gm_spec_step")
+
+
+def gm_spec_step_host(ctx: Context, st: State, k: int, temperature: float, seed: int, step: int, accept_len_host,
+                      next_token_host):
+    """accept_len_host / next_token_host: pinned (or pageable) CPU int32 tensors."""
+    s = st.struct()
+    assert not accept_len_host.is_cuda and not next_token_host.is_cuda
+    _check(lib().gm_spec_step_host(ctx.handle, C.byref(s), k, temperature, seed, step,
+                                   C.c_void_p(accept_len_host.data_ptr()), C.c_void_p(next_token_host.data_ptr())),
+           "gm_spec_step_host")
+
+
+def gm_draw(ctx: Context, logits, rows: int, temperature: float, u24, out_tok, dbg_prob=None):
+    _check(lib().gm_draw(ctx.handle, _p(logits), rows, temperature, _p(u24), _p(out_tok), _p(dbg_prob)), "gm_draw")
+
+
+def gm_gemm(ctx: Context, x, w, out, M: int, N: int, K: int, out_fp32: bool):
+    _check(lib().gm_gemm(ctx.handle, _p(x), _p(w), _p(out), M, N, K, 1 if out_fp32 else 0), "gm_gemm")
+
+
+def gm_profile(ctx: Context, class_mask: int):
+    _check(lib().gm_profile(ctx.handle, class_mask), "gm_profile")
+
+
+def gm_profile_read(ctx: Context, kernel_class: int):
+    ms, n = C.c_double(), C.c_int64()
+    _check(lib().gm_profile_read(ctx.handle, kernel_class, C.byref(ms), C.byref(n)), "gm_profile_read")
+    return ms.value, n.value
+
+
+def gm_launch_count(ctx: Context) -> int:
+    return lib().gm_launch_count(ctx.handle)
+
+
+def gm_last_status(ctx: Context) -> int:
+    return lib().gm_last_status(ctx.handle)

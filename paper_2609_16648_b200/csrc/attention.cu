@@ -1,0 +1,346 @@
+// Multi-query paged decode attention with grouped-query heads over ragged KV lengths.
+//
+// Work partition.  The pages every sequence attends are laid end to end (page_start is their
+// prefix sum) and cut into gridDim.x equal contiguous ranges, one per CTA, so every SM streams the
+// same number of bytes whatever the length mix.  A range may cover the tail of one sequence and
+// the head of the next: each (CTA, sequence) piece is a "segment" that yields an un-normalised
+// partial (max, sum, output); segment id = cta + sequence index, which is unique and consecutive
+// within a sequence.  A second kernel merges the segments of each sequence (log-sum-exp).
+//
+// Inside a CTA.  Warp h of the first HPC warps owns KV head h; one extra warp is the producer.
+// The producer walks the range page by page, looks the physical page up in the page table and
+// issues TMA tensor copies (128-byte swizzle) of that page's keys and values for all HPC heads
+// - 16 KB boxes, contiguous in the pool - into a ring of shared-memory stages guarded by
+// full/empty mbarriers.  A compute warp holds its (K+1) x group <= 16*MT query rows as mma.sync
+// A-fragments in registers, forms S = Q K^T for the page's 16 keys with m16n8k16 bf16 MMAs fed by
+// ldmatrix, runs the online softmax in registers (quad shuffles for the row statistics) and
+// accumulates O += P V with V fetched by ldmatrix.trans.  The 16-row M extent is why this is the
+// warp-level MMA and not tcgen05 (whose minimum M is 64).
+#include "common.cuh"
+#include "kernels.h"
+
+namespace gm {
+
+constexpr int ATT_MAX_HPC = 8;        // KV heads (= compute warps) per CTA
+constexpr int ATT_SMEM_BUDGET = 200 * 1024;
+
+template <int HD> struct AttCfg {
+  static constexpr int NSUB = HD / 64;                                   // 128-byte sub-tiles per row
+  static __host__ __device__ constexpr int tile_bytes(int hpc) { return hpc * 16 * 128; }       // one sub-tile
+  static __host__ __device__ constexpr int stage_bytes(int hpc) { return 2 * NSUB * tile_bytes(hpc); }
+};
+
+static int att_hpc(int n_kv) { return n_kv < ATT_MAX_HPC ? n_kv : ATT_MAX_HPC; }
+static int att_stages(int n_kv, int hd) {
+  const int sb = 2 * (hd / 64) * att_hpc(n_kv) * 16 * 128;
+  int s = ATT_SMEM_BUDGET / sb;
+  return s > 8 ? 8 : (s < 2 ? 2 : s);
+}
+size_t attention_smem_bytes(int n_kv, int hd) {
+  return static_cast<size_t>(att_stages(n_kv, hd)) * 2 * (hd / 64) * att_hpc(n_kv) * 16 * 128 + 1024 + 256;
+}
+int attention_max_ctas(int n_kv, int hd) {
+  (void)n_kv; (void)hd;
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  return sms;
+}
+
+// CTA that owns global page x when P pages are cut into G ranges [i*P/G, (i+1)*P/G).
+__device__ __forceinline__ int cta_of_page(long long x, long long P, long long G) {
+  return static_cast<int>(((x + 1) * G - 1) / P);
+}
+
+template <int HD, int MT>
+__global__ void __launch_bounds__((ATT_MAX_HPC + 1) * 32, 1)
+attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int nstages) {
+  using C = AttCfg<HD>;
+  constexpr int NSUB = C::NSUB;
+  constexpr int KSTEPS = HD / 16;
+  constexpr int NT = HD / 8;                    // 8-wide output column tiles
+
+  extern __shared__ unsigned char att_smem_raw[];
+  unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(att_smem_raw) + 1023) & ~uintptr_t(1023));
+  const int tile_b = C::tile_bytes(hpc);
+  const int stage_b = C::stage_bytes(hpc);
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem + static_cast<size_t>(nstages) * stage_b);
+  uint64_t *empty = full + 8;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int B = A.batch;
+  const long long G = gridDim.x;
+  const long long P = A.page_start[B];
+  const int lo = static_cast<int>(blockIdx.x * P / G), hi = static_cast<int>((blockIdx.x + 1) * P / G);
+  const int hg = blockIdx.y;                    // head group (n_kv > 8)
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < nstages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], hpc); }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (lo >= hi) return;
+
+  // first sequence of the range: largest b with page_start[b] <= lo
+  int b0 = 0;
+  {
+    int l = 0, r = B - 1;
+    while (l < r) { const int mid = (l + r + 1) >> 1; if (A.page_start[mid] <= lo) l = mid; else r = mid - 1; }
+    b0 = l;
+  }
+
+  if (warp == hpc) {
+    // ---- producer ------------------------------------------------------------------------------------------
+    if (lane == 0) {
+      tma_prefetch_desc(&A.kv_map);
+      int b = b0;
+      const long long rows_per_page = static_cast<long long>(A.n_kv) * 16;
+      for (int p = lo, it = 0; p < hi; ++p, ++it) {
+        while (p >= A.page_start[b + 1]) ++b;
+        int page = A.page_table[static_cast<size_t>(b) * A.max_pages_per_seq + (p - A.page_start[b])];
+        if (page < 0 || page >= A.num_pages) { set_status(A.status, ST_BAD_PAGE); page = 0; }
+        const int s = it % nstages;
+        if (!mbar_wait(&empty[s], ((it / nstages) & 1) ^ 1)) { set_status(A.status, ST_TIMEOUT); break; }
+        mbar_expect_tx(&full[s], stage_b);
+        unsigned char *dst = smem + static_cast<size_t>(s) * stage_b;
+        const long long row_k = ((static_cast<long long>(A.layer) * 2 + 0) * A.num_pages + page) * rows_per_page + hg * hpc * 16;
+        const long long row_v = ((static_cast<long long>(A.layer) * 2 + 1) * A.num_pages + page) * rows_per_page + hg * hpc * 16;
+#pragma unroll
+        for (int sub = 0; sub < NSUB; ++sub) {
+          tma_load_2d(dst + sub * tile_b, &A.kv_map, sub * 64, static_cast<int>(row_k), &full[s]);
+          tma_load_2d(dst + (NSUB + sub) * tile_b, &A.kv_map, sub * 64, static_cast<int>(row_v), &full[s]);
+        }
+      }
+    }
+    return;
+  }
+  if (warp > hpc) return;
+
+  // ---- compute warp: KV head = hg*hpc + warp -------------------------------------------------------------------
+  const int head = hg * hpc + warp;
+  const int t4 = lane & 3, r8 = lane >> 2;
+  const float c = A.scale_log2e;
+  const uint32_t smem_base = smem_u32(smem);
+  // per-lane ldmatrix offsets inside one 128-byte-row sub-tile (row index inside the warp's 16 rows)
+  const int mi = lane >> 3;
+  const int k_tok = (mi >> 1) * 8 + (lane & 7), k_chunk = mi & 1;        // K: non-transposed
+  const int v_tok = (mi & 1) * 8 + (lane & 7), v_chunk = mi >> 1;        // V: transposed
+  const uint32_t k_row_off = (warp * 16 + k_tok) * 128, v_row_off = (warp * 16 + v_tok) * 128;
+  const int k_sw = k_tok & 7, v_sw = v_tok & 7;
+
+  int it = 0;
+  bool dead = false;
+  for (int b = b0; b < B && !dead; ++b) {
+    const int ps = A.page_start[b], pe = A.page_start[b + 1];
+    if (ps >= hi) break;
+    const int seg_lo = max(lo, ps), seg_hi = min(hi, pe);
+    if (seg_lo >= seg_hi) continue;
+    const int qn = A.qn[b], qbase = A.qbase[b];
+
+    // query fragments
+    uint32_t qf[MT][KSTEPS][4];
+    const __nv_bfloat16 *qp = A.qbuf + (static_cast<size_t>(b) * A.n_kv + head) * A.qrows * HD;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+      for (int ks = 0; ks < KSTEPS; ++ks) {
+        const __nv_bfloat16 *r0 = qp + (mt * 16 + r8) * HD + ks * 16 + 2 * t4;
+        qf[mt][ks][0] = *reinterpret_cast<const uint32_t *>(r0);
+        qf[mt][ks][1] = *reinterpret_cast<const uint32_t *>(r0 + 8 * HD);
+        qf[mt][ks][2] = *reinterpret_cast<const uint32_t *>(r0 + 8);
+        qf[mt][ks][3] = *reinterpret_cast<const uint32_t *>(r0 + 8 * HD + 8);
+      }
+    float o[MT][NT][4];
+    float mrow[MT][2], lrow[MT][2];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+      mrow[mt][0] = mrow[mt][1] = -INFINITY;
+      lrow[mt][0] = lrow[mt][1] = 0.f;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) o[mt][nt][0] = o[mt][nt][1] = o[mt][nt][2] = o[mt][nt][3] = 0.f;
+    }
+
+    for (int p = seg_lo; p < seg_hi; ++p, ++it) {
+      const int s = it % nstages;
+      if (!mbar_wait(&full[s], (it / nstages) & 1)) { set_status(A.status, ST_TIMEOUT); dead = true; break; }
+      const uint32_t kbase = smem_base + s * stage_b, vbase = kbase + NSUB * tile_b;
+
+      float sc[MT][2][4];
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int n = 0; n < 2; ++n) sc[mt][n][0] = sc[mt][n][1] = sc[mt][n][2] = sc[mt][n][3] = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < KSTEPS; ++ks) {
+        uint32_t kf[4];
+        const int chunk = (ks & 3) * 2 + k_chunk;
+        ldmatrix_x4(kf, kbase + (ks >> 2) * tile_b + k_row_off + ((chunk ^ k_sw) << 4));
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          mma_16816(sc[mt][0], qf[mt][ks], kf[0], kf[1]);
+          mma_16816(sc[mt][1], qf[mt][ks], kf[2], kf[3]);
+        }
+      }
+
+      // causal / length mask: key position kp is visible to row r iff kp <= qbase + r/group and r/group < qn
+      const int kp0 = (p - ps) * 16;
+      const bool need_mask = kp0 + 15 > qbase;
+      uint32_t pa[MT][4];
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        if (need_mask) {
+#pragma unroll
+          for (int hrow = 0; hrow < 2; ++hrow) {
+            const int j = (mt * 16 + r8 + hrow * 8) / A.group;
+            const int lim = j < qn ? qbase + j : -1;
+#pragma unroll
+            for (int n = 0; n < 2; ++n)
+#pragma unroll
+              for (int e = 0; e < 2; ++e)
+                if (kp0 + n * 8 + 2 * t4 + e > lim) sc[mt][n][hrow * 2 + e] = -INFINITY;
+          }
+        }
+        float alpha[2];
+#pragma unroll
+        for (int hrow = 0; hrow < 2; ++hrow) {
+          float mx = fmaxf(fmaxf(sc[mt][0][hrow * 2], sc[mt][0][hrow * 2 + 1]),
+                           fmaxf(sc[mt][1][hrow * 2], sc[mt][1][hrow * 2 + 1]));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+          const float m_new = fmaxf(mrow[mt][hrow], mx);
+          const float m_use = m_new == -INFINITY ? 0.f : m_new;
+          alpha[hrow] = exp2f((mrow[mt][hrow] - m_use) * c);       // exp2(-inf) = 0 on the first page
+          mrow[mt][hrow] = m_new;
+          const float mc = m_use * c;
+          float rs = 0.f;
+#pragma unroll
+          for (int n = 0; n < 2; ++n)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const float pv = exp2f(fmaf(sc[mt][n][hrow * 2 + e], c, -mc));
+              sc[mt][n][hrow * 2 + e] = pv;
+              rs += pv;
+            }
+          lrow[mt][hrow] = lrow[mt][hrow] * alpha[hrow] + rs;
+        }
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          o[mt][nt][0] *= alpha[0]; o[mt][nt][1] *= alpha[0];
+          o[mt][nt][2] *= alpha[1]; o[mt][nt][3] *= alpha[1];
+        }
+        pa[mt][0] = pack_bf16(sc[mt][0][0], sc[mt][0][1]);
+        pa[mt][1] = pack_bf16(sc[mt][0][2], sc[mt][0][3]);
+        pa[mt][2] = pack_bf16(sc[mt][1][0], sc[mt][1][1]);
+        pa[mt][3] = pack_bf16(sc[mt][1][2], sc[mt][1][3]);
+      }
+
+      // O += P V
+#pragma unroll
+      for (int n2 = 0; n2 < NT / 2; ++n2) {
+        uint32_t vf[4];
+        const int chunk = (n2 & 3) * 2 + v_chunk;
+        ldmatrix_x4_trans(vf, vbase + (n2 >> 2) * tile_b + v_row_off + ((chunk ^ v_sw) << 4));
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          mma_16816(o[mt][2 * n2], pa[mt], vf[0], vf[1]);
+          mma_16816(o[mt][2 * n2 + 1], pa[mt], vf[2], vf[3]);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[s]);
+    }
+    if (dead) break;
+
+    // ---- write this segment's partial ----------------------------------------------------------------------
+    const size_t slot = static_cast<size_t>(blockIdx.x) + b;
+    float *po = A.part_o + ((slot * A.n_kv + head) * A.qrows) * HD;
+    float *pml = A.part_ml + ((slot * A.n_kv + head) * A.qrows) * 2;
+    const int rows_valid = qn * A.group;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+      for (int hrow = 0; hrow < 2; ++hrow) {
+        float l = lrow[mt][hrow];
+        l += __shfl_xor_sync(0xffffffffu, l, 1);
+        l += __shfl_xor_sync(0xffffffffu, l, 2);
+        const int row = mt * 16 + r8 + hrow * 8;
+        if (row < rows_valid) {
+          if (t4 == 0) {
+            pml[row * 2 + 0] = mrow[mt][hrow] == -INFINITY ? -INFINITY : mrow[mt][hrow] * c;
+            pml[row * 2 + 1] = l;
+          }
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+            *reinterpret_cast<float2 *>(po + static_cast<size_t>(row) * HD + nt * 8 + 2 * t4) =
+                make_float2(o[mt][nt][hrow * 2], o[mt][nt][hrow * 2 + 1]);
+        }
+      }
+  }
+}
+
+template <int HD, int MT>
+static cudaError_t launch_att(const AttnArgs &A, cudaStream_t stream) {
+  const int hpc = att_hpc(A.n_kv), nst = att_stages(A.n_kv, HD);
+  const size_t smem = attention_smem_bytes(A.n_kv, HD);
+  static size_t configured = 0;
+  if (smem > configured) {
+    cudaError_t e = cudaFuncSetAttribute(attention_kernel<HD, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    configured = smem;
+  }
+  dim3 grid(A.n_ctas, A.n_kv / hpc);
+  attention_kernel<HD, MT><<<grid, (hpc + 1) * 32, smem, stream>>>(A, hpc, nst);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attention(const AttnArgs &A, cudaStream_t stream) {
+  const int mt = A.qrows / 16;
+  if (A.n_kv % att_hpc(A.n_kv) != 0) return cudaErrorInvalidValue;
+  if (A.hd == 128 && mt == 1) return launch_att<128, 1>(A, stream);
+  if (A.hd == 128 && mt == 2) return launch_att<128, 2>(A, stream);
+  if (A.hd == 64 && mt == 1) return launch_att<64, 1>(A, stream);
+  if (A.hd == 64 && mt == 2) return launch_att<64, 2>(A, stream);
+  return cudaErrorInvalidValue;
+}
+
+// ---- merge the segments of each sequence ------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) attention_combine_kernel(const AttnCombineArgs A) {
+  const int b = blockIdx.x / A.n_kv, head = blockIdx.x % A.n_kv;
+  const int qn = A.qn[b];
+  const long long P = A.page_start[A.batch], G = A.n_ctas;
+  const int ps = A.page_start[b], pe = A.page_start[b + 1];
+  if (qn <= 0 || pe <= ps) return;
+  const int s_first = cta_of_page(ps, P, G) + b, s_last = cta_of_page(pe - 1, P, G) + b;
+  const int rows = qn * A.group, hd = A.hd;
+  for (int idx = threadIdx.x; idx < rows * (hd / 4); idx += blockDim.x) {
+    const int row = idx / (hd / 4), c4 = idx % (hd / 4);
+    float mt = -INFINITY;
+    for (int s = s_first; s <= s_last; ++s)
+      mt = fmaxf(mt, A.part_ml[((static_cast<size_t>(s) * A.n_kv + head) * A.qrows + row) * 2]);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float l = 0.f;
+    for (int s = s_first; s <= s_last; ++s) {
+      const size_t base = (static_cast<size_t>(s) * A.n_kv + head) * A.qrows + row;
+      const float ms = A.part_ml[base * 2];
+      if (ms == -INFINITY) continue;
+      const float w = exp2f(ms - mt);
+      l += w * A.part_ml[base * 2 + 1];
+      const float4 ov = reinterpret_cast<const float4 *>(A.part_o + base * hd)[c4];
+      acc.x += w * ov.x; acc.y += w * ov.y; acc.z += w * ov.z; acc.w += w * ov.w;
+    }
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+    const int j = row / A.group, g = row % A.group;
+    __nv_bfloat16 *dst = A.out + (static_cast<size_t>(b) * A.QT + j) * (A.n_kv * A.group * hd) +
+                         (static_cast<size_t>(head) * A.group + g) * hd + c4 * 4;
+    uint2 ov2;
+    ov2.x = pack_bf16(acc.x * inv, acc.y * inv);
+    ov2.y = pack_bf16(acc.z * inv, acc.w * inv);
+    *reinterpret_cast<uint2 *>(dst) = ov2;
+  }
+}
+cudaError_t launch_attention_combine(const AttnCombineArgs &A, cudaStream_t stream) {
+  attention_combine_kernel<<<A.batch * A.n_kv, 128, 0, stream>>>(A);
+  return cudaGetLastError();
+}
+
+}  // namespace gm

@@ -1,0 +1,314 @@
+// Memory-bound glue of the decoder: embedding gather, RMSNorm, rotary embedding + KV append,
+// SwiGLU, residual/split-K reduction, and the per-phase plan.  One CTA per token row; rows are
+// M = batch * QT with a fixed stride QT per sequence (rows j >= qn[b] are padding).
+#include "common.cuh"
+#include "kernels.h"
+
+namespace gm {
+
+constexpr int EW_THREADS = 256;
+constexpr int EW_MAXC = 8;            // float4 chunks per thread: rows up to 8192 wide
+
+__device__ __forceinline__ float block_sum(float v) {
+  __shared__ float red[EW_THREADS / 32];
+  __shared__ float total;
+  v = warp_sum(v);
+  __syncthreads();                    // protects `red`/`total` against a previous call
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float t = threadIdx.x < EW_THREADS / 32 ? red[threadIdx.x] : 0.f;
+    t = warp_sum(t);
+    if (threadIdx.x == 0) total = t;
+  }
+  __syncthreads();
+  return total;
+}
+
+// y = v * rsqrt(mean(v^2) + eps) * w, written as bf16; v holds this thread's chunks of the row.
+__device__ __forceinline__ void rmsnorm_store(const float4 (&v)[EW_MAXC], int d4, int d, float eps,
+                                              const __nv_bfloat16 *w, __nv_bfloat16 *out) {
+  float ss = 0.f;
+#pragma unroll
+  for (int c = 0; c < EW_MAXC; ++c) {
+    const int i = threadIdx.x + c * EW_THREADS;
+    if (i < d4) ss += v[c].x * v[c].x + v[c].y * v[c].y + v[c].z * v[c].z + v[c].w * v[c].w;
+  }
+  const float inv = rsqrtf(block_sum(ss) / static_cast<float>(d) + eps);
+#pragma unroll
+  for (int c = 0; c < EW_MAXC; ++c) {
+    const int i = threadIdx.x + c * EW_THREADS;
+    if (i < d4) {
+      const uint2 wv = *reinterpret_cast<const uint2 *>(w + 4 * i);
+      uint2 o;
+      o.x = pack_bf16(v[c].x * inv * bf16_lo(wv.x), v[c].y * inv * bf16_hi(wv.x));
+      o.y = pack_bf16(v[c].z * inv * bf16_lo(wv.y), v[c].w * inv * bf16_hi(wv.y));
+      *reinterpret_cast<uint2 *>(out + 4 * i) = o;
+    }
+  }
+}
+
+__device__ __forceinline__ float4 load_bf16x4(const __nv_bfloat16 *p) {
+  const uint2 r = *reinterpret_cast<const uint2 *>(p);
+  return make_float4(bf16_lo(r.x), bf16_hi(r.x), bf16_lo(r.y), bf16_hi(r.y));
+}
+
+// ---- plan -----------------------------------------------------------------------------------------------
+__global__ void plan_kernel(const PlanArgs A) {
+  __shared__ int pages[1024];
+  const int B = A.batch;
+  for (int b = threadIdx.x; b < B; b += blockDim.x) {
+    const int len = A.kv_len[b];
+    int qn, qbase;
+    if (A.mode == PHASE_VERIFY) { qn = A.k_or_j + 1; qbase = len; }
+    else if (A.mode == PHASE_DRAFT_FIRST) { qn = A.pending_n[b]; qbase = len - qn; }
+    else { qn = 1; qbase = len + A.k_or_j - 2; }
+    bool ok = qn >= 1 && qbase >= 0 && qbase + qn <= A.max_pages_per_seq * 16;
+    if (A.mode == PHASE_DRAFT_FIRST) ok = ok && qn <= A.k_or_j;     // k_or_j carries max_k + 1 here
+    if (!ok) { set_status(A.status, ST_KV_CAPACITY); qn = 0; qbase = 0; }
+    A.qn[b] = qn;
+    A.qbase[b] = qbase;
+    pages[b] = qn > 0 ? (qbase + qn + 15) >> 4 : 0;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int acc = 0;
+    for (int b = 0; b < B; ++b) { A.page_start[b] = acc; acc += pages[b]; }
+    A.page_start[B] = acc;
+  }
+}
+cudaError_t launch_plan(const PlanArgs &A, cudaStream_t stream) {
+  if (A.batch > 1024) return cudaErrorInvalidValue;
+  plan_kernel<<<1, 256, 0, stream>>>(A);
+  return cudaGetLastError();
+}
+
+// ---- embedding gather + first RMSNorm of the verify forward ------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS)
+embed_norm_kernel(const __nv_bfloat16 *embed, const __nv_bfloat16 *w, const int32_t *pending_tok,
+                  const int32_t *pending_n, const int32_t *draft_tok, int K, int max_k, int d, int vocab, float eps,
+                  float *x, __nv_bfloat16 *xn, uint32_t *status) {
+  const int m = blockIdx.x, b = m / (K + 1), j = m % (K + 1);
+  int tok;
+  if (j == 0) {
+    const int n = min(max(pending_n[b], 1), max_k + 1);
+    tok = pending_tok[b * (max_k + 1) + n - 1];
+  } else {
+    tok = draft_tok[b * K + j - 1];
+  }
+  if (tok < 0 || tok >= vocab) { if (threadIdx.x == 0) set_status(status, ST_BAD_TOKEN); tok = 0; }
+  const int d4 = d >> 2;
+  float4 v[EW_MAXC];
+#pragma unroll
+  for (int c = 0; c < EW_MAXC; ++c) {
+    const int i = threadIdx.x + c * EW_THREADS;
+    if (i < d4) {
+      v[c] = load_bf16x4(embed + static_cast<size_t>(tok) * d + 4 * i);
+      reinterpret_cast<float4 *>(x + static_cast<size_t>(m) * d)[i] = v[c];
+    }
+  }
+  rmsnorm_store(v, d4, d, eps, w, xn + static_cast<size_t>(m) * d);
+}
+cudaError_t launch_embed_norm(const __nv_bfloat16 *embed, const __nv_bfloat16 *w, const int32_t *pending_tok,
+                              const int32_t *pending_n, const int32_t *draft_tok, int batch, int K, int max_k, int d,
+                              int vocab, float eps, float *x, __nv_bfloat16 *xn, uint32_t *status,
+                              cudaStream_t stream) {
+  embed_norm_kernel<<<batch * (K + 1), EW_THREADS, 0, stream>>>(embed, w, pending_tok, pending_n, draft_tok, K, max_k,
+                                                                d, vocab, eps, x, xn, status);
+  return cudaGetLastError();
+}
+
+// ---- draft-head input: [RMSNorm_e(embedding) ; RMSNorm_h(hidden)] ---------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS) head_input_kernel(const HeadInputArgs A) {
+  const int m = blockIdx.x, b = m / A.QT, j = m % A.QT;
+  const int d = A.d, d4 = d >> 2;
+  __nv_bfloat16 *out = A.zin + static_cast<size_t>(m) * 2 * d;
+  int tok = 0;
+  bool valid = true;
+  const __nv_bfloat16 *hid_bf = nullptr;
+  const float *hid_f = nullptr;
+  if (A.mode == PHASE_DRAFT_FIRST) {
+    const int n = A.pending_n[b];
+    valid = j < n && n <= A.max_k + 1;
+    if (valid) {
+      tok = A.pending_tok[b * (A.max_k + 1) + j];
+      hid_bf = A.pending_hidden + (static_cast<size_t>(b) * (A.max_k + 1) + j) * d;
+    }
+  } else {
+    tok = A.draft_tok[b * A.k + A.j - 2];
+    hid_f = A.g_prev + static_cast<size_t>(b) * d;
+  }
+  if (!valid) {
+    for (int i = threadIdx.x; i < 2 * d4; i += EW_THREADS) reinterpret_cast<uint2 *>(out)[i] = make_uint2(0u, 0u);
+    return;
+  }
+  if (tok < 0 || tok >= A.vocab) { if (threadIdx.x == 0) set_status(A.status, ST_BAD_TOKEN); tok = 0; }
+  float4 v[EW_MAXC];
+#pragma unroll
+  for (int c = 0; c < EW_MAXC; ++c) {
+    const int i = threadIdx.x + c * EW_THREADS;
+    if (i < d4) v[c] = load_bf16x4(A.embed + static_cast<size_t>(tok) * d + 4 * i);
+  }
+  rmsnorm_store(v, d4, d, A.eps, A.we, out);
+#pragma unroll
+  for (int c = 0; c < EW_MAXC; ++c) {
+    const int i = threadIdx.x + c * EW_THREADS;
+    if (i < d4) v[c] = hid_bf ? load_bf16x4(hid_bf + 4 * i) : reinterpret_cast<const float4 *>(hid_f)[i];
+  }
+  rmsnorm_store(v, d4, d, A.eps, A.wh, out + d);
+}
+cudaError_t launch_head_input(const HeadInputArgs &A, cudaStream_t stream) {
+  head_input_kernel<<<A.batch * A.QT, EW_THREADS, 0, stream>>>(A);
+  return cudaGetLastError();
+}
+
+// ---- split-K reduction + residual add + RMSNorm -------------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS)
+reduce_residual_norm_kernel(const float *partial, int nsplit, size_t split_stride, float *x, int add_residual,
+                            const __nv_bfloat16 *w, __nv_bfloat16 *xn, __nv_bfloat16 *hidden_out, int d, float eps) {
+  const int m = blockIdx.x, d4 = d >> 2;
+  float4 v[EW_MAXC];
+#pragma unroll
+  for (int c = 0; c < EW_MAXC; ++c) {
+    const int i = threadIdx.x + c * EW_THREADS;
+    if (i < d4) {
+      float4 acc = add_residual ? reinterpret_cast<const float4 *>(x + static_cast<size_t>(m) * d)[i]
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int s = 0; s < nsplit; ++s) {
+        const float4 p = reinterpret_cast<const float4 *>(partial + s * split_stride + static_cast<size_t>(m) * d)[i];
+        acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+      }
+      v[c] = acc;
+      reinterpret_cast<float4 *>(x + static_cast<size_t>(m) * d)[i] = acc;
+      if (hidden_out) {
+        uint2 o;
+        o.x = pack_bf16(acc.x, acc.y);
+        o.y = pack_bf16(acc.z, acc.w);
+        *reinterpret_cast<uint2 *>(hidden_out + static_cast<size_t>(m) * d + 4 * i) = o;
+      }
+    }
+  }
+  if (xn) rmsnorm_store(v, d4, d, eps, w, xn + static_cast<size_t>(m) * d);
+}
+cudaError_t launch_reduce_residual_norm(const float *partial, int nsplit, size_t split_stride, float *x,
+                                        int add_residual, const __nv_bfloat16 *w, __nv_bfloat16 *xn,
+                                        __nv_bfloat16 *hidden_out, int M, int d, float eps, cudaStream_t stream) {
+  reduce_residual_norm_kernel<<<M, EW_THREADS, 0, stream>>>(partial, nsplit, split_stride, x, add_residual, w, xn,
+                                                            hidden_out, d, eps);
+  return cudaGetLastError();
+}
+
+// ---- rotary embedding + KV append + Q rearrangement --------------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS) rope_append_kernel(const RopeAppendArgs A) {
+  const int m = blockIdx.x, b = m / A.QT, j = m % A.QT;
+  const int hd = A.hd, half = hd >> 1, group = A.n_q / A.n_kv;
+  const int ncols = (A.n_q + 2 * A.n_kv) * hd;
+  const int qn = A.qn[b];
+  __nv_bfloat16 *qdst = A.qbuf + static_cast<size_t>(b) * A.n_kv * A.qrows * hd;
+  if (j >= qn) {                           // padding row: zero its query rows, append nothing
+    for (int i = threadIdx.x; i < A.n_q * hd; i += EW_THREADS) {
+      const int h = i / hd, e = i % hd;
+      qdst[(static_cast<size_t>(h / group) * A.qrows + j * group + h % group) * hd + e] = __float2bfloat16(0.f);
+    }
+    return;
+  }
+  const int pos = A.qbase[b] + j;
+  const int page = A.page_table[static_cast<size_t>(b) * A.max_pages_per_seq + (pos >> 4)];
+  const bool page_ok = page >= 0 && page < A.num_pages;
+  if (!page_ok && threadIdx.x == 0) set_status(A.status, ST_BAD_PAGE);
+  const float *src = A.qkv + static_cast<size_t>(m) * ncols;
+  auto val = [&](int col) {
+    float s = 0.f;
+    for (int sp = 0; sp < A.nsplit; ++sp) s += src[sp * A.split_stride + col];
+    return s;
+  };
+  const float2 *cs = A.rope + static_cast<size_t>(pos) * half;
+  const size_t page_elems = static_cast<size_t>(A.n_kv) * 16 * hd;
+  __nv_bfloat16 *kdst = A.pool + ((static_cast<size_t>(A.layer) * 2 + 0) * A.num_pages + page) * page_elems;
+  __nv_bfloat16 *vdst = A.pool + ((static_cast<size_t>(A.layer) * 2 + 1) * A.num_pages + page) * page_elems;
+  const int slot = pos & 15;
+  // rotate-half pairs of the query and key heads
+  const int npairs = (A.n_q + A.n_kv) * half;
+  for (int i = threadIdx.x; i < npairs; i += EW_THREADS) {
+    const int h = i / half, e = i % half;
+    const float x1 = val(h * hd + e), x2 = val(h * hd + e + half);
+    const float2 c = cs[e];
+    const float y1 = x1 * c.x - x2 * c.y, y2 = x2 * c.x + x1 * c.y;
+    if (h < A.n_q) {
+      __nv_bfloat16 *dst = qdst + (static_cast<size_t>(h / group) * A.qrows + j * group + h % group) * hd;
+      dst[e] = __float2bfloat16(y1);
+      dst[e + half] = __float2bfloat16(y2);
+    } else if (page_ok) {
+      __nv_bfloat16 *dst = kdst + (static_cast<size_t>(h - A.n_q) * 16 + slot) * hd;
+      dst[e] = __float2bfloat16(y1);
+      dst[e + half] = __float2bfloat16(y2);
+    }
+  }
+  if (page_ok) {
+    const int vbase = (A.n_q + A.n_kv) * hd;
+    for (int i = threadIdx.x; i < A.n_kv * hd; i += EW_THREADS) {
+      const int h = i / hd, e = i % hd;
+      vdst[(static_cast<size_t>(h) * 16 + slot) * hd + e] = __float2bfloat16(val(vbase + i));
+    }
+  }
+}
+cudaError_t launch_rope_append(const RopeAppendArgs &A, cudaStream_t stream) {
+  rope_append_kernel<<<A.batch * A.QT, EW_THREADS, 0, stream>>>(A);
+  return cudaGetLastError();
+}
+
+// ---- SwiGLU ---------------------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS)
+swiglu_kernel(const float *gu, int nsplit, size_t split_stride, __nv_bfloat16 *act, size_t total4) {
+  // one thread: 4 outputs = 8 interleaved inputs (gate, up, gate, up, ...)
+  for (size_t i = blockIdx.x * static_cast<size_t>(EW_THREADS) + threadIdx.x; i < total4;
+       i += static_cast<size_t>(gridDim.x) * EW_THREADS) {
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), c = a;
+    for (int s = 0; s < nsplit; ++s) {
+      const float4 *p = reinterpret_cast<const float4 *>(gu + s * split_stride) + 2 * i;
+      const float4 u = p[0], w = p[1];
+      a.x += u.x; a.y += u.y; a.z += u.z; a.w += u.w;
+      c.x += w.x; c.y += w.y; c.z += w.z; c.w += w.w;
+    }
+    auto f = [](float g, float u) { return g / (1.f + __expf(-g)) * u; };
+    uint2 o;
+    o.x = pack_bf16(f(a.x, a.y), f(a.z, a.w));
+    o.y = pack_bf16(f(c.x, c.y), f(c.z, c.w));
+    reinterpret_cast<uint2 *>(act)[i] = o;
+  }
+}
+cudaError_t launch_swiglu(const float *gu, int nsplit, size_t split_stride, __nv_bfloat16 *act, int M, int F,
+                          cudaStream_t stream) {
+  const size_t total4 = static_cast<size_t>(M) * F / 4;
+  size_t nb = (total4 + EW_THREADS - 1) / EW_THREADS;
+  if (nb > 148 * 8) nb = 148 * 8;
+  if (nb < 1) nb = 1;
+  swiglu_kernel<<<static_cast<int>(nb), EW_THREADS, 0, stream>>>(gu, nsplit, split_stride, act, total4);
+  return cudaGetLastError();
+}
+
+// ---- head output row: last valid row of each sequence + the head's final norm ----------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS)
+head_out_kernel(const float *x, const int32_t *qn, int QT, int d, const __nv_bfloat16 *w, float eps, float *g,
+                __nv_bfloat16 *gn) {
+  const int b = blockIdx.x, d4 = d >> 2;
+  const int j = min(max(qn[b], 1), QT) - 1;
+  const float4 *src = reinterpret_cast<const float4 *>(x + (static_cast<size_t>(b) * QT + j) * d);
+  float4 v[EW_MAXC];
+#pragma unroll
+  for (int c = 0; c < EW_MAXC; ++c) {
+    const int i = threadIdx.x + c * EW_THREADS;
+    if (i < d4) {
+      v[c] = src[i];
+      reinterpret_cast<float4 *>(g + static_cast<size_t>(b) * d)[i] = v[c];
+    }
+  }
+  rmsnorm_store(v, d4, d, eps, w, gn + static_cast<size_t>(b) * d);
+}
+cudaError_t launch_head_out(const float *x, const int32_t *qn, int batch, int QT, int d, const __nv_bfloat16 *w,
+                            float eps, float *g, __nv_bfloat16 *gn, cudaStream_t stream) {
+  head_out_kernel<<<batch, EW_THREADS, 0, stream>>>(x, qn, QT, d, w, eps, g, gn);
+  return cudaGetLastError();
+}
+
+}  // namespace gm

@@ -1,0 +1,654 @@
+// C ABI of libgm: context, workspaces, tensor maps and the launch sequences of the draft, verify and
+// accept phases.  Host code only; every step of the path runs in the kernels of this directory.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <new>
+#include <tuple>
+#include <vector>
+
+#include <cudaTypedefs.h>
+
+#include "../../include/gm.h"
+#include "common.cuh"
+#include "kernels.h"
+
+using namespace gm;
+
+namespace {
+
+struct LayerMaps { CUtensorMap wqkv, wo, wgu, wdown; };
+
+struct EventPair { cudaEvent_t a, b; };
+
+}  // namespace
+
+struct gm_ctx {
+  gm_config cfg;
+  gm_weights w;
+  std::vector<gm_layer_weights> layers;
+  cudaStream_t stream = nullptr;
+  int sm_count = 148;
+  PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+
+  // derived shapes
+  int d, q_dim, kv_dim, n_qkv, F, V, group, Mmax;
+
+  // tensor maps
+  std::vector<LayerMaps> lmaps;
+  LayerMaps head_maps;
+  CUtensorMap lm_head_map, head_proj_map;
+  std::map<std::tuple<const void *, int, int, int>, CUtensorMap> x_maps;   // (ptr, rows, K, box rows)
+  std::map<std::tuple<const void *, int, int>, CUtensorMap> w_maps;        // (ptr, N, K)   (gm_gemm only)
+  std::map<std::tuple<const void *, long long>, CUtensorMap> kv_maps;      // (pool, rows)
+
+  // workspaces (device)
+  float *x = nullptr, *part = nullptr, *g = nullptr, *part_o = nullptr, *part_ml = nullptr;
+  __nv_bfloat16 *xn = nullptr, *zin = nullptr, *qbuf = nullptr, *attn_out = nullptr, *act = nullptr, *gn = nullptr;
+  __nv_bfloat16 *ws_draft_logits = nullptr, *ws_target_logits = nullptr, *ws_target_hidden = nullptr;
+  int32_t *ws_draft_tok = nullptr, *ws_accept_len = nullptr, *ws_next_token = nullptr;
+  uint32_t *ws_u24 = nullptr;
+  int32_t *qn = nullptr, *qbase = nullptr, *page_start = nullptr;
+  float2 *rope = nullptr;
+  uint32_t *status = nullptr;
+  size_t part_elems = 0;
+  std::vector<void *> allocs;
+
+  // profiling
+  int prof_mask = 0;
+  std::vector<EventPair> events[GM_KC_COUNT];
+  size_t events_used[GM_KC_COUNT] = {0, 0, 0, 0};
+  int64_t launches = 0;
+  cudaError_t last_cuda = cudaSuccess;
+};
+
+namespace {
+
+#define GM_CUDA(ctx, call)                                   \
+  do {                                                       \
+    cudaError_t e__ = (call);                                \
+    if (e__ != cudaSuccess) { (ctx)->last_cuda = e__; return GM_ERR_CUDA; } \
+  } while (0)
+
+template <typename T>
+int dev_alloc(gm_ctx *c, T **p, size_t n, bool zero = true) {
+  void *q = nullptr;
+  GM_CUDA(c, cudaMalloc(&q, n * sizeof(T) > 0 ? n * sizeof(T) : 16));
+  c->allocs.push_back(q);
+  if (zero) GM_CUDA(c, cudaMemsetAsync(q, 0, n * sizeof(T), c->stream));
+  *p = static_cast<T *>(q);
+  return GM_OK;
+}
+
+struct Prof {
+  gm_ctx *c; int cls; bool on; EventPair ev{};
+  Prof(gm_ctx *c_, int cls_) : c(c_), cls(cls_), on((c_->prof_mask >> cls_) & 1) {
+    if (!on) return;
+    size_t &u = c->events_used[cls];
+    if (u == c->events[cls].size()) {
+      EventPair e;
+      cudaEventCreate(&e.a);
+      cudaEventCreate(&e.b);
+      c->events[cls].push_back(e);
+    }
+    ev = c->events[cls][u++];
+    cudaEventRecord(ev.a, c->stream);
+  }
+  ~Prof() {
+    if (on) cudaEventRecord(ev.b, c->stream);
+    c->launches++;
+  }
+};
+#define GM_LAUNCH(ctx, cls, call)           \
+  do {                                      \
+    cudaError_t e__;                        \
+    { Prof p__(ctx, cls); e__ = (call); }   \
+    if (e__ != cudaSuccess) { (ctx)->last_cuda = e__; return GM_ERR_CUDA; } \
+  } while (0)
+
+// 2-D bf16 tensor map: inner extent `cols` (contiguous), outer extent `rows`, box 64 x box_rows, 128-byte swizzle.
+int make_map(gm_ctx *c, CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = c->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? GM_OK : GM_ERR_CUDA;
+}
+
+int x_map(gm_ctx *c, const void *ptr, int rows, int K, int box_rows, CUtensorMap *out) {
+  auto key = std::make_tuple(ptr, rows, K, box_rows);
+  auto it = c->x_maps.find(key);
+  if (it == c->x_maps.end()) {
+    CUtensorMap m;
+    if (make_map(c, &m, ptr, rows, K, box_rows) != GM_OK) return GM_ERR_CUDA;
+    it = c->x_maps.emplace(key, m).first;
+  }
+  *out = it->second;
+  return GM_OK;
+}
+
+int kv_map(gm_ctx *c, const void *pool, int layers, int num_pages, CUtensorMap *out) {
+  const long long rows = static_cast<long long>(layers) * 2 * num_pages * c->cfg.n_kv_heads * 16;
+  auto key = std::make_tuple(pool, rows);
+  auto it = c->kv_maps.find(key);
+  if (it == c->kv_maps.end()) {
+    const int hpc = c->cfg.n_kv_heads < 8 ? c->cfg.n_kv_heads : 8;
+    CUtensorMap m;
+    if (make_map(c, &m, pool, rows, c->cfg.head_dim, hpc * 16) != GM_OK) return GM_ERR_CUDA;
+    it = c->kv_maps.emplace(key, m).first;
+  }
+  *out = it->second;
+  return GM_OK;
+}
+
+int round16(int v) { return (v + 15) & ~15; }
+
+// Split-K factor that fills the SMs when a projection has few output tiles.
+int pick_split(const gm_ctx *c, int M, int N, int K, int T) {
+  const int tiles = ((N + 127) / 128) * ((M + T - 1) / T);
+  if (tiles * 3 >= c->sm_count * 2) return 1;
+  int ns = c->sm_count / tiles;
+  const int KB = K / 64;
+  if (ns > KB) ns = KB;
+  if (ns > 16) ns = 16;
+  return ns < 1 ? 1 : ns;
+}
+
+// out = x[M, K] w[N, K]^T.  fp32 partials into c->part (returns the split count), or bf16 to `out_bf16`
+// with row stride ldo.
+int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *wmap, const __nv_bfloat16 *w, int M,
+             int N, int K, void *out, bool out_fp32, int *nsplit_out, size_t *split_stride_out) {
+  GemmArgs A;
+  std::memset(&A, 0, sizeof(A));
+  A.x = x; A.w = w; A.M = M; A.N = N; A.K = K; A.status = c->status;
+  A.out = out; A.out_fp32 = out_fp32 ? 1 : 0;
+  const bool simple = (c->cfg.flags & GM_FLAG_SIMPLE_GEMM) != 0 || (K % 64) != 0;
+  const int T = M >= 256 ? 256 : round16(M);
+  A.block_t = T;
+  A.nsplit = out_fp32 ? pick_split(c, M, N, K, T) : 1;
+  A.split_stride = static_cast<size_t>(M) * N;
+  A.ldo = N;
+  if (out_fp32 && A.split_stride * A.nsplit > c->part_elems && out == c->part) return GM_ERR_INVALID_ARG;
+  if (nsplit_out) *nsplit_out = A.nsplit;
+  if (split_stride_out) *split_stride_out = A.split_stride;
+  if (simple) {
+    GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_simple(A, c->stream));
+    return GM_OK;
+  }
+  A.w_map = *wmap;
+  int rc = x_map(c, x, x_rows, K, T, &A.x_map);
+  if (rc != GM_OK) return rc;
+  GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(A, c->stream));
+  return GM_OK;
+}
+
+struct PhaseShape { int B, QT, M, qrows; };
+
+// One decoder layer on rows x/xn [M, d] (xn = normed input).  `next_norm` is the RMSNorm weight applied to
+// the layer's output for whatever consumes it next (null: none); `hidden_out` optionally receives the
+// bf16 residual stream.
+int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const PhaseShape &ph, const CUtensorMap &kvm,
+              __nv_bfloat16 *pool, int layer, int num_pages, const int32_t *page_table,
+              const __nv_bfloat16 *next_norm, __nv_bfloat16 *hidden_out) {
+  const gm_config &cf = c->cfg;
+  int ns; size_t ss; int rc;
+  // QKV projection -> rotary + KV append + Q rearrangement
+  rc = run_gemm(c, c->xn, c->Mmax, &lm.wqkv, static_cast<const __nv_bfloat16 *>(lw.wqkv), ph.M, c->n_qkv, c->d,
+                c->part, true, &ns, &ss);
+  if (rc) return rc;
+  RopeAppendArgs R;
+  R.qkv = c->part; R.nsplit = ns; R.split_stride = ss;
+  R.batch = ph.B; R.QT = ph.QT; R.n_q = cf.n_q_heads; R.n_kv = cf.n_kv_heads; R.hd = cf.head_dim; R.layer = layer;
+  R.num_pages = num_pages; R.max_pages_per_seq = cf.max_pages_per_seq; R.qrows = ph.qrows;
+  R.qn = c->qn; R.qbase = c->qbase; R.page_table = page_table; R.rope = c->rope; R.qbuf = c->qbuf; R.pool = pool;
+  R.status = c->status;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rope_append(R, c->stream));
+  // attention over the pages + merge of the segments
+  AttnArgs T;
+  T.kv_map = kvm; T.qbuf = c->qbuf; T.qn = c->qn; T.qbase = c->qbase; T.page_start = c->page_start;
+  T.page_table = page_table; T.batch = ph.B; T.n_kv = cf.n_kv_heads; T.group = c->group; T.hd = cf.head_dim;
+  T.qrows = ph.qrows; T.layer = layer; T.num_pages = num_pages; T.max_pages_per_seq = cf.max_pages_per_seq;
+  T.n_ctas = c->sm_count; T.scale_log2e = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(cf.head_dim)));
+  T.part_o = c->part_o; T.part_ml = c->part_ml; T.status = c->status;
+  GM_LAUNCH(c, GM_KC_ATTENTION, launch_attention(T, c->stream));
+  AttnCombineArgs Cb;
+  Cb.part_o = c->part_o; Cb.part_ml = c->part_ml; Cb.qn = c->qn; Cb.page_start = c->page_start; Cb.batch = ph.B;
+  Cb.n_kv = cf.n_kv_heads; Cb.group = c->group; Cb.hd = cf.head_dim; Cb.qrows = ph.qrows; Cb.QT = ph.QT;
+  Cb.n_ctas = c->sm_count; Cb.out = c->attn_out;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_attention_combine(Cb, c->stream));
+  // output projection + residual + post-attention norm
+  rc = run_gemm(c, c->attn_out, c->Mmax, &lm.wo, static_cast<const __nv_bfloat16 *>(lw.wo), ph.M, c->d, c->q_dim,
+                c->part, true, &ns, &ss);
+  if (rc) return rc;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+            launch_reduce_residual_norm(c->part, ns, ss, c->x, 1, static_cast<const __nv_bfloat16 *>(lw.ln2), c->xn,
+                                        nullptr, ph.M, c->d, cf.rms_eps, c->stream));
+  // SwiGLU feed-forward
+  rc = run_gemm(c, c->xn, c->Mmax, &lm.wgu, static_cast<const __nv_bfloat16 *>(lw.w_gate_up), ph.M, 2 * c->F, c->d,
+                c->part, true, &ns, &ss);
+  if (rc) return rc;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_swiglu(c->part, ns, ss, c->act, ph.M, c->F, c->stream));
+  rc = run_gemm(c, c->act, c->Mmax, &lm.wdown, static_cast<const __nv_bfloat16 *>(lw.w_down), ph.M, c->d, c->F,
+                c->part, true, &ns, &ss);
+  if (rc) return rc;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+            launch_reduce_residual_norm(c->part, ns, ss, c->x, 1, next_norm, next_norm ? c->xn : nullptr, hidden_out,
+                                        ph.M, c->d, cf.rms_eps, c->stream));
+  return GM_OK;
+}
+
+int run_plan(gm_ctx *c, const gm_state *st, int mode, int k_or_j) {
+  PlanArgs P;
+  P.mode = mode; P.batch = st->batch; P.k_or_j = k_or_j; P.max_pages_per_seq = c->cfg.max_pages_per_seq;
+  P.n_ctas = c->sm_count; P.kv_len = st->kv_len; P.pending_n = st->pending_n; P.qn = c->qn; P.qbase = c->qbase;
+  P.page_start = c->page_start; P.status = c->status;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_plan(P, c->stream));
+  return GM_OK;
+}
+
+int check_state(const gm_ctx *c, const gm_state *st, int k) {
+  if (!c || !st) return GM_ERR_INVALID_ARG;
+  if (k < 1 || k > c->cfg.max_k) return k > c->cfg.max_k ? GM_ERR_UNSUPPORTED : GM_ERR_INVALID_ARG;
+  if (st->batch < 1 || st->batch > c->cfg.max_batch) return GM_ERR_INVALID_ARG;
+  if (!st->kv_len || !st->page_table || !st->kv_pool || !st->head_page_table || !st->head_kv_pool || !st->pending_n ||
+      !st->pending_tok || !st->pending_hidden)
+    return GM_ERR_INVALID_ARG;
+  return GM_OK;
+}
+
+int fill_sampler(gm_ctx *c, SamplerArgs &S, float temperature) {
+  if (!(temperature > 0.f) || !std::isfinite(temperature)) return GM_ERR_UNSUPPORTED;
+  std::memset(&S, 0, sizeof(S));
+  S.inv_temp = 1.0f / temperature;
+  S.V = c->V;
+  S.status = c->status;
+  S.slot_accept = SLOT_ACCEPT;
+  S.slot_final = SLOT_FINAL;
+  return GM_OK;
+}
+
+}  // namespace
+
+// ======================================================================================================================
+extern "C" {
+
+const char *gm_strerror(int code) {
+  switch (code) {
+    case GM_OK: return "ok";
+    case GM_ERR_INVALID_ARG: return "invalid argument";
+    case GM_ERR_UNSUPPORTED: return "unsupported configuration";
+    case GM_ERR_KV_CAPACITY: return "a sequence's pages cannot hold kv_len + k + 1 positions";
+    case GM_ERR_CUDA: return "CUDA call failed";
+    case GM_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    case GM_ERR_BAD_PAGE: return "page id or token id outside its range";
+    case GM_ERR_NO_EXTENSION: return "no sm_100 device";
+    default: return "unknown error";
+  }
+}
+
+int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_stream) {
+  if (!out || !cfg || !w) return GM_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cfg->n_layers < 1 || cfg->d_model < 64 || cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 || cfg->d_ffn < 64 ||
+      cfg->vocab < 8 || cfg->max_batch < 1 || cfg->max_k < 1 || cfg->max_pages_per_seq < 1 || cfg->num_pages < 1 ||
+      cfg->head_num_pages < 1 || !(cfg->rope_base > 1.f) || !(cfg->rms_eps >= 0.f))
+    return GM_ERR_INVALID_ARG;
+  if (cfg->page_size != GM_PAGE || cfg->max_k > GM_MAX_K || (cfg->vocab % 8) || (cfg->d_model % 64) ||
+      (cfg->d_ffn % 64) || (cfg->head_dim != 64 && cfg->head_dim != 128) || (cfg->n_q_heads % cfg->n_kv_heads) ||
+      cfg->d_model > 8192 || cfg->max_batch > 1024 || (cfg->n_kv_heads > 8 && cfg->n_kv_heads % 8))
+    return GM_ERR_UNSUPPORTED;
+  const int group = cfg->n_q_heads / cfg->n_kv_heads;
+  if ((cfg->max_k + 1) * group > 32) return GM_ERR_UNSUPPORTED;
+  if (!w->embed || !w->lm_head || !w->final_norm || !w->layers || !w->head_enorm || !w->head_hnorm || !w->head_proj ||
+      !w->head_final_norm)
+    return GM_ERR_INVALID_ARG;
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return GM_ERR_NO_EXTENSION;
+  cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  if (major != 10) return GM_ERR_NO_EXTENSION;
+
+  gm_ctx *c = new (std::nothrow) gm_ctx();
+  if (!c) return GM_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  c->w = *w;
+  c->layers.assign(w->layers, w->layers + cfg->n_layers);
+  c->w.layers = c->layers.data();
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  c->d = cfg->d_model; c->q_dim = cfg->n_q_heads * cfg->head_dim; c->kv_dim = cfg->n_kv_heads * cfg->head_dim;
+  c->n_qkv = c->q_dim + 2 * c->kv_dim; c->F = cfg->d_ffn; c->V = cfg->vocab; c->group = group;
+  c->Mmax = cfg->max_batch * (cfg->max_k + 1);
+
+  auto fail = [&](int code) { gm_destroy(c); return code; };
+  {
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn)
+      return fail(GM_ERR_CUDA);
+    c->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+  }
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    const gm_layer_weights &lw = c->layers[l];
+    if (!lw.ln1 || !lw.wqkv || !lw.wo || !lw.ln2 || !lw.w_gate_up || !lw.w_down) return fail(GM_ERR_INVALID_ARG);
+  }
+  {
+    const gm_layer_weights &lw = w->head_layer;
+    if (!lw.ln1 || !lw.wqkv || !lw.wo || !lw.ln2 || !lw.w_gate_up || !lw.w_down) return fail(GM_ERR_INVALID_ARG);
+  }
+  auto layer_maps = [&](const gm_layer_weights &lw, LayerMaps &lm) {
+    int rc = make_map(c, &lm.wqkv, lw.wqkv, c->n_qkv, c->d, 128);
+    if (!rc) rc = make_map(c, &lm.wo, lw.wo, c->d, c->q_dim, 128);
+    if (!rc) rc = make_map(c, &lm.wgu, lw.w_gate_up, 2 * c->F, c->d, 128);
+    if (!rc) rc = make_map(c, &lm.wdown, lw.w_down, c->d, c->F, 128);
+    return rc;
+  };
+  c->lmaps.resize(cfg->n_layers);
+  for (int l = 0; l < cfg->n_layers; ++l)
+    if (layer_maps(c->layers[l], c->lmaps[l])) return fail(GM_ERR_CUDA);
+  if (layer_maps(w->head_layer, c->head_maps)) return fail(GM_ERR_CUDA);
+  if (make_map(c, &c->lm_head_map, w->lm_head, c->V, c->d, 128)) return fail(GM_ERR_CUDA);
+  if (make_map(c, &c->head_proj_map, w->head_proj, c->d, 2 * c->d, 128)) return fail(GM_ERR_CUDA);
+
+  // workspaces
+  const size_t M = c->Mmax, B = cfg->max_batch;
+  const int qrows = round16((cfg->max_k + 1) * group);
+  size_t pe = 0;
+  auto upd = [&](int N, int K) {          // worst case of nsplit * M * N over every row count a call may use
+    for (int m = 1; m <= static_cast<int>(M); ++m) {
+      const int T = m >= 256 ? 256 : round16(m);
+      pe = std::max(pe, static_cast<size_t>(pick_split(c, m, N, K, T)) * m * N);
+    }
+  };
+  upd(c->n_qkv, c->d); upd(c->d, c->q_dim); upd(2 * c->F, c->d); upd(c->d, c->F); upd(c->d, 2 * c->d);
+  c->part_elems = pe;
+  int rc = GM_OK;
+  const size_t slots = static_cast<size_t>(c->sm_count) + B;
+#define A_(call) if ((rc = (call)) != GM_OK) return fail(rc)
+  A_(dev_alloc(c, &c->x, M * c->d));
+  A_(dev_alloc(c, &c->xn, M * c->d));
+  A_(dev_alloc(c, &c->zin, M * 2 * c->d));
+  A_(dev_alloc(c, &c->part, pe));
+  A_(dev_alloc(c, &c->qbuf, B * cfg->n_kv_heads * qrows * cfg->head_dim));
+  A_(dev_alloc(c, &c->attn_out, M * c->q_dim));
+  A_(dev_alloc(c, &c->act, M * c->F));
+  A_(dev_alloc(c, &c->g, B * c->d));
+  A_(dev_alloc(c, &c->gn, B * c->d));
+  A_(dev_alloc(c, &c->part_o, slots * cfg->n_kv_heads * qrows * cfg->head_dim));
+  A_(dev_alloc(c, &c->part_ml, slots * cfg->n_kv_heads * qrows * 2));
+  A_(dev_alloc(c, &c->ws_draft_logits, B * cfg->max_k * c->V, false));
+  A_(dev_alloc(c, &c->ws_target_logits, B * (cfg->max_k + 1) * c->V, false));
+  A_(dev_alloc(c, &c->ws_target_hidden, M * c->d));
+  A_(dev_alloc(c, &c->ws_draft_tok, B * cfg->max_k));
+  A_(dev_alloc(c, &c->ws_accept_len, B));
+  A_(dev_alloc(c, &c->ws_next_token, B));
+  A_(dev_alloc(c, &c->ws_u24, B * (2 * cfg->max_k + 1)));
+  A_(dev_alloc(c, &c->qn, B));
+  A_(dev_alloc(c, &c->qbase, B));
+  A_(dev_alloc(c, &c->page_start, B + 1));
+  A_(dev_alloc(c, &c->status, 1));
+  // rotary table: cos/sin of pos * base^(-2i/hd), computed in double precision on the host
+  {
+    const int half = cfg->head_dim / 2;
+    const size_t max_pos = static_cast<size_t>(cfg->max_pages_per_seq) * 16;
+    std::vector<float2> tab(max_pos * half);
+    for (int i = 0; i < half; ++i) {
+      const double inv = std::pow(static_cast<double>(cfg->rope_base), -2.0 * i / cfg->head_dim);
+      for (size_t p = 0; p < max_pos; ++p) {
+        const double a = static_cast<double>(p) * inv;
+        tab[p * half + i] = make_float2(static_cast<float>(std::cos(a)), static_cast<float>(std::sin(a)));
+      }
+    }
+    A_(dev_alloc(c, &c->rope, tab.size(), false));
+    if (cudaMemcpyAsync(c->rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
+      return fail(GM_ERR_CUDA);
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(GM_ERR_CUDA);
+  }
+#undef A_
+  *out = c;
+  return GM_OK;
+}
+
+void gm_destroy(gm_ctx *c) {
+  if (!c) return;
+  cudaStreamSynchronize(c->stream);
+  for (void *p : c->allocs) cudaFree(p);
+  for (auto &v : c->events)
+    for (auto &e : v) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+  delete c;
+}
+
+int gm_draft(gm_ctx *c, const gm_state *st, int k, float temperature, const uint32_t *u24_draft, uint64_t seed,
+             uint64_t step, int32_t *draft_tok, void *draft_logits, float *dbg_q) {
+  int rc = check_state(c, st, k);
+  if (rc) return rc;
+  if (!draft_tok || !draft_logits) return GM_ERR_INVALID_ARG;
+  SamplerArgs S;
+  if ((rc = fill_sampler(c, S, temperature)) != GM_OK) return rc;
+  const gm_config &cf = c->cfg;
+  CUtensorMap kvm;
+  if ((rc = kv_map(c, st->head_kv_pool, 1, cf.head_num_pages, &kvm)) != GM_OK) return rc;
+  __nv_bfloat16 *dl = static_cast<__nv_bfloat16 *>(draft_logits);
+  for (int j = 1; j <= k; ++j) {
+    const int mode = j == 1 ? PHASE_DRAFT_FIRST : PHASE_DRAFT_NEXT;
+    PhaseShape ph;
+    ph.B = st->batch; ph.QT = j == 1 ? cf.max_k + 1 : 1; ph.M = ph.B * ph.QT; ph.qrows = round16(ph.QT * c->group);
+    if ((rc = run_plan(c, st, mode, j == 1 ? cf.max_k + 1 : j)) != GM_OK) return rc;
+    HeadInputArgs H;
+    H.mode = mode; H.batch = ph.B; H.QT = ph.QT; H.d = c->d; H.vocab = c->V; H.max_k = cf.max_k; H.k = k; H.j = j;
+    H.eps = cf.rms_eps; H.embed = static_cast<const __nv_bfloat16 *>(c->w.embed);
+    H.we = static_cast<const __nv_bfloat16 *>(c->w.head_enorm); H.wh = static_cast<const __nv_bfloat16 *>(c->w.head_hnorm);
+    H.pending_tok = st->pending_tok; H.pending_n = st->pending_n;
+    H.pending_hidden = static_cast<const __nv_bfloat16 *>(st->pending_hidden); H.draft_tok = draft_tok; H.g_prev = c->g;
+    H.zin = c->zin; H.status = c->status;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_head_input(H, c->stream));
+    int ns; size_t ss;
+    rc = run_gemm(c, c->zin, c->Mmax, &c->head_proj_map, static_cast<const __nv_bfloat16 *>(c->w.head_proj), ph.M, c->d,
+                  2 * c->d, c->part, true, &ns, &ss);
+    if (rc) return rc;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+              launch_reduce_residual_norm(c->part, ns, ss, c->x, 0, static_cast<const __nv_bfloat16 *>(c->w.head_layer.ln1),
+                                          c->xn, nullptr, ph.M, c->d, cf.rms_eps, c->stream));
+    rc = run_layer(c, c->w.head_layer, c->head_maps, ph, kvm, static_cast<__nv_bfloat16 *>(st->head_kv_pool), 0,
+                   cf.head_num_pages, st->head_page_table, nullptr, nullptr);
+    if (rc) return rc;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+              launch_head_out(c->x, c->qn, ph.B, ph.QT, c->d, static_cast<const __nv_bfloat16 *>(c->w.head_final_norm),
+                              cf.rms_eps, c->g, c->gn, c->stream));
+    // shared LM head -> row j-1 of every sequence's draft logits (row stride k*V)
+    {
+      GemmArgs A;
+      std::memset(&A, 0, sizeof(A));
+      A.x = c->gn; A.w = static_cast<const __nv_bfloat16 *>(c->w.lm_head); A.M = ph.B; A.N = c->V; A.K = c->d;
+      A.out = dl + static_cast<size_t>(j - 1) * c->V; A.out_fp32 = 0; A.nsplit = 1; A.ldo = static_cast<size_t>(k) * c->V;
+      A.block_t = ph.B >= 256 ? 256 : round16(ph.B); A.status = c->status;
+      if (cf.flags & GM_FLAG_SIMPLE_GEMM) {
+        GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_simple(A, c->stream));
+      } else {
+        A.w_map = c->lm_head_map;
+        if ((rc = x_map(c, c->gn, cf.max_batch, c->d, A.block_t, &A.x_map)) != GM_OK) return rc;
+        GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(A, c->stream));
+      }
+    }
+    // d_j ~ softmax(logits / T): the sampler with depth 0
+    S.K = 0; S.target_logits = dl + static_cast<size_t>(j - 1) * c->V; S.tgt_bstride = static_cast<size_t>(k) * c->V;
+    S.draft_logits = nullptr; S.u24 = u24_draft ? u24_draft + (j - 1) : nullptr; S.u_stride = k;
+    S.seed = seed; S.step = step; S.slot_final = SLOT_DRAFT + (j - 1);
+    S.accept_len = nullptr; S.next_token = draft_tok + (j - 1); S.tok_out_stride = k;
+    S.dbg_p = dbg_q ? dbg_q + static_cast<size_t>(j - 1) * c->V : nullptr; S.dbg_q = nullptr; S.commit = 0;
+    GM_LAUNCH(c, GM_KC_SAMPLER, launch_sampler(S, ph.B, c->stream));
+  }
+  return GM_OK;
+}
+
+int gm_verify(gm_ctx *c, const gm_state *st, int k, const int32_t *draft_tok, void *target_logits,
+              void *target_hidden) {
+  int rc = check_state(c, st, k);
+  if (rc) return rc;
+  if (!draft_tok || !target_logits || !target_hidden) return GM_ERR_INVALID_ARG;
+  const gm_config &cf = c->cfg;
+  PhaseShape ph;
+  ph.B = st->batch; ph.QT = k + 1; ph.M = ph.B * ph.QT; ph.qrows = round16(ph.QT * c->group);
+  CUtensorMap kvm;
+  if ((rc = kv_map(c, st->kv_pool, cf.n_layers, cf.num_pages, &kvm)) != GM_OK) return rc;
+  if ((rc = run_plan(c, st, PHASE_VERIFY, k)) != GM_OK) return rc;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+            launch_embed_norm(static_cast<const __nv_bfloat16 *>(c->w.embed),
+                              static_cast<const __nv_bfloat16 *>(c->layers[0].ln1), st->pending_tok, st->pending_n,
+                              draft_tok, ph.B, k, cf.max_k, c->d, c->V, cf.rms_eps, c->x, c->xn, c->status, c->stream));
+  for (int l = 0; l < cf.n_layers; ++l) {
+    const bool last = l + 1 == cf.n_layers;
+    const __nv_bfloat16 *next_norm =
+        static_cast<const __nv_bfloat16 *>(last ? c->w.final_norm : c->layers[l + 1].ln1);
+    rc = run_layer(c, c->layers[l], c->lmaps[l], ph, kvm, static_cast<__nv_bfloat16 *>(st->kv_pool), l, cf.num_pages,
+                   st->page_table, next_norm, last ? static_cast<__nv_bfloat16 *>(target_hidden) : nullptr);
+    if (rc) return rc;
+  }
+  GemmArgs A;
+  std::memset(&A, 0, sizeof(A));
+  A.x = c->xn; A.w = static_cast<const __nv_bfloat16 *>(c->w.lm_head); A.M = ph.M; A.N = c->V; A.K = c->d;
+  A.out = target_logits; A.out_fp32 = 0; A.nsplit = 1; A.ldo = c->V;
+  A.block_t = ph.M >= 256 ? 256 : round16(ph.M); A.status = c->status;
+  if (cf.flags & GM_FLAG_SIMPLE_GEMM) {
+    GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_simple(A, c->stream));
+  } else {
+    A.w_map = c->lm_head_map;
+    if ((rc = x_map(c, c->xn, c->Mmax, c->d, A.block_t, &A.x_map)) != GM_OK) return rc;
+    GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(A, c->stream));
+  }
+  return GM_OK;
+}
+
+int gm_accept(gm_ctx *c, gm_state *st, int batch, int k, float temperature, const void *target_logits,
+              const void *draft_logits, const int32_t *draft_tok, const uint32_t *u24_accept, uint64_t seed,
+              uint64_t step, int32_t *accept_len, int32_t *next_token, float *dbg_p, float *dbg_q,
+              const void *target_hidden, int commit_state) {
+  if (!c || !target_logits || !draft_logits || !draft_tok || !accept_len || !next_token) return GM_ERR_INVALID_ARG;
+  if (k < 1 || batch < 1) return GM_ERR_INVALID_ARG;
+  if (k > GM_MAX_K) return GM_ERR_UNSUPPORTED;
+  if (commit_state) {
+    int rc = check_state(c, st, k);
+    if (rc) return rc;
+    if (!target_hidden || batch != st->batch) return GM_ERR_INVALID_ARG;
+  }
+  SamplerArgs S;
+  int rc = fill_sampler(c, S, temperature);
+  if (rc) return rc;
+  S.K = k;
+  S.target_logits = static_cast<const __nv_bfloat16 *>(target_logits); S.tgt_bstride = static_cast<size_t>(k + 1) * c->V;
+  S.draft_logits = static_cast<const __nv_bfloat16 *>(draft_logits); S.drf_bstride = static_cast<size_t>(k) * c->V;
+  S.draft_tok = draft_tok; S.tok_in_stride = k; S.u24 = u24_accept; S.u_stride = k + 1; S.seed = seed; S.step = step;
+  S.accept_len = accept_len; S.next_token = next_token; S.tok_out_stride = 1; S.dbg_p = dbg_p; S.dbg_q = dbg_q;
+  S.commit = commit_state ? 1 : 0;
+  if (commit_state) {
+    S.kv_len = st->kv_len; S.pending_n = st->pending_n; S.pending_tok = st->pending_tok;
+    S.pending_hidden = static_cast<__nv_bfloat16 *>(st->pending_hidden);
+    S.target_hidden = static_cast<const __nv_bfloat16 *>(target_hidden);
+    S.d_model = c->d; S.max_k = c->cfg.max_k;
+  }
+  GM_LAUNCH(c, GM_KC_SAMPLER, launch_sampler(S, batch, c->stream));
+  return GM_OK;
+}
+
+int gm_draw(gm_ctx *c, const void *logits, int rows, float temperature, const uint32_t *u24, int32_t *out_tok,
+            float *dbg_prob) {
+  if (!c || !logits || !u24 || !out_tok || rows < 1) return GM_ERR_INVALID_ARG;
+  SamplerArgs S;
+  int rc = fill_sampler(c, S, temperature);
+  if (rc) return rc;
+  S.K = 0; S.target_logits = static_cast<const __nv_bfloat16 *>(logits); S.tgt_bstride = c->V; S.u24 = u24; S.u_stride = 1;
+  S.next_token = out_tok; S.tok_out_stride = 1; S.dbg_p = dbg_prob;
+  GM_LAUNCH(c, GM_KC_SAMPLER, launch_sampler(S, rows, c->stream));
+  return GM_OK;
+}
+
+int gm_spec_step(gm_ctx *c, gm_state *st, int k, float temperature, uint64_t seed, uint64_t step, int32_t *accept_len,
+                 int32_t *next_token, int32_t *draft_tok) {
+  int rc = check_state(c, st, k);
+  if (rc) return rc;
+  if (!accept_len || !next_token) return GM_ERR_INVALID_ARG;
+  int32_t *dt = draft_tok ? draft_tok : c->ws_draft_tok;
+  if ((rc = gm_draft(c, st, k, temperature, nullptr, seed, step, dt, c->ws_draft_logits, nullptr)) != GM_OK) return rc;
+  if ((rc = gm_verify(c, st, k, dt, c->ws_target_logits, c->ws_target_hidden)) != GM_OK) return rc;
+  return gm_accept(c, st, st->batch, k, temperature, c->ws_target_logits, c->ws_draft_logits, dt, nullptr, seed, step,
+                   accept_len, next_token, nullptr, nullptr, c->ws_target_hidden, 1);
+}
+
+int gm_spec_step_host(gm_ctx *c, gm_state *st, int k, float temperature, uint64_t seed, uint64_t step,
+                      int32_t *accept_len_host, int32_t *next_token_host) {
+  if (!accept_len_host || !next_token_host) return GM_ERR_INVALID_ARG;
+  int rc = gm_spec_step(c, st, k, temperature, seed, step, c->ws_accept_len, c->ws_next_token, nullptr);
+  if (rc) return rc;
+  const size_t n = static_cast<size_t>(st->batch) * sizeof(int32_t);
+  GM_CUDA(c, cudaMemcpyAsync(accept_len_host, c->ws_accept_len, n, cudaMemcpyDeviceToHost, c->stream));
+  GM_CUDA(c, cudaMemcpyAsync(next_token_host, c->ws_next_token, n, cudaMemcpyDeviceToHost, c->stream));
+  GM_CUDA(c, cudaStreamSynchronize(c->stream));
+  return GM_OK;
+}
+
+int gm_gemm(gm_ctx *c, const void *x, const void *w, void *out, int M, int N, int K, int out_fp32) {
+  if (!c || !x || !w || !out || M < 1 || N < 1 || K < 1) return GM_ERR_INVALID_ARG;
+  if ((K % 64) || (N % 8)) return GM_ERR_UNSUPPORTED;
+  GemmArgs A;
+  std::memset(&A, 0, sizeof(A));
+  A.x = static_cast<const __nv_bfloat16 *>(x); A.w = static_cast<const __nv_bfloat16 *>(w); A.M = M; A.N = N; A.K = K;
+  A.out = out; A.out_fp32 = out_fp32 ? 1 : 0; A.nsplit = 1; A.ldo = N; A.split_stride = static_cast<size_t>(M) * N;
+  A.block_t = M >= 256 ? 256 : round16(M); A.status = c->status;
+  if (c->cfg.flags & GM_FLAG_SIMPLE_GEMM) {
+    GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_simple(A, c->stream));
+    return GM_OK;
+  }
+  auto key = std::make_tuple(w, N, K);
+  auto it = c->w_maps.find(key);
+  if (it == c->w_maps.end()) {
+    CUtensorMap m;
+    if (make_map(c, &m, w, N, K, 128) != GM_OK) return GM_ERR_CUDA;
+    it = c->w_maps.emplace(key, m).first;
+  }
+  A.w_map = it->second;
+  int rc = x_map(c, x, M, K, A.block_t, &A.x_map);
+  if (rc) return rc;
+  GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(A, c->stream));
+  return GM_OK;
+}
+
+int gm_profile(gm_ctx *c, int class_mask) {
+  if (!c) return GM_ERR_INVALID_ARG;
+  GM_CUDA(c, cudaStreamSynchronize(c->stream));
+  c->prof_mask = class_mask;
+  for (int i = 0; i < GM_KC_COUNT; ++i) c->events_used[i] = 0;
+  return GM_OK;
+}
+
+int gm_profile_read(gm_ctx *c, int kernel_class, double *total_ms, int64_t *launches) {
+  if (!c || kernel_class < 0 || kernel_class >= GM_KC_COUNT || !total_ms || !launches) return GM_ERR_INVALID_ARG;
+  GM_CUDA(c, cudaStreamSynchronize(c->stream));
+  double t = 0;
+  for (size_t i = 0; i < c->events_used[kernel_class]; ++i) {
+    float ms = 0.f;
+    GM_CUDA(c, cudaEventElapsedTime(&ms, c->events[kernel_class][i].a, c->events[kernel_class][i].b));
+    t += ms;
+  }
+  *total_ms = t;
+  *launches = static_cast<int64_t>(c->events_used[kernel_class]);
+  return GM_OK;
+}
+
+int64_t gm_launch_count(gm_ctx *c) { return c ? c->launches : 0; }
+
+int gm_last_status(gm_ctx *c) {
+  if (!c) return GM_ERR_INVALID_ARG;
+  uint32_t s = 0;
+  GM_CUDA(c, cudaStreamSynchronize(c->stream));
+  GM_CUDA(c, cudaMemcpy(&s, c->status, sizeof(s), cudaMemcpyDeviceToHost));
+  GM_CUDA(c, cudaMemset(c->status, 0, sizeof(s)));
+  if (s & ST_TIMEOUT) return GM_ERR_DEVICE_TIMEOUT;
+  if (s & ST_KV_CAPACITY) return GM_ERR_KV_CAPACITY;
+  if (s & (ST_BAD_PAGE | ST_BAD_TOKEN)) return GM_ERR_BAD_PAGE;
+  return GM_OK;
+}
+
+}  // extern "C"

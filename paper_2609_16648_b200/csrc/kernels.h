@@ -1,0 +1,132 @@
+// Internal declarations shared by the kernel files and the C-ABI layer (not part of the public ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gm {
+
+constexpr int GM_MAX_K_ = 7;
+constexpr int SAMP_THREADS = 512;
+constexpr int SAMP_CLUSTER = 8;
+
+// ---- sampler ------------------------------------------------------------------------------------------
+struct SamplerArgs {
+  const __nv_bfloat16 *target_logits;   // row (b, r) at target_logits + b*tgt_bstride + r*V, r = 0..K
+  const __nv_bfloat16 *draft_logits;    // row (b, r) at draft_logits + b*drf_bstride + r*V, r = 0..K-1 (null if K == 0)
+  size_t tgt_bstride, drf_bstride;      // in elements
+  const int32_t *draft_tok;             // d_{j+1} of row b at draft_tok[b*tok_in_stride + j]
+  int tok_in_stride;
+  const uint32_t *u24;                  // [b*u_stride + j], j = 0..K (K accept uniforms, then the final one); null = Philox
+  int u_stride;
+  uint64_t seed, step;
+  uint32_t slot_accept, slot_final;
+  float inv_temp;
+  int K, V;
+  int32_t *accept_len;                  // [b] or null
+  int32_t *next_token;                  // [b*tok_out_stride]
+  int tok_out_stride;
+  float *dbg_p, *dbg_q;                 // same strides as the logits, or null
+  int commit;                           // state commit (needs the fields below)
+  int32_t *kv_len, *pending_n, *pending_tok;
+  __nv_bfloat16 *pending_hidden;
+  const __nv_bfloat16 *target_hidden;   // [b, K+1, d_model]
+  int d_model, max_k;
+  uint32_t *status;
+};
+cudaError_t launch_sampler(const SamplerArgs &A, int batch, cudaStream_t stream);
+
+// ---- planning: query ranges of a phase and the balanced attention partition --------------------------
+enum PhaseMode { PHASE_VERIFY = 0, PHASE_DRAFT_FIRST = 1, PHASE_DRAFT_NEXT = 2 };
+struct PlanArgs {
+  int mode, batch, k_or_j;              // VERIFY: K;  DRAFT_NEXT: application index j (2..K)
+  int max_pages_per_seq, n_ctas;
+  const int32_t *kv_len, *pending_n;
+  int32_t *qn, *qbase;                  // [B] queries of this phase and the position of the first one
+  int32_t *page_start;                  // [B+1] exclusive prefix of pages attended per sequence
+  uint32_t *status;
+};
+cudaError_t launch_plan(const PlanArgs &A, cudaStream_t stream);
+
+// ---- element-wise --------------------------------------------------------------------------------------
+// x[m] = embed[token(m)] (fp32), xn[m] = RMSNorm(x[m]; w) (bf16); rows m = b*QT + j of the verify phase.
+cudaError_t launch_embed_norm(const __nv_bfloat16 *embed, const __nv_bfloat16 *w, const int32_t *pending_tok,
+                              const int32_t *pending_n, const int32_t *draft_tok, int batch, int K, int max_k, int d,
+                              int vocab, float eps, float *x, __nv_bfloat16 *xn, uint32_t *status,
+                              cudaStream_t stream);
+// zin[m] = [RMSNorm(embed[tok]; we) ; RMSNorm(hidden; wh)] (bf16 [M, 2d]) for the draft head.
+struct HeadInputArgs {
+  int mode, batch, QT, d, vocab, max_k, k, j;    // j: application index for DRAFT_NEXT
+  float eps;
+  const __nv_bfloat16 *embed, *we, *wh;
+  const int32_t *pending_tok, *pending_n;
+  const __nv_bfloat16 *pending_hidden;           // [B, max_k+1, d]
+  const int32_t *draft_tok;                      // [B, k]
+  const float *g_prev;                           // [B, d] head state of the previous application
+  __nv_bfloat16 *zin;                            // [B*QT, 2d]
+  uint32_t *status;
+};
+cudaError_t launch_head_input(const HeadInputArgs &A, cudaStream_t stream);
+// x_out[m] = (add_residual ? x[m] : 0) + sum_s partial[s][m];  xn[m] = RMSNorm(x_out[m]; w);  optional
+// bf16 copy of x_out (the hidden state handed to the caller).
+cudaError_t launch_reduce_residual_norm(const float *partial, int nsplit, size_t split_stride, float *x,
+                                        int add_residual, const __nv_bfloat16 *w, __nv_bfloat16 *xn,
+                                        __nv_bfloat16 *hidden_out, int M, int d, float eps, cudaStream_t stream);
+// Rotary embedding of q and k, KV append into the pages, Q rearranged per (sequence, kv head).
+struct RopeAppendArgs {
+  const float *qkv; int nsplit; size_t split_stride;   // fp32 [nsplit][M][(n_q + 2 n_kv) hd]
+  int batch, QT, n_q, n_kv, hd, layer, num_pages, max_pages_per_seq, qrows;
+  const int32_t *qn, *qbase, *page_table;
+  const float2 *rope;                                   // [max_pos][hd/2] (cos, sin)
+  __nv_bfloat16 *qbuf;                                  // [B][n_kv][qrows][hd], row = j*group + g
+  __nv_bfloat16 *pool;                                  // [L][2][num_pages][n_kv][16][hd]
+  uint32_t *status;
+};
+cudaError_t launch_rope_append(const RopeAppendArgs &A, cudaStream_t stream);
+// act[m][i] = silu(gate_i) * up_i from interleaved fp32 partials [nsplit][M][2F].
+cudaError_t launch_swiglu(const float *gu, int nsplit, size_t split_stride, __nv_bfloat16 *act, int M, int F,
+                          cudaStream_t stream);
+// g[b] = x[b*QT + qn[b]-1] (fp32), gn[b] = RMSNorm(g[b]; w) (bf16): the head's last valid row per sequence.
+cudaError_t launch_head_out(const float *x, const int32_t *qn, int batch, int QT, int d, const __nv_bfloat16 *w,
+                            float eps, float *g, __nv_bfloat16 *gn, cudaStream_t stream);
+
+// ---- attention -------------------------------------------------------------------------------------------
+struct AttnArgs {
+  CUtensorMap kv_map;                   // 2-D view of the pool: [rows of hd elements], box 64 x (heads*16)
+  const __nv_bfloat16 *qbuf;            // [B][n_kv][qrows][hd]
+  const int32_t *qn, *qbase, *page_start, *page_table;
+  int batch, n_kv, group, hd, qrows, layer, num_pages, max_pages_per_seq, n_ctas;
+  float scale_log2e;                    // 1/sqrt(hd) * log2(e)
+  float *part_o;                        // [n_ctas + B][n_kv][qrows][hd] partial outputs
+  float *part_ml;                       // [n_ctas + B][n_kv][qrows][2] partial (max, sum)
+  uint32_t *status;
+};
+cudaError_t launch_attention(const AttnArgs &A, cudaStream_t stream);
+struct AttnCombineArgs {
+  const float *part_o, *part_ml;
+  const int32_t *qn, *page_start;
+  int batch, n_kv, group, hd, qrows, QT, n_ctas;
+  __nv_bfloat16 *out;                   // [B*QT][n_q*hd]
+};
+cudaError_t launch_attention_combine(const AttnCombineArgs &A, cudaStream_t stream);
+int attention_max_ctas(int n_kv, int hd);   // CTAs the attention kernel wants for this shape (<= SM count)
+size_t attention_smem_bytes(int n_kv, int hd);
+
+// ---- GEMM --------------------------------------------------------------------------------------------------
+// out = x[M, K] * w[N, K]^T with fp32 accumulation.  nsplit > 1 (or out_fp32): fp32 partials
+// [nsplit][M][N]; otherwise bf16 [M][N].
+struct GemmArgs {
+  CUtensorMap w_map, x_map;             // tcgen05 path only
+  const __nv_bfloat16 *x, *w;
+  void *out; int out_fp32;
+  int M, N, K, nsplit, block_t;         // block_t: tokens per CTA (multiple of 16, <= 256)
+  size_t split_stride;                  // elements between partials
+  size_t ldo;                           // output row stride in elements (>= N)
+  uint32_t *status;
+};
+cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream);
+cudaError_t launch_gemm_simple(const GemmArgs &A, cudaStream_t stream);
+
+}  // namespace gm

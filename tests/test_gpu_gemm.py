@@ -1,0 +1,48 @@
+"""tcgen05 GEMM (gm_gemm) against an fp64 matmul, and against the plain mma.sync kernel."""
+import numpy as np
+import pytest
+import torch
+
+from synth_inputs import ModelConfig
+
+pytestmark = pytest.mark.gpu
+
+
+def _ctx(flags=0):
+    import paper_2609_16648_b200 as gmb
+    cfg = ModelConfig("g", 1, 64, 1, 1, 64, 64, 8, batch=4, k=1, kv_len_min=0, kv_len_max=0, length_law="uniform")
+    return gmb, gmb.Context(cfg, gmb.random_packed_weights(cfg, "cuda"), 4, 1, 4, 8, 8, flags=flags)
+
+
+SHAPES = [(1, 128, 64), (16, 128, 128), (4, 136, 256), (64, 2560, 2560), (100, 1000, 704), (256, 6144, 2560),
+          (300, 384, 512), (256, 2560, 9728), (20, 8, 64), (513, 264, 192)]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+@pytest.mark.parametrize("out_fp32", [True, False])
+def test_gemm_matches_fp64_matmul(M, N, K, out_fp32):
+    gmb, ctx = _ctx()
+    g = torch.Generator(device="cpu").manual_seed(M * 7 + N * 3 + K)
+    x = (torch.randn((M, K), generator=g)).to(torch.bfloat16)
+    w = (torch.randn((N, K), generator=g) * 0.05).to(torch.bfloat16)
+    ref = x.double().numpy() @ w.double().numpy().T
+    out = torch.full((M, N), float("nan"), dtype=torch.float32 if out_fp32 else torch.bfloat16, device="cuda")
+    gmb.gm_gemm(ctx, x.cuda(), w.cuda(), out, M, N, K, out_fp32)
+    assert gmb.gm_last_status(ctx) == 0
+    got = out.float().cpu().numpy().astype(np.float64)
+    tol = (1e-5 if out_fp32 else 5e-3) * np.abs(ref).max() + 1e-6
+    assert np.abs(got - ref).max() <= tol, np.abs(got - ref).max() / np.abs(ref).max()
+    ctx.close()
+
+
+def test_simple_kernel_agrees():
+    gmb, ctx = _ctx(flags=1)
+    M, N, K = 70, 200, 192
+    g = torch.Generator(device="cpu").manual_seed(5)
+    x = torch.randn((M, K), generator=g).to(torch.bfloat16)
+    w = torch.randn((N, K), generator=g).to(torch.bfloat16)
+    out = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+    gmb.gm_gemm(ctx, x.cuda(), w.cuda(), out, M, N, K, True)
+    ref = x.double().numpy() @ w.double().numpy().T
+    assert np.abs(out.cpu().numpy() - ref).max() <= 1e-5 * np.abs(ref).max()
+    ctx.close()

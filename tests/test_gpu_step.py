@@ -1,0 +1,227 @@
+"""Whole speculative step on the Tiny configuration: CUDA library vs the oracle, from a common state."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import philox, sampler as osampler, step as ostep
+from synth_inputs import get_config
+
+from helpers import push_state, rel_err, tiny_setup
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-2      # per-tensor normalised max error for bf16-path logits and hidden states
+
+
+def _bufs(B, K, V, d):
+    dev = "cuda"
+    z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=dev)
+    return dict(draft_tok=z((B, K), torch.int32), draft_logits=z((B, K, V), torch.bfloat16),
+                tgt_logits=z((B, K + 1, V), torch.bfloat16), tgt_hidden=z((B, K + 1, d), torch.bfloat16),
+                dbg_q=z((B, K, V), torch.float32), dbg_p=z((B, K + 1, V), torch.float32),
+                dbg_q2=z((B, K, V), torch.float32), a=z((B,), torch.int32), t=z((B,), torch.int32))
+
+
+def _run_phases(gmb, ctx, gst, K, seed, step, bufs, commit=False):
+    B = gst.batch
+    gmb.gm_draft(ctx, gst, K, 1.0, None, seed, step, bufs["draft_tok"], bufs["draft_logits"], bufs["dbg_q"])
+    gmb.gm_verify(ctx, gst, K, bufs["draft_tok"], bufs["tgt_logits"], bufs["tgt_hidden"])
+    gmb.gm_accept(ctx, gst, B, K, 1.0, bufs["tgt_logits"], bufs["draft_logits"], bufs["draft_tok"], None, seed, step,
+                  bufs["a"], bufs["t"], bufs["dbg_p"], bufs["dbg_q2"], bufs["tgt_hidden"], commit_state=commit)
+    assert gmb.gm_last_status(ctx) == 0
+
+
+@pytest.mark.parametrize("flags", [1, 0], ids=["mma_sync_gemm", "tcgen05_gemm"])
+def test_tiny_step_parity_from_common_state(flags):
+    """Every step starts from the oracle's state.  Logits/hidden within 2e-2; the device's decisions
+    equal the oracle's decision function on the device's own probabilities bit for bit; draft tokens and
+    accept bits agree with the oracle end to end on >= 99.5 % of positions."""
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny").with_(prompt_len=40)
+    K, B, V, d = cfg.k, cfg.batch, cfg.vocab, cfg.d_model
+    n_steps = 24
+    w, ost, ctx, gst = tiny_setup(cfg, cap_tokens=40 + n_steps * (K + 1) + 8, flags=flags)
+    bufs = _bufs(B, K, V, d)
+    seed = 5
+    agree = total = tok_agree = 0
+    worst = 0.0
+    for it in range(n_steps):
+        push_state(ost, gst, ctx)
+        step = ost.step
+        _run_phases(gmb, ctx, gst, K, seed, step, bufs)
+        g_dtok = bufs["draft_tok"].cpu().numpy()
+        g_dl = bufs["draft_logits"].float().cpu().numpy()
+        g_q = bufs["dbg_q"].cpu().numpy()
+        ud, ua = philox.u24_draft(seed, step, B, K), philox.u24_accept(seed, step, B, K)
+        # (1) draft draws are the integer inverse CDF of the device's own q
+        for b in range(B):
+            for k in range(K):
+                assert g_dtok[b, k] == osampler.draw_token(g_q[b, k], ud[b, k])[0]
+        assert torch.equal(bufs["dbg_q"], bufs["dbg_q2"])
+        # (2) decisions on the device's p, q
+        p, q = bufs["dbg_p"].cpu().numpy(), bufs["dbg_q2"].cpu().numpy()
+        for b in range(B):
+            ea, et, _ = osampler.decide(p[b], q[b], g_dtok[b], ua[b])
+            assert (ea, et) == (int(bufs["a"][b]), int(bufs["t"][b]))
+        # (3) oracle cycle on its own; compare tensors as long as the inputs are the same
+        ref = ostep.spec_step(w, cfg, ost, K, 1.0, seed=seed, do_commit=False)
+        worst = max(worst, rel_err(g_dl[:, 0], ref["draft_logits"][:, 0]))
+        same_d = (g_dtok == ref["draft_tok"])
+        prefix_same = np.cumprod(same_d, axis=1).astype(bool)        # drafts equal up to and including k
+        g_tl = bufs["tgt_logits"].float().cpu().numpy()
+        g_th = bufs["tgt_hidden"].float().cpu().numpy()
+        for b in range(B):
+            for j in range(K + 1):
+                if j == 0 or prefix_same[b, j - 1]:
+                    worst = max(worst, rel_err(g_tl[b, j], ref["target_logits"][b, j]),
+                                rel_err(g_th[b, j], ref["target_hidden"][b, j]))
+                if 0 < j < K and prefix_same[b, j - 1]:
+                    worst = max(worst, rel_err(g_dl[b, j], ref["draft_logits"][b, j]))
+        # (4) end-to-end agreement per position: draft token and accept bit
+        ga = bufs["a"].cpu().numpy()
+        for b in range(B):
+            for k in range(K):
+                total += 1
+                g_acc, o_acc = k < ga[b], k < ref["accept_len"][b]
+                if same_d[b, k] and g_acc == o_acc:
+                    agree += 1
+            tok_agree += int(int(bufs["t"][b]) == ref["next_token"][b] and ga[b] == ref["accept_len"][b])
+        # advance the oracle (its own decisions) to the next common state
+        ostep.spec_step(w, cfg, ost, K, 1.0, seed=seed, do_commit=True)
+    assert worst < TOL, worst
+    assert agree / total >= 0.995, (agree, total)
+    assert tok_agree / (n_steps * B) >= 0.97
+    ctx.close()
+
+
+def test_spec_step_equals_three_calls_and_commits_state():
+    """gm_spec_step == gm_draft; gm_verify; gm_accept(commit) bit for bit, and the committed state follows
+    the cycle's rules (kv_len += a+1, pending pairs = accepted drafts + final token with their hiddens)."""
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny").with_(prompt_len=33)
+    K, B, V, d = cfg.k, cfg.batch, cfg.vocab, cfg.d_model
+    w, ost, ctx, gst = tiny_setup(cfg, cap_tokens=160)
+    bufs = _bufs(B, K, V, d)
+    seed = 11
+    push_state(ost, gst, ctx)
+    snap = {n: getattr(gst, n).clone() for n in ("kv_len", "pending_n", "pending_tok", "pending_hidden", "kv_pool",
+                                                   "head_kv_pool")}
+    hist_a = []
+    for it in range(6):
+        _run_phases(gmb, ctx, gst, K, seed, 100 + it, bufs, commit=True)
+        a, t = bufs["a"].cpu().numpy(), bufs["t"].cpu().numpy()
+        hist_a.append((a.copy(), t.copy(), bufs["draft_tok"].cpu().numpy().copy()))
+        kv_prev = snap["kv_len"].cpu().numpy() if it == 0 else kv_after
+        kv_after = gst.kv_len.cpu().numpy()
+        np.testing.assert_array_equal(kv_after, kv_prev + a + 1)
+        np.testing.assert_array_equal(gst.pending_n.cpu().numpy(), a + 1)
+        pt, ph = gst.pending_tok.cpu().numpy(), gst.pending_hidden.float().cpu().numpy()
+        th = bufs["tgt_hidden"].float().cpu().numpy()
+        for b in range(B):
+            np.testing.assert_array_equal(pt[b, :a[b]], hist_a[-1][2][b, :a[b]])
+            assert pt[b, a[b]] == t[b]
+            np.testing.assert_array_equal(ph[b, :a[b] + 1], th[b, :a[b] + 1])
+    final = {n: getattr(gst, n).clone() for n in snap}
+    # replay with the fused call
+    for n, v in snap.items():
+        getattr(gst, n).copy_(v)
+    a2, t2 = torch.zeros_like(bufs["a"]), torch.zeros_like(bufs["t"])
+    dt2 = torch.zeros_like(bufs["draft_tok"])
+    for it in range(6):
+        gmb.gm_spec_step(ctx, gst, K, 1.0, seed, 100 + it, a2, t2, dt2)
+        np.testing.assert_array_equal(a2.cpu().numpy(), hist_a[it][0])
+        np.testing.assert_array_equal(t2.cpu().numpy(), hist_a[it][1])
+        np.testing.assert_array_equal(dt2.cpu().numpy(), hist_a[it][2])
+    assert gmb.gm_last_status(ctx) == 0
+    for n, v in final.items():
+        assert torch.equal(getattr(gst, n), v), n
+    # host-buffer form
+    for n, v in snap.items():
+        getattr(gst, n).copy_(v)
+    ah = torch.zeros(B, dtype=torch.int32).pin_memory()
+    th_ = torch.zeros(B, dtype=torch.int32).pin_memory()
+    gmb.gm_spec_step_host(ctx, gst, K, 1.0, seed, 100, ah, th_)
+    np.testing.assert_array_equal(ah.numpy(), hist_a[0][0])
+    np.testing.assert_array_equal(th_.numpy(), hist_a[0][1])
+    ctx.close()
+
+
+def test_free_running_rollout_keeps_caches_consistent():
+    """Let the device run many committed cycles on its own, then check its caches against an oracle
+    recomputation of the committed sequence: target KV everywhere, head KV behind the boundary."""
+    import paper_2609_16648_b200 as gmb
+    from oracle import model as omodel
+    cfg = get_config("tiny").with_(prompt_len=20)
+    K, B = cfg.k, cfg.batch
+    w, ost, ctx, gst = tiny_setup(cfg, cap_tokens=200)
+    push_state(ost, gst, ctx)
+    a = torch.zeros(B, dtype=torch.int32, device="cuda")
+    t = torch.zeros(B, dtype=torch.int32, device="cuda")
+    dt = torch.zeros((B, K), dtype=torch.int32, device="cuda")
+    seqs = [list(s.tokens) for s in ost.seqs]
+    n_acc = 0
+    for it in range(30):
+        gmb.gm_spec_step(ctx, gst, K, 1.0, 77, it, a, t, dt)
+        an, tn, dn = a.cpu().numpy(), t.cpu().numpy(), dt.cpu().numpy()
+        for b in range(B):
+            seqs[b] += [int(x) for x in dn[b, :an[b]]] + [int(tn[b])]
+            n_acc += an[b]
+    assert gmb.gm_last_status(ctx) == 0
+    kv_len = gst.kv_len.cpu().numpy()
+    pool = gst.kv_pool.float().cpu().numpy()
+    hpool = gst.head_kv_pool.float().cpu().numpy()
+    pn = gst.pending_n.cpu().numpy()
+    assert n_acc > 0
+    for b in range(B):
+        assert kv_len[b] == len(seqs[b]) - 1
+        L1 = int(kv_len[b])
+        kv = omodel.PagedKV(cfg.n_layers, cfg.n_kv_heads, cfg.head_dim, ost.kv.table, ost.kv.pool.shape[2])
+        H = omodel.target_forward(w, seqs[b][:L1], np.arange(L1), kv, b, cfg)
+        dev_kv = omodel.PagedKV(cfg.n_layers, cfg.n_kv_heads, cfg.head_dim, ost.kv.table, ost.kv.pool.shape[2])
+        dev_kv.pool = pool.astype(np.float64)
+        for l in range(cfg.n_layers):
+            for x, y in zip(dev_kv.gather(l, b, L1), kv.gather(l, b, L1)):
+                assert rel_err(x, y) < TOL
+        m = L1 - int(pn[b])
+        hkv = omodel.PagedKV(1, cfg.n_kv_heads, cfg.head_dim, ost.hkv.table, ost.hkv.pool.shape[2])
+        omodel.head_forward(w, H[:m], seqs[b][1:m + 1], np.arange(m), hkv, b, cfg)
+        dev_h = omodel.PagedKV(1, cfg.n_kv_heads, cfg.head_dim, ost.hkv.table, ost.hkv.pool.shape[2])
+        dev_h.pool = hpool.astype(np.float64)
+        for x, y in zip(dev_h.gather(0, b, m), hkv.gather(0, b, m)):
+            assert rel_err(x, y) < TOL
+    ctx.close()
+
+
+def test_device_seen_errors_and_host_validation():
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny").with_(prompt_len=20)
+    K, B = cfg.k, cfg.batch
+    w, ost, ctx, gst = tiny_setup(cfg, cap_tokens=32)       # 2 pages per row only
+    push_state(ost, gst, ctx)
+    a = torch.zeros(B, dtype=torch.int32, device="cuda")
+    t = torch.zeros(B, dtype=torch.int32, device="cuda")
+    with pytest.raises(gmb.GmError) as e:
+        gmb.gm_spec_step(ctx, gst, K + 1, 1.0, 0, 0, a, t)
+    assert e.value.code == gmb.GM_ERR_UNSUPPORTED
+    with pytest.raises(gmb.GmError) as e:
+        gmb.gm_spec_step(ctx, gst, K, -1.0, 0, 0, a, t)
+    assert e.value.code == gmb.GM_ERR_UNSUPPORTED
+    with pytest.raises(gmb.GmError) as e:
+        gmb.gm_spec_step(ctx, gst, K, 1.0, 0, 0, None, t)
+    assert e.value.code == gmb.GM_ERR_INVALID_ARG
+    # run until a row outgrows its two pages: the device reports it, nothing faults
+    code = 0
+    for it in range(12):
+        gmb.gm_spec_step(ctx, gst, K, 1.0, 3, it, a, t)
+        code = gmb.gm_last_status(ctx)
+        if code:
+            break
+    assert code == gmb.GM_ERR_KV_CAPACITY
+    # a page id outside the pool is reported too
+    w2, ost2, ctx2, gst2 = tiny_setup(cfg, cap_tokens=96)
+    push_state(ost2, gst2, ctx2)
+    gst2.page_table[1, 1] = 10 ** 6
+    gmb.gm_spec_step(ctx2, gst2, K, 1.0, 3, 0, a, t)
+    assert gmb.gm_last_status(ctx2) == gmb.GM_ERR_BAD_PAGE
+    ctx.close()
+    ctx2.close()
