@@ -76,8 +76,12 @@ def prefill(w, cfg, prompts, page_table, num_pages, head_page_table, head_num_pa
 
 
 def draft(w, cfg, st: BatchState, b: int, K: int, temperature: float, u24_draft,
-          round_interface=True):
-    """K recurrent applications of the head; returns (d[K], draft_logits[K, V], q[K, V])."""
+          round_interface=True, forced=None):
+    """K recurrent applications of the head; returns (d[K], draft_logits[K, V], q[K, V]).
+
+    ``forced``: K recorded draft tokens to feed back instead of sampling (the draft-path
+    reconstruction of Eq. 4: s_{k+1} = [s_k, d_k] with the recorded d_k, nothing sampled); the
+    distributions q_k are then those the head assigns along that recorded path."""
     s = st.seqs[b]
     n = len(s.pending_tok)
     L1 = s.kv_len                       # = Len - 1
@@ -89,7 +93,7 @@ def draft(w, cfg, st: BatchState, b: int, K: int, temperature: float, u24_draft,
         lg = _maybe_round(head_logits(w, g, cfg)[0], round_interface)
         q = sampler.softmax_probs(lg, temperature)
         tok, _ = sampler.draw_token(q, u24_draft[k - 1])
-        d.append(tok)
+        d.append(tok if forced is None else int(forced[k - 1]))
         logits_out.append(lg)
         q_out.append(q)
     return d, np.array(logits_out), np.array(q_out)
@@ -116,15 +120,17 @@ def commit(st: BatchState, b: int, d, a: int, t_star: int, H):
 
 def spec_step(w, cfg, st: BatchState, K: int, temperature: float = 1.0, seed: int = 0,
               do_commit: bool = True, round_interface: bool = True,
-              u24_draft=None, u24_accept=None):
-    """One cycle for every sequence.  Returns a dict of per-row outputs."""
+              u24_draft=None, u24_accept=None, forced_draft=None):
+    """One cycle for every sequence.  Returns a dict of per-row outputs.  ``forced_draft`` [B, K]
+    replays recorded draft tokens (see ``draft``)."""
     B = len(st.seqs)
     ud = philox.u24_draft(seed, st.step, B, K) if u24_draft is None else u24_draft
     ua = philox.u24_accept(seed, st.step, B, K) if u24_accept is None else u24_accept
     out = {k: [] for k in ("draft_tok", "draft_logits", "q", "target_logits", "target_hidden",
                            "p", "accept_len", "next_token", "warn")}
     for b in range(B):
-        d, dl, q = draft(w, cfg, st, b, K, temperature, ud[b], round_interface)
+        d, dl, q = draft(w, cfg, st, b, K, temperature, ud[b], round_interface,
+                         None if forced_draft is None else forced_draft[b])
         tl, H, p = verify(w, cfg, st, b, d, temperature, round_interface)
         a, t_star, warn = sampler.decide(p, q, d, ua[b])
         if do_commit:

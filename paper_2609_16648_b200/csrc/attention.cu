@@ -68,8 +68,11 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int B = A.batch;
-  const long long G = gridDim.x;
   const long long P = A.page_start[B];
+  // never more ranges than pages: every active CTA then owns at least one page, so the CTAs that hold
+  // pieces of one sequence are consecutive and so are its segment ids
+  const long long G = P < static_cast<long long>(gridDim.x) ? P : static_cast<long long>(gridDim.x);
+  if (static_cast<long long>(blockIdx.x) >= G) return;
   const int lo = static_cast<int>(blockIdx.x * P / G), hi = static_cast<int>((blockIdx.x + 1) * P / G);
   const int hg = blockIdx.y;                    // head group (n_kv > 8)
 
@@ -307,7 +310,8 @@ cudaError_t launch_attention(const AttnArgs &A, cudaStream_t stream) {
 __global__ void __launch_bounds__(128) attention_combine_kernel(const AttnCombineArgs A) {
   const int b = blockIdx.x / A.n_kv, head = blockIdx.x % A.n_kv;
   const int qn = A.qn[b];
-  const long long P = A.page_start[A.batch], G = A.n_ctas;
+  const long long P = A.page_start[A.batch];
+  const long long G = P < static_cast<long long>(A.n_ctas) ? P : static_cast<long long>(A.n_ctas);   // as in the kernel above
   const int ps = A.page_start[b], pe = A.page_start[b + 1];
   if (qn <= 0 || pe <= ps) return;
   const int s_first = cta_of_page(ps, P, G) + b, s_last = cta_of_page(pe - 1, P, G) + b;

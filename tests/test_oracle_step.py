@@ -168,3 +168,23 @@ def test_committed_tokens_follow_the_target_autoregressive_law():
     chi, pv = stats.chisquare(counts.ravel()[keep], expect.ravel()[keep] * counts.ravel()[keep].sum() / expect.ravel()[keep].sum())
     assert pv > 1e-4, (chi, pv)
     assert acc > 0.05 * N                          # drafts do get accepted, so the test exercises both branches
+
+
+def test_forced_drafts_replay_the_recorded_path():
+    """Feeding a cycle's own drafts back reproduces it exactly (Eq. 4: the reconstruction consumes the
+    recorded drafts and samples nothing); other drafts change q_2.. and p_2.. but not q_1, p_1."""
+    w, st, _ = _setup()
+    K = 3
+    free = step.spec_step(w, CFG, st, K, seed=5, do_commit=False, round_interface=False)
+    same = step.spec_step(w, CFG, st, K, seed=5, do_commit=False, round_interface=False,
+                          forced_draft=free["draft_tok"])
+    for key in ("draft_tok", "accept_len", "next_token"):
+        np.testing.assert_array_equal(free[key], same[key])
+    np.testing.assert_allclose(free["q"], same["q"], rtol=1e-12)
+    other = (free["draft_tok"] + 1) % CFG.vocab
+    alt = step.spec_step(w, CFG, st, K, seed=5, do_commit=False, round_interface=False, forced_draft=other)
+    np.testing.assert_array_equal(alt["draft_tok"], other)
+    np.testing.assert_allclose(alt["q"][:, 0], free["q"][:, 0], rtol=1e-12)
+    np.testing.assert_allclose(alt["p"][:, 0], free["p"][:, 0], rtol=1e-12)
+    assert np.abs(alt["q"][:, 1] - free["q"][:, 1]).max() > 1e-7
+    assert np.abs(alt["p"][:, 1] - free["p"][:, 1]).max() > 1e-7
