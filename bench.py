@@ -1,0 +1,446 @@
+#!/usr/bin/env python
+"""Benchmark of one speculative-decoding rollout step (draft k tokens, verify k+1 positions, accept).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 4b] [--impl reference]
+
+Prints ONE JSON line.  A "step" is one whole cycle (gm_spec_step: all draft applications, the target
+verify forward over the paged KV cache, rejection sampling and the state commit) over one batch of
+seeded synthetic sequences; consecutive steps feed on each other's committed state.  `value` is the
+whole-job committed tokens per second with all inputs resident in HBM; `e2e` is the same metric
+through the host-buffer entry point (uniforms copied from pinned host memory, results copied back,
+every step).  With N > 1 every rank runs an independent replica (no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "committed_tokens_per_s"
+UNIT = "tokens/s"
+SMI_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            p = json.load(open(path))
+            return float(p["hbm_gbs"]), float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "measured"
+        except Exception:
+            pass
+    return 6650.0, 1400.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs (read-only)."""
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.gpu = [], None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={SMI_QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[1]))
+                mx.append(float(r[2]))
+                for n, v in zip(names, r[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                continue
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---- workload -------------------------------------------------------------------------------------------------------
+
+def lengths_for(cfg, seed):
+    from synth_inputs import kv_lengths_lognormal, kv_lengths_uniform
+    if cfg.length_law == "lognormal":
+        return kv_lengths_lognormal(cfg.batch, 4096, 0.7, cfg.kv_len_min, cfg.kv_len_max, seed)
+    return kv_lengths_uniform(cfg.batch, cfg.kv_len_min, cfg.kv_len_max, seed)
+
+
+def build_workload(name: str, rank: int, total_steps: int, k: int, device):
+    """Random-init model of the named shape + a batch of sequences with ragged, fragmented KV caches."""
+    import torch
+    import paper_2609_16648_b200 as gmb
+    from synth_inputs import get_config, make_page_tables
+    cfg = get_config(name)
+    cfg = cfg.with_(k=k)
+    lens = lengths_for(cfg, seed=3 + rank).astype(np.int64)
+    free_b, _ = torch.cuda.mem_get_info()
+    w_bytes = 2 * (cfg.target_params() + cfg.layer_params() + 2 * cfg.d_model ** 2 + cfg.vocab * cfg.d_model)
+    logits_bytes = 2 * cfg.batch * (2 * k + 1) * cfg.vocab
+    budget = free_b - w_bytes - logits_bytes - (8 << 30)
+    grow = total_steps * (k + 1) + 2 * (k + 1)
+    per_tok = cfg.kv_bytes_per_token() + cfg.kv_bytes_per_token(1)
+    # keep the first B' sequences whose caches fit (the 7B and long-tail batches exceed one GPU as written)
+    keep, used = 0, 0
+    for b in range(cfg.batch):
+        need = ((lens[b] + grow + 15) // 16) * 16 * per_tok
+        if used + need > budget:
+            break
+        used += need
+        keep += 1
+    if keep == 0:
+        raise RuntimeError("no sequence fits in device memory")
+    lens = lens[:keep]
+    cfg = cfg.with_(batch=keep)
+    cap = lens + grow
+    pt, npg = make_page_tables(cap, 16, seed=7 + rank)
+    hpt, hnpg = make_page_tables(cap, 16, seed=8 + rank)
+    packed = gmb.random_packed_weights(cfg, device, seed=rank)
+    ctx = gmb.Context(cfg, packed, keep, k, pt.shape[1], npg, hnpg)
+    st = gmb.State(ctx, keep, np.where(pt < 0, 0, pt), np.where(hpt < 0, 0, hpt), device)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(100 + rank)
+
+    def fill(t):                                    # N(0,1) keys/values, in slabs
+        flat = t.view(-1)
+        step = 1 << 28
+        for i in range(0, flat.numel(), step):
+            n = min(step, flat.numel() - i)
+            flat[i:i + n] = torch.randn(n, device=device, generator=gen, dtype=torch.float32).to(torch.bfloat16)
+
+    fill(st.kv_pool)
+    fill(st.head_kv_pool)
+    st.kv_len.copy_(torch.from_numpy(lens.astype(np.int32)))
+    st.pending_n.fill_(1)
+    st.pending_tok.copy_(torch.randint(0, cfg.vocab, st.pending_tok.shape, device=device, generator=gen, dtype=torch.int32))
+    st.pending_hidden.copy_(torch.randn(st.pending_hidden.shape, device=device, generator=gen).to(torch.bfloat16))
+    torch.cuda.synchronize()
+    return cfg, ctx, st, lens
+
+
+def algorithmic_bytes_per_step(cfg, k, sum_len):
+    """What one cycle must move at least once: weights, KV, logits (bytes)."""
+    d, V = cfg.d_model, cfg.vocab
+    verify_w = 2 * cfg.target_params()
+    draft_w = k * 2 * (cfg.layer_params() + 2 * d * d + V * d)
+    kv = sum_len * cfg.kv_bytes_per_token() + k * sum_len * cfg.kv_bytes_per_token(1)
+    logits = 2 * 2 * cfg.batch * (2 * k + 1) * V
+    return verify_w + draft_w + kv + logits
+
+
+# ---- CPU oracle leg -----------------------------------------------------------------------------------------------------
+
+class OracleSample:
+    """Times the oracle, as it stands, on a bounded sample of the workload: ONE sequence of the named
+    shape at a typical KV length through the draft head (k applications), ONE of the target's decoder
+    layers, the LM head and the sampler; the layer time is multiplied by the layer count
+    (extrapolated).  The weights are generated once and handed over as float64 arrays, so that the
+    oracle's up-casts are no-ops and the time is spent on its arithmetic."""
+
+    def __init__(self, name: str, k: int, kv_len: int = 4608):
+        from oracle import model as omodel
+        from synth_inputs import get_config, make_page_tables, make_weights
+        t0 = time.time()
+        self.name, self.k, self.kv_len = name, k, kv_len
+        self.n_layers = get_config(name).n_layers
+        self.cfg = cfg = get_config(name).with_(k=k, batch=1)
+        if name == "tiny":
+            self.kv_len = kv_len = 200
+        w = make_weights(cfg, 0, n_layers=1)
+
+        def up(o):
+            if isinstance(o, dict):
+                return {k_: up(v) for k_, v in o.items()}
+            if isinstance(o, list):
+                return [up(v) for v in o]
+            return np.asarray(o, dtype=np.float64)
+        self.w = up(w)
+        rng = np.random.default_rng(0)
+        pt, npg = make_page_tables(np.array([kv_len + 2 * (k + 1)]), 16, seed=1)
+        self.kv = omodel.PagedKV(1, cfg.n_kv_heads, cfg.head_dim, pt, npg)
+        self.hkv = omodel.PagedKV(1, cfg.n_kv_heads, cfg.head_dim, pt, npg)
+        self.kv.pool[:] = rng.standard_normal(self.kv.pool.shape)
+        self.hkv.pool[:] = rng.standard_normal(self.hkv.pool.shape)
+        self.setup_s = time.time() - t0
+
+    def run(self, seed: int = 0):
+        from oracle import model as omodel, philox, sampler as osampler
+        cfg, w, k, kv_len = self.cfg, self.w, self.k, self.kv_len
+        rng = np.random.default_rng(seed)
+        hidden = rng.standard_normal((1, cfg.d_model))
+        tok = [int(rng.integers(cfg.vocab))]
+        t1 = time.time()
+        g = omodel.head_forward(w, hidden, tok, np.array([kv_len - 1]), self.hkv, 0, cfg)
+        d, q = [], []
+        for j in range(k):
+            if j > 0:
+                g = omodel.head_forward(w, g, [d[-1]], np.array([kv_len - 1 + j]), self.hkv, 0, cfg)
+            qj = osampler.softmax_probs(omodel.round_bf16(omodel.head_logits(w, g, cfg)[0]))
+            d.append(osampler.draw_token(qj, philox.u24(seed, 1, 0, j))[0])
+            q.append(qj)
+        t_draft = time.time() - t1
+        t3 = time.time()
+        x = w["embed"][tok + d]
+        H = omodel.decoder_layer(w["layers"][0], x, np.arange(kv_len, kv_len + k + 1), self.kv, 0, 0, cfg)
+        t_layer = time.time() - t3
+        t4 = time.time()
+        p = osampler.softmax_probs(omodel.round_bf16(omodel.target_logits(w, H, cfg)))
+        a, _, _ = osampler.decide(p, np.array(q), d, philox.u24_accept(seed, 1, 1, k)[0])
+        t_tail = time.time() - t4
+        step_s = t_draft + self.n_layers * t_layer + t_tail
+        return {"step_s": step_s, "committed": int(a + 1), "t_draft": t_draft, "t_layer": t_layer, "t_tail": t_tail,
+                "cpu_s": time.time() - t1}
+
+    def describe(self, runs, cpu_s):
+        import torch
+        return (f"{runs} x [1 sequence of the {self.name} shape at kv_len {self.kv_len}, k={self.k}: draft head x{self.k}, "
+                f"1 of {self.n_layers} target layers (its time extrapolated x{self.n_layers}), LM head + sampler]; "
+                f"{cpu_s:.1f} s of CPU work; sequences run one after another on the CPU, so tokens/s does not depend on "
+                f"the batch; float64 weights prepared once ({self.setup_s:.0f} s, excluded); "
+                f"BLAS threads {torch.get_num_threads()}")
+
+
+def host_cores():
+    return len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+
+
+def cpu_baseline(name: str, k: int, budget_s: float = 15.0, max_runs: int = 40):
+    smp = OracleSample(name, k)
+    runs, t0 = [], time.time()
+    while len(runs) < max_runs and (not runs or time.time() - t0 < budget_s):
+        runs.append(smp.run(seed=len(runs)))
+    value = sum(r["committed"] for r in runs) / sum(r["step_s"] for r in runs)
+    return {"value": value, "unit": UNIT, "cores": host_cores(), "kind": "oracle",
+            "sample": smp.describe(len(runs), sum(r["cpu_s"] for r in runs))}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    smp = OracleSample(args.workload, args.k)
+    runs = []
+    for i in range(args.warmup + args.steps):
+        r = smp.run(seed=i)
+        if i >= args.warmup:
+            runs.append(r)
+    value = sum(r["committed"] for r in runs) / sum(r["step_s"] for r in runs)
+    secs = float(np.mean([r["step_s"] for r in runs]))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "k": args.k,
+                       "note": "CPU oracle; every step is a bounded sample (one sequence, one layer extrapolated)"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_cores(), "kind": "oracle",
+                             "sample": smp.describe(len(runs), sum(r["cpu_s"] for r in runs))},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ---- product leg ---------------------------------------------------------------------------------------------------------
+
+def run_product(args):
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    from paper_2609_16648_b200.build import build
+    if rank == 0:
+        build()
+    if world > 1:
+        dist.barrier()
+    import paper_2609_16648_b200 as gmb
+
+    K, W, S = args.k, args.warmup, args.steps
+    total_steps = W + 2 * S + 12
+    cfg, ctx, st, lens = build_workload(args.workload, rank, total_steps, K, device)
+    B = cfg.batch
+    a_dev = torch.zeros(B, dtype=torch.int32, device=device)
+    t_dev = torch.zeros(B, dtype=torch.int32, device=device)
+    acc_sum = torch.zeros(1, dtype=torch.int64, device=device)
+    seed = 1234 + rank
+    step_id = 0
+
+    def one_step():
+        nonlocal step_id
+        gmb.gm_spec_step(ctx, st, K, 1.0, seed, step_id, a_dev, t_dev)
+        acc_sum.add_(a_dev.sum())
+        step_id += 1
+
+    for _ in range(W):
+        one_step()
+    torch.cuda.synchronize()
+    if gmb.gm_last_status(ctx) != 0:
+        raise RuntimeError("device status set during warm-up")
+    acc_sum.zero_()
+    len0 = int(st.kv_len.sum().item())
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    clocks = ClockSampler(local)
+    gmb.gm_profile(ctx, 1 << gmb.GM_KC_ATTENTION)
+    launches0 = gmb.gm_launch_count(ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    clocks.start()
+    e0.record()
+    for _ in range(S):
+        one_step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clk = clocks.stop()
+    launches = gmb.gm_launch_count(ctx) - launches0
+    att_ms, att_n = gmb.gm_profile_read(ctx, gmb.GM_KC_ATTENTION)
+    gmb.gm_profile(ctx, 0)
+    accepted = int(acc_sum.item())
+    committed = accepted + S * B
+    len1 = int(st.kv_len.sum().item())
+    status = gmb.gm_last_status(ctx)
+    if status != 0:
+        raise RuntimeError(f"device status {status} ({gmb.gm_strerror(status)}) during the timed region")
+
+    # ---- optional: device time per kernel class, from a separate pass with every launch bracketed by events ---------
+    breakdown = None
+    if args.breakdown:
+        gmb.gm_profile(ctx, 0xF)
+        nb = min(S, 5)
+        for _ in range(nb):
+            one_step()
+        names = {gmb.GM_KC_GEMM: "gemm", gmb.GM_KC_ATTENTION: "attention", gmb.GM_KC_ELEMENTWISE: "elementwise",
+                 gmb.GM_KC_SAMPLER: "sampler"}
+        breakdown = {}
+        for cls, nm in names.items():
+            t_ms, n = gmb.gm_profile_read(ctx, cls)
+            breakdown[nm] = {"ms_per_step": t_ms / nb, "launches_per_step": n / nb}
+        gmb.gm_profile(ctx, 0)
+
+    # ---- end to end through the host-buffer entry point -------------------------------------------------------------
+    ud_h = torch.randint(0, 1 << 24, (B, K), dtype=torch.int32).pin_memory()
+    ua_h = torch.randint(0, 1 << 24, (B, K + 1), dtype=torch.int32).pin_memory()
+    a_h = torch.zeros(B, dtype=torch.int32).pin_memory()
+    t_h = torch.zeros(B, dtype=torch.int32).pin_memory()
+    d_h = torch.zeros((B, K), dtype=torch.int32).pin_memory()
+    gmb.gm_spec_step_host(ctx, st, K, 1.0, seed, step_id, a_h, t_h, d_h, ud_h, ua_h)      # warm the path
+    barrier()
+    t0 = time.perf_counter()
+    committed_e2e = 0
+    for i in range(S):
+        gmb.gm_spec_step_host(ctx, st, K, 1.0, seed, step_id + 1 + i, a_h, t_h, d_h, ud_h, ua_h)
+        committed_e2e += int(a_h.sum()) + B
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    h2d = int(ud_h.numel() + ua_h.numel()) * 4
+    d2h = int(a_h.numel() + t_h.numel() + d_h.numel()) * 4
+
+    # ---- reduce over ranks (max time, summed tokens) ---------------------------------------------------------------------
+    stats = torch.tensor([ms, e2e_s * 1e3], dtype=torch.float64, device=device)
+    toks = torch.tensor([committed, committed_e2e, launches, B], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
+        dist.all_reduce(toks, op=dist.ReduceOp.SUM)
+    ms_max, e2e_ms_max = stats.tolist()
+    committed_all, committed_e2e_all, launches_all, batch_all = toks.tolist()
+
+    if rank == 0:
+        hbm, tflops, which = measured_peaks()
+        sum_len_avg = 0.5 * (len0 + len1) + B * (K + 1)               # positions attended per launch (incl. new ones)
+        att_bytes = sum_len_avg * cfg.kv_bytes_per_token(1)
+        att_avg_ms = att_ms / max(att_n, 1)
+        achieved = att_bytes / (att_avg_ms * 1e-3) / 1e9
+        step_bytes = algorithmic_bytes_per_step(cfg, K, 0.5 * (len0 + len1))
+        step_roof_ms = step_bytes / (hbm * 1e9) * 1e3
+        line = {
+            "metric": METRIC, "value": committed_all / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": S,
+            "warmup": W, "ms_per_step": ms_max / S, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "batch_per_gpu": B, "k": K, "temperature": 1.0,
+                       "kv_len_mean": float(lens.mean()), "kv_len_min": int(lens.min()), "kv_len_max": int(lens.max()),
+                       "page": 16, "tau": committed / (S * B), "parallelism": f"replicas x{world}",
+                       "l2": "per-step working set (weights + KV, tens of GB) >> 126 MB L2: no flush needed",
+                       "step_algorithmic_GB": step_bytes / 1e9, "step_roofline_ms": step_roof_ms,
+                       "step_roofline_frac": step_roof_ms / (ms / S), "peaks": which},
+            "clocks": clk,
+            "e2e": {"value": committed_e2e_all / (e2e_ms_max * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_max / S},
+            "gpu_launches": int(launches_all),
+            "roofline": {"kernel": "attention_kernel (paged multi-query decode attention, one layer per launch)",
+                         "bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s", "frac": achieved / hbm,
+                         "traffic": None, "launches": int(att_n), "avg_launch_ms": att_avg_ms,
+                         "algorithmic_bytes_per_launch": att_bytes, "peak_source": which},
+        }
+        if breakdown is not None:
+            line["config"]["breakdown"] = breakdown
+        if not args.no_cpu_baseline and world >= 1:
+            try:
+                line["cpu_baseline"] = cpu_baseline(args.workload, K)
+            except Exception as exc:                        # the baseline is reported, never required
+                line["cpu_baseline"] = {"value": None, "unit": UNIT, "cores": 0, "kind": "oracle",
+                                        "sample": f"failed: {exc}"}
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="4b", choices=["tiny", "4b", "7b", "longtail"])
+    ap.add_argument("--k", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--breakdown", action="store_true", help="add device time per kernel class (extra pass)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_product(args)
+
+
+if __name__ == "__main__":
+    main()

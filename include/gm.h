@@ -166,9 +166,14 @@ int gm_spec_step(gm_ctx *ctx, gm_state *st, int k, float temperature, uint64_t s
 int gm_draw(gm_ctx *ctx, const void *logits, int rows, float temperature, const uint32_t *u24,
             int32_t *out_tok, float *dbg_prob);
 
-/* Host-buffer form of the cycle: copies accept_len / next_token to HOST arrays and waits.   */
+/* Host-buffer form of the cycle, for callers that keep no device memory of their own besides the
+ * state: copies the uniforms from HOST arrays (u24_draft_host [B, k], u24_accept_host [B, k+1]; both
+ * NULL = Philox from seed/step), runs the cycle, copies accept_len [B], next_token [B] and (if not
+ * NULL) draft_tok [B, k] back to HOST arrays and waits for the stream.  Pinned host memory makes the
+ * copies asynchronous.                                                                        */
 int gm_spec_step_host(gm_ctx *ctx, gm_state *st, int k, float temperature, uint64_t seed,
-                      uint64_t step, int32_t *accept_len_host, int32_t *next_token_host);
+                      uint64_t step, const uint32_t *u24_draft_host, const uint32_t *u24_accept_host,
+                      int32_t *accept_len_host, int32_t *next_token_host, int32_t *draft_tok_host);
 
 /* Dense projection out[M, N] = x[M, K] w[N, K]^T on the context's stream (bf16 in, fp32
  * accumulate; the kernel every QKV / O / FFN / LM-head projection of the step uses).

@@ -70,7 +70,7 @@ def lib() -> C.CDLL:
     L.gm_verify.argtypes = [vp, C.POINTER(gm_state), i32, vp, vp, vp]
     L.gm_accept.argtypes = [vp, C.POINTER(gm_state), i32, i32, f32, vp, vp, vp, vp, u64, u64, vp, vp, vp, vp, vp, i32]
     L.gm_spec_step.argtypes = [vp, C.POINTER(gm_state), i32, f32, u64, u64, vp, vp, vp]
-    L.gm_spec_step_host.argtypes = [vp, C.POINTER(gm_state), i32, f32, u64, u64, vp, vp]
+    L.gm_spec_step_host.argtypes = [vp, C.POINTER(gm_state), i32, f32, u64, u64, vp, vp, vp, vp, vp]
     L.gm_draw.argtypes = [vp, vp, i32, f32, vp, vp, vp]
     L.gm_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
     L.gm_profile.argtypes = [vp, i32]
@@ -254,12 +254,14 @@ def gm_spec_step(ctx: Context, st: State, k: int, temperature: float, seed: int,
 
 
 def gm_spec_step_host(ctx: Context, st: State, k: int, temperature: float, seed: int, step: int, accept_len_host,
-                      next_token_host):
-    """accept_len_host / next_token_host: pinned (or pageable) CPU int32 tensors."""
+                      next_token_host, draft_tok_host=None, u24_draft_host=None, u24_accept_host=None):
+    """All tensor arguments are CPU tensors (pinned for asynchronous copies); int32 / uint32-valued."""
     s = st.struct()
-    assert not accept_len_host.is_cuda and not next_token_host.is_cuda
-    _check(lib().gm_spec_step_host(ctx.handle, C.byref(s), k, temperature, seed, step,
-                                   C.c_void_p(accept_len_host.data_ptr()), C.c_void_p(next_token_host.data_ptr())),
+    hp = lambda t: None if t is None else C.c_void_p(t.data_ptr())
+    for t in (accept_len_host, next_token_host, draft_tok_host, u24_draft_host, u24_accept_host):
+        assert t is None or (not t.is_cuda and t.is_contiguous())
+    _check(lib().gm_spec_step_host(ctx.handle, C.byref(s), k, temperature, seed, step, hp(u24_draft_host),
+                                   hp(u24_accept_host), hp(accept_len_host), hp(next_token_host), hp(draft_tok_host)),
            "gm_spec_step_host")
 
 

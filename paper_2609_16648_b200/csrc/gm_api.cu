@@ -565,26 +565,45 @@ int gm_draw(gm_ctx *c, const void *logits, int rows, float temperature, const ui
   return GM_OK;
 }
 
-int gm_spec_step(gm_ctx *c, gm_state *st, int k, float temperature, uint64_t seed, uint64_t step, int32_t *accept_len,
-                 int32_t *next_token, int32_t *draft_tok) {
+static int spec_step_impl(gm_ctx *c, gm_state *st, int k, float temperature, const uint32_t *u24_draft,
+                          const uint32_t *u24_accept, uint64_t seed, uint64_t step, int32_t *accept_len,
+                          int32_t *next_token, int32_t *draft_tok) {
   int rc = check_state(c, st, k);
   if (rc) return rc;
   if (!accept_len || !next_token) return GM_ERR_INVALID_ARG;
   int32_t *dt = draft_tok ? draft_tok : c->ws_draft_tok;
-  if ((rc = gm_draft(c, st, k, temperature, nullptr, seed, step, dt, c->ws_draft_logits, nullptr)) != GM_OK) return rc;
+  if ((rc = gm_draft(c, st, k, temperature, u24_draft, seed, step, dt, c->ws_draft_logits, nullptr)) != GM_OK) return rc;
   if ((rc = gm_verify(c, st, k, dt, c->ws_target_logits, c->ws_target_hidden)) != GM_OK) return rc;
-  return gm_accept(c, st, st->batch, k, temperature, c->ws_target_logits, c->ws_draft_logits, dt, nullptr, seed, step,
+  return gm_accept(c, st, st->batch, k, temperature, c->ws_target_logits, c->ws_draft_logits, dt, u24_accept, seed, step,
                    accept_len, next_token, nullptr, nullptr, c->ws_target_hidden, 1);
 }
 
+int gm_spec_step(gm_ctx *c, gm_state *st, int k, float temperature, uint64_t seed, uint64_t step, int32_t *accept_len,
+                 int32_t *next_token, int32_t *draft_tok) {
+  return spec_step_impl(c, st, k, temperature, nullptr, nullptr, seed, step, accept_len, next_token, draft_tok);
+}
+
 int gm_spec_step_host(gm_ctx *c, gm_state *st, int k, float temperature, uint64_t seed, uint64_t step,
-                      int32_t *accept_len_host, int32_t *next_token_host) {
-  if (!accept_len_host || !next_token_host) return GM_ERR_INVALID_ARG;
-  int rc = gm_spec_step(c, st, k, temperature, seed, step, c->ws_accept_len, c->ws_next_token, nullptr);
+                      const uint32_t *u24_draft_host, const uint32_t *u24_accept_host, int32_t *accept_len_host,
+                      int32_t *next_token_host, int32_t *draft_tok_host) {
+  int rc = check_state(c, st, k);
   if (rc) return rc;
-  const size_t n = static_cast<size_t>(st->batch) * sizeof(int32_t);
-  GM_CUDA(c, cudaMemcpyAsync(accept_len_host, c->ws_accept_len, n, cudaMemcpyDeviceToHost, c->stream));
-  GM_CUDA(c, cudaMemcpyAsync(next_token_host, c->ws_next_token, n, cudaMemcpyDeviceToHost, c->stream));
+  if (!accept_len_host || !next_token_host) return GM_ERR_INVALID_ARG;
+  if ((u24_draft_host == nullptr) != (u24_accept_host == nullptr)) return GM_ERR_INVALID_ARG;
+  const size_t B = static_cast<size_t>(st->batch);
+  uint32_t *ud = nullptr, *ua = nullptr;
+  if (u24_draft_host) {
+    ud = c->ws_u24;
+    ua = c->ws_u24 + B * k;
+    GM_CUDA(c, cudaMemcpyAsync(ud, u24_draft_host, B * k * sizeof(uint32_t), cudaMemcpyHostToDevice, c->stream));
+    GM_CUDA(c, cudaMemcpyAsync(ua, u24_accept_host, B * (k + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice, c->stream));
+  }
+  rc = spec_step_impl(c, st, k, temperature, ud, ua, seed, step, c->ws_accept_len, c->ws_next_token, c->ws_draft_tok);
+  if (rc) return rc;
+  GM_CUDA(c, cudaMemcpyAsync(accept_len_host, c->ws_accept_len, B * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
+  GM_CUDA(c, cudaMemcpyAsync(next_token_host, c->ws_next_token, B * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
+  if (draft_tok_host)
+    GM_CUDA(c, cudaMemcpyAsync(draft_tok_host, c->ws_draft_tok, B * k * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
   GM_CUDA(c, cudaStreamSynchronize(c->stream));
   return GM_OK;
 }
