@@ -96,13 +96,18 @@ def lengths_for(cfg, seed):
     return kv_lengths_uniform(cfg.batch, cfg.kv_len_min, cfg.kv_len_max, seed)
 
 
-def build_workload(name: str, rank: int, total_steps: int, k: int, device):
-    """Random-init model of the named shape + a batch of sequences with ragged, fragmented KV caches."""
+def build_workload(name: str, rank: int, total_steps: int, k: int, device, layers: int = 0, batch: int = 0):
+    """Random-init model of the named shape + a batch of sequences with ragged, fragmented KV caches.
+    `layers` / `batch` > 0 shrink the model depth / the batch (profiling captures on a few GB)."""
     import torch
     import paper_2609_16648_b200 as gmb
     from synth_inputs import get_config, make_page_tables
     cfg = get_config(name)
     cfg = cfg.with_(k=k)
+    if layers > 0:
+        cfg = cfg.with_(n_layers=layers)
+    if batch > 0:
+        cfg = cfg.with_(batch=batch)
     lens = lengths_for(cfg, seed=3 + rank).astype(np.int64)
     free_b, _ = torch.cuda.mem_get_info()
     w_bytes = 2 * (cfg.target_params() + cfg.layer_params() + 2 * cfg.d_model ** 2 + cfg.vocab * cfg.d_model)
@@ -290,7 +295,7 @@ def run_product(args):
 
     K, W, S = args.k, args.warmup, args.steps
     total_steps = W + 2 * S + 12
-    cfg, ctx, st, lens = build_workload(args.workload, rank, total_steps, K, device)
+    cfg, ctx, st, lens = build_workload(args.workload, rank, total_steps, K, device, args.layers, args.batch)
     B = cfg.batch
     a_dev = torch.zeros(B, dtype=torch.int32, device=device)
     t_dev = torch.zeros(B, dtype=torch.int32, device=device)
@@ -394,7 +399,7 @@ def run_product(args):
             "metric": METRIC, "value": committed_all / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": S,
             "warmup": W, "ms_per_step": ms_max / S, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": args.workload, "batch_per_gpu": B, "k": K, "temperature": 1.0,
+            "config": {"workload": args.workload, "n_layers": cfg.n_layers, "batch_per_gpu": B, "k": K, "temperature": 1.0,
                        "kv_len_mean": float(lens.mean()), "kv_len_min": int(lens.min()), "kv_len_max": int(lens.max()),
                        "page": 16, "tau": committed / (S * B), "parallelism": f"replicas x{world}",
                        "l2": "per-step working set (weights + KV, tens of GB) >> 126 MB L2: no flush needed",
@@ -432,6 +437,8 @@ def main():
     ap.add_argument("--workload", default="4b", choices=["tiny", "4b", "7b", "longtail"])
     ap.add_argument("--k", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (small profiling cases)")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch size (small profiling cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--breakdown", action="store_true", help="add device time per kernel class (extra pass)")
     args = ap.parse_args()
