@@ -307,39 +307,50 @@ cudaError_t launch_attention(const AttnArgs &A, cudaStream_t stream) {
 }
 
 // ---- merge the segments of each sequence ------------------------------------------------------------------------------
+// One warp per (sequence, kv head, query row): lanes first fetch the segments' (max, sum) pairs in parallel,
+// then each lane accumulates its 4 output dimensions over the segments with independent 16-byte loads.
 __global__ void __launch_bounds__(128) attention_combine_kernel(const AttnCombineArgs A) {
   const int b = blockIdx.x / A.n_kv, head = blockIdx.x % A.n_kv;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qn = A.qn[b];
   const long long P = A.page_start[A.batch];
   const long long G = P < static_cast<long long>(A.n_ctas) ? P : static_cast<long long>(A.n_ctas);   // as in the kernel above
   const int ps = A.page_start[b], pe = A.page_start[b + 1];
   if (qn <= 0 || pe <= ps) return;
   const int s_first = cta_of_page(ps, P, G) + b, s_last = cta_of_page(pe - 1, P, G) + b;
+  const int nseg = s_last - s_first + 1;
   const int rows = qn * A.group, hd = A.hd;
-  for (int idx = threadIdx.x; idx < rows * (hd / 4); idx += blockDim.x) {
-    const int row = idx / (hd / 4), c4 = idx % (hd / 4);
+  for (int row = warp; row < rows; row += 4) {
+    const size_t base0 = (static_cast<size_t>(s_first) * A.n_kv + head) * A.qrows + row;
+    const size_t seg_stride = static_cast<size_t>(A.n_kv) * A.qrows;
     float mt = -INFINITY;
-    for (int s = s_first; s <= s_last; ++s)
-      mt = fmaxf(mt, A.part_ml[((static_cast<size_t>(s) * A.n_kv + head) * A.qrows + row) * 2]);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = lane; s < nseg; s += 32) mt = fmaxf(mt, A.part_ml[(base0 + s * seg_stride) * 2]);
+    mt = warp_max(mt);
     float l = 0.f;
-    for (int s = s_first; s <= s_last; ++s) {
-      const size_t base = (static_cast<size_t>(s) * A.n_kv + head) * A.qrows + row;
-      const float ms = A.part_ml[base * 2];
-      if (ms == -INFINITY) continue;
-      const float w = exp2f(ms - mt);
-      l += w * A.part_ml[base * 2 + 1];
-      const float4 ov = reinterpret_cast<const float4 *>(A.part_o + base * hd)[c4];
-      acc.x += w * ov.x; acc.y += w * ov.y; acc.z += w * ov.z; acc.w += w * ov.w;
+    for (int s = lane; s < nseg; s += 32) {
+      const float ms = A.part_ml[(base0 + s * seg_stride) * 2];
+      if (ms != -INFINITY) l += exp2f(ms - mt) * A.part_ml[(base0 + s * seg_stride) * 2 + 1];
     }
+    l = warp_sum(l);
     const float inv = l > 0.f ? 1.f / l : 0.f;
-    const int j = row / A.group, g = row % A.group;
-    __nv_bfloat16 *dst = A.out + (static_cast<size_t>(b) * A.QT + j) * (A.n_kv * A.group * hd) +
-                         (static_cast<size_t>(head) * A.group + g) * hd + c4 * 4;
-    uint2 ov2;
-    ov2.x = pack_bf16(acc.x * inv, acc.y * inv);
-    ov2.y = pack_bf16(acc.z * inv, acc.w * inv);
-    *reinterpret_cast<uint2 *>(dst) = ov2;
+    const int c4 = lane;
+    if (c4 * 4 < hd) {
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+      for (int s = 0; s < nseg; ++s) {
+        const float ms = A.part_ml[(base0 + s * seg_stride) * 2];
+        const float w = ms == -INFINITY ? 0.f : exp2f(ms - mt);
+        const float4 ov = reinterpret_cast<const float4 *>(A.part_o + (base0 + s * seg_stride) * hd)[c4];
+        if (w != 0.f) { acc.x += w * ov.x; acc.y += w * ov.y; acc.z += w * ov.z; acc.w += w * ov.w; }
+      }
+      const int j = row / A.group, g = row % A.group;
+      __nv_bfloat16 *dst = A.out + (static_cast<size_t>(b) * A.QT + j) * (A.n_kv * A.group * hd) +
+                           (static_cast<size_t>(head) * A.group + g) * hd + c4 * 4;
+      uint2 ov2;
+      ov2.x = pack_bf16(acc.x * inv, acc.y * inv);
+      ov2.y = pack_bf16(acc.z * inv, acc.w * inv);
+      *reinterpret_cast<uint2 *>(dst) = ov2;
+    }
   }
 }
 cudaError_t launch_attention_combine(const AttnCombineArgs &A, cudaStream_t stream) {

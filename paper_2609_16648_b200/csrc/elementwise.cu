@@ -162,53 +162,54 @@ cudaError_t launch_head_input(const HeadInputArgs &A, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
-// ---- split-K reduction + residual add + RMSNorm -------------------------------------------------------------------
+// ---- RMSNorm of the fp32 residual stream ------------------------------------------------------------------------------
 __global__ void __launch_bounds__(EW_THREADS)
-reduce_residual_norm_kernel(const float *partial, int nsplit, size_t split_stride, float *x, int add_residual,
-                            const __nv_bfloat16 *w, __nv_bfloat16 *xn, __nv_bfloat16 *hidden_out, int d, float eps) {
+rmsnorm_kernel(const float *x, const __nv_bfloat16 *w, __nv_bfloat16 *xn, __nv_bfloat16 *hidden_out, int d, float eps) {
   const int m = blockIdx.x, d4 = d >> 2;
   float4 v[EW_MAXC];
 #pragma unroll
   for (int c = 0; c < EW_MAXC; ++c) {
     const int i = threadIdx.x + c * EW_THREADS;
     if (i < d4) {
-      float4 acc = add_residual ? reinterpret_cast<const float4 *>(x + static_cast<size_t>(m) * d)[i]
-                                : make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int s = 0; s < nsplit; ++s) {
-        const float4 p = reinterpret_cast<const float4 *>(partial + s * split_stride + static_cast<size_t>(m) * d)[i];
-        acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
-      }
-      v[c] = acc;
-      reinterpret_cast<float4 *>(x + static_cast<size_t>(m) * d)[i] = acc;
+      v[c] = reinterpret_cast<const float4 *>(x + static_cast<size_t>(m) * d)[i];
       if (hidden_out) {
         uint2 o;
-        o.x = pack_bf16(acc.x, acc.y);
-        o.y = pack_bf16(acc.z, acc.w);
+        o.x = pack_bf16(v[c].x, v[c].y);
+        o.y = pack_bf16(v[c].z, v[c].w);
         *reinterpret_cast<uint2 *>(hidden_out + static_cast<size_t>(m) * d + 4 * i) = o;
       }
     }
   }
   if (xn) rmsnorm_store(v, d4, d, eps, w, xn + static_cast<size_t>(m) * d);
 }
-cudaError_t launch_reduce_residual_norm(const float *partial, int nsplit, size_t split_stride, float *x,
-                                        int add_residual, const __nv_bfloat16 *w, __nv_bfloat16 *xn,
-                                        __nv_bfloat16 *hidden_out, int M, int d, float eps, cudaStream_t stream) {
-  reduce_residual_norm_kernel<<<M, EW_THREADS, 0, stream>>>(partial, nsplit, split_stride, x, add_residual, w, xn,
-                                                            hidden_out, d, eps);
+cudaError_t launch_rmsnorm(const float *x, const __nv_bfloat16 *w, __nv_bfloat16 *xn, __nv_bfloat16 *hidden_out,
+                           int M, int d, float eps, cudaStream_t stream) {
+  rmsnorm_kernel<<<M, EW_THREADS, 0, stream>>>(x, w, xn, hidden_out, d, eps);
   return cudaGetLastError();
 }
 
 // ---- rotary embedding + KV append + Q rearrangement --------------------------------------------------------------------
+// One CTA per token row; a work item is 8 consecutive head dimensions (one 16-byte load per half of the
+// rotate-half pair, two 16-byte stores).
+__device__ __forceinline__ void unpack8f(const uint4 &v, float (&x)[8]) {
+  x[0] = bf16_lo(v.x); x[1] = bf16_hi(v.x); x[2] = bf16_lo(v.y); x[3] = bf16_hi(v.y);
+  x[4] = bf16_lo(v.z); x[5] = bf16_hi(v.z); x[6] = bf16_lo(v.w); x[7] = bf16_hi(v.w);
+}
+__device__ __forceinline__ uint4 pack8f(const float (&x)[8]) {
+  return make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+}
 __global__ void __launch_bounds__(EW_THREADS) rope_append_kernel(const RopeAppendArgs A) {
   const int m = blockIdx.x, b = m / A.QT, j = m % A.QT;
   const int hd = A.hd, half = hd >> 1, group = A.n_q / A.n_kv;
   const int ncols = (A.n_q + 2 * A.n_kv) * hd;
   const int qn = A.qn[b];
+  const int hv = half >> 3;                                       // 8-wide items per half head
   __nv_bfloat16 *qdst = A.qbuf + static_cast<size_t>(b) * A.n_kv * A.qrows * hd;
   if (j >= qn) {                           // padding row: zero its query rows, append nothing
-    for (int i = threadIdx.x; i < A.n_q * hd; i += EW_THREADS) {
-      const int h = i / hd, e = i % hd;
-      qdst[(static_cast<size_t>(h / group) * A.qrows + j * group + h % group) * hd + e] = __float2bfloat16(0.f);
+    for (int i = threadIdx.x; i < A.n_q * (hd >> 3); i += EW_THREADS) {
+      const int h = i / (hd >> 3), e = (i % (hd >> 3)) * 8;
+      *reinterpret_cast<uint4 *>(qdst + (static_cast<size_t>(h / group) * A.qrows + j * group + h % group) * hd + e) =
+          make_uint4(0u, 0u, 0u, 0u);
     }
     return;
   }
@@ -216,74 +217,40 @@ __global__ void __launch_bounds__(EW_THREADS) rope_append_kernel(const RopeAppen
   const int page = A.page_table[static_cast<size_t>(b) * A.max_pages_per_seq + (pos >> 4)];
   const bool page_ok = page >= 0 && page < A.num_pages;
   if (!page_ok && threadIdx.x == 0) set_status(A.status, ST_BAD_PAGE);
-  const float *src = A.qkv + static_cast<size_t>(m) * ncols;
-  auto val = [&](int col) {
-    float s = 0.f;
-    for (int sp = 0; sp < A.nsplit; ++sp) s += src[sp * A.split_stride + col];
-    return s;
-  };
+  const __nv_bfloat16 *src = A.qkv + static_cast<size_t>(m) * ncols;
   const float2 *cs = A.rope + static_cast<size_t>(pos) * half;
   const size_t page_elems = static_cast<size_t>(A.n_kv) * 16 * hd;
-  __nv_bfloat16 *kdst = A.pool + ((static_cast<size_t>(A.layer) * 2 + 0) * A.num_pages + page) * page_elems;
-  __nv_bfloat16 *vdst = A.pool + ((static_cast<size_t>(A.layer) * 2 + 1) * A.num_pages + page) * page_elems;
+  __nv_bfloat16 *kdst = A.pool + ((static_cast<size_t>(A.layer) * 2 + 0) * A.num_pages + (page_ok ? page : 0)) * page_elems;
+  __nv_bfloat16 *vdst = A.pool + ((static_cast<size_t>(A.layer) * 2 + 1) * A.num_pages + (page_ok ? page : 0)) * page_elems;
   const int slot = pos & 15;
-  // rotate-half pairs of the query and key heads
-  const int npairs = (A.n_q + A.n_kv) * half;
-  for (int i = threadIdx.x; i < npairs; i += EW_THREADS) {
-    const int h = i / half, e = i % half;
-    const float x1 = val(h * hd + e), x2 = val(h * hd + e + half);
-    const float2 c = cs[e];
-    const float y1 = x1 * c.x - x2 * c.y, y2 = x2 * c.x + x1 * c.y;
-    if (h < A.n_q) {
-      __nv_bfloat16 *dst = qdst + (static_cast<size_t>(h / group) * A.qrows + j * group + h % group) * hd;
-      dst[e] = __float2bfloat16(y1);
-      dst[e + half] = __float2bfloat16(y2);
+  const int n_rot = (A.n_q + A.n_kv) * hv, n_v = A.n_kv * (hd >> 3);
+  for (int i = threadIdx.x; i < n_rot + n_v; i += EW_THREADS) {
+    if (i < n_rot) {
+      const int h = i / hv, e = (i % hv) * 8;
+      float x1[8], x2[8], y1[8], y2[8];
+      unpack8f(*reinterpret_cast<const uint4 *>(src + h * hd + e), x1);
+      unpack8f(*reinterpret_cast<const uint4 *>(src + h * hd + e + half), x2);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        const float2 c = cs[e + t];
+        y1[t] = x1[t] * c.x - x2[t] * c.y;
+        y2[t] = x2[t] * c.x + x1[t] * c.y;
+      }
+      __nv_bfloat16 *dst;
+      if (h < A.n_q) dst = qdst + (static_cast<size_t>(h / group) * A.qrows + j * group + h % group) * hd;
+      else if (page_ok) dst = kdst + (static_cast<size_t>(h - A.n_q) * 16 + slot) * hd;
+      else continue;
+      *reinterpret_cast<uint4 *>(dst + e) = pack8f(y1);
+      *reinterpret_cast<uint4 *>(dst + e + half) = pack8f(y2);
     } else if (page_ok) {
-      __nv_bfloat16 *dst = kdst + (static_cast<size_t>(h - A.n_q) * 16 + slot) * hd;
-      dst[e] = __float2bfloat16(y1);
-      dst[e + half] = __float2bfloat16(y2);
-    }
-  }
-  if (page_ok) {
-    const int vbase = (A.n_q + A.n_kv) * hd;
-    for (int i = threadIdx.x; i < A.n_kv * hd; i += EW_THREADS) {
-      const int h = i / hd, e = i % hd;
-      vdst[(static_cast<size_t>(h) * 16 + slot) * hd + e] = __float2bfloat16(val(vbase + i));
+      const int iv = i - n_rot, h = iv / (hd >> 3), e = (iv % (hd >> 3)) * 8;
+      *reinterpret_cast<uint4 *>(vdst + (static_cast<size_t>(h) * 16 + slot) * hd + e) =
+          *reinterpret_cast<const uint4 *>(src + (A.n_q + A.n_kv) * hd + h * hd + e);
     }
   }
 }
 cudaError_t launch_rope_append(const RopeAppendArgs &A, cudaStream_t stream) {
   rope_append_kernel<<<A.batch * A.QT, EW_THREADS, 0, stream>>>(A);
-  return cudaGetLastError();
-}
-
-// ---- SwiGLU ---------------------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(EW_THREADS)
-swiglu_kernel(const float *gu, int nsplit, size_t split_stride, __nv_bfloat16 *act, size_t total4) {
-  // one thread: 4 outputs = 8 interleaved inputs (gate, up, gate, up, ...)
-  for (size_t i = blockIdx.x * static_cast<size_t>(EW_THREADS) + threadIdx.x; i < total4;
-       i += static_cast<size_t>(gridDim.x) * EW_THREADS) {
-    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), c = a;
-    for (int s = 0; s < nsplit; ++s) {
-      const float4 *p = reinterpret_cast<const float4 *>(gu + s * split_stride) + 2 * i;
-      const float4 u = p[0], w = p[1];
-      a.x += u.x; a.y += u.y; a.z += u.z; a.w += u.w;
-      c.x += w.x; c.y += w.y; c.z += w.z; c.w += w.w;
-    }
-    auto f = [](float g, float u) { return g / (1.f + __expf(-g)) * u; };
-    uint2 o;
-    o.x = pack_bf16(f(a.x, a.y), f(a.z, a.w));
-    o.y = pack_bf16(f(c.x, c.y), f(c.z, c.w));
-    reinterpret_cast<uint2 *>(act)[i] = o;
-  }
-}
-cudaError_t launch_swiglu(const float *gu, int nsplit, size_t split_stride, __nv_bfloat16 *act, int M, int F,
-                          cudaStream_t stream) {
-  const size_t total4 = static_cast<size_t>(M) * F / 4;
-  size_t nb = (total4 + EW_THREADS - 1) / EW_THREADS;
-  if (nb > 148 * 8) nb = 148 * 8;
-  if (nb < 1) nb = 1;
-  swiglu_kernel<<<static_cast<int>(nb), EW_THREADS, 0, stream>>>(gu, nsplit, split_stride, act, total4);
   return cudaGetLastError();
 }
 

@@ -8,48 +8,105 @@
 // stage: a 128 x 64 weight box and a T x 64 activation box); warp 1 owns the tensor memory
 // allocation and one of its threads issues tcgen05.mma (four K=16 instructions per stage),
 // releasing each stage with tcgen05.commit; warps 2-5 read the fp32 accumulator out of tensor
-// memory with tcgen05.ld once the last commit lands and store it transposed (lanes = consecutive
-// features, so stores coalesce).  Optional split-K over blockIdx.z writes fp32 partials that the
-// consumer kernels sum in a fixed order.  Every wait is bounded; on expiry the kernel records
-// ST_TIMEOUT, still meets the final barrier and frees its tensor memory.
+// memory with tcgen05.ld once the last commit lands.
 //
-// gemm_simple_kernel: a plain warp-level mma.sync version with the same interface, kept as an
+// Split-K without a trip through HBM.  Projections with few output tiles (N = d_model gives 20)
+// are cut along K over blockIdx.z, and the CTAs of one output tile form a thread-block cluster.
+// Every CTA parks its accumulator in its own shared memory (the pipeline stages are free by
+// then), the cluster synchronises, and each CTA sums one slice of the tile's tokens over all
+// peers through distributed shared memory in rank order (so the result does not depend on
+// timing) and applies the epilogue: store bf16 / fp32, add into the fp32 residual stream, or
+// SwiGLU on interleaved gate/up rows.  Every wait is bounded; on expiry the kernel records
+// ST_TIMEOUT, still meets every barrier and frees its tensor memory.
+//
+// gemm_simple_kernel: a plain warp-level mma.sync version with the same epilogues, kept as an
 // independent on-device cross-check and for shapes the tcgen05 kernel does not take.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 #include "kernels.h"
 
+namespace cg = cooperative_groups;
+
 namespace gm {
 
-constexpr int GT_BN = 128;            // output features per CTA (MMA M)
+constexpr int GT_BN = 128;            // output features per MMA (its M extent); a CTA owns wt = 1 or 2 such sub-tiles
 constexpr int GT_BK = 64;             // K elements per stage (one 128-byte swizzle row)
 constexpr int GT_THREADS = 192;
 constexpr int GT_SMEM_BUDGET = 200 * 1024;
 
-static int gt_stages(int block_t) {
-  int s = GT_SMEM_BUDGET / (GT_BN * 128 + block_t * 128);
+static int gt_stages(int block_t, int wt) {
+  int s = GT_SMEM_BUDGET / (wt * GT_BN * 128 + block_t * 128);
   return s > 8 ? 8 : s;
 }
-static size_t gt_smem(int block_t) {
-  return static_cast<size_t>(gt_stages(block_t)) * (GT_BN * 128 + block_t * 128) + 1024 + 256;
+static size_t gt_smem(int block_t, int wt) {
+  size_t pipe = static_cast<size_t>(gt_stages(block_t, wt)) * (wt * GT_BN * 128 + block_t * 128);
+  const size_t park = static_cast<size_t>(block_t) * GT_BN * 4;      // one accumulator parked as fp32 [T][128]
+  if (park > pipe) pipe = park;
+  return pipe + 1024 + 256;
+}
+
+// Epilogue on four consecutive features n..n+3 of token row m.
+__device__ __forceinline__ void epilogue4(const GemmArgs &A, int m, int n, float4 v) {
+  if (A.epi == EPI_SWIGLU_BF16) {           // (gate, up, gate, up) -> two outputs
+    if (n + 1 >= A.N) return;
+    const float a0 = v.x / (1.f + __expf(-v.x)) * v.y;
+    __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(A.out) + static_cast<size_t>(m) * A.ldo + (n >> 1);
+    if (n + 3 < A.N) {
+      const float a1 = v.z / (1.f + __expf(-v.z)) * v.w;
+      *reinterpret_cast<uint32_t *>(out) = pack_bf16(a0, a1);
+    } else {
+      out[0] = __float2bfloat16(a0);
+    }
+    return;
+  }
+  const float e[4] = {v.x, v.y, v.z, v.w};
+  if (A.epi == EPI_STORE_BF16) {
+    __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(A.out) + static_cast<size_t>(m) * A.ldo + n;
+    if (n + 3 < A.N && (A.ldo & 3) == 0) {
+      uint2 o;
+      o.x = pack_bf16(v.x, v.y);
+      o.y = pack_bf16(v.z, v.w);
+      *reinterpret_cast<uint2 *>(out) = o;
+    } else {
+      for (int i = 0; i < 4 && n + i < A.N; ++i) out[i] = __float2bfloat16(e[i]);
+    }
+    return;
+  }
+  float *out = reinterpret_cast<float *>(A.out) + static_cast<size_t>(m) * A.ldo + n;
+  if (n + 3 < A.N && (A.ldo & 3) == 0) {
+    float4 o = v;
+    if (A.epi == EPI_ADD_F32) {
+      const float4 r = *reinterpret_cast<const float4 *>(out);
+      o.x += r.x; o.y += r.y; o.z += r.z; o.w += r.w;
+    }
+    *reinterpret_cast<float4 *>(out) = o;
+  } else {
+    for (int i = 0; i < 4 && n + i < A.N; ++i) out[i] = (A.epi == EPI_ADD_F32 ? out[i] : 0.f) + e[i];
+  }
 }
 
 __global__ void __launch_bounds__(GT_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
   extern __shared__ unsigned char gt_smem_raw[];
   unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(gt_smem_raw) + 1023) & ~uintptr_t(1023));
-  const int T = A.block_t;
-  const int a_bytes = GT_BN * 128, b_bytes = T * 128, stage_b = a_bytes + b_bytes;
-  uint64_t *full = reinterpret_cast<uint64_t *>(smem + static_cast<size_t>(nstages) * stage_b);
+  const int T = A.block_t, wt = A.wtiles;
+  const int a_bytes = wt * GT_BN * 128, b_bytes = T * 128, stage_b = a_bytes + b_bytes;
+  size_t pipe_b = static_cast<size_t>(nstages) * stage_b;
+  if (static_cast<size_t>(T) * GT_BN * 4 > pipe_b) pipe_b = static_cast<size_t>(T) * GT_BN * 4;
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem + pipe_b);
   uint64_t *empty = full + 8;
   uint64_t *acc_full = empty + 8;
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  float *park = reinterpret_cast<float *>(smem);                // [T][128] fp32, reuses the pipeline stages
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * GT_BN, m0 = blockIdx.y * T, split = blockIdx.z;
+  const int n0 = blockIdx.x * GT_BN * wt, m0 = blockIdx.y * T, split = blockIdx.z, ns = A.nsplit;
   const int KB = A.K / GT_BK;
-  const int kb_lo = static_cast<int>(static_cast<long long>(split) * KB / A.nsplit);
-  const int kb_hi = static_cast<int>(static_cast<long long>(split + 1) * KB / A.nsplit);
-  const uint32_t ncols = T <= 32 ? 32u : T <= 64 ? 64u : T <= 128 ? 128u : 256u;
+  const int kb_lo = static_cast<int>(static_cast<long long>(split) * KB / ns);
+  const int kb_hi = static_cast<int>(static_cast<long long>(split + 1) * KB / ns);
+  const uint32_t acc_cols = T <= 32 ? 32u : T <= 64 ? 64u : T <= 128 ? 128u : 256u;   // per accumulator
+  const uint32_t ncols = acc_cols * wt;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < nstages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -74,7 +131,7 @@ gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
         if (!mbar_wait(&empty[s], ((it / nstages) & 1) ^ 1)) { set_status(A.status, ST_TIMEOUT); break; }
         mbar_expect_tx(&full[s], stage_b);
         unsigned char *dst = smem + static_cast<size_t>(s) * stage_b;
-        tma_load_2d(dst, &A.w_map, kb * GT_BK, n0, &full[s]);
+        for (int a = 0; a < wt; ++a) tma_load_2d(dst + a * GT_BN * 128, &A.w_map, kb * GT_BK, n0 + a * GT_BN, &full[s]);
         tma_load_2d(dst + a_bytes, &A.x_map, kb * GT_BK, m0, &full[s]);
       }
     }
@@ -87,65 +144,122 @@ gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
         if (!mbar_wait(&full[s], (it / nstages) & 1)) { set_status(A.status, ST_TIMEOUT); ok = false; break; }
         tc_fence_after();
         const uint32_t a_addr = smem_u32(smem + static_cast<size_t>(s) * stage_b);
-        const uint64_t adesc = tc_smem_desc_sw128(a_addr), bdesc = tc_smem_desc_sw128(a_addr + a_bytes);
+        const uint64_t bdesc = tc_smem_desc_sw128(a_addr + a_bytes);
+        for (int a = 0; a < wt; ++a) {
+          const uint64_t adesc = tc_smem_desc_sw128(a_addr + a * GT_BN * 128);
 #pragma unroll
-        for (int k = 0; k < GT_BK / 16; ++k)      // +32 bytes (2 x 16-byte units) per K=16 step
-          tc_mma_bf16(tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < GT_BK / 16; ++k)    // +32 bytes (2 x 16-byte units) per K=16 step
+            tc_mma_bf16(tmem + a * acc_cols, adesc + 2 * k, bdesc + 2 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+        }
         tc_commit(&empty[s]);                      // the stage is free once these MMAs have read it
       }
-      if (ok) tc_commit(acc_full);                 // accumulator complete
+      if (ok) tc_commit(acc_full);                 // accumulators complete
     }
-  } else {
-    // ---- epilogue: TMEM -> registers -> global, transposed --------------------------------------------------
-    const int quad = warp & 3;                     // the TMEM lane quadrant this warp may read
-    const int n = n0 + quad * 32 + lane;
-    bool ok = kb_hi > kb_lo;
-    if (ok && !mbar_wait(acc_full, 0)) { set_status(A.status, ST_TIMEOUT); ok = false; }
+  }
+  bool acc_ok = kb_hi > kb_lo;
+  if (warp >= 2) {
+    if (acc_ok && !mbar_wait(acc_full, 0)) { set_status(A.status, ST_TIMEOUT); acc_ok = false; }
     tc_fence_after();
-    if (ok) {
+  }
+  cg::cluster_group cluster = cg::this_cluster();
+  const int per = (T + ns - 1) / ns;               // this CTA reduces tokens [c_lo, c_hi) of every sub-tile
+  const int c_lo = split * per, c_hi = min(T, c_lo + per);
+  for (int a = 0; a < wt; ++a) {
+    __syncthreads();                               // the pipeline stages (first pass) / the previous sub-tile are done with
+    if (warp >= 2) {
+      // TMEM -> registers -> parked fp32 tile in shared memory (lanes = consecutive features: no bank conflicts)
+      const int quad = warp & 3;                   // the TMEM lane quadrant this warp may read
+      const int r = quad * 32 + lane;
       for (int c0 = 0; c0 < T; c0 += 16) {
-        uint32_t r[16];
-        tc_ld_32x16(tmem + (static_cast<uint32_t>(quad * 32) << 16) + c0, r);
-        tc_wait_ld();
-        if (n < A.N) {
-          if (A.out_fp32) {
-            float *out = reinterpret_cast<float *>(A.out) + split * A.split_stride;
+        uint32_t v[16];
+        if (acc_ok) {
+          tc_ld_32x16(tmem + (static_cast<uint32_t>(quad * 32) << 16) + a * acc_cols + c0, v);
+          tc_wait_ld();
+        } else {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int m = m0 + c0 + j;
-              if (m < A.M) out[static_cast<size_t>(m) * A.ldo + n] = __uint_as_float(r[j]);
-            }
-          } else {
-            __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(A.out);
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int m = m0 + c0 + j;
-              if (m < A.M) out[static_cast<size_t>(m) * A.ldo + n] = __float2bfloat16(__uint_as_float(r[j]));
-            }
-          }
+          for (int j = 0; j < 16; ++j) v[j] = 0u;
         }
+#pragma unroll
+        for (int j = 0; j < 16; ++j) park[(c0 + j) * GT_BN + r] = __uint_as_float(v[j]);
       }
     }
+    __syncthreads();
+    if (ns > 1) cluster.sync();
+    // sum the cluster's K slices in rank order (all peer loads issued before the adds) and apply the epilogue
+    for (int idx = threadIdx.x; idx < (c_hi - c_lo) * (GT_BN / 4); idx += GT_THREADS) {
+      const int c = c_lo + idx / (GT_BN / 4), r4 = (idx % (GT_BN / 4)) * 4;
+      const int m = m0 + c, n = n0 + a * GT_BN + r4;
+      if (m >= A.M || n >= A.N) continue;
+      float4 acc;
+      if (ns == 1) {
+        acc = *reinterpret_cast<const float4 *>(park + c * GT_BN + r4);
+      } else {
+        float4 v[8];
+#pragma unroll
+        for (int p = 0; p < 8; ++p)
+          v[p] = p < ns ? *reinterpret_cast<const float4 *>(cluster.map_shared_rank(park, p) + c * GT_BN + r4)
+                        : make_float4(0.f, 0.f, 0.f, 0.f);
+        acc = v[0];
+#pragma unroll
+        for (int p = 1; p < 8; ++p) { acc.x += v[p].x; acc.y += v[p].y; acc.z += v[p].z; acc.w += v[p].w; }
+      }
+      epilogue4(A, m, n, acc);
+    }
+    if (ns > 1) cluster.sync();                    // peers may still be reading this CTA's parked tile
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tc_dealloc(tmem, ncols);
 }
 
+// The kernel may use the whole opt-in shared memory of an SM (227 KB); set once per process.
+static cudaError_t gt_configure() {
+  static bool done = false;
+  if (done) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) done = true;
+  return e;
+}
+
+cudaError_t gemm_tc_max_clusters(int block_t, int nsplit, int *out) {
+  const size_t smem = gt_smem(block_t, 1);
+  cudaError_t e = gt_configure();
+  if (e != cudaSuccess) return e;
+  if (nsplit > 8) {
+    e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return e;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(1, 1, nsplit);
+  cfg.blockDim = dim3(GT_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = nsplit;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaOccupancyMaxActiveClusters(out, gemm_tc_kernel, &cfg);
+}
+
 cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream) {
   const int T = A.block_t;
-  if (T < 16 || T > 256 || (T & 15) || (A.K % GT_BK) || A.nsplit < 1 || A.nsplit > A.K / GT_BK) return cudaErrorInvalidValue;
-  if (!A.out_fp32 && A.nsplit != 1) return cudaErrorInvalidValue;
-  const size_t smem = gt_smem(T);
-  static size_t configured = 0;
-  if (smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    configured = smem;
-  }
-  dim3 grid((A.N + GT_BN - 1) / GT_BN, (A.M + T - 1) / T, A.nsplit);
-  gemm_tc_kernel<<<grid, GT_THREADS, smem, stream>>>(A, gt_stages(T));
-  return cudaGetLastError();
+  if (T < 16 || T > 256 || (T & 15) || (A.K % GT_BK) || A.nsplit < 1 || A.nsplit > A.K / GT_BK || A.nsplit > 8 ||
+      A.wtiles < 1 || A.wtiles > 2)
+    return cudaErrorInvalidValue;
+  const size_t smem = gt_smem(T, A.wtiles);
+  cudaError_t ec = gt_configure();
+  if (ec != cudaSuccess) return ec;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((A.N + GT_BN * A.wtiles - 1) / (GT_BN * A.wtiles), (A.M + T - 1) / T, A.nsplit);
+  cfg.blockDim = dim3(GT_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = A.nsplit;
+  cfg.attrs = attr;
+  cfg.numAttrs = A.nsplit > 1 ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel, A, gt_stages(T, A.wtiles));
 }
 
 // ---- plain mma.sync GEMM ----------------------------------------------------------------------------------------------
@@ -153,14 +267,12 @@ cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream) {
 // straight from global memory (both operands are K-major, so fragments are plain 32-bit loads).
 __global__ void __launch_bounds__(128) gemm_simple_kernel(const GemmArgs A) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, t4 = lane & 3, r8 = lane >> 2;
-  const int m0 = blockIdx.y * 64 + warp * 16, n0 = blockIdx.x * 64, split = blockIdx.z;
-  const int k_lo = static_cast<int>(static_cast<long long>(split) * (A.K / 16) / A.nsplit) * 16;
-  const int k_hi = static_cast<int>(static_cast<long long>(split + 1) * (A.K / 16) / A.nsplit) * 16;
+  const int m0 = blockIdx.y * 64 + warp * 16, n0 = blockIdx.x * 64;
   float acc[8][4];
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
   const int ra = m0 + r8, rb = m0 + r8 + 8;
-  for (int k = k_lo; k < k_hi; k += 16) {
+  for (int k = 0; k < A.K; k += 16) {
     uint32_t a[4];
     const __nv_bfloat16 *pa = A.x + static_cast<size_t>(ra) * A.K + k + 2 * t4;
     const __nv_bfloat16 *pb = A.x + static_cast<size_t>(rb) * A.K + k + 2 * t4;
@@ -180,25 +292,34 @@ __global__ void __launch_bounds__(128) gemm_simple_kernel(const GemmArgs A) {
       mma_16816(acc[nt], a, b0, b1);
     }
   }
+  // each thread holds column pairs (n, n+1) with n even: (gate, up) of one SwiGLU output
 #pragma unroll
   for (int nt = 0; nt < 8; ++nt)
 #pragma unroll
-    for (int h = 0; h < 2; ++h)
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int m = m0 + r8 + h * 8, n = n0 + nt * 8 + 2 * t4 + e;
-        if (m < A.M && n < A.N) {
-          const float v = acc[nt][h * 2 + e];
-          if (A.out_fp32) reinterpret_cast<float *>(A.out)[split * A.split_stride + static_cast<size_t>(m) * A.ldo + n] = v;
-          else reinterpret_cast<__nv_bfloat16 *>(A.out)[static_cast<size_t>(m) * A.ldo + n] = __float2bfloat16(v);
-        }
+    for (int h = 0; h < 2; ++h) {
+      const int m = m0 + r8 + h * 8, n = n0 + nt * 8 + 2 * t4;
+      if (m >= A.M) continue;
+      const float v0 = acc[nt][h * 2], v1 = acc[nt][h * 2 + 1];
+      if (A.epi == EPI_SWIGLU_BF16) {
+        if (n + 1 < A.N)
+          reinterpret_cast<__nv_bfloat16 *>(A.out)[static_cast<size_t>(m) * A.ldo + (n >> 1)] =
+              __float2bfloat16(v0 / (1.f + __expf(-v0)) * v1);
+        continue;
       }
+      for (int e = 0; e < 2; ++e) {
+        if (n + e >= A.N) continue;
+        const float v = e ? v1 : v0;
+        const size_t o = static_cast<size_t>(m) * A.ldo + n + e;
+        if (A.epi == EPI_STORE_BF16) reinterpret_cast<__nv_bfloat16 *>(A.out)[o] = __float2bfloat16(v);
+        else if (A.epi == EPI_ADD_F32) reinterpret_cast<float *>(A.out)[o] += v;
+        else reinterpret_cast<float *>(A.out)[o] = v;
+      }
+    }
 }
 
 cudaError_t launch_gemm_simple(const GemmArgs &A, cudaStream_t stream) {
-  if ((A.K % 16) || A.nsplit < 1 || A.nsplit > A.K / 16) return cudaErrorInvalidValue;
-  if (!A.out_fp32 && A.nsplit != 1) return cudaErrorInvalidValue;
-  dim3 grid((A.N + 63) / 64, (A.M + 63) / 64, A.nsplit);
+  if (A.K % 16) return cudaErrorInvalidValue;
+  dim3 grid((A.N + 63) / 64, (A.M + 63) / 64, 1);
   gemm_simple_kernel<<<grid, 128, 0, stream>>>(A);
   return cudaGetLastError();
 }

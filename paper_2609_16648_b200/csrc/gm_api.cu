@@ -2,6 +2,7 @@
 // accept phases.  Host code only; every step of the path runs in the kernels of this directory.
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <new>
@@ -44,15 +45,15 @@ struct gm_ctx {
   std::map<std::tuple<const void *, long long>, CUtensorMap> kv_maps;      // (pool, rows)
 
   // workspaces (device)
-  float *x = nullptr, *part = nullptr, *g = nullptr, *part_o = nullptr, *part_ml = nullptr;
-  __nv_bfloat16 *xn = nullptr, *zin = nullptr, *qbuf = nullptr, *attn_out = nullptr, *act = nullptr, *gn = nullptr;
+  float *x = nullptr, *g = nullptr, *part_o = nullptr, *part_ml = nullptr;
+  __nv_bfloat16 *xn = nullptr, *zin = nullptr, *qkv = nullptr, *qbuf = nullptr, *attn_out = nullptr, *act = nullptr, *gn = nullptr;
+  int max_clusters[17][9];            // resident clusters of the GEMM kernel by (block_t / 16, cluster size); -1 = not asked yet
   __nv_bfloat16 *ws_draft_logits = nullptr, *ws_target_logits = nullptr, *ws_target_hidden = nullptr;
   int32_t *ws_draft_tok = nullptr, *ws_accept_len = nullptr, *ws_next_token = nullptr;
   uint32_t *ws_u24 = nullptr;
   int32_t *qn = nullptr, *qbase = nullptr, *page_start = nullptr;
   float2 *rope = nullptr;
   uint32_t *status = nullptr;
-  size_t part_elems = 0;
   std::vector<void *> allocs;
 
   // profiling
@@ -104,7 +105,11 @@ struct Prof {
   do {                                      \
     cudaError_t e__;                        \
     { Prof p__(ctx, cls); e__ = (call); }   \
-    if (e__ != cudaSuccess) { (ctx)->last_cuda = e__; return GM_ERR_CUDA; } \
+    if (e__ != cudaSuccess) {               \
+      (ctx)->last_cuda = e__;               \
+      if (std::getenv("GM_DEBUG")) std::fprintf(stderr, "[gm] %s failed: %s\n", #call, cudaGetErrorString(e__)); \
+      return GM_ERR_CUDA;                   \
+    }                                       \
   } while (0)
 
 // 2-D bf16 tensor map: inner extent `cols` (contiguous), outer extent `rows`, box 64 x box_rows, 128-byte swizzle.
@@ -147,38 +152,45 @@ int kv_map(gm_ctx *c, const void *pool, int layers, int num_pages, CUtensorMap *
 
 int round16(int v) { return (v + 15) & ~15; }
 
-// Split-K factor that fills the SMs when a projection has few output tiles.
-int pick_split(const gm_ctx *c, int M, int N, int K, int T) {
+// K slices (= cluster size) for a projection with few output tiles: the largest count whose clusters are all
+// resident at once (GPC packing decides), so the slices of a tile run concurrently and the SMs are filled.
+int pick_split(gm_ctx *c, int M, int N, int K, int T) {
   const int tiles = ((N + 127) / 128) * ((M + T - 1) / T);
   if (tiles * 3 >= c->sm_count * 2) return 1;
-  int ns = c->sm_count / tiles;
   const int KB = K / 64;
-  if (ns > KB) ns = KB;
-  if (ns > 16) ns = 16;
-  return ns < 1 ? 1 : ns;
+  int best = 1;
+  for (int ns = 2; ns <= 8 && ns <= KB; ++ns) {
+    int &cap = c->max_clusters[T / 16][ns];
+    if (cap < 0) {
+      int v = 0;
+      cudaError_t e = gemm_tc_max_clusters(T, ns, &v);
+      if (e != cudaSuccess) { v = 0; (void)cudaGetLastError(); }
+      if (std::getenv("GM_DEBUG")) std::fprintf(stderr, "[gm] resident clusters T=%d size=%d: %d (%s)\n", T, ns, v, cudaGetErrorString(e));
+      cap = v;
+    }
+    if (cap >= tiles) best = ns;
+  }
+  return best;
 }
 
-// out = x[M, K] w[N, K]^T.  fp32 partials into c->part (returns the split count), or bf16 to `out_bf16`
-// with row stride ldo.
+// out = epilogue(x[M, K] w[N, K]^T) on the tcgen05 kernel (or the plain one under GM_FLAG_SIMPLE_GEMM).
 int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *wmap, const __nv_bfloat16 *w, int M,
-             int N, int K, void *out, bool out_fp32, int *nsplit_out, size_t *split_stride_out) {
+             int N, int K, void *out, int epi, size_t ldo) {
   GemmArgs A;
   std::memset(&A, 0, sizeof(A));
   A.x = x; A.w = w; A.M = M; A.N = N; A.K = K; A.status = c->status;
-  A.out = out; A.out_fp32 = out_fp32 ? 1 : 0;
-  const bool simple = (c->cfg.flags & GM_FLAG_SIMPLE_GEMM) != 0 || (K % 64) != 0;
+  A.out = out; A.epi = epi; A.ldo = ldo;
   const int T = M >= 256 ? 256 : round16(M);
   A.block_t = T;
-  A.nsplit = out_fp32 ? pick_split(c, M, N, K, T) : 1;
-  A.split_stride = static_cast<size_t>(M) * N;
-  A.ldo = N;
-  if (out_fp32 && A.split_stride * A.nsplit > c->part_elems && out == c->part) return GM_ERR_INVALID_ARG;
-  if (nsplit_out) *nsplit_out = A.nsplit;
-  if (split_stride_out) *split_stride_out = A.split_stride;
-  if (simple) {
+  A.nsplit = 1;
+  A.wtiles = 1;
+  if ((c->cfg.flags & GM_FLAG_SIMPLE_GEMM) != 0 || (K % 64) != 0) {
     GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_simple(A, c->stream));
     return GM_OK;
   }
+  A.nsplit = pick_split(c, M, N, K, T);
+  // wide projections: two sub-tiles per CTA halve the activation re-reads from L2
+  if (A.nsplit == 1 && ((N + 127) / 128) * ((M + T - 1) / T) >= c->sm_count) A.wtiles = 2;
   A.w_map = *wmap;
   int rc = x_map(c, x, x_rows, K, T, &A.x_map);
   if (rc != GM_OK) return rc;
@@ -195,13 +207,13 @@ int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const 
               __nv_bfloat16 *pool, int layer, int num_pages, const int32_t *page_table,
               const __nv_bfloat16 *next_norm, __nv_bfloat16 *hidden_out) {
   const gm_config &cf = c->cfg;
-  int ns; size_t ss; int rc;
-  // QKV projection -> rotary + KV append + Q rearrangement
+  int rc;
+  // QKV projection (bf16) -> rotary + KV append + Q rearrangement
   rc = run_gemm(c, c->xn, c->Mmax, &lm.wqkv, static_cast<const __nv_bfloat16 *>(lw.wqkv), ph.M, c->n_qkv, c->d,
-                c->part, true, &ns, &ss);
+                c->qkv, EPI_STORE_BF16, c->n_qkv);
   if (rc) return rc;
   RopeAppendArgs R;
-  R.qkv = c->part; R.nsplit = ns; R.split_stride = ss;
+  R.qkv = c->qkv;
   R.batch = ph.B; R.QT = ph.QT; R.n_q = cf.n_q_heads; R.n_kv = cf.n_kv_heads; R.hd = cf.head_dim; R.layer = layer;
   R.num_pages = num_pages; R.max_pages_per_seq = cf.max_pages_per_seq; R.qrows = ph.qrows;
   R.qn = c->qn; R.qbase = c->qbase; R.page_table = page_table; R.rope = c->rope; R.qbuf = c->qbuf; R.pool = pool;
@@ -220,24 +232,24 @@ int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const 
   Cb.n_kv = cf.n_kv_heads; Cb.group = c->group; Cb.hd = cf.head_dim; Cb.qrows = ph.qrows; Cb.QT = ph.QT;
   Cb.n_ctas = c->sm_count; Cb.out = c->attn_out;
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_attention_combine(Cb, c->stream));
-  // output projection + residual + post-attention norm
+  // output projection added into the residual stream, then the post-attention norm
   rc = run_gemm(c, c->attn_out, c->Mmax, &lm.wo, static_cast<const __nv_bfloat16 *>(lw.wo), ph.M, c->d, c->q_dim,
-                c->part, true, &ns, &ss);
+                c->x, EPI_ADD_F32, c->d);
   if (rc) return rc;
   GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-            launch_reduce_residual_norm(c->part, ns, ss, c->x, 1, static_cast<const __nv_bfloat16 *>(lw.ln2), c->xn,
-                                        nullptr, ph.M, c->d, cf.rms_eps, c->stream));
-  // SwiGLU feed-forward
+            launch_rmsnorm(c->x, static_cast<const __nv_bfloat16 *>(lw.ln2), c->xn, nullptr, ph.M, c->d, cf.rms_eps,
+                           c->stream));
+  // SwiGLU feed-forward: gate/up projection with the activation in its epilogue, down projection into the residual
   rc = run_gemm(c, c->xn, c->Mmax, &lm.wgu, static_cast<const __nv_bfloat16 *>(lw.w_gate_up), ph.M, 2 * c->F, c->d,
-                c->part, true, &ns, &ss);
+                c->act, EPI_SWIGLU_BF16, c->F);
   if (rc) return rc;
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_swiglu(c->part, ns, ss, c->act, ph.M, c->F, c->stream));
   rc = run_gemm(c, c->act, c->Mmax, &lm.wdown, static_cast<const __nv_bfloat16 *>(lw.w_down), ph.M, c->d, c->F,
-                c->part, true, &ns, &ss);
+                c->x, EPI_ADD_F32, c->d);
   if (rc) return rc;
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-            launch_reduce_residual_norm(c->part, ns, ss, c->x, 1, next_norm, next_norm ? c->xn : nullptr, hidden_out,
-                                        ph.M, c->d, cf.rms_eps, c->stream));
+  if (next_norm || hidden_out)
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+              launch_rmsnorm(c->x, next_norm, next_norm ? c->xn : nullptr, hidden_out, ph.M, c->d, cf.rms_eps,
+                             c->stream));
   return GM_OK;
 }
 
@@ -356,22 +368,15 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
   // workspaces
   const size_t M = c->Mmax, B = cfg->max_batch;
   const int qrows = round16((cfg->max_k + 1) * group);
-  size_t pe = 0;
-  auto upd = [&](int N, int K) {          // worst case of nsplit * M * N over every row count a call may use
-    for (int m = 1; m <= static_cast<int>(M); ++m) {
-      const int T = m >= 256 ? 256 : round16(m);
-      pe = std::max(pe, static_cast<size_t>(pick_split(c, m, N, K, T)) * m * N);
-    }
-  };
-  upd(c->n_qkv, c->d); upd(c->d, c->q_dim); upd(2 * c->F, c->d); upd(c->d, c->F); upd(c->d, 2 * c->d);
-  c->part_elems = pe;
+  for (auto &row : c->max_clusters)
+    for (int &v : row) v = -1;
   int rc = GM_OK;
   const size_t slots = static_cast<size_t>(c->sm_count) + B;
 #define A_(call) if ((rc = (call)) != GM_OK) return fail(rc)
   A_(dev_alloc(c, &c->x, M * c->d));
   A_(dev_alloc(c, &c->xn, M * c->d));
   A_(dev_alloc(c, &c->zin, M * 2 * c->d));
-  A_(dev_alloc(c, &c->part, pe));
+  A_(dev_alloc(c, &c->qkv, M * c->n_qkv));
   A_(dev_alloc(c, &c->qbuf, B * cfg->n_kv_heads * qrows * cfg->head_dim));
   A_(dev_alloc(c, &c->attn_out, M * c->q_dim));
   A_(dev_alloc(c, &c->act, M * c->F));
@@ -445,13 +450,12 @@ int gm_draft(gm_ctx *c, const gm_state *st, int k, float temperature, const uint
     H.pending_hidden = static_cast<const __nv_bfloat16 *>(st->pending_hidden); H.draft_tok = draft_tok; H.g_prev = c->g;
     H.zin = c->zin; H.status = c->status;
     GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_head_input(H, c->stream));
-    int ns; size_t ss;
     rc = run_gemm(c, c->zin, c->Mmax, &c->head_proj_map, static_cast<const __nv_bfloat16 *>(c->w.head_proj), ph.M, c->d,
-                  2 * c->d, c->part, true, &ns, &ss);
+                  2 * c->d, c->x, EPI_STORE_F32, c->d);
     if (rc) return rc;
     GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-              launch_reduce_residual_norm(c->part, ns, ss, c->x, 0, static_cast<const __nv_bfloat16 *>(c->w.head_layer.ln1),
-                                          c->xn, nullptr, ph.M, c->d, cf.rms_eps, c->stream));
+              launch_rmsnorm(c->x, static_cast<const __nv_bfloat16 *>(c->w.head_layer.ln1), c->xn, nullptr, ph.M, c->d,
+                             cf.rms_eps, c->stream));
     rc = run_layer(c, c->w.head_layer, c->head_maps, ph, kvm, static_cast<__nv_bfloat16 *>(st->head_kv_pool), 0,
                    cf.head_num_pages, st->head_page_table, nullptr, nullptr);
     if (rc) return rc;
@@ -459,20 +463,9 @@ int gm_draft(gm_ctx *c, const gm_state *st, int k, float temperature, const uint
               launch_head_out(c->x, c->qn, ph.B, ph.QT, c->d, static_cast<const __nv_bfloat16 *>(c->w.head_final_norm),
                               cf.rms_eps, c->g, c->gn, c->stream));
     // shared LM head -> row j-1 of every sequence's draft logits (row stride k*V)
-    {
-      GemmArgs A;
-      std::memset(&A, 0, sizeof(A));
-      A.x = c->gn; A.w = static_cast<const __nv_bfloat16 *>(c->w.lm_head); A.M = ph.B; A.N = c->V; A.K = c->d;
-      A.out = dl + static_cast<size_t>(j - 1) * c->V; A.out_fp32 = 0; A.nsplit = 1; A.ldo = static_cast<size_t>(k) * c->V;
-      A.block_t = ph.B >= 256 ? 256 : round16(ph.B); A.status = c->status;
-      if (cf.flags & GM_FLAG_SIMPLE_GEMM) {
-        GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_simple(A, c->stream));
-      } else {
-        A.w_map = c->lm_head_map;
-        if ((rc = x_map(c, c->gn, cf.max_batch, c->d, A.block_t, &A.x_map)) != GM_OK) return rc;
-        GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(A, c->stream));
-      }
-    }
+    rc = run_gemm(c, c->gn, cf.max_batch, &c->lm_head_map, static_cast<const __nv_bfloat16 *>(c->w.lm_head), ph.B, c->V,
+                  c->d, dl + static_cast<size_t>(j - 1) * c->V, EPI_STORE_BF16, static_cast<size_t>(k) * c->V);
+    if (rc) return rc;
     // d_j ~ softmax(logits / T): the sampler with depth 0
     S.K = 0; S.target_logits = dl + static_cast<size_t>(j - 1) * c->V; S.tgt_bstride = static_cast<size_t>(k) * c->V;
     S.draft_logits = nullptr; S.u24 = u24_draft ? u24_draft + (j - 1) : nullptr; S.u_stride = k;
@@ -507,19 +500,8 @@ int gm_verify(gm_ctx *c, const gm_state *st, int k, const int32_t *draft_tok, vo
                    st->page_table, next_norm, last ? static_cast<__nv_bfloat16 *>(target_hidden) : nullptr);
     if (rc) return rc;
   }
-  GemmArgs A;
-  std::memset(&A, 0, sizeof(A));
-  A.x = c->xn; A.w = static_cast<const __nv_bfloat16 *>(c->w.lm_head); A.M = ph.M; A.N = c->V; A.K = c->d;
-  A.out = target_logits; A.out_fp32 = 0; A.nsplit = 1; A.ldo = c->V;
-  A.block_t = ph.M >= 256 ? 256 : round16(ph.M); A.status = c->status;
-  if (cf.flags & GM_FLAG_SIMPLE_GEMM) {
-    GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_simple(A, c->stream));
-  } else {
-    A.w_map = c->lm_head_map;
-    if ((rc = x_map(c, c->xn, c->Mmax, c->d, A.block_t, &A.x_map)) != GM_OK) return rc;
-    GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(A, c->stream));
-  }
-  return GM_OK;
+  return run_gemm(c, c->xn, c->Mmax, &c->lm_head_map, static_cast<const __nv_bfloat16 *>(c->w.lm_head), ph.M, c->V, c->d,
+                  target_logits, EPI_STORE_BF16, c->V);
 }
 
 int gm_accept(gm_ctx *c, gm_state *st, int batch, int k, float temperature, const void *target_logits,
@@ -611,27 +593,20 @@ int gm_spec_step_host(gm_ctx *c, gm_state *st, int k, float temperature, uint64_
 int gm_gemm(gm_ctx *c, const void *x, const void *w, void *out, int M, int N, int K, int out_fp32) {
   if (!c || !x || !w || !out || M < 1 || N < 1 || K < 1) return GM_ERR_INVALID_ARG;
   if ((K % 64) || (N % 8)) return GM_ERR_UNSUPPORTED;
-  GemmArgs A;
-  std::memset(&A, 0, sizeof(A));
-  A.x = static_cast<const __nv_bfloat16 *>(x); A.w = static_cast<const __nv_bfloat16 *>(w); A.M = M; A.N = N; A.K = K;
-  A.out = out; A.out_fp32 = out_fp32 ? 1 : 0; A.nsplit = 1; A.ldo = N; A.split_stride = static_cast<size_t>(M) * N;
-  A.block_t = M >= 256 ? 256 : round16(M); A.status = c->status;
-  if (c->cfg.flags & GM_FLAG_SIMPLE_GEMM) {
-    GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_simple(A, c->stream));
-    return GM_OK;
+  CUtensorMap wm;
+  std::memset(&wm, 0, sizeof(wm));
+  if (!(c->cfg.flags & GM_FLAG_SIMPLE_GEMM)) {
+    auto key = std::make_tuple(w, N, K);
+    auto it = c->w_maps.find(key);
+    if (it == c->w_maps.end()) {
+      CUtensorMap m;
+      if (make_map(c, &m, w, N, K, 128) != GM_OK) return GM_ERR_CUDA;
+      it = c->w_maps.emplace(key, m).first;
+    }
+    wm = it->second;
   }
-  auto key = std::make_tuple(w, N, K);
-  auto it = c->w_maps.find(key);
-  if (it == c->w_maps.end()) {
-    CUtensorMap m;
-    if (make_map(c, &m, w, N, K, 128) != GM_OK) return GM_ERR_CUDA;
-    it = c->w_maps.emplace(key, m).first;
-  }
-  A.w_map = it->second;
-  int rc = x_map(c, x, M, K, A.block_t, &A.x_map);
-  if (rc) return rc;
-  GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(A, c->stream));
-  return GM_OK;
+  return run_gemm(c, static_cast<const __nv_bfloat16 *>(x), M, &wm, static_cast<const __nv_bfloat16 *>(w), M, N, K, out,
+                  out_fp32 ? EPI_STORE_F32 : EPI_STORE_BF16, N);
 }
 
 int gm_profile(gm_ctx *c, int class_mask) {

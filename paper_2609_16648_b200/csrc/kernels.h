@@ -69,14 +69,13 @@ struct HeadInputArgs {
   uint32_t *status;
 };
 cudaError_t launch_head_input(const HeadInputArgs &A, cudaStream_t stream);
-// x_out[m] = (add_residual ? x[m] : 0) + sum_s partial[s][m];  xn[m] = RMSNorm(x_out[m]; w);  optional
-// bf16 copy of x_out (the hidden state handed to the caller).
-cudaError_t launch_reduce_residual_norm(const float *partial, int nsplit, size_t split_stride, float *x,
-                                        int add_residual, const __nv_bfloat16 *w, __nv_bfloat16 *xn,
-                                        __nv_bfloat16 *hidden_out, int M, int d, float eps, cudaStream_t stream);
+// xn[m] = RMSNorm(x[m]; w) (bf16) from the fp32 residual stream; optional bf16 copy of x (the hidden state
+// handed to the caller).
+cudaError_t launch_rmsnorm(const float *x, const __nv_bfloat16 *w, __nv_bfloat16 *xn, __nv_bfloat16 *hidden_out,
+                           int M, int d, float eps, cudaStream_t stream);
 // Rotary embedding of q and k, KV append into the pages, Q rearranged per (sequence, kv head).
 struct RopeAppendArgs {
-  const float *qkv; int nsplit; size_t split_stride;   // fp32 [nsplit][M][(n_q + 2 n_kv) hd]
+  const __nv_bfloat16 *qkv;                             // bf16 [M][(n_q + 2 n_kv) hd]
   int batch, QT, n_q, n_kv, hd, layer, num_pages, max_pages_per_seq, qrows;
   const int32_t *qn, *qbase, *page_table;
   const float2 *rope;                                   // [max_pos][hd/2] (cos, sin)
@@ -85,9 +84,6 @@ struct RopeAppendArgs {
   uint32_t *status;
 };
 cudaError_t launch_rope_append(const RopeAppendArgs &A, cudaStream_t stream);
-// act[m][i] = silu(gate_i) * up_i from interleaved fp32 partials [nsplit][M][2F].
-cudaError_t launch_swiglu(const float *gu, int nsplit, size_t split_stride, __nv_bfloat16 *act, int M, int F,
-                          cudaStream_t stream);
 // g[b] = x[b*QT + qn[b]-1] (fp32), gn[b] = RMSNorm(g[b]; w) (bf16): the head's last valid row per sequence.
 cudaError_t launch_head_out(const float *x, const int32_t *qn, int batch, int QT, int d, const __nv_bfloat16 *w,
                             float eps, float *g, __nv_bfloat16 *gn, cudaStream_t stream);
@@ -115,18 +111,27 @@ int attention_max_ctas(int n_kv, int hd);   // CTAs the attention kernel wants f
 size_t attention_smem_bytes(int n_kv, int hd);
 
 // ---- GEMM --------------------------------------------------------------------------------------------------
-// out = x[M, K] * w[N, K]^T with fp32 accumulation.  nsplit > 1 (or out_fp32): fp32 partials
-// [nsplit][M][N]; otherwise bf16 [M][N].
+// out = epilogue(x[M, K] * w[N, K]^T) with fp32 accumulation.
+enum GemmEpilogue {
+  EPI_STORE_BF16 = 0,    // out bf16 [M, ldo]
+  EPI_STORE_F32 = 1,     // out fp32 [M, ldo]
+  EPI_ADD_F32 = 2,       // out fp32 [M, ldo] += result   (residual stream update)
+  EPI_SWIGLU_BF16 = 3,   // rows of w interleaved (gate_i, up_i): out bf16 [M, ldo], column i = silu(gate_i) * up_i
+};
 struct GemmArgs {
   CUtensorMap w_map, x_map;             // tcgen05 path only
   const __nv_bfloat16 *x, *w;
-  void *out; int out_fp32;
-  int M, N, K, nsplit, block_t;         // block_t: tokens per CTA (multiple of 16, <= 256)
-  size_t split_stride;                  // elements between partials
-  size_t ldo;                           // output row stride in elements (>= N)
+  void *out; int epi;
+  int M, N, K;
+  int nsplit;                           // K slices = cluster size along z (1..8); the simple kernel ignores it
+  int block_t;                          // tokens per CTA (multiple of 16, <= 256)
+  int wtiles;                           // 128-feature sub-tiles per CTA sharing one activation tile (1 or 2)
+  size_t ldo;                           // output row stride in elements
   uint32_t *status;
 };
 cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream);
 cudaError_t launch_gemm_simple(const GemmArgs &A, cudaStream_t stream);
+// How many clusters of `nsplit` CTAs of the tcgen05 kernel can be resident at once (GPC packing).
+cudaError_t gemm_tc_max_clusters(int block_t, int nsplit, int *out);
 
 }  // namespace gm
