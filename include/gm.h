@@ -181,6 +181,21 @@ int gm_spec_step_host(gm_ctx *ctx, gm_state *st, int k, float temperature, uint6
 int gm_gemm(gm_ctx *ctx, const void *x, const void *w, void *out, int M, int N, int K,
             int out_fp32);
 
+/* Multi-query paged decode attention as a stand-alone call: the kernel both phases run once per layer
+ * (Sec. 2.2: the target verifies all K candidates in a single forward pass; App. B.1: the head keeps a KV
+ * cache of its own).  For every sequence b, q_count[b] queries at positions q_base[b] .. q_base[b] +
+ * q_count[b] - 1 attend the cached positions <= their own; the caller has already written the new
+ * keys/values into the pages.  Grouped-query: query head h reads KV head h / (n_q / n_kv).
+ *   q        bf16 [B][n_kv][q_rows][head_dim], q_rows = 16 * ceil(q_stride * group / 16); row j*group + g is
+ *            query j of head kv*group + g, rotary embedding already applied; unused rows must be finite
+ *   kv_pool  bf16 [pool_layers][2][num_pages][n_kv][16][head_dim]; `layer` selects the slab
+ *   page_table [B, max_pages_per_seq];  q_count, q_base [B];  q_stride <= max_k + 1 (rows per sequence in out)
+ *   out      bf16 [B * q_stride][n_q * head_dim]; rows j >= q_count[b] are left untouched
+ * A sequence whose queries do not fit its page-table row sets GM_ERR_KV_CAPACITY and is skipped.          */
+int gm_attention(gm_ctx *ctx, const void *q, const void *kv_pool, int pool_layers, int num_pages, int layer,
+                 const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch,
+                 int q_stride, void *out);
+
 /* Kernel-class timing.  gm_profile(ctx, mask) makes later calls bracket every launch of the
  * selected classes with CUDA events on the context's stream; gm_profile_read waits for the
  * stream and returns the accumulated device time and launch count of one class since the

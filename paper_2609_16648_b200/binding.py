@@ -22,7 +22,7 @@ GM_FLAG_SIMPLE_GEMM = 1
 GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER = 0, 1, 2, 3
 
 EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw",
-           "gm_spec_step_host", "gm_gemm", "gm_profile", "gm_profile_read", "gm_launch_count",
+           "gm_spec_step_host", "gm_gemm", "gm_attention", "gm_profile", "gm_profile_read", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
 
 
@@ -73,6 +73,7 @@ def lib() -> C.CDLL:
     L.gm_spec_step_host.argtypes = [vp, C.POINTER(gm_state), i32, f32, u64, u64, vp, vp, vp, vp, vp]
     L.gm_draw.argtypes = [vp, vp, i32, f32, vp, vp, vp]
     L.gm_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
+    L.gm_attention.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, i32, i32, vp]
     L.gm_profile.argtypes = [vp, i32]
     L.gm_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     L.gm_launch_count.argtypes = [vp]
@@ -271,6 +272,12 @@ def gm_draw(ctx: Context, logits, rows: int, temperature: float, u24, out_tok, d
 
 def gm_gemm(ctx: Context, x, w, out, M: int, N: int, K: int, out_fp32: bool):
     _check(lib().gm_gemm(ctx.handle, _p(x), _p(w), _p(out), M, N, K, 1 if out_fp32 else 0), "gm_gemm")
+
+
+def gm_attention(ctx: Context, q, kv_pool, layer: int, page_table, q_count, q_base, batch: int, q_stride: int, out):
+    """kv_pool: bf16 [pool_layers, 2, num_pages, n_kv, 16, head_dim]."""
+    _check(lib().gm_attention(ctx.handle, _p(q), _p(kv_pool), kv_pool.shape[0], kv_pool.shape[2], layer,
+                              _p(page_table), _p(q_count), _p(q_base), batch, q_stride, _p(out)), "gm_attention")
 
 
 def gm_profile(ctx: Context, class_mask: int):

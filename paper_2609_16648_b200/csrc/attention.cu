@@ -358,4 +358,26 @@ cudaError_t launch_attention_combine(const AttnCombineArgs &A, cudaStream_t stre
   return cudaGetLastError();
 }
 
+// ---- page prefix for a caller-given query layout (stand-alone attention calls) -------------------------------------------
+// page_start[b] = pages attended by the sequences before b; a sequence whose queries do not fit its page-table row
+// is reported and given no pages (its output rows are then left untouched).
+__global__ void page_prefix_kernel(const int32_t *qn, const int32_t *qbase, int batch, int max_pages_per_seq,
+                                   int q_stride, int32_t *page_start, uint32_t *status) {
+  if (threadIdx.x != 0) return;
+  int acc = 0;
+  for (int b = 0; b < batch; ++b) {
+    page_start[b] = acc;
+    const int n = qn[b], base = qbase[b];
+    const bool ok = n >= 1 && n <= q_stride && base >= 0 && base + n <= max_pages_per_seq * 16;
+    if (!ok && n != 0) set_status(status, ST_KV_CAPACITY);
+    acc += ok ? (base + n + 15) >> 4 : 0;
+  }
+  page_start[batch] = acc;
+}
+cudaError_t launch_page_prefix(const int32_t *qn, const int32_t *qbase, int batch, int max_pages_per_seq, int q_stride,
+                               int32_t *page_start, uint32_t *status, cudaStream_t stream) {
+  page_prefix_kernel<<<1, 32, 0, stream>>>(qn, qbase, batch, max_pages_per_seq, q_stride, page_start, status);
+  return cudaGetLastError();
+}
+
 }  // namespace gm

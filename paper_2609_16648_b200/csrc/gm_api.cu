@@ -609,6 +609,36 @@ int gm_gemm(gm_ctx *c, const void *x, const void *w, void *out, int M, int N, in
                   out_fp32 ? EPI_STORE_F32 : EPI_STORE_BF16, N);
 }
 
+int gm_attention(gm_ctx *c, const void *q, const void *kv_pool, int pool_layers, int num_pages, int layer,
+                 const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch, int q_stride,
+                 void *out) {
+  if (!c || !q || !kv_pool || !page_table || !q_count || !q_base || !out) return GM_ERR_INVALID_ARG;
+  if (batch < 1 || batch > c->cfg.max_batch || q_stride < 1 || pool_layers < 1 || layer < 0 || layer >= pool_layers ||
+      num_pages < 1)
+    return GM_ERR_INVALID_ARG;
+  if (q_stride > c->cfg.max_k + 1) return GM_ERR_UNSUPPORTED;
+  const gm_config &cf = c->cfg;
+  CUtensorMap kvm;
+  int rc = kv_map(c, kv_pool, pool_layers, num_pages, &kvm);
+  if (rc) return rc;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+            launch_page_prefix(q_count, q_base, batch, cf.max_pages_per_seq, q_stride, c->page_start, c->status, c->stream));
+  const int qrows = round16(q_stride * c->group);
+  AttnArgs T;
+  T.kv_map = kvm; T.qbuf = static_cast<const __nv_bfloat16 *>(q); T.qn = q_count; T.qbase = q_base;
+  T.page_start = c->page_start; T.page_table = page_table; T.batch = batch; T.n_kv = cf.n_kv_heads; T.group = c->group;
+  T.hd = cf.head_dim; T.qrows = qrows; T.layer = layer; T.num_pages = num_pages; T.max_pages_per_seq = cf.max_pages_per_seq;
+  T.n_ctas = c->sm_count; T.scale_log2e = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(cf.head_dim)));
+  T.part_o = c->part_o; T.part_ml = c->part_ml; T.status = c->status;
+  GM_LAUNCH(c, GM_KC_ATTENTION, launch_attention(T, c->stream));
+  AttnCombineArgs Cb;
+  Cb.part_o = c->part_o; Cb.part_ml = c->part_ml; Cb.qn = q_count; Cb.page_start = c->page_start; Cb.batch = batch;
+  Cb.n_kv = cf.n_kv_heads; Cb.group = c->group; Cb.hd = cf.head_dim; Cb.qrows = qrows; Cb.QT = q_stride;
+  Cb.n_ctas = c->sm_count; Cb.out = static_cast<__nv_bfloat16 *>(out);
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_attention_combine(Cb, c->stream));
+  return GM_OK;
+}
+
 int gm_profile(gm_ctx *c, int class_mask) {
   if (!c) return GM_ERR_INVALID_ARG;
   GM_CUDA(c, cudaStreamSynchronize(c->stream));
