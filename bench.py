@@ -274,6 +274,19 @@ def run_reference(args):
 
 # ---- product leg ---------------------------------------------------------------------------------------------------------
 
+def reduce_over_ranks(maxima, sums, device, world):
+    """Replicas share nothing on the data path; only the report is reduced: times as the max over ranks,
+    token and launch counts as sums.  Works on any backend (NCCL on GPUs, gloo in the CPU tests)."""
+    import torch
+    mx = torch.tensor(list(maxima), dtype=torch.float64, device=device)
+    sm = torch.tensor(list(sums), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+        dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+    return mx.tolist(), sm.tolist()
+
+
 def run_product(args):
     import torch
     rank = int(os.environ.get("RANK", "0"))
@@ -379,13 +392,8 @@ def run_product(args):
     d2h = int(a_h.numel() + t_h.numel() + d_h.numel()) * 4
 
     # ---- reduce over ranks (max time, summed tokens) ---------------------------------------------------------------------
-    stats = torch.tensor([ms, e2e_s * 1e3], dtype=torch.float64, device=device)
-    toks = torch.tensor([committed, committed_e2e, launches, B], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
-        dist.all_reduce(toks, op=dist.ReduceOp.SUM)
-    ms_max, e2e_ms_max = stats.tolist()
-    committed_all, committed_e2e_all, launches_all, batch_all = toks.tolist()
+    (ms_max, e2e_ms_max), (committed_all, committed_e2e_all, launches_all, batch_all) = reduce_over_ranks(
+        [ms, e2e_s * 1e3], [committed, committed_e2e, launches, B], device, world)
 
     if rank == 0:
         hbm, tflops, which = measured_peaks()
