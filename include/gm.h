@@ -51,6 +51,7 @@ extern "C" {
 #define GM_ERR_DEVICE_TIMEOUT (-5)  /* a bounded device-side wait expired (device-seen)         */
 #define GM_ERR_BAD_PAGE      (-6)   /* a page id outside the pool (device-seen)                 */
 #define GM_ERR_NO_EXTENSION  (-7)   /* not an sm_100 device                                     */
+#define GM_ERR_SCRATCH_LIMIT (-8)   /* request larger than the static scratch of a no-alloc call */
 
 #define GM_MAX_K 7
 #define GM_PAGE  16
@@ -195,6 +196,32 @@ int gm_gemm(gm_ctx *ctx, const void *x, const void *w, void *out, int M, int N, 
 int gm_attention(gm_ctx *ctx, const void *q, const void *kv_pool, int pool_layers, int num_pages, int layer,
                  const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch,
                  int q_stride, void *out);
+
+/* gm_attention for callers that cannot allocate (the paper has no counterpart: this is a packaging
+ * variant of the attention kernel, not a step of the method).  Same computation and argument meaning as
+ * gm_attention, but it takes no context - the model shape is passed directly - and it calls no cudaMalloc,
+ * cudaFree or any other allocating routine: the per-segment partial outputs, the page prefix and a status
+ * word live in ONE static device array of GM_NOALLOC_SCRATCH_BYTES (16 MiB) that every GPU loading the
+ * library holds until the process exits.  It is meant for callers such as a latency-critical serving
+ * thread that must not trigger a device allocation, a plug-in that is given a stream but owns no memory
+ * pool, or a process whose device memory is fully managed by another allocator.
+ *   Limits: batch <= GM_NOALLOC_MAX_BATCH and
+ *   4096 + (SMs + batch) * n_kv * q_rows * (head_dim + 2) * 4 bytes <= GM_NOALLOC_SCRATCH_BYTES
+ *   (e.g. 64 sequences, 8 KV heads, 16 query rows, head_dim 128 on 148 SMs need 14.1 MB); anything larger
+ *   returns GM_ERR_SCRATCH_LIMIT and launches nothing.
+ *   Set-up: the FIRST call on each device resolves the array's device address (cudaGetSymbolAddress) with
+ *   that device current; make that first call before any stream capture begins.
+ *   Sharing: every call uses the same array, which keeps the previous call's contents; the call clears what
+ *   must start at zero itself.  Two calls that overlap on the GPU (different streams, or two host threads)
+ *   race on it - serialise them.  Device-seen conditions are not reported: a sequence that does not fit its
+ *   page-table row is skipped (its output rows stay untouched) and an out-of-range page id reads page 0.
+ *   cuda_stream: a cudaStream_t (NULL = the default stream) of the current device.                        */
+#define GM_NOALLOC_SCRATCH_BYTES (16u << 20)
+#define GM_NOALLOC_MAX_BATCH 256
+int gm_attention_noalloc(int n_q_heads, int n_kv_heads, int head_dim, int max_pages_per_seq, const void *q,
+                         const void *kv_pool, int pool_layers, int num_pages, int layer,
+                         const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch,
+                         int q_stride, void *out, void *cuda_stream);
 
 /* Kernel-class timing.  gm_profile(ctx, mask) makes later calls bracket every launch of the
  * selected classes with CUDA events on the context's stream; gm_profile_read waits for the

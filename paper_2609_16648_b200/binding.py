@@ -16,13 +16,14 @@ LIB_PATH = os.path.join(HERE, "libgm.so")
 
 GM_OK = 0
 GM_ERR_INVALID_ARG, GM_ERR_UNSUPPORTED, GM_ERR_KV_CAPACITY, GM_ERR_CUDA = -1, -2, -3, -4
-GM_ERR_DEVICE_TIMEOUT, GM_ERR_BAD_PAGE, GM_ERR_NO_EXTENSION = -5, -6, -7
+GM_ERR_DEVICE_TIMEOUT, GM_ERR_BAD_PAGE, GM_ERR_NO_EXTENSION, GM_ERR_SCRATCH_LIMIT = -5, -6, -7, -8
+GM_NOALLOC_SCRATCH_BYTES, GM_NOALLOC_MAX_BATCH = 16 << 20, 256
 GM_MAX_K, GM_PAGE = 7, 16
 GM_FLAG_SIMPLE_GEMM = 1
 GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER = 0, 1, 2, 3
 
 EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw",
-           "gm_spec_step_host", "gm_gemm", "gm_attention", "gm_profile", "gm_profile_read", "gm_launch_count",
+           "gm_spec_step_host", "gm_gemm", "gm_attention", "gm_attention_noalloc", "gm_profile", "gm_profile_read", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
 
 
@@ -74,6 +75,7 @@ def lib() -> C.CDLL:
     L.gm_draw.argtypes = [vp, vp, i32, f32, vp, vp, vp]
     L.gm_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
     L.gm_attention.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, i32, i32, vp]
+    L.gm_attention_noalloc.argtypes = [i32, i32, i32, i32, vp, vp, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp]
     L.gm_profile.argtypes = [vp, i32]
     L.gm_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     L.gm_launch_count.argtypes = [vp]
@@ -278,6 +280,17 @@ def gm_attention(ctx: Context, q, kv_pool, layer: int, page_table, q_count, q_ba
     """kv_pool: bf16 [pool_layers, 2, num_pages, n_kv, 16, head_dim]."""
     _check(lib().gm_attention(ctx.handle, _p(q), _p(kv_pool), kv_pool.shape[0], kv_pool.shape[2], layer,
                               _p(page_table), _p(q_count), _p(q_base), batch, q_stride, _p(out)), "gm_attention")
+
+
+def gm_attention_noalloc(n_q_heads: int, n_kv_heads: int, head_dim: int, q, kv_pool, layer: int, page_table, q_count,
+                         q_base, batch: int, q_stride: int, out, stream=None):
+    """gm_attention without a context and without any allocation inside the library: for callers that are
+    handed device buffers and a stream but may not allocate (the scratch is a fixed 16 MiB array inside the
+    library).  Raises GmError(GM_ERR_SCRATCH_LIMIT) when the request does not fit that array."""
+    stream = torch.cuda.current_stream() if stream is None else stream
+    _check(lib().gm_attention_noalloc(n_q_heads, n_kv_heads, head_dim, page_table.shape[1], _p(q), _p(kv_pool),
+                                      kv_pool.shape[0], kv_pool.shape[2], layer, _p(page_table), _p(q_count), _p(q_base),
+                                      batch, q_stride, _p(out), C.c_void_p(stream.cuda_stream)), "gm_attention_noalloc")
 
 
 def gm_profile(ctx: Context, class_mask: int):

@@ -298,6 +298,7 @@ const char *gm_strerror(int code) {
     case GM_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
     case GM_ERR_BAD_PAGE: return "page id or token id outside its range";
     case GM_ERR_NO_EXTENSION: return "no sm_100 device";
+    case GM_ERR_SCRATCH_LIMIT: return "request exceeds the static scratch of the no-alloc entry point (see GM_NOALLOC_SCRATCH_BYTES)";
     default: return "unknown error";
   }
 }
