@@ -88,3 +88,37 @@ def test_capacity_is_reported_not_faulted():
         gmb.gm_attention(ctx, z((2, 2, 16, 64), torch.bfloat16), z((1, 2, 8, 2, 16, 64), torch.bfloat16), 0,
                          z((2, 2), torch.int32), z((2,), torch.int32), z((2,), torch.int32), 2, 5, out)
     ctx.close()
+
+
+def test_4b_shape_batch_on_sampled_sequences():
+    """The benchmark's attention launch (64 sequences, KV uniform 1k..8k, 32 q / 8 kv heads, head_dim 128,
+    4 queries per sequence): three sampled sequences against the oracle, every row finite."""
+    import paper_2609_16648_b200 as gmb
+    from synth_inputs import kv_lengths_uniform
+    n_q, n_kv, hd, qs, B = 32, 8, 128, 4, 64
+    lens = kv_lengths_uniform(B, 1024, 8192, seed=3).astype(np.int64)
+    pt, npg = make_page_tables(lens + qs, 16, seed=7)
+    cfg = ModelConfig("a", 1, 64, n_q, n_kv, hd, 64, 8, batch=B, k=3, kv_len_min=0, kv_len_max=0, length_law="uniform")
+    ctx = gmb.Context(cfg, gmb.random_packed_weights(cfg, "cuda"), B, 3, pt.shape[1], npg, 4)
+    g = torch.Generator(device="cuda").manual_seed(1)
+    pool = torch.randn((1, 2, npg, n_kv, 16, hd), device="cuda", generator=g).to(torch.bfloat16)
+    q = torch.randn((B, n_kv, 16, hd), device="cuda", generator=g).to(torch.bfloat16)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device="cuda", dtype=torch.int32)
+    out = torch.zeros((B * qs, n_q * hd), dtype=torch.bfloat16, device="cuda")
+    gmb.gm_attention(ctx, q, pool, 0, dev(np.where(pt < 0, 0, pt)), dev(np.full(B, qs)), dev(lens), B, qs, out)
+    assert gmb.gm_last_status(ctx) == 0
+    got = out.float().cpu().numpy().reshape(B, qs, n_q, hd)
+    assert np.isfinite(got).all()
+    pool_h, q_h = pool.float().cpu().numpy(), q.float().cpu().numpy()
+    for b in (0, int(np.argmax(lens)), int(np.argmin(lens))):
+        S = int(lens[b]) + qs
+        idx = np.arange(S)
+        k = pool_h[0, 0, pt[b, idx // 16], :, idx % 16, :]
+        v = pool_h[0, 1, pt[b, idx // 16], :, idx % 16, :]
+        qq = np.zeros((qs, n_q, hd))
+        for j in range(qs):
+            for h in range(n_q):
+                qq[j, h] = q_h[b, h // 4, j * 4 + h % 4]
+        ref = omodel.attention(qq, k, v, np.arange(lens[b], S), idx)
+        assert np.abs(got[b] - ref).max() / np.abs(ref).max() < 1.5e-2
+    ctx.close()

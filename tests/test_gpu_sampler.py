@@ -141,3 +141,36 @@ def test_argument_validation():
         gmb.gm_accept(ctx, None, 4, 9, 1.0, lg, lg, z, None, 0, 0, z, z)
     assert e.value.code == gmb.GM_ERR_UNSUPPORTED
     ctx.close()
+
+
+def test_sampler_only_workload_full_size_all_rows():
+    """The sampler-only configuration at full size (256 sequences x 4 positions, vocabulary 151936, draft =
+    target + N(0, 0.908) noise): the device's decisions equal the oracle's decision function on the device's
+    probabilities for ALL 256 rows, and the mean acceptance is near the closed form 0.65."""
+    gmb, ctx = _ctx(151936, max_batch=256, max_k=3)
+    B, K, V = 256, 3, 151936
+    tgt, drf = sampler_only_logits(B, K, V, sigma=0.908, seed=4)
+    t_dev, d_dev = _bf16(tgt), _bf16(drf)
+    us = random_u24((B, K), seed=5)
+    dtok = torch.zeros((B, K), dtype=torch.int32, device="cuda")
+    for k in range(K):                                            # drafts drawn on the device from q_k
+        col = torch.zeros(B, dtype=torch.int32, device="cuda")
+        gmb.gm_draw(ctx, d_dev[:, k].contiguous(), B, 1.0, torch.from_numpy(us[:, k].astype(np.int32)).cuda(), col)
+        dtok[:, k] = col
+    u24 = random_u24((B, K + 1), seed=6)
+    a = torch.zeros(B, dtype=torch.int32, device="cuda")
+    t = torch.zeros(B, dtype=torch.int32, device="cuda")
+    dp = torch.zeros((B, K + 1, V), dtype=torch.float32, device="cuda")
+    dq = torch.zeros((B, K, V), dtype=torch.float32, device="cuda")
+    gmb.gm_accept(ctx, None, B, K, 1.0, t_dev, d_dev, dtok, torch.from_numpy(u24.astype(np.int32)).cuda(), 0, 0, a, t, dp, dq)
+    assert gmb.gm_last_status(ctx) == 0
+    p, q, dt = dp.cpu().numpy(), dq.cpu().numpy(), dtok.cpu().numpy()
+    an, tn = a.cpu().numpy(), t.cpu().numpy()
+    for b in range(B):
+        for k in range(K):
+            assert dt[b, k] == osampler.draw_token(q[b, k], us[b, k])[0]
+        ea, et, warn = osampler.decide(p[b], q[b], dt[b], u24[b])
+        assert (ea, et, warn) == (an[b], tn[b], 0), b
+    first = (an >= 1).mean()
+    assert 0.5 < first < 0.8, first                               # per-token acceptance ~ 0.65 (+- sampling noise)
+    ctx.close()
