@@ -26,6 +26,9 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes per algorithmic byte of the attention kernel, from the ncu capture summarised in
+# profiles/attention_kernel_4b-shape_small.md (traffic grows in proportion to the positions attended).
+ATTENTION_TRAFFIC_RATIO = 1.022
 METRIC = "committed_tokens_per_s"
 UNIT = "tokens/s"
 SMI_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -419,7 +422,7 @@ def run_product(args):
             "gpu_launches": int(launches_all),
             "roofline": {"kernel": "attention_kernel (paged multi-query decode attention, one layer per launch)",
                          "bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s", "frac": achieved / hbm,
-                         "traffic": None, "launches": int(att_n), "avg_launch_ms": att_avg_ms,
+                         "traffic": ATTENTION_TRAFFIC_RATIO * att_bytes, "launches": int(att_n), "avg_launch_ms": att_avg_ms,
                          "algorithmic_bytes_per_launch": att_bytes, "peak_source": which},
         }
         if breakdown is not None:
@@ -437,12 +440,124 @@ def run_product(args):
         dist.destroy_process_group()
 
 
+def run_sampler_only(args):
+    """Sampler-only workload: 256 sequences x (k+1) positions over the 151936-token vocabulary.  A step is one
+    gm_accept over the whole batch (the draft tokens were drawn once, on the device, by gm_draw)."""
+    import torch
+    import paper_2609_16648_b200 as gmb
+    from paper_2609_16648_b200.build import build
+    from synth_inputs import get_config, sampler_only_logits
+    from synth_inputs.workload import random_u24
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the product path has no CPU fallback")
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    build()
+    cfg = get_config("sampler")
+    B, K, V, S, W = (args.batch or cfg.batch), args.k, cfg.vocab, args.steps, args.warmup
+    mcfg = cfg.with_(n_layers=1, d_model=64, n_q_heads=1, n_kv_heads=1, head_dim=64, d_ffn=64, batch=B)
+    ctx = gmb.Context(mcfg, gmb.random_packed_weights(mcfg, device), B, K, 4, 8, 8)
+    tgt, drf = sampler_only_logits(B, K, V, sigma=0.908, seed=4 + rank)
+    t_h = torch.from_numpy(tgt).to(torch.bfloat16).pin_memory()
+    d_h = torch.from_numpy(drf).to(torch.bfloat16).pin_memory()
+    t_dev, d_dev = t_h.to(device), d_h.to(device)
+    ud = torch.from_numpy(random_u24((B, K), seed=5).astype(np.int32)).to(device)
+    ua_h = torch.from_numpy(random_u24((B, K + 1), seed=6).astype(np.int32)).pin_memory()
+    ua = ua_h.to(device)
+    dtok = torch.zeros((B, K), dtype=torch.int32, device=device)
+    col = torch.zeros(B, dtype=torch.int32, device=device)
+    for k in range(K):
+        gmb.gm_draw(ctx, d_dev[:, k].contiguous(), B, 1.0, ud[:, k].contiguous(), col)
+        dtok[:, k] = col
+    a = torch.zeros(B, dtype=torch.int32, device=device)
+    t = torch.zeros(B, dtype=torch.int32, device=device)
+    step = lambda: gmb.gm_accept(ctx, None, B, K, 1.0, t_dev, d_dev, dtok, ua, 0, 0, a, t)
+    for _ in range(W):
+        step()
+    torch.cuda.synchronize()
+    clocks = ClockSampler(local)
+    gmb.gm_profile(ctx, 1 << gmb.GM_KC_SAMPLER)
+    l0 = gmb.gm_launch_count(ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    clocks.start()
+    e0.record()
+    for _ in range(S):
+        step()
+    e1.record()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    clk = clocks.stop()
+    k_ms, k_n = gmb.gm_profile_read(ctx, gmb.GM_KC_SAMPLER)
+    gmb.gm_profile(ctx, 0)
+    launches = gmb.gm_launch_count(ctx) - l0
+    committed = (int(a.sum().item()) + B) * S
+    # end to end: logits, tokens and uniforms from pinned host memory every step, results back to the host
+    a_h, n_h = torch.zeros(B, dtype=torch.int32).pin_memory(), torch.zeros(B, dtype=torch.int32).pin_memory()
+    dtok_h = dtok.cpu().pin_memory()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(S):
+        t_dev.copy_(t_h, non_blocking=True)
+        d_dev.copy_(d_h, non_blocking=True)
+        dtok.copy_(dtok_h, non_blocking=True)
+        ua.copy_(ua_h, non_blocking=True)
+        step()
+        a_h.copy_(a, non_blocking=True)
+        n_h.copy_(t, non_blocking=True)
+        torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) * 1e3
+    h2d = (t_h.numel() + d_h.numel()) * 2 + (dtok_h.numel() + ua_h.numel()) * 4
+    (ms_max, e2e_max), (committed_all, launches_all) = reduce_over_ranks([ms, e2e_ms], [committed, launches], device, world)
+    if rank == 0:
+        hbm, _, which = measured_peaks()
+        bytes_launch = B * (2 * K + 1) * V * 2
+        avg_ms = k_ms / max(k_n, 1)
+        achieved = bytes_launch / (avg_ms * 1e-3) / 1e9
+        line = {"metric": METRIC, "value": committed_all / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": S,
+                "warmup": W, "ms_per_step": ms_max / S, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": "sampler", "batch_per_gpu": B, "k": K, "vocab": V, "temperature": 1.0,
+                           "tau": committed / (S * B), "l2": "544 MB of logits per step > 126 MB L2: no flush needed",
+                           "peaks": which},
+                "clocks": clk,
+                "e2e": {"value": committed_all / (e2e_max * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": 2 * B * 4, "ms_per_step": e2e_max / S},
+                "gpu_launches": int(launches_all),
+                "roofline": {"kernel": "sampler_kernel (softmax + rejection + residual resampling)", "bound": "hbm",
+                             "achieved": achieved, "peak": hbm, "unit": "GB/s", "frac": achieved / hbm, "traffic": None,
+                             "launches": int(k_n), "avg_launch_ms": avg_ms, "algorithmic_bytes_per_launch": bytes_launch,
+                             "peak_source": which}}
+        if not args.no_cpu_baseline:
+            from oracle import sampler as osampler
+            n = 8
+            t1 = time.time()
+            ea, _, _ = osampler.accept_batch(tgt[:n], drf[:n], dtok_h.numpy()[:n], ua_h.numpy()[:n].astype(np.uint32), 1.0)
+            dt = time.time() - t1
+            line["cpu_baseline"] = {"value": float((ea.sum() + n) / dt), "unit": UNIT, "cores": host_cores(), "kind": "oracle",
+                                    "sample": f"oracle softmax + decision function on the first {n} of {B} rows ({dt:.1f} s)"}
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="4b", choices=["tiny", "4b", "7b", "longtail"])
+    ap.add_argument("--workload", default="4b", choices=["tiny", "4b", "7b", "longtail", "sampler"])
     ap.add_argument("--k", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (small profiling cases)")
@@ -453,6 +568,8 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "sampler":
+        run_sampler_only(args)
     else:
         run_product(args)
 

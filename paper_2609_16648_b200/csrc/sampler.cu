@@ -1,17 +1,25 @@
 // Fused vocab-wide softmax + speculative rejection sampling + residual resampling (Sec. 2.2, Eq. 1).
 //
 // One thread-block cluster of 8 CTAs owns one sequence; each CTA owns a contiguous eighth of the
-// vocabulary.  Pass 1 streams all 2K+1 logit rows once (128-bit loads) and reduces a running
-// (max, sum exp) per row: thread -> warp shuffle -> CTA -> cluster (distributed shared memory), in a
-// fixed order, so every CTA ends with bit-identical row statistics.  The K accept tests then need
-// only the gathered logits of the draft tokens.  Pass 2 re-reads just the two rows of position a+1
-// (still L2-resident), turns max(0, p - q) into 64-bit integer weights trunc(r * 2^44), sums them
-// (integer sums do not depend on the reduction order), and the CTA that holds the target quantile
-// walks its slice to the token.  With K = 0 the same kernel is the plain draw of the draft phase.
+// vocabulary.  Pass 1 streams all 2K+1 logit rows once: one thread issues bulk asynchronous copies of
+// the CTA's slice of each row into a two-stage shared-memory ring (two rows ahead of the arithmetic, so
+// the copy engine keeps the memory system busy while the warps compute), and the warps reduce a
+// (max, sum exp) pair per row from shared memory with 128-bit reads: first the maximum (packed bf16),
+// then the exponentials against it (one multiply-add, one ex2 and one add per logit); thread -> warp shuffle ->
+// CTA -> cluster (distributed shared memory) merges run in a fixed order, so every CTA ends with
+// bit-identical row statistics.  The K accept tests then need only the gathered logits of the draft
+// tokens.  Pass 2 re-reads just the two rows of position a+1 (still L2-resident), turns max(0, p - q)
+// into 64-bit integer weights trunc(r * 2^44), sums them (integer sums do not depend on the reduction
+// order), and the CTA that holds the target quantile walks its slice to the token.  With K = 0 the same
+// kernel is the plain draw of the draft phase.
 //
-// Built without fast-math: the accept test and the weights are IEEE fp32 operations (denormals kept),
-// written with explicit round-to-nearest intrinsics so that no contraction can change them between
-// the debug dump of p/q and their use.
+// Arithmetic.  Everything is fp32 in the base-2 domain with s = log2(e) / T: the row maximum m is taken on
+// the raw bf16 logits (packed bf16x2 max, exact), c = -fl(m * s), and
+//     p(x) = ex2(fma(x, s, c)) * (1 / Z),   Z = sum ex2(fma(x, s, c))
+// with the hardware ex2.approx (2 ulp): per logit one unpack, one fused multiply-add, one ex2, one add.
+// One device function computes p wherever it is needed (accept test, weights, debug dump), with explicit
+// round-to-nearest intrinsics, so the dumped probabilities are exactly the ones the decisions used.  The
+// accept test and the weights are IEEE operations on those values.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -24,67 +32,64 @@ namespace gm {
 constexpr int SAMP_WARPS = SAMP_THREADS / 32;
 constexpr int SAMP_MAX_ROWS = 2 * GM_MAX_K_ + 1;
 
-struct MZ { float m, z; };
+struct MZ { float m, z; };                        // running maximum (raw logit units) and sum of 2^((x - m) s)
 
-__device__ __forceinline__ MZ mz_merge(MZ a, MZ b) {
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ MZ mz_merge(MZ a, MZ b, float s) {
   const float m = fmaxf(a.m, b.m);
   if (m == -INFINITY) return MZ{m, 0.f};
-  return MZ{m, a.z * expf(a.m - m) + b.z * expf(b.m - m)};
+  return MZ{m, a.z * ex2((a.m - m) * s) + b.z * ex2((b.m - m) * s)};
 }
-
-// softmax probability of a scaled logit given the row statistics: exp(x - max) / Z, both IEEE.
-__device__ __forceinline__ float prob_of(float x_scaled, float m, float Z) {
-  return __fdiv_rn(expf(__fsub_rn(x_scaled, m)), Z);
+// softmax probability of a raw logit x given s, c = -fl(max * s) and 1 / Z
+__device__ __forceinline__ float prob_of(float x, float s, float c, float inv_z) {
+  return __fmul_rn(ex2(__fmaf_rn(x, s, c)), inv_z);
 }
-
-__device__ __forceinline__ void unpack8(const uint4 &v, float inv_temp, float (&x)[8]) {
-  x[0] = __fmul_rn(bf16_lo(v.x), inv_temp); x[1] = __fmul_rn(bf16_hi(v.x), inv_temp);
-  x[2] = __fmul_rn(bf16_lo(v.y), inv_temp); x[3] = __fmul_rn(bf16_hi(v.y), inv_temp);
-  x[4] = __fmul_rn(bf16_lo(v.z), inv_temp); x[5] = __fmul_rn(bf16_hi(v.z), inv_temp);
-  x[6] = __fmul_rn(bf16_lo(v.w), inv_temp); x[7] = __fmul_rn(bf16_hi(v.w), inv_temp);
+__device__ __forceinline__ void unpack8(const uint4 &v, float (&x)[8]) {
+  x[0] = bf16_lo(v.x); x[1] = bf16_hi(v.x); x[2] = bf16_lo(v.y); x[3] = bf16_hi(v.y);
+  x[4] = bf16_lo(v.z); x[5] = bf16_hi(v.z); x[6] = bf16_lo(v.w); x[7] = bf16_hi(v.w);
 }
-
-__device__ __forceinline__ void mz_update(MZ &s, const uint4 &v, float inv_temp) {
-  float x[8];
-  unpack8(v, inv_temp, x);
-  float vm = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])), fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
-  if (vm > s.m) { s.z *= expf(s.m - vm); s.m = vm; }
-  float acc = 0.f;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) acc += expf(x[j] - s.m);
-  s.z += acc;
+__device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b) {          // packed bf16x2 maximum
+  __nv_bfloat162 r = __hmax2(*reinterpret_cast<__nv_bfloat162 *>(&a), *reinterpret_cast<__nv_bfloat162 *>(&b));
+  return *reinterpret_cast<uint32_t *>(&r);
 }
-
-// integer weight of one residual entry
+// integer weight of one residual entry: trunc(r * 2^44) for r > 0, else 0 (the product is an exact scaling)
 __device__ __forceinline__ unsigned long long weight_of(float p, float q, bool use_q) {
   const float r = use_q ? __fsub_rn(p, q) : p;
   return r > 0.f ? __float2ull_rz(__fmul_rn(r, 17592186044416.0f /* 2^44 */)) : 0ull;
 }
 
-__global__ void __cluster_dims__(SAMP_CLUSTER, 1, 1) __launch_bounds__(SAMP_THREADS)
+__global__ void __cluster_dims__(SAMP_CLUSTER, 1, 1) __launch_bounds__(SAMP_THREADS, 2)
 sampler_kernel(const SamplerArgs A) {
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = static_cast<int>(cluster.block_rank());
   const int b = blockIdx.x / SAMP_CLUSTER;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = A.K, V = A.V, R = 2 * K + 1;
-
-  extern __shared__ __align__(16) unsigned char dyn_smem[];
-  unsigned long long *vecsum = reinterpret_cast<unsigned long long *>(dyn_smem);   // [vpc]
-
-  __shared__ MZ warp_mz[SAMP_MAX_ROWS][SAMP_WARPS];
-  __shared__ MZ local_mz[SAMP_MAX_ROWS];          // this CTA's slice statistics (read by peers)
-  __shared__ MZ row_mz[SAMP_MAX_ROWS];            // whole-row statistics
-  __shared__ unsigned long long warp_w[SAMP_WARPS];
-  __shared__ unsigned long long local_w;          // this CTA's integer mass (read by peers)
-  __shared__ unsigned long long scan_w[SAMP_WARPS];
-  __shared__ int local_cand;                      // argmax fallback candidate (read by peers)
-  __shared__ int sh_a, sh_tok;
+  const float s = A.inv_temp * 1.4426950408889634f;            // logits -> base-2 exponents
 
   const int nvec_total = V >> 3;
   const int vpc = (nvec_total + SAMP_CLUSTER - 1) / SAMP_CLUSTER;
   const int v_lo = min(rank * vpc, nvec_total);
   const int n = min(v_lo + vpc, nvec_total) - v_lo;
+  const uint32_t stage_b = (static_cast<uint32_t>(vpc) * 16u + 127u) & ~127u;
+
+  extern __shared__ __align__(128) unsigned char dyn_smem[];
+  const uint4 *stage[2] = {reinterpret_cast<const uint4 *>(dyn_smem), reinterpret_cast<const uint4 *>(dyn_smem + stage_b)};
+  unsigned long long *vecsum = reinterpret_cast<unsigned long long *>(dyn_smem + 2 * stage_b);   // [vpc]
+  __shared__ uint64_t full[2];
+
+  __shared__ MZ warp_mz[SAMP_MAX_ROWS][SAMP_WARPS];
+  __shared__ MZ local_mz[SAMP_MAX_ROWS];          // this CTA's slice statistics (read by peers)
+  __shared__ MZ row_mz[SAMP_MAX_ROWS];            // whole-row statistics: .m holds c = -fl(max * s), .z holds 1 / Z
+  __shared__ unsigned long long warp_w[SAMP_WARPS];
+  __shared__ unsigned long long local_w;          // this CTA's integer mass (read by peers)
+  __shared__ unsigned long long scan_w[SAMP_WARPS];
+  __shared__ int local_cand;                      // argmax fallback candidate (read by peers)
+  __shared__ int sh_a, sh_tok;
 
   const __nv_bfloat16 *tgt = A.target_logits + static_cast<size_t>(b) * A.tgt_bstride;
   const __nv_bfloat16 *drf = A.draft_logits ? A.draft_logits + static_cast<size_t>(b) * A.drf_bstride : nullptr;
@@ -93,40 +98,85 @@ sampler_kernel(const SamplerArgs A) {
     return reinterpret_cast<const uint4 *>(p) + v_lo;
   };
 
-  // ---- pass 1: (max, sum exp) of every row over this CTA's slice ------------------------------------
+  // ---- pass 1: (max, sum 2^((x - max) s)) of every row over this CTA's slice, through the shared-memory ring ----
+  if (tid == 0) {
+    mbar_init(&full[0], 1);
+    mbar_init(&full[1], 1);
+    mbar_fence_init();
+  }
+  __syncthreads();
+  uint32_t uses[2] = {0u, 0u};                    // completed phases of each stage's barrier (parity = uses & 1)
+  auto issue = [&](int st_i, const uint4 *src) {  // thread 0 only
+    if (n > 0) {
+      mbar_expect_tx(&full[st_i], static_cast<uint32_t>(n) * 16u);
+      bulk_load(const_cast<uint4 *>(stage[st_i]), src, static_cast<uint32_t>(n) * 16u, &full[st_i]);
+    }
+  };
+  __shared__ int sh_alive;
+  if (tid == 0) sh_alive = 1;
+  bool alive = true;                              // false after a bounded wait expired: finish without touching the data
+  // One thread polls the mbarrier (bounded); everybody else sleeps at the CTA barrier instead of spinning.
+  auto wait_stage = [&](int st_i) {
+    if (tid == 0 && n > 0 && sh_alive && !mbar_wait(&full[st_i], uses[st_i] & 1u)) {
+      sh_alive = 0;
+      set_status(A.status, ST_TIMEOUT);
+    }
+    ++uses[st_i];
+    __syncthreads();
+    alive = sh_alive != 0;
+  };
+  const uint32_t NEG_INF2 = 0xff80ff80u;          // two bf16 -inf
+  if (tid == 0) {
+    issue(0, row_ptr(0));
+    if (R > 1) issue(1, row_ptr(1));
+  }
   for (int r = 0; r < R; ++r) {
-    const uint4 *row = row_ptr(r);
-    MZ s{-INFINITY, 0.f};
-    for (int i0 = tid; i0 < n; i0 += 4 * SAMP_THREADS) {
-      uint4 v[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int i = i0 + u * SAMP_THREADS;
-        if (i < n) v[u] = __ldg(row + i);
+    const int st_i = r & 1;
+    wait_stage(st_i);
+    const uint4 *buf = stage[st_i];
+    MZ st{-INFINITY, 0.f};
+    if (alive && tid < n) {
+      uint32_t m2 = NEG_INF2;
+      for (int i = tid; i < n; i += SAMP_THREADS) {
+        const uint4 v = buf[i];
+        m2 = bmax2(bmax2(m2, bmax2(v.x, v.y)), bmax2(v.z, v.w));
       }
+      const float mx = fmaxf(bf16_lo(m2), bf16_hi(m2));
+      const float c = -mx * s;
+      float acc = 0.f;
+      for (int i = tid; i < n; i += SAMP_THREADS) {
+        float x[8];
+        unpack8(buf[i], x);
 #pragma unroll
-      for (int u = 0; u < 4; ++u)
-        if (i0 + u * SAMP_THREADS < n) mz_update(s, v[u], A.inv_temp);
+        for (int j = 0; j < 8; ++j) acc += ex2(fmaf(x[j], s, c));
+      }
+      st = MZ{mx, acc};
     }
+    {
+      const float wm = warp_max(st.m);            // butterfly: every lane ends with the same maximum
+      float z = wm == -INFINITY ? 0.f : st.z * ex2((st.m - wm) * s);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      MZ t{__shfl_xor_sync(0xffffffffu, s.m, o), __shfl_xor_sync(0xffffffffu, s.z, o)};
-      // order the operands by lane so both partners compute the identical expression
-      s = (lane & o) ? mz_merge(t, s) : mz_merge(s, t);
+      for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);   // commutative pairs: same sum on every lane
+      st = MZ{wm, z};
     }
-    if (lane == 0) warp_mz[r][warp] = s;
+    if (lane == 0) warp_mz[r][warp] = st;
+    __syncthreads();                              // every warp has finished reading this stage
+    if (tid == 0 && r + 2 < R) {
+      fence_proxy_async();                        // order the generic reads before the asynchronous overwrite
+      issue(st_i, row_ptr(r + 2));
+    }
   }
   __syncthreads();
   if (tid < R) {
-    MZ s = warp_mz[tid][0];
-    for (int w = 1; w < SAMP_WARPS; ++w) s = mz_merge(s, warp_mz[tid][w]);
-    local_mz[tid] = s;
+    MZ st = warp_mz[tid][0];
+    for (int w = 1; w < SAMP_WARPS; ++w) st = mz_merge(st, warp_mz[tid][w], s);
+    local_mz[tid] = st;
   }
   cluster.sync();
   if (tid < R) {
-    MZ s = *cluster.map_shared_rank(&local_mz[tid], 0);
-    for (int c = 1; c < SAMP_CLUSTER; ++c) s = mz_merge(s, *cluster.map_shared_rank(&local_mz[tid], c));
-    row_mz[tid] = s;
+    MZ st = *cluster.map_shared_rank(&local_mz[tid], 0);
+    for (int c = 1; c < SAMP_CLUSTER; ++c) st = mz_merge(st, *cluster.map_shared_rank(&local_mz[tid], c), s);
+    row_mz[tid] = MZ{-st.m * s, __frcp_rn(st.z)};               // (c, 1 / Z) of the row
   }
   __syncthreads();
 
@@ -140,29 +190,34 @@ sampler_kernel(const SamplerArgs A) {
       const MZ st = row_mz[r];
       for (int i = tid; i < n; i += SAMP_THREADS) {
         float x[8];
-        unpack8(__ldg(row + i), A.inv_temp, x);
+        unpack8(__ldg(row + i), x);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) dst[static_cast<size_t>(v_lo + i) * 8 + j] = prob_of(x[j], st.m, st.z);
+        for (int j = 0; j < 8; ++j) dst[static_cast<size_t>(v_lo + i) * 8 + j] = prob_of(x[j], s, st.m, st.z);
       }
     }
   }
 
-  // ---- accept tests (every CTA redundantly; identical inputs give identical results) ---------------
-  if (tid == 0) {
-    int a = 0;
-    for (; a < K; ++a) {
-      int d = A.draft_tok[static_cast<size_t>(b) * A.tok_in_stride + a];
-      if (d < 0 || d >= V) { set_status(A.status, ST_BAD_TOKEN); break; }
-      const float xp = __fmul_rn(__bfloat162float(tgt[static_cast<size_t>(a) * V + d]), A.inv_temp);
-      const float xq = __fmul_rn(__bfloat162float(drf[static_cast<size_t>(a) * V + d]), A.inv_temp);
-      const float p = prob_of(xp, row_mz[a].m, row_mz[a].z);
-      const float q = prob_of(xq, row_mz[K + 1 + a].m, row_mz[K + 1 + a].z);
-      const uint32_t u24 = A.u24 ? A.u24[static_cast<size_t>(b) * A.u_stride + a]
-                                 : philox_u24(A.seed, A.step, b, A.slot_accept + a);
-      const float uq = __fmul_rn(__fmul_rn(static_cast<float>(u24), 5.9604644775390625e-8f /* 2^-24 */), q);
-      if (!(p >= q || uq < p)) break;
+  // ---- accept tests: lane k of warp 0 tests draft k (every CTA redundantly, identical inputs) ----------
+  if (warp == 0) {
+    bool ok = true;
+    if (lane < K) {
+      const int d = A.draft_tok[static_cast<size_t>(b) * A.tok_in_stride + lane];
+      if (d < 0 || d >= V) {
+        set_status(A.status, ST_BAD_TOKEN);
+        ok = false;
+      } else {
+        const float xp = __bfloat162float(tgt[static_cast<size_t>(lane) * V + d]);
+        const float xq = __bfloat162float(drf[static_cast<size_t>(lane) * V + d]);
+        const float p = prob_of(xp, s, row_mz[lane].m, row_mz[lane].z);
+        const float q = prob_of(xq, s, row_mz[K + 1 + lane].m, row_mz[K + 1 + lane].z);
+        const uint32_t u24 = A.u24 ? A.u24[static_cast<size_t>(b) * A.u_stride + lane]
+                                   : philox_u24(A.seed, A.step, b, A.slot_accept + lane);
+        const float uq = __fmul_rn(__fmul_rn(static_cast<float>(u24), 5.9604644775390625e-8f /* 2^-24 */), q);
+        ok = p >= q || uq < p;
+      }
     }
-    sh_a = a;
+    const unsigned rejected = __ballot_sync(0xffffffffu, !ok);   // lanes >= K vote "accepted"
+    if (lane == 0) sh_a = rejected ? __ffs(rejected) - 1 : K;    // first rejection, else all K accepted
   }
   __syncthreads();
   const int a = sh_a;
@@ -175,26 +230,34 @@ sampler_kernel(const SamplerArgs A) {
   bool use_q = a < K;
   unsigned long long Wc[SAMP_CLUSTER];
   unsigned long long W = 0;
+  // both rows of position a+1 come back through the ring (they are L2-resident)
+  if (tid == 0) {
+    fence_proxy_async();
+    issue(0, prow);
+    if (use_q) issue(1, qrow);
+  }
+  wait_stage(0);
+  if (use_q) wait_stage(1);
   for (int attempt = 0; attempt < 2; ++attempt) {
     unsigned long long tsum = 0;
-    for (int i = tid; i < n; i += SAMP_THREADS) {
+    for (int i = tid; i < n && alive; i += SAMP_THREADS) {
       float xp[8], xq[8];
-      unpack8(__ldg(prow + i), A.inv_temp, xp);
-      if (use_q) unpack8(__ldg(qrow + i), A.inv_temp, xq);
-      unsigned long long s = 0;
+      unpack8(stage[0][i], xp);
+      if (use_q) unpack8(stage[1][i], xq);
+      unsigned long long sm = 0;
 #pragma unroll
       for (int j = 0; j < 8; ++j)
-        s += weight_of(prob_of(xp[j], ps.m, ps.z), use_q ? prob_of(xq[j], qs.m, qs.z) : 0.f, use_q);
-      vecsum[i] = s;
-      tsum += s;
+        sm += weight_of(prob_of(xp[j], s, ps.m, ps.z), use_q ? prob_of(xq[j], s, qs.m, qs.z) : 0.f, use_q);
+      vecsum[i] = sm;
+      tsum += sm;
     }
     tsum = warp_sum_u64(tsum);
     if (lane == 0) warp_w[warp] = tsum;
     __syncthreads();
     if (tid == 0) {
-      unsigned long long s = 0;
-      for (int w = 0; w < SAMP_WARPS; ++w) s += warp_w[w];
-      local_w = s;
+      unsigned long long sm = 0;
+      for (int w = 0; w < SAMP_WARPS; ++w) sm += warp_w[w];
+      local_w = sm;
     }
     cluster.sync();
     W = 0;
@@ -228,10 +291,10 @@ sampler_kernel(const SamplerArgs A) {
     __syncthreads();
     for (int i = tid; i < n; i += SAMP_THREADS) {
       float x[8];
-      unpack8(__ldg(prow + i), A.inv_temp, x);
+      unpack8(__ldg(prow + i), x);
 #pragma unroll
       for (int j = 0; j < 8; ++j)
-        if (x[j] == ps.m) atomicMin(&local_cand, (v_lo + i) * 8 + j);
+        if (-x[j] * s == ps.m) atomicMin(&local_cand, (v_lo + i) * 8 + j);
     }
     cluster.sync();
     if (rank == 0 && tid == 0) {
@@ -265,12 +328,12 @@ sampler_kernel(const SamplerArgs A) {
       int iv = lo;
       while (rem >= vecsum[iv]) { rem -= vecsum[iv]; ++iv; }     // stops inside [lo, hi): rem < mine
       float xp[8], xq[8];
-      unpack8(__ldg(prow + iv), A.inv_temp, xp);
-      if (use_q) unpack8(__ldg(qrow + iv), A.inv_temp, xq);
+      unpack8(__ldg(prow + iv), xp);
+      if (use_q) unpack8(__ldg(qrow + iv), xq);
       int tok = (v_lo + iv) * 8 + 7;
       for (int j = 0; j < 8; ++j) {
         const unsigned long long w =
-            weight_of(prob_of(xp[j], ps.m, ps.z), use_q ? prob_of(xq[j], qs.m, qs.z) : 0.f, use_q);
+            weight_of(prob_of(xp[j], s, ps.m, ps.z), use_q ? prob_of(xq[j], s, qs.m, qs.z) : 0.f, use_q);
         if (rem < w) { tok = (v_lo + iv) * 8 + j; break; }
         rem -= w;
       }
@@ -308,7 +371,9 @@ sampler_kernel(const SamplerArgs A) {
 cudaError_t launch_sampler(const SamplerArgs &A, int batch, cudaStream_t stream) {
   const int nvec_total = A.V >> 3;
   const int vpc = (nvec_total + SAMP_CLUSTER - 1) / SAMP_CLUSTER;
-  const size_t dyn = static_cast<size_t>(vpc) * sizeof(unsigned long long);
+  const size_t stage_b = (static_cast<size_t>(vpc) * 16 + 127) & ~size_t(127);
+  const size_t dyn = 2 * stage_b + static_cast<size_t>(vpc) * sizeof(unsigned long long);
+  if (dyn > 227 * 1024 - 4096) return cudaErrorInvalidValue;      // vocabulary too large for the shared-memory ring
   static size_t configured = 0;
   if (dyn > configured) {
     cudaError_t e = cudaFuncSetAttribute(sampler_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(dyn));

@@ -53,8 +53,9 @@ def test_accept_decisions_bit_exact_on_dumped_probabilities(B, K, V, sigma, temp
     # the dumped probabilities are the softmax of the logits (fp32 arithmetic on the device)
     ref_p = osampler.softmax_probs(tgt, temp)
     ref_q = osampler.softmax_probs(drf, temp)
-    assert np.abs(p - ref_p).max() <= 2e-6 * ref_p.max() + 1e-9
-    assert np.abs(q - ref_q).max() <= 2e-6 * ref_q.max() + 1e-9
+    # exponent arguments reach 2^5, so each of their three roundings (c of the thread, of the merge, of the row) moves p by <= 1.3e-6
+    assert np.abs(p - ref_p).max() <= 5e-6 * ref_p.max() + 1e-9
+    assert np.abs(q - ref_q).max() <= 5e-6 * ref_q.max() + 1e-9
     np.testing.assert_allclose(p.sum(-1), 1.0, atol=2e-5)
     # end to end (oracle softmax in fp64 instead of the device's): decisions agree on almost every row
     ea, et, _ = osampler.accept_batch(tgt, drf, dtok, u24, temp)
