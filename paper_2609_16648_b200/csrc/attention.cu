@@ -31,13 +31,17 @@ template <int HD> struct AttCfg {
 };
 
 static int att_hpc(int n_kv) { return n_kv < ATT_MAX_HPC ? n_kv : ATT_MAX_HPC; }
-static int att_stages(int n_kv, int hd) {
+// With two 16-row query tiles the Q fragments do not fit in registers next to the output accumulators:
+// they are kept in shared memory (32 rows x head_dim per KV head) and fetched with ldmatrix per page.
+static int att_q_bytes(int n_kv, int hd, int mt) { return mt >= 2 ? att_hpc(n_kv) * 32 * hd * 2 : 0; }
+static int att_stages(int n_kv, int hd, int mt) {
   const int sb = 2 * (hd / 64) * att_hpc(n_kv) * 16 * 128;
-  int s = ATT_SMEM_BUDGET / sb;
+  int s = (ATT_SMEM_BUDGET - att_q_bytes(n_kv, hd, mt)) / sb;
   return s > 8 ? 8 : (s < 2 ? 2 : s);
 }
-size_t attention_smem_bytes(int n_kv, int hd) {
-  return static_cast<size_t>(att_stages(n_kv, hd)) * 2 * (hd / 64) * att_hpc(n_kv) * 16 * 128 + 1024 + 256;
+size_t attention_smem_bytes(int n_kv, int hd, int mt) {
+  return static_cast<size_t>(att_stages(n_kv, hd, mt)) * 2 * (hd / 64) * att_hpc(n_kv) * 16 * 128 + 1024 + 1024 +
+         att_q_bytes(n_kv, hd, mt);
 }
 int attention_max_ctas(int n_kv, int hd) {
   (void)n_kv; (void)hd;
@@ -65,6 +69,8 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
   const int stage_b = C::stage_bytes(hpc);
   uint64_t *full = reinterpret_cast<uint64_t *>(smem + static_cast<size_t>(nstages) * stage_b);
   uint64_t *empty = full + 8;
+  // Q staging area (two-tile variant only), 1024-byte aligned after the barriers
+  unsigned char *qsm = smem + ((static_cast<size_t>(nstages) * stage_b + 128 + 1023) & ~size_t(1023));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int B = A.batch;
@@ -139,19 +145,33 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
     if (seg_lo >= seg_hi) continue;
     const int qn = A.qn[b], qbase = A.qbase[b];
 
-    // query fragments
-    uint32_t qf[MT][KSTEPS][4];
+    // query fragments: in registers for one 16-row tile; staged in shared memory (128-byte rows, XOR swizzle)
+    // for two tiles and fetched per page
+    constexpr int QREG = MT == 1 ? KSTEPS : 1;
+    uint32_t qf[MT][QREG][4];
     const __nv_bfloat16 *qp = A.qbuf + (static_cast<size_t>(b) * A.n_kv + head) * A.qrows * HD;
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
+    const uint32_t q_smem = smem_u32(qsm) + warp * (32 * HD * 2);
+    if constexpr (MT == 1) {
 #pragma unroll
       for (int ks = 0; ks < KSTEPS; ++ks) {
-        const __nv_bfloat16 *r0 = qp + (mt * 16 + r8) * HD + ks * 16 + 2 * t4;
-        qf[mt][ks][0] = *reinterpret_cast<const uint32_t *>(r0);
-        qf[mt][ks][1] = *reinterpret_cast<const uint32_t *>(r0 + 8 * HD);
-        qf[mt][ks][2] = *reinterpret_cast<const uint32_t *>(r0 + 8);
-        qf[mt][ks][3] = *reinterpret_cast<const uint32_t *>(r0 + 8 * HD + 8);
+        const __nv_bfloat16 *r0 = qp + r8 * HD + ks * 16 + 2 * t4;
+        qf[0][ks][0] = *reinterpret_cast<const uint32_t *>(r0);
+        qf[0][ks][1] = *reinterpret_cast<const uint32_t *>(r0 + 8 * HD);
+        qf[0][ks][2] = *reinterpret_cast<const uint32_t *>(r0 + 8);
+        qf[0][ks][3] = *reinterpret_cast<const uint32_t *>(r0 + 8 * HD + 8);
       }
+    } else {
+      __syncwarp();                               // the previous segment's fragment reads are done
+      constexpr int CPR = HD / 8;                 // 16-byte chunks per row
+      for (int idx = lane; idx < 32 * CPR; idx += 32) {
+        const int row = idx / CPR, ch = idx % CPR;
+        const uint4 v = *reinterpret_cast<const uint4 *>(qp + row * HD + ch * 8);
+        unsigned char *dst = qsm + warp * (32 * HD * 2) + (ch >> 3) * (32 * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4);
+        *reinterpret_cast<uint4 *>(dst) = v;
+      }
+      __syncwarp();
+    }
+    const int q_row = (lane & 7) + ((lane >> 3) & 1) * 8, q_chunk = lane >> 4;   // ldmatrix lane address (A fragment)
     float o[MT][NT][4];
     float mrow[MT][2], lrow[MT][2];
 #pragma unroll
@@ -179,8 +199,15 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
         ldmatrix_x4(kf, kbase + (ks >> 2) * tile_b + k_row_off + ((chunk ^ k_sw) << 4));
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-          mma_16816(sc[mt][0], qf[mt][ks], kf[0], kf[1]);
-          mma_16816(sc[mt][1], qf[mt][ks], kf[2], kf[3]);
+          if constexpr (MT == 1) {
+            mma_16816(sc[mt][0], qf[mt][ks], kf[0], kf[1]);
+            mma_16816(sc[mt][1], qf[mt][ks], kf[2], kf[3]);
+          } else {
+            const int row = mt * 16 + q_row;
+            ldmatrix_x4(qf[mt][0], q_smem + (ks >> 2) * (32 * 128) + row * 128 + ((((ks & 3) * 2 + q_chunk) ^ (row & 7)) << 4));
+            mma_16816(sc[mt][0], qf[mt][0], kf[0], kf[1]);
+            mma_16816(sc[mt][1], qf[mt][0], kf[2], kf[3]);
+          }
         }
       }
 
@@ -282,8 +309,8 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
 
 template <int HD, int MT>
 static cudaError_t launch_att(const AttnArgs &A, cudaStream_t stream) {
-  const int hpc = att_hpc(A.n_kv), nst = att_stages(A.n_kv, HD);
-  const size_t smem = attention_smem_bytes(A.n_kv, HD);
+  const int hpc = att_hpc(A.n_kv), nst = att_stages(A.n_kv, HD, MT);
+  const size_t smem = attention_smem_bytes(A.n_kv, HD, MT);
   static size_t configured = 0;
   if (smem > configured) {
     cudaError_t e = cudaFuncSetAttribute(attention_kernel<HD, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,

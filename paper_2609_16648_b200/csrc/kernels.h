@@ -110,7 +110,7 @@ cudaError_t launch_attention_combine(const AttnCombineArgs &A, cudaStream_t stre
 cudaError_t launch_page_prefix(const int32_t *qn, const int32_t *qbase, int batch, int max_pages_per_seq, int q_stride,
                                int32_t *page_start, uint32_t *status, cudaStream_t stream);
 int attention_max_ctas(int n_kv, int hd);   // CTAs the attention kernel wants for this shape (<= SM count)
-size_t attention_smem_bytes(int n_kv, int hd);
+size_t attention_smem_bytes(int n_kv, int hd, int mt);
 
 // ---- GEMM --------------------------------------------------------------------------------------------------
 // out = epilogue(x[M, K] * w[N, K]^T) with fp32 accumulation.
