@@ -74,6 +74,7 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int B = A.batch;
+  pdl_prologue();
   const long long P = A.page_start[B];
   // never more ranges than pages: every active CTA then owns at least one page, so the CTAs that hold
   // pieces of one sequence are consecutive and so are its segment ids
@@ -319,8 +320,7 @@ static cudaError_t launch_att(const AttnArgs &A, cudaStream_t stream) {
     configured = smem;
   }
   dim3 grid(A.n_ctas, A.n_kv / hpc);
-  attention_kernel<HD, MT><<<grid, (hpc + 1) * 32, smem, stream>>>(A, hpc, nst);
-  return cudaGetLastError();
+  return launch_k(attention_kernel<HD, MT>, grid, dim3((hpc + 1) * 32), smem, stream, 1, A, hpc, nst);
 }
 
 cudaError_t launch_attention(const AttnArgs &A, cudaStream_t stream) {
@@ -339,6 +339,7 @@ cudaError_t launch_attention(const AttnArgs &A, cudaStream_t stream) {
 __global__ void __launch_bounds__(128) attention_combine_kernel(const AttnCombineArgs A) {
   const int b = blockIdx.x / A.n_kv, head = blockIdx.x % A.n_kv;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_prologue();
   const int qn = A.qn[b];
   const long long P = A.page_start[A.batch];
   const long long G = P < static_cast<long long>(A.n_ctas) ? P : static_cast<long long>(A.n_ctas);   // as in the kernel above
@@ -381,8 +382,7 @@ __global__ void __launch_bounds__(128) attention_combine_kernel(const AttnCombin
   }
 }
 cudaError_t launch_attention_combine(const AttnCombineArgs &A, cudaStream_t stream) {
-  attention_combine_kernel<<<A.batch * A.n_kv, 128, 0, stream>>>(A);
-  return cudaGetLastError();
+  return launch_k(attention_combine_kernel, dim3(A.batch * A.n_kv), dim3(128), 0, stream, 1, A);
 }
 
 // ---- page prefix for a caller-given query layout (stand-alone attention calls) -------------------------------------------
@@ -390,6 +390,7 @@ cudaError_t launch_attention_combine(const AttnCombineArgs &A, cudaStream_t stre
 // is reported and given no pages (its output rows are then left untouched).
 __global__ void page_prefix_kernel(const int32_t *qn, const int32_t *qbase, int batch, int max_pages_per_seq,
                                    int q_stride, int32_t *page_start, uint32_t *status) {
+  pdl_prologue();
   if (threadIdx.x != 0) return;
   int acc = 0;
   for (int b = 0; b < batch; ++b) {
@@ -403,8 +404,8 @@ __global__ void page_prefix_kernel(const int32_t *qn, const int32_t *qbase, int 
 }
 cudaError_t launch_page_prefix(const int32_t *qn, const int32_t *qbase, int batch, int max_pages_per_seq, int q_stride,
                                int32_t *page_start, uint32_t *status, cudaStream_t stream) {
-  page_prefix_kernel<<<1, 32, 0, stream>>>(qn, qbase, batch, max_pages_per_seq, q_stride, page_start, status);
-  return cudaGetLastError();
+  return launch_k(page_prefix_kernel, dim3(1), dim3(32), 0, stream, 1, qn, qbase, batch, max_pages_per_seq, q_stride,
+                  page_start, status);
 }
 
 }  // namespace gm

@@ -20,6 +20,16 @@ enum : uint32_t {
 
 __device__ __forceinline__ void set_status(uint32_t *status, uint32_t bit) { atomicOr(status, bit); }
 
+// ---- programmatic dependent launch ------------------------------------------------------------------
+// Every kernel of the library starts with pdl_prologue(): it lets the next kernel of the stream begin its launch
+// (that kernel's CTAs take SM slots as this grid's CTAs retire and run their own set-up), then waits until the
+// previous kernel has completed and its memory is visible.  Nothing before this call may touch global memory.
+// Without the launch attribute both instructions are no-ops.
+__device__ __forceinline__ void pdl_prologue() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ---- small math -----------------------------------------------------------------------------------
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }

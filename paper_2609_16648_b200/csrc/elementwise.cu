@@ -57,6 +57,7 @@ __device__ __forceinline__ float4 load_bf16x4(const __nv_bfloat16 *p) {
 __global__ void plan_kernel(const PlanArgs A) {
   __shared__ int pages[1024];
   const int B = A.batch;
+  pdl_prologue();
   for (int b = threadIdx.x; b < B; b += blockDim.x) {
     const int len = A.kv_len[b];
     int qn, qbase;
@@ -79,8 +80,7 @@ __global__ void plan_kernel(const PlanArgs A) {
 }
 cudaError_t launch_plan(const PlanArgs &A, cudaStream_t stream) {
   if (A.batch > 1024) return cudaErrorInvalidValue;
-  plan_kernel<<<1, 256, 0, stream>>>(A);
-  return cudaGetLastError();
+  return launch_k(plan_kernel, dim3(1), dim3(256), 0, stream, 1, A);
 }
 
 // ---- embedding gather + first RMSNorm of the verify forward ------------------------------------------------
@@ -89,6 +89,7 @@ embed_norm_kernel(const __nv_bfloat16 *embed, const __nv_bfloat16 *w, const int3
                   const int32_t *pending_n, const int32_t *draft_tok, int K, int max_k, int d, int vocab, float eps,
                   float *x, __nv_bfloat16 *xn, uint32_t *status) {
   const int m = blockIdx.x, b = m / (K + 1), j = m % (K + 1);
+  pdl_prologue();
   int tok;
   if (j == 0) {
     const int n = min(max(pending_n[b], 1), max_k + 1);
@@ -113,9 +114,8 @@ cudaError_t launch_embed_norm(const __nv_bfloat16 *embed, const __nv_bfloat16 *w
                               const int32_t *pending_n, const int32_t *draft_tok, int batch, int K, int max_k, int d,
                               int vocab, float eps, float *x, __nv_bfloat16 *xn, uint32_t *status,
                               cudaStream_t stream) {
-  embed_norm_kernel<<<batch * (K + 1), EW_THREADS, 0, stream>>>(embed, w, pending_tok, pending_n, draft_tok, K, max_k,
-                                                                d, vocab, eps, x, xn, status);
-  return cudaGetLastError();
+  return launch_k(embed_norm_kernel, dim3(batch * (K + 1)), dim3(EW_THREADS), 0, stream, 1, embed, w, pending_tok,
+                  pending_n, draft_tok, K, max_k, d, vocab, eps, x, xn, status);
 }
 
 // ---- draft-head input: [RMSNorm_e(embedding) ; RMSNorm_h(hidden)] ---------------------------------------------
@@ -123,6 +123,7 @@ __global__ void __launch_bounds__(EW_THREADS) head_input_kernel(const HeadInputA
   const int m = blockIdx.x, b = m / A.QT, j = m % A.QT;
   const int d = A.d, d4 = d >> 2;
   __nv_bfloat16 *out = A.zin + static_cast<size_t>(m) * 2 * d;
+  pdl_prologue();
   int tok = 0;
   bool valid = true;
   const __nv_bfloat16 *hid_bf = nullptr;
@@ -158,14 +159,14 @@ __global__ void __launch_bounds__(EW_THREADS) head_input_kernel(const HeadInputA
   rmsnorm_store(v, d4, d, A.eps, A.wh, out + d);
 }
 cudaError_t launch_head_input(const HeadInputArgs &A, cudaStream_t stream) {
-  head_input_kernel<<<A.batch * A.QT, EW_THREADS, 0, stream>>>(A);
-  return cudaGetLastError();
+  return launch_k(head_input_kernel, dim3(A.batch * A.QT), dim3(EW_THREADS), 0, stream, 1, A);
 }
 
 // ---- RMSNorm of the fp32 residual stream ------------------------------------------------------------------------------
 __global__ void __launch_bounds__(EW_THREADS)
 rmsnorm_kernel(const float *x, const __nv_bfloat16 *w, __nv_bfloat16 *xn, __nv_bfloat16 *hidden_out, int d, float eps) {
   const int m = blockIdx.x, d4 = d >> 2;
+  pdl_prologue();
   float4 v[EW_MAXC];
 #pragma unroll
   for (int c = 0; c < EW_MAXC; ++c) {
@@ -184,8 +185,7 @@ rmsnorm_kernel(const float *x, const __nv_bfloat16 *w, __nv_bfloat16 *xn, __nv_b
 }
 cudaError_t launch_rmsnorm(const float *x, const __nv_bfloat16 *w, __nv_bfloat16 *xn, __nv_bfloat16 *hidden_out,
                            int M, int d, float eps, cudaStream_t stream) {
-  rmsnorm_kernel<<<M, EW_THREADS, 0, stream>>>(x, w, xn, hidden_out, d, eps);
-  return cudaGetLastError();
+  return launch_k(rmsnorm_kernel, dim3(M), dim3(EW_THREADS), 0, stream, 1, x, w, xn, hidden_out, d, eps);
 }
 
 // ---- rotary embedding + KV append + Q rearrangement --------------------------------------------------------------------
@@ -202,6 +202,7 @@ __global__ void __launch_bounds__(EW_THREADS) rope_append_kernel(const RopeAppen
   const int m = blockIdx.x, b = m / A.QT, j = m % A.QT;
   const int hd = A.hd, half = hd >> 1, group = A.n_q / A.n_kv;
   const int ncols = (A.n_q + 2 * A.n_kv) * hd;
+  pdl_prologue();
   const int qn = A.qn[b];
   const int hv = half >> 3;                                       // 8-wide items per half head
   __nv_bfloat16 *qdst = A.qbuf + static_cast<size_t>(b) * A.n_kv * A.qrows * hd;
@@ -250,8 +251,7 @@ __global__ void __launch_bounds__(EW_THREADS) rope_append_kernel(const RopeAppen
   }
 }
 cudaError_t launch_rope_append(const RopeAppendArgs &A, cudaStream_t stream) {
-  rope_append_kernel<<<A.batch * A.QT, EW_THREADS, 0, stream>>>(A);
-  return cudaGetLastError();
+  return launch_k(rope_append_kernel, dim3(A.batch * A.QT), dim3(EW_THREADS), 0, stream, 1, A);
 }
 
 // ---- head output row: last valid row of each sequence + the head's final norm ----------------------------------------------
@@ -259,6 +259,7 @@ __global__ void __launch_bounds__(EW_THREADS)
 head_out_kernel(const float *x, const int32_t *qn, int QT, int d, const __nv_bfloat16 *w, float eps, float *g,
                 __nv_bfloat16 *gn) {
   const int b = blockIdx.x, d4 = d >> 2;
+  pdl_prologue();
   const int j = min(max(qn[b], 1), QT) - 1;
   const float4 *src = reinterpret_cast<const float4 *>(x + (static_cast<size_t>(b) * QT + j) * d);
   float4 v[EW_MAXC];
@@ -274,8 +275,7 @@ head_out_kernel(const float *x, const int32_t *qn, int QT, int d, const __nv_bfl
 }
 cudaError_t launch_head_out(const float *x, const int32_t *qn, int batch, int QT, int d, const __nv_bfloat16 *w,
                             float eps, float *g, __nv_bfloat16 *gn, cudaStream_t stream) {
-  head_out_kernel<<<batch, EW_THREADS, 0, stream>>>(x, qn, QT, d, w, eps, g, gn);
-  return cudaGetLastError();
+  return launch_k(head_out_kernel, dim3(batch), dim3(EW_THREADS), 0, stream, 1, x, qn, QT, d, w, eps, g, gn);
 }
 
 }  // namespace gm

@@ -117,15 +117,18 @@ gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
     tc_alloc(tmem_slot, ncols);
     tc_relinquish();
   }
+  if (warp == 0 && lane == 0) {
+    tma_prefetch_desc(&A.w_map);
+    tma_prefetch_desc(&A.x_map);
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  pdl_prologue();                                  // everything above touches no global data: it overlaps the previous kernel
 
   if (warp == 0) {
     if (lane == 0) {
-      tma_prefetch_desc(&A.w_map);
-      tma_prefetch_desc(&A.x_map);
       for (int kb = kb_lo, it = 0; kb < kb_hi; ++kb, ++it) {
         const int s = it % nstages;
         if (!mbar_wait(&empty[s], ((it / nstages) & 1) ^ 1)) { set_status(A.status, ST_TIMEOUT); break; }
@@ -249,17 +252,8 @@ cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream) {
   const size_t smem = gt_smem(T, A.wtiles);
   cudaError_t ec = gt_configure();
   if (ec != cudaSuccess) return ec;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((A.N + GT_BN * A.wtiles - 1) / (GT_BN * A.wtiles), (A.M + T - 1) / T, A.nsplit);
-  cfg.blockDim = dim3(GT_THREADS);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = A.nsplit;
-  cfg.attrs = attr;
-  cfg.numAttrs = A.nsplit > 1 ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel, A, gt_stages(T, A.wtiles));
+  const dim3 grid((A.N + GT_BN * A.wtiles - 1) / (GT_BN * A.wtiles), (A.M + T - 1) / T, A.nsplit);
+  return launch_k(gemm_tc_kernel, grid, dim3(GT_THREADS), smem, stream, A.nsplit, A, gt_stages(T, A.wtiles));
 }
 
 // ---- plain mma.sync GEMM ----------------------------------------------------------------------------------------------
@@ -268,6 +262,7 @@ cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream) {
 __global__ void __launch_bounds__(128) gemm_simple_kernel(const GemmArgs A) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, t4 = lane & 3, r8 = lane >> 2;
   const int m0 = blockIdx.y * 64 + warp * 16, n0 = blockIdx.x * 64;
+  pdl_prologue();
   float acc[8][4];
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
@@ -320,8 +315,7 @@ __global__ void __launch_bounds__(128) gemm_simple_kernel(const GemmArgs A) {
 cudaError_t launch_gemm_simple(const GemmArgs &A, cudaStream_t stream) {
   if (A.K % 16) return cudaErrorInvalidValue;
   dim3 grid((A.N + 63) / 64, (A.M + 63) / 64, 1);
-  gemm_simple_kernel<<<grid, 128, 0, stream>>>(A);
-  return cudaGetLastError();
+  return launch_k(gemm_simple_kernel, grid, dim3(128), 0, stream, 1, A);
 }
 
 }  // namespace gm

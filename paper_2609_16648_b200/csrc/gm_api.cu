@@ -17,6 +17,13 @@
 
 using namespace gm;
 
+namespace gm {
+bool pdl_enabled() {
+  static const bool on = std::getenv("GM_NO_PDL") == nullptr;
+  return on;
+}
+}  // namespace gm
+
 namespace {
 
 struct LayerMaps { CUtensorMap wqkv, wo, wgu, wdown; };

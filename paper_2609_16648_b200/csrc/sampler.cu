@@ -70,6 +70,7 @@ sampler_kernel(const SamplerArgs A) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = A.K, V = A.V, R = 2 * K + 1;
   const float s = A.inv_temp * 1.4426950408889634f;            // logits -> base-2 exponents
+  pdl_prologue();
 
   const int nvec_total = V >> 3;
   const int vpc = (nvec_total + SAMP_CLUSTER - 1) / SAMP_CLUSTER;
@@ -380,8 +381,7 @@ cudaError_t launch_sampler(const SamplerArgs &A, int batch, cudaStream_t stream)
     if (e != cudaSuccess) return e;
     configured = dyn;
   }
-  sampler_kernel<<<batch * SAMP_CLUSTER, SAMP_THREADS, dyn, stream>>>(A);
-  return cudaGetLastError();
+  return launch_k(sampler_kernel, dim3(batch * SAMP_CLUSTER), dim3(SAMP_THREADS), dyn, stream, 1, A);
 }
 
 }  // namespace gm
