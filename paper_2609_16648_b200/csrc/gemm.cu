@@ -101,7 +101,7 @@ gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
   float *park = reinterpret_cast<float *>(smem);                // [T][128] fp32, reuses the pipeline stages
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * GT_BN * wt, m0 = blockIdx.y * T, split = blockIdx.z, ns = A.nsplit;
+  const int n0 = A.n_base + blockIdx.x * GT_BN * wt, m0 = blockIdx.y * T, split = blockIdx.z, ns = A.nsplit;
   const int KB = A.K / GT_BK;
   const int kb_lo = static_cast<int>(static_cast<long long>(split) * KB / ns);
   const int kb_hi = static_cast<int>(static_cast<long long>(split + 1) * KB / ns);
@@ -247,12 +247,12 @@ cudaError_t gemm_tc_max_clusters(int block_t, int nsplit, int *out) {
 cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream) {
   const int T = A.block_t;
   if (T < 16 || T > 256 || (T & 15) || (A.K % GT_BK) || A.nsplit < 1 || A.nsplit > A.K / GT_BK || A.nsplit > 8 ||
-      A.wtiles < 1 || A.wtiles > 2)
+      A.wtiles < 1 || A.wtiles > 2 || A.n_tiles < 1 || A.n_base < 0)
     return cudaErrorInvalidValue;
   const size_t smem = gt_smem(T, A.wtiles);
   cudaError_t ec = gt_configure();
   if (ec != cudaSuccess) return ec;
-  const dim3 grid((A.N + GT_BN * A.wtiles - 1) / (GT_BN * A.wtiles), (A.M + T - 1) / T, A.nsplit);
+  const dim3 grid(A.n_tiles, (A.M + T - 1) / T, A.nsplit);
   return launch_k(gemm_tc_kernel, grid, dim3(GT_THREADS), smem, stream, A.nsplit, A, gt_stages(T, A.wtiles));
 }
 

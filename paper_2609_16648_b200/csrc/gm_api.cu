@@ -195,12 +195,37 @@ int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *w
     GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_simple(A, c->stream));
     return GM_OK;
   }
-  A.nsplit = pick_split(c, M, N, K, T);
-  // wide projections: two sub-tiles per CTA halve the activation re-reads from L2
-  if (A.nsplit == 1 && ((N + 127) / 128) * ((M + T - 1) / T) >= c->sm_count) A.wtiles = 2;
-  A.w_map = *wmap;
   int rc = x_map(c, x, x_rows, K, T, &A.x_map);
   if (rc != GM_OK) return rc;
+  A.w_map = *wmap;
+  const int mblocks = (M + T - 1) / T;
+  const int tiles128 = (N + 127) / 128;
+  A.nsplit = pick_split(c, M, N, K, T);
+  // very wide projections: two sub-tiles per CTA halve the activation re-reads from L2
+  if (A.nsplit == 1 && tiles128 * mblocks >= 2 * c->sm_count) A.wtiles = 2;
+  const int units = (tiles128 + A.wtiles - 1) / A.wtiles;          // CTAs along N
+  A.n_base = 0;
+  A.n_tiles = units;
+  // Wave quantisation: a few CTAs more than a multiple of the SM count would cost a whole extra wave.  Run the full
+  // waves as they are and the leftover features as a short launch whose tiles are split along K over clusters.
+  const int rem = (units * mblocks) % c->sm_count;
+  if (A.nsplit == 1 && mblocks == 1 && units > c->sm_count && rem != 0 && rem * 4 <= c->sm_count) {
+    A.n_tiles = units - rem;
+    GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(A, c->stream));
+    GemmArgs Tl = A;
+    Tl.n_base = A.n_tiles * 128 * A.wtiles;
+    Tl.wtiles = 1;
+    Tl.n_tiles = (N - Tl.n_base + 127) / 128;
+    Tl.nsplit = 1;
+    const int KB = K / 64;
+    for (int ns = 2; ns <= 8 && ns <= KB; ++ns) {
+      int &cap = c->max_clusters[T / 16][ns];
+      if (cap < 0) { int v = 0; if (gemm_tc_max_clusters(T, ns, &v) != cudaSuccess) { v = 0; (void)cudaGetLastError(); } cap = v; }
+      if (cap >= Tl.n_tiles) Tl.nsplit = ns;
+    }
+    GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(Tl, c->stream));
+    return GM_OK;
+  }
   GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(A, c->stream));
   return GM_OK;
 }

@@ -153,6 +153,8 @@ struct GemmArgs {
   const __nv_bfloat16 *x, *w;
   void *out; int epi;
   int M, N, K;
+  int n_base;                           // first output feature of this launch (a projection may be issued as main part + tail)
+  int n_tiles;                          // CTAs along N of this launch
   int nsplit;                           // K slices = cluster size along z (1..8); the simple kernel ignores it
   int block_t;                          // tokens per CTA (multiple of 16, <= 256)
   int wtiles;                           // 128-feature sub-tiles per CTA sharing one activation tile (1 or 2)
