@@ -7,8 +7,9 @@
 // elected thread) is the TMA producer filling a ring of 128-byte-swizzled stages (64 K-elements per
 // stage: a 128 x 64 weight box and a T x 64 activation box); warp 1 owns the tensor memory
 // allocation and one of its threads issues tcgen05.mma (four K=16 instructions per stage),
-// releasing each stage with tcgen05.commit; warps 2-5 read the fp32 accumulator out of tensor
-// memory with tcgen05.ld once the last commit lands.
+// releasing each stage with tcgen05.commit; warps 2-9 read the fp32 accumulator out of tensor
+// memory with tcgen05.ld once the last commit lands (two warps per TMEM lane quadrant, alternating
+// 16-column chunks), and all 16 warps run the reduction and the epilogue.
 //
 // Split-K without a trip through HBM.  Projections with few output tiles (N = d_model gives 20)
 // are cut along K over blockIdx.z, and the CTAs of one output tile form a thread-block cluster.
@@ -32,7 +33,7 @@ namespace gm {
 
 constexpr int GT_BN = 128;            // output features per MMA (its M extent); a CTA owns wt = 1 or 2 such sub-tiles
 constexpr int GT_BK = 64;             // K elements per stage (one 128-byte swizzle row)
-constexpr int GT_THREADS = 192;
+constexpr int GT_THREADS = 512;     // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: TMEM readers; all 16 warps reduce + store
 constexpr int GT_SMEM_BUDGET = 200 * 1024;
 
 static int gt_stages(int block_t, int wt) {
@@ -160,7 +161,8 @@ gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
     }
   }
   bool acc_ok = kb_hi > kb_lo;
-  if (warp >= 2) {
+  const bool reader = warp >= 2 && warp < 10;
+  if (reader) {
     if (acc_ok && !mbar_wait(acc_full, 0)) { set_status(A.status, ST_TIMEOUT); acc_ok = false; }
     tc_fence_after();
   }
@@ -169,11 +171,11 @@ gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
   const int c_lo = split * per, c_hi = min(T, c_lo + per);
   for (int a = 0; a < wt; ++a) {
     __syncthreads();                               // the pipeline stages (first pass) / the previous sub-tile are done with
-    if (warp >= 2) {
+    if (reader) {
       // TMEM -> registers -> parked fp32 tile in shared memory (lanes = consecutive features: no bank conflicts)
       const int quad = warp & 3;                   // the TMEM lane quadrant this warp may read
       const int r = quad * 32 + lane;
-      for (int c0 = 0; c0 < T; c0 += 16) {
+      for (int c0 = ((warp - 2) >> 2) * 16; c0 < T; c0 += 32) {
         uint32_t v[16];
         if (acc_ok) {
           tc_ld_32x16(tmem + (static_cast<uint32_t>(quad * 32) << 16) + a * acc_cols + c0, v);
