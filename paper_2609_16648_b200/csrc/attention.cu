@@ -341,6 +341,7 @@ __global__ void __launch_bounds__(128) attention_combine_kernel(const AttnCombin
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   pdl_prologue();
   const int qn = A.qn[b];
+  const int row_first = blockIdx.y * 4 + warp;     // one query row per warp: the dependent loads of a row are paid once
   const long long P = A.page_start[A.batch];
   const long long G = P < static_cast<long long>(A.n_ctas) ? P : static_cast<long long>(A.n_ctas);   // as in the kernel above
   const int ps = A.page_start[b], pe = A.page_start[b + 1];
@@ -348,7 +349,7 @@ __global__ void __launch_bounds__(128) attention_combine_kernel(const AttnCombin
   const int s_first = cta_of_page(ps, P, G) + b, s_last = cta_of_page(pe - 1, P, G) + b;
   const int nseg = s_last - s_first + 1;
   const int rows = qn * A.group, hd = A.hd;
-  for (int row = warp; row < rows; row += 4) {
+  for (int row = row_first; row < rows; row += 4 * gridDim.y) {
     const size_t base0 = (static_cast<size_t>(s_first) * A.n_kv + head) * A.qrows + row;
     const size_t seg_stride = static_cast<size_t>(A.n_kv) * A.qrows;
     float mt = -INFINITY;
@@ -382,7 +383,7 @@ __global__ void __launch_bounds__(128) attention_combine_kernel(const AttnCombin
   }
 }
 cudaError_t launch_attention_combine(const AttnCombineArgs &A, cudaStream_t stream) {
-  return launch_k(attention_combine_kernel, dim3(A.batch * A.n_kv), dim3(128), 0, stream, 1, A);
+  return launch_k(attention_combine_kernel, dim3(A.batch * A.n_kv, (A.QT * A.group + 3) / 4), dim3(128), 0, stream, 1, A);
 }
 
 // ---- page prefix for a caller-given query layout (stand-alone attention calls) -------------------------------------------
