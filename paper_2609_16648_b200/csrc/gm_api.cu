@@ -163,8 +163,12 @@ int round16(int v) { return (v + 15) & ~15; }
 // resident at once (GPC packing decides), so the slices of a tile run concurrently and the SMs are filled.
 int pick_split(gm_ctx *c, int M, int N, int K, int T) {
   const int tiles = ((N + 127) / 128) * ((M + T - 1) / T);
-  if (tiles * 3 >= c->sm_count * 2) return 1;
   const int KB = K / 64;
+  if (const char *ov = std::getenv("GM_GEMM_SPLIT")) {            // tuning aid: force the K-split of small projections
+    const int ns = std::atoi(ov);
+    if (ns >= 1 && ns <= 8 && ns <= KB && tiles * 3 < c->sm_count * 2) return ns;
+  }
+  if (tiles * 3 >= c->sm_count * 2) return 1;
   int best = 1;
   for (int ns = 2; ns <= 8 && ns <= KB; ++ns) {
     int &cap = c->max_clusters[T / 16][ns];
