@@ -319,9 +319,15 @@ def run_product(args):
     seed = 1234 + rank
     step_id = 0
 
+    rec = gmb.Record(B, K, cfg.d_model, device) if args.record else None
+    d_dev = torch.zeros((B, K), dtype=torch.int32, device=device)
+
     def one_step():
         nonlocal step_id
-        gmb.gm_spec_step(ctx, st, K, 1.0, seed, step_id, a_dev, t_dev)
+        if rec is not None:
+            gmb.gm_spec_step_rec(ctx, st, K, 1.0, seed, step_id, a_dev, t_dev, d_dev, rec)
+        else:
+            gmb.gm_spec_step(ctx, st, K, 1.0, seed, step_id, a_dev, t_dev)
         acc_sum.add_(a_dev.sum())
         step_id += 1
 
@@ -339,7 +345,7 @@ def run_product(args):
         torch.cuda.synchronize()
 
     clocks = ClockSampler(local)
-    gmb.gm_profile(ctx, 1 << gmb.GM_KC_ATTENTION)
+    gmb.gm_profile(ctx, (1 << gmb.GM_KC_ATTENTION) | (1 << gmb.GM_KC_RECORD))
     launches0 = gmb.gm_launch_count(ctx)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -353,6 +359,7 @@ def run_product(args):
     clk = clocks.stop()
     launches = gmb.gm_launch_count(ctx) - launches0
     att_ms, att_n = gmb.gm_profile_read(ctx, gmb.GM_KC_ATTENTION)
+    rec_ms, rec_n = gmb.gm_profile_read(ctx, gmb.GM_KC_RECORD)
     gmb.gm_profile(ctx, 0)
     accepted = int(acc_sum.item())
     committed = accepted + S * B
@@ -427,6 +434,11 @@ def run_product(args):
         }
         if breakdown is not None:
             line["config"]["breakdown"] = breakdown
+        if rec is not None and rec_n:
+            rb = B * K * cfg.vocab * 2
+            line["config"]["record"] = {"what": "per-cycle record (top-64 target log-probs of k positions + 4 small items)",
+                                        "topk_ms_per_launch": rec_ms / rec_n, "algorithmic_bytes": rb,
+                                        "GB_per_s": rb / (rec_ms / rec_n * 1e-3) / 1e9}
         if not args.no_cpu_baseline and world >= 1:
             try:
                 line["cpu_baseline"] = cpu_baseline(args.workload, K)
@@ -562,6 +574,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (small profiling cases)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (small profiling cases)")
+    ap.add_argument("--record", action="store_true", help="also write the per-cycle verification record every step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--breakdown", action="store_true", help="add device time per kernel class (extra pass)")
     args = ap.parse_args()

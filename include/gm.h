@@ -176,6 +176,30 @@ int gm_spec_step_host(gm_ctx *ctx, gm_state *st, int k, float temperature, uint6
                       uint64_t step, const uint32_t *u24_draft_host, const uint32_t *u24_accept_host,
                       int32_t *accept_len_host, int32_t *next_token_host, int32_t *draft_tok_host);
 
+/* The record a cycle leaves for the head update (App. D.2 "Recording in Rollout"): the backbone hidden state
+ * at the cycle's start, the k drafts, the verification distributions kept as the target's top-64
+ * log-probabilities in bf16 WITH full-vocabulary normalisation (not renormalised over the retained set), the
+ * accepted length with the final token counted, and the absolute position of the start.  Entries of a row
+ * are ordered by logit descending, ties by token id ascending; rows with fewer than 64 tokens are padded with
+ * index -1 / log-probability -inf.  All pointers are device buffers owned by the caller.                  */
+typedef struct {
+  void    *start_hidden;            /* bf16 [B, d]      hidden state the first draft application consumed   */
+  int32_t *start_pos;               /* [B]              context length at which drafting starts (kv_len+1)  */
+  int32_t *drafts;                  /* [B, k]                                                                */
+  void    *top_logprob;             /* bf16 [B, k, 64]  log p_j at the target's 64 largest logits, j = 1..k  */
+  int32_t *top_index;               /* [B, k, 64]       their token ids                                      */
+  int32_t *accepted;                /* [B]              accepted drafts + 1                                  */
+} gm_record;
+/* gm_record_begin: call before the cycle (fills start_hidden, start_pos from the state).
+ * gm_record_end:   call after gm_accept (fills drafts, top_logprob, top_index, accepted from the cycle's
+ *                  target logits [B, k+1, V], draft tokens [B, k] and accept_len [B]).
+ * gm_spec_step_rec: gm_spec_step with both calls around it; the cycle itself is unchanged bit for bit.       */
+int gm_record_begin(gm_ctx *ctx, const gm_state *st, gm_record *rec);
+int gm_record_end(gm_ctx *ctx, int batch, int k, float temperature, const void *target_logits,
+                  const int32_t *draft_tok, const int32_t *accept_len, gm_record *rec);
+int gm_spec_step_rec(gm_ctx *ctx, gm_state *st, int k, float temperature, uint64_t seed, uint64_t step,
+                     int32_t *accept_len, int32_t *next_token, int32_t *draft_tok, gm_record *rec);
+
 /* Dense projection out[M, N] = x[M, K] w[N, K]^T on the context's stream (bf16 in, fp32
  * accumulate; the kernel every QKV / O / FFN / LM-head projection of the step uses).
  *   out_fp32 != 0: out is fp32 [M, N]; else bf16 [M, N].  K % 64 == 0, N % 8 == 0, M >= 1.   */
@@ -231,7 +255,8 @@ int gm_attention_noalloc(int n_q_heads, int n_kv_heads, int head_dim, int max_pa
 #define GM_KC_ATTENTION  1
 #define GM_KC_ELEMENTWISE 2
 #define GM_KC_SAMPLER    3
-#define GM_KC_COUNT      4
+#define GM_KC_RECORD     4
+#define GM_KC_COUNT      5
 int gm_profile(gm_ctx *ctx, int class_mask);
 int gm_profile_read(gm_ctx *ctx, int kernel_class, double *total_ms, int64_t *launches);
 

@@ -20,10 +20,11 @@ GM_ERR_DEVICE_TIMEOUT, GM_ERR_BAD_PAGE, GM_ERR_NO_EXTENSION, GM_ERR_SCRATCH_LIMI
 GM_NOALLOC_SCRATCH_BYTES, GM_NOALLOC_MAX_BATCH = 16 << 20, 256
 GM_MAX_K, GM_PAGE = 7, 16
 GM_FLAG_SIMPLE_GEMM = 1
-GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER = 0, 1, 2, 3
+GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER, GM_KC_RECORD = 0, 1, 2, 3, 4
 
 EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw",
-           "gm_spec_step_host", "gm_gemm", "gm_attention", "gm_attention_noalloc", "gm_profile", "gm_profile_read", "gm_launch_count",
+           "gm_spec_step_host", "gm_gemm", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
+           "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
 
 
@@ -51,6 +52,10 @@ class gm_state(C.Structure):
                 ("pending_tok", C.c_void_p), ("pending_hidden", C.c_void_p)]
 
 
+class gm_record(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("start_hidden", "start_pos", "drafts", "top_logprob", "top_index", "accepted")]
+
+
 _lib = None
 
 
@@ -76,6 +81,9 @@ def lib() -> C.CDLL:
     L.gm_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
     L.gm_attention.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, i32, i32, vp]
     L.gm_attention_noalloc.argtypes = [i32, i32, i32, i32, vp, vp, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp]
+    L.gm_record_begin.argtypes = [vp, C.POINTER(gm_state), C.POINTER(gm_record)]
+    L.gm_record_end.argtypes = [vp, i32, i32, f32, vp, vp, vp, C.POINTER(gm_record)]
+    L.gm_spec_step_rec.argtypes = [vp, C.POINTER(gm_state), i32, f32, u64, u64, vp, vp, vp, C.POINTER(gm_record)]
     L.gm_profile.argtypes = [vp, i32]
     L.gm_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     L.gm_launch_count.argtypes = [vp]
@@ -291,6 +299,41 @@ def gm_attention_noalloc(n_q_heads: int, n_kv_heads: int, head_dim: int, q, kv_p
     _check(lib().gm_attention_noalloc(n_q_heads, n_kv_heads, head_dim, page_table.shape[1], _p(q), _p(kv_pool),
                                       kv_pool.shape[0], kv_pool.shape[2], layer, _p(page_table), _p(q_count), _p(q_base),
                                       batch, q_stride, _p(out), C.c_void_p(stream.cuda_stream)), "gm_attention_noalloc")
+
+
+class Record:
+    """Device tensors of struct gm_record."""
+
+    def __init__(self, batch: int, k: int, d_model: int, device="cuda"):
+        z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=device)
+        self.start_hidden = z((batch, d_model), torch.bfloat16)
+        self.start_pos = z((batch,), torch.int32)
+        self.drafts = z((batch, k), torch.int32)
+        self.top_logprob = z((batch, k, 64), torch.bfloat16)
+        self.top_index = z((batch, k, 64), torch.int32)
+        self.accepted = z((batch,), torch.int32)
+
+    def struct(self) -> gm_record:
+        return gm_record(*[getattr(self, n).data_ptr() for n in ("start_hidden", "start_pos", "drafts", "top_logprob",
+                                                                  "top_index", "accepted")])
+
+
+def gm_record_begin(ctx: Context, st: State, rec: Record):
+    s, r = st.struct(), rec.struct()
+    _check(lib().gm_record_begin(ctx.handle, C.byref(s), C.byref(r)), "gm_record_begin")
+
+
+def gm_record_end(ctx: Context, batch: int, k: int, temperature: float, target_logits, draft_tok, accept_len, rec: Record):
+    r = rec.struct()
+    _check(lib().gm_record_end(ctx.handle, batch, k, temperature, _p(target_logits), _p(draft_tok), _p(accept_len),
+                               C.byref(r)), "gm_record_end")
+
+
+def gm_spec_step_rec(ctx: Context, st: State, k: int, temperature: float, seed: int, step: int, accept_len, next_token,
+                     draft_tok, rec: Record):
+    s, r = st.struct(), rec.struct()
+    _check(lib().gm_spec_step_rec(ctx.handle, C.byref(s), k, temperature, seed, step, _p(accept_len), _p(next_token),
+                                  _p(draft_tok), C.byref(r)), "gm_spec_step_rec")
 
 
 def gm_profile(ctx: Context, class_mask: int):

@@ -66,7 +66,7 @@ struct gm_ctx {
   // profiling
   int prof_mask = 0;
   std::vector<EventPair> events[GM_KC_COUNT];
-  size_t events_used[GM_KC_COUNT] = {0, 0, 0, 0};
+  size_t events_used[GM_KC_COUNT] = {};
   int64_t launches = 0;
   cudaError_t last_cuda = cudaSuccess;
 };
@@ -625,6 +625,44 @@ int gm_spec_step_host(gm_ctx *c, gm_state *st, int k, float temperature, uint64_
     GM_CUDA(c, cudaMemcpyAsync(draft_tok_host, c->ws_draft_tok, B * k * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
   GM_CUDA(c, cudaStreamSynchronize(c->stream));
   return GM_OK;
+}
+
+int gm_record_begin(gm_ctx *c, const gm_state *st, gm_record *rec) {
+  if (!c || !st || !rec || !rec->start_hidden || !rec->start_pos) return GM_ERR_INVALID_ARG;
+  if (st->batch < 1 || st->batch > c->cfg.max_batch || !st->kv_len || !st->pending_n || !st->pending_hidden)
+    return GM_ERR_INVALID_ARG;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+            launch_record_begin(st->kv_len, st->pending_n, static_cast<const __nv_bfloat16 *>(st->pending_hidden), st->batch,
+                                c->cfg.max_k, c->d, static_cast<__nv_bfloat16 *>(rec->start_hidden), rec->start_pos,
+                                c->stream));
+  return GM_OK;
+}
+
+int gm_record_end(gm_ctx *c, int batch, int k, float temperature, const void *target_logits, const int32_t *draft_tok,
+                  const int32_t *accept_len, gm_record *rec) {
+  if (!c || !rec || !target_logits || !draft_tok || !accept_len || !rec->drafts || !rec->top_logprob || !rec->top_index ||
+      !rec->accepted)
+    return GM_ERR_INVALID_ARG;
+  if (batch < 1 || k < 1) return GM_ERR_INVALID_ARG;
+  if (k > GM_MAX_K || !(temperature > 0.f) || !std::isfinite(temperature)) return GM_ERR_UNSUPPORTED;
+  RecordTopkArgs R;
+  R.target_logits = static_cast<const __nv_bfloat16 *>(target_logits); R.bstride = static_cast<size_t>(k + 1) * c->V;
+  R.K = k; R.V = c->V; R.inv_temp = 1.0f / temperature; R.top_logprob = static_cast<__nv_bfloat16 *>(rec->top_logprob);
+  R.top_index = rec->top_index; R.status = c->status;
+  GM_LAUNCH(c, GM_KC_RECORD, launch_record_topk(R, batch, c->stream));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_record_end(draft_tok, accept_len, batch, k, rec->drafts, rec->accepted, c->stream));
+  return GM_OK;
+}
+
+int gm_spec_step_rec(gm_ctx *c, gm_state *st, int k, float temperature, uint64_t seed, uint64_t step, int32_t *accept_len,
+                     int32_t *next_token, int32_t *draft_tok, gm_record *rec) {
+  int rc = check_state(c, st, k);
+  if (rc) return rc;
+  if (!accept_len || !next_token || !rec) return GM_ERR_INVALID_ARG;
+  if ((rc = gm_record_begin(c, st, rec)) != GM_OK) return rc;
+  int32_t *dt = draft_tok ? draft_tok : c->ws_draft_tok;
+  if ((rc = spec_step_impl(c, st, k, temperature, nullptr, nullptr, seed, step, accept_len, next_token, dt)) != GM_OK) return rc;
+  return gm_record_end(c, st->batch, k, temperature, c->ws_target_logits, dt, accept_len, rec);
 }
 
 int gm_gemm(gm_ctx *c, const void *x, const void *w, void *out, int M, int N, int K, int out_fp32) {

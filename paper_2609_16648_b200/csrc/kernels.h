@@ -66,6 +66,23 @@ struct SamplerArgs {
 };
 cudaError_t launch_sampler(const SamplerArgs &A, int batch, cudaStream_t stream);
 
+// ---- cycle record (top-64 target log-probabilities and the other recorded items) ---------------------------------
+struct RecordTopkArgs {
+  const __nv_bfloat16 *target_logits;   // row (b, k) at target_logits + b*bstride + k*V, k = 0..K-1
+  size_t bstride;
+  int K, V;
+  float inv_temp;
+  __nv_bfloat16 *top_logprob;           // [B, K, 64]
+  int32_t *top_index;                   // [B, K, 64]
+  uint32_t *status;
+};
+cudaError_t launch_record_topk(const RecordTopkArgs &A, int batch, cudaStream_t stream);
+cudaError_t launch_record_begin(const int32_t *kv_len, const int32_t *pending_n, const __nv_bfloat16 *pending_hidden,
+                                int batch, int max_k, int d, __nv_bfloat16 *start_hidden, int32_t *start_pos,
+                                cudaStream_t stream);
+cudaError_t launch_record_end(const int32_t *draft_tok, const int32_t *accept_len, int batch, int k, int32_t *drafts,
+                              int32_t *accepted, cudaStream_t stream);
+
 // ---- planning: query ranges of a phase and the balanced attention partition --------------------------
 enum PhaseMode { PHASE_VERIFY = 0, PHASE_DRAFT_FIRST = 1, PHASE_DRAFT_NEXT = 2 };
 struct PlanArgs {
