@@ -1,17 +1,17 @@
 // Fused vocab-wide softmax + speculative rejection sampling + residual resampling (Sec. 2.2, Eq. 1).
 //
 // One thread-block cluster of 8 CTAs owns one sequence; each CTA owns a contiguous eighth of the
-// vocabulary.  Pass 1 streams all 2K+1 logit rows once: one thread issues bulk asynchronous copies of
-// the CTA's slice of each row into a two-stage shared-memory ring (two rows ahead of the arithmetic, so
-// the copy engine keeps the memory system busy while the warps compute), and the warps reduce a
-// (max, sum exp) pair per row from shared memory with 128-bit reads: first the maximum (packed bf16),
-// then the exponentials against it (one multiply-add, one ex2 and one add per logit); thread -> warp shuffle ->
+// vocabulary.  Positions are walked in order: one thread issues bulk asynchronous copies of the CTA's
+// slices of the rows p_k and q_k into a two-stage shared-memory ring, the warps reduce a (max, sum exp)
+// pair per row from shared memory with 128-bit reads - first the maximum (packed bf16), then the
+// exponentials against it (one multiply-add, one ex2 and one add per logit); thread -> warp shuffle ->
 // CTA -> cluster (distributed shared memory) merges run in a fixed order, so every CTA ends with
-// bit-identical row statistics.  The K accept tests then need only the gathered logits of the draft
-// tokens.  Pass 2 re-reads just the two rows of position a+1 (still L2-resident), turns max(0, p - q)
-// into 64-bit integer weights trunc(r * 2^44), sums them (integer sums do not depend on the reduction
-// order), and the CTA that holds the target quantile walks its slice to the token.  With K = 0 the same
-// kernel is the plain draw of the draft phase.
+// bit-identical row statistics - and accept test k needs only the gathered logits of draft k.  The walk
+// stops at the first rejection (or at the bonus position): rows of later positions are never read, and the
+// two rows of position a+1 are still in the ring, so the resampling pass turns max(0, p - q) into 64-bit
+// integer weights trunc(r * 2^44) straight from shared memory, sums them (integer sums do not depend on
+// the reduction order), and the CTA that holds the target quantile walks its slice to the token.  With
+// K = 0 the same kernel is the plain draw of the draft phase.
 //
 // Arithmetic.  Everything is fp32 in the base-2 domain with s = log2(e) / T: the row maximum m is taken on
 // the raw bf16 logits (packed bf16x2 max, exact), c = -fl(m * s), and
@@ -84,7 +84,7 @@ sampler_kernel(const SamplerArgs A) {
   __shared__ uint64_t full[2];
 
   __shared__ MZ warp_mz[SAMP_MAX_ROWS][SAMP_WARPS];
-  __shared__ MZ local_mz[SAMP_MAX_ROWS];          // this CTA's slice statistics (read by peers)
+  __shared__ MZ local_mz[2][2];                   // this CTA's slice statistics (read by peers), double-buffered by call parity
   __shared__ MZ row_mz[SAMP_MAX_ROWS];            // whole-row statistics: .m holds c = -fl(max * s), .z holds 1 / Z
   __shared__ unsigned long long warp_w[SAMP_WARPS];
   __shared__ unsigned long long local_w;          // this CTA's integer mass (read by peers)
@@ -99,7 +99,7 @@ sampler_kernel(const SamplerArgs A) {
     return reinterpret_cast<const uint4 *>(p) + v_lo;
   };
 
-  // ---- pass 1: (max, sum 2^((x - max) s)) of every row over this CTA's slice, through the shared-memory ring ----
+  // ---- shared-memory ring: stage 0 holds the target row, stage 1 the draft row of the position in flight ----------
   if (tid == 0) {
     mbar_init(&full[0], 1);
     mbar_init(&full[1], 1);
@@ -127,14 +127,8 @@ sampler_kernel(const SamplerArgs A) {
     alive = sh_alive != 0;
   };
   const uint32_t NEG_INF2 = 0xff80ff80u;          // two bf16 -inf
-  if (tid == 0) {
-    issue(0, row_ptr(0));
-    if (R > 1) issue(1, row_ptr(1));
-  }
-  for (int r = 0; r < R; ++r) {
-    const int st_i = r & 1;
-    wait_stage(st_i);
-    const uint4 *buf = stage[st_i];
+  // (max, sum 2^((x - max) s)) of the row slice in `buf`, per warp, into warp_mz[slot]
+  auto slice_stats = [&](const uint4 *buf, int slot) {
     MZ st{-INFINITY, 0.f};
     if (alive && tid < n) {
       uint32_t m2 = NEG_INF2;
@@ -153,92 +147,98 @@ sampler_kernel(const SamplerArgs A) {
       }
       st = MZ{mx, acc};
     }
-    {
-      const float wm = warp_max(st.m);            // butterfly: every lane ends with the same maximum
-      float z = wm == -INFINITY ? 0.f : st.z * ex2((st.m - wm) * s);
+    const float wm = warp_max(st.m);              // butterfly: every lane ends with the same maximum
+    float z = wm == -INFINITY ? 0.f : st.z * ex2((st.m - wm) * s);
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);   // commutative pairs: same sum on every lane
-      st = MZ{wm, z};
+    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);   // commutative pairs: same sum on every lane
+    if (lane == 0) warp_mz[slot][warp] = MZ{wm, z};
+  };
+  // whole-row (c, 1 / Z) of slots 0..nslots-1 from the slice statistics: warps, then the 8 CTAs in rank order, so
+  // that every CTA of the cluster holds bit-identical values in row_mz
+  int stats_calls = 0;                            // same sequence in every CTA of the cluster
+  auto finish_stats = [&](int nslots) {
+    MZ *mine = local_mz[stats_calls & 1];         // a buffer is rewritten two calls later: the call in between has a
+    ++stats_calls;                                // cluster barrier that every peer passes only after reading it
+    __syncthreads();                              // also: every warp has finished reading the stages
+    if (tid < nslots) {
+      MZ st = warp_mz[tid][0];
+      for (int w = 1; w < SAMP_WARPS; ++w) st = mz_merge(st, warp_mz[tid][w], s);
+      mine[tid] = st;
     }
-    if (lane == 0) warp_mz[r][warp] = st;
-    __syncthreads();                              // every warp has finished reading this stage
-    if (tid == 0 && r + 2 < R) {
-      fence_proxy_async();                        // order the generic reads before the asynchronous overwrite
-      issue(st_i, row_ptr(r + 2));
+    cluster.sync();
+    if (tid < nslots) {
+      MZ st = *cluster.map_shared_rank(&mine[tid], 0);
+      for (int c = 1; c < SAMP_CLUSTER; ++c) st = mz_merge(st, *cluster.map_shared_rank(&mine[tid], c), s);
+      row_mz[tid] = MZ{-st.m * s, __frcp_rn(st.z)};
     }
-  }
-  __syncthreads();
-  if (tid < R) {
-    MZ st = warp_mz[tid][0];
-    for (int w = 1; w < SAMP_WARPS; ++w) st = mz_merge(st, warp_mz[tid][w], s);
-    local_mz[tid] = st;
-  }
-  cluster.sync();
-  if (tid < R) {
-    MZ st = *cluster.map_shared_rank(&local_mz[tid], 0);
-    for (int c = 1; c < SAMP_CLUSTER; ++c) st = mz_merge(st, *cluster.map_shared_rank(&local_mz[tid], c), s);
-    row_mz[tid] = MZ{-st.m * s, __frcp_rn(st.z)};               // (c, 1 / Z) of the row
-  }
-  __syncthreads();
+    __syncthreads();
+  };
 
-  // ---- optional dump of the probabilities the decisions use ------------------------------------------
+  // ---- optional dump of the probabilities (debug): every row through the same statistics code ---------------------
   if (A.dbg_p != nullptr || A.dbg_q != nullptr) {
     for (int r = 0; r < R; ++r) {
       float *dst = r <= K ? (A.dbg_p ? A.dbg_p + static_cast<size_t>(b) * A.tgt_bstride + static_cast<size_t>(r) * V : nullptr)
                           : (A.dbg_q ? A.dbg_q + static_cast<size_t>(b) * A.drf_bstride + static_cast<size_t>(r - K - 1) * V : nullptr);
-      if (dst == nullptr) continue;
-      const uint4 *row = row_ptr(r);
-      const MZ st = row_mz[r];
-      for (int i = tid; i < n; i += SAMP_THREADS) {
-        float x[8];
-        unpack8(__ldg(row + i), x);
+      if (tid == 0) { fence_proxy_async(); issue(0, row_ptr(r)); }
+      wait_stage(0);
+      slice_stats(stage[0], 0);
+      finish_stats(1);
+      const MZ st = row_mz[0];
+      if (dst != nullptr && alive)
+        for (int i = tid; i < n; i += SAMP_THREADS) {
+          float x[8];
+          unpack8(stage[0][i], x);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) dst[static_cast<size_t>(v_lo + i) * 8 + j] = prob_of(x[j], s, st.m, st.z);
-      }
+          for (int j = 0; j < 8; ++j) dst[static_cast<size_t>(v_lo + i) * 8 + j] = prob_of(x[j], s, st.m, st.z);
+        }
+      __syncthreads();
     }
   }
 
-  // ---- accept tests: lane k of warp 0 tests draft k (every CTA redundantly, identical inputs) ----------
-  if (warp == 0) {
-    bool ok = true;
-    if (lane < K) {
-      const int d = A.draft_tok[static_cast<size_t>(b) * A.tok_in_stride + lane];
+  // ---- positions in order: statistics of (p_k, q_k), accept test k; stop at the first rejection -----------------
+  // The rows of the position where the walk stops are then still in the ring: the resampling pass reads them from
+  // shared memory, and the rows of later positions are never loaded.
+  int a = K;
+  for (int k = 0; k <= K; ++k) {
+    const bool bonus = k == K;
+    if (tid == 0) {
+      fence_proxy_async();                        // order the generic reads of the stages before the asynchronous overwrite
+      issue(0, row_ptr(k));
+      if (!bonus) issue(1, row_ptr(K + 1 + k));
+    }
+    wait_stage(0);
+    if (!bonus) wait_stage(1);
+    slice_stats(stage[0], 0);
+    if (!bonus) slice_stats(stage[1], 1);
+    finish_stats(bonus ? 1 : 2);
+    if (bonus) break;
+    if (tid == 0) {                               // every CTA redundantly, identical inputs
+      bool ok = false;
+      const int d = A.draft_tok[static_cast<size_t>(b) * A.tok_in_stride + k];
       if (d < 0 || d >= V) {
         set_status(A.status, ST_BAD_TOKEN);
-        ok = false;
       } else {
-        const float xp = __bfloat162float(tgt[static_cast<size_t>(lane) * V + d]);
-        const float xq = __bfloat162float(drf[static_cast<size_t>(lane) * V + d]);
-        const float p = prob_of(xp, s, row_mz[lane].m, row_mz[lane].z);
-        const float q = prob_of(xq, s, row_mz[K + 1 + lane].m, row_mz[K + 1 + lane].z);
-        const uint32_t u24 = A.u24 ? A.u24[static_cast<size_t>(b) * A.u_stride + lane]
-                                   : philox_u24(A.seed, A.step, b, A.slot_accept + lane);
+        const float xp = __bfloat162float(tgt[static_cast<size_t>(k) * V + d]);
+        const float xq = __bfloat162float(drf[static_cast<size_t>(k) * V + d]);
+        const float p = prob_of(xp, s, row_mz[0].m, row_mz[0].z);
+        const float q = prob_of(xq, s, row_mz[1].m, row_mz[1].z);
+        const uint32_t u24 = A.u24 ? A.u24[static_cast<size_t>(b) * A.u_stride + k]
+                                   : philox_u24(A.seed, A.step, b, A.slot_accept + k);
         const float uq = __fmul_rn(__fmul_rn(static_cast<float>(u24), 5.9604644775390625e-8f /* 2^-24 */), q);
         ok = p >= q || uq < p;
       }
+      sh_a = ok ? 1 : 0;
     }
-    const unsigned rejected = __ballot_sync(0xffffffffu, !ok);   // lanes >= K vote "accepted"
-    if (lane == 0) sh_a = rejected ? __ffs(rejected) - 1 : K;    // first rejection, else all K accepted
+    __syncthreads();
+    if (!sh_a) { a = k; break; }
   }
-  __syncthreads();
-  const int a = sh_a;
 
-  // ---- pass 2: integer weights of position a+1 and the draw -----------------------------------------
-  const uint4 *prow = row_ptr(a);
-  const uint4 *qrow = a < K ? row_ptr(K + 1 + a) : nullptr;
-  const MZ ps = row_mz[a];
-  const MZ qs = a < K ? row_mz[K + 1 + a] : MZ{0.f, 1.f};
+  // ---- resampling at position a+1 from the rows in the ring: integer weights and the draw -------------------------
+  const MZ ps = row_mz[0];
+  const MZ qs = a < K ? row_mz[1] : MZ{0.f, 1.f};
   bool use_q = a < K;
   unsigned long long Wc[SAMP_CLUSTER];
   unsigned long long W = 0;
-  // both rows of position a+1 come back through the ring (they are L2-resident)
-  if (tid == 0) {
-    fence_proxy_async();
-    issue(0, prow);
-    if (use_q) issue(1, qrow);
-  }
-  wait_stage(0);
-  if (use_q) wait_stage(1);
   for (int attempt = 0; attempt < 2; ++attempt) {
     unsigned long long tsum = 0;
     for (int i = tid; i < n && alive; i += SAMP_THREADS) {
@@ -292,7 +292,7 @@ sampler_kernel(const SamplerArgs A) {
     __syncthreads();
     for (int i = tid; i < n; i += SAMP_THREADS) {
       float x[8];
-      unpack8(__ldg(prow + i), x);
+      unpack8(stage[0][i], x);
 #pragma unroll
       for (int j = 0; j < 8; ++j)
         if (-x[j] * s == ps.m) atomicMin(&local_cand, (v_lo + i) * 8 + j);
@@ -329,8 +329,8 @@ sampler_kernel(const SamplerArgs A) {
       int iv = lo;
       while (rem >= vecsum[iv]) { rem -= vecsum[iv]; ++iv; }     // stops inside [lo, hi): rem < mine
       float xp[8], xq[8];
-      unpack8(__ldg(prow + iv), xp);
-      if (use_q) unpack8(__ldg(qrow + iv), xq);
+      unpack8(stage[0][iv], xp);
+      if (use_q) unpack8(stage[1][iv], xq);
       int tok = (v_lo + iv) * 8 + 7;
       for (int j = 0; j < 8; ++j) {
         const unsigned long long w =
