@@ -58,6 +58,8 @@ extern "C" {
 
 /* gm_config.flags */
 #define GM_FLAG_SIMPLE_GEMM 1       /* debug: route every GEMM through the plain mma.sync kernel */
+#define GM_FLAG_SAMPLER_CLUSTER 2   /* always map the sampler as one 8-CTA cluster per sequence  */
+#define GM_FLAG_SAMPLER_STREAM 4    /* always map the sampler as one CTA per sequence            */
 
 typedef struct gm_ctx gm_ctx;       /* opaque */
 

@@ -308,6 +308,16 @@ int check_state(const gm_ctx *c, const gm_state *st, int k) {
   return GM_OK;
 }
 
+// Mapping of the sampler: a cluster per sequence while sequences are few, one CTA per sequence once there are enough
+// of them to fill the SMs (the flags force one or the other).
+cudaError_t run_sampler(gm_ctx *c, const SamplerArgs &S, int batch) {
+  bool stream_variant = batch * 3 >= c->sm_count * 2;
+  if (c->cfg.flags & GM_FLAG_SAMPLER_CLUSTER) stream_variant = false;
+  if (c->cfg.flags & GM_FLAG_SAMPLER_STREAM) stream_variant = true;
+  if (stream_variant && sampler_stream_supported(S.V)) return launch_sampler_stream(S, batch, c->stream);
+  return launch_sampler(S, batch, c->stream);
+}
+
 int fill_sampler(gm_ctx *c, SamplerArgs &S, float temperature) {
   if (!(temperature > 0.f) || !std::isfinite(temperature)) return GM_ERR_UNSUPPORTED;
   std::memset(&S, 0, sizeof(S));
@@ -509,7 +519,7 @@ int gm_draft(gm_ctx *c, const gm_state *st, int k, float temperature, const uint
     S.seed = seed; S.step = step; S.slot_final = SLOT_DRAFT + (j - 1);
     S.accept_len = nullptr; S.next_token = draft_tok + (j - 1); S.tok_out_stride = k;
     S.dbg_p = dbg_q ? dbg_q + static_cast<size_t>(j - 1) * c->V : nullptr; S.dbg_q = nullptr; S.commit = 0;
-    GM_LAUNCH(c, GM_KC_SAMPLER, launch_sampler(S, ph.B, c->stream));
+    GM_LAUNCH(c, GM_KC_SAMPLER, run_sampler(c, S, ph.B));
   }
   return GM_OK;
 }
@@ -568,7 +578,7 @@ int gm_accept(gm_ctx *c, gm_state *st, int batch, int k, float temperature, cons
     S.target_hidden = static_cast<const __nv_bfloat16 *>(target_hidden);
     S.d_model = c->d; S.max_k = c->cfg.max_k;
   }
-  GM_LAUNCH(c, GM_KC_SAMPLER, launch_sampler(S, batch, c->stream));
+  GM_LAUNCH(c, GM_KC_SAMPLER, run_sampler(c, S, batch));
   return GM_OK;
 }
 
@@ -580,7 +590,7 @@ int gm_draw(gm_ctx *c, const void *logits, int rows, float temperature, const ui
   if (rc) return rc;
   S.K = 0; S.target_logits = static_cast<const __nv_bfloat16 *>(logits); S.tgt_bstride = c->V; S.u24 = u24; S.u_stride = 1;
   S.next_token = out_tok; S.tok_out_stride = 1; S.dbg_p = dbg_prob;
-  GM_LAUNCH(c, GM_KC_SAMPLER, launch_sampler(S, rows, c->stream));
+  GM_LAUNCH(c, GM_KC_SAMPLER, run_sampler(c, S, rows));
   return GM_OK;
 }
 

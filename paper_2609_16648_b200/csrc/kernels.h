@@ -64,7 +64,9 @@ struct SamplerArgs {
   int d_model, max_k;
   uint32_t *status;
 };
-cudaError_t launch_sampler(const SamplerArgs &A, int batch, cudaStream_t stream);
+cudaError_t launch_sampler(const SamplerArgs &A, int batch, cudaStream_t stream);          // cluster of 8 CTAs per sequence
+cudaError_t launch_sampler_stream(const SamplerArgs &A, int batch, cudaStream_t stream);   // one CTA per sequence
+bool sampler_stream_supported(int V);
 
 // ---- cycle record (top-64 target log-probabilities and the other recorded items) ---------------------------------
 struct RecordTopkArgs {

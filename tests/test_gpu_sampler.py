@@ -10,12 +10,22 @@ from synth_inputs.workload import random_u24
 pytestmark = pytest.mark.gpu
 
 
+MAPPING = {"flags": 0}
+
+
+@pytest.fixture(autouse=True, params=[2, 4], ids=["cluster_per_sequence", "cta_per_sequence"])
+def _mapping(request):
+    """Every test of this file runs with both mappings of the sampler kernel."""
+    MAPPING["flags"] = request.param
+    yield
+
+
 def _ctx(vocab, max_batch=256, max_k=7):
     import paper_2609_16648_b200 as gmb
     cfg = ModelConfig("s", 1, 64, 1, 1, 64, 64, vocab, batch=max_batch, k=max_k, kv_len_min=0, kv_len_max=0,
                       length_law="uniform")
     packed = gmb.random_packed_weights(cfg, "cuda")      # the sampler itself reads no weights
-    return gmb, gmb.Context(cfg, packed, max_batch, max_k, 4, 8, 8)
+    return gmb, gmb.Context(cfg, packed, max_batch, max_k, 4, 8, 8, flags=MAPPING["flags"])
 
 
 def _bf16(x):
