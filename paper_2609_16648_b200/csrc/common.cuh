@@ -91,7 +91,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, uint32
   return false;
 }
 
-// ---- TMA (tensor-map copies, no multicast anywhere) ---------------------------------------------------
+// ---- TMA (tensor-map copies; every CTA fetches its own tiles) ------------------------------------------
 __device__ __forceinline__ void tma_load_2d(void *smem_dst, const void *tmap, int x, int y, uint64_t *bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"

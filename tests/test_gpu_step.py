@@ -227,3 +227,51 @@ def test_device_seen_errors_and_host_validation():
     assert gmb.gm_last_status(ctx2) == gmb.GM_ERR_BAD_PAGE
     ctx.close()
     ctx2.close()
+
+
+def test_rerun_is_bit_identical_and_resume_equals_uninterrupted():
+    """Counter-based uniforms and fixed-order reductions: the same state and (seed, step) give bit-identical
+    tokens and state on a second run, and a rollout that is stopped, copied to the host, restored into fresh
+    buffers and continued equals the uninterrupted one."""
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny").with_(prompt_len=25)
+    K, B = cfg.k, cfg.batch
+    w, ost, ctx, gst = tiny_setup(cfg, cap_tokens=200)
+    push_state(ost, gst, ctx)
+    names = ("kv_len", "pending_n", "pending_tok", "pending_hidden", "kv_pool", "head_kv_pool")
+    snap = {n: getattr(gst, n).clone() for n in names}
+    a = torch.zeros(B, dtype=torch.int32, device="cuda")
+    t = torch.zeros(B, dtype=torch.int32, device="cuda")
+    d = torch.zeros((B, K), dtype=torch.int32, device="cuda")
+
+    def rollout(state, first, n):
+        out = []
+        for it in range(first, first + n):
+            gmb.gm_spec_step(ctx, state, K, 1.0, 21, it, a, t, d)
+            out.append((a.cpu().clone(), t.cpu().clone(), d.cpu().clone()))
+        return out
+
+    ref = rollout(gst, 0, 12)
+    end = {n: getattr(gst, n).clone() for n in names}
+    for n, v in snap.items():
+        getattr(gst, n).copy_(v)
+    again = rollout(gst, 0, 12)
+    for x, y in zip(ref, again):
+        assert all(torch.equal(p, q) for p, q in zip(x, y))
+    for n in names:
+        assert torch.equal(getattr(gst, n), end[n]), n
+    # stop after 5 steps, checkpoint to the host, restore into a new state object, continue
+    for n, v in snap.items():
+        getattr(gst, n).copy_(v)
+    first = rollout(gst, 0, 5)
+    ckpt = {n: getattr(gst, n).cpu() for n in names}
+    gst2 = gmb.State(ctx, B, gst.page_table.cpu().numpy(), gst.head_page_table.cpu().numpy())
+    for n, v in ckpt.items():
+        getattr(gst2, n).copy_(v)
+    rest = rollout(gst2, 5, 7)
+    for x, y in zip(ref, first + rest):
+        assert all(torch.equal(p, q) for p, q in zip(x, y))
+    for n in names:
+        assert torch.equal(getattr(gst2, n), end[n]), n
+    assert gmb.gm_last_status(ctx) == 0
+    ctx.close()
