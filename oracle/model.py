@@ -1,7 +1,11 @@
 """Dense decoder blocks, paged KV cache and the recurrent MTP draft head, in fp64.
 
 Target model: a generic pre-norm decoder (RMSNorm, rotary positions, grouped-query
-attention, SwiGLU feed-forward, no biases).  Draft head (App. B.1, "MTP
+attention, SwiGLU feed-forward).  The decoder-layer families the paper names (App. B.1)
+differ in the attention projections only: one adds a bias to the query/key/value
+projections (keys "bq", "bk", "bv" of a layer), one normalises every query and key head
+with an RMSNorm over the head dimension before the rotary embedding (keys "qnorm",
+"knorm").  A layer without those keys has neither.  Draft head (App. B.1, "MTP
 Architecture"): ONE such decoder layer.  For each position it drafts, it consumes the
 hidden state and the token embedding of the position before it: the two are
 normalised by separate RMSNorms, concatenated, projected back to the model width by a
@@ -116,6 +120,27 @@ class PagedKV:
 
 # ---- decoder layer, target forward, draft head ----------------------------------------------
 
+def project_qkv(lw, h, cfg):
+    """Query/key/value heads of normalised rows h [T, d], before the rotary embedding.
+
+    q [T, n_q, hd], k and v [T, n_kv, hd].  Optional per-family steps (App. B.1): a bias
+    on each projection; an RMSNorm over the head dimension on every query and key head.
+    """
+    T = h.shape[0]
+    q = h @ f64(lw["wq"]).T
+    k = h @ f64(lw["wk"]).T
+    v = h @ f64(lw["wv"]).T
+    if "bq" in lw:
+        q, k, v = q + f64(lw["bq"]), k + f64(lw["bk"]), v + f64(lw["bv"])
+    q = q.reshape(T, cfg.n_q_heads, cfg.head_dim)
+    k = k.reshape(T, cfg.n_kv_heads, cfg.head_dim)
+    v = v.reshape(T, cfg.n_kv_heads, cfg.head_dim)
+    if "qnorm" in lw:
+        q = rmsnorm(q, lw["qnorm"], cfg.rms_eps)
+        k = rmsnorm(k, lw["knorm"], cfg.rms_eps)
+    return q, k, v
+
+
 def decoder_layer(lw, x, pos, kv: PagedKV, layer: int, b: int, cfg) -> np.ndarray:
     """One pre-norm decoder layer over new rows x [T, d] at positions pos, against the cache.
 
@@ -126,9 +151,7 @@ def decoder_layer(lw, x, pos, kv: PagedKV, layer: int, b: int, cfg) -> np.ndarra
     T = x.shape[0]
     pos = np.asarray(pos)
     h = rmsnorm(x, lw["ln1"], cfg.rms_eps)
-    q = (h @ f64(lw["wq"]).T).reshape(T, cfg.n_q_heads, cfg.head_dim)
-    k = (h @ f64(lw["wk"]).T).reshape(T, cfg.n_kv_heads, cfg.head_dim)
-    v = (h @ f64(lw["wv"]).T).reshape(T, cfg.n_kv_heads, cfg.head_dim)
+    q, k, v = project_qkv(lw, h, cfg)
     q = rope(q, pos, cfg.rope_base)
     k = rope(k, pos, cfg.rope_base)
     kv.write(layer, b, pos, k, v)
@@ -157,11 +180,17 @@ def target_logits(w, hidden, cfg) -> np.ndarray:
 
 def head_forward(w, hidden, tokens, pos, hkv: PagedKV, b: int, cfg) -> np.ndarray:
     """Draft head over pairs (hidden_i, token_i) at positions pos; returns g [T, d], the
-    head layer's residual output (its recurrent state)."""
+    head layer's residual output (its recurrent state).
+
+    The two normalised inputs are concatenated [embedding ; hidden]; a head whose
+    "concat" entry is "hidden_first" takes them in the opposite order (App. B.1: one
+    family's native head does)."""
     hw = w["head"]
     e = f64(w["embed"])[np.asarray(tokens)]
-    z = np.concatenate([rmsnorm(e, hw["enorm"], cfg.rms_eps),
-                        rmsnorm(hidden, hw["hnorm"], cfg.rms_eps)], axis=-1)
+    parts = [rmsnorm(e, hw["enorm"], cfg.rms_eps), rmsnorm(hidden, hw["hnorm"], cfg.rms_eps)]
+    if hw.get("concat", "embedding_first") == "hidden_first":
+        parts.reverse()
+    z = np.concatenate(parts, axis=-1)
     z = z @ f64(hw["proj"]).T
     return decoder_layer(hw["layer"], z, pos, hkv, 0, b, cfg)
 

@@ -33,6 +33,8 @@ class ModelConfig:
     temperature: float = 1.0
     init_std: float = 0.02      # standard deviation of every linear / embedding weight
     prompt_len: int = 0         # Tiny only: prompts are prefetched by a real prefill
+    qkv_bias: bool = False      # decoder-layer family with a bias on the q/k/v projections
+    qk_norm: bool = False       # decoder-layer family with an RMSNorm on every query and key head
 
     @property
     def q_dim(self) -> int:

@@ -29,7 +29,7 @@ def _normal(rng: np.random.Generator, shape, std: float) -> np.ndarray:
 def _layer(rng: np.random.Generator, cfg: ModelConfig) -> dict:
     d, f = cfg.d_model, cfg.d_ffn
     s = cfg.init_std
-    return {
+    lw = {
         "ln1": np.ones(d, np.float32),
         "wq": _normal(rng, (cfg.q_dim, d), s),
         "wk": _normal(rng, (cfg.kv_dim, d), s),
@@ -40,6 +40,16 @@ def _layer(rng: np.random.Generator, cfg: ModelConfig) -> dict:
         "wu": _normal(rng, (f, d), s),
         "wd": _normal(rng, (d, f), s),
     }
+    # family extras; the biases are drawn four times wider than the weights so that a consumer
+    # that drops them is far outside any parity tolerance
+    if cfg.qkv_bias:
+        lw["bq"] = _normal(rng, (cfg.q_dim,), 4 * s)
+        lw["bk"] = _normal(rng, (cfg.kv_dim,), 4 * s)
+        lw["bv"] = _normal(rng, (cfg.kv_dim,), 4 * s)
+    if cfg.qk_norm:
+        lw["qnorm"] = np.ones(cfg.head_dim, np.float32)
+        lw["knorm"] = np.ones(cfg.head_dim, np.float32)
+    return lw
 
 
 def make_weights(cfg: ModelConfig, seed: int = 0, n_layers: int | None = None) -> dict:
@@ -82,6 +92,9 @@ def perturb_norm_weights(w: dict, seed: int = 123, spread: float = 0.25) -> dict
     for lw in w["layers"] + [w["head"]["layer"]]:
         lw["ln1"] = pert(lw["ln1"])
         lw["ln2"] = pert(lw["ln2"])
+        for name in ("qnorm", "knorm"):
+            if name in lw:
+                lw[name] = pert(lw[name])
     for name in ("enorm", "hnorm", "final_norm"):
         w["head"][name] = pert(w["head"][name])
     return w

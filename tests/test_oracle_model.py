@@ -1,4 +1,5 @@
 """Pins for the oracle's decoder blocks: closed forms, library routines, brute force, invariants."""
+import dataclasses
 import math
 
 import numpy as np
@@ -172,9 +173,13 @@ def _torch_layer(lw, x, cfg):
     t = lambda a: torch.from_numpy(np.asarray(a, np.float64))
     T = x.shape[0]
     h = F.rms_norm(t(x), (cfg.d_model,), t(lw["ln1"]), eps=cfg.rms_eps)
-    q = (h @ t(lw["wq"]).T).view(T, cfg.n_q_heads, cfg.head_dim)
-    k = (h @ t(lw["wk"]).T).view(T, cfg.n_kv_heads, cfg.head_dim)
-    v = (h @ t(lw["wv"]).T).view(T, cfg.n_kv_heads, cfg.head_dim)
+    bias = lambda n: t(lw[n]) if n in lw else None
+    q = F.linear(h, t(lw["wq"]), bias("bq")).view(T, cfg.n_q_heads, cfg.head_dim)
+    k = F.linear(h, t(lw["wk"]), bias("bk")).view(T, cfg.n_kv_heads, cfg.head_dim)
+    v = F.linear(h, t(lw["wv"]), bias("bv")).view(T, cfg.n_kv_heads, cfg.head_dim)
+    if "qnorm" in lw:
+        q = F.rms_norm(q, (cfg.head_dim,), t(lw["qnorm"]), eps=cfg.rms_eps)
+        k = F.rms_norm(k, (cfg.head_dim,), t(lw["knorm"]), eps=cfg.rms_eps)
     half = cfg.head_dim // 2
     ang = torch.arange(T, dtype=torch.float64)[:, None] * cfg.rope_base ** (
         -torch.arange(half, dtype=torch.float64) * 2 / cfg.head_dim)
@@ -226,3 +231,77 @@ def test_head_forward_structure():
     assert lg.shape == (5, CFG.vocab)
     np.testing.assert_allclose(lg, model.rmsnorm(g, w["head"]["final_norm"], CFG.rms_eps)
                                @ w["lm_head"].astype(np.float64).T, rtol=1e-12)
+
+
+# ---- decoder-layer families and the head's concatenation order (App. B.1) ---------------------------
+
+@pytest.mark.parametrize("bias,qkn", [(True, False), (False, True), (True, True)])
+def test_family_layers_against_library_composition(bias, qkn):
+    cfg = dataclasses.replace(CFG, qkv_bias=bias, qk_norm=qkn)
+    w = _weights(cfg)
+    lw = w["layers"][1]
+    assert ("bq" in lw) == bias and ("qnorm" in lw) == qkn
+    rng = np.random.default_rng(17)
+    x = rng.normal(size=(11, cfg.d_model))
+    out = model.decoder_layer(lw, x, np.arange(11), _kv(cfg, cfg.n_layers, 64), 1, 0, cfg)
+    np.testing.assert_allclose(out, _torch_layer(lw, x, cfg), rtol=1e-9, atol=1e-11)
+    # and the extras matter: dropping them changes the output
+    plain = {k: v for k, v in lw.items() if k not in ("bq", "bk", "bv", "qnorm", "knorm")}
+    out0 = model.decoder_layer(plain, x, np.arange(11), _kv(cfg, cfg.n_layers, 64), 1, 0, cfg)
+    assert np.abs(out0 - out).max() > 1e-3
+
+
+def test_projection_bias_is_an_extra_input_column():
+    """h W^T + b == [h, 1] [W, b]^T; a zero bias changes nothing."""
+    cfg = dataclasses.replace(CFG, qkv_bias=True)
+    lw = _weights(cfg)["layers"][0]
+    rng = np.random.default_rng(18)
+    h = rng.normal(size=(7, cfg.d_model))
+    q, k, v = model.project_qkv(lw, h, cfg)
+    h1 = np.concatenate([h, np.ones((7, 1))], 1)
+    for got, wn, bn in ((q, "wq", "bq"), (k, "wk", "bk"), (v, "wv", "bv")):
+        aug = np.concatenate([lw[wn].astype(np.float64), lw[bn].astype(np.float64)[:, None]], 1)
+        np.testing.assert_allclose(got.reshape(7, -1), h1 @ aug.T, rtol=1e-12, atol=1e-14)
+    zero = dict(lw, bq=np.zeros_like(lw["bq"]), bk=np.zeros_like(lw["bk"]), bv=np.zeros_like(lw["bv"]))
+    plain = {k_: v_ for k_, v_ in lw.items() if k_ not in ("bq", "bk", "bv")}
+    for a, b in zip(model.project_qkv(zero, h, cfg), model.project_qkv(plain, h, cfg)):
+        np.testing.assert_array_equal(a, b)
+
+
+def test_query_key_norm_properties():
+    """With unit weights every query and key head has mean square 1 (up to eps), whatever the scale of
+    the projection; values are not normalised; the weight multiplies element-wise after the division."""
+    cfg = dataclasses.replace(CFG, qk_norm=True)
+    lw = make_weights(cfg, seed=3)["layers"][0]            # norm weights are one
+    rng = np.random.default_rng(19)
+    h = rng.normal(size=(9, cfg.d_model))
+    q, k, v = model.project_qkv(lw, h, cfg)
+    np.testing.assert_allclose((q * q).mean(-1), 1.0, rtol=1e-3)
+    np.testing.assert_allclose((k * k).mean(-1), 1.0, rtol=1e-3)
+    assert abs((v * v).mean() - 1.0) > 0.1
+    big = dict(lw, wq=lw["wq"] * 8.0, wv=lw["wv"] * 8.0)
+    q8, k8, v8 = model.project_qkv(big, h, cfg)
+    np.testing.assert_allclose(q8, q, rtol=1e-3, atol=1e-6)
+    np.testing.assert_allclose(v8, 8.0 * v, rtol=1e-12)
+    g = rng.uniform(0.5, 1.5, cfg.head_dim)
+    qg, _, _ = model.project_qkv(dict(lw, qnorm=g), h, cfg)
+    np.testing.assert_allclose(qg, q * g, rtol=1e-12)
+    # the norm comes before the rotary embedding: rotating afterwards keeps the head's mean square
+    qr = model.rope(q, np.arange(9), cfg.rope_base)
+    np.testing.assert_allclose((qr * qr).mean(-1), 1.0, rtol=1e-3)
+
+
+def test_opposite_concatenation_order_is_a_swap_of_the_projection_halves():
+    w = _weights(CFG)
+    rng = np.random.default_rng(20)
+    hid = rng.normal(size=(5, CFG.d_model))
+    toks = rng.integers(0, CFG.vocab, 5)
+    g = model.head_forward(w, hid, toks, np.arange(5), _kv(CFG, 1, 64), 0, CFG)
+    d = CFG.d_model
+    proj = w["head"]["proj"]
+    w2 = dict(w, head=dict(w["head"], concat="hidden_first", proj=np.concatenate([proj[:, d:], proj[:, :d]], 1)))
+    g2 = model.head_forward(w2, hid, toks, np.arange(5), _kv(CFG, 1, 64), 0, CFG)
+    np.testing.assert_allclose(g2, g, rtol=1e-10, atol=1e-12)
+    w3 = dict(w, head=dict(w["head"], concat="hidden_first"))      # same matrix, other order: a different function
+    g3 = model.head_forward(w3, hid, toks, np.arange(5), _kv(CFG, 1, 64), 0, CFG)
+    assert np.abs(g3 - g).max() > 1e-3
