@@ -77,7 +77,11 @@ typedef struct {
 } gm_config;
 
 /* One decoder layer.  wqkv rows: all query heads, then all key heads, then all value heads.
- * w_gate_up rows are interleaved: row 2i = gate_i, row 2i+1 = up_i.                       */
+ * w_gate_up rows are interleaved: row 2i = gate_i, row 2i+1 = up_i.
+ * The last three members select the decoder-layer family (App. B.1) and may each be NULL:
+ * b_qkv is a bias added to the fused projection (same row order as wqkv); q_norm / k_norm are
+ * the weights of an RMSNorm over head_dim applied to every query / key head after the bias and
+ * before the rotary embedding (both or neither).                                           */
 typedef struct {
   const void *ln1;                  /* [d]                                  */
   const void *wqkv;                 /* [(n_q + 2 n_kv) head_dim, d]         */
@@ -85,11 +89,16 @@ typedef struct {
   const void *ln2;                  /* [d]                                  */
   const void *w_gate_up;            /* [2 d_ffn, d]                         */
   const void *w_down;               /* [d, d_ffn]                           */
+  const void *b_qkv;                /* [(n_q + 2 n_kv) head_dim] or NULL    */
+  const void *q_norm;               /* [head_dim] or NULL                   */
+  const void *k_norm;               /* [head_dim] or NULL                   */
 } gm_layer_weights;
 
 /* Model weights (App. B.1: the head has neither embedding nor output projection and takes
  * both from the backbone; its two inputs go through separate RMSNorms, are concatenated
- * [embedding ; hidden] and projected by a bias-free linear layer).                       */
+ * [embedding ; hidden] and projected by a bias-free linear layer).  A head trained with the
+ * opposite order [hidden ; embedding] is loaded by swapping the two column halves of
+ * head_proj, as the paper's own loader does.                                              */
 typedef struct {
   const void *embed;                /* [vocab, d]                           */
   const void *lm_head;              /* [vocab, d]                           */

@@ -36,7 +36,7 @@ class gm_config(C.Structure):
 
 
 class gm_layer_weights(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("ln1", "wqkv", "wo", "ln2", "w_gate_up", "w_down")]
+    _fields_ = [(n, C.c_void_p) for n in ("ln1", "wqkv", "wo", "ln2", "w_gate_up", "w_down", "b_qkv", "q_norm", "k_norm")]
 
 
 class gm_weights(C.Structure):
@@ -122,10 +122,17 @@ def _p(t):
 
 def pack_layer(lw: dict, device) -> dict:
     """Canonical per-projection matrices -> the library's fused layout (bf16 on `device`):
-    wqkv = [wq; wk; wv] stacked by rows, w_gate_up rows interleaved (2i = gate_i, 2i+1 = up_i)."""
+    wqkv = [wq; wk; wv] stacked by rows, w_gate_up rows interleaved (2i = gate_i, 2i+1 = up_i).
+    Family extras when present: b_qkv = [bq; bk; bv], q_norm, k_norm."""
     bf = lambda a: torch.as_tensor(a).to(device=device, dtype=torch.bfloat16).contiguous()
     wg, wu = torch.as_tensor(lw["wg"]), torch.as_tensor(lw["wu"])
+    extra = {}
+    if "bq" in lw:
+        extra["b_qkv"] = bf(torch.cat([torch.as_tensor(lw[n]) for n in ("bq", "bk", "bv")], 0))
+    if "qnorm" in lw:
+        extra["q_norm"], extra["k_norm"] = bf(lw["qnorm"]), bf(lw["knorm"])
     return {
+        **extra,
         "ln1": bf(lw["ln1"]), "ln2": bf(lw["ln2"]),
         "wqkv": bf(torch.cat([torch.as_tensor(lw["wq"]), torch.as_tensor(lw["wk"]), torch.as_tensor(lw["wv"])], 0)),
         "wo": bf(lw["wo"]),
@@ -135,7 +142,15 @@ def pack_layer(lw: dict, device) -> dict:
 
 
 def pack_weights(w: dict, device="cuda") -> dict:
+    """Canonical weights -> the library's layout.  A head whose "concat" entry is "hidden_first" was
+    trained on [hidden ; embedding]: the two column halves of its projection are swapped here, so the
+    library's fixed order [embedding ; hidden] computes the same function (App. B.1)."""
     bf = lambda a: torch.as_tensor(a).to(device=device, dtype=torch.bfloat16).contiguous()
+    proj = torch.as_tensor(w["head"]["proj"])
+    if w["head"].get("concat", "embedding_first") == "hidden_first":
+        d = proj.shape[0]
+        proj = torch.cat([proj[:, d:], proj[:, :d]], 1)
+    w = dict(w, head=dict(w["head"], proj=proj))
     return {
         "embed": bf(w["embed"]), "lm_head": bf(w["lm_head"]), "final_norm": bf(w["final_norm"]),
         "layers": [pack_layer(lw, device) for lw in w["layers"]],
@@ -161,8 +176,13 @@ def random_packed_weights(cfg, device="cuda", seed=0, std=0.02) -> dict:
     d, f = cfg.d_model, cfg.d_ffn
 
     def layer():
-        return {"ln1": ones(d), "ln2": ones(d), "wqkv": rnd(cfg.q_dim + 2 * cfg.kv_dim, d), "wo": rnd(d, cfg.q_dim),
-                "w_gate_up": rnd(2 * f, d), "w_down": rnd(d, f)}
+        lw = {"ln1": ones(d), "ln2": ones(d), "wqkv": rnd(cfg.q_dim + 2 * cfg.kv_dim, d), "wo": rnd(d, cfg.q_dim),
+              "w_gate_up": rnd(2 * f, d), "w_down": rnd(d, f)}
+        if getattr(cfg, "qkv_bias", False):
+            lw["b_qkv"] = rnd(cfg.q_dim + 2 * cfg.kv_dim, 1).reshape(-1)
+        if getattr(cfg, "qk_norm", False):
+            lw["q_norm"], lw["k_norm"] = ones(cfg.head_dim), ones(cfg.head_dim)
+        return lw
 
     return {"embed": rnd(cfg.vocab, d), "lm_head": rnd(cfg.vocab, d), "final_norm": ones(d),
             "layers": [layer() for _ in range(cfg.n_layers)],
@@ -171,7 +191,8 @@ def random_packed_weights(cfg, device="cuda", seed=0, std=0.02) -> dict:
 
 
 def _layer_struct(lw: dict) -> gm_layer_weights:
-    return gm_layer_weights(*[lw[n].data_ptr() for n in ("ln1", "wqkv", "wo", "ln2", "w_gate_up", "w_down")])
+    opt = [lw[n].data_ptr() if n in lw else None for n in ("b_qkv", "q_norm", "k_norm")]
+    return gm_layer_weights(*[lw[n].data_ptr() for n in ("ln1", "wqkv", "wo", "ln2", "w_gate_up", "w_down")], *opt)
 
 
 class Context:

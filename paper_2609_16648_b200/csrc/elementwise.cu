@@ -225,12 +225,35 @@ __global__ void __launch_bounds__(EW_THREADS) rope_append_kernel(const RopeAppen
   __nv_bfloat16 *vdst = A.pool + ((static_cast<size_t>(A.layer) * 2 + 1) * A.num_pages + (page_ok ? page : 0)) * page_elems;
   const int slot = pos & 15;
   const int n_rot = (A.n_q + A.n_kv) * hv, n_v = A.n_kv * (hd >> 3);
+  // the hv lanes that share one head are consecutive and aligned (hv is a power of two <= 32)
+  const unsigned lane = threadIdx.x & 31u;
+  const unsigned head_lanes = hv >= 32 ? 0xffffffffu : ((1u << hv) - 1u) << (lane & ~static_cast<unsigned>(hv - 1));
   for (int i = threadIdx.x; i < n_rot + n_v; i += EW_THREADS) {
     if (i < n_rot) {
       const int h = i / hv, e = (i % hv) * 8;
       float x1[8], x2[8], y1[8], y2[8];
       unpack8f(*reinterpret_cast<const uint4 *>(src + h * hd + e), x1);
       unpack8f(*reinterpret_cast<const uint4 *>(src + h * hd + e + half), x2);
+      if (A.bias) {
+        float b1[8], b2[8];
+        unpack8f(*reinterpret_cast<const uint4 *>(A.bias + h * hd + e), b1);
+        unpack8f(*reinterpret_cast<const uint4 *>(A.bias + h * hd + e + half), b2);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) { x1[t] += b1[t]; x2[t] += b2[t]; }
+      }
+      const __nv_bfloat16 *nw = h < A.n_q ? A.qnorm : A.knorm;
+      if (nw) {                                       // RMSNorm over the head dimension, before the rotation
+        float ss = 0.f;
+#pragma unroll
+        for (int t = 0; t < 8; ++t) ss += x1[t] * x1[t] + x2[t] * x2[t];
+        for (int off = hv >> 1; off >= 1; off >>= 1) ss += __shfl_xor_sync(head_lanes, ss, off);
+        const float inv = rsqrtf(ss / static_cast<float>(hd) + A.eps);
+        float w1[8], w2[8];
+        unpack8f(*reinterpret_cast<const uint4 *>(nw + e), w1);
+        unpack8f(*reinterpret_cast<const uint4 *>(nw + e + half), w2);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) { x1[t] = x1[t] * inv * w1[t]; x2[t] = x2[t] * inv * w2[t]; }
+      }
 #pragma unroll
       for (int t = 0; t < 8; ++t) {
         const float2 c = cs[e + t];
@@ -245,8 +268,16 @@ __global__ void __launch_bounds__(EW_THREADS) rope_append_kernel(const RopeAppen
       *reinterpret_cast<uint4 *>(dst + e + half) = pack8f(y2);
     } else if (page_ok) {
       const int iv = i - n_rot, h = iv / (hd >> 3), e = (iv % (hd >> 3)) * 8;
-      *reinterpret_cast<uint4 *>(vdst + (static_cast<size_t>(h) * 16 + slot) * hd + e) =
-          *reinterpret_cast<const uint4 *>(src + (A.n_q + A.n_kv) * hd + h * hd + e);
+      uint4 val = *reinterpret_cast<const uint4 *>(src + (A.n_q + A.n_kv) * hd + h * hd + e);
+      if (A.bias) {
+        float x[8], bv[8];
+        unpack8f(val, x);
+        unpack8f(*reinterpret_cast<const uint4 *>(A.bias + (A.n_q + A.n_kv) * hd + h * hd + e), bv);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) x[t] += bv[t];
+        val = pack8f(x);
+      }
+      *reinterpret_cast<uint4 *>(vdst + (static_cast<size_t>(h) * 16 + slot) * hd + e) = val;
     }
   }
 }

@@ -254,6 +254,9 @@ int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const 
   R.num_pages = num_pages; R.max_pages_per_seq = cf.max_pages_per_seq; R.qrows = ph.qrows;
   R.qn = c->qn; R.qbase = c->qbase; R.page_table = page_table; R.rope = c->rope; R.qbuf = c->qbuf; R.pool = pool;
   R.status = c->status;
+  R.bias = static_cast<const __nv_bfloat16 *>(lw.b_qkv);
+  R.qnorm = static_cast<const __nv_bfloat16 *>(lw.q_norm); R.knorm = static_cast<const __nv_bfloat16 *>(lw.k_norm);
+  R.eps = cf.rms_eps;
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rope_append(R, c->stream));
   // attention over the pages + merge of the segments
   AttnArgs T;
@@ -392,11 +395,13 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
   }
   for (int l = 0; l < cfg->n_layers; ++l) {
     const gm_layer_weights &lw = c->layers[l];
-    if (!lw.ln1 || !lw.wqkv || !lw.wo || !lw.ln2 || !lw.w_gate_up || !lw.w_down) return fail(GM_ERR_INVALID_ARG);
+    if (!lw.ln1 || !lw.wqkv || !lw.wo || !lw.ln2 || !lw.w_gate_up || !lw.w_down || !lw.q_norm != !lw.k_norm)
+      return fail(GM_ERR_INVALID_ARG);
   }
   {
     const gm_layer_weights &lw = w->head_layer;
-    if (!lw.ln1 || !lw.wqkv || !lw.wo || !lw.ln2 || !lw.w_gate_up || !lw.w_down) return fail(GM_ERR_INVALID_ARG);
+    if (!lw.ln1 || !lw.wqkv || !lw.wo || !lw.ln2 || !lw.w_gate_up || !lw.w_down || !lw.q_norm != !lw.k_norm)
+      return fail(GM_ERR_INVALID_ARG);
   }
   auto layer_maps = [&](const gm_layer_weights &lw, LayerMaps &lm) {
     int rc = make_map(c, &lm.wqkv, lw.wqkv, c->n_qkv, c->d, 128);

@@ -126,6 +126,9 @@ struct RopeAppendArgs {
   int batch, QT, n_q, n_kv, hd, layer, num_pages, max_pages_per_seq, qrows;
   const int32_t *qn, *qbase, *page_table;
   const float2 *rope;                                   // [max_pos][hd/2] (cos, sin)
+  const __nv_bfloat16 *bias = nullptr;                  // [(n_q + 2 n_kv) hd] added to the projection, or null
+  const __nv_bfloat16 *qnorm = nullptr, *knorm = nullptr;  // [hd] RMSNorm weights of the query / key heads, or null
+  float eps = 0.f;
   __nv_bfloat16 *qbuf;                                  // [B][n_kv][qrows][hd], row = j*group + g
   __nv_bfloat16 *pool;                                  // [L][2][num_pages][n_kv][16][hd]
   uint32_t *status;

@@ -14,11 +14,13 @@ def rel_err(a, b):
     return float(np.abs(a - b).max() / max(np.abs(b).max(), 1e-30))
 
 
-def tiny_setup(cfg, cap_tokens, seed=0, perturb=True, flags=0, max_k=None, prompt_seed=1, rounding=True):
+def tiny_setup(cfg, cap_tokens, seed=0, perturb=True, flags=0, max_k=None, prompt_seed=1, rounding=True, concat=None):
     """Oracle prefill of the prompts + a CUDA context/state sharing the same page tables."""
     w = make_weights(cfg, seed)
     if perturb:
         w = perturb_norm_weights(w)
+    if concat is not None:
+        w["head"]["concat"] = concat          # the order the head's two inputs are concatenated in
     prompts = random_prompts(cfg.batch, cfg.prompt_len, cfg.vocab, seed=prompt_seed)
     pt, npg = make_page_tables(np.full(cfg.batch, cap_tokens), cfg.page_size, seed=7, slack_pages=3)
     hpt, hnpg = make_page_tables(np.full(cfg.batch, cap_tokens), cfg.page_size, seed=8, slack_pages=2)

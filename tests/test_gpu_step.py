@@ -31,22 +31,10 @@ def _run_phases(gmb, ctx, gst, K, seed, step, bufs, commit=False):
     assert gmb.gm_last_status(ctx) == 0
 
 
-@pytest.mark.parametrize("flags", [1, 0], ids=["mma_sync_gemm", "tcgen05_gemm"])
-def test_tiny_step_parity_from_common_state(flags):
-    """Every step starts from the oracle's state.
-    (1) the device's draft draws and accept/resample decisions equal the oracle's decision function on the
-        device's own probabilities, bit for bit;
-    (2) with the device's drafts fed back to the oracle (the recorded-path replay of Eq. 4), every logit row
-        and hidden state agrees within 2e-2 and the accept bits agree on >= 99.5 % of the positions both
-        sides evaluate;
-    (3) free-running (each side sampling its own drafts from the same uniforms) the sampled tokens agree on
-        most positions - a looser bar, because an inverse-CDF draw turns a relative logit error e into a
-        disagreement probability of order e * sqrt(V)."""
+def _parity_from_common_state(cfg, flags, n_steps, concat=None):
     import paper_2609_16648_b200 as gmb
-    cfg = get_config("tiny").with_(prompt_len=40)
     K, B, V, d = cfg.k, cfg.batch, cfg.vocab, cfg.d_model
-    n_steps = 24
-    w, ost, ctx, gst = tiny_setup(cfg, cap_tokens=40 + n_steps * (K + 1) + 8, flags=flags)
+    w, ost, ctx, gst = tiny_setup(cfg, cap_tokens=cfg.prompt_len + n_steps * (K + 1) + 8, flags=flags, concat=concat)
     bufs = _bufs(B, K, V, d)
     seed = 5
     bit_agree = bit_total = tok_same = tok_total = fin_same = fin_total = 0
@@ -87,13 +75,47 @@ def test_tiny_step_parity_from_common_state(flags):
         free = ostep.spec_step(w, cfg, ost, K, 1.0, seed=seed, do_commit=True)
         tok_total += B
         tok_same += int((g_dtok[:, 0] == free["draft_tok"][:, 0]).sum())
-    assert worst < TOL, worst
-    assert bit_agree / bit_total >= 0.995, (bit_agree, bit_total)
-    assert tok_same / tok_total >= 0.85, (tok_same, tok_total)
-    assert fin_same / max(fin_total, 1) >= 0.85, (fin_same, fin_total)
+    ctx.close()
     print(f"worst rel err {worst:.3e}; accept bits {bit_agree}/{bit_total}; first draft token {tok_same}/{tok_total}; "
           f"final token {fin_same}/{fin_total}")
-    ctx.close()
+    return worst, (bit_agree, bit_total), (tok_same, tok_total), (fin_same, fin_total)
+
+
+@pytest.mark.parametrize("flags", [1, 0], ids=["mma_sync_gemm", "tcgen05_gemm"])
+def test_tiny_step_parity_from_common_state(flags):
+    """Every step starts from the oracle's state.
+    (1) the device's draft draws and accept/resample decisions equal the oracle's decision function on the
+        device's own probabilities, bit for bit;
+    (2) with the device's drafts fed back to the oracle (the recorded-path replay of Eq. 4), every logit row
+        and hidden state agrees within 2e-2 and the accept bits agree on >= 99.5 % of the positions both
+        sides evaluate;
+    (3) free-running (each side sampling its own drafts from the same uniforms) the sampled tokens agree on
+        most positions - a looser bar, because an inverse-CDF draw turns a relative logit error e into a
+        disagreement probability of order e * sqrt(V)."""
+    cfg = get_config("tiny").with_(prompt_len=40)
+    worst, bits, toks, fins = _parity_from_common_state(cfg, flags, n_steps=24)
+    assert worst < TOL, worst
+    assert bits[0] / bits[1] >= 0.995, bits
+    assert toks[0] / toks[1] >= 0.85, toks
+    assert fins[0] / max(fins[1], 1) >= 0.85, fins
+
+
+@pytest.mark.parametrize("extras", [dict(qkv_bias=True), dict(qk_norm=True),
+                                    dict(qkv_bias=True, qk_norm=True, concat="hidden_first"),
+                                    dict(qkv_bias=True, qk_norm=True, n_q_heads=2, n_kv_heads=1, head_dim=128),
+                                    dict(k=7), dict(k=1)],
+                         ids=["qkv_bias", "qk_norm", "bias_norm_hidden_first", "bias_norm_head128", "depth7", "depth1"])
+def test_tiny_step_parity_variants(extras):
+    """The same bars for the other operating points of the cycle: the decoder-layer families of App. B.1
+    (projection bias; query/key head norms), a head that concatenates [hidden ; embedding], and the
+    smallest and largest drafting depth."""
+    extras = dict(extras)
+    concat = extras.pop("concat", None)
+    cfg = get_config("tiny").with_(prompt_len=40, **extras)
+    worst, bits, toks, fins = _parity_from_common_state(cfg, 0, n_steps=10, concat=concat)
+    assert worst < TOL, worst
+    assert bits[0] / bits[1] >= 0.995, bits
+    assert toks[0] / toks[1] >= 0.8, toks
 
 
 def test_spec_step_equals_three_calls_and_commits_state():
