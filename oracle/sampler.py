@@ -104,8 +104,8 @@ def decide(p: np.ndarray, q: np.ndarray, d, u24s):
     return a, tok, warn
 
 
-def accept_batch(target_logits, draft_logits, draft_tok, u24s, temperature: float = 1.0):
-    """Rows of a batch through softmax + decide.
+def accept_batch(target_logits, draft_logits, draft_tok, u24s, temperature: float = 1.0, top_p: float = 1.0):
+    """Rows of a batch through softmax (+ top-p truncation of the target rows) + decide.
 
     target_logits [B, K+1, V], draft_logits [B, K, V], draft_tok [B, K], u24s [B, K+1].
     Returns (accept_len[B], next_token[B], warn[B]).
@@ -115,10 +115,60 @@ def accept_batch(target_logits, draft_logits, draft_tok, u24s, temperature: floa
     t_out = np.zeros(B, np.int32)
     w_out = np.zeros(B, np.int32)
     for b in range(B):
-        p = softmax_probs(target_logits[b], temperature)
+        p = nucleus_filter(softmax_probs(target_logits[b], temperature), top_p)
         q = softmax_probs(draft_logits[b], temperature)
         a_out[b], t_out[b], w_out[b] = decide(p, q, draft_tok[b], u24s[b])
     return a_out, t_out, w_out
+
+
+# ---- nucleus (top-p) truncation of the target distribution ---------------------------------
+#
+# The paper's evaluation samples with top-p 0.7 (its rollouts with top-p 1, i.e. none).  The
+# truncation is applied to the distribution whose samples the cycle must reproduce - the
+# target's p_1..p_{K+1}; the head's q is left as it is (the accept rule is exact for any q).
+# Stated so that it is single-valued whatever order the masses are added in: with integer
+# weights w = trunc(r * 2^44), W = sum w and tp24 = round(top_p * 2^24), token v is kept iff
+# w[v] > 0 and  (sum of w over tokens with r strictly larger than r[v]) * 2^24 < tp24 * W.
+# That is the textbook rule (sort by probability, keep tokens while the mass before them is
+# below top_p) with every member of a tie at the cut kept.
+
+def nucleus_keep(r, top_p: float) -> np.ndarray:
+    """Boolean mask of the top-p set of non-negative weights r (fp32, any normalisation)."""
+    if not (0.0 < float(top_p) <= 1.0):
+        raise ValueError("top_p must be in (0, 1]")
+    r = np.asarray(r, dtype=np.float32)
+    w = integer_weights(r)
+    tp24 = int(round(float(np.float32(top_p)) * (1 << 24)))
+    W = int(w.sum(dtype=np.uint64))
+    order = np.argsort(-r, kind="stable")
+    keep = np.zeros(r.shape, bool)
+    above = 0                       # weight of the tokens strictly larger than the current tie group
+    i = 0
+    while i < len(order):
+        j = i
+        group = 0
+        while j < len(order) and r[order[j]] == r[order[i]]:
+            group += int(w[order[j]])
+            j += 1
+        if (above << 24) < tp24 * W:
+            for t in order[i:j]:
+                keep[t] = w[t] > 0
+        above += group
+        i = j
+    return keep
+
+
+def nucleus_filter(p, top_p: float) -> np.ndarray:
+    """Rows of p [..., V] truncated to their top-p sets and renormalised (fp64 division), fp32 out."""
+    p = np.asarray(p, dtype=np.float32)
+    if float(top_p) >= 1.0:
+        return p
+    flat = p.reshape(-1, p.shape[-1])
+    out = np.zeros_like(flat)
+    for i, row in enumerate(flat):
+        kept = np.where(nucleus_keep(row, top_p), row.astype(np.float64), 0.0)
+        out[i] = (kept / kept.sum()).astype(np.float32)
+    return out.reshape(p.shape)
 
 
 # ---- closed forms used as pins (Eq. 5 and Eq. 6) ---------------------------------------

@@ -99,14 +99,15 @@ def draft(w, cfg, st: BatchState, b: int, K: int, temperature: float, u24_draft,
     return d, np.array(logits_out), np.array(q_out)
 
 
-def verify(w, cfg, st: BatchState, b: int, d, temperature: float, round_interface=True):
-    """Target forward over [x[Len-1], d_1..d_K]; returns (logits[K+1, V], H[K+1, d], p[K+1, V])."""
+def verify(w, cfg, st: BatchState, b: int, d, temperature: float, round_interface=True, top_p: float = 1.0):
+    """Target forward over [x[Len-1], d_1..d_K]; returns (logits[K+1, V], H[K+1, d], p[K+1, V]);
+    p is truncated to its top-p sets when top_p < 1."""
     s = st.seqs[b]
     toks = [s.tokens[-1]] + list(d)
     pos = np.arange(s.kv_len, s.kv_len + len(toks))
     H = _maybe_round(target_forward(w, toks, pos, st.kv, b, cfg), round_interface)
     logits = _maybe_round(target_logits(w, H, cfg), round_interface)
-    return logits, H, sampler.softmax_probs(logits, temperature)
+    return logits, H, sampler.nucleus_filter(sampler.softmax_probs(logits, temperature), top_p)
 
 
 def commit(st: BatchState, b: int, d, a: int, t_star: int, H):
@@ -120,9 +121,10 @@ def commit(st: BatchState, b: int, d, a: int, t_star: int, H):
 
 def spec_step(w, cfg, st: BatchState, K: int, temperature: float = 1.0, seed: int = 0,
               do_commit: bool = True, round_interface: bool = True,
-              u24_draft=None, u24_accept=None, forced_draft=None):
+              u24_draft=None, u24_accept=None, forced_draft=None, top_p: float = 1.0):
     """One cycle for every sequence.  Returns a dict of per-row outputs.  ``forced_draft`` [B, K]
-    replays recorded draft tokens (see ``draft``)."""
+    replays recorded draft tokens (see ``draft``).  ``top_p`` < 1 truncates the target's
+    distributions to their nucleus before the accept test."""
     B = len(st.seqs)
     ud = philox.u24_draft(seed, st.step, B, K) if u24_draft is None else u24_draft
     ua = philox.u24_accept(seed, st.step, B, K) if u24_accept is None else u24_accept
@@ -131,7 +133,7 @@ def spec_step(w, cfg, st: BatchState, K: int, temperature: float = 1.0, seed: in
     for b in range(B):
         d, dl, q = draft(w, cfg, st, b, K, temperature, ud[b], round_interface,
                          None if forced_draft is None else forced_draft[b])
-        tl, H, p = verify(w, cfg, st, b, d, temperature, round_interface)
+        tl, H, p = verify(w, cfg, st, b, d, temperature, round_interface, top_p)
         a, t_star, warn = sampler.decide(p, q, d, ua[b])
         if do_commit:
             commit(st, b, d, a, t_star, H)

@@ -9,6 +9,8 @@ import numpy as np
 import pytest
 from scipy import stats
 
+import torch
+
 from oracle import sampler
 
 V = 16
@@ -265,3 +267,99 @@ def test_noisy_logit_acceptance_closed_form():
                                                      sampler.softmax_probs(dr[i])) for i in range(4)])
         assert abs(al - math.erfc(sigma / (2 * math.sqrt(2)))) < 0.01
     assert abs(math.erfc(0.908 / (2 * math.sqrt(2))) - 0.65) < 2e-3
+
+
+# ---- nucleus (top-p) truncation -----------------------------------------------------------------------
+
+def _textbook_top_p(p, top_p):
+    """Sort descending, keep a token while the mass before it is below top_p (exact rationals)."""
+    from fractions import Fraction
+    order = sorted(range(len(p)), key=lambda i: -p[i])
+    total = sum(Fraction(float(x)) for x in p)
+    keep, before = np.zeros(len(p), bool), Fraction(0)
+    for i in order:
+        if before < Fraction(float(np.float32(top_p))) * total:
+            keep[i] = True
+        before += Fraction(float(p[i]))
+    return keep
+
+
+def test_nucleus_equals_textbook_rule_without_ties():
+    rng = np.random.default_rng(31)
+    for trial in range(40):
+        v = int(rng.integers(2, 60))
+        p = _dist(rng, v, conc=float(rng.choice([0.2, 1.0, 5.0])))
+        assert len(np.unique(p)) == v
+        top_p = float(rng.uniform(0.05, 0.99))
+        # 2^-44 quantisation can move a cut only if the mass before a token is within V * 2^-44 of it
+        ref = _textbook_top_p(p, top_p)
+        srt = np.sort(p.astype(np.float64))[::-1]
+        margin = np.abs(np.concatenate([[0.0], np.cumsum(srt)[:-1]]) - np.float32(top_p) * srt.sum()).min()
+        if margin > 1e-9:
+            np.testing.assert_array_equal(sampler.nucleus_keep(p, top_p), ref)
+
+
+def test_nucleus_against_library_sort_and_cumsum():
+    rng = np.random.default_rng(32)
+    p = _dist(rng, 500, conc=0.3)
+    for top_p in (0.1, 0.5, 0.7, 0.9):
+        t = torch.from_numpy(p.astype(np.float64))
+        srt, idx = torch.sort(t, descending=True)
+        before = torch.cumsum(srt, 0) - srt
+        keep = torch.zeros(500, dtype=torch.bool)
+        keep[idx[before < top_p * float(t.sum())]] = True
+        np.testing.assert_array_equal(sampler.nucleus_keep(p, top_p), keep.numpy())
+
+
+def test_nucleus_properties():
+    rng = np.random.default_rng(33)
+    p = _dist(rng, 200, conc=0.5)
+    for top_p in (0.3, 0.7, 0.95):
+        keep = sampler.nucleus_keep(p, top_p)
+        kept = np.sort(p[keep].astype(np.float64))
+        assert kept.sum() >= top_p * p.sum(dtype=np.float64) - 1e-9          # covers top_p of the mass
+        assert kept.sum() - kept[0] < top_p * p.sum(dtype=np.float64)        # and is minimal
+        assert p[keep].min() > p[~keep].max()                               # a prefix of the sorted order
+        assert keep[np.argmax(p)]
+        f = sampler.nucleus_filter(p, top_p)
+        np.testing.assert_allclose(f.sum(dtype=np.float64), 1.0, atol=1e-6)
+        np.testing.assert_allclose(f[keep], p[keep] / kept.sum(), rtol=1e-6)
+        assert (f[~keep] == 0).all()
+    assert sampler.nucleus_keep(p, 1e-6).sum() == 1                        # only the mode
+    assert sampler.nucleus_keep(p, 1.0).all()                              # everything with mass
+    np.testing.assert_array_equal(sampler.nucleus_filter(p, 1.0), p)
+    # scale of the weights does not matter (unnormalised weights give the same set)
+    np.testing.assert_array_equal(sampler.nucleus_keep(p * np.float32(0.25), 0.7), sampler.nucleus_keep(p, 0.7))
+    with pytest.raises(ValueError):
+        sampler.nucleus_keep(p, 0.0)
+
+
+def test_nucleus_keeps_every_member_of_a_tie_at_the_cut():
+    p = np.array([0.4, 0.2, 0.2, 0.1, 0.1], np.float32)
+    np.testing.assert_array_equal(sampler.nucleus_keep(p, 0.5), [True, True, True, False, False])
+    np.testing.assert_array_equal(sampler.nucleus_keep(p, 0.4), [True, False, False, False, False])
+    np.testing.assert_array_equal(sampler.nucleus_keep(p, 0.41), [True, True, True, False, False])
+    np.testing.assert_array_equal(sampler.nucleus_keep(p, 0.85), [True, True, True, True, True])
+    z = np.array([0.5, 0.0, 0.5, 0.0], np.float32)                          # zero-mass tokens are never kept
+    np.testing.assert_array_equal(sampler.nucleus_keep(z, 1.0), [True, False, True, False])
+
+
+def test_cycle_with_truncated_target_follows_the_truncated_law():
+    """Losslessness with top-p: the first committed token of a cycle is distributed as the truncated
+    target, although the head's distribution is not truncated (chi-square, 200k cycles)."""
+    from scipy import stats
+    rng = np.random.default_rng(34)
+    v = 24
+    p = np.stack([_dist(rng, v, 0.6), _dist(rng, v, 0.6)])
+    q = _dist(rng, v, 0.6)[None]
+    pf = sampler.nucleus_filter(p, 0.7)
+    assert 1 < (pf[0] > 0).sum() < v
+    n = 200_000
+    d = sampler.icdf_draw_many(q[0], _u24(rng, n))[:, None]
+    a, tok = sampler.decide_many(pf, q, d, _u24(rng, (n, 2)))
+    first = np.where(a >= 1, d[:, 0], tok)
+    support = pf[0] > 0
+    assert not np.isin(first, np.nonzero(~support)[0]).any()
+    obs = np.bincount(first, minlength=v)[support]
+    chi = stats.chisquare(obs, pf[0][support].astype(np.float64) / pf[0][support].sum(dtype=np.float64) * n)
+    assert chi.pvalue > 1e-4, chi
