@@ -99,7 +99,8 @@ def lengths_for(cfg, seed):
     return kv_lengths_uniform(cfg.batch, cfg.kv_len_min, cfg.kv_len_max, seed)
 
 
-def build_workload(name: str, rank: int, total_steps: int, k: int, device, layers: int = 0, batch: int = 0):
+def build_workload(name: str, rank: int, total_steps: int, k: int, device, layers: int = 0, batch: int = 0,
+                   top_p: float = 1.0):
     """Random-init model of the named shape + a batch of sequences with ragged, fragmented KV caches.
     `layers` / `batch` > 0 shrink the model depth / the batch (profiling captures on a few GB)."""
     import torch
@@ -135,6 +136,8 @@ def build_workload(name: str, rank: int, total_steps: int, k: int, device, layer
     hpt, hnpg = make_page_tables(cap, 16, seed=8 + rank)
     packed = gmb.random_packed_weights(cfg, device, seed=rank)
     ctx = gmb.Context(cfg, packed, keep, k, pt.shape[1], npg, hnpg)
+    if top_p < 1.0:
+        gmb.gm_set_top_p(ctx, top_p)
     st = gmb.State(ctx, keep, np.where(pt < 0, 0, pt), np.where(hpt < 0, 0, hpt), device)
     gen = torch.Generator(device=device)
     gen.manual_seed(100 + rank)
@@ -311,7 +314,7 @@ def run_product(args):
 
     K, W, S = args.k, args.warmup, args.steps
     total_steps = W + 2 * S + 12
-    cfg, ctx, st, lens = build_workload(args.workload, rank, total_steps, K, device, args.layers, args.batch)
+    cfg, ctx, st, lens = build_workload(args.workload, rank, total_steps, K, device, args.layers, args.batch, args.top_p)
     B = cfg.batch
     a_dev = torch.zeros(B, dtype=torch.int32, device=device)
     t_dev = torch.zeros(B, dtype=torch.int32, device=device)
@@ -418,7 +421,7 @@ def run_product(args):
             "warmup": W, "ms_per_step": ms_max / S, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "n_layers": cfg.n_layers, "batch_per_gpu": B, "k": K, "temperature": 1.0,
-                       "kv_len_mean": float(lens.mean()), "kv_len_min": int(lens.min()), "kv_len_max": int(lens.max()),
+                       "top_p": args.top_p, "kv_len_mean": float(lens.mean()), "kv_len_min": int(lens.min()), "kv_len_max": int(lens.max()),
                        "page": 16, "tau": committed / (S * B), "parallelism": f"replicas x{world}",
                        "l2": "per-step working set (weights + KV, tens of GB) >> 126 MB L2: no flush needed",
                        "step_algorithmic_GB": step_bytes / 1e9, "step_roofline_ms": step_roof_ms,
@@ -474,6 +477,8 @@ def run_sampler_only(args):
     B, K, V, S, W = (args.batch or cfg.batch), args.k, cfg.vocab, args.steps, args.warmup
     mcfg = cfg.with_(n_layers=1, d_model=64, n_q_heads=1, n_kv_heads=1, head_dim=64, d_ffn=64, batch=B)
     ctx = gmb.Context(mcfg, gmb.random_packed_weights(mcfg, device), B, K, 4, 8, 8)
+    if args.top_p < 1.0:
+        gmb.gm_set_top_p(ctx, args.top_p)
     tgt, drf = sampler_only_logits(B, K, V, sigma=0.908, seed=4 + rank)
     t_h = torch.from_numpy(tgt).to(torch.bfloat16).pin_memory()
     d_h = torch.from_numpy(drf).to(torch.bfloat16).pin_memory()
@@ -538,7 +543,7 @@ def run_sampler_only(args):
         line = {"metric": METRIC, "value": committed_all / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": S,
                 "warmup": W, "ms_per_step": ms_max / S, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": "sampler", "batch_per_gpu": B, "k": K, "vocab": V, "temperature": 1.0,
+                "config": {"workload": "sampler", "batch_per_gpu": B, "k": K, "vocab": V, "temperature": 1.0, "top_p": args.top_p,
                            "tau": committed / (S * B), "l2": "544 MB of logits per step > 126 MB L2: no flush needed",
                            "peaks": which},
                 "clocks": clk,
@@ -575,6 +580,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (small profiling cases)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (small profiling cases)")
     ap.add_argument("--record", action="store_true", help="also write the per-cycle verification record every step")
+    ap.add_argument("--top-p", type=float, default=1.0,
+                    help="nucleus of the target distributions (1 = none, the paper's rollout setting; its evaluation uses 0.7)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--breakdown", action="store_true", help="add device time per kernel class (extra pass)")
     args = ap.parse_args()

@@ -172,6 +172,27 @@ int gm_accept(gm_ctx *ctx, gm_state *st, int batch, int k, float temperature,
 int gm_spec_step(gm_ctx *ctx, gm_state *st, int k, float temperature, uint64_t seed,
                  uint64_t step, int32_t *accept_len, int32_t *next_token, int32_t *draft_tok);
 
+/* Nucleus (top-p) sampling of the target (the paper's evaluation uses top-p 0.7, its rollouts
+ * top-p 1 = none, Sec. 4 / App. B).  gm_set_top_p stores the value in the context (default 1);
+ * while it is below 1, gm_accept - and therefore gm_spec_step and its variants - first
+ * truncates every target row to its top-p set and renormalises, so the committed tokens
+ * follow the truncated target law; the head's distributions are not truncated, and the
+ * cycle record still holds the full distribution.  The first call with top_p < 1 allocates a
+ * buffer of max_batch (max_k + 1) V bf16.  top_p outside (0, 1] -> GM_ERR_UNSUPPORTED.
+ *
+ * The set is order-free: with e[v] = 2^((x[v] - max) log2(e) / T) in fp32, w[v] = trunc(e[v] 2^44),
+ * W = sum w and tp24 = round(top_p 2^24), v is kept iff
+ *     (sum of w over entries whose logit is larger than x[v]) * 2^24  <  tp24 * W,
+ * i.e. tokens in decreasing probability while the mass before them is below top_p, every
+ * member of a tie at the cut kept.
+ *
+ * gm_nucleus is the truncation as a stand-alone call: logits bf16 [rows, V] in, out bf16
+ * [rows, V] = the same rows with entries outside the set replaced by -inf (out must not alias
+ * logits); dbg_weight fp32 [rows, V] receives e or is NULL.  It needs top_p < 1.             */
+int gm_set_top_p(gm_ctx *ctx, float top_p);
+int gm_nucleus(gm_ctx *ctx, const void *logits, int rows, float temperature, float top_p,
+               void *out, float *dbg_weight);
+
 /* Draw one token per row from softmax(logits / T) by the integer inverse CDF (the draw of the
  * draft phase as a stand-alone call).  logits bf16 [rows, V]; u24 [rows]; out_tok [rows];
  * dbg_prob fp32 [rows, V] or NULL.                                                           */

@@ -22,7 +22,7 @@ GM_MAX_K, GM_PAGE = 7, 16
 GM_FLAG_SIMPLE_GEMM, GM_FLAG_SAMPLER_CLUSTER, GM_FLAG_SAMPLER_STREAM = 1, 2, 4
 GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER, GM_KC_RECORD = 0, 1, 2, 3, 4
 
-EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw",
+EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw", "gm_set_top_p", "gm_nucleus",
            "gm_spec_step_host", "gm_gemm", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
            "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
@@ -78,6 +78,8 @@ def lib() -> C.CDLL:
     L.gm_spec_step.argtypes = [vp, C.POINTER(gm_state), i32, f32, u64, u64, vp, vp, vp]
     L.gm_spec_step_host.argtypes = [vp, C.POINTER(gm_state), i32, f32, u64, u64, vp, vp, vp, vp, vp]
     L.gm_draw.argtypes = [vp, vp, i32, f32, vp, vp, vp]
+    L.gm_set_top_p.argtypes = [vp, f32]
+    L.gm_nucleus.argtypes = [vp, vp, i32, f32, f32, vp, vp]
     L.gm_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
     L.gm_attention.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, i32, i32, vp]
     L.gm_attention_noalloc.argtypes = [i32, i32, i32, i32, vp, vp, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp]
@@ -299,6 +301,14 @@ def gm_spec_step_host(ctx: Context, st: State, k: int, temperature: float, seed:
 
 def gm_draw(ctx: Context, logits, rows: int, temperature: float, u24, out_tok, dbg_prob=None):
     _check(lib().gm_draw(ctx.handle, _p(logits), rows, temperature, _p(u24), _p(out_tok), _p(dbg_prob)), "gm_draw")
+
+
+def gm_set_top_p(ctx: Context, top_p: float):
+    _check(lib().gm_set_top_p(ctx.handle, top_p), "gm_set_top_p")
+
+
+def gm_nucleus(ctx: Context, logits, rows: int, temperature: float, top_p: float, out, dbg_weight=None):
+    _check(lib().gm_nucleus(ctx.handle, _p(logits), rows, temperature, top_p, _p(out), _p(dbg_weight)), "gm_nucleus")
 
 
 def gm_gemm(ctx: Context, x, w, out, M: int, N: int, K: int, out_fp32: bool):

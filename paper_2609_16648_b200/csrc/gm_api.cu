@@ -61,6 +61,8 @@ struct gm_ctx {
   int32_t *qn = nullptr, *qbase = nullptr, *page_start = nullptr;
   float2 *rope = nullptr;
   uint32_t *status = nullptr;
+  float top_p = 1.f;                    // nucleus of the target distributions (1 = none)
+  __nv_bfloat16 *ws_nucleus = nullptr;  // [max_batch (max_k + 1)][V] filtered target rows, allocated by gm_set_top_p
   std::vector<void *> allocs;
 
   // profiling
@@ -556,6 +558,8 @@ int gm_verify(gm_ctx *c, const gm_state *st, int k, const int32_t *draft_tok, vo
                   target_logits, EPI_STORE_BF16, c->V);
 }
 
+static int run_nucleus(gm_ctx *c, const void *logits, int rows, float temperature, float top_p, void *out, float *dbg_e);
+
 int gm_accept(gm_ctx *c, gm_state *st, int batch, int k, float temperature, const void *target_logits,
               const void *draft_logits, const int32_t *draft_tok, const uint32_t *u24_accept, uint64_t seed,
               uint64_t step, int32_t *accept_len, int32_t *next_token, float *dbg_p, float *dbg_q,
@@ -572,6 +576,11 @@ int gm_accept(gm_ctx *c, gm_state *st, int batch, int k, float temperature, cons
   int rc = fill_sampler(c, S, temperature);
   if (rc) return rc;
   S.K = k;
+  if (c->top_p < 1.f) {                 // truncate the target rows to their nucleus first; the head's rows stay as they are
+    if (batch > c->cfg.max_batch || k > c->cfg.max_k) return GM_ERR_INVALID_ARG;
+    if ((rc = run_nucleus(c, target_logits, batch * (k + 1), temperature, c->top_p, c->ws_nucleus, nullptr)) != GM_OK) return rc;
+    target_logits = c->ws_nucleus;
+  }
   S.target_logits = static_cast<const __nv_bfloat16 *>(target_logits); S.tgt_bstride = static_cast<size_t>(k + 1) * c->V;
   S.draft_logits = static_cast<const __nv_bfloat16 *>(draft_logits); S.drf_bstride = static_cast<size_t>(k) * c->V;
   S.draft_tok = draft_tok; S.tok_in_stride = k; S.u24 = u24_accept; S.u_stride = k + 1; S.seed = seed; S.step = step;
@@ -584,6 +593,35 @@ int gm_accept(gm_ctx *c, gm_state *st, int batch, int k, float temperature, cons
     S.d_model = c->d; S.max_k = c->cfg.max_k;
   }
   GM_LAUNCH(c, GM_KC_SAMPLER, run_sampler(c, S, batch));
+  return GM_OK;
+}
+
+static int run_nucleus(gm_ctx *c, const void *logits, int rows, float temperature, float top_p, void *out, float *dbg_e) {
+  if (!(temperature > 0.f) || !std::isfinite(temperature) || !(top_p > 0.f) || !(top_p < 1.f)) return GM_ERR_UNSUPPORTED;
+  NucleusArgs N;
+  N.in = static_cast<const __nv_bfloat16 *>(logits); N.out = static_cast<__nv_bfloat16 *>(out); N.dbg_e = dbg_e;
+  N.rows = rows; N.V = c->V; N.inv_temp = 1.0f / temperature;
+  N.tp24 = static_cast<uint32_t>(std::nearbyint(static_cast<double>(top_p) * 16777216.0));
+  if (N.tp24 < 1u) N.tp24 = 1u;
+  if (N.tp24 > 16777215u) N.tp24 = 16777215u;
+  GM_LAUNCH(c, GM_KC_SAMPLER, launch_nucleus(N, c->stream));
+  return GM_OK;
+}
+
+int gm_nucleus(gm_ctx *c, const void *logits, int rows, float temperature, float top_p, void *out, float *dbg_weight) {
+  if (!c || !logits || !out || rows < 1 || logits == out) return GM_ERR_INVALID_ARG;
+  return run_nucleus(c, logits, rows, temperature, top_p, out, dbg_weight);
+}
+
+int gm_set_top_p(gm_ctx *c, float top_p) {
+  if (!c) return GM_ERR_INVALID_ARG;
+  if (!(top_p > 0.f) || !(top_p <= 1.f)) return GM_ERR_UNSUPPORTED;
+  if (top_p < 1.f && !c->ws_nucleus) {
+    const size_t n = static_cast<size_t>(c->cfg.max_batch) * (c->cfg.max_k + 1) * c->V;
+    int rc = dev_alloc(c, &c->ws_nucleus, n, false);
+    if (rc) return rc;
+  }
+  c->top_p = top_p;
   return GM_OK;
 }
 

@@ -85,6 +85,17 @@ cudaError_t launch_record_begin(const int32_t *kv_len, const int32_t *pending_n,
 cudaError_t launch_record_end(const int32_t *draft_tok, const int32_t *accept_len, int batch, int k, int32_t *drafts,
                               int32_t *accepted, cudaStream_t stream);
 
+// ---- nucleus (top-p) truncation of logit rows: entries outside the top-p set become -inf ---------------
+struct NucleusArgs {
+  const __nv_bfloat16 *in;              // [rows][V]
+  __nv_bfloat16 *out;                   // [rows][V] (may not alias in)
+  float *dbg_e;                         // [rows][V] fp32 weights 2^((x - max) s) or null
+  int rows, V;
+  float inv_temp;
+  uint32_t tp24;                        // round(top_p * 2^24), 1 .. 2^24 - 1
+};
+cudaError_t launch_nucleus(const NucleusArgs &A, cudaStream_t stream);
+
 // ---- planning: query ranges of a phase and the balanced attention partition --------------------------
 enum PhaseMode { PHASE_VERIFY = 0, PHASE_DRAFT_FIRST = 1, PHASE_DRAFT_NEXT = 2 };
 struct PlanArgs {

@@ -105,11 +105,13 @@ sampler_kernel(const SamplerArgs A) {
       const float mx = fmaxf(bf16_lo(m2), bf16_hi(m2));
       const float c = -mx * s;
       float acc = 0.f;
-      for (int i = tid; i < n; i += SAMP_THREADS) {
-        float x[8];
-        unpack8(buf[i], x);
+      if (mx != -INFINITY) {                      // a thread that saw only -inf (masked-out) logits contributes nothing
+        for (int i = tid; i < n; i += SAMP_THREADS) {
+          float x[8];
+          unpack8(buf[i], x);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc += ex2(fmaf(x[j], s, c));
+          for (int j = 0; j < 8; ++j) acc += ex2(fmaf(x[j], s, c));
+        }
       }
       st = MZ{mx, acc};
     }

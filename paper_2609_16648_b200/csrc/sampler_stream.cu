@@ -148,12 +148,14 @@ __global__ void __launch_bounds__(SS_THREADS, 2) sampler_stream_kernel(const Sam
           if (mx > st.m) { st.z *= ex2((st.m - mx) * s); st.m = mx; }          // 0 * 2^-inf = 0 on the first chunk
           const float c = -st.m * s;
           float acc = 0.f;
+          if (st.m != -INFINITY) {                                              // only -inf (masked-out) logits so far: nothing to add
 #pragma unroll
-          for (int t = 0; t < 3; ++t) {
-            float x[8];
-            unpack8(v[t], x);
+            for (int t = 0; t < 3; ++t) {
+              float x[8];
+              unpack8(v[t], x);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) acc += ex2(fmaf(x[j], s, c));           // padding lanes: 2^-inf = 0
+              for (int j = 0; j < 8; ++j) acc += ex2(fmaf(x[j], s, c));         // padding lanes: 2^-inf = 0
+            }
           }
           st.z += acc;
         }

@@ -185,3 +185,110 @@ def test_sampler_only_workload_full_size_all_rows():
     first = (an >= 1).mean()
     assert 0.5 < first < 0.8, first                               # per-token acceptance ~ 0.65 (+- sampling noise)
     ctx.close()
+
+
+# ---- nucleus (top-p) truncation of the target rows ----------------------------------------------------------
+
+@pytest.mark.parametrize("rows,V,temp,top_p", [(6, 4096, 1.0, 0.7), (3, 4104, 0.6, 0.3), (4, 151936, 1.0, 0.7),
+                                               (2, 151936, 1.5, 0.95), (2, 8, 1.0, 0.5)])
+def test_nucleus_set_is_the_oracles_on_the_device_weights(rows, V, temp, top_p):
+    gmb, ctx = _ctx(V)
+    rng = np.random.default_rng(70 + rows)
+    x = (rng.standard_normal((rows, V)) * 3.0).astype(np.float32)
+    x[0, : V // 2] = x[0, V // 2: 2 * (V // 2)]          # plenty of exact ties in the first row
+    xin = _bf16(x)
+    out = torch.zeros_like(xin)
+    e = torch.zeros((rows, V), dtype=torch.float32, device="cuda")
+    gmb.gm_nucleus(ctx, xin, rows, temp, top_p, out, e)
+    assert gmb.gm_last_status(ctx) == 0
+    xb, ob, ev = xin.float().cpu().numpy(), out.float().cpu().numpy(), e.cpu().numpy()
+    kept = np.isfinite(ob)
+    np.testing.assert_array_equal(ob[kept], xb[kept])                        # kept entries pass through unchanged
+    assert np.isneginf(ob[~kept]).all()
+    ref_e = np.exp2((xb.astype(np.float64) - xb.max(1, keepdims=True)) * (np.log2(np.e) / temp))
+    assert np.abs(ev - ref_e).max() <= 5e-6
+    for r in range(rows):
+        want = osampler.nucleus_keep(ev[r], top_p)
+        diff = np.nonzero(want != kept[r])[0]
+        # distinct logits whose weights round to the same fp32 value may fall on either side of the cut
+        assert len(diff) == 0 or (len(np.unique(ev[r][diff])) == 1 and ev[r][diff[0]] == ev[r][kept[r]].min()), (r, diff[:8])
+        assert len(diff) <= 4
+        lo = xb[r][kept[r]].min()
+        assert (xb[r][~kept[r]] < lo).all() or len(diff)                      # a threshold on the logit
+    # without the weight dump the result is the same
+    out2 = torch.zeros_like(xin)
+    gmb.gm_nucleus(ctx, xin, rows, temp, top_p, out2)
+    assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
+    ctx.close()
+
+
+def test_accept_with_top_p_truncates_the_target_only():
+    gmb, ctx = _ctx(8200, max_batch=8, max_k=3)
+    B, K, V, top_p = 8, 3, 8200, 0.7
+    tgt, drf = sampler_only_logits(B, K, V, sigma=0.9, seed=81)
+    dtok = _draft_tokens(drf, seed=82)
+    u24 = random_u24((B, K + 1), seed=83)
+    args = (_bf16(tgt), _bf16(drf), torch.from_numpy(dtok).cuda(), torch.from_numpy(u24.astype(np.int32)).cuda(), 0, 0)
+
+    def run():
+        a = torch.zeros(B, dtype=torch.int32, device="cuda")
+        t = torch.zeros(B, dtype=torch.int32, device="cuda")
+        dp = torch.zeros((B, K + 1, V), dtype=torch.float32, device="cuda")
+        dq = torch.zeros((B, K, V), dtype=torch.float32, device="cuda")
+        gmb.gm_accept(ctx, None, B, K, 1.0, *args, a, t, dp, dq)
+        assert gmb.gm_last_status(ctx) == 0
+        return a.cpu().numpy(), t.cpu().numpy(), dp.cpu().numpy(), dq.cpu().numpy()
+
+    a0, t0, p0, q0 = run()
+    gmb.gm_set_top_p(ctx, top_p)
+    a1, t1, p1, q1 = run()
+    np.testing.assert_array_equal(q1, q0)                                    # the head's rows are untouched
+    ref = osampler.nucleus_filter(osampler.softmax_probs(_bf16(tgt).float().cpu().numpy()), top_p)
+    support_diff = ((p1 > 0) != (ref > 0)).sum()
+    assert support_diff <= 2, support_diff                                   # a cut within rounding of a token's mass
+    if support_diff == 0:
+        assert np.abs(p1 - ref).max() <= 1e-5 * ref.max()
+    np.testing.assert_allclose(p1.sum(-1), 1.0, atol=2e-5)
+    assert ((p1 > 0).sum(-1) < (p0 > 0).sum(-1)).all()
+    for b in range(B):                                                       # decisions: the oracle on the dumped rows
+        ea, et, _ = osampler.decide(p1[b], q1[b], dtok[b], u24[b])
+        assert (int(a1[b]), int(t1[b])) == (ea, et)
+        assert p1[b, a1[b], t1[b]] > 0                                       # the final token lies in the nucleus
+    gmb.gm_set_top_p(ctx, 1.0)
+    a2, t2, p2, _ = run()
+    np.testing.assert_array_equal(a2, a0)
+    np.testing.assert_array_equal(t2, t0)
+    np.testing.assert_array_equal(p2, p0)
+    with pytest.raises(RuntimeError):
+        gmb.gm_set_top_p(ctx, 0.0)
+    ctx.close()
+
+
+def test_nucleus_flat_negative_constant_and_peaked_rows():
+    """Rows whose cut lies far below the maximum in key space (the kernel's key window has to slide), below zero,
+    on a tie that spans the row, or right at the mode."""
+    V, top_p = 8192, 0.9
+    gmb, ctx = _ctx(V)
+    rng = np.random.default_rng(91)
+    x = np.zeros((6, V), np.float32)
+    x[0] = rng.standard_normal(V) * 0.02                   # flat around zero: the cut is a small negative logit
+    x[1] = -np.abs(rng.standard_normal(V)) * 4.0 - 1.0     # all negative
+    x[2] = 1.25                                            # constant: one tie, everything kept
+    x[3] = rng.standard_normal(V)
+    x[3, 77] = 40.0                                        # one token holds all the mass
+    x[4] = rng.standard_normal(V) * 1e-3 - 5.0             # flat, negative
+    x[5] = np.where(rng.random(V) < 0.5, 3.0, -3.0)        # two ties
+    xin = _bf16(x)
+    out = torch.zeros_like(xin)
+    e = torch.zeros((6, V), dtype=torch.float32, device="cuda")
+    gmb.gm_nucleus(ctx, xin, 6, 1.0, top_p, out, e)
+    assert gmb.gm_last_status(ctx) == 0
+    kept, ev = np.isfinite(out.float().cpu().numpy()), e.cpu().numpy()
+    for r in range(6):
+        want = osampler.nucleus_keep(ev[r], top_p)
+        diff = np.nonzero(want != kept[r])[0]
+        assert len(diff) == 0 or len(np.unique(ev[r][diff])) == 1, (r, len(diff))
+    assert kept[2].all() and kept[3].sum() == 1 and kept[3, 77]
+    assert (xin[0].float().cpu().numpy()[kept[0]] < 0).any() and 0.85 * V < kept[0].sum() < 0.95 * V
+    np.testing.assert_array_equal(kept[5], xin[5].float().cpu().numpy() > 0)
+    ctx.close()

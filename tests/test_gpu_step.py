@@ -31,10 +31,11 @@ def _run_phases(gmb, ctx, gst, K, seed, step, bufs, commit=False):
     assert gmb.gm_last_status(ctx) == 0
 
 
-def _parity_from_common_state(cfg, flags, n_steps, concat=None):
+def _parity_from_common_state(cfg, flags, n_steps, concat=None, top_p=1.0):
     import paper_2609_16648_b200 as gmb
     K, B, V, d = cfg.k, cfg.batch, cfg.vocab, cfg.d_model
     w, ost, ctx, gst = tiny_setup(cfg, cap_tokens=cfg.prompt_len + n_steps * (K + 1) + 8, flags=flags, concat=concat)
+    gmb.gm_set_top_p(ctx, top_p)
     bufs = _bufs(B, K, V, d)
     seed = 5
     bit_agree = bit_total = tok_same = tok_total = fin_same = fin_total = 0
@@ -56,7 +57,7 @@ def _parity_from_common_state(cfg, flags, n_steps, concat=None):
             ea, et, _ = osampler.decide(p[b], q[b], g_dtok[b], ua[b])
             assert (ea, et) == (int(ga[b]), int(gt[b]))
         # (2) replay of the device's drafts through the oracle
-        ref = ostep.spec_step(w, cfg, ost, K, 1.0, seed=seed, do_commit=False, forced_draft=g_dtok)
+        ref = ostep.spec_step(w, cfg, ost, K, 1.0, seed=seed, do_commit=False, forced_draft=g_dtok, top_p=top_p)
         worst = max(worst,
                     rel_err(bufs["draft_logits"].float().cpu().numpy(), ref["draft_logits"]),
                     rel_err(bufs["tgt_logits"].float().cpu().numpy(), ref["target_logits"]),
@@ -72,7 +73,7 @@ def _parity_from_common_state(cfg, flags, n_steps, concat=None):
                 fin_total += 1
                 fin_same += int(gt[b] == ref["next_token"][b])
         # (3) free-running oracle from the same state and uniforms
-        free = ostep.spec_step(w, cfg, ost, K, 1.0, seed=seed, do_commit=True)
+        free = ostep.spec_step(w, cfg, ost, K, 1.0, seed=seed, do_commit=True, top_p=top_p)
         tok_total += B
         tok_same += int((g_dtok[:, 0] == free["draft_tok"][:, 0]).sum())
     ctx.close()
@@ -103,16 +104,18 @@ def test_tiny_step_parity_from_common_state(flags):
 @pytest.mark.parametrize("extras", [dict(qkv_bias=True), dict(qk_norm=True),
                                     dict(qkv_bias=True, qk_norm=True, concat="hidden_first"),
                                     dict(qkv_bias=True, qk_norm=True, n_q_heads=2, n_kv_heads=1, head_dim=128),
-                                    dict(k=7), dict(k=1)],
-                         ids=["qkv_bias", "qk_norm", "bias_norm_hidden_first", "bias_norm_head128", "depth7", "depth1"])
+                                    dict(k=7), dict(k=1), dict(top_p=0.7)],
+                         ids=["qkv_bias", "qk_norm", "bias_norm_hidden_first", "bias_norm_head128", "depth7", "depth1",
+                              "top_p_0.7"])
 def test_tiny_step_parity_variants(extras):
     """The same bars for the other operating points of the cycle: the decoder-layer families of App. B.1
     (projection bias; query/key head norms), a head that concatenates [hidden ; embedding], and the
-    smallest and largest drafting depth."""
+    smallest and largest drafting depth, and the evaluation's nucleus sampling of the target."""
     extras = dict(extras)
     concat = extras.pop("concat", None)
+    top_p = extras.pop("top_p", 1.0)
     cfg = get_config("tiny").with_(prompt_len=40, **extras)
-    worst, bits, toks, fins = _parity_from_common_state(cfg, 0, n_steps=10, concat=concat)
+    worst, bits, toks, fins = _parity_from_common_state(cfg, 0, n_steps=10, concat=concat, top_p=top_p)
     assert worst < TOL, worst
     assert bits[0] / bits[1] >= 0.995, bits
     assert toks[0] / toks[1] >= 0.8, toks
