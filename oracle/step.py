@@ -57,13 +57,15 @@ def prefill(w, cfg, prompts, page_table, num_pages, head_page_table, head_num_pa
             temperature=1.0, seed=0, round_interface=True) -> BatchState:
     """Full causal forward over each prompt; samples the first response token (slot FINAL of
     step 0), fills the head cache from the pairs (H_{i-1}, x_i), i = 1..P-1, and leaves the
-    pair (H_{P-1}, x_P) pending."""
-    B, P = prompts.shape
+    pair (H_{P-1}, x_P) pending.  ``prompts`` is a [B, P] array or a list of B token
+    sequences of different lengths (each at least one token)."""
+    B = len(prompts)
     kv = PagedKV(cfg.n_layers, cfg.n_kv_heads, cfg.head_dim, page_table, num_pages, cfg.page_size)
     hkv = PagedKV(1, cfg.n_kv_heads, cfg.head_dim, head_page_table, head_num_pages, cfg.page_size)
     seqs = []
     for b in range(B):
         toks = [int(t) for t in prompts[b]]
+        P = len(toks)
         H = target_forward(w, toks, np.arange(P), kv, b, cfg)
         H = _maybe_round(H, round_interface)
         logits = _maybe_round(target_logits(w, H[-1:], cfg), round_interface)

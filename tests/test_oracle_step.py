@@ -28,6 +28,33 @@ def test_prefill_state():
     assert st.step == 1
 
 
+def test_ragged_prefill_equals_each_sequence_alone():
+    """Prompts of different lengths: every sequence ends in the state it reaches when prefilled on its own
+    (own first token, own pending pair, own cache rows), and the head cache holds pairs 1..P-1 at positions 0..P-2."""
+    w = perturb_norm_weights(make_weights(CFG, 0))
+    rng = np.random.default_rng(3)
+    prompts = [rng.integers(0, CFG.vocab, n) for n in (1, 7, 20)]
+    pt, npg = make_page_tables(np.full(3, 64), CFG.page_size, seed=7)
+    hpt, hnpg = make_page_tables(np.full(3, 64), CFG.page_size, seed=8)
+    st = step.prefill(w, CFG, prompts, pt, npg, hpt, hnpg, seed=5, round_interface=False)
+    for b, pr in enumerate(prompts):
+        s = st.seqs[b]
+        assert s.tokens[:-1] == [int(t) for t in pr] and s.kv_len == len(pr) and len(s.pending_tok) == 1
+        kv1 = model.PagedKV(CFG.n_layers, CFG.n_kv_heads, CFG.head_dim, pt[b:b + 1], npg)
+        H = model.target_forward(w, pr, np.arange(len(pr)), kv1, 0, CFG)
+        np.testing.assert_allclose(s.pending_hidden[0], H[-1], rtol=1e-12)
+        p = sampler.softmax_probs(model.target_logits(w, H[-1:], CFG)[0])
+        assert s.tokens[-1] == sampler.draw_token(p, philox.u24(5, 0, b, philox.SLOT_FINAL))[0]
+        for l in range(CFG.n_layers):
+            for a, c in zip(st.kv.gather(l, b, len(pr)), kv1.gather(l, 0, len(pr))):
+                np.testing.assert_allclose(a, c, rtol=1e-12)
+        if len(pr) > 1:
+            hk1 = model.PagedKV(1, CFG.n_kv_heads, CFG.head_dim, hpt[b:b + 1], hnpg)
+            model.head_forward(w, H[:-1], pr[1:], np.arange(len(pr) - 1), hk1, 0, CFG)
+            for a, c in zip(st.hkv.gather(0, b, len(pr) - 1), hk1.gather(0, 0, len(pr) - 1)):
+                np.testing.assert_allclose(a, c, rtol=1e-12)
+
+
 def test_cycle_invariants_and_restart_cache_composition():
     """After several cycles: every cycle commits between 1 and K+1 tokens; the target cache and the
     head cache BEHIND the boundary equal those of a fresh pass over the committed sequence that
