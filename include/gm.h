@@ -130,6 +130,25 @@ typedef struct {
 int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_stream);
 void gm_destroy(gm_ctx *ctx);
 
+/* Prompt prefill: the state a rollout starts from (App. B.2: prompts of at most 1024 tokens; App. D.2:
+ * the rollout-time hidden states of the prompt prefill the draft head).  For every sequence b with prompt
+ * x[0..L_b-1], L_b = prompt_len[b]:
+ *   - the backbone runs causally over the prompt and fills target-cache positions 0..L_b-1;
+ *   - the draft head runs over the pairs (H_{i-1}, x_i), i = 1..L_b-1, filling head-cache positions 0..L_b-2;
+ *   - the first response token x[L_b] is drawn from softmax(logits(H_{L_b-1}) / T) with the uniform
+ *     u24_first[b], or Philox (key = seed, counter = (slot 16 >> 2, row, 0, 0)) when u24_first is NULL;
+ *   - kv_len[b] = L_b, pending_n[b] = 1, pending pair = (H_{L_b-1}, x[L_b]).
+ * The prompts are processed max_k + 1 positions per sequence and pass, every pass through the kernels of the
+ * verify and draft phases; ceil(max_prompt_len / (max_k + 1)) passes.
+ *   prompt_tok  device int32 [B, prompt_stride], row b holds L_b tokens;  prompt_len device int32 [B];
+ *   max_prompt_len  host value >= every L_b (a longer or empty prompt raises GM_ERR_KV_CAPACITY in
+ *                   gm_last_status and its sequence is left untouched);
+ *   first_token device int32 [B] out or NULL;  dbg_p fp32 [B, V] out or NULL (the distributions drawn from).
+ * The page tables of `st` must cover max_prompt_len + max_k + 1 positions (else GM_ERR_KV_CAPACITY).     */
+int gm_prefill(gm_ctx *ctx, gm_state *st, const int32_t *prompt_tok, const int32_t *prompt_len,
+               int prompt_stride, int max_prompt_len, float temperature, const uint32_t *u24_first,
+               uint64_t seed, int32_t *first_token, float *dbg_p);
+
 /* Draft phase (App. E, restart equations).  Application 1 runs the head over the pending pairs,
  * overwriting head-cache entries of the previous chain; applications 2..k feed the head its own
  * output and the previous draft.  After each application q_j = softmax(logits / T) and d_j is

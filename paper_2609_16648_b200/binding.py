@@ -22,7 +22,7 @@ GM_MAX_K, GM_PAGE = 7, 16
 GM_FLAG_SIMPLE_GEMM, GM_FLAG_SAMPLER_CLUSTER, GM_FLAG_SAMPLER_STREAM = 1, 2, 4
 GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER, GM_KC_RECORD = 0, 1, 2, 3, 4
 
-EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw", "gm_set_top_p", "gm_nucleus",
+EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw", "gm_set_top_p", "gm_nucleus", "gm_prefill",
            "gm_spec_step_host", "gm_gemm", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
            "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
@@ -79,6 +79,7 @@ def lib() -> C.CDLL:
     L.gm_spec_step_host.argtypes = [vp, C.POINTER(gm_state), i32, f32, u64, u64, vp, vp, vp, vp, vp]
     L.gm_draw.argtypes = [vp, vp, i32, f32, vp, vp, vp]
     L.gm_set_top_p.argtypes = [vp, f32]
+    L.gm_prefill.argtypes = [vp, C.POINTER(gm_state), vp, vp, i32, i32, f32, vp, u64, vp, vp]
     L.gm_nucleus.argtypes = [vp, vp, i32, f32, f32, vp, vp]
     L.gm_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
     L.gm_attention.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, i32, i32, vp]
@@ -301,6 +302,13 @@ def gm_spec_step_host(ctx: Context, st: State, k: int, temperature: float, seed:
 
 def gm_draw(ctx: Context, logits, rows: int, temperature: float, u24, out_tok, dbg_prob=None):
     _check(lib().gm_draw(ctx.handle, _p(logits), rows, temperature, _p(u24), _p(out_tok), _p(dbg_prob)), "gm_draw")
+
+
+def gm_prefill(ctx: Context, st, prompt_tok, prompt_len, max_prompt_len: int, temperature: float, u24_first, seed: int,
+               first_token=None, dbg_p=None):
+    """prompt_tok int32 [B, stride] and prompt_len int32 [B] on the device; max_prompt_len a host integer."""
+    _check(lib().gm_prefill(ctx.handle, C.byref(st.struct()), _p(prompt_tok), _p(prompt_len), prompt_tok.shape[1],
+                            max_prompt_len, temperature, _p(u24_first), seed, _p(first_token), _p(dbg_p)), "gm_prefill")
 
 
 def gm_set_top_p(ctx: Context, top_p: float):

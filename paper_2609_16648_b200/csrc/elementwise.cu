@@ -63,8 +63,13 @@ __global__ void plan_kernel(const PlanArgs A) {
     int qn, qbase;
     if (A.mode == PHASE_VERIFY) { qn = A.k_or_j + 1; qbase = len; }
     else if (A.mode == PHASE_DRAFT_FIRST) { qn = A.pending_n[b]; qbase = len - qn; }
+    else if (A.mode == PHASE_CHUNK) { qn = A.row_n[b]; qbase = A.k_or_j; }
     else { qn = 1; qbase = len + A.k_or_j - 2; }
     bool ok = qn >= 1 && qbase >= 0 && qbase + qn <= A.max_pages_per_seq * 16;
+    if (A.mode == PHASE_CHUNK) {
+      if (qn == 0) { A.qn[b] = 0; A.qbase[b] = 0; pages[b] = 0; continue; }      // sits this pass out
+      ok = ok && qn <= A.QT;
+    }
     if (A.mode == PHASE_DRAFT_FIRST) ok = ok && qn <= A.k_or_j;     // k_or_j carries max_k + 1 here
     if (!ok) { set_status(A.status, ST_KV_CAPACITY); qn = 0; qbase = 0; }
     A.qn[b] = qn;
@@ -81,6 +86,87 @@ __global__ void plan_kernel(const PlanArgs A) {
 cudaError_t launch_plan(const PlanArgs &A, cudaStream_t stream) {
   if (A.batch > 1024) return cudaErrorInvalidValue;
   return launch_k(plan_kernel, dim3(1), dim3(256), 0, stream, 1, A);
+}
+
+// ---- prompt prefill: chunk bookkeeping ----------------------------------------------------------------------
+__global__ void chunk_setup_kernel(const ChunkSetupArgs A) {
+  pdl_prologue();
+  for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < A.batch; b += gridDim.x * blockDim.x) {
+    const int L = A.prompt_len[b];
+    const bool bad = L < 1 || L > A.max_len || L > A.stride;
+    if (bad && A.base == 0) set_status(A.status, ST_KV_CAPACITY);
+    const int n = bad ? 0 : min(max(L - A.base, 0), A.QT);
+    const int hn = bad ? 0 : min(max(L - 1 - A.base, 0), A.QT);
+    A.row_n[b] = n;
+    A.head_n[b] = hn;
+    for (int j = 0; j < A.QT; ++j)
+      A.pair_tok[b * A.pair_stride + j] = j < hn ? A.prompt_tok[static_cast<size_t>(b) * A.stride + A.base + j + 1] : 0;
+  }
+}
+cudaError_t launch_chunk_setup(const ChunkSetupArgs &A, cudaStream_t stream) {
+  return launch_k(chunk_setup_kernel, dim3((A.batch + 127) / 128), dim3(128), 0, stream, 1, A);
+}
+
+__global__ void __launch_bounds__(EW_THREADS)
+embed_chunk_kernel(const __nv_bfloat16 *embed, const __nv_bfloat16 *w, const int32_t *prompt_tok, int stride, int base,
+                   const int32_t *row_n, int QT, int d, int vocab, float eps, float *x, __nv_bfloat16 *xn,
+                   uint32_t *status) {
+  const int m = blockIdx.x, b = m / QT, j = m % QT;
+  pdl_prologue();
+  int tok = j < row_n[b] ? prompt_tok[static_cast<size_t>(b) * stride + base + j] : 0;
+  if (tok < 0 || tok >= vocab) { if (threadIdx.x == 0) set_status(status, ST_BAD_TOKEN); tok = 0; }
+  const int d4 = d >> 2;
+  float4 v[EW_MAXC];
+#pragma unroll
+  for (int c = 0; c < EW_MAXC; ++c) {
+    const int i = threadIdx.x + c * EW_THREADS;
+    if (i < d4) {
+      v[c] = load_bf16x4(embed + static_cast<size_t>(tok) * d + 4 * i);
+      reinterpret_cast<float4 *>(x + static_cast<size_t>(m) * d)[i] = v[c];
+    }
+  }
+  rmsnorm_store(v, d4, d, eps, w, xn + static_cast<size_t>(m) * d);
+}
+cudaError_t launch_embed_chunk(const __nv_bfloat16 *embed, const __nv_bfloat16 *w, const int32_t *prompt_tok, int stride,
+                               int base, const int32_t *row_n, int batch, int QT, int d, int vocab, float eps, float *x,
+                               __nv_bfloat16 *xn, uint32_t *status, cudaStream_t stream) {
+  return launch_k(embed_chunk_kernel, dim3(batch * QT), dim3(EW_THREADS), 0, stream, 1, embed, w, prompt_tok, stride,
+                  base, row_n, QT, d, vocab, eps, x, xn, status);
+}
+
+__global__ void __launch_bounds__(EW_THREADS)
+prefill_last_kernel(const float *x, const __nv_bfloat16 *hidden, const int32_t *row_n, const int32_t *prompt_len,
+                    int base, int QT, int d, int pend_stride, float *xlast, __nv_bfloat16 *pending_hidden) {
+  const int b = blockIdx.x;
+  pdl_prologue();
+  const int n = row_n[b];
+  if (n < 1 || base + n != prompt_len[b]) return;
+  const size_t m = static_cast<size_t>(b) * QT + n - 1;
+  for (int i = threadIdx.x; i < d; i += EW_THREADS) {
+    xlast[static_cast<size_t>(b) * d + i] = x[m * d + i];
+    pending_hidden[static_cast<size_t>(b) * pend_stride * d + i] = hidden[m * d + i];
+  }
+}
+cudaError_t launch_prefill_last(const float *x, const __nv_bfloat16 *hidden, const int32_t *row_n,
+                                const int32_t *prompt_len, int batch, int base, int QT, int d, int pend_stride,
+                                float *xlast, __nv_bfloat16 *pending_hidden, cudaStream_t stream) {
+  return launch_k(prefill_last_kernel, dim3(batch), dim3(EW_THREADS), 0, stream, 1, x, hidden, row_n, prompt_len, base,
+                  QT, d, pend_stride, xlast, pending_hidden);
+}
+
+__global__ void prefill_finish_kernel(const int32_t *prompt_len, const int32_t *first_tok, int batch, int pend_stride,
+                                      int32_t *kv_len, int32_t *pending_n, int32_t *pending_tok) {
+  pdl_prologue();
+  for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < batch; b += gridDim.x * blockDim.x) {
+    kv_len[b] = prompt_len[b];
+    pending_n[b] = 1;
+    pending_tok[b * pend_stride] = first_tok[b];
+  }
+}
+cudaError_t launch_prefill_finish(const int32_t *prompt_len, const int32_t *first_tok, int batch, int pend_stride,
+                                  int32_t *kv_len, int32_t *pending_n, int32_t *pending_tok, cudaStream_t stream) {
+  return launch_k(prefill_finish_kernel, dim3((batch + 127) / 128), dim3(128), 0, stream, 1, prompt_len, first_tok, batch,
+                  pend_stride, kv_len, pending_n, pending_tok);
 }
 
 // ---- embedding gather + first RMSNorm of the verify forward ------------------------------------------------

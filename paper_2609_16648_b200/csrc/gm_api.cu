@@ -61,6 +61,10 @@ struct gm_ctx {
   int32_t *qn = nullptr, *qbase = nullptr, *page_start = nullptr;
   float2 *rope = nullptr;
   uint32_t *status = nullptr;
+  // prompt prefill: per-chunk bookkeeping, the chunk's hidden states, the row of each prompt's last token
+  int32_t *pf_row_n = nullptr, *pf_head_n = nullptr, *pf_pair_tok = nullptr, *pf_first = nullptr;
+  __nv_bfloat16 *pf_hidden = nullptr;
+  float *pf_xlast = nullptr;
   float top_p = 1.f;                    // nucleus of the target distributions (1 = none)
   __nv_bfloat16 *ws_nucleus = nullptr;  // [max_batch (max_k + 1)][V] filtered target rows, allocated by gm_set_top_p
   std::vector<void *> allocs;
@@ -303,6 +307,15 @@ int run_plan(gm_ctx *c, const gm_state *st, int mode, int k_or_j) {
   return GM_OK;
 }
 
+int run_plan_chunk(gm_ctx *c, int batch, const int32_t *row_n, int base, int QT) {
+  PlanArgs P;
+  P.mode = PHASE_CHUNK; P.batch = batch; P.k_or_j = base; P.max_pages_per_seq = c->cfg.max_pages_per_seq;
+  P.n_ctas = c->sm_count; P.kv_len = row_n; P.pending_n = row_n; P.row_n = row_n; P.QT = QT; P.qn = c->qn; P.qbase = c->qbase;
+  P.page_start = c->page_start; P.status = c->status;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_plan(P, c->stream));
+  return GM_OK;
+}
+
 int check_state(const gm_ctx *c, const gm_state *st, int k) {
   if (!c || !st) return GM_ERR_INVALID_ARG;
   if (k < 1 || k > c->cfg.max_k) return k > c->cfg.max_k ? GM_ERR_UNSUPPORTED : GM_ERR_INVALID_ARG;
@@ -448,6 +461,12 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
   A_(dev_alloc(c, &c->qn, B));
   A_(dev_alloc(c, &c->qbase, B));
   A_(dev_alloc(c, &c->page_start, B + 1));
+  A_(dev_alloc(c, &c->pf_row_n, B));
+  A_(dev_alloc(c, &c->pf_head_n, B));
+  A_(dev_alloc(c, &c->pf_first, B));
+  A_(dev_alloc(c, &c->pf_pair_tok, B * (cfg->max_k + 1)));
+  A_(dev_alloc(c, &c->pf_hidden, M * c->d));
+  A_(dev_alloc(c, &c->pf_xlast, B * c->d));
   A_(dev_alloc(c, &c->status, 1));
   // rotary table: cos/sin of pos * base^(-2i/hd), computed in double precision on the host
   {
@@ -559,6 +578,83 @@ int gm_verify(gm_ctx *c, const gm_state *st, int k, const int32_t *draft_tok, vo
 }
 
 static int run_nucleus(gm_ctx *c, const void *logits, int rows, float temperature, float top_p, void *out, float *dbg_e);
+
+int gm_prefill(gm_ctx *c, gm_state *st, const int32_t *prompt_tok, const int32_t *prompt_len, int prompt_stride,
+               int max_prompt_len, float temperature, const uint32_t *u24_first, uint64_t seed, int32_t *first_token,
+               float *dbg_p) {
+  int rc = check_state(c, st, 1);
+  if (rc) return rc;
+  if (!prompt_tok || !prompt_len || max_prompt_len < 1 || prompt_stride < max_prompt_len) return GM_ERR_INVALID_ARG;
+  const gm_config &cf = c->cfg;
+  if (max_prompt_len + cf.max_k + 1 > cf.max_pages_per_seq * GM_PAGE) return GM_ERR_KV_CAPACITY;
+  SamplerArgs S;
+  if ((rc = fill_sampler(c, S, temperature)) != GM_OK) return rc;
+  const int B = st->batch, QT = cf.max_k + 1;
+  PhaseShape ph;
+  ph.B = B; ph.QT = QT; ph.M = B * QT; ph.qrows = round16(QT * c->group);
+  CUtensorMap kvm, hkvm;
+  if ((rc = kv_map(c, st->kv_pool, cf.n_layers, cf.num_pages, &kvm)) != GM_OK) return rc;
+  if ((rc = kv_map(c, st->head_kv_pool, 1, cf.head_num_pages, &hkvm)) != GM_OK) return rc;
+  for (int base = 0; base < max_prompt_len; base += QT) {
+    ChunkSetupArgs Cs;
+    Cs.prompt_tok = prompt_tok; Cs.prompt_len = prompt_len; Cs.batch = B; Cs.stride = prompt_stride; Cs.base = base;
+    Cs.QT = QT; Cs.max_len = max_prompt_len; Cs.pair_stride = QT; Cs.row_n = c->pf_row_n; Cs.head_n = c->pf_head_n;
+    Cs.pair_tok = c->pf_pair_tok; Cs.status = c->status;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_chunk_setup(Cs, c->stream));
+    // the backbone over positions base .. base + QT - 1 of every prompt that reaches them
+    if ((rc = run_plan_chunk(c, B, c->pf_row_n, base, QT)) != GM_OK) return rc;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+              launch_embed_chunk(static_cast<const __nv_bfloat16 *>(c->w.embed),
+                                 static_cast<const __nv_bfloat16 *>(c->layers[0].ln1), prompt_tok, prompt_stride, base,
+                                 c->pf_row_n, B, QT, c->d, c->V, cf.rms_eps, c->x, c->xn, c->status, c->stream));
+    for (int l = 0; l < cf.n_layers; ++l) {
+      const bool last = l + 1 == cf.n_layers;
+      rc = run_layer(c, c->layers[l], c->lmaps[l], ph, kvm, static_cast<__nv_bfloat16 *>(st->kv_pool), l, cf.num_pages,
+                     st->page_table, last ? nullptr : static_cast<const __nv_bfloat16 *>(c->layers[l + 1].ln1),
+                     last ? c->pf_hidden : nullptr);
+      if (rc) return rc;
+    }
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+              launch_prefill_last(c->x, c->pf_hidden, c->pf_row_n, prompt_len, B, base, QT, c->d, QT, c->pf_xlast,
+                                  static_cast<__nv_bfloat16 *>(st->pending_hidden), c->stream));
+    // the draft head over the pairs (hidden of position t, token t + 1) of the same chunk, at head positions t
+    if (base + 1 < max_prompt_len) {
+      if ((rc = run_plan_chunk(c, B, c->pf_head_n, base, QT)) != GM_OK) return rc;
+      HeadInputArgs H;
+      H.mode = PHASE_DRAFT_FIRST; H.batch = B; H.QT = QT; H.d = c->d; H.vocab = c->V; H.max_k = cf.max_k; H.k = 1; H.j = 1;
+      H.eps = cf.rms_eps; H.embed = static_cast<const __nv_bfloat16 *>(c->w.embed);
+      H.we = static_cast<const __nv_bfloat16 *>(c->w.head_enorm); H.wh = static_cast<const __nv_bfloat16 *>(c->w.head_hnorm);
+      H.pending_tok = c->pf_pair_tok; H.pending_n = c->pf_head_n; H.pending_hidden = c->pf_hidden; H.draft_tok = nullptr;
+      H.g_prev = c->g; H.zin = c->zin; H.status = c->status;
+      GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_head_input(H, c->stream));
+      rc = run_gemm(c, c->zin, c->Mmax, &c->head_proj_map, static_cast<const __nv_bfloat16 *>(c->w.head_proj), ph.M, c->d,
+                    2 * c->d, c->x, EPI_STORE_F32, c->d);
+      if (rc) return rc;
+      GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+                launch_rmsnorm(c->x, static_cast<const __nv_bfloat16 *>(c->w.head_layer.ln1), c->xn, nullptr, ph.M, c->d,
+                               cf.rms_eps, c->stream));
+      rc = run_layer(c, c->w.head_layer, c->head_maps, ph, hkvm, static_cast<__nv_bfloat16 *>(st->head_kv_pool), 0,
+                     cf.head_num_pages, st->head_page_table, nullptr, nullptr);
+      if (rc) return rc;
+    }
+  }
+  // first response token: final norm + LM head on the hidden state of each prompt's last token, one draw per sequence
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+            launch_rmsnorm(c->pf_xlast, static_cast<const __nv_bfloat16 *>(c->w.final_norm), c->xn, nullptr, B, c->d,
+                           cf.rms_eps, c->stream));
+  rc = run_gemm(c, c->xn, c->Mmax, &c->lm_head_map, static_cast<const __nv_bfloat16 *>(c->w.lm_head), B, c->V, c->d,
+                c->ws_target_logits, EPI_STORE_BF16, c->V);
+  if (rc) return rc;
+  S.K = 0; S.target_logits = c->ws_target_logits; S.tgt_bstride = c->V; S.draft_logits = nullptr;
+  S.u24 = u24_first; S.u_stride = 1; S.seed = seed; S.step = 0; S.slot_final = SLOT_FINAL;
+  S.accept_len = nullptr; S.next_token = c->pf_first; S.tok_out_stride = 1; S.dbg_p = dbg_p; S.dbg_q = nullptr; S.commit = 0;
+  GM_LAUNCH(c, GM_KC_SAMPLER, run_sampler(c, S, B));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+            launch_prefill_finish(prompt_len, c->pf_first, B, QT, st->kv_len, st->pending_n, st->pending_tok, c->stream));
+  if (first_token)
+    GM_CUDA(c, cudaMemcpyAsync(first_token, c->pf_first, sizeof(int32_t) * B, cudaMemcpyDeviceToDevice, c->stream));
+  return GM_OK;
+}
 
 int gm_accept(gm_ctx *c, gm_state *st, int batch, int k, float temperature, const void *target_logits,
               const void *draft_logits, const int32_t *draft_tok, const uint32_t *u24_accept, uint64_t seed,

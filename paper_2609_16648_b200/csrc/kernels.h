@@ -97,16 +97,43 @@ struct NucleusArgs {
 cudaError_t launch_nucleus(const NucleusArgs &A, cudaStream_t stream);
 
 // ---- planning: query ranges of a phase and the balanced attention partition --------------------------
-enum PhaseMode { PHASE_VERIFY = 0, PHASE_DRAFT_FIRST = 1, PHASE_DRAFT_NEXT = 2 };
+enum PhaseMode { PHASE_VERIFY = 0, PHASE_DRAFT_FIRST = 1, PHASE_DRAFT_NEXT = 2, PHASE_CHUNK = 3 };
 struct PlanArgs {
-  int mode, batch, k_or_j;              // VERIFY: K;  DRAFT_NEXT: application index j (2..K)
+  int mode, batch, k_or_j;              // VERIFY: K;  DRAFT_NEXT: application index j (2..K);  CHUNK: first position
   int max_pages_per_seq, n_ctas;
   const int32_t *kv_len, *pending_n;
+  const int32_t *row_n = nullptr;       // CHUNK: queries per sequence (0 = the sequence sits this pass out)
+  int QT = 0;                           // CHUNK: most queries a sequence may have
   int32_t *qn, *qbase;                  // [B] queries of this phase and the position of the first one
   int32_t *page_start;                  // [B+1] exclusive prefix of pages attended per sequence
   uint32_t *status;
 };
 cudaError_t launch_plan(const PlanArgs &A, cudaStream_t stream);
+
+// ---- prompt prefill in chunks of QT positions per sequence ------------------------------------------------
+// Chunk `base / QT` of every prompt: row_n[b] = positions of prompt b inside [base, base + QT) (0 when the prompt
+// ended before), head_n[b] = how many of them have a successor token inside the prompt (the pairs the draft head
+// is prefilled with), pair_tok[b][j] = token at position base + j + 1.  A prompt shorter than 1 or longer than
+// max_len raises ST_KV_CAPACITY and sits out.
+struct ChunkSetupArgs {
+  const int32_t *prompt_tok, *prompt_len;
+  int batch, stride, base, QT, max_len, pair_stride;
+  int32_t *row_n, *head_n, *pair_tok;
+  uint32_t *status;
+};
+cudaError_t launch_chunk_setup(const ChunkSetupArgs &A, cudaStream_t stream);
+// x[m] = embed[prompt_tok[b][base + j]] (fp32), xn[m] = RMSNorm(x[m]; w) (bf16) for j < row_n[b]; other rows token 0.
+cudaError_t launch_embed_chunk(const __nv_bfloat16 *embed, const __nv_bfloat16 *w, const int32_t *prompt_tok, int stride,
+                               int base, const int32_t *row_n, int batch, int QT, int d, int vocab, float eps, float *x,
+                               __nv_bfloat16 *xn, uint32_t *status, cudaStream_t stream);
+// For the sequences whose prompt ends inside this chunk: xlast[b] = x[row of the last prompt token] (fp32) and
+// pending_hidden[b][0] = the same row of `hidden` (bf16).
+cudaError_t launch_prefill_last(const float *x, const __nv_bfloat16 *hidden, const int32_t *row_n,
+                                const int32_t *prompt_len, int batch, int base, int QT, int d, int pend_stride,
+                                float *xlast, __nv_bfloat16 *pending_hidden, cudaStream_t stream);
+// kv_len[b] = prompt_len[b], pending_n[b] = 1, pending_tok[b][0] = first_tok[b].
+cudaError_t launch_prefill_finish(const int32_t *prompt_len, const int32_t *first_tok, int batch, int pend_stride,
+                                  int32_t *kv_len, int32_t *pending_n, int32_t *pending_tok, cudaStream_t stream);
 
 // ---- element-wise --------------------------------------------------------------------------------------
 // x[m] = embed[token(m)] (fp32), xn[m] = RMSNorm(x[m]; w) (bf16); rows m = b*QT + j of the verify phase.
