@@ -146,3 +146,49 @@ def spec_step(w, cfg, st: BatchState, K: int, temperature: float = 1.0, seed: in
     if do_commit:
         st.step += 1
     return {k: np.array(v) for k, v in out.items()}
+
+
+# ---- a whole rollout: cycles until every response has ended --------------------------------------------
+#
+# Responses are capped (App. B.2: 8192 tokens, 16384 for one model).  A response is the token the prefill
+# drew followed by the tokens each cycle commits; it ends with the first end-of-sequence token (kept) or when
+# it reaches the cap; what a cycle commits beyond either is dropped.  A finished sequence sits out the remaining
+# cycles with its state frozen.  A row's uniforms depend on (seed, step, row) only, so the others are unaffected.
+
+RUNNING, HIT_EOS, HIT_CAP = 0, 1, 2
+
+
+def append_committed(response: list, new_tokens, eos: int, max_new: int) -> int:
+    """Append a cycle's committed tokens to ``response``; returns RUNNING, HIT_EOS or HIT_CAP."""
+    if len(response) >= max_new:
+        return HIT_CAP
+    for t in new_tokens:
+        response.append(int(t))
+        if int(t) == eos:
+            return HIT_EOS
+        if len(response) >= max_new:
+            return HIT_CAP
+    return RUNNING
+
+
+def rollout(w, cfg, st: BatchState, K: int, temperature: float = 1.0, seed: int = 0, max_steps: int = 1 << 30,
+            eos: int = -1, max_new: int = 8192, round_interface: bool = True, top_p: float = 1.0):
+    """Run cycles from a prefilled state.  Returns (responses, status[B], cycles run)."""
+    B = len(st.seqs)
+    responses = [[] for _ in range(B)]
+    status = [append_committed(responses[b], [st.seqs[b].tokens[-1]], eos, max_new) for b in range(B)]
+    steps = 0
+    while steps < max_steps and any(s == RUNNING for s in status):
+        ud = philox.u24_draft(seed, st.step, B, K)
+        ua = philox.u24_accept(seed, st.step, B, K)
+        for b in range(B):
+            if status[b] != RUNNING:
+                continue
+            d, _, q = draft(w, cfg, st, b, K, temperature, ud[b], round_interface)
+            _, H, p = verify(w, cfg, st, b, d, temperature, round_interface, top_p)
+            a, t_star, _ = sampler.decide(p, q, d, ua[b])
+            commit(st, b, d, a, t_star, H)
+            status[b] = append_committed(responses[b], list(d[:a]) + [t_star], eos, max_new)
+        st.step += 1
+        steps += 1
+    return responses, status, steps

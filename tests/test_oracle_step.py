@@ -215,3 +215,42 @@ def test_forced_drafts_replay_the_recorded_path():
     np.testing.assert_allclose(alt["p"][:, 0], free["p"][:, 0], rtol=1e-12)
     assert np.abs(alt["q"][:, 1] - free["q"][:, 1]).max() > 1e-7
     assert np.abs(alt["p"][:, 1] - free["p"][:, 1]).max() > 1e-7
+
+
+# ---- whole rollouts: stopping rules -----------------------------------------------------------------------
+
+def test_append_committed_rules():
+    r = [5]
+    assert step.append_committed(r, [1, 2, 3], eos=9, max_new=10) == step.RUNNING and r == [5, 1, 2, 3]
+    assert step.append_committed(r, [4, 9, 7, 7], eos=9, max_new=10) == step.HIT_EOS and r == [5, 1, 2, 3, 4, 9]
+    r = [5, 1]
+    assert step.append_committed(r, [2, 3, 4], eos=9, max_new=4) == step.HIT_CAP and r == [5, 1, 2, 3]
+    assert step.append_committed(r, [8], eos=9, max_new=4) == step.HIT_CAP and r == [5, 1, 2, 3]
+    r = []
+    assert step.append_committed(r, [9], eos=9, max_new=1) == step.HIT_EOS and r == [9]      # EOS wins on the last slot
+    r = []
+    assert step.append_committed(r, [3], eos=-1, max_new=1) == step.HIT_CAP and r == [3]
+
+
+def test_rollout_is_the_concatenation_of_its_cycles_and_rows_are_independent():
+    """(a) With no stopping rule a rollout's responses are the committed tokens of plain cycles; (b) with a cap and
+    an end-of-sequence token each response is that stream cut by the rules; (c) a row's response does not depend
+    on when the other rows stop (rolled out alone it gives the same tokens)."""
+    w, st, _ = _setup(cap=160)
+    w2, st2, _ = _setup(cap=160)
+    resp, status, n = step.rollout(w, CFG, st, 3, seed=5, max_steps=6, eos=-1, max_new=1000, round_interface=False)
+    assert n == 6 and status == [step.RUNNING] * CFG.batch
+    for b, s in enumerate(st.seqs):
+        assert resp[b] == s.tokens[CFG.prompt_len:]
+    stream = [list(r) for r in resp]
+    eos = stream[0][4]                                   # a token row 0 emits early
+    resp2, status2, n2 = step.rollout(w2, CFG, st2, 3, seed=5, max_steps=6, eos=eos, max_new=11, round_interface=False)
+    for b in range(CFG.batch):
+        want = []
+        code = step.append_committed(want, stream[b], eos, 11)
+        assert resp2[b] == want and status2[b] == code
+    assert status2[0] == step.HIT_EOS and resp2[0][-1] == eos
+    assert n2 <= 6 and all(len(r) <= 11 for r in resp2)
+    # frozen state of a finished row: its committed tokens stop where its response stopped (up to the dropped tail)
+    for b, s in enumerate(st2.seqs):
+        assert s.tokens[CFG.prompt_len:CFG.prompt_len + len(resp2[b])] == resp2[b]
