@@ -149,6 +149,57 @@ int gm_prefill(gm_ctx *ctx, gm_state *st, const int32_t *prompt_tok, const int32
                int prompt_stride, int max_prompt_len, float temperature, const uint32_t *u24_first,
                uint64_t seed, int32_t *first_token, float *dbg_p);
 
+/* ---- A whole rollout: cycles until every response has ended (App. B.2: responses capped at 8192 / 16384
+ * tokens).  A response is the token the prefill drew followed by what each cycle commits; it ends with the
+ * first eos_token (kept) or when it holds max_new tokens; what a cycle commits beyond either is dropped.  A
+ * finished row sits out the remaining cycles: it gets no queries and no pages in any phase, the sampler
+ * skips it, and its state (kv_len, pending_*, caches) stays as it was.  A row's uniforms depend on seed,
+ * step and row only, so its response does not depend on when the others end - up to floating-point
+ * rounding in attention at scale: the pages of all running rows are cut into equal ranges over the SMs,
+ * so which partial results are merged for a row shifts when another row leaves (with fewer pages than
+ * SMs every range is one page and the results are bit-identical).  All pointers are device memory.      */
+typedef struct {
+  int32_t *out_tok;                 /* [B, out_stride] responses                                         */
+  int32_t *out_len;                 /* [B] tokens held by each response                                  */
+  int32_t *finished;                /* [B] 0 running, 1 ended with eos_token, 2 reached max_new          */
+  int32_t *n_running;               /* [1] rows still running after the last call                        */
+  int32_t  out_stride;              /* >= max_new                                                        */
+  int32_t  eos_token;               /* < 0: none                                                         */
+  int32_t  max_new;                 /* response cap, >= 1                                                */
+} gm_rollout;
+
+/* After gm_prefill (or with any state whose pending_tok[b][0] is the first response token): response b =
+ * [that token], finished / n_running set by the rules above.                                            */
+int gm_rollout_begin(gm_ctx *ctx, const gm_state *st, const gm_rollout *ro);
+/* One cycle (gm_spec_step) over the running rows, then the append of what it committed.  With the page
+ * allocator on (gm_pages_reset) it first reserves pages for kv_len + k + 1 positions of every running row
+ * and afterwards returns the pages of the rows that finished.                                           */
+int gm_rollout_step(gm_ctx *ctx, gm_state *st, const gm_rollout *ro, int k, float temperature,
+                    uint64_t seed, uint64_t step);
+/* Host loop: gm_rollout_step with step = first_step, first_step + 1, ... until no row is running or
+ * max_steps cycles ran.  n_running is read back (one stream synchronisation) every check_every cycles, so
+ * up to check_every - 1 cycles may run with every row sitting out.  steps_run / rows_running: host
+ * outputs, may be NULL.                                                                                 */
+int gm_rollout_run(gm_ctx *ctx, gm_state *st, const gm_rollout *ro, int k, float temperature,
+                   uint64_t seed, uint64_t first_step, int max_steps, int check_every,
+                   int32_t *steps_run, int32_t *rows_running);
+
+/* ---- Page allocator (the paper's serving engine allocates cache pages as sequences grow; no passage
+ * describes it).  The context keeps one stack of free page ids per pool (target, draft head).
+ *   gm_pages_reset    every page free, both page tables of `st` emptied (-1), switches the allocator on;
+ *   gm_pages_reserve  every row (finished[b] == 0 when finished is given) receives pages until its two
+ *                     tables cover length[b] + extra positions (length NULL = kv_len); a row that needs
+ *                     more than max_pages_per_seq pages, or an empty stack, raises GM_ERR_KV_CAPACITY in
+ *                     gm_last_status;
+ *   gm_pages_release  rows with finished[b] != 0 hand their pages back;
+ *   gm_pages_free_count  free pages per pool (host outputs; synchronises the stream).
+ * One thread walks the rows in order, so page assignment is the same on every run.  A context serves one
+ * state at a time while the allocator is on.                                                            */
+int gm_pages_reset(gm_ctx *ctx, gm_state *st);
+int gm_pages_reserve(gm_ctx *ctx, gm_state *st, const int32_t *length, int extra, const int32_t *finished);
+int gm_pages_release(gm_ctx *ctx, gm_state *st, const int32_t *finished);
+int gm_pages_free_count(gm_ctx *ctx, int32_t *target_free, int32_t *head_free);
+
 /* Draft phase (App. E, restart equations).  Application 1 runs the head over the pending pairs,
  * overwriting head-cache entries of the previous chain; applications 2..k feed the head its own
  * output and the previous draft.  After each application q_j = softmax(logits / T) and d_j is

@@ -23,6 +23,8 @@ GM_FLAG_SIMPLE_GEMM, GM_FLAG_SAMPLER_CLUSTER, GM_FLAG_SAMPLER_STREAM = 1, 2, 4
 GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER, GM_KC_RECORD = 0, 1, 2, 3, 4
 
 EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw", "gm_set_top_p", "gm_nucleus", "gm_prefill",
+           "gm_rollout_begin", "gm_rollout_step", "gm_rollout_run", "gm_pages_reset", "gm_pages_reserve",
+           "gm_pages_release", "gm_pages_free_count",
            "gm_spec_step_host", "gm_gemm", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
            "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
@@ -52,6 +54,11 @@ class gm_state(C.Structure):
                 ("pending_tok", C.c_void_p), ("pending_hidden", C.c_void_p)]
 
 
+class gm_rollout(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("out_tok", "out_len", "finished", "n_running")] + \
+               [(n, C.c_int32) for n in ("out_stride", "eos_token", "max_new")]
+
+
 class gm_record(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("start_hidden", "start_pos", "drafts", "top_logprob", "top_index", "accepted")]
 
@@ -79,6 +86,14 @@ def lib() -> C.CDLL:
     L.gm_spec_step_host.argtypes = [vp, C.POINTER(gm_state), i32, f32, u64, u64, vp, vp, vp, vp, vp]
     L.gm_draw.argtypes = [vp, vp, i32, f32, vp, vp, vp]
     L.gm_set_top_p.argtypes = [vp, f32]
+    L.gm_rollout_begin.argtypes = [vp, C.POINTER(gm_state), C.POINTER(gm_rollout)]
+    L.gm_rollout_step.argtypes = [vp, C.POINTER(gm_state), C.POINTER(gm_rollout), i32, f32, u64, u64]
+    L.gm_rollout_run.argtypes = [vp, C.POINTER(gm_state), C.POINTER(gm_rollout), i32, f32, u64, u64, i32, i32,
+                                 C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    L.gm_pages_reset.argtypes = [vp, C.POINTER(gm_state)]
+    L.gm_pages_reserve.argtypes = [vp, C.POINTER(gm_state), vp, i32, vp]
+    L.gm_pages_release.argtypes = [vp, C.POINTER(gm_state), vp]
+    L.gm_pages_free_count.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     L.gm_prefill.argtypes = [vp, C.POINTER(gm_state), vp, vp, i32, i32, f32, vp, u64, vp, vp]
     L.gm_nucleus.argtypes = [vp, vp, i32, f32, f32, vp, vp]
     L.gm_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
@@ -309,6 +324,62 @@ def gm_prefill(ctx: Context, st, prompt_tok, prompt_len, max_prompt_len: int, te
     """prompt_tok int32 [B, stride] and prompt_len int32 [B] on the device; max_prompt_len a host integer."""
     _check(lib().gm_prefill(ctx.handle, C.byref(st.struct()), _p(prompt_tok), _p(prompt_len), prompt_tok.shape[1],
                             max_prompt_len, temperature, _p(u24_first), seed, _p(first_token), _p(dbg_p)), "gm_prefill")
+
+
+class Rollout:
+    """Device tensors of struct gm_rollout."""
+
+    def __init__(self, batch: int, max_new: int, eos_token: int = -1, device="cuda"):
+        i32 = dict(device=device, dtype=torch.int32)
+        self.max_new, self.eos_token = max_new, eos_token
+        self.out_tok = torch.zeros((batch, max_new), **i32)
+        self.out_len = torch.zeros(batch, **i32)
+        self.finished = torch.zeros(batch, **i32)
+        self.n_running = torch.zeros(1, **i32)
+
+    def struct(self) -> gm_rollout:
+        return gm_rollout(self.out_tok.data_ptr(), self.out_len.data_ptr(), self.finished.data_ptr(),
+                          self.n_running.data_ptr(), self.out_tok.shape[1], self.eos_token, self.max_new)
+
+    def responses(self):
+        tok, n = self.out_tok.cpu().numpy(), self.out_len.cpu().numpy()
+        return [tok[b, :n[b]].tolist() for b in range(len(n))]
+
+
+def gm_rollout_begin(ctx: Context, st: State, ro: Rollout):
+    _check(lib().gm_rollout_begin(ctx.handle, C.byref(st.struct()), C.byref(ro.struct())), "gm_rollout_begin")
+
+
+def gm_rollout_step(ctx: Context, st: State, ro: Rollout, k: int, temperature: float, seed: int, step: int):
+    _check(lib().gm_rollout_step(ctx.handle, C.byref(st.struct()), C.byref(ro.struct()), k, temperature, seed, step),
+           "gm_rollout_step")
+
+
+def gm_rollout_run(ctx: Context, st: State, ro: Rollout, k: int, temperature: float, seed: int, first_step: int,
+                   max_steps: int, check_every: int = 8):
+    """Returns (cycles run, rows still running)."""
+    steps, running = C.c_int32(0), C.c_int32(0)
+    _check(lib().gm_rollout_run(ctx.handle, C.byref(st.struct()), C.byref(ro.struct()), k, temperature, seed, first_step,
+                                max_steps, check_every, C.byref(steps), C.byref(running)), "gm_rollout_run")
+    return steps.value, running.value
+
+
+def gm_pages_reset(ctx: Context, st: State):
+    _check(lib().gm_pages_reset(ctx.handle, C.byref(st.struct())), "gm_pages_reset")
+
+
+def gm_pages_reserve(ctx: Context, st: State, length, extra: int, finished=None):
+    _check(lib().gm_pages_reserve(ctx.handle, C.byref(st.struct()), _p(length), extra, _p(finished)), "gm_pages_reserve")
+
+
+def gm_pages_release(ctx: Context, st: State, finished):
+    _check(lib().gm_pages_release(ctx.handle, C.byref(st.struct()), _p(finished)), "gm_pages_release")
+
+
+def gm_pages_free_count(ctx: Context):
+    a, b = C.c_int32(0), C.c_int32(0)
+    _check(lib().gm_pages_free_count(ctx.handle, C.byref(a), C.byref(b)), "gm_pages_free_count")
+    return a.value, b.value
 
 
 def gm_set_top_p(ctx: Context, top_p: float):

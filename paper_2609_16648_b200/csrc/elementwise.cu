@@ -66,6 +66,7 @@ __global__ void plan_kernel(const PlanArgs A) {
     else if (A.mode == PHASE_CHUNK) { qn = A.row_n[b]; qbase = A.k_or_j; }
     else { qn = 1; qbase = len + A.k_or_j - 2; }
     bool ok = qn >= 1 && qbase >= 0 && qbase + qn <= A.max_pages_per_seq * 16;
+    if (A.finished && A.finished[b]) { A.qn[b] = 0; A.qbase[b] = 0; pages[b] = 0; continue; }    // sits the phase out
     if (A.mode == PHASE_CHUNK) {
       if (qn == 0) { A.qn[b] = 0; A.qbase[b] = 0; pages[b] = 0; continue; }      // sits this pass out
       ok = ok && qn <= A.QT;
@@ -86,6 +87,88 @@ __global__ void plan_kernel(const PlanArgs A) {
 cudaError_t launch_plan(const PlanArgs &A, cudaStream_t stream) {
   if (A.batch > 1024) return cudaErrorInvalidValue;
   return launch_k(plan_kernel, dim3(1), dim3(256), 0, stream, 1, A);
+}
+
+// ---- rollout bookkeeping ------------------------------------------------------------------------------------
+__global__ void rollout_append_kernel(const RolloutArgs A, int begin) {
+  __shared__ int running;
+  pdl_prologue();
+  if (threadIdx.x == 0) running = 0;
+  __syncthreads();
+  for (int b = threadIdx.x; b < A.batch; b += blockDim.x) {
+    int fin = begin ? 0 : A.finished[b];
+    int len = begin ? 0 : A.out_len[b];
+    if (!fin) {
+      const int n_new = begin ? 1 : A.accept_len[b] + 1;
+      int32_t *row = A.out_tok + static_cast<size_t>(b) * A.out_stride;
+      if (len >= A.max_new) fin = 2;
+      for (int i = 0; i < n_new && !fin; ++i) {
+        const int tok = begin ? A.pending_tok[b * A.pend_stride]
+                              : (i < n_new - 1 ? A.draft_tok[b * A.k + i] : A.next_token[b]);
+        row[len++] = tok;
+        if (tok == A.eos_token) fin = 1;
+        else if (len >= A.max_new) fin = 2;
+      }
+      A.out_len[b] = len;
+      A.finished[b] = fin;
+    }
+    if (!fin) atomicAdd(&running, 1);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) *A.n_running = running;
+}
+cudaError_t launch_rollout_append(const RolloutArgs &A, bool begin, cudaStream_t stream) {
+  return launch_k(rollout_append_kernel, dim3(1), dim3(256), 0, stream, 1, A, begin ? 1 : 0);
+}
+
+__global__ void page_reset_kernel(const PageAllocArgs A) {
+  pdl_prologue();
+  const int t = blockIdx.x * blockDim.x + threadIdx.x, n = gridDim.x * blockDim.x;
+  for (int i = t; i < A.num_pages; i += n) A.free_list[i] = A.num_pages - 1 - i;      // page 0 is handed out first
+  for (int i = t; i < A.batch * A.max_pages_per_seq; i += n) A.page_table[i] = -1;
+  for (int i = t; i < A.batch; i += n) A.held[i] = 0;
+  if (t == 0) *A.free_top = A.num_pages;
+}
+cudaError_t launch_page_reset(const PageAllocArgs &A, cudaStream_t stream) {
+  return launch_k(page_reset_kernel, dim3(64), dim3(256), 0, stream, 1, A);
+}
+__global__ void page_reserve_kernel(const PageAllocArgs A) {
+  pdl_prologue();
+  if (threadIdx.x != 0) return;
+  int top = *A.free_top;
+  for (int b = 0; b < A.batch; ++b) {
+    if (A.finished && A.finished[b]) continue;
+    const int need = (A.length[b] + A.extra + 15) >> 4;
+    int have = A.held[b];
+    if (need > A.max_pages_per_seq) { set_status(A.status, ST_KV_CAPACITY); continue; }
+    while (have < need) {
+      if (top <= 0) { set_status(A.status, ST_KV_CAPACITY); break; }
+      A.page_table[static_cast<size_t>(b) * A.max_pages_per_seq + have++] = A.free_list[--top];
+    }
+    A.held[b] = have;
+  }
+  *A.free_top = top;
+}
+cudaError_t launch_page_reserve(const PageAllocArgs &A, cudaStream_t stream) {
+  return launch_k(page_reserve_kernel, dim3(1), dim3(32), 0, stream, 1, A);
+}
+__global__ void page_release_kernel(const PageAllocArgs A) {
+  pdl_prologue();
+  if (threadIdx.x != 0) return;
+  int top = *A.free_top;
+  for (int b = 0; b < A.batch; ++b) {
+    if (!A.finished[b]) continue;
+    int32_t *row = A.page_table + static_cast<size_t>(b) * A.max_pages_per_seq;
+    for (int i = A.held[b] - 1; i >= 0; --i) {
+      if (top < A.num_pages) A.free_list[top++] = row[i];
+      row[i] = -1;
+    }
+    A.held[b] = 0;
+  }
+  *A.free_top = top;
+}
+cudaError_t launch_page_release(const PageAllocArgs &A, cudaStream_t stream) {
+  return launch_k(page_release_kernel, dim3(1), dim3(32), 0, stream, 1, A);
 }
 
 // ---- prompt prefill: chunk bookkeeping ----------------------------------------------------------------------

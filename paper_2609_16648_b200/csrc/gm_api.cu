@@ -65,6 +65,11 @@ struct gm_ctx {
   int32_t *pf_row_n = nullptr, *pf_head_n = nullptr, *pf_pair_tok = nullptr, *pf_first = nullptr;
   __nv_bfloat16 *pf_hidden = nullptr;
   float *pf_xlast = nullptr;
+  int32_t *ro_accept = nullptr, *ro_next = nullptr;   // per-step outputs of a rollout step
+  const int32_t *finished_mask = nullptr;   // set around the phases of a rollout step: rows that sit out
+  // page allocator (gm_pages_*): one stack of free page ids per pool
+  bool alloc_on = false;
+  int32_t *free_list[2] = {nullptr, nullptr}, *free_top[2] = {nullptr, nullptr}, *held[2] = {nullptr, nullptr};
   float top_p = 1.f;                    // nucleus of the target distributions (1 = none)
   __nv_bfloat16 *ws_nucleus = nullptr;  // [max_batch (max_k + 1)][V] filtered target rows, allocated by gm_set_top_p
   std::vector<void *> allocs;
@@ -302,7 +307,7 @@ int run_plan(gm_ctx *c, const gm_state *st, int mode, int k_or_j) {
   PlanArgs P;
   P.mode = mode; P.batch = st->batch; P.k_or_j = k_or_j; P.max_pages_per_seq = c->cfg.max_pages_per_seq;
   P.n_ctas = c->sm_count; P.kv_len = st->kv_len; P.pending_n = st->pending_n; P.qn = c->qn; P.qbase = c->qbase;
-  P.page_start = c->page_start; P.status = c->status;
+  P.page_start = c->page_start; P.status = c->status; P.finished = c->finished_mask;
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_plan(P, c->stream));
   return GM_OK;
 }
@@ -344,6 +349,7 @@ int fill_sampler(gm_ctx *c, SamplerArgs &S, float temperature) {
   S.status = c->status;
   S.slot_accept = SLOT_ACCEPT;
   S.slot_final = SLOT_FINAL;
+  S.finished = c->finished_mask;
   return GM_OK;
 }
 
@@ -461,6 +467,8 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
   A_(dev_alloc(c, &c->qn, B));
   A_(dev_alloc(c, &c->qbase, B));
   A_(dev_alloc(c, &c->page_start, B + 1));
+  A_(dev_alloc(c, &c->ro_accept, B));
+  A_(dev_alloc(c, &c->ro_next, B));
   A_(dev_alloc(c, &c->pf_row_n, B));
   A_(dev_alloc(c, &c->pf_head_n, B));
   A_(dev_alloc(c, &c->pf_first, B));
@@ -860,6 +868,132 @@ int gm_attention(gm_ctx *c, const void *q, const void *kv_pool, int pool_layers,
   Cb.n_kv = cf.n_kv_heads; Cb.group = c->group; Cb.hd = cf.head_dim; Cb.qrows = qrows; Cb.QT = q_stride;
   Cb.n_ctas = c->sm_count; Cb.out = static_cast<__nv_bfloat16 *>(out);
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_attention_combine(Cb, c->stream));
+  return GM_OK;
+}
+
+// ---- rollout driver and page allocator ------------------------------------------------------------------------------
+static int rollout_args_ok(const gm_ctx *c, const gm_state *st, const gm_rollout *ro) {
+  if (!c || !st || !ro || !ro->out_tok || !ro->out_len || !ro->finished || !ro->n_running) return GM_ERR_INVALID_ARG;
+  if (ro->max_new < 1 || ro->out_stride < ro->max_new) return GM_ERR_INVALID_ARG;
+  if (st->batch < 1 || st->batch > c->cfg.max_batch) return GM_ERR_INVALID_ARG;
+  return GM_OK;
+}
+
+static void fill_alloc(gm_ctx *c, gm_state *st, int pool, PageAllocArgs &P) {
+  P.batch = st->batch; P.max_pages_per_seq = c->cfg.max_pages_per_seq;
+  P.num_pages = pool ? c->cfg.head_num_pages : c->cfg.num_pages; P.extra = 0;
+  P.length = nullptr; P.finished = nullptr;
+  P.page_table = pool ? st->head_page_table : st->page_table;
+  P.held = c->held[pool]; P.free_list = c->free_list[pool]; P.free_top = c->free_top[pool]; P.status = c->status;
+}
+
+int gm_pages_reset(gm_ctx *c, gm_state *st) {
+  if (!c || !st || !st->page_table || !st->head_page_table || st->batch < 1 || st->batch > c->cfg.max_batch)
+    return GM_ERR_INVALID_ARG;
+  for (int pool = 0; pool < 2; ++pool) {
+    if (!c->free_list[pool]) {
+      int rc;
+      if ((rc = dev_alloc(c, &c->free_list[pool], pool ? c->cfg.head_num_pages : c->cfg.num_pages, false)) != GM_OK) return rc;
+      if ((rc = dev_alloc(c, &c->free_top[pool], 1)) != GM_OK) return rc;
+      if ((rc = dev_alloc(c, &c->held[pool], c->cfg.max_batch)) != GM_OK) return rc;
+    }
+    PageAllocArgs P;
+    fill_alloc(c, st, pool, P);
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_page_reset(P, c->stream));
+  }
+  c->alloc_on = true;
+  return GM_OK;
+}
+
+int gm_pages_reserve(gm_ctx *c, gm_state *st, const int32_t *length, int extra, const int32_t *finished) {
+  if (!c || !st || extra < 0) return GM_ERR_INVALID_ARG;
+  if (!c->alloc_on) return GM_ERR_INVALID_ARG;
+  for (int pool = 0; pool < 2; ++pool) {
+    PageAllocArgs P;
+    fill_alloc(c, st, pool, P);
+    P.length = length ? length : st->kv_len; P.extra = extra; P.finished = finished;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_page_reserve(P, c->stream));
+  }
+  return GM_OK;
+}
+
+int gm_pages_release(gm_ctx *c, gm_state *st, const int32_t *finished) {
+  if (!c || !st || !finished) return GM_ERR_INVALID_ARG;
+  if (!c->alloc_on) return GM_ERR_INVALID_ARG;
+  for (int pool = 0; pool < 2; ++pool) {
+    PageAllocArgs P;
+    fill_alloc(c, st, pool, P);
+    P.finished = finished;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_page_release(P, c->stream));
+  }
+  return GM_OK;
+}
+
+int gm_pages_free_count(gm_ctx *c, int32_t *target_free, int32_t *head_free) {
+  if (!c || !c->alloc_on) return GM_ERR_INVALID_ARG;
+  int32_t v[2] = {0, 0};
+  for (int pool = 0; pool < 2; ++pool)
+    GM_CUDA(c, cudaMemcpyAsync(&v[pool], c->free_top[pool], sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
+  GM_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (target_free) *target_free = v[0];
+  if (head_free) *head_free = v[1];
+  return GM_OK;
+}
+
+static void fill_rollout(const gm_ctx *c, const gm_state *st, const gm_rollout *ro, int k, RolloutArgs &R) {
+  R.batch = st->batch; R.k = k; R.out_stride = ro->out_stride; R.eos_token = ro->eos_token; R.max_new = ro->max_new;
+  R.pend_stride = c->cfg.max_k + 1; R.draft_tok = c->ws_draft_tok; R.accept_len = c->ro_accept; R.next_token = c->ro_next;
+  R.pending_tok = st->pending_tok; R.out_tok = ro->out_tok; R.out_len = ro->out_len; R.finished = ro->finished;
+  R.n_running = ro->n_running;
+}
+
+int gm_rollout_begin(gm_ctx *c, const gm_state *st, const gm_rollout *ro) {
+  int rc = rollout_args_ok(c, st, ro);
+  if (rc) return rc;
+  if (!st->pending_tok) return GM_ERR_INVALID_ARG;
+  RolloutArgs R;
+  fill_rollout(c, st, ro, 1, R);
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rollout_append(R, true, c->stream));
+  return GM_OK;
+}
+
+int gm_rollout_step(gm_ctx *c, gm_state *st, const gm_rollout *ro, int k, float temperature, uint64_t seed, uint64_t step) {
+  int rc = rollout_args_ok(c, st, ro);
+  if (rc) return rc;
+  if ((rc = check_state(c, st, k)) != GM_OK) return rc;
+  if (c->alloc_on && (rc = gm_pages_reserve(c, st, nullptr, k + 1, ro->finished)) != GM_OK) return rc;
+  c->finished_mask = ro->finished;
+  rc = spec_step_impl(c, st, k, temperature, nullptr, nullptr, seed, step, c->ro_accept, c->ro_next, c->ws_draft_tok);
+  c->finished_mask = nullptr;
+  if (rc) return rc;
+  RolloutArgs R;
+  fill_rollout(c, st, ro, k, R);
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rollout_append(R, false, c->stream));
+  if (c->alloc_on && (rc = gm_pages_release(c, st, ro->finished)) != GM_OK) return rc;
+  return GM_OK;
+}
+
+int gm_rollout_run(gm_ctx *c, gm_state *st, const gm_rollout *ro, int k, float temperature, uint64_t seed,
+                   uint64_t first_step, int max_steps, int check_every, int32_t *steps_run, int32_t *rows_running) {
+  if (max_steps < 0 || check_every < 1) return GM_ERR_INVALID_ARG;
+  int rc = rollout_args_ok(c, st, ro);
+  if (rc) return rc;
+  int done = 0;
+  int32_t running = st->batch;
+  auto poll = [&]() -> int {
+    GM_CUDA(c, cudaMemcpyAsync(&running, ro->n_running, sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
+    GM_CUDA(c, cudaStreamSynchronize(c->stream));
+    return GM_OK;
+  };
+  if ((rc = poll()) != GM_OK) return rc;
+  while (done < max_steps && running > 0) {
+    if ((rc = gm_rollout_step(c, st, ro, k, temperature, seed, first_step + done)) != GM_OK) return rc;
+    ++done;
+    if (done % check_every == 0 || done == max_steps)
+      if ((rc = poll()) != GM_OK) return rc;
+  }
+  if (steps_run) *steps_run = done;
+  if (rows_running) *rows_running = running;
   return GM_OK;
 }
 

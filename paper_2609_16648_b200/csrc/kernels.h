@@ -63,6 +63,7 @@ struct SamplerArgs {
   const __nv_bfloat16 *target_hidden;   // [b, K+1, d_model]
   int d_model, max_k;
   uint32_t *status;
+  const int32_t *finished;              // [b] non-zero: the row sits out (accept_len 0, next_token -1 (0 from a plain draw), state untouched); or null
 };
 cudaError_t launch_sampler(const SamplerArgs &A, int batch, cudaStream_t stream);          // cluster of 8 CTAs per sequence
 cudaError_t launch_sampler_stream(const SamplerArgs &A, int batch, cudaStream_t stream);   // one CTA per sequence
@@ -102,6 +103,7 @@ struct PlanArgs {
   int mode, batch, k_or_j;              // VERIFY: K;  DRAFT_NEXT: application index j (2..K);  CHUNK: first position
   int max_pages_per_seq, n_ctas;
   const int32_t *kv_len, *pending_n;
+  const int32_t *finished = nullptr;    // [B] non-zero: the sequence sits the phase out (no queries, no pages); or null
   const int32_t *row_n = nullptr;       // CHUNK: queries per sequence (0 = the sequence sits this pass out)
   int QT = 0;                           // CHUNK: most queries a sequence may have
   int32_t *qn, *qbase;                  // [B] queries of this phase and the position of the first one
@@ -134,6 +136,30 @@ cudaError_t launch_prefill_last(const float *x, const __nv_bfloat16 *hidden, con
 // kv_len[b] = prompt_len[b], pending_n[b] = 1, pending_tok[b][0] = first_tok[b].
 cudaError_t launch_prefill_finish(const int32_t *prompt_len, const int32_t *first_tok, int batch, int pend_stride,
                                   int32_t *kv_len, int32_t *pending_n, int32_t *pending_tok, cudaStream_t stream);
+
+// ---- rollout bookkeeping: responses, stopping, page allocation ------------------------------------------------
+struct RolloutArgs {
+  int batch, k, out_stride, eos_token, max_new, pend_stride;
+  const int32_t *draft_tok;             // [B, k] drafts of the cycle (null for the begin call)
+  const int32_t *accept_len, *next_token;   // [B] (null for the begin call: the token is pending_tok[b][0])
+  const int32_t *pending_tok;
+  int32_t *out_tok, *out_len, *finished, *n_running;
+};
+// begin: response = [first token]; append: response += accepted drafts + final token of the cycle, cut at the first
+// end-of-sequence token (kept) or at max_new tokens; finished[b] = 1 / 2 accordingly; n_running = rows still running.
+cudaError_t launch_rollout_append(const RolloutArgs &A, bool begin, cudaStream_t stream);
+// Page allocator: a stack of free page ids per pool.  reserve: every running row gets pages until its table covers
+// length[b] + extra positions (ST_KV_CAPACITY when the stack or the table row runs out); release: the pages of
+// finished rows go back on the stack.  One thread walks the rows in order, so the assignment is deterministic.
+struct PageAllocArgs {
+  int batch, max_pages_per_seq, num_pages, extra;
+  const int32_t *length, *finished;     // finished may be null
+  int32_t *page_table, *held, *free_list, *free_top;
+  uint32_t *status;
+};
+cudaError_t launch_page_reset(const PageAllocArgs &A, cudaStream_t stream);
+cudaError_t launch_page_reserve(const PageAllocArgs &A, cudaStream_t stream);
+cudaError_t launch_page_release(const PageAllocArgs &A, cudaStream_t stream);
 
 // ---- element-wise --------------------------------------------------------------------------------------
 // x[m] = embed[token(m)] (fp32), xn[m] = RMSNorm(x[m]; w) (bf16); rows m = b*QT + j of the verify phase.

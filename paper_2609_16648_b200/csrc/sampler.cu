@@ -37,6 +37,13 @@ sampler_kernel(const SamplerArgs A) {
   const int K = A.K, V = A.V, R = 2 * K + 1;
   const float s = A.inv_temp * 1.4426950408889634f;            // logits -> base-2 exponents
   pdl_prologue();
+  if (A.finished && A.finished[b]) {               // the row sits out: the whole cluster leaves before any barrier
+    if (rank == 0 && tid == 0) {
+      if (A.accept_len) A.accept_len[b] = 0;
+      A.next_token[static_cast<size_t>(b) * A.tok_out_stride] = A.accept_len ? -1 : 0;   // a plain draw leaves a valid id
+    }
+    return;
+  }
 
   const int nvec_total = V >> 3;
   const int vpc = (nvec_total + SAMP_CLUSTER - 1) / SAMP_CLUSTER;

@@ -53,6 +53,13 @@ __global__ void __launch_bounds__(SS_THREADS, 2) sampler_stream_kernel(const Sam
   __shared__ int sh_ok, sh_tok;
 
   pdl_prologue();
+  if (A.finished && A.finished[b]) {                  // the row sits out
+    if (tid == 0) {
+      if (A.accept_len) A.accept_len[b] = 0;
+      A.next_token[static_cast<size_t>(b) * A.tok_out_stride] = A.accept_len ? -1 : 0;   // a plain draw leaves a valid id
+    }
+    return;
+  }
   if (tid == 0) {
     for (int i = 0; i < SS_NST; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], SS_CWARPS); }
     mbar_fence_init();
