@@ -60,6 +60,9 @@ extern "C" {
 #define GM_FLAG_SIMPLE_GEMM 1       /* debug: route every GEMM through the plain mma.sync kernel */
 #define GM_FLAG_SAMPLER_CLUSTER 2   /* always map the sampler as one 8-CTA cluster per sequence  */
 #define GM_FLAG_SAMPLER_STREAM 4    /* always map the sampler as one CTA per sequence            */
+#define GM_FLAG_GRAPH 8             /* gm_spec_step, gm_spec_step_host and gm_rollout_run replay a
+                                       captured CUDA graph of one cycle (needs a context created on a
+                                       stream of its own: on a default stream the flag has no effect) */
 
 typedef struct gm_ctx gm_ctx;       /* opaque */
 
@@ -179,7 +182,12 @@ int gm_rollout_step(gm_ctx *ctx, gm_state *st, const gm_rollout *ro, int k, floa
 /* Host loop: gm_rollout_step with step = first_step, first_step + 1, ... until no row is running or
  * max_steps cycles ran.  n_running is read back (one stream synchronisation) every check_every cycles, so
  * up to check_every - 1 cycles may run with every row sitting out.  steps_run / rows_running: host
- * outputs, may be NULL.                                                                                 */
+ * outputs, may be NULL.  With GM_FLAG_GRAPH the first call captures one cycle (all its launches,
+ * with their programmatic dependencies, the page reserve / release and the append) into a CUDA graph and
+ * every cycle is one graph launch; the step index then lives in device memory and is advanced by the
+ * append kernel.  The graph is re-captured when the state, the rollout buffers, k, the temperature or
+ * the seed change.  Results are bit-identical to the host-launched loop.  The context must have been
+ * created on a stream of its own: the default streams cannot be captured, and the flag is ignored there. */
 int gm_rollout_run(gm_ctx *ctx, gm_state *st, const gm_rollout *ro, int k, float temperature,
                    uint64_t seed, uint64_t first_step, int max_steps, int check_every,
                    int32_t *steps_run, int32_t *rows_running);
@@ -238,7 +246,9 @@ int gm_accept(gm_ctx *ctx, gm_state *st, int batch, int k, float temperature,
               float *dbg_p, float *dbg_q, const void *target_hidden, int commit_state);
 
 /* One whole cycle: gm_draft, gm_verify, gm_accept(commit_state = 1) on library-owned logit
- * buffers, bit-for-bit the same as the three calls.  draft_tok [B, k] may be NULL.          */
+ * buffers, bit-for-bit the same as the three calls.  draft_tok [B, k] may be NULL.  With
+ * GM_FLAG_GRAPH the cycle is captured once per (state, k, temperature, seed, output pointers)
+ * and every call is one graph launch plus a one-thread kernel that stores the step index.    */
 int gm_spec_step(gm_ctx *ctx, gm_state *st, int k, float temperature, uint64_t seed,
                  uint64_t step, int32_t *accept_len, int32_t *next_token, int32_t *draft_tok);
 

@@ -115,10 +115,21 @@ __global__ void rollout_append_kernel(const RolloutArgs A, int begin) {
     if (!fin) atomicAdd(&running, 1);
   }
   __syncthreads();
-  if (threadIdx.x == 0) *A.n_running = running;
+  if (threadIdx.x == 0) {
+    *A.n_running = running;
+    if (A.step_counter) *A.step_counter += 1;
+  }
 }
 cudaError_t launch_rollout_append(const RolloutArgs &A, bool begin, cudaStream_t stream) {
   return launch_k(rollout_append_kernel, dim3(1), dim3(256), 0, stream, 1, A, begin ? 1 : 0);
+}
+
+__global__ void set_step_kernel(uint64_t *dst, uint64_t value) {
+  pdl_prologue();
+  if (threadIdx.x == 0) *dst = value;
+}
+cudaError_t launch_set_step(uint64_t *dst, uint64_t value, cudaStream_t stream) {
+  return launch_k(set_step_kernel, dim3(1), dim3(32), 0, stream, 1, dst, value);
 }
 
 __global__ void page_reset_kernel(const PageAllocArgs A) {

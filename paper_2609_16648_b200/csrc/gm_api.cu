@@ -66,6 +66,14 @@ struct gm_ctx {
   __nv_bfloat16 *pf_hidden = nullptr;
   float *pf_xlast = nullptr;
   int32_t *ro_accept = nullptr, *ro_next = nullptr;   // per-step outputs of a rollout step
+  // captured rollout cycle (GM_FLAG_ROLLOUT_GRAPH)
+  uint64_t *dev_step = nullptr;             // step index of the captured cycle
+  uint64_t *step_ptr = nullptr;             // non-null while a cycle is being captured: kernels read the step from here
+  struct GraphSlot {                        // one captured sequence of launches and what it was captured for
+    cudaGraphExec_t exec = nullptr;
+    int64_t launches = 0;
+    std::vector<unsigned char> key;
+  } graph_rollout, graph_step;
   const int32_t *finished_mask = nullptr;   // set around the phases of a rollout step: rows that sit out
   // page allocator (gm_pages_*): one stack of free page ids per pool
   bool alloc_on = false;
@@ -350,6 +358,49 @@ int fill_sampler(gm_ctx *c, SamplerArgs &S, float temperature) {
   S.slot_accept = SLOT_ACCEPT;
   S.slot_final = SLOT_FINAL;
   S.finished = c->finished_mask;
+  S.step_ptr = c->step_ptr;
+  return GM_OK;
+}
+
+// ---- captured cycles (GM_FLAG_GRAPH) ----------------------------------------------------------------------------------
+struct KeyBytes {
+  std::vector<unsigned char> bytes;
+  template <typename T> void add(const T &v) {
+    const unsigned char *p = reinterpret_cast<const unsigned char *>(&v);
+    bytes.insert(bytes.end(), p, p + sizeof(T));
+  }
+};
+bool graph_capable(const gm_ctx *c) {
+  return (c->cfg.flags & GM_FLAG_GRAPH) && c->stream != nullptr && c->stream != cudaStreamLegacy &&
+         c->stream != cudaStreamPerThread;
+}
+// Makes `slot` hold a graph of the launches `body` issues (with the step index read from c->dev_step), re-capturing
+// when `key` differs from what the slot was captured for.  Nothing of `body` runs here.
+template <typename F>
+int graph_prepare(gm_ctx *c, gm_ctx::GraphSlot &slot, const std::vector<unsigned char> &key, F &&body) {
+  if (slot.exec && slot.key == key) return GM_OK;
+  if (slot.exec) { cudaGraphExecDestroy(slot.exec); slot.exec = nullptr; }
+  int rc;
+  if (!c->dev_step && (rc = dev_alloc(c, &c->dev_step, 1)) != GM_OK) return rc;
+  const int64_t before = c->launches;
+  GM_CUDA(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeRelaxed));
+  c->step_ptr = c->dev_step;
+  rc = body();
+  c->step_ptr = nullptr;
+  cudaGraph_t graph = nullptr;
+  const cudaError_t e = cudaStreamEndCapture(c->stream, &graph);         // always leave capture mode
+  const int64_t n = c->launches - before;
+  c->launches = before;                                                  // nothing has run yet
+  if (rc != GM_OK || e != cudaSuccess || !graph) {
+    if (graph) cudaGraphDestroy(graph);
+    if (e != cudaSuccess) { c->last_cuda = e; (void)cudaGetLastError(); }
+    return rc != GM_OK ? rc : GM_ERR_CUDA;
+  }
+  const cudaError_t ei = cudaGraphInstantiate(&slot.exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (ei != cudaSuccess) { c->last_cuda = ei; slot.exec = nullptr; return GM_ERR_CUDA; }
+  slot.launches = n;
+  slot.key = key;
   return GM_OK;
 }
 
@@ -501,6 +552,8 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
 void gm_destroy(gm_ctx *c) {
   if (!c) return;
   cudaStreamSynchronize(c->stream);
+  if (c->graph_rollout.exec) cudaGraphExecDestroy(c->graph_rollout.exec);
+  if (c->graph_step.exec) cudaGraphExecDestroy(c->graph_step.exec);
   for (void *p : c->allocs) cudaFree(p);
   for (auto &v : c->events)
     for (auto &e : v) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
@@ -743,6 +796,32 @@ int gm_draw(gm_ctx *c, const void *logits, int rows, float temperature, const ui
 
 static int spec_step_impl(gm_ctx *c, gm_state *st, int k, float temperature, const uint32_t *u24_draft,
                           const uint32_t *u24_accept, uint64_t seed, uint64_t step, int32_t *accept_len,
+                          int32_t *next_token, int32_t *draft_tok);
+
+// One cycle, host-launched or (GM_FLAG_GRAPH on a capturable stream) as a replay of the captured cycle.
+static int spec_step_run(gm_ctx *c, gm_state *st, int k, float temperature, const uint32_t *u24_draft,
+                         const uint32_t *u24_accept, uint64_t seed, uint64_t step, int32_t *accept_len,
+                         int32_t *next_token, int32_t *draft_tok) {
+  if (!c || !graph_capable(c) || c->prof_mask != 0)          // per-launch timing needs host-launched kernels
+    return spec_step_impl(c, st, k, temperature, u24_draft, u24_accept, seed, step, accept_len, next_token, draft_tok);
+  int rc = check_state(c, st, k);
+  if (rc) return rc;
+  if (!accept_len || !next_token) return GM_ERR_INVALID_ARG;
+  KeyBytes key;
+  key.add(*st); key.add(k); key.add(temperature); key.add(u24_draft); key.add(u24_accept); key.add(seed);
+  key.add(accept_len); key.add(next_token); key.add(draft_tok); key.add(c->top_p);
+  rc = graph_prepare(c, c->graph_step, key.bytes, [&]() {
+    return spec_step_impl(c, st, k, temperature, u24_draft, u24_accept, seed, 0, accept_len, next_token, draft_tok);
+  });
+  if (rc) return rc;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_set_step(c->dev_step, step, c->stream));
+  GM_CUDA(c, cudaGraphLaunch(c->graph_step.exec, c->stream));
+  c->launches += c->graph_step.launches;
+  return GM_OK;
+}
+
+static int spec_step_impl(gm_ctx *c, gm_state *st, int k, float temperature, const uint32_t *u24_draft,
+                          const uint32_t *u24_accept, uint64_t seed, uint64_t step, int32_t *accept_len,
                           int32_t *next_token, int32_t *draft_tok) {
   int rc = check_state(c, st, k);
   if (rc) return rc;
@@ -756,7 +835,7 @@ static int spec_step_impl(gm_ctx *c, gm_state *st, int k, float temperature, con
 
 int gm_spec_step(gm_ctx *c, gm_state *st, int k, float temperature, uint64_t seed, uint64_t step, int32_t *accept_len,
                  int32_t *next_token, int32_t *draft_tok) {
-  return spec_step_impl(c, st, k, temperature, nullptr, nullptr, seed, step, accept_len, next_token, draft_tok);
+  return spec_step_run(c, st, k, temperature, nullptr, nullptr, seed, step, accept_len, next_token, draft_tok);
 }
 
 int gm_spec_step_host(gm_ctx *c, gm_state *st, int k, float temperature, uint64_t seed, uint64_t step,
@@ -774,7 +853,7 @@ int gm_spec_step_host(gm_ctx *c, gm_state *st, int k, float temperature, uint64_
     GM_CUDA(c, cudaMemcpyAsync(ud, u24_draft_host, B * k * sizeof(uint32_t), cudaMemcpyHostToDevice, c->stream));
     GM_CUDA(c, cudaMemcpyAsync(ua, u24_accept_host, B * (k + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice, c->stream));
   }
-  rc = spec_step_impl(c, st, k, temperature, ud, ua, seed, step, c->ws_accept_len, c->ws_next_token, c->ws_draft_tok);
+  rc = spec_step_run(c, st, k, temperature, ud, ua, seed, step, c->ws_accept_len, c->ws_next_token, c->ws_draft_tok);
   if (rc) return rc;
   GM_CUDA(c, cudaMemcpyAsync(accept_len_host, c->ws_accept_len, B * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
   GM_CUDA(c, cudaMemcpyAsync(next_token_host, c->ws_next_token, B * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
@@ -944,7 +1023,7 @@ static void fill_rollout(const gm_ctx *c, const gm_state *st, const gm_rollout *
   R.batch = st->batch; R.k = k; R.out_stride = ro->out_stride; R.eos_token = ro->eos_token; R.max_new = ro->max_new;
   R.pend_stride = c->cfg.max_k + 1; R.draft_tok = c->ws_draft_tok; R.accept_len = c->ro_accept; R.next_token = c->ro_next;
   R.pending_tok = st->pending_tok; R.out_tok = ro->out_tok; R.out_len = ro->out_len; R.finished = ro->finished;
-  R.n_running = ro->n_running;
+  R.n_running = ro->n_running; R.step_counter = c->step_ptr;
 }
 
 int gm_rollout_begin(gm_ctx *c, const gm_state *st, const gm_rollout *ro) {
@@ -986,8 +1065,22 @@ int gm_rollout_run(gm_ctx *c, gm_state *st, const gm_rollout *ro, int k, float t
     return GM_OK;
   };
   if ((rc = poll()) != GM_OK) return rc;
+  const bool use_graph = graph_capable(c);
+  if (use_graph && running > 0 && max_steps > 0) {
+    KeyBytes key;
+    key.add(*st); key.add(*ro); key.add(k); key.add(temperature); key.add(seed); key.add(c->alloc_on); key.add(c->top_p);
+    if ((rc = check_state(c, st, k)) != GM_OK) return rc;
+    rc = graph_prepare(c, c->graph_rollout, key.bytes, [&]() { return gm_rollout_step(c, st, ro, k, temperature, seed, 0); });
+    if (rc) return rc;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_set_step(c->dev_step, first_step, c->stream));
+  }
   while (done < max_steps && running > 0) {
-    if ((rc = gm_rollout_step(c, st, ro, k, temperature, seed, first_step + done)) != GM_OK) return rc;
+    if (use_graph) {
+      GM_CUDA(c, cudaGraphLaunch(c->graph_rollout.exec, c->stream));
+      c->launches += c->graph_rollout.launches;
+    } else if ((rc = gm_rollout_step(c, st, ro, k, temperature, seed, first_step + done)) != GM_OK) {
+      return rc;
+    }
     ++done;
     if (done % check_every == 0 || done == max_steps)
       if ((rc = poll()) != GM_OK) return rc;

@@ -63,6 +63,7 @@ struct SamplerArgs {
   const __nv_bfloat16 *target_hidden;   // [b, K+1, d_model]
   int d_model, max_k;
   uint32_t *status;
+  const uint64_t *step_ptr;             // when set, the step index is read from device memory instead of `step`
   const int32_t *finished;              // [b] non-zero: the row sits out (accept_len 0, next_token -1 (0 from a plain draw), state untouched); or null
 };
 cudaError_t launch_sampler(const SamplerArgs &A, int batch, cudaStream_t stream);          // cluster of 8 CTAs per sequence
@@ -144,10 +145,12 @@ struct RolloutArgs {
   const int32_t *accept_len, *next_token;   // [B] (null for the begin call: the token is pending_tok[b][0])
   const int32_t *pending_tok;
   int32_t *out_tok, *out_len, *finished, *n_running;
+  uint64_t *step_counter = nullptr;     // when set, incremented once per append (the step index of a captured cycle)
 };
 // begin: response = [first token]; append: response += accepted drafts + final token of the cycle, cut at the first
 // end-of-sequence token (kept) or at max_new tokens; finished[b] = 1 / 2 accordingly; n_running = rows still running.
 cudaError_t launch_rollout_append(const RolloutArgs &A, bool begin, cudaStream_t stream);
+cudaError_t launch_set_step(uint64_t *dst, uint64_t value, cudaStream_t stream);      // *dst = value
 // Page allocator: a stack of free page ids per pool.  reserve: every running row gets pages until its table covers
 // length[b] + extra positions (ST_KV_CAPACITY when the stack or the table row runs out); release: the pages of
 // finished rows go back on the stack.  One thread walks the rows in order, so the assignment is deterministic.

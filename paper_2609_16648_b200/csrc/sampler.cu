@@ -198,7 +198,7 @@ sampler_kernel(const SamplerArgs A) {
         const float p = prob_of(xp, s, row_mz[0].m, row_mz[0].z);
         const float q = prob_of(xq, s, row_mz[1].m, row_mz[1].z);
         const uint32_t u24 = A.u24 ? A.u24[static_cast<size_t>(b) * A.u_stride + k]
-                                   : philox_u24(A.seed, A.step, b, A.slot_accept + k);
+                                   : philox_u24(A.seed, step_of(A), b, A.slot_accept + k);
         const float uq = __fmul_rn(__fmul_rn(static_cast<float>(u24), 5.9604644775390625e-8f /* 2^-24 */), q);
         ok = p >= q || uq < p;
       }
@@ -246,7 +246,7 @@ sampler_kernel(const SamplerArgs A) {
   }
 
   const uint32_t u_final = A.u24 ? A.u24[static_cast<size_t>(b) * A.u_stride + K]
-                                 : philox_u24(A.seed, A.step, b, A.slot_final);
+                                 : philox_u24(A.seed, step_of(A), b, A.slot_final);
   int winner = -1;                          // CTA that owns the quantile
   unsigned long long t_local = 0;
   if (W != 0) {

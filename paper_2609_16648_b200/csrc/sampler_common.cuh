@@ -35,6 +35,7 @@ __device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b) {          // 
   __nv_bfloat162 r = __hmax2(*reinterpret_cast<__nv_bfloat162 *>(&a), *reinterpret_cast<__nv_bfloat162 *>(&b));
   return *reinterpret_cast<uint32_t *>(&r);
 }
+__device__ __forceinline__ uint64_t step_of(const SamplerArgs &A) { return A.step_ptr ? *A.step_ptr : A.step; }
 // integer weight of one residual entry: trunc(r * 2^44) for r > 0, else 0 (the product is an exact scaling)
 __device__ __forceinline__ unsigned long long weight_of(float p, float q, bool use_q) {
   const float r = use_q ? __fsub_rn(p, q) : p;

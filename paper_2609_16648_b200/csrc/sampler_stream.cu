@@ -227,7 +227,7 @@ __global__ void __launch_bounds__(SS_THREADS, 2) sampler_stream_kernel(const Sam
         const float p = prob_of(xp, s, row_mz[0].m, row_mz[0].z);
         const float q = prob_of(xq, s, row_mz[1].m, row_mz[1].z);
         const uint32_t u24 = A.u24 ? A.u24[static_cast<size_t>(b) * A.u_stride + k]
-                                   : philox_u24(A.seed, A.step, b, A.slot_accept + k);
+                                   : philox_u24(A.seed, step_of(A), b, A.slot_accept + k);
         const float uq = __fmul_rn(__fmul_rn(static_cast<float>(u24), 5.9604644775390625e-8f /* 2^-24 */), q);
         ok = p >= q || uq < p;
       }
@@ -287,7 +287,7 @@ __global__ void __launch_bounds__(SS_THREADS, 2) sampler_stream_kernel(const Sam
   }
 
   const uint32_t u_final = A.u24 ? A.u24[static_cast<size_t>(b) * A.u_stride + K]
-                                 : philox_u24(A.seed, A.step, b, A.slot_final);
+                                 : philox_u24(A.seed, step_of(A), b, A.slot_final);
   if (W != 0) {
     const unsigned long long t = static_cast<unsigned long long>(u_final) * (W >> 24) +
                                  ((static_cast<unsigned long long>(u_final) * (W & 0xFFFFFFull)) >> 24);

@@ -152,3 +152,47 @@ def test_page_allocator_rollout_equals_static_tables_and_returns_pages():
     t = st.page_table.cpu().numpy()
     assert t.max() < npg and len(set(t[t >= 0].tolist())) == (t >= 0).sum()
     ctx.close()
+
+
+def _two_rollouts(gmb, cfg, n_steps, flags):
+    K, B = cfg.k, cfg.batch
+    w, ost, ctx, gst = tiny_setup(cfg, cap_tokens=20 + n_steps * (K + 1) + 8, flags=flags)
+    push_state(ost, gst, ctx)
+    snap = {n: getattr(gst, n).clone() for n in STATE_FIELDS}
+    ro = gmb.Rollout(B, 17, -1)
+    runs = []
+    for rep in range(2):
+        for n, v in snap.items():
+            getattr(gst, n).copy_(v)
+        gmb.gm_rollout_begin(ctx, gst, ro)
+        l0 = gmb.gm_launch_count(ctx)
+        steps, running = gmb.gm_rollout_run(ctx, gst, ro, K, 1.0, 5, 1 + 100 * rep, n_steps, check_every=2)
+        assert gmb.gm_last_status(ctx) == 0
+        runs.append((steps, running, ro.responses(), ro.finished.cpu().numpy().copy(), gst.kv_len.cpu().numpy().copy(),
+                     gst.pending_hidden.clone().cpu(), gmb.gm_launch_count(ctx) - l0))
+    ctx.close()
+    return runs
+
+
+def test_graph_replayed_rollout_equals_host_launched_rollout():
+    """One captured cycle replayed per step (step index on the device) gives the same responses, stop codes and
+    final state as the host-launched loop; a second rollout through the same buffers reuses the graph."""
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny").with_(prompt_len=20)
+    K, B = cfg.k, cfg.batch
+    n_steps = 9
+    results = {}
+    side = torch.cuda.Stream()                                   # the default stream cannot be captured
+    for flags in (0, 8):
+        with torch.cuda.stream(side):
+            runs = _two_rollouts(gmb, cfg, n_steps, flags)
+        side.synchronize()
+        results[flags] = runs
+    for rep in range(2):
+        h, g = results[0][rep], results[8][rep]
+        assert h[0] == g[0] and h[1] == g[1] and h[2] == g[2]
+        np.testing.assert_array_equal(h[3], g[3])
+        np.testing.assert_array_equal(h[4], g[4])
+        assert torch.equal(h[5], g[5])
+        assert g[6] == h[6] + 1 > 1                              # the replayed kernels are counted, plus one store of the first step index
+    assert results[0][0][2] != results[0][1][2]                  # different step indices: different uniforms

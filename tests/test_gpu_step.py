@@ -300,3 +300,49 @@ def test_rerun_is_bit_identical_and_resume_equals_uninterrupted():
         assert torch.equal(getattr(gst2, n), end[n]), n
     assert gmb.gm_last_status(ctx) == 0
     ctx.close()
+
+
+def test_graph_replayed_cycle_equals_host_launched_cycle():
+    """GM_FLAG_GRAPH on a stream of its own: gm_spec_step and gm_spec_step_host replay a captured cycle; accept
+    lengths, tokens, drafts and the final state are bit-identical to the host-launched cycle, across re-captures
+    (other output buffers) and with the step index changing every call."""
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny").with_(prompt_len=33)
+    K, B = cfg.k, cfg.batch
+    out = {}
+    side = torch.cuda.Stream()
+    for flags in (0, gmb.GM_FLAG_GRAPH):
+        with torch.cuda.stream(side):
+            w, ost, ctx, gst = tiny_setup(cfg, cap_tokens=160, flags=flags)
+            push_state(ost, gst, ctx)
+            z = lambda *shape: torch.zeros(shape, dtype=torch.int32, device="cuda")
+            a, t, d, a2, t2 = z(B), z(B), z(B, K), z(B), z(B)
+            hist = []
+            l0 = gmb.gm_launch_count(ctx)
+            for it in range(6):
+                gmb.gm_spec_step(ctx, gst, K, 1.0, 11, 100 + 7 * it, a, t, d)
+                hist.append((a.cpu().numpy().copy(), t.cpu().numpy().copy(), d.cpu().numpy().copy()))
+            for it in range(3):                                   # other output pointers: a second capture
+                gmb.gm_spec_step(ctx, gst, K, 1.0, 11, 200 + it, a2, t2)
+                hist.append((a2.cpu().numpy().copy(), t2.cpu().numpy().copy()))
+            ud = torch.randint(0, 1 << 24, (B, K), dtype=torch.int32).pin_memory()
+            ua = torch.randint(0, 1 << 24, (B, K + 1), dtype=torch.int32, generator=torch.Generator().manual_seed(3)).pin_memory()
+            ah, th = torch.zeros(B, dtype=torch.int32).pin_memory(), torch.zeros(B, dtype=torch.int32).pin_memory()
+            dh = torch.zeros((B, K), dtype=torch.int32).pin_memory()
+            torch.manual_seed(5)
+            for it in range(3):
+                ud.copy_(torch.randint(0, 1 << 24, (B, K), dtype=torch.int32))
+                gmb.gm_spec_step_host(ctx, gst, K, 1.0, 11, 300 + it, ah, th, dh, ud, ua)
+                hist.append((ah.numpy().copy(), th.numpy().copy(), dh.numpy().copy()))
+            assert gmb.gm_last_status(ctx) == 0
+            out[flags] = (hist, gst.kv_len.cpu().numpy().copy(), gst.pending_hidden.clone().cpu(), gst.kv_pool.clone().cpu(),
+                          gmb.gm_launch_count(ctx) - l0)
+            ctx.close()
+        side.synchronize()
+    h0, h1 = out[0], out[gmb.GM_FLAG_GRAPH]
+    for x, y in zip(h0[0], h1[0]):
+        for u, v in zip(x, y):
+            np.testing.assert_array_equal(u, v)
+    np.testing.assert_array_equal(h0[1], h1[1])
+    assert torch.equal(h0[2], h1[2]) and torch.equal(h0[3], h1[3])
+    assert h1[4] == h0[4] + 12                                     # the same kernels + one step-index store per replay
