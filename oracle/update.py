@@ -1,0 +1,92 @@
+"""Forward pass of the draft-head update: draft-path reconstruction and the acceptance objective
+(Sec. 3.2 Eq. 4; Sec. 3.3 Eq. 5-7; Sec. 3.4 Eq. 8-9; App. D.2-D.3).  Test infrastructure only.
+
+Reconstruction.  A recorded cycle r started at context length Len (its record's start position) with the
+committed tokens x[0..Len-1].  The head's chain is replayed on recorded inputs: its cache is rebuilt from
+the recorded pairs (H_{i-1}, x_i), i = 1..Len-1 (the rollout-time target hidden states and token ids),
+restricted to the committed prefix; the first application's output at head position Len-2 is the state
+g_1; application k >= 2 consumes (g_{k-1}, d_{k-1}) - the *recorded* draft - at head position Len+k-3,
+seeing the prefix and the chain's own earlier entries only.  Nothing is sampled.  q_k = softmax(logits(g_k)/T).
+
+Objective.  alpha_k = sum_d min(p_k(d), q_k(d)) (Eq. 5), estimated from the record's top-64 target
+log-probabilities plus one residual bin (App. D.2); the chain surrogate -sum_l prod_{i<=l} alpha_i (Eq. 6),
+its logarithmic form (Eq. 7) and the truncation of the chain sum at min(j, K), j the first rejected
+position, K+1 if none (Eq. 9).  The update minimises the mean over cycles.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from . import record, sampler
+from .model import PagedKV, head_forward, head_logits, round_bf16
+
+
+def reconstruct_chain(w, cfg, seq_hidden, seq_tokens, start_len: int, drafts, temperature: float = 1.0,
+                      round_interface: bool = True):
+    """Eq. 4 for one cycle.  seq_hidden[i] = H_i, the target hidden state that produced token x_{i+1};
+    seq_tokens = the sequence's committed tokens; start_len = Len >= 2 (a prompt token and the first
+    response token at least).
+    Returns (q[K, V] fp32, logits[K, V])."""
+    Len, K = int(start_len), len(drafts)
+    assert Len >= 2 and len(seq_tokens) >= Len and len(seq_hidden) >= Len - 1
+    pages = (Len + K + cfg.page_size) // cfg.page_size + 1
+    hkv = PagedKV(1, cfg.n_kv_heads, cfg.head_dim, np.arange(pages)[None, :], pages, cfg.page_size)
+    g = head_forward(w, np.asarray(seq_hidden)[:Len - 1], list(seq_tokens[1:Len]), np.arange(Len - 1), hkv, 0, cfg)[-1:]
+    qs, lgs = [], []
+    for k in range(1, K + 1):
+        if k > 1:
+            g = head_forward(w, g, [int(drafts[k - 2])], np.array([Len + k - 3]), hkv, 0, cfg)
+        lg = head_logits(w, g, cfg)[0]
+        if round_interface:
+            lg = round_bf16(lg).astype(np.float64)
+        lgs.append(lg)
+        qs.append(sampler.softmax_probs(lg, temperature))
+    return np.array(qs), np.array(lgs)
+
+
+def chain_alphas(rec: dict, q) -> np.ndarray:
+    """alpha_k, k = 1..K, of one recorded cycle from its top-64 record and the reconstructed q[K, V]."""
+    return np.array([record.sparsified_overlap(rec["top_index"][k], rec["top_logprob"][k], q[k])
+                     for k in range(len(q))])
+
+
+def tv_chain_loss(alphas) -> float:
+    """L_TV = - sum_{l=1..K} prod_{i<=l} alpha_i   (Eq. 6)."""
+    return -float(np.cumprod(np.asarray(alphas, np.float64)).sum())
+
+
+def dca_loss(alphas, j: int | None = None) -> float:
+    """L_DCA = - log sum_{l=1..L} exp(sum_{i<=l} log alpha_i), L = K (Eq. 7) or min(j, K) (Eq. 9)."""
+    a = np.asarray(alphas, np.float64)
+    L = len(a) if j is None else min(int(j), len(a))
+    assert L >= 1
+    with np.errstate(divide="ignore"):
+        s = np.cumsum(np.log(a[:L]))
+    m = s.max()
+    if not np.isfinite(m):
+        return float("inf")
+    return -float(m + np.log(np.exp(s - m).sum()))
+
+
+def dca_position_weights(alphas) -> np.ndarray:
+    """-dL_DCA/dalpha_k = (prod_{i<k} alpha_i) D_k / (-L_TV), D_k = sum_{l>=k} prod_{i=k+1..l} alpha_i   (Eq. 8)."""
+    a = np.asarray(alphas, np.float64)
+    K = len(a)
+    out = np.zeros(K)
+    for k in range(K):
+        D = sum(np.prod(a[k + 1:l + 1]) for l in range(k, K))
+        out[k] = np.prod(a[:k]) * D / (-tv_chain_loss(a))
+    return out
+
+
+def head_update_loss(w, cfg, sequences, records, temperature: float = 1.0, round_interface: bool = True):
+    """Mean of Eq. 9 over recorded cycles.  sequences[s] = (seq_hidden, seq_tokens); records = list of
+    (s, record dict as oracle.record.cycle_record builds it).  Returns (loss, alphas[n_cycles, K])."""
+    losses, alphas = [], []
+    for s, rec in records:
+        hid, toks = sequences[s]
+        q, _ = reconstruct_chain(w, cfg, hid, toks, rec["start_pos"], rec["drafts"], temperature, round_interface)
+        a = chain_alphas(rec, q)
+        alphas.append(a)
+        losses.append(dca_loss(a, rec["accepted"]))
+    return float(np.mean(losses)), np.array(alphas)

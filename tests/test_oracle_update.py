@@ -1,0 +1,125 @@
+"""Pins for the oracle's head-update forward: draft-path reconstruction (Eq. 4) and the DCA / VGM objective
+(Eq. 5-9)."""
+import numpy as np
+import pytest
+
+from oracle import model, record, sampler, step, update
+from synth_inputs import ModelConfig, make_weights, make_page_tables, random_prompts
+from synth_inputs.weights import perturb_norm_weights
+
+T = 0.02        # random-init logits are almost flat; a low temperature makes head and target disagree
+CFG = ModelConfig("t", 2, 64, 4, 2, 16, 96, 50, batch=3, k=3, kv_len_min=0, kv_len_max=0,
+                  length_law="prompt", prompt_len=9)
+
+
+def _rollout_with_records(rounding, n_steps=5, K=3):
+    w = perturb_norm_weights(make_weights(CFG, 0))
+    prompts = random_prompts(CFG.batch, CFG.prompt_len, CFG.vocab, seed=1)
+    pt, npg = make_page_tables(np.full(CFG.batch, 96), CFG.page_size, seed=7)
+    hpt, hnpg = make_page_tables(np.full(CFG.batch, 96), CFG.page_size, seed=8)
+    st = step.prefill(w, CFG, prompts, pt, npg, hpt, hnpg, temperature=T, seed=5, round_interface=rounding)
+    cycles = []
+    for it in range(n_steps):
+        lens = [len(s.tokens) for s in st.seqs]
+        start_h = [s.pending_hidden[-1].copy() for s in st.seqs]
+        out = step.spec_step(w, CFG, st, K, T, seed=5, round_interface=rounding)
+        for b in range(CFG.batch):
+            rec = record.cycle_record(start_h[b], out["draft_tok"][b], out["target_logits"][b], out["accept_len"][b], lens[b], T)
+            cycles.append((b, rec, out["q"][b], out["p"][b]))
+    return w, st, cycles
+
+
+def _sequence_features(w, st, rounding):
+    seqs = []
+    for s in st.seqs:
+        kv = model.PagedKV(CFG.n_layers, CFG.n_kv_heads, CFG.head_dim, np.arange(16)[None, :], 16)
+        H = model.target_forward(w, s.tokens[:-1], np.arange(len(s.tokens) - 1), kv, 0, CFG)
+        seqs.append((model.round_bf16(H).astype(np.float64) if rounding else H, list(s.tokens)))
+    return seqs
+
+
+def test_reconstruction_reproduces_the_rollouts_head_distributions():
+    """Eq. 4 on recorded inputs recomputes exactly the states drafting ran: every q_k of every cycle of a rollout,
+    although the rollout's head cache was written incrementally and partly overwritten by rejected chains."""
+    w, st, cycles = _rollout_with_records(rounding=False)
+    seqs = _sequence_features(w, st, rounding=False)
+    assert any(rec["accepted"] <= 3 for _, rec, _, _ in cycles)          # some chains were cut short
+    for b, rec, q_roll, _ in cycles:
+        q, _ = update.reconstruct_chain(w, CFG, seqs[b][0], seqs[b][1], rec["start_pos"], rec["drafts"], T,
+                                        round_interface=False)
+        np.testing.assert_allclose(q, q_roll, rtol=1e-6, atol=1e-12)
+        # the start hidden of the record is the feature the chain starts from
+        np.testing.assert_allclose(rec["start_hidden"], seqs[b][0][rec["start_pos"] - 2], rtol=1e-9, atol=1e-12)
+
+
+def test_reconstruction_depends_on_the_recorded_drafts_not_on_the_committed_path():
+    w, st, cycles = _rollout_with_records(rounding=False)
+    seqs = _sequence_features(w, st, rounding=False)
+    b, rec, q_roll, _ = next(c for c in cycles if c[1]["accepted"] == 1)   # first draft rejected
+    other = (rec["drafts"] + 1) % CFG.vocab
+    q2, _ = update.reconstruct_chain(w, CFG, seqs[b][0], seqs[b][1], rec["start_pos"], other, T, round_interface=False)
+    np.testing.assert_allclose(q2[0], q_roll[0], rtol=1e-6)                # depth 1 sees no draft
+    assert np.abs(q2[1] - q_roll[1]).max() > 1e-4                          # depth 2 is conditioned on d_1
+    # feeding the committed continuation instead of the recorded (rejected) draft gives another state
+    committed = np.array(seqs[b][1][rec["start_pos"]:rec["start_pos"] + 3])
+    assert committed[0] != rec["drafts"][0]
+    q3, _ = update.reconstruct_chain(w, CFG, seqs[b][0], seqs[b][1], rec["start_pos"], committed, T, round_interface=False)
+    assert np.abs(q3[1] - q_roll[1]).max() > 1e-4
+
+
+def test_alpha_from_the_record_is_close_to_the_full_overlap_and_bounds_it():
+    w, st, cycles = _rollout_with_records(rounding=True)
+    for b, rec, q, p in cycles[:6]:
+        a = update.chain_alphas(rec, q)
+        full = np.array([sampler.acceptance_probability(p[k], q[k]) for k in range(3)])
+        # vocabulary 50 < 64 retained entries: the residual bin is empty and the estimate is the overlap itself
+        np.testing.assert_allclose(a, full, atol=4e-3)                      # bf16 log-probabilities
+        assert (a > 0).all() and (a <= 1 + 1e-3).all()
+
+
+def test_chain_losses_closed_forms():
+    a = np.array([0.9, 0.5, 0.25])
+    assert update.tv_chain_loss(a) == pytest.approx(-(0.9 + 0.45 + 0.1125))
+    assert update.dca_loss(a) == pytest.approx(-np.log(0.9 + 0.45 + 0.1125))
+    assert update.dca_loss(a) == pytest.approx(-np.log(-update.tv_chain_loss(a)))          # Eq. 7 = -log(-L_TV)
+    assert update.dca_loss(np.ones(5)) == pytest.approx(-np.log(5.0))
+    assert update.dca_loss([0.3]) == pytest.approx(-np.log(0.3))
+    # verify-gated masking: chain sum cut at min(j, K); j = 1 keeps the first position only
+    assert update.dca_loss(a, j=1) == pytest.approx(-np.log(0.9))
+    assert update.dca_loss(a, j=2) == pytest.approx(-np.log(0.9 + 0.45))
+    assert update.dca_loss(a, j=3) == update.dca_loss(a, j=4) == update.dca_loss(a)
+    assert update.dca_loss([0.0, 0.5]) == float("inf")
+    assert np.isfinite(update.dca_loss([0.5, 0.0, 0.7]))
+
+
+def test_gradient_weights_of_eq8_match_finite_differences():
+    rng = np.random.default_rng(4)
+    for K in (1, 2, 5, 7):
+        a = rng.uniform(0.05, 0.95, K)
+        w = update.dca_position_weights(a)
+        for k in range(K):
+            e = np.zeros(K)
+            e[k] = 1e-6
+            fd = -(update.dca_loss(a + e) - update.dca_loss(a - e)) / 2e-6
+            assert w[k] == pytest.approx(fd, rel=1e-5)
+        # the tail term lies in [1, K-k+1] (k counted from 1)
+        D = w * (-update.tv_chain_loss(a)) / np.concatenate([[1.0], np.cumprod(a)[:-1]])
+        assert (D >= 1 - 1e-12).all() and (D <= K - np.arange(K) + 1e-12).all()
+        # gradient of the logarithmic form = gradient of the chain form / M
+        for k in range(K):
+            e = np.zeros(K)
+            e[k] = 1e-6
+            fd_tv = -(update.tv_chain_loss(a + e) - update.tv_chain_loss(a - e)) / 2e-6
+            assert w[k] == pytest.approx(fd_tv / (-update.tv_chain_loss(a)), rel=1e-5)
+
+
+def test_head_update_loss_is_the_mean_over_cycles():
+    w, st, cycles = _rollout_with_records(rounding=True, n_steps=3)
+    seqs = _sequence_features(w, st, rounding=True)
+    recs = [(b, rec) for b, rec, _, _ in cycles]
+    loss, alphas = update.head_update_loss(w, CFG, seqs, recs, T)
+    assert alphas.shape == (len(recs), 3)
+    per = [update.dca_loss(alphas[i], recs[i][1]["accepted"]) for i in range(len(recs))]
+    assert loss == pytest.approx(np.mean(per))
+    # a perfect head (q = p) would give alpha = 1 everywhere and loss -log(min(j, K)) per cycle: the bound
+    assert loss >= -np.mean([np.log(min(r["accepted"], 3)) for _, r in recs]) - 1e-9
