@@ -312,6 +312,43 @@ int gm_record_end(gm_ctx *ctx, int batch, int k, float temperature, const void *
 int gm_spec_step_rec(gm_ctx *ctx, gm_state *st, int k, float temperature, uint64_t seed, uint64_t step,
                      int32_t *accept_len, int32_t *next_token, int32_t *draft_tok, gm_record *rec);
 
+/* ---- Forward pass of the draft-head update on recorded cycles (Sec. 3.2 Eq. 4; Sec. 3.3-3.4 Eq. 5-9; App. D.2,
+ * D.3).  The recorded inputs: per sequence its committed tokens x[0..L-1] and the rollout-time target hidden
+ * states H_0..H_{L-2} (H_i produced x_{i+1}); per cycle a gm_record entry.  Forward only: no gradients.
+ *
+ * gm_head_prefill rebuilds the head cache of every sequence from its recorded pairs (H_{i-1}, x_i),
+ *   i = 1..L_b-1, at head positions 0..L_b-2 (the shared prefix every chain attends).
+ *   seq_hidden bf16 [B, hid_stride, d];  seq_tok int32 [B, tok_stride];  seq_len int32 [B] = L_b (device);
+ *   max_len host value >= every L_b;  hid_stride >= max_len - 1, tok_stride >= max_len.
+ *
+ * gm_reconstruct replays the draft chain of n_cycles recorded cycles (Eq. 4): chain r belongs to sequence
+ *   cycle_seq[r], starts at context length rec->start_pos[r] from the hidden rec->start_hidden[r], and feeds
+ *   back the recorded drafts rec->drafts[r]; nothing is sampled.  All chains advance together, one draft
+ *   application per depth, max_batch chains per pass.  Every chain sees the shared prefix up to its start
+ *   and only its own draft entries: it runs as a virtual sequence whose page-table row shares its sequence's
+ *   head-cache pages before the page of its first entry and owns the two pages scratch_pages[r][0..1] (ids
+ *   in the head pool that no sequence uses) from there on.  draft_logits bf16 [n_cycles, k, V] out.
+ *   The state's head cache must have been prefilled (gm_head_prefill, or the rollout that made the record);
+ *   it is not modified outside the scratch pages.
+ *
+ * gm_overlap: alpha[r, j] = sum over the record's 64 retained tokens of min(p, q) + min(1 - sum p, 1 - sum q)
+ *   (Eq. 5 on the sparsified record, App. D.2), q = softmax(draft_logits / T) over the full vocabulary.
+ *   alpha fp32 [n_cycles, k] out.
+ *
+ * gm_dca_loss: loss[r] = -log sum_{l=1..min(accepted[r], k)} prod_{i<=l} alpha[r, i] (Eq. 9; accepted =
+ *   accepted drafts + 1 = the first rejected position, k + 1 if none), evaluated in the log domain (Eq. 7);
+ *   mean[0] = their mean, added in a fixed order.  A chain whose first overlap is 0 gives +inf.           */
+int gm_head_prefill(gm_ctx *ctx, gm_state *st, const void *seq_hidden, int hid_stride,
+                    const int32_t *seq_tok, int tok_stride, const int32_t *seq_len, int max_len);
+int gm_reconstruct(gm_ctx *ctx, gm_state *st, int n_cycles, int k, const int32_t *cycle_seq,
+                   const gm_record *rec, const int32_t *seq_tok, int tok_stride,
+                   const int32_t *scratch_pages, void *draft_logits);
+int gm_overlap(gm_ctx *ctx, int n_cycles, int k, float temperature, const void *draft_logits,
+               const gm_record *rec, float *alpha);
+int gm_dca_loss(gm_ctx *ctx, int n_cycles, int k, const float *alpha, const int32_t *accepted,
+                float *loss, float *mean);
+
+
 /* Dense projection out[M, N] = x[M, K] w[N, K]^T on the context's stream (bf16 in, fp32
  * accumulate; the kernel every QKV / O / FFN / LM-head projection of the step uses).
  *   out_fp32 != 0: out is fp32 [M, N]; else bf16 [M, N].  K % 64 == 0, N % 8 == 0, M >= 1.   */

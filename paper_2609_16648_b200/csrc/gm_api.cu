@@ -78,6 +78,9 @@ struct gm_ctx {
   // page allocator (gm_pages_*): one stack of free page ids per pool
   bool alloc_on = false;
   int32_t *free_list[2] = {nullptr, nullptr}, *free_top[2] = {nullptr, nullptr}, *held[2] = {nullptr, nullptr};
+  // chains of a reconstruction: virtual sequences (allocated on first use)
+  int32_t *v_kv_len = nullptr, *v_pending_n = nullptr, *v_pending_tok = nullptr, *v_table = nullptr;
+  __nv_bfloat16 *v_pending_hidden = nullptr;
   float top_p = 1.f;                    // nucleus of the target distributions (1 = none)
   __nv_bfloat16 *ws_nucleus = nullptr;  // [max_batch (max_k + 1)][V] filtered target rows, allocated by gm_set_top_p
   std::vector<void *> allocs;
@@ -560,8 +563,17 @@ void gm_destroy(gm_ctx *c) {
   delete c;
 }
 
+// forced: draft_tok holds recorded drafts that are fed back instead of sampled ones (Eq. 4); nothing is drawn
+static int draft_impl(gm_ctx *c, const gm_state *st, int k, float temperature, const uint32_t *u24_draft, uint64_t seed,
+                      uint64_t step, int32_t *draft_tok, void *draft_logits, float *dbg_q, bool forced);
+
 int gm_draft(gm_ctx *c, const gm_state *st, int k, float temperature, const uint32_t *u24_draft, uint64_t seed,
              uint64_t step, int32_t *draft_tok, void *draft_logits, float *dbg_q) {
+  return draft_impl(c, st, k, temperature, u24_draft, seed, step, draft_tok, draft_logits, dbg_q, false);
+}
+
+static int draft_impl(gm_ctx *c, const gm_state *st, int k, float temperature, const uint32_t *u24_draft, uint64_t seed,
+                      uint64_t step, int32_t *draft_tok, void *draft_logits, float *dbg_q, bool forced) {
   int rc = check_state(c, st, k);
   if (rc) return rc;
   if (!draft_tok || !draft_logits) return GM_ERR_INVALID_ARG;
@@ -606,7 +618,7 @@ int gm_draft(gm_ctx *c, const gm_state *st, int k, float temperature, const uint
     S.seed = seed; S.step = step; S.slot_final = SLOT_DRAFT + (j - 1);
     S.accept_len = nullptr; S.next_token = draft_tok + (j - 1); S.tok_out_stride = k;
     S.dbg_p = dbg_q ? dbg_q + static_cast<size_t>(j - 1) * c->V : nullptr; S.dbg_q = nullptr; S.commit = 0;
-    GM_LAUNCH(c, GM_KC_SAMPLER, run_sampler(c, S, ph.B));
+    if (!forced) GM_LAUNCH(c, GM_KC_SAMPLER, run_sampler(c, S, ph.B));
   }
   return GM_OK;
 }
@@ -947,6 +959,108 @@ int gm_attention(gm_ctx *c, const void *q, const void *kv_pool, int pool_layers,
   Cb.n_kv = cf.n_kv_heads; Cb.group = c->group; Cb.hd = cf.head_dim; Cb.qrows = qrows; Cb.QT = q_stride;
   Cb.n_ctas = c->sm_count; Cb.out = static_cast<__nv_bfloat16 *>(out);
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_attention_combine(Cb, c->stream));
+  return GM_OK;
+}
+
+// ---- forward pass of the head update on recorded cycles -------------------------------------------------------------
+int gm_head_prefill(gm_ctx *c, gm_state *st, const void *seq_hidden, int hid_stride, const int32_t *seq_tok,
+                    int tok_stride, const int32_t *seq_len, int max_len) {
+  int rc = check_state(c, st, 1);
+  if (rc) return rc;
+  if (!seq_hidden || !seq_tok || !seq_len || max_len < 1 || tok_stride < max_len || hid_stride < max_len - 1)
+    return GM_ERR_INVALID_ARG;
+  const gm_config &cf = c->cfg;
+  if (max_len + cf.max_k + 1 > cf.max_pages_per_seq * GM_PAGE) return GM_ERR_KV_CAPACITY;
+  const int B = st->batch, QT = cf.max_k + 1;
+  PhaseShape ph;
+  ph.B = B; ph.QT = QT; ph.M = B * QT; ph.qrows = round16(QT * c->group);
+  CUtensorMap hkvm;
+  if ((rc = kv_map(c, st->head_kv_pool, 1, cf.head_num_pages, &hkvm)) != GM_OK) return rc;
+  for (int base = 0; base + 1 < max_len; base += QT) {
+    ChunkSetupArgs Cs;
+    Cs.prompt_tok = seq_tok; Cs.prompt_len = seq_len; Cs.batch = B; Cs.stride = tok_stride; Cs.base = base; Cs.QT = QT;
+    Cs.max_len = max_len; Cs.pair_stride = QT; Cs.row_n = c->pf_row_n; Cs.head_n = c->pf_head_n;
+    Cs.pair_tok = c->pf_pair_tok; Cs.status = c->status;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_chunk_setup(Cs, c->stream));
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+              launch_gather_chunk_hidden(static_cast<const __nv_bfloat16 *>(seq_hidden), hid_stride, base, B, QT, c->d,
+                                         c->pf_head_n, c->pf_hidden, c->stream));
+    if ((rc = run_plan_chunk(c, B, c->pf_head_n, base, QT)) != GM_OK) return rc;
+    HeadInputArgs H;
+    H.mode = PHASE_DRAFT_FIRST; H.batch = B; H.QT = QT; H.d = c->d; H.vocab = c->V; H.max_k = cf.max_k; H.k = 1; H.j = 1;
+    H.eps = cf.rms_eps; H.embed = static_cast<const __nv_bfloat16 *>(c->w.embed);
+    H.we = static_cast<const __nv_bfloat16 *>(c->w.head_enorm); H.wh = static_cast<const __nv_bfloat16 *>(c->w.head_hnorm);
+    H.pending_tok = c->pf_pair_tok; H.pending_n = c->pf_head_n; H.pending_hidden = c->pf_hidden; H.draft_tok = nullptr;
+    H.g_prev = c->g; H.zin = c->zin; H.status = c->status;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_head_input(H, c->stream));
+    rc = run_gemm(c, c->zin, c->Mmax, &c->head_proj_map, static_cast<const __nv_bfloat16 *>(c->w.head_proj), ph.M, c->d,
+                  2 * c->d, c->x, EPI_STORE_F32, c->d);
+    if (rc) return rc;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+              launch_rmsnorm(c->x, static_cast<const __nv_bfloat16 *>(c->w.head_layer.ln1), c->xn, nullptr, ph.M, c->d,
+                             cf.rms_eps, c->stream));
+    rc = run_layer(c, c->w.head_layer, c->head_maps, ph, hkvm, static_cast<__nv_bfloat16 *>(st->head_kv_pool), 0,
+                   cf.head_num_pages, st->head_page_table, nullptr, nullptr);
+    if (rc) return rc;
+  }
+  return GM_OK;
+}
+
+int gm_reconstruct(gm_ctx *c, gm_state *st, int n_cycles, int k, const int32_t *cycle_seq, const gm_record *rec,
+                   const int32_t *seq_tok, int tok_stride, const int32_t *scratch_pages, void *draft_logits) {
+  int rc = check_state(c, st, k);
+  if (rc) return rc;
+  if (n_cycles < 1 || !cycle_seq || !rec || !rec->start_hidden || !rec->start_pos || !rec->drafts || !seq_tok ||
+      tok_stride < 2 || !scratch_pages || !draft_logits)
+    return GM_ERR_INVALID_ARG;
+  const gm_config &cf = c->cfg;
+  const int MB = cf.max_batch, PS = cf.max_k + 1;
+  if (!c->v_table) {
+    if ((rc = dev_alloc(c, &c->v_kv_len, MB)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->v_pending_n, MB)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->v_pending_tok, static_cast<size_t>(MB) * PS)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->v_pending_hidden, static_cast<size_t>(MB) * PS * c->d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->v_table, static_cast<size_t>(MB) * cf.max_pages_per_seq)) != GM_OK) return rc;
+  }
+  for (int off = 0; off < n_cycles; off += MB) {
+    const int m = std::min(MB, n_cycles - off);
+    ChainSetupArgs A;
+    A.cycle_seq = cycle_seq + off; A.start_pos = rec->start_pos + off;
+    A.start_hidden = static_cast<const __nv_bfloat16 *>(rec->start_hidden) + static_cast<size_t>(off) * c->d;
+    A.seq_tok = seq_tok; A.scratch_pages = scratch_pages + 2 * static_cast<size_t>(off);
+    A.head_page_table = st->head_page_table; A.pool = static_cast<__nv_bfloat16 *>(st->head_kv_pool);
+    A.n_seq = st->batch; A.tok_stride = tok_stride; A.k = k; A.d = c->d; A.vocab = c->V;
+    A.max_pages_per_seq = cf.max_pages_per_seq; A.num_pages = cf.head_num_pages;
+    A.page_elems = cf.n_kv_heads * GM_PAGE * cf.head_dim; A.pend_stride = PS;
+    A.v_kv_len = c->v_kv_len; A.v_pending_n = c->v_pending_n; A.v_pending_tok = c->v_pending_tok; A.v_table = c->v_table;
+    A.v_pending_hidden = c->v_pending_hidden; A.status = c->status;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_chain_setup(A, m, c->stream));
+    gm_state vs = *st;
+    vs.batch = m; vs.kv_len = c->v_kv_len; vs.head_page_table = c->v_table; vs.pending_n = c->v_pending_n;
+    vs.pending_tok = c->v_pending_tok; vs.pending_hidden = c->v_pending_hidden;
+    rc = draft_impl(c, &vs, k, 1.0f, nullptr, 0, 0, rec->drafts + static_cast<size_t>(off) * k,
+                    static_cast<__nv_bfloat16 *>(draft_logits) + static_cast<size_t>(off) * k * c->V, nullptr, true);
+    if (rc) return rc;
+  }
+  return GM_OK;
+}
+
+int gm_overlap(gm_ctx *c, int n_cycles, int k, float temperature, const void *draft_logits, const gm_record *rec,
+               float *alpha) {
+  if (!c || n_cycles < 1 || k < 1 || k > GM_MAX_K || !draft_logits || !rec || !rec->top_index || !rec->top_logprob || !alpha)
+    return GM_ERR_INVALID_ARG;
+  if (!(temperature > 0.f) || !std::isfinite(temperature)) return GM_ERR_UNSUPPORTED;
+  OverlapArgs A;
+  A.logits = static_cast<const __nv_bfloat16 *>(draft_logits); A.top_index = rec->top_index;
+  A.top_logprob = static_cast<const __nv_bfloat16 *>(rec->top_logprob); A.alpha = alpha; A.V = c->V;
+  A.inv_temp = 1.0f / temperature;
+  GM_LAUNCH(c, GM_KC_RECORD, launch_overlap(A, n_cycles * k, c->stream));
+  return GM_OK;
+}
+
+int gm_dca_loss(gm_ctx *c, int n_cycles, int k, const float *alpha, const int32_t *accepted, float *loss, float *mean) {
+  if (!c || n_cycles < 1 || k < 1 || k > GM_MAX_K || !alpha || !accepted || !loss || !mean) return GM_ERR_INVALID_ARG;
+  GM_LAUNCH(c, GM_KC_RECORD, launch_dca_loss(alpha, accepted, n_cycles, k, loss, mean, c->stream));
   return GM_OK;
 }
 

@@ -164,6 +164,37 @@ cudaError_t launch_page_reset(const PageAllocArgs &A, cudaStream_t stream);
 cudaError_t launch_page_reserve(const PageAllocArgs &A, cudaStream_t stream);
 cudaError_t launch_page_release(const PageAllocArgs &A, cudaStream_t stream);
 
+// ---- forward pass of the head update on recorded cycles ---------------------------------------------------
+// A chain = a virtual sequence: shared head-cache pages of its sequence before the page of its first entry, two
+// private pages from there (the first a copy of the shared one); pending pair = (start hidden, token at start - 1).
+struct ChainSetupArgs {
+  const int32_t *cycle_seq, *start_pos;            // [chains] sequence of the cycle; context length at its start
+  const __nv_bfloat16 *start_hidden;               // [chains, d]
+  const int32_t *seq_tok;                          // [n_seq, tok_stride] committed tokens
+  const int32_t *scratch_pages;                    // [chains, 2] private page ids in the head pool
+  const int32_t *head_page_table;                  // [n_seq, max_pages_per_seq]
+  __nv_bfloat16 *pool;                             // head pool [1][2][num_pages][n_kv][16][hd]
+  int n_seq, tok_stride, k, d, vocab, max_pages_per_seq, num_pages, page_elems, pend_stride;
+  int32_t *v_kv_len, *v_pending_n, *v_pending_tok, *v_table;
+  __nv_bfloat16 *v_pending_hidden;
+  uint32_t *status;
+};
+cudaError_t launch_chain_setup(const ChainSetupArgs &A, int chains, cudaStream_t stream);
+// out[b*QT + j] = seq_hidden[b][base + j] for j < row_n[b]
+cudaError_t launch_gather_chunk_hidden(const __nv_bfloat16 *seq_hidden, int hid_stride, int base, int batch, int QT, int d,
+                                       const int32_t *row_n, __nv_bfloat16 *out, cudaStream_t stream);
+struct OverlapArgs {
+  const __nv_bfloat16 *logits;                     // [rows, V] head logits of the reconstructed chains
+  const int32_t *top_index;                        // [rows, 64]
+  const __nv_bfloat16 *top_logprob;                // [rows, 64]
+  float *alpha;                                    // [rows]
+  int V;
+  float inv_temp;
+};
+cudaError_t launch_overlap(const OverlapArgs &A, int rows, cudaStream_t stream);
+cudaError_t launch_dca_loss(const float *alpha, const int32_t *accepted, int n, int K, float *loss, float *mean,
+                            cudaStream_t stream);
+
 // ---- element-wise --------------------------------------------------------------------------------------
 // x[m] = embed[token(m)] (fp32), xn[m] = RMSNorm(x[m]; w) (bf16); rows m = b*QT + j of the verify phase.
 cudaError_t launch_embed_norm(const __nv_bfloat16 *embed, const __nv_bfloat16 *w, const int32_t *pending_tok,

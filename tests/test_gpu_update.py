@@ -1,0 +1,143 @@
+"""Forward pass of the head update on the device (head-cache rebuild from recorded pairs, draft-path reconstruction
+through virtual page tables, overlaps from the top-64 record, DCA / VGM objective) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import model as omodel, record as orecord, sampler as osampler, step as ostep, update as oupdate
+from synth_inputs import get_config, make_page_tables, make_weights, random_prompts
+from synth_inputs.weights import perturb_norm_weights
+
+from helpers import rel_err
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-2
+T = 0.2          # sharpens the nearly flat random-init distributions so that chains get rejected
+
+
+def _oracle_rollout(cfg, w, n_steps):
+    B, K = cfg.batch, cfg.k
+    prompts = random_prompts(B, cfg.prompt_len, cfg.vocab, seed=1)
+    pt, npg = make_page_tables(np.full(B, 96), cfg.page_size, seed=7)
+    hpt, hnpg = make_page_tables(np.full(B, 96), cfg.page_size, seed=8)
+    st = ostep.prefill(w, cfg, prompts, pt, npg, hpt, hnpg, temperature=T, seed=5)
+    cycles = []
+    for it in range(n_steps):
+        lens = [len(s.tokens) for s in st.seqs]
+        start_h = [s.pending_hidden[-1].copy() for s in st.seqs]
+        out = ostep.spec_step(w, cfg, st, K, T, seed=5)
+        for b in range(B):
+            cycles.append((b, orecord.cycle_record(start_h[b], out["draft_tok"][b], out["target_logits"][b],
+                                                   out["accept_len"][b], lens[b], T)))
+    seqs = []
+    for s in st.seqs:
+        kv = omodel.PagedKV(cfg.n_layers, cfg.n_kv_heads, cfg.head_dim, np.arange(16)[None, :], 16)
+        H = omodel.target_forward(w, s.tokens[:-1], np.arange(len(s.tokens) - 1), kv, 0, cfg)
+        seqs.append((omodel.round_bf16(H).astype(np.float64), list(s.tokens)))
+    return st, cycles, seqs, hpt, hnpg
+
+
+def test_head_update_forward_matches_the_oracle():
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny").with_(prompt_len=12)
+    B, K, V, d = cfg.batch, cfg.k, cfg.vocab, cfg.d_model
+    w = perturb_norm_weights(make_weights(cfg, 0))
+    st, cycles, seqs, hpt, hnpg = _oracle_rollout(cfg, w, n_steps=5)
+    n = len(cycles)
+    assert any(r["accepted"] <= K for _, r in cycles) and any(r["accepted"] == K + 1 for _, r in cycles)
+
+    ctx = gmb.Context(cfg, gmb.pack_weights(w), B, K, hpt.shape[1], hnpg, hnpg + 2 * n)     # spare pages for the chains
+    gst = gmb.State(ctx, B, hpt, hpt)
+    S = max(len(t) for _, t in seqs)
+    seq_tok = np.zeros((B, S), np.int32)
+    seq_hid = np.zeros((B, S, d), np.float32)
+    seq_len = np.zeros(B, np.int32)
+    for b, (H, toks) in enumerate(seqs):
+        seq_tok[b, :len(toks)] = toks
+        seq_hid[b, :len(toks) - 1] = H
+        seq_len[b] = len(toks)
+    tok_d = torch.from_numpy(seq_tok).cuda()
+    hid_d = torch.from_numpy(seq_hid).to(device="cuda", dtype=torch.bfloat16)
+    gmb.gm_head_prefill(ctx, gst, hid_d, tok_d, torch.from_numpy(seq_len).cuda(), int(seq_len.max()))
+    assert gmb.gm_last_status(ctx) == 0
+    # the rebuilt prefix cache = the oracle's head over the recorded pairs
+    hkv = omodel.PagedKV(1, cfg.n_kv_heads, cfg.head_dim, hpt, hnpg + 2 * n, cfg.page_size)
+    hkv.pool = gst.head_kv_pool.float().cpu().numpy().astype(np.float64)
+    for b, (H, toks) in enumerate(seqs):
+        L = len(toks)
+        ref = omodel.PagedKV(1, cfg.n_kv_heads, cfg.head_dim, np.arange(8)[None, :], 8, cfg.page_size)
+        omodel.head_forward(w, H, toks[1:], np.arange(L - 1), ref, 0, cfg)
+        for got, want in zip(hkv.gather(0, b, L - 1), ref.gather(0, 0, L - 1)):
+            assert rel_err(got, want) < TOL
+
+    rec = gmb.Record(n, K, d)
+    rec.start_hidden.copy_(torch.from_numpy(np.stack([r["start_hidden"] for _, r in cycles])).to(torch.bfloat16))
+    rec.start_pos.copy_(torch.tensor([r["start_pos"] for _, r in cycles], dtype=torch.int32))
+    rec.drafts.copy_(torch.from_numpy(np.stack([r["drafts"] for _, r in cycles]).astype(np.int32)))
+    rec.top_index.copy_(torch.from_numpy(np.stack([r["top_index"] for _, r in cycles]).astype(np.int32)))
+    rec.top_logprob.copy_(torch.from_numpy(np.stack([r["top_logprob"] for _, r in cycles])).to(torch.bfloat16))
+    rec.accepted.copy_(torch.tensor([r["accepted"] for _, r in cycles], dtype=torch.int32))
+    cycle_seq = torch.tensor([b for b, _ in cycles], dtype=torch.int32, device="cuda")
+    scratch = torch.arange(hnpg, hnpg + 2 * n, dtype=torch.int32, device="cuda").reshape(n, 2)
+    logits = torch.zeros((n, K, V), dtype=torch.bfloat16, device="cuda")
+    shared = torch.as_tensor(hpt[hpt >= 0], device="cuda", dtype=torch.long)
+    before = gst.head_kv_pool[:, :, shared].clone()
+    gmb.gm_reconstruct(ctx, gst, n, K, cycle_seq, rec, tok_d, scratch, logits)        # 20 chains, 4 per pass
+    assert gmb.gm_last_status(ctx) == 0
+    assert torch.equal(gst.head_kv_pool[:, :, shared], before)                         # chains wrote to their own pages only
+
+    lg = logits.float().cpu().numpy()
+    worst = 0.0
+    ref_alpha = np.zeros((n, K))
+    for i, (b, r) in enumerate(cycles):
+        q, ref_lg = oupdate.reconstruct_chain(w, cfg, seqs[b][0], seqs[b][1], r["start_pos"], r["drafts"], T)
+        worst = max(worst, rel_err(lg[i], ref_lg))
+        ref_alpha[i] = oupdate.chain_alphas(r, q)
+    assert worst < TOL, worst
+
+    alpha = torch.zeros((n, K), dtype=torch.float32, device="cuda")
+    gmb.gm_overlap(ctx, n, K, T, logits, rec, alpha)
+    al = alpha.cpu().numpy()
+    for i, (b, r) in enumerate(cycles):                     # the kernel itself: the oracle's overlap on the device's logits
+        want = oupdate.chain_alphas(r, osampler.softmax_probs(lg[i], T))
+        np.testing.assert_allclose(al[i], want, atol=3e-5)
+    assert np.abs(al - ref_alpha).max() < 3e-2              # end to end: bf16 forward passes on both sides
+    assert al.min() > 0 and al.max() <= 1 + 1e-4 and al.std() > 1e-3
+
+    loss = torch.zeros(n, dtype=torch.float32, device="cuda")
+    mean = torch.zeros(1, dtype=torch.float32, device="cuda")
+    gmb.gm_dca_loss(ctx, n, K, alpha, rec.accepted, loss, mean)
+    want = np.array([oupdate.dca_loss(al[i], cycles[i][1]["accepted"]) for i in range(n)])
+    np.testing.assert_allclose(loss.cpu().numpy(), want, rtol=2e-5, atol=2e-6)
+    assert float(mean[0]) == pytest.approx(want.mean(), rel=1e-5)
+    ref_loss, _ = oupdate.head_update_loss(w, cfg, seqs, cycles, T)
+    assert abs(float(mean[0]) - ref_loss) < 3e-2
+    ctx.close()
+
+
+def test_loss_kernel_edge_cases():
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny")
+    ctx = gmb.Context(cfg, gmb.random_packed_weights(cfg, "cuda"), 4, 7, 4, 8, 8)
+    rng = np.random.default_rng(2)
+    n, K = 2500, 7
+    al = rng.uniform(0.01, 1.0, (n, K)).astype(np.float32)
+    acc = rng.integers(1, K + 2, n).astype(np.int32)
+    al[0] = 1.0; acc[0] = K + 1                              # perfect head: -log K
+    al[1, 0] = 0.0                                           # dead chain: +inf
+    al[2, 1] = 0.0; acc[2] = 5                               # dies after the first position: -log alpha_1
+    loss = torch.zeros(n, dtype=torch.float32, device="cuda")
+    mean = torch.zeros(1, dtype=torch.float32, device="cuda")
+    gmb.gm_dca_loss(ctx, n, K, torch.from_numpy(al).cuda(), torch.from_numpy(acc).cuda(), loss, mean)
+    got = loss.cpu().numpy()
+    want = np.array([oupdate.dca_loss(al[i], acc[i]) for i in range(n)])
+    assert got[0] == pytest.approx(-np.log(K), rel=1e-6) and np.isinf(got[1]) and got[2] == pytest.approx(-np.log(al[2, 0]), rel=1e-5)
+    fin = np.isfinite(want)
+    np.testing.assert_allclose(got[fin], want[fin], rtol=3e-5, atol=3e-6)
+    assert np.isinf(float(mean[0]))
+    al[1, 0] = 0.5
+    gmb.gm_dca_loss(ctx, n, K, torch.from_numpy(al).cuda(), torch.from_numpy(acc).cuda(), loss, mean)
+    want = np.array([oupdate.dca_loss(al[i], acc[i]) for i in range(n)])
+    assert float(mean[0]) == pytest.approx(want.mean(), rel=1e-5)
+    ctx.close()
