@@ -338,6 +338,13 @@ int gm_spec_step_rec(gm_ctx *ctx, gm_state *st, int k, float temperature, uint64
  * gm_dca_loss: loss[r] = -log sum_{l=1..min(accepted[r], k)} prod_{i<=l} alpha[r, i] (Eq. 9; accepted =
  *   accepted drafts + 1 = the first rejected position, k + 1 if none), evaluated in the log domain (Eq. 7);
  *   mean[0] = their mean, added in a fixed order.  A chain whose first overlap is 0 gives +inf.           */
+/* Rollout-time capture of the target hidden states (App. D.2: every sequence also stores the rollout-time
+ * target hidden states of the prompt and of all committed tokens).  While seq_hidden (device bf16
+ * [max_batch, stride, d]) is set, gm_prefill writes H_0..H_{L-1} of every prompt and every committing
+ * gm_accept / gm_spec_step* / gm_rollout_step writes the hidden states of the positions it commits, so that
+ * row b holds H_i at index i - what gm_head_prefill consumes.  Positions >= stride are dropped.  NULL
+ * switches the capture off.  A captured CUDA graph (GM_FLAG_GRAPH) keeps the setting it was captured with. */
+int gm_capture_hidden(gm_ctx *ctx, void *seq_hidden, int stride);
 int gm_head_prefill(gm_ctx *ctx, gm_state *st, const void *seq_hidden, int hid_stride,
                     const int32_t *seq_tok, int tok_stride, const int32_t *seq_len, int max_len);
 int gm_reconstruct(gm_ctx *ctx, gm_state *st, int n_cycles, int k, const int32_t *cycle_seq,

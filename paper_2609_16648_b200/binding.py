@@ -24,7 +24,7 @@ GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER, GM_KC_RECORD = 0,
 
 EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw", "gm_set_top_p", "gm_nucleus", "gm_prefill",
            "gm_rollout_begin", "gm_rollout_step", "gm_rollout_run", "gm_pages_reset", "gm_pages_reserve",
-           "gm_pages_release", "gm_pages_free_count", "gm_head_prefill", "gm_reconstruct", "gm_overlap", "gm_dca_loss",
+           "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_overlap", "gm_dca_loss",
            "gm_spec_step_host", "gm_gemm", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
            "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
@@ -91,6 +91,7 @@ def lib() -> C.CDLL:
     L.gm_rollout_run.argtypes = [vp, C.POINTER(gm_state), C.POINTER(gm_rollout), i32, f32, u64, u64, i32, i32,
                                  C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     L.gm_pages_reset.argtypes = [vp, C.POINTER(gm_state)]
+    L.gm_capture_hidden.argtypes = [vp, vp, i32]
     L.gm_head_prefill.argtypes = [vp, C.POINTER(gm_state), vp, i32, vp, i32, vp, i32]
     L.gm_reconstruct.argtypes = [vp, C.POINTER(gm_state), i32, i32, vp, C.POINTER(gm_record), vp, i32, vp, vp]
     L.gm_overlap.argtypes = [vp, i32, i32, f32, vp, C.POINTER(gm_record), vp]
@@ -366,6 +367,13 @@ def gm_rollout_run(ctx: Context, st: State, ro: Rollout, k: int, temperature: fl
     _check(lib().gm_rollout_run(ctx.handle, C.byref(st.struct()), C.byref(ro.struct()), k, temperature, seed, first_step,
                                 max_steps, check_every, C.byref(steps), C.byref(running)), "gm_rollout_run")
     return steps.value, running.value
+
+
+def gm_capture_hidden(ctx: Context, seq_hidden):
+    """seq_hidden: bf16 [max_batch, stride, d] on the device, or None to stop capturing."""
+    ctx._capture = seq_hidden                                # keeps the buffer alive
+    _check(lib().gm_capture_hidden(ctx.handle, _p(seq_hidden), 0 if seq_hidden is None else seq_hidden.shape[1]),
+           "gm_capture_hidden")
 
 
 def gm_head_prefill(ctx: Context, st: State, seq_hidden, seq_tok, seq_len, max_len: int):

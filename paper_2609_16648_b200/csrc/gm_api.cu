@@ -81,6 +81,8 @@ struct gm_ctx {
   // chains of a reconstruction: virtual sequences (allocated on first use)
   int32_t *v_kv_len = nullptr, *v_pending_n = nullptr, *v_pending_tok = nullptr, *v_table = nullptr;
   __nv_bfloat16 *v_pending_hidden = nullptr;
+  __nv_bfloat16 *capture = nullptr;         // gm_capture_hidden: [max_batch, capture_stride, d] or null
+  int capture_stride = 0;
   float top_p = 1.f;                    // nucleus of the target distributions (1 = none)
   __nv_bfloat16 *ws_nucleus = nullptr;  // [max_batch (max_k + 1)][V] filtered target rows, allocated by gm_set_top_p
   std::vector<void *> allocs;
@@ -687,6 +689,9 @@ int gm_prefill(gm_ctx *c, gm_state *st, const int32_t *prompt_tok, const int32_t
                      last ? c->pf_hidden : nullptr);
       if (rc) return rc;
     }
+    if (c->capture)
+      GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+                launch_capture_chunk(c->pf_hidden, c->pf_row_n, B, QT, base, c->d, c->capture, c->capture_stride, c->stream));
     GM_LAUNCH(c, GM_KC_ELEMENTWISE,
               launch_prefill_last(c->x, c->pf_hidden, c->pf_row_n, prompt_len, B, base, QT, c->d, QT, c->pf_xlast,
                                   static_cast<__nv_bfloat16 *>(st->pending_hidden), c->stream));
@@ -762,6 +767,17 @@ int gm_accept(gm_ctx *c, gm_state *st, int batch, int k, float temperature, cons
     S.d_model = c->d; S.max_k = c->cfg.max_k;
   }
   GM_LAUNCH(c, GM_KC_SAMPLER, run_sampler(c, S, batch));
+  if (commit_state && c->capture)
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+              launch_capture_cycle(static_cast<const __nv_bfloat16 *>(target_hidden), accept_len, st->kv_len,
+                                   c->finished_mask, batch, k, c->d, c->capture, c->capture_stride, c->stream));
+  return GM_OK;
+}
+
+int gm_capture_hidden(gm_ctx *c, void *seq_hidden, int stride) {
+  if (!c || (seq_hidden && stride < 1)) return GM_ERR_INVALID_ARG;
+  c->capture = static_cast<__nv_bfloat16 *>(seq_hidden);
+  c->capture_stride = seq_hidden ? stride : 0;
   return GM_OK;
 }
 

@@ -192,6 +192,16 @@ struct OverlapArgs {
   float inv_temp;
 };
 cudaError_t launch_overlap(const OverlapArgs &A, int rows, cudaStream_t stream);
+// Rollout-time capture of the target hidden states of committed positions (App. D.2: "each sequence additionally
+// stores the rollout-time target hidden states"): dst[b][pos] = the hidden state computed at position pos.
+//   chunk form (prefill): rows j < row_n[b] of src [B, QT, d] go to positions base + j;
+//   cycle form: rows l <= accept_len[b] of src [B, k+1, d] go to positions kv_len[b] - (accept_len[b] + 1) + l, with
+//   kv_len already advanced by the commit; rows of finished sequences are skipped.
+cudaError_t launch_capture_chunk(const __nv_bfloat16 *src, const int32_t *row_n, int batch, int QT, int base, int d,
+                                 __nv_bfloat16 *dst, int dst_stride, cudaStream_t stream);
+cudaError_t launch_capture_cycle(const __nv_bfloat16 *src, const int32_t *accept_len, const int32_t *kv_len,
+                                 const int32_t *finished, int batch, int k, int d, __nv_bfloat16 *dst, int dst_stride,
+                                 cudaStream_t stream);
 cudaError_t launch_dca_loss(const float *alpha, const int32_t *accepted, int n, int K, float *loss, float *mean,
                             cudaStream_t stream);
 

@@ -164,7 +164,42 @@ __global__ void __launch_bounds__(DL_THREADS) dca_loss_kernel(const float *alpha
   if (threadIdx.x == 0) *mean = static_cast<float>(red[0] / static_cast<double>(n));
 }
 
+__global__ void __launch_bounds__(128)
+capture_chunk_kernel(const __nv_bfloat16 *src, const int32_t *row_n, int QT, int base, int d, __nv_bfloat16 *dst,
+                     int dst_stride) {
+  const int m = blockIdx.x, b = m / QT, j = m % QT;
+  pdl_prologue();
+  if (j >= row_n[b] || base + j >= dst_stride) return;
+  const uint4 *s = reinterpret_cast<const uint4 *>(src + static_cast<size_t>(m) * d);
+  uint4 *o = reinterpret_cast<uint4 *>(dst + (static_cast<size_t>(b) * dst_stride + base + j) * d);
+  for (int i = threadIdx.x; i < d / 8; i += blockDim.x) o[i] = s[i];
+}
+__global__ void __launch_bounds__(128)
+capture_cycle_kernel(const __nv_bfloat16 *src, const int32_t *accept_len, const int32_t *kv_len, const int32_t *finished,
+                     int k, int d, __nv_bfloat16 *dst, int dst_stride) {
+  const int b = blockIdx.x / (k + 1), l = blockIdx.x % (k + 1);
+  pdl_prologue();
+  if (finished && finished[b]) return;
+  const int a = accept_len[b];
+  const int pos = kv_len[b] - (a + 1) + l;
+  if (l > a || pos < 0 || pos >= dst_stride) return;
+  const uint4 *s = reinterpret_cast<const uint4 *>(src + static_cast<size_t>(blockIdx.x) * d);
+  uint4 *o = reinterpret_cast<uint4 *>(dst + (static_cast<size_t>(b) * dst_stride + pos) * d);
+  for (int i = threadIdx.x; i < d / 8; i += blockDim.x) o[i] = s[i];
+}
+
 }  // namespace
+
+cudaError_t launch_capture_chunk(const __nv_bfloat16 *src, const int32_t *row_n, int batch, int QT, int base, int d,
+                                 __nv_bfloat16 *dst, int dst_stride, cudaStream_t stream) {
+  return launch_k(capture_chunk_kernel, dim3(batch * QT), dim3(128), 0, stream, 1, src, row_n, QT, base, d, dst, dst_stride);
+}
+cudaError_t launch_capture_cycle(const __nv_bfloat16 *src, const int32_t *accept_len, const int32_t *kv_len,
+                                 const int32_t *finished, int batch, int k, int d, __nv_bfloat16 *dst, int dst_stride,
+                                 cudaStream_t stream) {
+  return launch_k(capture_cycle_kernel, dim3(batch * (k + 1)), dim3(128), 0, stream, 1, src, accept_len, kv_len, finished,
+                  k, d, dst, dst_stride);
+}
 
 cudaError_t launch_chain_setup(const ChainSetupArgs &A, int chains, cudaStream_t stream) {
   return launch_k(chain_setup_kernel, dim3(chains), dim3(128), 0, stream, 1, A);

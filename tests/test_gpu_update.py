@@ -141,3 +141,81 @@ def test_loss_kernel_edge_cases():
     want = np.array([oupdate.dca_loss(al[i], acc[i]) for i in range(n)])
     assert float(mean[0]) == pytest.approx(want.mean(), rel=1e-5)
     ctx.close()
+
+
+def test_device_pipeline_reconstruction_reproduces_the_rollouts_draft_logits():
+    """Prefill -> cycles with records and hidden capture -> head-cache rebuild in a fresh state -> reconstruction:
+    the replayed chains give back the draft logits the rollout itself computed (the property Eq. 4 is built for),
+    through the device path alone, with ragged prompts and rejected chains."""
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny")
+    B, K, V, d = cfg.batch, cfg.k, cfg.vocab, cfg.d_model
+    w = perturb_norm_weights(make_weights(cfg, 0))
+    lengths = [9, 14, 20, 11]
+    n_steps = 6
+    n = n_steps * B
+    cap = max(lengths) + n_steps * (K + 1) + 8
+    pt, npg = make_page_tables(np.full(B, cap), cfg.page_size, seed=7)
+    hpt, hnpg = make_page_tables(np.full(B, cap), cfg.page_size, seed=8)
+    ctx = gmb.Context(cfg, gmb.pack_weights(w), B, K, pt.shape[1], npg, hnpg + 2 * n)
+    st = gmb.State(ctx, B, pt, hpt)
+    rng = np.random.default_rng(5)
+    S = cap + 4
+    seq_tok = np.zeros((B, S), np.int32)
+    for b, L in enumerate(lengths):
+        seq_tok[b, :L] = rng.integers(0, V, L)
+    capture = torch.zeros((B, S, d), dtype=torch.bfloat16, device="cuda")
+    gmb.gm_capture_hidden(ctx, capture)
+    first = torch.zeros(B, dtype=torch.int32, device="cuda")
+    gmb.gm_prefill(ctx, st, torch.from_numpy(seq_tok).cuda(), torch.tensor(lengths, dtype=torch.int32, device="cuda"),
+                   max(lengths), T, None, 3, first)
+    cur = list(lengths)
+    for b in range(B):
+        seq_tok[b, cur[b]] = int(first[b]); cur[b] += 1
+    z = lambda shape, dt: torch.zeros(shape, dtype=dt, device="cuda")
+    big = gmb.Record(n, K, d)
+    saved_logits, accepted_all = [], []
+    for it in range(n_steps):
+        rec = gmb.Record(B, K, d)
+        dtok, dl = z((B, K), torch.int32), z((B, K, V), torch.bfloat16)
+        tl, th = z((B, K + 1, V), torch.bfloat16), z((B, K + 1, d), torch.bfloat16)
+        a, t = z((B,), torch.int32), z((B,), torch.int32)
+        gmb.gm_record_begin(ctx, st, rec)
+        gmb.gm_draft(ctx, st, K, T, None, 3, 1 + it, dtok, dl)
+        gmb.gm_verify(ctx, st, K, dtok, tl, th)
+        gmb.gm_accept(ctx, st, B, K, T, tl, dl, dtok, None, 3, 1 + it, a, t, None, None, th, commit_state=True)
+        gmb.gm_record_end(ctx, B, K, T, tl, dtok, a, rec)
+        saved_logits.append(dl.clone())
+        an, tn, dn = a.cpu().numpy(), t.cpu().numpy(), dtok.cpu().numpy()
+        accepted_all.append(an.copy())
+        for b in range(B):
+            new = [int(x) for x in dn[b, :an[b]]] + [int(tn[b])]
+            seq_tok[b, cur[b]:cur[b] + len(new)] = new
+            cur[b] += len(new)
+        for name in ("start_hidden", "start_pos", "drafts", "top_logprob", "top_index", "accepted"):
+            getattr(big, name)[it * B:(it + 1) * B].copy_(getattr(rec, name))
+    assert gmb.gm_last_status(ctx) == 0
+    gmb.gm_capture_hidden(ctx, None)
+    acc = np.concatenate(accepted_all)
+    assert (acc < K).any()                                                   # some chains were cut short
+    np.testing.assert_array_equal(st.kv_len.cpu().numpy() + 1, cur)
+    # the captured hidden of the position before each cycle's start is that cycle's recorded start hidden
+    sp = big.start_pos.cpu().numpy()
+    for i in range(n):
+        assert torch.equal(capture[i % B, sp[i] - 2], big.start_hidden[i])
+
+    st2 = gmb.State(ctx, B, pt, hpt)                                          # a fresh state: only recorded inputs
+    tok_d = torch.from_numpy(seq_tok).cuda()
+    gmb.gm_head_prefill(ctx, st2, capture, tok_d, torch.tensor(cur, dtype=torch.int32, device="cuda"), max(cur))
+    cycle_seq = torch.arange(n, dtype=torch.int32, device="cuda") % B
+    scratch = torch.arange(hnpg, hnpg + 2 * n, dtype=torch.int32, device="cuda").reshape(n, 2)
+    logits = z((n, K, V), torch.bfloat16)
+    gmb.gm_reconstruct(ctx, st2, n, K, cycle_seq, big, tok_d, scratch, logits)
+    assert gmb.gm_last_status(ctx) == 0
+    want = torch.cat(saved_logits).float().cpu().numpy()
+    got = logits.float().cpu().numpy()
+    err = max(rel_err(got[i], want[i]) for i in range(n))
+    exact = float((got == want).mean())
+    print(f"reconstructed vs rollout-time draft logits: worst rel err {err:.2e}, bit-identical entries {exact:.4f}")
+    assert err < 1e-2 and exact > 0.9
+    ctx.close()
