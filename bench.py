@@ -313,6 +313,9 @@ def run_product(args):
     if world > 1:
         dist.barrier()
     import paper_2609_16648_b200 as gmb
+    # a stream of this rank's own (the default stream cannot be captured into a CUDA graph); everything below -
+    # the library's context, the torch ops and the timing events - runs on it
+    torch.cuda.set_stream(torch.cuda.Stream(device))
 
     K, W, S = args.k, args.warmup, args.steps
     total_steps = W + 2 * S + 12
@@ -595,12 +598,7 @@ def main():
     elif args.workload == "sampler":
         run_sampler_only(args)
     else:
-        import torch
-        if torch.cuda.is_available():
-            with torch.cuda.stream(torch.cuda.Stream()):      # a capturable stream for the library's context
-                run_product(args)
-        else:
-            run_product(args)                                 # raises: no CPU fallback
+        run_product(args)
 
 
 if __name__ == "__main__":
