@@ -462,6 +462,126 @@ def run_product(args):
         dist.destroy_process_group()
 
 
+def run_rollout(args):
+    """Whole-rollout workload on the 4B shape (not the default line): prompts of 128..1024 random tokens are
+    prefilled on the device, pages come from the library's allocator, and the rollout driver runs cycles (one
+    captured CUDA graph per cycle) with responses collected on the device.  A step is one cycle over the batch;
+    `e2e` is the whole job (prompt upload, prefill, warm-up + timed cycles, response download) by the host clock."""
+    import torch
+    import paper_2609_16648_b200 as gmb
+    from paper_2609_16648_b200.build import build
+    from synth_inputs import get_config
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the product path has no CPU fallback")
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    if rank == 0:
+        build()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.set_stream(torch.cuda.Stream(device))
+    K, W, S = args.k, args.warmup, args.steps
+    cfg = get_config("4b").with_(k=K)
+    if args.layers > 0:
+        cfg = cfg.with_(n_layers=args.layers)
+    if args.batch > 0:
+        cfg = cfg.with_(batch=args.batch)
+    B, V = cfg.batch, cfg.vocab
+    rng = np.random.default_rng(11 + rank)
+    plen = rng.integers(128, 1025, B).astype(np.int32)
+    pmax = int(plen.max())
+    tok = np.zeros((B, pmax), np.int32)
+    for b in range(B):
+        tok[b, :plen[b]] = rng.integers(0, V, plen[b])
+    cycles = W + S
+    max_new = cycles * (K + 1) + 1
+    per_seq_pages = (pmax + max_new + K + 1 + 15) // 16 + 1
+    npg = int(sum((int(l) + max_new + K + 1 + 15) // 16 + 1 for l in plen))       # what the batch can need, not B x the cap
+    packed = gmb.random_packed_weights(cfg, device, seed=rank)
+    ctx = gmb.Context(cfg, packed, B, K, per_seq_pages, npg, npg, flags=gmb.GM_FLAG_GRAPH)
+    empty = np.full((B, per_seq_pages), -1, np.int32)
+    st = gmb.State(ctx, B, empty, empty, device)
+    ro = gmb.Rollout(B, max_new, -1, device)
+    tok_h, len_h = torch.from_numpy(tok).pin_memory(), torch.from_numpy(plen).pin_memory()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    barrier()
+    t_job = time.perf_counter()
+    tok_d, len_d = tok_h.to(device, non_blocking=True), len_h.to(device, non_blocking=True)
+    gmb.gm_pages_reset(ctx, st)
+    gmb.gm_pages_reserve(ctx, st, len_d, K + 1)
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    e[0].record()
+    gmb.gm_prefill(ctx, st, tok_d, len_d, pmax, 1.0, None, 77 + rank)
+    e[1].record()
+    gmb.gm_rollout_begin(ctx, st, ro)
+    gmb.gm_rollout_run(ctx, st, ro, K, 1.0, 77 + rank, 1, W, W)
+    n0 = int(ro.out_len.sum().item())
+    len0 = int(st.kv_len.sum().item())
+    clocks = ClockSampler(local)
+    launches0 = gmb.gm_launch_count(ctx)
+    barrier()
+    clocks.start()
+    e[2].record()
+    steps, running = gmb.gm_rollout_run(ctx, st, ro, K, 1.0, 77 + rank, 1 + W, S, S)
+    e[3].record()
+    barrier()
+    clk = clocks.stop()
+    ms = e[2].elapsed_time(e[3])
+    prefill_ms = e[0].elapsed_time(e[1])
+    launches = gmb.gm_launch_count(ctx) - launches0
+    out_len = ro.out_len.cpu()
+    resp = ro.out_tok.cpu()                                   # the responses leave the device
+    torch.cuda.synchronize()
+    job_s = time.perf_counter() - t_job
+    committed = int(out_len.sum().item()) - n0
+    len1 = int(st.kv_len.sum().item())
+    status = gmb.gm_last_status(ctx)
+    if status != 0 or steps != S or running != B:
+        raise RuntimeError(f"rollout workload: status {status}, {steps} cycles, {running} rows running")
+    free_t, free_h = gmb.gm_pages_free_count(ctx)
+    (ms_max, job_ms_max, prefill_ms_max), (committed_all, launches_all, tokens_job, prompt_tokens) = reduce_over_ranks(
+        [ms, job_s * 1e3, prefill_ms], [committed, launches, int(out_len.sum().item()), int(plen.sum())], device, world)
+    if rank == 0:
+        hbm, _, which = measured_peaks()
+        step_bytes = algorithmic_bytes_per_step(cfg, K, 0.5 * (len0 + len1))
+        achieved = step_bytes / (ms_max / S * 1e-3) / 1e9
+        line = {"metric": METRIC, "value": committed_all / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": S,
+                "warmup": W, "ms_per_step": ms_max / S, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": "rollout", "n_layers": cfg.n_layers, "batch_per_gpu": B, "k": K, "temperature": 1.0,
+                           "prompt_len": "uniform 128..1024", "prompt_tokens": int(prompt_tokens),
+                           "prefill_ms": prefill_ms_max, "prefill_tokens_per_s": prompt_tokens / (prefill_ms_max * 1e-3),
+                           "kv_len_mean": 0.5 * (len0 + len1) / B, "tau": committed / (S * B),
+                           "pages": {"pool": npg, "free_after": free_t}, "launch": "one captured CUDA graph per cycle",
+                           "parallelism": f"replicas x{world}",
+                           "l2": "per-cycle working set (weights + KV) >> 126 MB L2: no flush needed", "peaks": which},
+                "clocks": clk,
+                "e2e": {"value": tokens_job / (job_ms_max * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 0,
+                        "d2h_bytes_per_step": 0, "h2d_bytes_per_job": int(tok.nbytes + plen.nbytes),
+                        "d2h_bytes_per_job": int(resp.numel() * 4 + out_len.numel() * 4), "job_ms": job_ms_max,
+                        "note": "whole job by the host clock: prompt upload, page reservation, prefill, warm-up and timed "
+                                "cycles, response download; response tokens / job time"},
+                "gpu_launches": int(launches_all),
+                "roofline": {"kernel": "whole cycle (per-kernel events are not recorded inside a replayed graph)",
+                             "bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s", "frac": achieved / hbm,
+                             "traffic": None, "algorithmic_bytes_per_launch": step_bytes, "peak_source": which},
+                "cpu_baseline": None}
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def run_sampler_only(args):
     """Sampler-only workload: 256 sequences x (k+1) positions over the 151936-token vocabulary.  A step is one
     gm_accept over the whole batch (the draft tokens were drawn once, on the device, by gm_draw)."""
@@ -581,7 +701,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="4b", choices=["tiny", "4b", "7b", "longtail", "sampler"])
+    ap.add_argument("--workload", default="4b", choices=["tiny", "4b", "7b", "longtail", "sampler", "rollout"])
     ap.add_argument("--k", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (small profiling cases)")
@@ -597,6 +717,8 @@ def main():
         run_reference(args)
     elif args.workload == "sampler":
         run_sampler_only(args)
+    elif args.workload == "rollout":
+        run_rollout(args)
     else:
         run_product(args)
 
