@@ -88,15 +88,11 @@ __device__ __forceinline__ void epilogue4(const GemmArgs &A, int m, int n, float
 }
 
 __global__ void __launch_bounds__(GT_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages_arg) {
+gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
   extern __shared__ unsigned char gt_smem_raw[];
   unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(gt_smem_raw) + 1023) & ~uintptr_t(1023));
-  // n_double > 0: a one-wave launch whose first n_double CTAs take two 128-feature sub-tiles and the rest one (their
-  // stage size, and so their stage count, differ); otherwise every CTA takes A.wtiles sub-tiles
-  const bool mixed = A.n_double > 0;
-  const int T = A.block_t, wt = mixed ? (static_cast<int>(blockIdx.x) < A.n_double ? 2 : 1) : A.wtiles;
+  const int T = A.block_t, wt = A.wtiles;
   const int a_bytes = wt * GT_BN * 128, b_bytes = T * 128, stage_b = a_bytes + b_bytes;
-  const int nstages = mixed ? min(8, GT_SMEM_BUDGET / stage_b) : nstages_arg;
   size_t pipe_b = static_cast<size_t>(nstages) * stage_b;
   if (static_cast<size_t>(T) * GT_BN * 4 > pipe_b) pipe_b = static_cast<size_t>(T) * GT_BN * 4;
   uint64_t *full = reinterpret_cast<uint64_t *>(smem + pipe_b);
@@ -106,9 +102,7 @@ gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages_arg) {
   float *park = reinterpret_cast<float *>(smem);                // [T][128] fp32, reuses the pipeline stages
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int bx = static_cast<int>(blockIdx.x);
-  const int n0 = A.n_base + (mixed ? (bx < A.n_double ? bx * 2 * GT_BN : (A.n_double + bx) * GT_BN) : bx * GT_BN * wt);
-  const int m0 = blockIdx.y * T, split = blockIdx.z, ns = A.nsplit;
+  const int n0 = A.n_base + blockIdx.x * GT_BN * wt, m0 = blockIdx.y * T, split = blockIdx.z, ns = A.nsplit;
   const int KB = A.K / GT_BK;
   const int kb_lo = static_cast<int>(static_cast<long long>(split) * KB / ns);
   const int kb_hi = static_cast<int>(static_cast<long long>(split + 1) * KB / ns);
@@ -255,10 +249,9 @@ cudaError_t gemm_tc_max_clusters(int block_t, int nsplit, int *out) {
 cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream) {
   const int T = A.block_t;
   if (T < 16 || T > 256 || (T & 15) || (A.K % GT_BK) || A.nsplit < 1 || A.nsplit > A.K / GT_BK || A.nsplit > 8 ||
-      A.wtiles < 1 || A.wtiles > 2 || A.n_tiles < 1 || A.n_base < 0 || A.n_double < 0 || A.n_double > A.n_tiles ||
-      (A.n_double > 0 && (A.nsplit != 1 || A.wtiles != 1)))
+      A.wtiles < 1 || A.wtiles > 2 || A.n_tiles < 1 || A.n_base < 0)
     return cudaErrorInvalidValue;
-  const size_t smem = A.n_double > 0 ? std::max(gt_smem(T, 1), gt_smem(T, 2)) : gt_smem(T, A.wtiles);
+  const size_t smem = gt_smem(T, A.wtiles);
   cudaError_t ec = gt_configure();
   if (ec != cudaSuccess) return ec;
   const dim3 grid(A.n_tiles, (A.M + T - 1) / T, A.nsplit);

@@ -237,15 +237,6 @@ int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *w
   // Wave quantisation: a few CTAs more than a multiple of the SM count would cost a whole extra wave.  Run the full
   // waves as they are and the leftover features as a short launch whose tiles are split along K over clusters.
   const int rem = (units * mblocks) % c->sm_count;
-  // A few tiles more than one wave: one launch of exactly one CTA per SM in which the first `rem` CTAs take two tiles.
-  static const bool no_mixed = std::getenv("GM_NO_MIXED_WAVE") != nullptr;
-  if (!no_mixed && A.nsplit == 1 && A.wtiles == 1 && mblocks == 1 && units > c->sm_count && units < 2 * c->sm_count &&
-      rem * 4 <= c->sm_count) {
-    A.n_double = rem;
-    A.n_tiles = c->sm_count;
-    GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(A, c->stream));
-    return GM_OK;
-  }
   if (A.nsplit == 1 && mblocks == 1 && units > c->sm_count && rem != 0 && rem * 4 <= c->sm_count) {
     A.n_tiles = units - rem;
     GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(A, c->stream));

@@ -290,7 +290,6 @@ struct GemmArgs {
   int wtiles;                           // 128-feature sub-tiles per CTA sharing one activation tile (1 or 2)
   size_t ldo;                           // output row stride in elements
   uint32_t *status;
-  int n_double;                         // > 0: the first n_double CTAs along N take two 128-feature sub-tiles, the others one
 };
 cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream);
 cudaError_t launch_gemm_simple(const GemmArgs &A, cudaStream_t stream);
