@@ -185,8 +185,8 @@ int gm_rollout_step(gm_ctx *ctx, gm_state *st, const gm_rollout *ro, int k, floa
  * outputs, may be NULL.  With GM_FLAG_GRAPH the first call captures one cycle (all its launches,
  * with their programmatic dependencies, the page reserve / release and the append) into a CUDA graph and
  * every cycle is one graph launch; the step index then lives in device memory and is advanced by the
- * append kernel.  The graph is re-captured when the state, the rollout buffers, k, the temperature or
- * the seed change.  Results are bit-identical to the host-launched loop.  The context must have been
+ * append kernel.  The graph is re-captured when the state, the rollout buffers, k, the temperature, the
+ * seed, top-p or the hidden-state capture change.  Results are bit-identical to the host-launched loop.  The context must have been
  * created on a stream of its own: the default streams cannot be captured, and the flag is ignored there. */
 int gm_rollout_run(gm_ctx *ctx, gm_state *st, const gm_rollout *ro, int k, float temperature,
                    uint64_t seed, uint64_t first_step, int max_steps, int check_every,
@@ -343,7 +343,7 @@ int gm_spec_step_rec(gm_ctx *ctx, gm_state *st, int k, float temperature, uint64
  * [max_batch, stride, d]) is set, gm_prefill writes H_0..H_{L-1} of every prompt and every committing
  * gm_accept / gm_spec_step* / gm_rollout_step writes the hidden states of the positions it commits, so that
  * row b holds H_i at index i - what gm_head_prefill consumes.  Positions >= stride are dropped.  NULL
- * switches the capture off.  A captured CUDA graph (GM_FLAG_GRAPH) keeps the setting it was captured with. */
+ * switches the capture off (a cycle captured as a CUDA graph is captured again when the setting changes).  */
 int gm_capture_hidden(gm_ctx *ctx, void *seq_hidden, int stride);
 int gm_head_prefill(gm_ctx *ctx, gm_state *st, const void *seq_hidden, int hid_stride,
                     const int32_t *seq_tok, int tok_stride, const int32_t *seq_len, int max_len);

@@ -838,6 +838,7 @@ static int spec_step_run(gm_ctx *c, gm_state *st, int k, float temperature, cons
   KeyBytes key;
   key.add(*st); key.add(k); key.add(temperature); key.add(u24_draft); key.add(u24_accept); key.add(seed);
   key.add(accept_len); key.add(next_token); key.add(draft_tok); key.add(c->top_p);
+  key.add(c->capture); key.add(c->capture_stride);
   rc = graph_prepare(c, c->graph_step, key.bytes, [&]() {
     return spec_step_impl(c, st, k, temperature, u24_draft, u24_accept, seed, 0, accept_len, next_token, draft_tok);
   });
@@ -1199,6 +1200,7 @@ int gm_rollout_run(gm_ctx *c, gm_state *st, const gm_rollout *ro, int k, float t
   if (use_graph && running > 0 && max_steps > 0) {
     KeyBytes key;
     key.add(*st); key.add(*ro); key.add(k); key.add(temperature); key.add(seed); key.add(c->alloc_on); key.add(c->top_p);
+    key.add(c->capture); key.add(c->capture_stride);
     if ((rc = check_state(c, st, k)) != GM_OK) return rc;
     rc = graph_prepare(c, c->graph_rollout, key.bytes, [&]() { return gm_rollout_step(c, st, ro, k, temperature, seed, 0); });
     if (rc) return rc;
