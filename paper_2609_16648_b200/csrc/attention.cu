@@ -16,6 +16,8 @@
 // ldmatrix, runs the online softmax in registers (quad shuffles for the row statistics) and
 // accumulates O += P V with V fetched by ldmatrix.trans.  The 16-row M extent is why this is the
 // warp-level MMA and not tcgen05 (whose minimum M is 64).
+#include <cstdlib>
+
 #include "common.cuh"
 #include "kernels.h"
 
@@ -308,6 +310,262 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
   }
 }
 
+
+// ---- transposed formulation for 17..24 query rows -----------------------------------------------------------------------
+// With two 16-row M tiles (rows padded to 32) the kernel above is bound by the warp-level MMA rate, not by HBM.  Here the
+// roles are swapped: the page's 16 keys are the M extent and the query rows the N extent (tiles of 8, so 24 rows are
+// exactly three tiles):  S^T = K Q^T  with K as the A operand (same ldmatrix loads, registers permuted) and Q^T as B
+// fragments held in registers;  O^T += V^T P^T  with V^T as the A operand (same ldmatrix.trans loads) and P^T obtained
+// from the S^T accumulators by an 8x8 register transpose (movmatrix).  48 MMAs per page instead of 64.
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+
+template <int HD, int NR>
+__global__ void __launch_bounds__((ATT_MAX_HPC + 1) * 32, 1)
+attention_t_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int nstages) {
+  using C = AttCfg<HD>;
+  constexpr int NSUB = C::NSUB;
+  constexpr int KSTEPS = HD / 16;
+  constexpr int MTILES = HD / 16;               // 16-wide tiles of the head dimension (M extent of O^T)
+
+  extern __shared__ unsigned char att_smem_raw[];
+  unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(att_smem_raw) + 1023) & ~uintptr_t(1023));
+  const int tile_b = C::tile_bytes(hpc);
+  const int stage_b = C::stage_bytes(hpc);
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem + static_cast<size_t>(nstages) * stage_b);
+  uint64_t *empty = full + 8;
+  unsigned char *qsm = smem + ((static_cast<size_t>(nstages) * stage_b + 128 + 1023) & ~size_t(1023));   // Q staging
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int B = A.batch;
+  pdl_prologue();
+  const long long P = A.page_start[B];
+  const long long G = P < static_cast<long long>(gridDim.x) ? P : static_cast<long long>(gridDim.x);
+  if (static_cast<long long>(blockIdx.x) >= G) return;
+  const int lo = static_cast<int>(blockIdx.x * P / G), hi = static_cast<int>((blockIdx.x + 1) * P / G);
+  const int hg = blockIdx.y;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < nstages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], hpc); }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (lo >= hi) return;
+
+  int b0 = 0;
+  {
+    int l = 0, r = B - 1;
+    while (l < r) { const int mid = (l + r + 1) >> 1; if (A.page_start[mid] <= lo) l = mid; else r = mid - 1; }
+    b0 = l;
+  }
+
+  if (warp == hpc) {
+    // ---- producer: identical to the kernel above ---------------------------------------------------------------
+    if (lane == 0) {
+      tma_prefetch_desc(&A.kv_map);
+      int b = b0;
+      const long long rows_per_page = static_cast<long long>(A.n_kv) * 16;
+      for (int p = lo, it = 0; p < hi; ++p, ++it) {
+        while (p >= A.page_start[b + 1]) ++b;
+        int page = A.page_table[static_cast<size_t>(b) * A.max_pages_per_seq + (p - A.page_start[b])];
+        if (page < 0 || page >= A.num_pages) { set_status(A.status, ST_BAD_PAGE); page = 0; }
+        const int s = it % nstages;
+        if (!mbar_wait(&empty[s], ((it / nstages) & 1) ^ 1)) { set_status(A.status, ST_TIMEOUT); break; }
+        mbar_expect_tx(&full[s], stage_b);
+        unsigned char *dst = smem + static_cast<size_t>(s) * stage_b;
+        const long long row_k = ((static_cast<long long>(A.layer) * 2 + 0) * A.num_pages + page) * rows_per_page + hg * hpc * 16;
+        const long long row_v = ((static_cast<long long>(A.layer) * 2 + 1) * A.num_pages + page) * rows_per_page + hg * hpc * 16;
+#pragma unroll
+        for (int sub = 0; sub < NSUB; ++sub) {
+          tma_load_2d(dst + sub * tile_b, &A.kv_map, sub * 64, static_cast<int>(row_k), &full[s]);
+          tma_load_2d(dst + (NSUB + sub) * tile_b, &A.kv_map, sub * 64, static_cast<int>(row_v), &full[s]);
+        }
+      }
+    }
+    return;
+  }
+  if (warp > hpc) return;
+
+  const int head = hg * hpc + warp;
+  const int t4 = lane & 3, r8 = lane >> 2;
+  const float c = A.scale_log2e;
+  const uint32_t smem_base = smem_u32(smem);
+  const int mi = lane >> 3;
+  const int k_tok = (mi >> 1) * 8 + (lane & 7), k_chunk = mi & 1;
+  const int v_tok = (mi & 1) * 8 + (lane & 7), v_chunk = mi >> 1;
+  const uint32_t k_row_off = (warp * 16 + k_tok) * 128, v_row_off = (warp * 16 + v_tok) * 128;
+  const int k_sw = k_tok & 7, v_sw = v_tok & 7;
+
+  int it = 0;
+  bool dead = false;
+  for (int b = b0; b < B && !dead; ++b) {
+    const int ps = A.page_start[b], pe = A.page_start[b + 1];
+    if (ps >= hi) break;
+    const int seg_lo = max(lo, ps), seg_hi = min(hi, pe);
+    if (seg_lo >= seg_hi) continue;
+    const int qn = A.qn[b], qbase = A.qbase[b];
+
+    // Q rows staged in shared memory (128-byte rows, XOR swizzle), fetched per page as B fragments with ldmatrix: one
+    // x4 load gives (k lo, k hi) of two consecutive K steps for the 8 rows of a tile.  (In registers they would be 48
+    // more per thread, and this kernel's 9 warps are limited to 168.)
+    const __nv_bfloat16 *qp = A.qbuf + (static_cast<size_t>(b) * A.n_kv + head) * A.qrows * HD;
+    unsigned char *q_stage = qsm + warp * (NR * 8 * HD * 2);
+    const uint32_t q_smem = smem_u32(q_stage);
+    __syncwarp();                                 // the previous segment's fragment reads are done
+    {
+      constexpr int CPR = HD / 8;                 // 16-byte chunks per row
+      for (int idx = lane; idx < NR * 8 * CPR; idx += 32) {
+        const int row = idx / CPR, ch = idx % CPR;
+        const uint4 v = *reinterpret_cast<const uint4 *>(qp + row * HD + ch * 8);
+        *reinterpret_cast<uint4 *>(q_stage + (ch >> 3) * (NR * 8 * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) = v;
+      }
+    }
+    __syncwarp();
+    const int qb_row = lane & 7, qb_chunk = lane >> 3;   // ldmatrix lane address: 8 rows x (4 chunks = 2 K steps)
+    float ot[MTILES][NR][4];
+    float mrow[NR][2], lrow[NR][2];
+#pragma unroll
+    for (int nr = 0; nr < NR; ++nr) {
+      mrow[nr][0] = mrow[nr][1] = -INFINITY;
+      lrow[nr][0] = lrow[nr][1] = 0.f;
+#pragma unroll
+      for (int mt = 0; mt < MTILES; ++mt) ot[mt][nr][0] = ot[mt][nr][1] = ot[mt][nr][2] = ot[mt][nr][3] = 0.f;
+    }
+
+    for (int p = seg_lo; p < seg_hi; ++p, ++it) {
+      const int s = it % nstages;
+      if (!mbar_wait(&full[s], (it / nstages) & 1)) { set_status(A.status, ST_TIMEOUT); dead = true; break; }
+      const uint32_t kbase = smem_base + s * stage_b, vbase = kbase + NSUB * tile_b;
+
+      // S^T[key][row]: accumulator e of tile nr = (key r8 + 8*(e>>1), row nr*8 + 2*t4 + (e&1))
+      float st[NR][4];
+#pragma unroll
+      for (int nr = 0; nr < NR; ++nr) st[nr][0] = st[nr][1] = st[nr][2] = st[nr][3] = 0.f;
+#pragma unroll
+      for (int kp = 0; kp < KSTEPS / 2; ++kp) {
+        uint32_t kf0[4], kf1[4];
+        const int ks0 = 2 * kp, ks1 = 2 * kp + 1;
+        ldmatrix_x4(kf0, kbase + (ks0 >> 2) * tile_b + k_row_off + (((((ks0 & 3) * 2 + k_chunk)) ^ k_sw) << 4));
+        ldmatrix_x4(kf1, kbase + (ks1 >> 2) * tile_b + k_row_off + (((((ks1 & 3) * 2 + k_chunk)) ^ k_sw) << 4));
+        // A operand = keys x k: (keys 0-7, k lo) (keys 8-15, k lo) (keys 0-7, k hi) (keys 8-15, k hi)
+        const uint32_t a0[4] = {kf0[0], kf0[2], kf0[1], kf0[3]};
+        const uint32_t a1[4] = {kf1[0], kf1[2], kf1[1], kf1[3]};
+#pragma unroll
+        for (int nr = 0; nr < NR; ++nr) {
+          uint32_t qf[4];                               // (ks0: k lo, k hi) (ks1: k lo, k hi) of rows nr*8 .. nr*8+7
+          const int row = nr * 8 + qb_row, ch = (ks0 & 3) * 2 + qb_chunk;
+          ldmatrix_x4(qf, q_smem + (ks0 >> 2) * (NR * 8 * 128) + row * 128 + ((ch ^ (row & 7)) << 4));
+          mma_16816(st[nr], a0, qf[0], qf[1]);
+          mma_16816(st[nr], a1, qf[2], qf[3]);
+        }
+      }
+
+      const int kp0 = (p - ps) * 16;
+      const bool need_mask = kp0 + 15 > qbase;
+      uint32_t pb[NR][2];
+#pragma unroll
+      for (int nr = 0; nr < NR; ++nr) {
+        if (need_mask) {                                         // only the last pages of a sequence come here
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            // accumulator columns are query rows nr*8 + 2*t4 + e: the last key position the row may see
+            const int j = (nr * 8 + 2 * t4 + e) / A.group;
+            const int lim = j < qn ? qbase + j : -1;
+            if (kp0 + r8 > lim) st[nr][e] = -INFINITY;
+            if (kp0 + r8 + 8 > lim) st[nr][e + 2] = -INFINITY;
+          }
+        }
+        float alpha[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          float mx = fmaxf(st[nr][e], st[nr][e + 2]);             // this thread's two keys of the row
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+          const float m_new = fmaxf(mrow[nr][e], mx);
+          const float m_use = m_new == -INFINITY ? 0.f : m_new;
+          alpha[e] = exp2f((mrow[nr][e] - m_use) * c);
+          mrow[nr][e] = m_new;
+          const float mc = m_use * c;
+          const float p0 = exp2f(fmaf(st[nr][e], c, -mc)), p1 = exp2f(fmaf(st[nr][e + 2], c, -mc));
+          st[nr][e] = p0; st[nr][e + 2] = p1;
+          lrow[nr][e] = lrow[nr][e] * alpha[e] + p0 + p1;         // this thread's keys only; lanes are added at the end
+        }
+#pragma unroll
+        for (int mt = 0; mt < MTILES; ++mt) {
+          ot[mt][nr][0] *= alpha[0]; ot[mt][nr][1] *= alpha[1];
+          ot[mt][nr][2] *= alpha[0]; ot[mt][nr][3] *= alpha[1];
+        }
+        // P^T as B fragments: transpose the two 8x8 blocks (keys 0-7 and keys 8-15) held as (key r8, rows 2*t4, 2*t4+1)
+        pb[nr][0] = movmatrix_trans(pack_bf16(st[nr][0], st[nr][1]));
+        pb[nr][1] = movmatrix_trans(pack_bf16(st[nr][2], st[nr][3]));
+      }
+
+      // O^T += V^T P^T
+#pragma unroll
+      for (int n2 = 0; n2 < MTILES; ++n2) {
+        uint32_t vf[4];
+        const int chunk = (n2 & 3) * 2 + v_chunk;
+        ldmatrix_x4_trans(vf, vbase + (n2 >> 2) * tile_b + v_row_off + ((chunk ^ v_sw) << 4));
+        const uint32_t af[4] = {vf[0], vf[2], vf[1], vf[3]};      // (hd 0-7,keys lo) (hd 8-15,keys lo) (hd 0-7,keys hi) (hd 8-15,keys hi)
+#pragma unroll
+        for (int nr = 0; nr < NR; ++nr) mma_16816(ot[n2][nr], af, pb[nr][0], pb[nr][1]);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[s]);
+    }
+    if (dead) break;
+
+    // ---- write this segment's partial: part_o[slot][head][row][hd], part_ml[slot][head][row][2] ----------------------
+    const size_t slot = static_cast<size_t>(blockIdx.x) + b;
+    float *po = A.part_o + ((slot * A.n_kv + head) * A.qrows) * HD;
+    float *pml = A.part_ml + ((slot * A.n_kv + head) * A.qrows) * 2;
+    const int rows_valid = qn * A.group;
+#pragma unroll
+    for (int nr = 0; nr < NR; ++nr)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        float l = lrow[nr][e];
+        l += __shfl_xor_sync(0xffffffffu, l, 4);
+        l += __shfl_xor_sync(0xffffffffu, l, 8);
+        l += __shfl_xor_sync(0xffffffffu, l, 16);
+        const int row = nr * 8 + 2 * t4 + e;
+        if (row < rows_valid) {
+          if (r8 == 0) {
+            pml[row * 2 + 0] = mrow[nr][e] == -INFINITY ? -INFINITY : mrow[nr][e] * c;
+            pml[row * 2 + 1] = l;
+          }
+#pragma unroll
+          for (int mt = 0; mt < MTILES; ++mt) {
+            po[static_cast<size_t>(row) * HD + mt * 16 + r8] = ot[mt][nr][e];
+            po[static_cast<size_t>(row) * HD + mt * 16 + r8 + 8] = ot[mt][nr][e + 2];
+          }
+        }
+      }
+  }
+}
+
+template <int HD, int NR>
+static cudaError_t launch_att_t(const AttnArgs &A, cudaStream_t stream) {
+  // shared-memory layout of the two-tile variant: its 32-row Q staging area holds this kernel's 8*NR rows.  (A third
+  // stage - first tile's fragments in registers, smaller staging area - was measured and is no faster: the kernel is
+  // bound by instruction issue, not by the depth of the ring.)
+  const int hpc = att_hpc(A.n_kv), nst = att_stages(A.n_kv, HD, 2);
+  const size_t smem = attention_smem_bytes(A.n_kv, HD, 2);
+  static size_t configured = 0;
+  if (smem > configured) {
+    cudaError_t e = cudaFuncSetAttribute(attention_t_kernel<HD, NR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    configured = smem;
+  }
+  dim3 grid(A.n_ctas, A.n_kv / hpc);
+  return launch_k(attention_t_kernel<HD, NR>, grid, dim3((hpc + 1) * 32), smem, stream, 1, A, hpc, nst);
+}
+
 template <int HD, int MT>
 static cudaError_t launch_att(const AttnArgs &A, cudaStream_t stream) {
   const int hpc = att_hpc(A.n_kv), nst = att_stages(A.n_kv, HD, MT);
@@ -326,6 +584,9 @@ static cudaError_t launch_att(const AttnArgs &A, cudaStream_t stream) {
 cudaError_t launch_attention(const AttnArgs &A, cudaStream_t stream) {
   const int mt = A.qrows / 16;
   if (A.n_kv % att_hpc(A.n_kv) != 0) return cudaErrorInvalidValue;
+  // 17..24 query rows: the transposed formulation (three 8-row tiles) instead of two padded 16-row tiles
+  static const bool no_t = std::getenv("GM_NO_ATT_T") != nullptr;
+  if (!no_t && A.hd == 128 && mt == 2 && A.rows_used > 16 && A.rows_used <= 24) return launch_att_t<128, 3>(A, stream);
   if (A.hd == 128 && mt == 1) return launch_att<128, 1>(A, stream);
   if (A.hd == 128 && mt == 2) return launch_att<128, 2>(A, stream);
   if (A.hd == 64 && mt == 1) return launch_att<64, 1>(A, stream);

@@ -288,7 +288,7 @@ int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const 
   T.page_table = page_table; T.batch = ph.B; T.n_kv = cf.n_kv_heads; T.group = c->group; T.hd = cf.head_dim;
   T.qrows = ph.qrows; T.layer = layer; T.num_pages = num_pages; T.max_pages_per_seq = cf.max_pages_per_seq;
   T.n_ctas = c->sm_count; T.scale_log2e = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(cf.head_dim)));
-  T.part_o = c->part_o; T.part_ml = c->part_ml; T.status = c->status;
+  T.part_o = c->part_o; T.part_ml = c->part_ml; T.status = c->status; T.rows_used = ph.QT * c->group;
   GM_LAUNCH(c, GM_KC_ATTENTION, launch_attention(T, c->stream));
   AttnCombineArgs Cb;
   Cb.part_o = c->part_o; Cb.part_ml = c->part_ml; Cb.qn = c->qn; Cb.page_start = c->page_start; Cb.batch = ph.B;
@@ -969,7 +969,7 @@ int gm_attention(gm_ctx *c, const void *q, const void *kv_pool, int pool_layers,
   T.page_start = c->page_start; T.page_table = page_table; T.batch = batch; T.n_kv = cf.n_kv_heads; T.group = c->group;
   T.hd = cf.head_dim; T.qrows = qrows; T.layer = layer; T.num_pages = num_pages; T.max_pages_per_seq = cf.max_pages_per_seq;
   T.n_ctas = c->sm_count; T.scale_log2e = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(cf.head_dim)));
-  T.part_o = c->part_o; T.part_ml = c->part_ml; T.status = c->status;
+  T.part_o = c->part_o; T.part_ml = c->part_ml; T.status = c->status; T.rows_used = q_stride * c->group;
   GM_LAUNCH(c, GM_KC_ATTENTION, launch_attention(T, c->stream));
   AttnCombineArgs Cb;
   Cb.part_o = c->part_o; Cb.part_ml = c->part_ml; Cb.qn = q_count; Cb.page_start = c->page_start; Cb.batch = batch;

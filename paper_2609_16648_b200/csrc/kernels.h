@@ -256,6 +256,7 @@ struct AttnArgs {
   float *part_o;                        // [n_ctas + B][n_kv][qrows][hd] partial outputs
   float *part_ml;                       // [n_ctas + B][n_kv][qrows][2] partial (max, sum)
   uint32_t *status;
+  int rows_used = 0;                    // query rows a sequence can have (q positions x group); 0 = unknown (qrows is assumed)
 };
 cudaError_t launch_attention(const AttnArgs &A, cudaStream_t stream);
 struct AttnCombineArgs {
