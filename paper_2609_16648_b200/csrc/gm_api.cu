@@ -1,21 +1,6 @@
 // C ABI of libgm: context, workspaces, tensor maps and the launch sequences of the draft, verify and
 // accept phases.  Host code only; every step of the path runs in the kernels of this directory.
-#include <cmath>
-#include <cstdio>
-#include <cstdlib>
-#include <cstring>
-#include <map>
-#include <new>
-#include <tuple>
-#include <vector>
-
-#include <cudaTypedefs.h>
-
-#include "../../include/gm.h"
-#include "common.cuh"
-#include "kernels.h"
-
-using namespace gm;
+#include "gm_internal.h"
 
 namespace gm {
 bool pdl_enabled() {
@@ -24,124 +9,7 @@ bool pdl_enabled() {
 }
 }  // namespace gm
 
-namespace {
-
-struct LayerMaps { CUtensorMap wqkv, wo, wgu, wdown; };
-
-struct EventPair { cudaEvent_t a, b; };
-
-}  // namespace
-
-struct gm_ctx {
-  gm_config cfg;
-  gm_weights w;
-  std::vector<gm_layer_weights> layers;
-  cudaStream_t stream = nullptr;
-  int sm_count = 148;
-  PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
-
-  // derived shapes
-  int d, q_dim, kv_dim, n_qkv, F, V, group, Mmax;
-
-  // tensor maps
-  std::vector<LayerMaps> lmaps;
-  LayerMaps head_maps;
-  CUtensorMap lm_head_map, head_proj_map;
-  std::map<std::tuple<const void *, int, int, int>, CUtensorMap> x_maps;   // (ptr, rows, K, box rows)
-  std::map<std::tuple<const void *, int, int>, CUtensorMap> w_maps;        // (ptr, N, K)   (gm_gemm only)
-  std::map<std::tuple<const void *, long long>, CUtensorMap> kv_maps;      // (pool, rows)
-
-  // workspaces (device)
-  float *x = nullptr, *g = nullptr, *part_o = nullptr, *part_ml = nullptr;
-  __nv_bfloat16 *xn = nullptr, *zin = nullptr, *qkv = nullptr, *qbuf = nullptr, *attn_out = nullptr, *act = nullptr, *gn = nullptr;
-  int max_clusters[17][9];            // resident clusters of the GEMM kernel by (block_t / 16, cluster size); -1 = not asked yet
-  __nv_bfloat16 *ws_draft_logits = nullptr, *ws_target_logits = nullptr, *ws_target_hidden = nullptr;
-  int32_t *ws_draft_tok = nullptr, *ws_accept_len = nullptr, *ws_next_token = nullptr;
-  uint32_t *ws_u24 = nullptr;
-  int32_t *qn = nullptr, *qbase = nullptr, *page_start = nullptr;
-  float2 *rope = nullptr;
-  uint32_t *status = nullptr;
-  // prompt prefill: per-chunk bookkeeping, the chunk's hidden states, the row of each prompt's last token
-  int32_t *pf_row_n = nullptr, *pf_head_n = nullptr, *pf_pair_tok = nullptr, *pf_first = nullptr;
-  __nv_bfloat16 *pf_hidden = nullptr;
-  float *pf_xlast = nullptr;
-  int32_t *ro_accept = nullptr, *ro_next = nullptr;   // per-step outputs of a rollout step
-  // captured rollout cycle (GM_FLAG_ROLLOUT_GRAPH)
-  uint64_t *dev_step = nullptr;             // step index of the captured cycle
-  uint64_t *step_ptr = nullptr;             // non-null while a cycle is being captured: kernels read the step from here
-  struct GraphSlot {                        // one captured sequence of launches and what it was captured for
-    cudaGraphExec_t exec = nullptr;
-    int64_t launches = 0;
-    std::vector<unsigned char> key;
-  } graph_rollout, graph_step;
-  const int32_t *finished_mask = nullptr;   // set around the phases of a rollout step: rows that sit out
-  // page allocator (gm_pages_*): one stack of free page ids per pool
-  bool alloc_on = false;
-  int32_t *free_list[2] = {nullptr, nullptr}, *free_top[2] = {nullptr, nullptr}, *held[2] = {nullptr, nullptr};
-  // chains of a reconstruction: virtual sequences (allocated on first use)
-  int32_t *v_kv_len = nullptr, *v_pending_n = nullptr, *v_pending_tok = nullptr, *v_table = nullptr;
-  __nv_bfloat16 *v_pending_hidden = nullptr;
-  __nv_bfloat16 *capture = nullptr;         // gm_capture_hidden: [max_batch, capture_stride, d] or null
-  int capture_stride = 0;
-  float top_p = 1.f;                    // nucleus of the target distributions (1 = none)
-  __nv_bfloat16 *ws_nucleus = nullptr;  // [max_batch (max_k + 1)][V] filtered target rows, allocated by gm_set_top_p
-  std::vector<void *> allocs;
-
-  // profiling
-  int prof_mask = 0;
-  std::vector<EventPair> events[GM_KC_COUNT];
-  size_t events_used[GM_KC_COUNT] = {};
-  int64_t launches = 0;
-  cudaError_t last_cuda = cudaSuccess;
-};
-
-namespace {
-
-#define GM_CUDA(ctx, call)                                   \
-  do {                                                       \
-    cudaError_t e__ = (call);                                \
-    if (e__ != cudaSuccess) { (ctx)->last_cuda = e__; return GM_ERR_CUDA; } \
-  } while (0)
-
-template <typename T>
-int dev_alloc(gm_ctx *c, T **p, size_t n, bool zero = true) {
-  void *q = nullptr;
-  GM_CUDA(c, cudaMalloc(&q, n * sizeof(T) > 0 ? n * sizeof(T) : 16));
-  c->allocs.push_back(q);
-  if (zero) GM_CUDA(c, cudaMemsetAsync(q, 0, n * sizeof(T), c->stream));
-  *p = static_cast<T *>(q);
-  return GM_OK;
-}
-
-struct Prof {
-  gm_ctx *c; int cls; bool on; EventPair ev{};
-  Prof(gm_ctx *c_, int cls_) : c(c_), cls(cls_), on((c_->prof_mask >> cls_) & 1) {
-    if (!on) return;
-    size_t &u = c->events_used[cls];
-    if (u == c->events[cls].size()) {
-      EventPair e;
-      cudaEventCreate(&e.a);
-      cudaEventCreate(&e.b);
-      c->events[cls].push_back(e);
-    }
-    ev = c->events[cls][u++];
-    cudaEventRecord(ev.a, c->stream);
-  }
-  ~Prof() {
-    if (on) cudaEventRecord(ev.b, c->stream);
-    c->launches++;
-  }
-};
-#define GM_LAUNCH(ctx, cls, call)           \
-  do {                                      \
-    cudaError_t e__;                        \
-    { Prof p__(ctx, cls); e__ = (call); }   \
-    if (e__ != cudaSuccess) {               \
-      (ctx)->last_cuda = e__;               \
-      if (std::getenv("GM_DEBUG")) std::fprintf(stderr, "[gm] %s failed: %s\n", #call, cudaGetErrorString(e__)); \
-      return GM_ERR_CUDA;                   \
-    }                                       \
-  } while (0)
+namespace gmh {
 
 // 2-D bf16 tensor map: inner extent `cols` (contiguous), outer extent `rows`, box 64 x box_rows, 128-byte swizzle.
 int make_map(gm_ctx *c, CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
@@ -258,8 +126,6 @@ int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *w
   return GM_OK;
 }
 
-struct PhaseShape { int B, QT, M, qrows; };
-
 // One decoder layer on rows x/xn [M, d] (xn = normed input).  `next_norm` is the RMSNorm weight applied to
 // the layer's output for whatever consumes it next (null: none); `hidden_out` optionally receives the
 // bf16 residual stream.
@@ -367,49 +233,7 @@ int fill_sampler(gm_ctx *c, SamplerArgs &S, float temperature) {
   return GM_OK;
 }
 
-// ---- captured cycles (GM_FLAG_GRAPH) ----------------------------------------------------------------------------------
-struct KeyBytes {
-  std::vector<unsigned char> bytes;
-  template <typename T> void add(const T &v) {
-    const unsigned char *p = reinterpret_cast<const unsigned char *>(&v);
-    bytes.insert(bytes.end(), p, p + sizeof(T));
-  }
-};
-bool graph_capable(const gm_ctx *c) {
-  return (c->cfg.flags & GM_FLAG_GRAPH) && c->stream != nullptr && c->stream != cudaStreamLegacy &&
-         c->stream != cudaStreamPerThread;
-}
-// Makes `slot` hold a graph of the launches `body` issues (with the step index read from c->dev_step), re-capturing
-// when `key` differs from what the slot was captured for.  Nothing of `body` runs here.
-template <typename F>
-int graph_prepare(gm_ctx *c, gm_ctx::GraphSlot &slot, const std::vector<unsigned char> &key, F &&body) {
-  if (slot.exec && slot.key == key) return GM_OK;
-  if (slot.exec) { cudaGraphExecDestroy(slot.exec); slot.exec = nullptr; }
-  int rc;
-  if (!c->dev_step && (rc = dev_alloc(c, &c->dev_step, 1)) != GM_OK) return rc;
-  const int64_t before = c->launches;
-  GM_CUDA(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeRelaxed));
-  c->step_ptr = c->dev_step;
-  rc = body();
-  c->step_ptr = nullptr;
-  cudaGraph_t graph = nullptr;
-  const cudaError_t e = cudaStreamEndCapture(c->stream, &graph);         // always leave capture mode
-  const int64_t n = c->launches - before;
-  c->launches = before;                                                  // nothing has run yet
-  if (rc != GM_OK || e != cudaSuccess || !graph) {
-    if (graph) cudaGraphDestroy(graph);
-    if (e != cudaSuccess) { c->last_cuda = e; (void)cudaGetLastError(); }
-    return rc != GM_OK ? rc : GM_ERR_CUDA;
-  }
-  const cudaError_t ei = cudaGraphInstantiate(&slot.exec, graph, 0);
-  cudaGraphDestroy(graph);
-  if (ei != cudaSuccess) { c->last_cuda = ei; slot.exec = nullptr; return GM_ERR_CUDA; }
-  slot.launches = n;
-  slot.key = key;
-  return GM_OK;
-}
-
-}  // namespace
+}  // namespace gmh
 
 // ======================================================================================================================
 extern "C" {
@@ -565,17 +389,15 @@ void gm_destroy(gm_ctx *c) {
   delete c;
 }
 
-// forced: draft_tok holds recorded drafts that are fed back instead of sampled ones (Eq. 4); nothing is drawn
-static int draft_impl(gm_ctx *c, const gm_state *st, int k, float temperature, const uint32_t *u24_draft, uint64_t seed,
-                      uint64_t step, int32_t *draft_tok, void *draft_logits, float *dbg_q, bool forced);
-
 int gm_draft(gm_ctx *c, const gm_state *st, int k, float temperature, const uint32_t *u24_draft, uint64_t seed,
              uint64_t step, int32_t *draft_tok, void *draft_logits, float *dbg_q) {
   return draft_impl(c, st, k, temperature, u24_draft, seed, step, draft_tok, draft_logits, dbg_q, false);
 }
 
-static int draft_impl(gm_ctx *c, const gm_state *st, int k, float temperature, const uint32_t *u24_draft, uint64_t seed,
-                      uint64_t step, int32_t *draft_tok, void *draft_logits, float *dbg_q, bool forced) {
+}  // extern "C"
+
+int gmh::draft_impl(gm_ctx *c, const gm_state *st, int k, float temperature, const uint32_t *u24_draft, uint64_t seed,
+                    uint64_t step, int32_t *draft_tok, void *draft_logits, float *dbg_q, bool forced) {
   int rc = check_state(c, st, k);
   if (rc) return rc;
   if (!draft_tok || !draft_logits) return GM_ERR_INVALID_ARG;
@@ -625,6 +447,8 @@ static int draft_impl(gm_ctx *c, const gm_state *st, int k, float temperature, c
   return GM_OK;
 }
 
+extern "C" {
+
 int gm_verify(gm_ctx *c, const gm_state *st, int k, const int32_t *draft_tok, void *target_logits,
               void *target_hidden) {
   int rc = check_state(c, st, k);
@@ -650,88 +474,6 @@ int gm_verify(gm_ctx *c, const gm_state *st, int k, const int32_t *draft_tok, vo
   }
   return run_gemm(c, c->xn, c->Mmax, &c->lm_head_map, static_cast<const __nv_bfloat16 *>(c->w.lm_head), ph.M, c->V, c->d,
                   target_logits, EPI_STORE_BF16, c->V);
-}
-
-static int run_nucleus(gm_ctx *c, const void *logits, int rows, float temperature, float top_p, void *out, float *dbg_e);
-
-int gm_prefill(gm_ctx *c, gm_state *st, const int32_t *prompt_tok, const int32_t *prompt_len, int prompt_stride,
-               int max_prompt_len, float temperature, const uint32_t *u24_first, uint64_t seed, int32_t *first_token,
-               float *dbg_p) {
-  int rc = check_state(c, st, 1);
-  if (rc) return rc;
-  if (!prompt_tok || !prompt_len || max_prompt_len < 1 || prompt_stride < max_prompt_len) return GM_ERR_INVALID_ARG;
-  const gm_config &cf = c->cfg;
-  if (max_prompt_len + cf.max_k + 1 > cf.max_pages_per_seq * GM_PAGE) return GM_ERR_KV_CAPACITY;
-  SamplerArgs S;
-  if ((rc = fill_sampler(c, S, temperature)) != GM_OK) return rc;
-  const int B = st->batch, QT = cf.max_k + 1;
-  PhaseShape ph;
-  ph.B = B; ph.QT = QT; ph.M = B * QT; ph.qrows = round16(QT * c->group);
-  CUtensorMap kvm, hkvm;
-  if ((rc = kv_map(c, st->kv_pool, cf.n_layers, cf.num_pages, &kvm)) != GM_OK) return rc;
-  if ((rc = kv_map(c, st->head_kv_pool, 1, cf.head_num_pages, &hkvm)) != GM_OK) return rc;
-  for (int base = 0; base < max_prompt_len; base += QT) {
-    ChunkSetupArgs Cs;
-    Cs.prompt_tok = prompt_tok; Cs.prompt_len = prompt_len; Cs.batch = B; Cs.stride = prompt_stride; Cs.base = base;
-    Cs.QT = QT; Cs.max_len = max_prompt_len; Cs.pair_stride = QT; Cs.row_n = c->pf_row_n; Cs.head_n = c->pf_head_n;
-    Cs.pair_tok = c->pf_pair_tok; Cs.status = c->status;
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_chunk_setup(Cs, c->stream));
-    // the backbone over positions base .. base + QT - 1 of every prompt that reaches them
-    if ((rc = run_plan_chunk(c, B, c->pf_row_n, base, QT)) != GM_OK) return rc;
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-              launch_embed_chunk(static_cast<const __nv_bfloat16 *>(c->w.embed),
-                                 static_cast<const __nv_bfloat16 *>(c->layers[0].ln1), prompt_tok, prompt_stride, base,
-                                 c->pf_row_n, B, QT, c->d, c->V, cf.rms_eps, c->x, c->xn, c->status, c->stream));
-    for (int l = 0; l < cf.n_layers; ++l) {
-      const bool last = l + 1 == cf.n_layers;
-      rc = run_layer(c, c->layers[l], c->lmaps[l], ph, kvm, static_cast<__nv_bfloat16 *>(st->kv_pool), l, cf.num_pages,
-                     st->page_table, last ? nullptr : static_cast<const __nv_bfloat16 *>(c->layers[l + 1].ln1),
-                     last ? c->pf_hidden : nullptr);
-      if (rc) return rc;
-    }
-    if (c->capture)
-      GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-                launch_capture_chunk(c->pf_hidden, c->pf_row_n, B, QT, base, c->d, c->capture, c->capture_stride, c->stream));
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-              launch_prefill_last(c->x, c->pf_hidden, c->pf_row_n, prompt_len, B, base, QT, c->d, QT, c->pf_xlast,
-                                  static_cast<__nv_bfloat16 *>(st->pending_hidden), c->stream));
-    // the draft head over the pairs (hidden of position t, token t + 1) of the same chunk, at head positions t
-    if (base + 1 < max_prompt_len) {
-      if ((rc = run_plan_chunk(c, B, c->pf_head_n, base, QT)) != GM_OK) return rc;
-      HeadInputArgs H;
-      H.mode = PHASE_DRAFT_FIRST; H.batch = B; H.QT = QT; H.d = c->d; H.vocab = c->V; H.max_k = cf.max_k; H.k = 1; H.j = 1;
-      H.eps = cf.rms_eps; H.embed = static_cast<const __nv_bfloat16 *>(c->w.embed);
-      H.we = static_cast<const __nv_bfloat16 *>(c->w.head_enorm); H.wh = static_cast<const __nv_bfloat16 *>(c->w.head_hnorm);
-      H.pending_tok = c->pf_pair_tok; H.pending_n = c->pf_head_n; H.pending_hidden = c->pf_hidden; H.draft_tok = nullptr;
-      H.g_prev = c->g; H.zin = c->zin; H.status = c->status;
-      GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_head_input(H, c->stream));
-      rc = run_gemm(c, c->zin, c->Mmax, &c->head_proj_map, static_cast<const __nv_bfloat16 *>(c->w.head_proj), ph.M, c->d,
-                    2 * c->d, c->x, EPI_STORE_F32, c->d);
-      if (rc) return rc;
-      GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-                launch_rmsnorm(c->x, static_cast<const __nv_bfloat16 *>(c->w.head_layer.ln1), c->xn, nullptr, ph.M, c->d,
-                               cf.rms_eps, c->stream));
-      rc = run_layer(c, c->w.head_layer, c->head_maps, ph, hkvm, static_cast<__nv_bfloat16 *>(st->head_kv_pool), 0,
-                     cf.head_num_pages, st->head_page_table, nullptr, nullptr);
-      if (rc) return rc;
-    }
-  }
-  // first response token: final norm + LM head on the hidden state of each prompt's last token, one draw per sequence
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-            launch_rmsnorm(c->pf_xlast, static_cast<const __nv_bfloat16 *>(c->w.final_norm), c->xn, nullptr, B, c->d,
-                           cf.rms_eps, c->stream));
-  rc = run_gemm(c, c->xn, c->Mmax, &c->lm_head_map, static_cast<const __nv_bfloat16 *>(c->w.lm_head), B, c->V, c->d,
-                c->ws_target_logits, EPI_STORE_BF16, c->V);
-  if (rc) return rc;
-  S.K = 0; S.target_logits = c->ws_target_logits; S.tgt_bstride = c->V; S.draft_logits = nullptr;
-  S.u24 = u24_first; S.u_stride = 1; S.seed = seed; S.step = 0; S.slot_final = SLOT_FINAL;
-  S.accept_len = nullptr; S.next_token = c->pf_first; S.tok_out_stride = 1; S.dbg_p = dbg_p; S.dbg_q = nullptr; S.commit = 0;
-  GM_LAUNCH(c, GM_KC_SAMPLER, run_sampler(c, S, B));
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-            launch_prefill_finish(prompt_len, c->pf_first, B, QT, st->kv_len, st->pending_n, st->pending_tok, c->stream));
-  if (first_token)
-    GM_CUDA(c, cudaMemcpyAsync(first_token, c->pf_first, sizeof(int32_t) * B, cudaMemcpyDeviceToDevice, c->stream));
-  return GM_OK;
 }
 
 int gm_accept(gm_ctx *c, gm_state *st, int batch, int k, float temperature, const void *target_logits,
@@ -774,42 +516,6 @@ int gm_accept(gm_ctx *c, gm_state *st, int batch, int k, float temperature, cons
   return GM_OK;
 }
 
-int gm_capture_hidden(gm_ctx *c, void *seq_hidden, int stride) {
-  if (!c || (seq_hidden && stride < 1)) return GM_ERR_INVALID_ARG;
-  c->capture = static_cast<__nv_bfloat16 *>(seq_hidden);
-  c->capture_stride = seq_hidden ? stride : 0;
-  return GM_OK;
-}
-
-static int run_nucleus(gm_ctx *c, const void *logits, int rows, float temperature, float top_p, void *out, float *dbg_e) {
-  if (!(temperature > 0.f) || !std::isfinite(temperature) || !(top_p > 0.f) || !(top_p < 1.f)) return GM_ERR_UNSUPPORTED;
-  NucleusArgs N;
-  N.in = static_cast<const __nv_bfloat16 *>(logits); N.out = static_cast<__nv_bfloat16 *>(out); N.dbg_e = dbg_e;
-  N.rows = rows; N.V = c->V; N.inv_temp = 1.0f / temperature;
-  N.tp24 = static_cast<uint32_t>(std::nearbyint(static_cast<double>(top_p) * 16777216.0));
-  if (N.tp24 < 1u) N.tp24 = 1u;
-  if (N.tp24 > 16777215u) N.tp24 = 16777215u;
-  GM_LAUNCH(c, GM_KC_SAMPLER, launch_nucleus(N, c->stream));
-  return GM_OK;
-}
-
-int gm_nucleus(gm_ctx *c, const void *logits, int rows, float temperature, float top_p, void *out, float *dbg_weight) {
-  if (!c || !logits || !out || rows < 1 || logits == out) return GM_ERR_INVALID_ARG;
-  return run_nucleus(c, logits, rows, temperature, top_p, out, dbg_weight);
-}
-
-int gm_set_top_p(gm_ctx *c, float top_p) {
-  if (!c) return GM_ERR_INVALID_ARG;
-  if (!(top_p > 0.f) || !(top_p <= 1.f)) return GM_ERR_UNSUPPORTED;
-  if (top_p < 1.f && !c->ws_nucleus) {
-    const size_t n = static_cast<size_t>(c->cfg.max_batch) * (c->cfg.max_k + 1) * c->V;
-    int rc = dev_alloc(c, &c->ws_nucleus, n, false);
-    if (rc) return rc;
-  }
-  c->top_p = top_p;
-  return GM_OK;
-}
-
 int gm_draw(gm_ctx *c, const void *logits, int rows, float temperature, const uint32_t *u24, int32_t *out_tok,
             float *dbg_prob) {
   if (!c || !logits || !u24 || !out_tok || rows < 1) return GM_ERR_INVALID_ARG;
@@ -821,10 +527,6 @@ int gm_draw(gm_ctx *c, const void *logits, int rows, float temperature, const ui
   GM_LAUNCH(c, GM_KC_SAMPLER, run_sampler(c, S, rows));
   return GM_OK;
 }
-
-static int spec_step_impl(gm_ctx *c, gm_state *st, int k, float temperature, const uint32_t *u24_draft,
-                          const uint32_t *u24_accept, uint64_t seed, uint64_t step, int32_t *accept_len,
-                          int32_t *next_token, int32_t *draft_tok);
 
 // One cycle, host-launched or (GM_FLAG_GRAPH on a capturable stream) as a replay of the captured cycle.
 static int spec_step_run(gm_ctx *c, gm_state *st, int k, float temperature, const uint32_t *u24_draft,
@@ -849,9 +551,11 @@ static int spec_step_run(gm_ctx *c, gm_state *st, int k, float temperature, cons
   return GM_OK;
 }
 
-static int spec_step_impl(gm_ctx *c, gm_state *st, int k, float temperature, const uint32_t *u24_draft,
-                          const uint32_t *u24_accept, uint64_t seed, uint64_t step, int32_t *accept_len,
-                          int32_t *next_token, int32_t *draft_tok) {
+}  // extern "C"
+
+int gmh::spec_step_impl(gm_ctx *c, gm_state *st, int k, float temperature, const uint32_t *u24_draft,
+                        const uint32_t *u24_accept, uint64_t seed, uint64_t step, int32_t *accept_len,
+                        int32_t *next_token, int32_t *draft_tok) {
   int rc = check_state(c, st, k);
   if (rc) return rc;
   if (!accept_len || !next_token) return GM_ERR_INVALID_ARG;
@@ -861,6 +565,8 @@ static int spec_step_impl(gm_ctx *c, gm_state *st, int k, float temperature, con
   return gm_accept(c, st, st->batch, k, temperature, c->ws_target_logits, c->ws_draft_logits, dt, u24_accept, seed, step,
                    accept_len, next_token, nullptr, nullptr, c->ws_target_hidden, 1);
 }
+
+extern "C" {
 
 int gm_spec_step(gm_ctx *c, gm_state *st, int k, float temperature, uint64_t seed, uint64_t step, int32_t *accept_len,
                  int32_t *next_token, int32_t *draft_tok) {
@@ -889,336 +595,6 @@ int gm_spec_step_host(gm_ctx *c, gm_state *st, int k, float temperature, uint64_
   if (draft_tok_host)
     GM_CUDA(c, cudaMemcpyAsync(draft_tok_host, c->ws_draft_tok, B * k * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
   GM_CUDA(c, cudaStreamSynchronize(c->stream));
-  return GM_OK;
-}
-
-int gm_record_begin(gm_ctx *c, const gm_state *st, gm_record *rec) {
-  if (!c || !st || !rec || !rec->start_hidden || !rec->start_pos) return GM_ERR_INVALID_ARG;
-  if (st->batch < 1 || st->batch > c->cfg.max_batch || !st->kv_len || !st->pending_n || !st->pending_hidden)
-    return GM_ERR_INVALID_ARG;
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-            launch_record_begin(st->kv_len, st->pending_n, static_cast<const __nv_bfloat16 *>(st->pending_hidden), st->batch,
-                                c->cfg.max_k, c->d, static_cast<__nv_bfloat16 *>(rec->start_hidden), rec->start_pos,
-                                c->stream));
-  return GM_OK;
-}
-
-int gm_record_end(gm_ctx *c, int batch, int k, float temperature, const void *target_logits, const int32_t *draft_tok,
-                  const int32_t *accept_len, gm_record *rec) {
-  if (!c || !rec || !target_logits || !draft_tok || !accept_len || !rec->drafts || !rec->top_logprob || !rec->top_index ||
-      !rec->accepted)
-    return GM_ERR_INVALID_ARG;
-  if (batch < 1 || k < 1) return GM_ERR_INVALID_ARG;
-  if (k > GM_MAX_K || !(temperature > 0.f) || !std::isfinite(temperature)) return GM_ERR_UNSUPPORTED;
-  RecordTopkArgs R;
-  R.target_logits = static_cast<const __nv_bfloat16 *>(target_logits); R.bstride = static_cast<size_t>(k + 1) * c->V;
-  R.K = k; R.V = c->V; R.inv_temp = 1.0f / temperature; R.top_logprob = static_cast<__nv_bfloat16 *>(rec->top_logprob);
-  R.top_index = rec->top_index; R.status = c->status;
-  GM_LAUNCH(c, GM_KC_RECORD, launch_record_topk(R, batch, c->stream));
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_record_end(draft_tok, accept_len, batch, k, rec->drafts, rec->accepted, c->stream));
-  return GM_OK;
-}
-
-int gm_spec_step_rec(gm_ctx *c, gm_state *st, int k, float temperature, uint64_t seed, uint64_t step, int32_t *accept_len,
-                     int32_t *next_token, int32_t *draft_tok, gm_record *rec) {
-  int rc = check_state(c, st, k);
-  if (rc) return rc;
-  if (!accept_len || !next_token || !rec) return GM_ERR_INVALID_ARG;
-  if ((rc = gm_record_begin(c, st, rec)) != GM_OK) return rc;
-  int32_t *dt = draft_tok ? draft_tok : c->ws_draft_tok;
-  if ((rc = spec_step_impl(c, st, k, temperature, nullptr, nullptr, seed, step, accept_len, next_token, dt)) != GM_OK) return rc;
-  return gm_record_end(c, st->batch, k, temperature, c->ws_target_logits, dt, accept_len, rec);
-}
-
-int gm_gemm(gm_ctx *c, const void *x, const void *w, void *out, int M, int N, int K, int out_fp32) {
-  if (!c || !x || !w || !out || M < 1 || N < 1 || K < 1) return GM_ERR_INVALID_ARG;
-  if ((K % 64) || (N % 8)) return GM_ERR_UNSUPPORTED;
-  CUtensorMap wm;
-  std::memset(&wm, 0, sizeof(wm));
-  if (!(c->cfg.flags & GM_FLAG_SIMPLE_GEMM)) {
-    auto key = std::make_tuple(w, N, K);
-    auto it = c->w_maps.find(key);
-    if (it == c->w_maps.end()) {
-      CUtensorMap m;
-      if (make_map(c, &m, w, N, K, 128) != GM_OK) return GM_ERR_CUDA;
-      it = c->w_maps.emplace(key, m).first;
-    }
-    wm = it->second;
-  }
-  return run_gemm(c, static_cast<const __nv_bfloat16 *>(x), M, &wm, static_cast<const __nv_bfloat16 *>(w), M, N, K, out,
-                  out_fp32 ? EPI_STORE_F32 : EPI_STORE_BF16, N);
-}
-
-int gm_attention(gm_ctx *c, const void *q, const void *kv_pool, int pool_layers, int num_pages, int layer,
-                 const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch, int q_stride,
-                 void *out) {
-  if (!c || !q || !kv_pool || !page_table || !q_count || !q_base || !out) return GM_ERR_INVALID_ARG;
-  if (batch < 1 || batch > c->cfg.max_batch || q_stride < 1 || pool_layers < 1 || layer < 0 || layer >= pool_layers ||
-      num_pages < 1)
-    return GM_ERR_INVALID_ARG;
-  if (q_stride > c->cfg.max_k + 1) return GM_ERR_UNSUPPORTED;
-  const gm_config &cf = c->cfg;
-  CUtensorMap kvm;
-  int rc = kv_map(c, kv_pool, pool_layers, num_pages, &kvm);
-  if (rc) return rc;
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-            launch_page_prefix(q_count, q_base, batch, cf.max_pages_per_seq, q_stride, c->page_start, c->status, c->stream));
-  const int qrows = round16(q_stride * c->group);
-  AttnArgs T;
-  T.kv_map = kvm; T.qbuf = static_cast<const __nv_bfloat16 *>(q); T.qn = q_count; T.qbase = q_base;
-  T.page_start = c->page_start; T.page_table = page_table; T.batch = batch; T.n_kv = cf.n_kv_heads; T.group = c->group;
-  T.hd = cf.head_dim; T.qrows = qrows; T.layer = layer; T.num_pages = num_pages; T.max_pages_per_seq = cf.max_pages_per_seq;
-  T.n_ctas = c->sm_count; T.scale_log2e = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(cf.head_dim)));
-  T.part_o = c->part_o; T.part_ml = c->part_ml; T.status = c->status; T.rows_used = q_stride * c->group;
-  GM_LAUNCH(c, GM_KC_ATTENTION, launch_attention(T, c->stream));
-  AttnCombineArgs Cb;
-  Cb.part_o = c->part_o; Cb.part_ml = c->part_ml; Cb.qn = q_count; Cb.page_start = c->page_start; Cb.batch = batch;
-  Cb.n_kv = cf.n_kv_heads; Cb.group = c->group; Cb.hd = cf.head_dim; Cb.qrows = qrows; Cb.QT = q_stride;
-  Cb.n_ctas = c->sm_count; Cb.out = static_cast<__nv_bfloat16 *>(out);
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_attention_combine(Cb, c->stream));
-  return GM_OK;
-}
-
-// ---- forward pass of the head update on recorded cycles -------------------------------------------------------------
-int gm_head_prefill(gm_ctx *c, gm_state *st, const void *seq_hidden, int hid_stride, const int32_t *seq_tok,
-                    int tok_stride, const int32_t *seq_len, int max_len) {
-  int rc = check_state(c, st, 1);
-  if (rc) return rc;
-  if (!seq_hidden || !seq_tok || !seq_len || max_len < 1 || tok_stride < max_len || hid_stride < max_len - 1)
-    return GM_ERR_INVALID_ARG;
-  const gm_config &cf = c->cfg;
-  if (max_len + cf.max_k + 1 > cf.max_pages_per_seq * GM_PAGE) return GM_ERR_KV_CAPACITY;
-  const int B = st->batch, QT = cf.max_k + 1;
-  PhaseShape ph;
-  ph.B = B; ph.QT = QT; ph.M = B * QT; ph.qrows = round16(QT * c->group);
-  CUtensorMap hkvm;
-  if ((rc = kv_map(c, st->head_kv_pool, 1, cf.head_num_pages, &hkvm)) != GM_OK) return rc;
-  for (int base = 0; base + 1 < max_len; base += QT) {
-    ChunkSetupArgs Cs;
-    Cs.prompt_tok = seq_tok; Cs.prompt_len = seq_len; Cs.batch = B; Cs.stride = tok_stride; Cs.base = base; Cs.QT = QT;
-    Cs.max_len = max_len; Cs.pair_stride = QT; Cs.row_n = c->pf_row_n; Cs.head_n = c->pf_head_n;
-    Cs.pair_tok = c->pf_pair_tok; Cs.status = c->status;
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_chunk_setup(Cs, c->stream));
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-              launch_gather_chunk_hidden(static_cast<const __nv_bfloat16 *>(seq_hidden), hid_stride, base, B, QT, c->d,
-                                         c->pf_head_n, c->pf_hidden, c->stream));
-    if ((rc = run_plan_chunk(c, B, c->pf_head_n, base, QT)) != GM_OK) return rc;
-    HeadInputArgs H;
-    H.mode = PHASE_DRAFT_FIRST; H.batch = B; H.QT = QT; H.d = c->d; H.vocab = c->V; H.max_k = cf.max_k; H.k = 1; H.j = 1;
-    H.eps = cf.rms_eps; H.embed = static_cast<const __nv_bfloat16 *>(c->w.embed);
-    H.we = static_cast<const __nv_bfloat16 *>(c->w.head_enorm); H.wh = static_cast<const __nv_bfloat16 *>(c->w.head_hnorm);
-    H.pending_tok = c->pf_pair_tok; H.pending_n = c->pf_head_n; H.pending_hidden = c->pf_hidden; H.draft_tok = nullptr;
-    H.g_prev = c->g; H.zin = c->zin; H.status = c->status;
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_head_input(H, c->stream));
-    rc = run_gemm(c, c->zin, c->Mmax, &c->head_proj_map, static_cast<const __nv_bfloat16 *>(c->w.head_proj), ph.M, c->d,
-                  2 * c->d, c->x, EPI_STORE_F32, c->d);
-    if (rc) return rc;
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-              launch_rmsnorm(c->x, static_cast<const __nv_bfloat16 *>(c->w.head_layer.ln1), c->xn, nullptr, ph.M, c->d,
-                             cf.rms_eps, c->stream));
-    rc = run_layer(c, c->w.head_layer, c->head_maps, ph, hkvm, static_cast<__nv_bfloat16 *>(st->head_kv_pool), 0,
-                   cf.head_num_pages, st->head_page_table, nullptr, nullptr);
-    if (rc) return rc;
-  }
-  return GM_OK;
-}
-
-int gm_reconstruct(gm_ctx *c, gm_state *st, int n_cycles, int k, const int32_t *cycle_seq, const gm_record *rec,
-                   const int32_t *seq_tok, int tok_stride, const int32_t *scratch_pages, void *draft_logits) {
-  int rc = check_state(c, st, k);
-  if (rc) return rc;
-  if (n_cycles < 1 || !cycle_seq || !rec || !rec->start_hidden || !rec->start_pos || !rec->drafts || !seq_tok ||
-      tok_stride < 2 || !scratch_pages || !draft_logits)
-    return GM_ERR_INVALID_ARG;
-  const gm_config &cf = c->cfg;
-  const int MB = cf.max_batch, PS = cf.max_k + 1;
-  if (!c->v_table) {
-    if ((rc = dev_alloc(c, &c->v_kv_len, MB)) != GM_OK) return rc;
-    if ((rc = dev_alloc(c, &c->v_pending_n, MB)) != GM_OK) return rc;
-    if ((rc = dev_alloc(c, &c->v_pending_tok, static_cast<size_t>(MB) * PS)) != GM_OK) return rc;
-    if ((rc = dev_alloc(c, &c->v_pending_hidden, static_cast<size_t>(MB) * PS * c->d)) != GM_OK) return rc;
-    if ((rc = dev_alloc(c, &c->v_table, static_cast<size_t>(MB) * cf.max_pages_per_seq)) != GM_OK) return rc;
-  }
-  for (int off = 0; off < n_cycles; off += MB) {
-    const int m = std::min(MB, n_cycles - off);
-    ChainSetupArgs A;
-    A.cycle_seq = cycle_seq + off; A.start_pos = rec->start_pos + off;
-    A.start_hidden = static_cast<const __nv_bfloat16 *>(rec->start_hidden) + static_cast<size_t>(off) * c->d;
-    A.seq_tok = seq_tok; A.scratch_pages = scratch_pages + 2 * static_cast<size_t>(off);
-    A.head_page_table = st->head_page_table; A.pool = static_cast<__nv_bfloat16 *>(st->head_kv_pool);
-    A.n_seq = st->batch; A.tok_stride = tok_stride; A.k = k; A.d = c->d; A.vocab = c->V;
-    A.max_pages_per_seq = cf.max_pages_per_seq; A.num_pages = cf.head_num_pages;
-    A.page_elems = cf.n_kv_heads * GM_PAGE * cf.head_dim; A.pend_stride = PS;
-    A.v_kv_len = c->v_kv_len; A.v_pending_n = c->v_pending_n; A.v_pending_tok = c->v_pending_tok; A.v_table = c->v_table;
-    A.v_pending_hidden = c->v_pending_hidden; A.status = c->status;
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_chain_setup(A, m, c->stream));
-    gm_state vs = *st;
-    vs.batch = m; vs.kv_len = c->v_kv_len; vs.head_page_table = c->v_table; vs.pending_n = c->v_pending_n;
-    vs.pending_tok = c->v_pending_tok; vs.pending_hidden = c->v_pending_hidden;
-    rc = draft_impl(c, &vs, k, 1.0f, nullptr, 0, 0, rec->drafts + static_cast<size_t>(off) * k,
-                    static_cast<__nv_bfloat16 *>(draft_logits) + static_cast<size_t>(off) * k * c->V, nullptr, true);
-    if (rc) return rc;
-  }
-  return GM_OK;
-}
-
-int gm_overlap(gm_ctx *c, int n_cycles, int k, float temperature, const void *draft_logits, const gm_record *rec,
-               float *alpha) {
-  if (!c || n_cycles < 1 || k < 1 || k > GM_MAX_K || !draft_logits || !rec || !rec->top_index || !rec->top_logprob || !alpha)
-    return GM_ERR_INVALID_ARG;
-  if (!(temperature > 0.f) || !std::isfinite(temperature)) return GM_ERR_UNSUPPORTED;
-  OverlapArgs A;
-  A.logits = static_cast<const __nv_bfloat16 *>(draft_logits); A.top_index = rec->top_index;
-  A.top_logprob = static_cast<const __nv_bfloat16 *>(rec->top_logprob); A.alpha = alpha; A.V = c->V;
-  A.inv_temp = 1.0f / temperature;
-  GM_LAUNCH(c, GM_KC_RECORD, launch_overlap(A, n_cycles * k, c->stream));
-  return GM_OK;
-}
-
-int gm_dca_loss(gm_ctx *c, int n_cycles, int k, const float *alpha, const int32_t *accepted, float *loss, float *mean) {
-  if (!c || n_cycles < 1 || k < 1 || k > GM_MAX_K || !alpha || !accepted || !loss || !mean) return GM_ERR_INVALID_ARG;
-  GM_LAUNCH(c, GM_KC_RECORD, launch_dca_loss(alpha, accepted, n_cycles, k, loss, mean, c->stream));
-  return GM_OK;
-}
-
-// ---- rollout driver and page allocator ------------------------------------------------------------------------------
-static int rollout_args_ok(const gm_ctx *c, const gm_state *st, const gm_rollout *ro) {
-  if (!c || !st || !ro || !ro->out_tok || !ro->out_len || !ro->finished || !ro->n_running) return GM_ERR_INVALID_ARG;
-  if (ro->max_new < 1 || ro->out_stride < ro->max_new) return GM_ERR_INVALID_ARG;
-  if (st->batch < 1 || st->batch > c->cfg.max_batch) return GM_ERR_INVALID_ARG;
-  return GM_OK;
-}
-
-static void fill_alloc(gm_ctx *c, gm_state *st, int pool, PageAllocArgs &P) {
-  P.batch = st->batch; P.max_pages_per_seq = c->cfg.max_pages_per_seq;
-  P.num_pages = pool ? c->cfg.head_num_pages : c->cfg.num_pages; P.extra = 0;
-  P.length = nullptr; P.finished = nullptr;
-  P.page_table = pool ? st->head_page_table : st->page_table;
-  P.held = c->held[pool]; P.free_list = c->free_list[pool]; P.free_top = c->free_top[pool]; P.status = c->status;
-}
-
-int gm_pages_reset(gm_ctx *c, gm_state *st) {
-  if (!c || !st || !st->page_table || !st->head_page_table || st->batch < 1 || st->batch > c->cfg.max_batch)
-    return GM_ERR_INVALID_ARG;
-  for (int pool = 0; pool < 2; ++pool) {
-    if (!c->free_list[pool]) {
-      int rc;
-      if ((rc = dev_alloc(c, &c->free_list[pool], pool ? c->cfg.head_num_pages : c->cfg.num_pages, false)) != GM_OK) return rc;
-      if ((rc = dev_alloc(c, &c->free_top[pool], 1)) != GM_OK) return rc;
-      if ((rc = dev_alloc(c, &c->held[pool], c->cfg.max_batch)) != GM_OK) return rc;
-    }
-    PageAllocArgs P;
-    fill_alloc(c, st, pool, P);
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_page_reset(P, c->stream));
-  }
-  c->alloc_on = true;
-  return GM_OK;
-}
-
-int gm_pages_reserve(gm_ctx *c, gm_state *st, const int32_t *length, int extra, const int32_t *finished) {
-  if (!c || !st || extra < 0) return GM_ERR_INVALID_ARG;
-  if (!c->alloc_on) return GM_ERR_INVALID_ARG;
-  for (int pool = 0; pool < 2; ++pool) {
-    PageAllocArgs P;
-    fill_alloc(c, st, pool, P);
-    P.length = length ? length : st->kv_len; P.extra = extra; P.finished = finished;
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_page_reserve(P, c->stream));
-  }
-  return GM_OK;
-}
-
-int gm_pages_release(gm_ctx *c, gm_state *st, const int32_t *finished) {
-  if (!c || !st || !finished) return GM_ERR_INVALID_ARG;
-  if (!c->alloc_on) return GM_ERR_INVALID_ARG;
-  for (int pool = 0; pool < 2; ++pool) {
-    PageAllocArgs P;
-    fill_alloc(c, st, pool, P);
-    P.finished = finished;
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_page_release(P, c->stream));
-  }
-  return GM_OK;
-}
-
-int gm_pages_free_count(gm_ctx *c, int32_t *target_free, int32_t *head_free) {
-  if (!c || !c->alloc_on) return GM_ERR_INVALID_ARG;
-  int32_t v[2] = {0, 0};
-  for (int pool = 0; pool < 2; ++pool)
-    GM_CUDA(c, cudaMemcpyAsync(&v[pool], c->free_top[pool], sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
-  GM_CUDA(c, cudaStreamSynchronize(c->stream));
-  if (target_free) *target_free = v[0];
-  if (head_free) *head_free = v[1];
-  return GM_OK;
-}
-
-static void fill_rollout(const gm_ctx *c, const gm_state *st, const gm_rollout *ro, int k, RolloutArgs &R) {
-  R.batch = st->batch; R.k = k; R.out_stride = ro->out_stride; R.eos_token = ro->eos_token; R.max_new = ro->max_new;
-  R.pend_stride = c->cfg.max_k + 1; R.draft_tok = c->ws_draft_tok; R.accept_len = c->ro_accept; R.next_token = c->ro_next;
-  R.pending_tok = st->pending_tok; R.out_tok = ro->out_tok; R.out_len = ro->out_len; R.finished = ro->finished;
-  R.n_running = ro->n_running; R.step_counter = c->step_ptr;
-}
-
-int gm_rollout_begin(gm_ctx *c, const gm_state *st, const gm_rollout *ro) {
-  int rc = rollout_args_ok(c, st, ro);
-  if (rc) return rc;
-  if (!st->pending_tok) return GM_ERR_INVALID_ARG;
-  RolloutArgs R;
-  fill_rollout(c, st, ro, 1, R);
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rollout_append(R, true, c->stream));
-  return GM_OK;
-}
-
-int gm_rollout_step(gm_ctx *c, gm_state *st, const gm_rollout *ro, int k, float temperature, uint64_t seed, uint64_t step) {
-  int rc = rollout_args_ok(c, st, ro);
-  if (rc) return rc;
-  if ((rc = check_state(c, st, k)) != GM_OK) return rc;
-  if (c->alloc_on && (rc = gm_pages_reserve(c, st, nullptr, k + 1, ro->finished)) != GM_OK) return rc;
-  c->finished_mask = ro->finished;
-  rc = spec_step_impl(c, st, k, temperature, nullptr, nullptr, seed, step, c->ro_accept, c->ro_next, c->ws_draft_tok);
-  c->finished_mask = nullptr;
-  if (rc) return rc;
-  RolloutArgs R;
-  fill_rollout(c, st, ro, k, R);
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rollout_append(R, false, c->stream));
-  if (c->alloc_on && (rc = gm_pages_release(c, st, ro->finished)) != GM_OK) return rc;
-  return GM_OK;
-}
-
-int gm_rollout_run(gm_ctx *c, gm_state *st, const gm_rollout *ro, int k, float temperature, uint64_t seed,
-                   uint64_t first_step, int max_steps, int check_every, int32_t *steps_run, int32_t *rows_running) {
-  if (max_steps < 0 || check_every < 1) return GM_ERR_INVALID_ARG;
-  int rc = rollout_args_ok(c, st, ro);
-  if (rc) return rc;
-  int done = 0;
-  int32_t running = st->batch;
-  auto poll = [&]() -> int {
-    GM_CUDA(c, cudaMemcpyAsync(&running, ro->n_running, sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
-    GM_CUDA(c, cudaStreamSynchronize(c->stream));
-    return GM_OK;
-  };
-  if ((rc = poll()) != GM_OK) return rc;
-  const bool use_graph = graph_capable(c);
-  if (use_graph && running > 0 && max_steps > 0) {
-    KeyBytes key;
-    key.add(*st); key.add(*ro); key.add(k); key.add(temperature); key.add(seed); key.add(c->alloc_on); key.add(c->top_p);
-    key.add(c->capture); key.add(c->capture_stride);
-    if ((rc = check_state(c, st, k)) != GM_OK) return rc;
-    rc = graph_prepare(c, c->graph_rollout, key.bytes, [&]() { return gm_rollout_step(c, st, ro, k, temperature, seed, 0); });
-    if (rc) return rc;
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_set_step(c->dev_step, first_step, c->stream));
-  }
-  while (done < max_steps && running > 0) {
-    if (use_graph) {
-      GM_CUDA(c, cudaGraphLaunch(c->graph_rollout.exec, c->stream));
-      c->launches += c->graph_rollout.launches;
-    } else if ((rc = gm_rollout_step(c, st, ro, k, temperature, seed, first_step + done)) != GM_OK) {
-      return rc;
-    }
-    ++done;
-    if (done % check_every == 0 || done == max_steps)
-      if ((rc = poll()) != GM_OK) return rc;
-  }
-  if (steps_run) *steps_run = done;
-  if (rows_running) *rows_running = running;
   return GM_OK;
 }
 

@@ -1,0 +1,211 @@
+// Internals of libgm shared by its host-side translation units: the context, error / launch macros, and the helpers
+// that issue the launch sequences.  Not part of the C ABI.
+#pragma once
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <new>
+#include <tuple>
+#include <vector>
+
+#include <cudaTypedefs.h>
+
+#include "../../include/gm.h"
+#include "common.cuh"
+#include "kernels.h"
+
+using namespace gm;
+
+
+namespace gmh {
+
+struct LayerMaps { CUtensorMap wqkv, wo, wgu, wdown; };
+
+struct EventPair { cudaEvent_t a, b; };
+
+}  // namespace gmh
+using namespace gmh;
+
+struct gm_ctx {
+  gm_config cfg;
+  gm_weights w;
+  std::vector<gm_layer_weights> layers;
+  cudaStream_t stream = nullptr;
+  int sm_count = 148;
+  PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+
+  // derived shapes
+  int d, q_dim, kv_dim, n_qkv, F, V, group, Mmax;
+
+  // tensor maps
+  std::vector<LayerMaps> lmaps;
+  LayerMaps head_maps;
+  CUtensorMap lm_head_map, head_proj_map;
+  std::map<std::tuple<const void *, int, int, int>, CUtensorMap> x_maps;   // (ptr, rows, K, box rows)
+  std::map<std::tuple<const void *, int, int>, CUtensorMap> w_maps;        // (ptr, N, K)   (gm_gemm only)
+  std::map<std::tuple<const void *, long long>, CUtensorMap> kv_maps;      // (pool, rows)
+
+  // workspaces (device)
+  float *x = nullptr, *g = nullptr, *part_o = nullptr, *part_ml = nullptr;
+  __nv_bfloat16 *xn = nullptr, *zin = nullptr, *qkv = nullptr, *qbuf = nullptr, *attn_out = nullptr, *act = nullptr, *gn = nullptr;
+  int max_clusters[17][9];            // resident clusters of the GEMM kernel by (block_t / 16, cluster size); -1 = not asked yet
+  __nv_bfloat16 *ws_draft_logits = nullptr, *ws_target_logits = nullptr, *ws_target_hidden = nullptr;
+  int32_t *ws_draft_tok = nullptr, *ws_accept_len = nullptr, *ws_next_token = nullptr;
+  uint32_t *ws_u24 = nullptr;
+  int32_t *qn = nullptr, *qbase = nullptr, *page_start = nullptr;
+  float2 *rope = nullptr;
+  uint32_t *status = nullptr;
+  // prompt prefill: per-chunk bookkeeping, the chunk's hidden states, the row of each prompt's last token
+  int32_t *pf_row_n = nullptr, *pf_head_n = nullptr, *pf_pair_tok = nullptr, *pf_first = nullptr;
+  __nv_bfloat16 *pf_hidden = nullptr;
+  float *pf_xlast = nullptr;
+  int32_t *ro_accept = nullptr, *ro_next = nullptr;   // per-step outputs of a rollout step
+  // captured rollout cycle (GM_FLAG_ROLLOUT_GRAPH)
+  uint64_t *dev_step = nullptr;             // step index of the captured cycle
+  uint64_t *step_ptr = nullptr;             // non-null while a cycle is being captured: kernels read the step from here
+  struct GraphSlot {                        // one captured sequence of launches and what it was captured for
+    cudaGraphExec_t exec = nullptr;
+    int64_t launches = 0;
+    std::vector<unsigned char> key;
+  } graph_rollout, graph_step;
+  const int32_t *finished_mask = nullptr;   // set around the phases of a rollout step: rows that sit out
+  // page allocator (gm_pages_*): one stack of free page ids per pool
+  bool alloc_on = false;
+  int32_t *free_list[2] = {nullptr, nullptr}, *free_top[2] = {nullptr, nullptr}, *held[2] = {nullptr, nullptr};
+  // chains of a reconstruction: virtual sequences (allocated on first use)
+  int32_t *v_kv_len = nullptr, *v_pending_n = nullptr, *v_pending_tok = nullptr, *v_table = nullptr;
+  __nv_bfloat16 *v_pending_hidden = nullptr;
+  __nv_bfloat16 *capture = nullptr;         // gm_capture_hidden: [max_batch, capture_stride, d] or null
+  int capture_stride = 0;
+  float top_p = 1.f;                    // nucleus of the target distributions (1 = none)
+  __nv_bfloat16 *ws_nucleus = nullptr;  // [max_batch (max_k + 1)][V] filtered target rows, allocated by gm_set_top_p
+  std::vector<void *> allocs;
+
+  // profiling
+  int prof_mask = 0;
+  std::vector<EventPair> events[GM_KC_COUNT];
+  size_t events_used[GM_KC_COUNT] = {};
+  int64_t launches = 0;
+  cudaError_t last_cuda = cudaSuccess;
+};
+
+namespace gmh {
+
+#define GM_CUDA(ctx, call)                                   \
+  do {                                                       \
+    cudaError_t e__ = (call);                                \
+    if (e__ != cudaSuccess) { (ctx)->last_cuda = e__; return GM_ERR_CUDA; } \
+  } while (0)
+
+template <typename T>
+int dev_alloc(gm_ctx *c, T **p, size_t n, bool zero = true) {
+  void *q = nullptr;
+  GM_CUDA(c, cudaMalloc(&q, n * sizeof(T) > 0 ? n * sizeof(T) : 16));
+  c->allocs.push_back(q);
+  if (zero) GM_CUDA(c, cudaMemsetAsync(q, 0, n * sizeof(T), c->stream));
+  *p = static_cast<T *>(q);
+  return GM_OK;
+}
+
+struct Prof {
+  gm_ctx *c; int cls; bool on; EventPair ev{};
+  Prof(gm_ctx *c_, int cls_) : c(c_), cls(cls_), on((c_->prof_mask >> cls_) & 1) {
+    if (!on) return;
+    size_t &u = c->events_used[cls];
+    if (u == c->events[cls].size()) {
+      EventPair e;
+      cudaEventCreate(&e.a);
+      cudaEventCreate(&e.b);
+      c->events[cls].push_back(e);
+    }
+    ev = c->events[cls][u++];
+    cudaEventRecord(ev.a, c->stream);
+  }
+  ~Prof() {
+    if (on) cudaEventRecord(ev.b, c->stream);
+    c->launches++;
+  }
+};
+#define GM_LAUNCH(ctx, cls, call)           \
+  do {                                      \
+    cudaError_t e__;                        \
+    { Prof p__(ctx, cls); e__ = (call); }   \
+    if (e__ != cudaSuccess) {               \
+      (ctx)->last_cuda = e__;               \
+      if (std::getenv("GM_DEBUG")) std::fprintf(stderr, "[gm] %s failed: %s\n", #call, cudaGetErrorString(e__)); \
+      return GM_ERR_CUDA;                   \
+    }                                       \
+  } while (0)
+
+
+// ---- host helpers shared by the api_*.cu files (defined in gm_api.cu) -------------------------------------------------
+int make_map(gm_ctx *c, CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t cols, uint32_t box_rows);
+int x_map(gm_ctx *c, const void *ptr, int rows, int K, int box_rows, CUtensorMap *out);
+int kv_map(gm_ctx *c, const void *pool, int layers, int num_pages, CUtensorMap *out);
+int round16(int v);
+int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *wmap, const __nv_bfloat16 *w, int M,
+             int N, int K, void *out, int epi, size_t ldo);
+struct PhaseShape { int B, QT, M, qrows; };
+int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const PhaseShape &ph, const CUtensorMap &kvm,
+              __nv_bfloat16 *pool, int layer, int num_pages, const int32_t *page_table,
+              const __nv_bfloat16 *next_norm, __nv_bfloat16 *hidden_out);
+int run_plan(gm_ctx *c, const gm_state *st, int mode, int k_or_j);
+int run_plan_chunk(gm_ctx *c, int batch, const int32_t *row_n, int base, int QT);
+int check_state(const gm_ctx *c, const gm_state *st, int k);
+cudaError_t run_sampler(gm_ctx *c, const SamplerArgs &S, int batch);
+int fill_sampler(gm_ctx *c, SamplerArgs &S, float temperature);
+// forced: draft_tok holds recorded drafts that are fed back instead of sampled ones (Eq. 4); nothing is drawn
+int draft_impl(gm_ctx *c, const gm_state *st, int k, float temperature, const uint32_t *u24_draft, uint64_t seed,
+               uint64_t step, int32_t *draft_tok, void *draft_logits, float *dbg_q, bool forced);
+int spec_step_impl(gm_ctx *c, gm_state *st, int k, float temperature, const uint32_t *u24_draft,
+                   const uint32_t *u24_accept, uint64_t seed, uint64_t step, int32_t *accept_len,
+                   int32_t *next_token, int32_t *draft_tok);
+int run_nucleus(gm_ctx *c, const void *logits, int rows, float temperature, float top_p, void *out, float *dbg_e);
+
+// ---- captured cycles (GM_FLAG_GRAPH) ----------------------------------------------------------------------------------
+struct KeyBytes {
+  std::vector<unsigned char> bytes;
+  template <typename T> void add(const T &v) {
+    const unsigned char *p = reinterpret_cast<const unsigned char *>(&v);
+    bytes.insert(bytes.end(), p, p + sizeof(T));
+  }
+};
+inline bool graph_capable(const gm_ctx *c) {
+  return (c->cfg.flags & GM_FLAG_GRAPH) && c->stream != nullptr && c->stream != cudaStreamLegacy &&
+         c->stream != cudaStreamPerThread;
+}
+// Makes `slot` hold a graph of the launches `body` issues (with the step index read from c->dev_step), re-capturing
+// when `key` differs from what the slot was captured for.  Nothing of `body` runs here.
+template <typename F>
+int graph_prepare(gm_ctx *c, gm_ctx::GraphSlot &slot, const std::vector<unsigned char> &key, F &&body) {
+  if (slot.exec && slot.key == key) return GM_OK;
+  if (slot.exec) { cudaGraphExecDestroy(slot.exec); slot.exec = nullptr; }
+  int rc;
+  if (!c->dev_step && (rc = dev_alloc(c, &c->dev_step, 1)) != GM_OK) return rc;
+  const int64_t before = c->launches;
+  GM_CUDA(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeRelaxed));
+  c->step_ptr = c->dev_step;
+  rc = body();
+  c->step_ptr = nullptr;
+  cudaGraph_t graph = nullptr;
+  const cudaError_t e = cudaStreamEndCapture(c->stream, &graph);         // always leave capture mode
+  const int64_t n = c->launches - before;
+  c->launches = before;                                                  // nothing has run yet
+  if (rc != GM_OK || e != cudaSuccess || !graph) {
+    if (graph) cudaGraphDestroy(graph);
+    if (e != cudaSuccess) { c->last_cuda = e; (void)cudaGetLastError(); }
+    return rc != GM_OK ? rc : GM_ERR_CUDA;
+  }
+  const cudaError_t ei = cudaGraphInstantiate(&slot.exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (ei != cudaSuccess) { c->last_cuda = ei; slot.exec = nullptr; return GM_ERR_CUDA; }
+  slot.launches = n;
+  slot.key = key;
+  return GM_OK;
+}
+
+
+}  // namespace gmh
