@@ -90,19 +90,21 @@ def test_capacity_is_reported_not_faulted():
     ctx.close()
 
 
-def test_4b_shape_batch_on_sampled_sequences():
+@pytest.mark.parametrize("qs", [4, 6, 8], ids=["k3_one_tile", "k5_transposed", "k7_two_tiles"])
+def test_4b_shape_batch_on_sampled_sequences(qs):
     """The benchmark's attention launch (64 sequences, KV uniform 1k..8k, 32 q / 8 kv heads, head_dim 128,
-    4 queries per sequence): three sampled sequences against the oracle, every row finite."""
+    4 queries per sequence; also 6 and 8 queries, which take the other two kernels): three sampled sequences
+    against the oracle, every row finite."""
     import paper_2609_16648_b200 as gmb
     from synth_inputs import kv_lengths_uniform
-    n_q, n_kv, hd, qs, B = 32, 8, 128, 4, 64
+    n_q, n_kv, hd, B = 32, 8, 128, 64
     lens = kv_lengths_uniform(B, 1024, 8192, seed=3).astype(np.int64)
     pt, npg = make_page_tables(lens + qs, 16, seed=7)
-    cfg = ModelConfig("a", 1, 64, n_q, n_kv, hd, 64, 8, batch=B, k=3, kv_len_min=0, kv_len_max=0, length_law="uniform")
-    ctx = gmb.Context(cfg, gmb.random_packed_weights(cfg, "cuda"), B, 3, pt.shape[1], npg, 4)
+    cfg = ModelConfig("a", 1, 64, n_q, n_kv, hd, 64, 8, batch=B, k=qs - 1, kv_len_min=0, kv_len_max=0, length_law="uniform")
+    ctx = gmb.Context(cfg, gmb.random_packed_weights(cfg, "cuda"), B, qs - 1, pt.shape[1], npg, 4)
     g = torch.Generator(device="cuda").manual_seed(1)
     pool = torch.randn((1, 2, npg, n_kv, 16, hd), device="cuda", generator=g).to(torch.bfloat16)
-    q = torch.randn((B, n_kv, 16, hd), device="cuda", generator=g).to(torch.bfloat16)
+    q = torch.randn((B, n_kv, 16 * ((qs * 4 + 15) // 16), hd), device="cuda", generator=g).to(torch.bfloat16)
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device="cuda", dtype=torch.int32)
     out = torch.zeros((B * qs, n_q * hd), dtype=torch.bfloat16, device="cuda")
     gmb.gm_attention(ctx, q, pool, 0, dev(np.where(pt < 0, 0, pt)), dev(np.full(B, qs)), dev(lens), B, qs, out)
