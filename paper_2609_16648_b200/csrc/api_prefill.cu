@@ -14,42 +14,49 @@ int gm_prefill(gm_ctx *c, gm_state *st, const int32_t *prompt_tok, const int32_t
   if (max_prompt_len + cf.max_k + 1 > cf.max_pages_per_seq * GM_PAGE) return GM_ERR_KV_CAPACITY;
   SamplerArgs S;
   if ((rc = fill_sampler(c, S, temperature)) != GM_OK) return rc;
-  const int B = st->batch, QT = cf.max_k + 1;
+  // Every pass gives each prompt VR consecutive chunks of QT positions: VR "virtual rows" per sequence, which the
+  // planner, the rotary/append kernel and attention treat as independent sequences sharing the prompt's page table
+  // (all keys of the pass are appended before attention runs, and each row attends only positions up to its own).
+  const int B = st->batch, QT = cf.max_k + 1, VR = c->pf_vr, R = B * VR;
   PhaseShape ph;
-  ph.B = B; ph.QT = QT; ph.M = B * QT; ph.qrows = round16(QT * c->group);
+  ph.B = R; ph.QT = QT; ph.M = R * QT; ph.qrows = round16(QT * c->group);
   CUtensorMap kvm, hkvm;
   if ((rc = kv_map(c, st->kv_pool, cf.n_layers, cf.num_pages, &kvm)) != GM_OK) return rc;
   if ((rc = kv_map(c, st->head_kv_pool, 1, cf.head_num_pages, &hkvm)) != GM_OK) return rc;
-  for (int base = 0; base < max_prompt_len; base += QT) {
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_dup_table_rows(st->page_table, B, VR, cf.max_pages_per_seq, c->pf_vtable[0], c->stream));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_dup_table_rows(st->head_page_table, B, VR, cf.max_pages_per_seq, c->pf_vtable[1], c->stream));
+  for (int base = 0; base < max_prompt_len; base += VR * QT) {
     ChunkSetupArgs Cs;
     Cs.prompt_tok = prompt_tok; Cs.prompt_len = prompt_len; Cs.batch = B; Cs.stride = prompt_stride; Cs.base = base;
-    Cs.QT = QT; Cs.max_len = max_prompt_len; Cs.pair_stride = QT; Cs.row_n = c->pf_row_n; Cs.head_n = c->pf_head_n;
-    Cs.pair_tok = c->pf_pair_tok; Cs.status = c->status;
+    Cs.QT = QT; Cs.max_len = max_prompt_len; Cs.pair_stride = QT; Cs.vr = VR; Cs.row_n = c->pf_row_n; Cs.head_n = c->pf_head_n;
+    Cs.pair_tok = c->pf_pair_tok; Cs.row_base = c->pf_row_base; Cs.status = c->status;
     GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_chunk_setup(Cs, c->stream));
-    // the backbone over positions base .. base + QT - 1 of every prompt that reaches them
-    if ((rc = run_plan_chunk(c, B, c->pf_row_n, base, QT)) != GM_OK) return rc;
+    // the backbone over positions base .. base + VR * QT - 1 of every prompt that reaches them
+    if ((rc = run_plan_chunk(c, R, c->pf_row_n, c->pf_row_base, QT)) != GM_OK) return rc;
     GM_LAUNCH(c, GM_KC_ELEMENTWISE,
               launch_embed_chunk(static_cast<const __nv_bfloat16 *>(c->w.embed),
-                                 static_cast<const __nv_bfloat16 *>(c->layers[0].ln1), prompt_tok, prompt_stride, base,
-                                 c->pf_row_n, B, QT, c->d, c->V, cf.rms_eps, c->x, c->xn, c->status, c->stream));
+                                 static_cast<const __nv_bfloat16 *>(c->layers[0].ln1), prompt_tok, prompt_stride,
+                                 c->pf_row_base, c->pf_row_n, R, VR, QT, c->d, c->V, cf.rms_eps, c->x, c->xn, c->status,
+                                 c->stream));
     for (int l = 0; l < cf.n_layers; ++l) {
       const bool last = l + 1 == cf.n_layers;
       rc = run_layer(c, c->layers[l], c->lmaps[l], ph, kvm, static_cast<__nv_bfloat16 *>(st->kv_pool), l, cf.num_pages,
-                     st->page_table, last ? nullptr : static_cast<const __nv_bfloat16 *>(c->layers[l + 1].ln1),
+                     c->pf_vtable[0], last ? nullptr : static_cast<const __nv_bfloat16 *>(c->layers[l + 1].ln1),
                      last ? c->pf_hidden : nullptr);
       if (rc) return rc;
     }
     if (c->capture)
       GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-                launch_capture_chunk(c->pf_hidden, c->pf_row_n, B, QT, base, c->d, c->capture, c->capture_stride, c->stream));
+                launch_capture_chunk(c->pf_hidden, c->pf_row_n, c->pf_row_base, R, VR, QT, c->d, c->capture,
+                                     c->capture_stride, c->stream));
     GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-              launch_prefill_last(c->x, c->pf_hidden, c->pf_row_n, prompt_len, B, base, QT, c->d, QT, c->pf_xlast,
-                                  static_cast<__nv_bfloat16 *>(st->pending_hidden), c->stream));
+              launch_prefill_last(c->x, c->pf_hidden, c->pf_row_n, c->pf_row_base, prompt_len, R, VR, QT, c->d, QT,
+                                  c->pf_xlast, static_cast<__nv_bfloat16 *>(st->pending_hidden), c->stream));
     // the draft head over the pairs (hidden of position t, token t + 1) of the same chunk, at head positions t
     if (base + 1 < max_prompt_len) {
-      if ((rc = run_plan_chunk(c, B, c->pf_head_n, base, QT)) != GM_OK) return rc;
+      if ((rc = run_plan_chunk(c, R, c->pf_head_n, c->pf_row_base, QT)) != GM_OK) return rc;
       HeadInputArgs H;
-      H.mode = PHASE_DRAFT_FIRST; H.batch = B; H.QT = QT; H.d = c->d; H.vocab = c->V; H.max_k = cf.max_k; H.k = 1; H.j = 1;
+      H.mode = PHASE_DRAFT_FIRST; H.batch = R; H.QT = QT; H.d = c->d; H.vocab = c->V; H.max_k = cf.max_k; H.k = 1; H.j = 1;
       H.eps = cf.rms_eps; H.embed = static_cast<const __nv_bfloat16 *>(c->w.embed);
       H.we = static_cast<const __nv_bfloat16 *>(c->w.head_enorm); H.wh = static_cast<const __nv_bfloat16 *>(c->w.head_hnorm);
       H.pending_tok = c->pf_pair_tok; H.pending_n = c->pf_head_n; H.pending_hidden = c->pf_hidden; H.draft_tok = nullptr;
@@ -62,7 +69,7 @@ int gm_prefill(gm_ctx *c, gm_state *st, const int32_t *prompt_tok, const int32_t
                 launch_rmsnorm(c->x, static_cast<const __nv_bfloat16 *>(c->w.head_layer.ln1), c->xn, nullptr, ph.M, c->d,
                                cf.rms_eps, c->stream));
       rc = run_layer(c, c->w.head_layer, c->head_maps, ph, hkvm, static_cast<__nv_bfloat16 *>(st->head_kv_pool), 0,
-                     cf.head_num_pages, st->head_page_table, nullptr, nullptr);
+                     cf.head_num_pages, c->pf_vtable[1], nullptr, nullptr);
       if (rc) return rc;
     }
   }
@@ -93,23 +100,24 @@ int gm_head_prefill(gm_ctx *c, gm_state *st, const void *seq_hidden, int hid_str
     return GM_ERR_INVALID_ARG;
   const gm_config &cf = c->cfg;
   if (max_len + cf.max_k + 1 > cf.max_pages_per_seq * GM_PAGE) return GM_ERR_KV_CAPACITY;
-  const int B = st->batch, QT = cf.max_k + 1;
+  const int B = st->batch, QT = cf.max_k + 1, VR = c->pf_vr, R = B * VR;          // virtual rows as in gm_prefill
   PhaseShape ph;
-  ph.B = B; ph.QT = QT; ph.M = B * QT; ph.qrows = round16(QT * c->group);
+  ph.B = R; ph.QT = QT; ph.M = R * QT; ph.qrows = round16(QT * c->group);
   CUtensorMap hkvm;
   if ((rc = kv_map(c, st->head_kv_pool, 1, cf.head_num_pages, &hkvm)) != GM_OK) return rc;
-  for (int base = 0; base + 1 < max_len; base += QT) {
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_dup_table_rows(st->head_page_table, B, VR, cf.max_pages_per_seq, c->pf_vtable[1], c->stream));
+  for (int base = 0; base + 1 < max_len; base += VR * QT) {
     ChunkSetupArgs Cs;
     Cs.prompt_tok = seq_tok; Cs.prompt_len = seq_len; Cs.batch = B; Cs.stride = tok_stride; Cs.base = base; Cs.QT = QT;
-    Cs.max_len = max_len; Cs.pair_stride = QT; Cs.row_n = c->pf_row_n; Cs.head_n = c->pf_head_n;
-    Cs.pair_tok = c->pf_pair_tok; Cs.status = c->status;
+    Cs.max_len = max_len; Cs.pair_stride = QT; Cs.vr = VR; Cs.row_n = c->pf_row_n; Cs.head_n = c->pf_head_n;
+    Cs.pair_tok = c->pf_pair_tok; Cs.row_base = c->pf_row_base; Cs.status = c->status;
     GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_chunk_setup(Cs, c->stream));
     GM_LAUNCH(c, GM_KC_ELEMENTWISE,
-              launch_gather_chunk_hidden(static_cast<const __nv_bfloat16 *>(seq_hidden), hid_stride, base, B, QT, c->d,
-                                         c->pf_head_n, c->pf_hidden, c->stream));
-    if ((rc = run_plan_chunk(c, B, c->pf_head_n, base, QT)) != GM_OK) return rc;
+              launch_gather_chunk_hidden(static_cast<const __nv_bfloat16 *>(seq_hidden), hid_stride, c->pf_row_base, R, VR, QT,
+                                         c->d, c->pf_head_n, c->pf_hidden, c->stream));
+    if ((rc = run_plan_chunk(c, R, c->pf_head_n, c->pf_row_base, QT)) != GM_OK) return rc;
     HeadInputArgs H;
-    H.mode = PHASE_DRAFT_FIRST; H.batch = B; H.QT = QT; H.d = c->d; H.vocab = c->V; H.max_k = cf.max_k; H.k = 1; H.j = 1;
+    H.mode = PHASE_DRAFT_FIRST; H.batch = R; H.QT = QT; H.d = c->d; H.vocab = c->V; H.max_k = cf.max_k; H.k = 1; H.j = 1;
     H.eps = cf.rms_eps; H.embed = static_cast<const __nv_bfloat16 *>(c->w.embed);
     H.we = static_cast<const __nv_bfloat16 *>(c->w.head_enorm); H.wh = static_cast<const __nv_bfloat16 *>(c->w.head_hnorm);
     H.pending_tok = c->pf_pair_tok; H.pending_n = c->pf_head_n; H.pending_hidden = c->pf_hidden; H.draft_tok = nullptr;
@@ -122,7 +130,7 @@ int gm_head_prefill(gm_ctx *c, gm_state *st, const void *seq_hidden, int hid_str
               launch_rmsnorm(c->x, static_cast<const __nv_bfloat16 *>(c->w.head_layer.ln1), c->xn, nullptr, ph.M, c->d,
                              cf.rms_eps, c->stream));
     rc = run_layer(c, c->w.head_layer, c->head_maps, ph, hkvm, static_cast<__nv_bfloat16 *>(st->head_kv_pool), 0,
-                   cf.head_num_pages, st->head_page_table, nullptr, nullptr);
+                   cf.head_num_pages, c->pf_vtable[1], nullptr, nullptr);
     if (rc) return rc;
   }
   return GM_OK;

@@ -63,7 +63,7 @@ __global__ void plan_kernel(const PlanArgs A) {
     int qn, qbase;
     if (A.mode == PHASE_VERIFY) { qn = A.k_or_j + 1; qbase = len; }
     else if (A.mode == PHASE_DRAFT_FIRST) { qn = A.pending_n[b]; qbase = len - qn; }
-    else if (A.mode == PHASE_CHUNK) { qn = A.row_n[b]; qbase = A.k_or_j; }
+    else if (A.mode == PHASE_CHUNK) { qn = A.row_n[b]; qbase = A.row_base ? A.row_base[b] : A.k_or_j; }
     else { qn = 1; qbase = len + A.k_or_j - 2; }
     bool ok = qn >= 1 && qbase >= 0 && qbase + qn <= A.max_pages_per_seq * 16;
     if (A.finished && A.finished[b]) { A.qn[b] = 0; A.qbase[b] = 0; pages[b] = 0; continue; }    // sits the phase out
@@ -185,29 +185,40 @@ cudaError_t launch_page_release(const PageAllocArgs &A, cudaStream_t stream) {
 // ---- prompt prefill: chunk bookkeeping ----------------------------------------------------------------------
 __global__ void chunk_setup_kernel(const ChunkSetupArgs A) {
   pdl_prologue();
-  for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < A.batch; b += gridDim.x * blockDim.x) {
+  for (int v = blockIdx.x * blockDim.x + threadIdx.x; v < A.batch * A.vr; v += gridDim.x * blockDim.x) {
+    const int b = v / A.vr, p0 = A.base + (v % A.vr) * A.QT;
     const int L = A.prompt_len[b];
     const bool bad = L < 1 || L > A.max_len || L > A.stride;
-    if (bad && A.base == 0) set_status(A.status, ST_KV_CAPACITY);
-    const int n = bad ? 0 : min(max(L - A.base, 0), A.QT);
-    const int hn = bad ? 0 : min(max(L - 1 - A.base, 0), A.QT);
-    A.row_n[b] = n;
-    A.head_n[b] = hn;
+    if (bad && p0 == 0) set_status(A.status, ST_KV_CAPACITY);
+    const int n = bad ? 0 : min(max(L - p0, 0), A.QT);
+    const int hn = bad ? 0 : min(max(L - 1 - p0, 0), A.QT);
+    A.row_n[v] = n;
+    A.head_n[v] = hn;
+    A.row_base[v] = p0;
     for (int j = 0; j < A.QT; ++j)
-      A.pair_tok[b * A.pair_stride + j] = j < hn ? A.prompt_tok[static_cast<size_t>(b) * A.stride + A.base + j + 1] : 0;
+      A.pair_tok[v * A.pair_stride + j] = j < hn ? A.prompt_tok[static_cast<size_t>(b) * A.stride + p0 + j + 1] : 0;
   }
 }
 cudaError_t launch_chunk_setup(const ChunkSetupArgs &A, cudaStream_t stream) {
-  return launch_k(chunk_setup_kernel, dim3((A.batch + 127) / 128), dim3(128), 0, stream, 1, A);
+  return launch_k(chunk_setup_kernel, dim3((A.batch * A.vr + 127) / 128), dim3(128), 0, stream, 1, A);
+}
+
+__global__ void dup_table_rows_kernel(const int32_t *src, int vr, int cols, int32_t *dst) {
+  pdl_prologue();
+  const int v = blockIdx.x;
+  for (int i = threadIdx.x; i < cols; i += blockDim.x) dst[static_cast<size_t>(v) * cols + i] = src[static_cast<size_t>(v / vr) * cols + i];
+}
+cudaError_t launch_dup_table_rows(const int32_t *src, int rows, int vr, int cols, int32_t *dst, cudaStream_t stream) {
+  return launch_k(dup_table_rows_kernel, dim3(rows * vr), dim3(128), 0, stream, 1, src, vr, cols, dst);
 }
 
 __global__ void __launch_bounds__(EW_THREADS)
-embed_chunk_kernel(const __nv_bfloat16 *embed, const __nv_bfloat16 *w, const int32_t *prompt_tok, int stride, int base,
-                   const int32_t *row_n, int QT, int d, int vocab, float eps, float *x, __nv_bfloat16 *xn,
-                   uint32_t *status) {
-  const int m = blockIdx.x, b = m / QT, j = m % QT;
+embed_chunk_kernel(const __nv_bfloat16 *embed, const __nv_bfloat16 *w, const int32_t *prompt_tok, int stride,
+                   const int32_t *row_base, const int32_t *row_n, int vr, int QT, int d, int vocab, float eps, float *x,
+                   __nv_bfloat16 *xn, uint32_t *status) {
+  const int m = blockIdx.x, vrow = m / QT, j = m % QT;
   pdl_prologue();
-  int tok = j < row_n[b] ? prompt_tok[static_cast<size_t>(b) * stride + base + j] : 0;
+  int tok = j < row_n[vrow] ? prompt_tok[static_cast<size_t>(vrow / vr) * stride + row_base[vrow] + j] : 0;
   if (tok < 0 || tok >= vocab) { if (threadIdx.x == 0) set_status(status, ST_BAD_TOKEN); tok = 0; }
   const int d4 = d >> 2;
   float4 v[EW_MAXC];
@@ -222,30 +233,31 @@ embed_chunk_kernel(const __nv_bfloat16 *embed, const __nv_bfloat16 *w, const int
   rmsnorm_store(v, d4, d, eps, w, xn + static_cast<size_t>(m) * d);
 }
 cudaError_t launch_embed_chunk(const __nv_bfloat16 *embed, const __nv_bfloat16 *w, const int32_t *prompt_tok, int stride,
-                               int base, const int32_t *row_n, int batch, int QT, int d, int vocab, float eps, float *x,
-                               __nv_bfloat16 *xn, uint32_t *status, cudaStream_t stream) {
-  return launch_k(embed_chunk_kernel, dim3(batch * QT), dim3(EW_THREADS), 0, stream, 1, embed, w, prompt_tok, stride,
-                  base, row_n, QT, d, vocab, eps, x, xn, status);
+                               const int32_t *row_base, const int32_t *row_n, int rows, int vr, int QT, int d, int vocab,
+                               float eps, float *x, __nv_bfloat16 *xn, uint32_t *status, cudaStream_t stream) {
+  return launch_k(embed_chunk_kernel, dim3(rows * QT), dim3(EW_THREADS), 0, stream, 1, embed, w, prompt_tok, stride,
+                  row_base, row_n, vr, QT, d, vocab, eps, x, xn, status);
 }
 
 __global__ void __launch_bounds__(EW_THREADS)
-prefill_last_kernel(const float *x, const __nv_bfloat16 *hidden, const int32_t *row_n, const int32_t *prompt_len,
-                    int base, int QT, int d, int pend_stride, float *xlast, __nv_bfloat16 *pending_hidden) {
-  const int b = blockIdx.x;
+prefill_last_kernel(const float *x, const __nv_bfloat16 *hidden, const int32_t *row_n, const int32_t *row_base,
+                    const int32_t *prompt_len, int vr, int QT, int d, int pend_stride, float *xlast,
+                    __nv_bfloat16 *pending_hidden) {
+  const int v = blockIdx.x, b = v / vr;
   pdl_prologue();
-  const int n = row_n[b];
-  if (n < 1 || base + n != prompt_len[b]) return;
-  const size_t m = static_cast<size_t>(b) * QT + n - 1;
+  const int n = row_n[v];
+  if (n < 1 || row_base[v] + n != prompt_len[b]) return;
+  const size_t m = static_cast<size_t>(v) * QT + n - 1;
   for (int i = threadIdx.x; i < d; i += EW_THREADS) {
     xlast[static_cast<size_t>(b) * d + i] = x[m * d + i];
     pending_hidden[static_cast<size_t>(b) * pend_stride * d + i] = hidden[m * d + i];
   }
 }
 cudaError_t launch_prefill_last(const float *x, const __nv_bfloat16 *hidden, const int32_t *row_n,
-                                const int32_t *prompt_len, int batch, int base, int QT, int d, int pend_stride,
-                                float *xlast, __nv_bfloat16 *pending_hidden, cudaStream_t stream) {
-  return launch_k(prefill_last_kernel, dim3(batch), dim3(EW_THREADS), 0, stream, 1, x, hidden, row_n, prompt_len, base,
-                  QT, d, pend_stride, xlast, pending_hidden);
+                                const int32_t *row_base, const int32_t *prompt_len, int rows, int vr, int QT, int d,
+                                int pend_stride, float *xlast, __nv_bfloat16 *pending_hidden, cudaStream_t stream) {
+  return launch_k(prefill_last_kernel, dim3(rows), dim3(EW_THREADS), 0, stream, 1, x, hidden, row_n, row_base,
+                  prompt_len, vr, QT, d, pend_stride, xlast, pending_hidden);
 }
 
 __global__ void prefill_finish_kernel(const int32_t *prompt_len, const int32_t *first_tok, int batch, int pend_stride,

@@ -102,7 +102,8 @@ gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
   float *park = reinterpret_cast<float *>(smem);                // [T][128] fp32, reuses the pipeline stages
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = A.n_base + blockIdx.x * GT_BN * wt, m0 = blockIdx.y * T, split = blockIdx.z, ns = A.nsplit;
+  // token blocks vary fastest in the grid, so that the CTAs that share a weight tile run together and it leaves HBM once
+  const int n0 = A.n_base + blockIdx.y * GT_BN * wt, m0 = blockIdx.x * T, split = blockIdx.z, ns = A.nsplit;
   const int KB = A.K / GT_BK;
   const int kb_lo = static_cast<int>(static_cast<long long>(split) * KB / ns);
   const int kb_hi = static_cast<int>(static_cast<long long>(split + 1) * KB / ns);
@@ -254,7 +255,7 @@ cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream) {
   const size_t smem = gt_smem(T, A.wtiles);
   cudaError_t ec = gt_configure();
   if (ec != cudaSuccess) return ec;
-  const dim3 grid(A.n_tiles, (A.M + T - 1) / T, A.nsplit);
+  const dim3 grid((A.M + T - 1) / T, A.n_tiles, A.nsplit);
   return launch_k(gemm_tc_kernel, grid, dim3(GT_THREADS), smem, stream, A.nsplit, A, gt_stages(T, A.wtiles));
 }
 

@@ -191,9 +191,9 @@ int run_plan(gm_ctx *c, const gm_state *st, int mode, int k_or_j) {
   return GM_OK;
 }
 
-int run_plan_chunk(gm_ctx *c, int batch, const int32_t *row_n, int base, int QT) {
+int run_plan_chunk(gm_ctx *c, int batch, const int32_t *row_n, const int32_t *row_base, int QT) {
   PlanArgs P;
-  P.mode = PHASE_CHUNK; P.batch = batch; P.k_or_j = base; P.max_pages_per_seq = c->cfg.max_pages_per_seq;
+  P.mode = PHASE_CHUNK; P.batch = batch; P.k_or_j = 0; P.row_base = row_base; P.max_pages_per_seq = c->cfg.max_pages_per_seq;
   P.n_ctas = c->sm_count; P.kv_len = row_n; P.pending_n = row_n; P.row_n = row_n; P.QT = QT; P.qn = c->qn; P.qbase = c->qbase;
   P.page_start = c->page_start; P.status = c->status;
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_plan(P, c->stream));
@@ -319,7 +319,11 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
   if (make_map(c, &c->head_proj_map, w->head_proj, c->d, 2 * c->d, 128)) return fail(GM_ERR_CUDA);
 
   // workspaces
-  const size_t M = c->Mmax, B = cfg->max_batch;
+  // Sized for the widest phase: a prefill pass of pf_vr virtual rows per sequence (at most 1024 rows for the planner).
+  c->pf_vr = std::max(1, std::min(8, 1024 / cfg->max_batch));
+  const size_t B1 = cfg->max_batch, M1 = c->Mmax;                  // rows of a cycle
+  const size_t B = B1 * c->pf_vr, M = M1 * c->pf_vr;                // rows of a prefill pass
+  c->Mmax = static_cast<int>(M);
   const int qrows = round16((cfg->max_k + 1) * group);
   for (auto &row : c->max_clusters)
     for (int &v : row) v = -1;
@@ -333,28 +337,31 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
   A_(dev_alloc(c, &c->qbuf, B * cfg->n_kv_heads * qrows * cfg->head_dim));
   A_(dev_alloc(c, &c->attn_out, M * c->q_dim));
   A_(dev_alloc(c, &c->act, M * c->F));
-  A_(dev_alloc(c, &c->g, B * c->d));
-  A_(dev_alloc(c, &c->gn, B * c->d));
+  A_(dev_alloc(c, &c->g, B1 * c->d));
+  A_(dev_alloc(c, &c->gn, B1 * c->d));
   A_(dev_alloc(c, &c->part_o, slots * cfg->n_kv_heads * qrows * cfg->head_dim));
   A_(dev_alloc(c, &c->part_ml, slots * cfg->n_kv_heads * qrows * 2));
-  A_(dev_alloc(c, &c->ws_draft_logits, B * cfg->max_k * c->V, false));
-  A_(dev_alloc(c, &c->ws_target_logits, B * (cfg->max_k + 1) * c->V, false));
-  A_(dev_alloc(c, &c->ws_target_hidden, M * c->d));
-  A_(dev_alloc(c, &c->ws_draft_tok, B * cfg->max_k));
-  A_(dev_alloc(c, &c->ws_accept_len, B));
-  A_(dev_alloc(c, &c->ws_next_token, B));
-  A_(dev_alloc(c, &c->ws_u24, B * (2 * cfg->max_k + 1)));
+  A_(dev_alloc(c, &c->ws_draft_logits, B1 * cfg->max_k * c->V, false));
+  A_(dev_alloc(c, &c->ws_target_logits, B1 * (cfg->max_k + 1) * c->V, false));
+  A_(dev_alloc(c, &c->ws_target_hidden, M1 * c->d));
+  A_(dev_alloc(c, &c->ws_draft_tok, B1 * cfg->max_k));
+  A_(dev_alloc(c, &c->ws_accept_len, B1));
+  A_(dev_alloc(c, &c->ws_next_token, B1));
+  A_(dev_alloc(c, &c->ws_u24, B1 * (2 * cfg->max_k + 1)));
   A_(dev_alloc(c, &c->qn, B));
   A_(dev_alloc(c, &c->qbase, B));
   A_(dev_alloc(c, &c->page_start, B + 1));
-  A_(dev_alloc(c, &c->ro_accept, B));
-  A_(dev_alloc(c, &c->ro_next, B));
+  A_(dev_alloc(c, &c->ro_accept, B1));
+  A_(dev_alloc(c, &c->ro_next, B1));
   A_(dev_alloc(c, &c->pf_row_n, B));
   A_(dev_alloc(c, &c->pf_head_n, B));
-  A_(dev_alloc(c, &c->pf_first, B));
+  A_(dev_alloc(c, &c->pf_row_base, B));
+  A_(dev_alloc(c, &c->pf_vtable[0], B * cfg->max_pages_per_seq));
+  A_(dev_alloc(c, &c->pf_vtable[1], B * cfg->max_pages_per_seq));
+  A_(dev_alloc(c, &c->pf_first, B1));
   A_(dev_alloc(c, &c->pf_pair_tok, B * (cfg->max_k + 1)));
   A_(dev_alloc(c, &c->pf_hidden, M * c->d));
-  A_(dev_alloc(c, &c->pf_xlast, B * c->d));
+  A_(dev_alloc(c, &c->pf_xlast, B1 * c->d));
   A_(dev_alloc(c, &c->status, 1));
   // rotary table: cos/sin of pos * base^(-2i/hd), computed in double precision on the host
   {

@@ -59,6 +59,10 @@ struct gm_ctx {
   float2 *rope = nullptr;
   uint32_t *status = nullptr;
   // prompt prefill: per-chunk bookkeeping, the chunk's hidden states, the row of each prompt's last token
+  // A prefill pass gives every prompt pf_vr consecutive chunks of max_k + 1 positions ("virtual rows" that share the
+  // prompt's page table), so the M-sized workspaces below hold max_batch * pf_vr * (max_k + 1) rows.
+  int pf_vr = 1;
+  int32_t *pf_row_base = nullptr, *pf_vtable[2] = {nullptr, nullptr};   // first position and page-table row per virtual row
   int32_t *pf_row_n = nullptr, *pf_head_n = nullptr, *pf_pair_tok = nullptr, *pf_first = nullptr;
   __nv_bfloat16 *pf_hidden = nullptr;
   float *pf_xlast = nullptr;
@@ -153,7 +157,7 @@ int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const 
               __nv_bfloat16 *pool, int layer, int num_pages, const int32_t *page_table,
               const __nv_bfloat16 *next_norm, __nv_bfloat16 *hidden_out);
 int run_plan(gm_ctx *c, const gm_state *st, int mode, int k_or_j);
-int run_plan_chunk(gm_ctx *c, int batch, const int32_t *row_n, int base, int QT);
+int run_plan_chunk(gm_ctx *c, int batch, const int32_t *row_n, const int32_t *row_base, int QT);
 int check_state(const gm_ctx *c, const gm_state *st, int k);
 cudaError_t run_sampler(gm_ctx *c, const SamplerArgs &S, int batch);
 int fill_sampler(gm_ctx *c, SamplerArgs &S, float temperature);

@@ -106,6 +106,7 @@ struct PlanArgs {
   const int32_t *kv_len, *pending_n;
   const int32_t *finished = nullptr;    // [B] non-zero: the sequence sits the phase out (no queries, no pages); or null
   const int32_t *row_n = nullptr;       // CHUNK: queries per sequence (0 = the sequence sits this pass out)
+  const int32_t *row_base = nullptr;    // CHUNK: first position per sequence (null: k_or_j for all)
   int QT = 0;                           // CHUNK: most queries a sequence may have
   int32_t *qn, *qbase;                  // [B] queries of this phase and the position of the first one
   int32_t *page_start;                  // [B+1] exclusive prefix of pages attended per sequence
@@ -118,22 +119,27 @@ cudaError_t launch_plan(const PlanArgs &A, cudaStream_t stream);
 // ended before), head_n[b] = how many of them have a successor token inside the prompt (the pairs the draft head
 // is prefilled with), pair_tok[b][j] = token at position base + j + 1.  A prompt shorter than 1 or longer than
 // max_len raises ST_KV_CAPACITY and sits out.
+// A pass may give every prompt `vr` consecutive chunks ("virtual rows": row v = b * vr + i holds positions
+// base + i * QT .. + QT - 1 of prompt b), which the planner and the attention kernel see as vr independent
+// sequences sharing a page table; row_base[v] = its first position.
 struct ChunkSetupArgs {
   const int32_t *prompt_tok, *prompt_len;
-  int batch, stride, base, QT, max_len, pair_stride;
-  int32_t *row_n, *head_n, *pair_tok;
+  int batch, stride, base, QT, max_len, pair_stride, vr;
+  int32_t *row_n, *head_n, *pair_tok, *row_base;
   uint32_t *status;
 };
 cudaError_t launch_chunk_setup(const ChunkSetupArgs &A, cudaStream_t stream);
 // x[m] = embed[prompt_tok[b][base + j]] (fp32), xn[m] = RMSNorm(x[m]; w) (bf16) for j < row_n[b]; other rows token 0.
 cudaError_t launch_embed_chunk(const __nv_bfloat16 *embed, const __nv_bfloat16 *w, const int32_t *prompt_tok, int stride,
-                               int base, const int32_t *row_n, int batch, int QT, int d, int vocab, float eps, float *x,
-                               __nv_bfloat16 *xn, uint32_t *status, cudaStream_t stream);
+                               const int32_t *row_base, const int32_t *row_n, int rows, int vr, int QT, int d, int vocab,
+                               float eps, float *x, __nv_bfloat16 *xn, uint32_t *status, cudaStream_t stream);
+// dst[v] = src[v / vr] for v < rows * vr: the page-table rows of the virtual rows
+cudaError_t launch_dup_table_rows(const int32_t *src, int rows, int vr, int cols, int32_t *dst, cudaStream_t stream);
 // For the sequences whose prompt ends inside this chunk: xlast[b] = x[row of the last prompt token] (fp32) and
 // pending_hidden[b][0] = the same row of `hidden` (bf16).
 cudaError_t launch_prefill_last(const float *x, const __nv_bfloat16 *hidden, const int32_t *row_n,
-                                const int32_t *prompt_len, int batch, int base, int QT, int d, int pend_stride,
-                                float *xlast, __nv_bfloat16 *pending_hidden, cudaStream_t stream);
+                                const int32_t *row_base, const int32_t *prompt_len, int rows, int vr, int QT, int d,
+                                int pend_stride, float *xlast, __nv_bfloat16 *pending_hidden, cudaStream_t stream);
 // kv_len[b] = prompt_len[b], pending_n[b] = 1, pending_tok[b][0] = first_tok[b].
 cudaError_t launch_prefill_finish(const int32_t *prompt_len, const int32_t *first_tok, int batch, int pend_stride,
                                   int32_t *kv_len, int32_t *pending_n, int32_t *pending_tok, cudaStream_t stream);
@@ -180,9 +186,9 @@ struct ChainSetupArgs {
   uint32_t *status;
 };
 cudaError_t launch_chain_setup(const ChainSetupArgs &A, int chains, cudaStream_t stream);
-// out[b*QT + j] = seq_hidden[b][base + j] for j < row_n[b]
-cudaError_t launch_gather_chunk_hidden(const __nv_bfloat16 *seq_hidden, int hid_stride, int base, int batch, int QT, int d,
-                                       const int32_t *row_n, __nv_bfloat16 *out, cudaStream_t stream);
+// out[v*QT + j] = seq_hidden[v / vr][row_base[v] + j] for j < row_n[v]
+cudaError_t launch_gather_chunk_hidden(const __nv_bfloat16 *seq_hidden, int hid_stride, const int32_t *row_base, int rows,
+                                       int vr, int QT, int d, const int32_t *row_n, __nv_bfloat16 *out, cudaStream_t stream);
 struct OverlapArgs {
   const __nv_bfloat16 *logits;                     // [rows, V] head logits of the reconstructed chains
   const int32_t *top_index;                        // [rows, 64]
@@ -194,11 +200,11 @@ struct OverlapArgs {
 cudaError_t launch_overlap(const OverlapArgs &A, int rows, cudaStream_t stream);
 // Rollout-time capture of the target hidden states of committed positions (App. D.2: "each sequence additionally
 // stores the rollout-time target hidden states"): dst[b][pos] = the hidden state computed at position pos.
-//   chunk form (prefill): rows j < row_n[b] of src [B, QT, d] go to positions base + j;
+//   chunk form (prefill): rows j < row_n[v] of src [rows, QT, d] go to positions row_base[v] + j of sequence v / vr;
 //   cycle form: rows l <= accept_len[b] of src [B, k+1, d] go to positions kv_len[b] - (accept_len[b] + 1) + l, with
 //   kv_len already advanced by the commit; rows of finished sequences are skipped.
-cudaError_t launch_capture_chunk(const __nv_bfloat16 *src, const int32_t *row_n, int batch, int QT, int base, int d,
-                                 __nv_bfloat16 *dst, int dst_stride, cudaStream_t stream);
+cudaError_t launch_capture_chunk(const __nv_bfloat16 *src, const int32_t *row_n, const int32_t *row_base, int rows, int vr,
+                                 int QT, int d, __nv_bfloat16 *dst, int dst_stride, cudaStream_t stream);
 cudaError_t launch_capture_cycle(const __nv_bfloat16 *src, const int32_t *accept_len, const int32_t *kv_len,
                                  const int32_t *finished, int batch, int k, int d, __nv_bfloat16 *dst, int dst_stride,
                                  cudaStream_t stream);

@@ -56,12 +56,12 @@ __global__ void __launch_bounds__(128) chain_setup_kernel(const ChainSetupArgs A
 }
 
 __global__ void __launch_bounds__(128)
-gather_chunk_hidden_kernel(const __nv_bfloat16 *seq_hidden, int hid_stride, int base, int QT, int d, const int32_t *row_n,
-                           __nv_bfloat16 *out) {
-  const int m = blockIdx.x, b = m / QT, j = m % QT;
+gather_chunk_hidden_kernel(const __nv_bfloat16 *seq_hidden, int hid_stride, const int32_t *row_base, int vr, int QT, int d,
+                           const int32_t *row_n, __nv_bfloat16 *out) {
+  const int m = blockIdx.x, v = m / QT, j = m % QT;
   pdl_prologue();
-  if (j >= row_n[b]) return;
-  const uint4 *s = reinterpret_cast<const uint4 *>(seq_hidden + (static_cast<size_t>(b) * hid_stride + base + j) * d);
+  if (j >= row_n[v]) return;
+  const uint4 *s = reinterpret_cast<const uint4 *>(seq_hidden + (static_cast<size_t>(v / vr) * hid_stride + row_base[v] + j) * d);
   uint4 *o = reinterpret_cast<uint4 *>(out + static_cast<size_t>(m) * d);
   for (int i = threadIdx.x; i < d / 8; i += blockDim.x) o[i] = s[i];
 }
@@ -165,13 +165,13 @@ __global__ void __launch_bounds__(DL_THREADS) dca_loss_kernel(const float *alpha
 }
 
 __global__ void __launch_bounds__(128)
-capture_chunk_kernel(const __nv_bfloat16 *src, const int32_t *row_n, int QT, int base, int d, __nv_bfloat16 *dst,
-                     int dst_stride) {
-  const int m = blockIdx.x, b = m / QT, j = m % QT;
+capture_chunk_kernel(const __nv_bfloat16 *src, const int32_t *row_n, const int32_t *row_base, int vr, int QT, int d,
+                     __nv_bfloat16 *dst, int dst_stride) {
+  const int m = blockIdx.x, v = m / QT, j = m % QT;
   pdl_prologue();
-  if (j >= row_n[b] || base + j >= dst_stride) return;
+  if (j >= row_n[v] || row_base[v] + j >= dst_stride) return;
   const uint4 *s = reinterpret_cast<const uint4 *>(src + static_cast<size_t>(m) * d);
-  uint4 *o = reinterpret_cast<uint4 *>(dst + (static_cast<size_t>(b) * dst_stride + base + j) * d);
+  uint4 *o = reinterpret_cast<uint4 *>(dst + (static_cast<size_t>(v / vr) * dst_stride + row_base[v] + j) * d);
   for (int i = threadIdx.x; i < d / 8; i += blockDim.x) o[i] = s[i];
 }
 __global__ void __launch_bounds__(128)
@@ -190,9 +190,10 @@ capture_cycle_kernel(const __nv_bfloat16 *src, const int32_t *accept_len, const 
 
 }  // namespace
 
-cudaError_t launch_capture_chunk(const __nv_bfloat16 *src, const int32_t *row_n, int batch, int QT, int base, int d,
-                                 __nv_bfloat16 *dst, int dst_stride, cudaStream_t stream) {
-  return launch_k(capture_chunk_kernel, dim3(batch * QT), dim3(128), 0, stream, 1, src, row_n, QT, base, d, dst, dst_stride);
+cudaError_t launch_capture_chunk(const __nv_bfloat16 *src, const int32_t *row_n, const int32_t *row_base, int rows, int vr,
+                                 int QT, int d, __nv_bfloat16 *dst, int dst_stride, cudaStream_t stream) {
+  return launch_k(capture_chunk_kernel, dim3(rows * QT), dim3(128), 0, stream, 1, src, row_n, row_base, vr, QT, d, dst,
+                  dst_stride);
 }
 cudaError_t launch_capture_cycle(const __nv_bfloat16 *src, const int32_t *accept_len, const int32_t *kv_len,
                                  const int32_t *finished, int batch, int k, int d, __nv_bfloat16 *dst, int dst_stride,
@@ -204,10 +205,10 @@ cudaError_t launch_capture_cycle(const __nv_bfloat16 *src, const int32_t *accept
 cudaError_t launch_chain_setup(const ChainSetupArgs &A, int chains, cudaStream_t stream) {
   return launch_k(chain_setup_kernel, dim3(chains), dim3(128), 0, stream, 1, A);
 }
-cudaError_t launch_gather_chunk_hidden(const __nv_bfloat16 *seq_hidden, int hid_stride, int base, int batch, int QT, int d,
-                                       const int32_t *row_n, __nv_bfloat16 *out, cudaStream_t stream) {
-  return launch_k(gather_chunk_hidden_kernel, dim3(batch * QT), dim3(128), 0, stream, 1, seq_hidden, hid_stride, base, QT,
-                  d, row_n, out);
+cudaError_t launch_gather_chunk_hidden(const __nv_bfloat16 *seq_hidden, int hid_stride, const int32_t *row_base, int rows,
+                                       int vr, int QT, int d, const int32_t *row_n, __nv_bfloat16 *out, cudaStream_t stream) {
+  return launch_k(gather_chunk_hidden_kernel, dim3(rows * QT), dim3(128), 0, stream, 1, seq_hidden, hid_stride, row_base, vr,
+                  QT, d, row_n, out);
 }
 cudaError_t launch_overlap(const OverlapArgs &A, int rows, cudaStream_t stream) {
   return launch_k(overlap_kernel, dim3(rows), dim3(OV_THREADS), 0, stream, 1, A);
