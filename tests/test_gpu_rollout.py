@@ -196,3 +196,46 @@ def test_graph_replayed_rollout_equals_host_launched_rollout():
         assert torch.equal(h[5], g[5])
         assert g[6] == h[6] + 1 > 1                              # the replayed kernels are counted, plus one store of the first step index
     assert results[0][0][2] != results[0][1][2]                  # different step indices: different uniforms
+
+
+def test_graph_replay_with_on_demand_pages_and_stopping():
+    """The captured cycle includes the page reserve / release kernels and the finished mask: a graph-replayed rollout
+    with on-demand pages, an end-of-sequence token and a cap equals the host-launched one, and every page comes back."""
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny")
+    K, B, V = cfg.k, cfg.batch, cfg.vocab
+    w = perturb_norm_weights(make_weights(cfg, 0))
+    lengths = [5, 21, 12, 30]
+    rng = np.random.default_rng(4)
+    tok = np.zeros((B, 32), np.int32)
+    for b, n in enumerate(lengths):
+        tok[b, :n] = rng.integers(0, V, n)
+    max_new, n_steps = 20, 12
+    pt, npg = make_page_tables(np.full(B, 30 + max_new + 2 * (K + 1)), cfg.page_size, seed=7)
+    out = {}
+    side = torch.cuda.Stream()
+    for flags in (0, gmb.GM_FLAG_GRAPH):
+        with torch.cuda.stream(side):
+            ctx = gmb.Context(cfg, gmb.pack_weights(w), B, K, pt.shape[1], npg, npg, flags=flags)
+            st = gmb.State(ctx, B, np.full_like(pt, -1), np.full_like(pt, -1))
+            tok_d = torch.from_numpy(tok).cuda()
+            len_d = torch.tensor(lengths, dtype=torch.int32, device="cuda")
+            gmb.gm_pages_reset(ctx, st)
+            gmb.gm_pages_reserve(ctx, st, len_d, K + 1)
+            gmb.gm_prefill(ctx, st, tok_d, len_d, max(lengths), 1.0, None, 9)
+            eos = int(st.pending_tok[1, 0])                      # row 1 ends at once; the others run on
+            ro = gmb.Rollout(B, max_new, eos)
+            gmb.gm_rollout_begin(ctx, st, ro)
+            steps, running = gmb.gm_rollout_run(ctx, st, ro, K, 1.0, 9, 1, n_steps, check_every=4)
+            assert gmb.gm_last_status(ctx) == 0
+            out[flags] = (steps, running, ro.responses(), ro.finished.cpu().numpy().copy(), gmb.gm_pages_free_count(ctx),
+                          st.kv_len.cpu().numpy().copy())
+            ctx.close()
+        side.synchronize()
+    h, g = out[0], out[gmb.GM_FLAG_GRAPH]
+    assert h[2] == g[2] and (h[3] == g[3]).all() and (h[5] == g[5]).all() and h[1] == g[1]
+    assert h[3][1] == 1 and len(h[2][1]) == 1                    # ended on its first token
+    assert g[0] >= h[0] and g[0] - h[0] < 4                      # the replayed loop may run up to check_every - 1 idle cycles
+    assert h[4] == g[4]
+    if h[1] == 0:
+        assert h[4] == (npg, npg)
