@@ -104,9 +104,11 @@ def test_tiny_step_parity_from_common_state(flags):
 @pytest.mark.parametrize("extras", [dict(qkv_bias=True), dict(qk_norm=True),
                                     dict(qkv_bias=True, qk_norm=True, concat="hidden_first"),
                                     dict(qkv_bias=True, qk_norm=True, n_q_heads=2, n_kv_heads=1, head_dim=128),
-                                    dict(k=7), dict(k=1), dict(top_p=0.7)],
+                                    dict(k=7), dict(k=1), dict(top_p=0.7),
+                                    dict(k=5, n_q_heads=8, n_kv_heads=2, head_dim=128),
+                                    dict(k=7, n_q_heads=8, n_kv_heads=2, head_dim=128)],
                          ids=["qkv_bias", "qk_norm", "bias_norm_hidden_first", "bias_norm_head128", "depth7", "depth1",
-                              "top_p_0.7"])
+                              "top_p_0.7", "depth5_group4_24_rows", "depth7_group4_32_rows"])
 def test_tiny_step_parity_variants(extras):
     """The same bars for the other operating points of the cycle: the decoder-layer families of App. B.1
     (projection bias; query/key head norms), a head that concatenates [hidden ; embedding], and the
