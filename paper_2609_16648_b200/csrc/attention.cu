@@ -613,26 +613,49 @@ __global__ void __launch_bounds__(128) attention_combine_kernel(const AttnCombin
   for (int row = row_first; row < rows; row += 4 * gridDim.y) {
     const size_t base0 = (static_cast<size_t>(s_first) * A.n_kv + head) * A.qrows + row;
     const size_t seg_stride = static_cast<size_t>(A.n_kv) * A.qrows;
-    float mt = -INFINITY;
-    for (int s = lane; s < nseg; s += 32) mt = fmaxf(mt, A.part_ml[(base0 + s * seg_stride) * 2]);
+    const int c4 = lane;
+    // the partial outputs of the first segments are requested before the statistics are reduced: their latency
+    // overlaps the two warp reductions (most sequences have at most four segments)
+    constexpr int NPRE = 4;
+    float4 pre[NPRE];
+#pragma unroll
+    for (int s = 0; s < NPRE; ++s)
+      pre[s] = (s < nseg && c4 * 4 < hd) ? reinterpret_cast<const float4 *>(A.part_o + (base0 + s * seg_stride) * hd)[c4]
+                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+    // lane s holds (max, sum) of segment s (and s + 32, ...)
+    float2 ml = make_float2(-INFINITY, 0.f);
+    if (lane < nseg) ml = *reinterpret_cast<const float2 *>(A.part_ml + (base0 + lane * seg_stride) * 2);
+    float mt = ml.x;
+    for (int s = lane + 32; s < nseg; s += 32) mt = fmaxf(mt, A.part_ml[(base0 + s * seg_stride) * 2]);
     mt = warp_max(mt);
-    float l = 0.f;
-    for (int s = lane; s < nseg; s += 32) {
+    float l = ml.x != -INFINITY ? exp2f(ml.x - mt) * ml.y : 0.f;
+    for (int s = lane + 32; s < nseg; s += 32) {
       const float ms = A.part_ml[(base0 + s * seg_stride) * 2];
       if (ms != -INFINITY) l += exp2f(ms - mt) * A.part_ml[(base0 + s * seg_stride) * 2 + 1];
     }
     l = warp_sum(l);
     const float inv = l > 0.f ? 1.f / l : 0.f;
-    const int c4 = lane;
-    if (c4 * 4 < hd) {
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-      for (int s = 0; s < nseg; ++s) {
+    const float w_lane = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mt);      // weight of segment `lane`
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int s = 0; s < NPRE; ++s) {
+      const float w = __shfl_sync(0xffffffffu, w_lane, s);
+      if (s < nseg && w != 0.f) { acc.x += w * pre[s].x; acc.y += w * pre[s].y; acc.z += w * pre[s].z; acc.w += w * pre[s].w; }
+    }
+    for (int s = NPRE; s < nseg; ++s) {
+      float w;
+      if (s < 32) {
+        w = __shfl_sync(0xffffffffu, w_lane, s);
+      } else {
         const float ms = A.part_ml[(base0 + s * seg_stride) * 2];
-        const float w = ms == -INFINITY ? 0.f : exp2f(ms - mt);
-        const float4 ov = reinterpret_cast<const float4 *>(A.part_o + (base0 + s * seg_stride) * hd)[c4];
-        if (w != 0.f) { acc.x += w * ov.x; acc.y += w * ov.y; acc.z += w * ov.z; acc.w += w * ov.w; }
+        w = ms == -INFINITY ? 0.f : exp2f(ms - mt);
       }
+      if (c4 * 4 < hd && w != 0.f) {
+        const float4 ov = reinterpret_cast<const float4 *>(A.part_o + (base0 + s * seg_stride) * hd)[c4];
+        acc.x += w * ov.x; acc.y += w * ov.y; acc.z += w * ov.z; acc.w += w * ov.w;
+      }
+    }
+    if (c4 * 4 < hd) {
       const int j = row / A.group, g = row % A.group;
       __nv_bfloat16 *dst = A.out + (static_cast<size_t>(b) * A.QT + j) * (A.n_kv * A.group * hd) +
                            (static_cast<size_t>(head) * A.group + g) * hd + c4 * 4;
