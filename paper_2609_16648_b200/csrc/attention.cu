@@ -76,6 +76,12 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int B = A.batch;
+  // barrier set-up touches shared memory only: it runs before the wait for the previous kernel
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < nstages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], hpc); }
+    mbar_fence_init();
+  }
+  __syncthreads();
   pdl_prologue();
   const long long P = A.page_start[B];
   // never more ranges than pages: every active CTA then owns at least one page, so the CTAs that hold
@@ -84,12 +90,6 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
   if (static_cast<long long>(blockIdx.x) >= G) return;
   const int lo = static_cast<int>(blockIdx.x * P / G), hi = static_cast<int>((blockIdx.x + 1) * P / G);
   const int hg = blockIdx.y;                    // head group (n_kv > 8)
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < nstages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], hpc); }
-    mbar_fence_init();
-  }
-  __syncthreads();
   if (lo >= hi) return;
 
   // first sequence of the range: largest b with page_start[b] <= lo
@@ -341,18 +341,17 @@ attention_t_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int B = A.batch;
+  if (threadIdx.x == 0) {                       // shared memory only: before the wait for the previous kernel
+    for (int s = 0; s < nstages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], hpc); }
+    mbar_fence_init();
+  }
+  __syncthreads();
   pdl_prologue();
   const long long P = A.page_start[B];
   const long long G = P < static_cast<long long>(gridDim.x) ? P : static_cast<long long>(gridDim.x);
   if (static_cast<long long>(blockIdx.x) >= G) return;
   const int lo = static_cast<int>(blockIdx.x * P / G), hi = static_cast<int>((blockIdx.x + 1) * P / G);
   const int hg = blockIdx.y;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < nstages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], hpc); }
-    mbar_fence_init();
-  }
-  __syncthreads();
   if (lo >= hi) return;
 
   int b0 = 0;

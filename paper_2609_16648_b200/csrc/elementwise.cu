@@ -29,20 +29,24 @@ __device__ __forceinline__ float block_sum(float v) {
 __device__ __forceinline__ void rmsnorm_store(const float4 (&v)[EW_MAXC], int d4, int d, float eps,
                                               const __nv_bfloat16 *w, __nv_bfloat16 *out) {
   float ss = 0.f;
+  uint2 wv[EW_MAXC];                         // the weights are requested before the reduction: their latency hides behind it
 #pragma unroll
   for (int c = 0; c < EW_MAXC; ++c) {
     const int i = threadIdx.x + c * EW_THREADS;
-    if (i < d4) ss += v[c].x * v[c].x + v[c].y * v[c].y + v[c].z * v[c].z + v[c].w * v[c].w;
+    wv[c] = make_uint2(0u, 0u);
+    if (i < d4) {
+      wv[c] = *reinterpret_cast<const uint2 *>(w + 4 * i);
+      ss += v[c].x * v[c].x + v[c].y * v[c].y + v[c].z * v[c].z + v[c].w * v[c].w;
+    }
   }
   const float inv = rsqrtf(block_sum(ss) / static_cast<float>(d) + eps);
 #pragma unroll
   for (int c = 0; c < EW_MAXC; ++c) {
     const int i = threadIdx.x + c * EW_THREADS;
     if (i < d4) {
-      const uint2 wv = *reinterpret_cast<const uint2 *>(w + 4 * i);
       uint2 o;
-      o.x = pack_bf16(v[c].x * inv * bf16_lo(wv.x), v[c].y * inv * bf16_hi(wv.x));
-      o.y = pack_bf16(v[c].z * inv * bf16_lo(wv.y), v[c].w * inv * bf16_hi(wv.y));
+      o.x = pack_bf16(v[c].x * inv * bf16_lo(wv[c].x), v[c].y * inv * bf16_hi(wv[c].x));
+      o.y = pack_bf16(v[c].z * inv * bf16_lo(wv[c].y), v[c].w * inv * bf16_hi(wv[c].y));
       *reinterpret_cast<uint2 *>(out + 4 * i) = o;
     }
   }
@@ -395,8 +399,22 @@ __global__ void __launch_bounds__(EW_THREADS) rope_append_kernel(const RopeAppen
   const int hd = A.hd, half = hd >> 1, group = A.n_q / A.n_kv;
   const int ncols = (A.n_q + 2 * A.n_kv) * hd;
   pdl_prologue();
+  // Everything that does not depend on another load is requested at once: the query count, the first position and
+  // this thread's first work item of the projection row (the kernel is a chain of latencies, not of bandwidth).
   const int qn = A.qn[b];
+  const int qb = A.qbase[b];
   const int hv = half >> 3;                                       // 8-wide items per half head
+  const __nv_bfloat16 *src = A.qkv + static_cast<size_t>(m) * ncols;
+  const int n_rot = (A.n_q + A.n_kv) * hv, n_v = A.n_kv * (hd >> 3);
+  uint4 first1 = make_uint4(0u, 0u, 0u, 0u), first2 = first1;
+  if (static_cast<int>(threadIdx.x) < n_rot) {
+    const int h = threadIdx.x / hv, e = (threadIdx.x % hv) * 8;
+    first1 = *reinterpret_cast<const uint4 *>(src + h * hd + e);
+    first2 = *reinterpret_cast<const uint4 *>(src + h * hd + e + half);
+  } else if (static_cast<int>(threadIdx.x) < n_rot + n_v) {
+    const int iv = threadIdx.x - n_rot, h = iv / (hd >> 3), e = (iv % (hd >> 3)) * 8;
+    first1 = *reinterpret_cast<const uint4 *>(src + (A.n_q + A.n_kv) * hd + h * hd + e);
+  }
   __nv_bfloat16 *qdst = A.qbuf + static_cast<size_t>(b) * A.n_kv * A.qrows * hd;
   if (j >= qn) {                           // padding row: zero its query rows, append nothing
     for (int i = threadIdx.x; i < A.n_q * (hd >> 3); i += EW_THREADS) {
@@ -406,17 +424,15 @@ __global__ void __launch_bounds__(EW_THREADS) rope_append_kernel(const RopeAppen
     }
     return;
   }
-  const int pos = A.qbase[b] + j;
+  const int pos = qb + j;
   const int page = A.page_table[static_cast<size_t>(b) * A.max_pages_per_seq + (pos >> 4)];
   const bool page_ok = page >= 0 && page < A.num_pages;
   if (!page_ok && threadIdx.x == 0) set_status(A.status, ST_BAD_PAGE);
-  const __nv_bfloat16 *src = A.qkv + static_cast<size_t>(m) * ncols;
   const float2 *cs = A.rope + static_cast<size_t>(pos) * half;
   const size_t page_elems = static_cast<size_t>(A.n_kv) * 16 * hd;
   __nv_bfloat16 *kdst = A.pool + ((static_cast<size_t>(A.layer) * 2 + 0) * A.num_pages + (page_ok ? page : 0)) * page_elems;
   __nv_bfloat16 *vdst = A.pool + ((static_cast<size_t>(A.layer) * 2 + 1) * A.num_pages + (page_ok ? page : 0)) * page_elems;
   const int slot = pos & 15;
-  const int n_rot = (A.n_q + A.n_kv) * hv, n_v = A.n_kv * (hd >> 3);
   // the hv lanes that share one head are consecutive and aligned (hv is a power of two <= 32)
   const unsigned lane = threadIdx.x & 31u;
   const unsigned head_lanes = hv >= 32 ? 0xffffffffu : ((1u << hv) - 1u) << (lane & ~static_cast<unsigned>(hv - 1));
@@ -424,8 +440,9 @@ __global__ void __launch_bounds__(EW_THREADS) rope_append_kernel(const RopeAppen
     if (i < n_rot) {
       const int h = i / hv, e = (i % hv) * 8;
       float x1[8], x2[8], y1[8], y2[8];
-      unpack8f(*reinterpret_cast<const uint4 *>(src + h * hd + e), x1);
-      unpack8f(*reinterpret_cast<const uint4 *>(src + h * hd + e + half), x2);
+      const bool is_first = i == static_cast<int>(threadIdx.x);
+      unpack8f(is_first ? first1 : *reinterpret_cast<const uint4 *>(src + h * hd + e), x1);
+      unpack8f(is_first ? first2 : *reinterpret_cast<const uint4 *>(src + h * hd + e + half), x2);
       if (A.bias) {
         float b1[8], b2[8];
         unpack8f(*reinterpret_cast<const uint4 *>(A.bias + h * hd + e), b1);
@@ -460,7 +477,8 @@ __global__ void __launch_bounds__(EW_THREADS) rope_append_kernel(const RopeAppen
       *reinterpret_cast<uint4 *>(dst + e + half) = pack8f(y2);
     } else if (page_ok) {
       const int iv = i - n_rot, h = iv / (hd >> 3), e = (iv % (hd >> 3)) * 8;
-      uint4 val = *reinterpret_cast<const uint4 *>(src + (A.n_q + A.n_kv) * hd + h * hd + e);
+      uint4 val = i == static_cast<int>(threadIdx.x) ? first1
+                                                     : *reinterpret_cast<const uint4 *>(src + (A.n_q + A.n_kv) * hd + h * hd + e);
       if (A.bias) {
         float x[8], bv[8];
         unpack8f(val, x);
