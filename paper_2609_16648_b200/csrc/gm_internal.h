@@ -67,7 +67,7 @@ struct gm_ctx {
   __nv_bfloat16 *pf_hidden = nullptr;
   float *pf_xlast = nullptr;
   int32_t *ro_accept = nullptr, *ro_next = nullptr;   // per-step outputs of a rollout step
-  // captured rollout cycle (GM_FLAG_ROLLOUT_GRAPH)
+  // captured cycles (GM_FLAG_GRAPH)
   uint64_t *dev_step = nullptr;             // step index of the captured cycle
   uint64_t *step_ptr = nullptr;             // non-null while a cycle is being captured: kernels read the step from here
   struct GraphSlot {                        // one captured sequence of launches and what it was captured for
