@@ -35,6 +35,27 @@ def test_error_strings_and_null_handling_need_no_gpu():
     out = ctypes.c_void_p()
     assert L.gm_init(ctypes.byref(out), None, None, None) == gmb.GM_ERR_INVALID_ARG
     L.gm_destroy(None)
+    # every entry point checks its context before anything else: a null context is an argument error, not a crash
+    inv = gmb.GM_ERR_INVALID_ARG
+    assert L.gm_draft(None, None, 3, 1.0, None, 0, 0, None, None, None) == inv
+    assert L.gm_verify(None, None, 3, None, None, None) == inv
+    assert L.gm_accept(None, None, 1, 3, 1.0, None, None, None, None, 0, 0, None, None, None, None, None, 0) == inv
+    assert L.gm_spec_step(None, None, 3, 1.0, 0, 0, None, None, None) == inv
+    assert L.gm_prefill(None, None, None, None, 0, 0, 1.0, None, 0, None, None) == inv
+    assert L.gm_set_top_p(None, 0.7) == inv
+    assert L.gm_nucleus(None, None, 1, 1.0, 0.7, None, None) == inv
+    assert L.gm_capture_hidden(None, None, 0) == inv
+    assert L.gm_head_prefill(None, None, None, 0, None, 0, None, 0) == inv
+    assert L.gm_reconstruct(None, None, 1, 3, None, None, None, 0, None, None) == inv
+    assert L.gm_overlap(None, 1, 3, 1.0, None, None, None) == inv
+    assert L.gm_dca_loss(None, 1, 3, None, None, None, None) == inv
+    assert L.gm_rollout_begin(None, None, None) == inv
+    assert L.gm_rollout_step(None, None, None, 3, 1.0, 0, 0) == inv
+    assert L.gm_rollout_run(None, None, None, 3, 1.0, 0, 0, 1, 1, None, None) == inv
+    assert L.gm_pages_reset(None, None) == inv
+    assert L.gm_pages_reserve(None, None, None, 1, None) == inv
+    assert L.gm_pages_release(None, None, None) == inv
+    assert L.gm_pages_free_count(None, None, None) == inv
 
 
 def test_product_path_does_not_import_the_oracle():
