@@ -401,9 +401,11 @@ def run_product(args):
     barrier()
     t0 = time.perf_counter()
     committed_e2e = 0
+    accept_hist = np.zeros(K + 1, np.int64)                # accepted lengths seen on the host (free: they arrive anyway)
     for i in range(S):
         gmb.gm_spec_step_host(ctx, st, K, 1.0, seed, step_id + 1 + i, a_h, t_h, d_h, ud_h, ua_h)
         committed_e2e += int(a_h.sum()) + B
+        accept_hist += np.bincount(a_h.numpy(), minlength=K + 1)[:K + 1]
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
     h2d = int(ud_h.numel() + ua_h.numel()) * 4
@@ -427,7 +429,11 @@ def run_product(args):
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "n_layers": cfg.n_layers, "batch_per_gpu": B, "k": K, "temperature": 1.0,
                        "top_p": args.top_p, "kv_len_mean": float(lens.mean()), "kv_len_min": int(lens.min()), "kv_len_max": int(lens.max()),
-                       "page": 16, "tau": committed / (S * B), "parallelism": f"replicas x{world}",
+                       "page": 16, "tau": committed / (S * B),
+                       # per-position acceptance alpha_k = P(draft k accepted | drafts 1..k-1 accepted), rank 0, e2e region
+                       "accept_by_position": [float(accept_hist[k:].sum() / max(accept_hist[k - 1:].sum(), 1))
+                                              for k in range(1, K + 1)],
+                       "parallelism": f"replicas x{world}",
                        "l2": "per-step working set (weights + KV, tens of GB) >> 126 MB L2: no flush needed",
                        "step_algorithmic_GB": step_bytes / 1e9, "step_roofline_ms": step_roof_ms,
                        "step_roofline_frac": step_roof_ms / (ms / S), "peaks": which},

@@ -406,7 +406,9 @@ int gm_attention_noalloc(int n_q_heads, int n_kv_heads, int head_dim, int max_pa
 /* Kernel-class timing.  gm_profile(ctx, mask) makes later calls bracket every launch of the
  * selected classes with CUDA events on the context's stream; gm_profile_read waits for the
  * stream and returns the accumulated device time and launch count of one class since the
- * last gm_profile call.                                                                     */
+ * last gm_profile call.  Independently of that, with the environment variable GM_NVTX set,
+ * gm_draft, gm_verify, gm_accept, gm_prefill, gm_head_prefill, gm_rollout_step and
+ * gm_reconstruct are wrapped in NVTX ranges of the same names.                              */
 #define GM_KC_GEMM       0
 #define GM_KC_ATTENTION  1
 #define GM_KC_ELEMENTWISE 2

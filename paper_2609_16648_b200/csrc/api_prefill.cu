@@ -7,6 +7,7 @@ extern "C" {
 int gm_prefill(gm_ctx *c, gm_state *st, const int32_t *prompt_tok, const int32_t *prompt_len, int prompt_stride,
                int max_prompt_len, float temperature, const uint32_t *u24_first, uint64_t seed, int32_t *first_token,
                float *dbg_p) {
+  NvtxRange nvtx_range("gm_prefill");
   int rc = check_state(c, st, 1);
   if (rc) return rc;
   if (!prompt_tok || !prompt_len || max_prompt_len < 1 || prompt_stride < max_prompt_len) return GM_ERR_INVALID_ARG;
@@ -94,6 +95,7 @@ int gm_prefill(gm_ctx *c, gm_state *st, const int32_t *prompt_tok, const int32_t
 // ---- forward pass of the head update on recorded cycles -------------------------------------------------------------
 int gm_head_prefill(gm_ctx *c, gm_state *st, const void *seq_hidden, int hid_stride, const int32_t *seq_tok,
                     int tok_stride, const int32_t *seq_len, int max_len) {
+  NvtxRange nvtx_range("gm_head_prefill");
   int rc = check_state(c, st, 1);
   if (rc) return rc;
   if (!seq_hidden || !seq_tok || !seq_len || max_len < 1 || tok_stride < max_len || hid_stride < max_len - 1)

@@ -91,6 +91,7 @@ int gm_rollout_begin(gm_ctx *c, const gm_state *st, const gm_rollout *ro) {
 }
 
 int gm_rollout_step(gm_ctx *c, gm_state *st, const gm_rollout *ro, int k, float temperature, uint64_t seed, uint64_t step) {
+  NvtxRange nvtx_range("gm_rollout_step");
   int rc = rollout_args_ok(c, st, ro);
   if (rc) return rc;
   if ((rc = check_state(c, st, k)) != GM_OK) return rc;

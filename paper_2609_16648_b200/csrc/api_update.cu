@@ -13,6 +13,7 @@ int gm_capture_hidden(gm_ctx *c, void *seq_hidden, int stride) {
 
 int gm_reconstruct(gm_ctx *c, gm_state *st, int n_cycles, int k, const int32_t *cycle_seq, const gm_record *rec,
                    const int32_t *seq_tok, int tok_stride, const int32_t *scratch_pages, void *draft_logits) {
+  NvtxRange nvtx_range("gm_reconstruct");
   int rc = check_state(c, st, k);
   if (rc) return rc;
   if (n_cycles < 1 || !cycle_seq || !rec || !rec->start_hidden || !rec->start_pos || !rec->drafts || !seq_tok ||

@@ -405,6 +405,7 @@ int gm_draft(gm_ctx *c, const gm_state *st, int k, float temperature, const uint
 
 int gmh::draft_impl(gm_ctx *c, const gm_state *st, int k, float temperature, const uint32_t *u24_draft, uint64_t seed,
                     uint64_t step, int32_t *draft_tok, void *draft_logits, float *dbg_q, bool forced) {
+  NvtxRange nvtx_range("gm_draft");
   int rc = check_state(c, st, k);
   if (rc) return rc;
   if (!draft_tok || !draft_logits) return GM_ERR_INVALID_ARG;
@@ -458,6 +459,7 @@ extern "C" {
 
 int gm_verify(gm_ctx *c, const gm_state *st, int k, const int32_t *draft_tok, void *target_logits,
               void *target_hidden) {
+  NvtxRange nvtx_range("gm_verify");
   int rc = check_state(c, st, k);
   if (rc) return rc;
   if (!draft_tok || !target_logits || !target_hidden) return GM_ERR_INVALID_ARG;
@@ -487,6 +489,7 @@ int gm_accept(gm_ctx *c, gm_state *st, int batch, int k, float temperature, cons
               const void *draft_logits, const int32_t *draft_tok, const uint32_t *u24_accept, uint64_t seed,
               uint64_t step, int32_t *accept_len, int32_t *next_token, float *dbg_p, float *dbg_q,
               const void *target_hidden, int commit_state) {
+  NvtxRange nvtx_range("gm_accept");
   if (!c || !target_logits || !draft_logits || !draft_tok || !accept_len || !next_token) return GM_ERR_INVALID_ARG;
   if (k < 1 || batch < 1) return GM_ERR_INVALID_ARG;
   if (k > GM_MAX_K) return GM_ERR_UNSUPPORTED;

@@ -12,6 +12,7 @@
 #include <vector>
 
 #include <cudaTypedefs.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include "../../include/gm.h"
 #include "common.cuh"
@@ -144,6 +145,17 @@ struct Prof {
     }                                       \
   } while (0)
 
+
+// NVTX range around an entry point (GM_NVTX=1): lets a profiler group the launches of a phase.  Off by default.
+struct NvtxRange {
+  bool on;
+  explicit NvtxRange(const char *name) : on(enabled()) { if (on) nvtxRangePushA(name); }
+  ~NvtxRange() { if (on) nvtxRangePop(); }
+  static bool enabled() {
+    static const bool e = std::getenv("GM_NVTX") != nullptr;
+    return e;
+  }
+};
 
 // ---- host helpers shared by the api_*.cu files (defined in gm_api.cu) -------------------------------------------------
 int make_map(gm_ctx *c, CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t cols, uint32_t box_rows);
