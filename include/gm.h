@@ -52,6 +52,7 @@ extern "C" {
 #define GM_ERR_BAD_PAGE      (-6)   /* a page id outside the pool (device-seen)                 */
 #define GM_ERR_NO_EXTENSION  (-7)   /* not an sm_100 device                                     */
 #define GM_ERR_SCRATCH_LIMIT (-8)   /* request larger than the static scratch of a no-alloc call */
+#define GM_ERR_OVERRUN       (-9)   /* a guard word behind a library workspace was overwritten   */
 
 #define GM_MAX_K 7
 #define GM_PAGE  16
@@ -402,6 +403,10 @@ int gm_attention_noalloc(int n_q_heads, int n_kv_heads, int head_dim, int max_pa
                          const void *kv_pool, int pool_layers, int num_pages, int layer,
                          const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch,
                          int q_stride, void *out, void *cuda_stream);
+
+/* Guard words (a stand-in for a memory checker): every workspace the library allocates is followed by 256
+ * bytes of a fixed pattern.  With the environment variable GM_CANARY set when the context is created,
+ * gm_last_status also reads the guards back and returns GM_ERR_OVERRUN if any byte changed.             */
 
 /* Kernel-class timing.  gm_profile(ctx, mask) makes later calls bracket every launch of the
  * selected classes with CUDA events on the context's stream; gm_profile_read waits for the

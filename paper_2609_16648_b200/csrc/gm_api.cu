@@ -248,6 +248,7 @@ const char *gm_strerror(int code) {
     case GM_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
     case GM_ERR_BAD_PAGE: return "page id or token id outside its range";
     case GM_ERR_NO_EXTENSION: return "no sm_100 device";
+    case GM_ERR_OVERRUN: return "a guard word behind a library workspace was overwritten";
     case GM_ERR_SCRATCH_LIMIT: return "request exceeds the static scratch of the no-alloc entry point (see GM_NOALLOC_SCRATCH_BYTES)";
     default: return "unknown error";
   }
@@ -281,6 +282,7 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
   c->layers.assign(w->layers, w->layers + cfg->n_layers);
   c->w.layers = c->layers.data();
   c->stream = static_cast<cudaStream_t>(cuda_stream);
+  c->check_guards = std::getenv("GM_CANARY") != nullptr;
   cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev);
   c->d = cfg->d_model; c->q_dim = cfg->n_q_heads * cfg->head_dim; c->kv_dim = cfg->n_kv_heads * cfg->head_dim;
   c->n_qkv = c->q_dim + 2 * c->kv_dim; c->F = cfg->d_ffn; c->V = cfg->vocab; c->group = group;
@@ -641,6 +643,14 @@ int gm_last_status(gm_ctx *c) {
   if (s & ST_TIMEOUT) return GM_ERR_DEVICE_TIMEOUT;
   if (s & ST_KV_CAPACITY) return GM_ERR_KV_CAPACITY;
   if (s & (ST_BAD_PAGE | ST_BAD_TOKEN)) return GM_ERR_BAD_PAGE;
+  if (c->check_guards) {
+    unsigned char host[GM_GUARD_BYTES];
+    for (unsigned char *g : c->guards) {
+      GM_CUDA(c, cudaMemcpy(host, g, GM_GUARD_BYTES, cudaMemcpyDeviceToHost));
+      for (size_t i = 0; i < GM_GUARD_BYTES; ++i)
+        if (host[i] != GM_GUARD_PATTERN) return GM_ERR_OVERRUN;
+    }
+  }
   return GM_OK;
 }
 

@@ -88,6 +88,8 @@ struct gm_ctx {
   float top_p = 1.f;                    // nucleus of the target distributions (1 = none)
   __nv_bfloat16 *ws_nucleus = nullptr;  // [max_batch (max_k + 1)][V] filtered target rows, allocated by gm_set_top_p
   std::vector<void *> allocs;
+  std::vector<unsigned char *> guards;      // 256 guard bytes behind every workspace
+  bool check_guards = false;                // GM_CANARY: gm_last_status verifies them
 
   // profiling
   int prof_mask = 0;
@@ -105,11 +107,18 @@ namespace gmh {
     if (e__ != cudaSuccess) { (ctx)->last_cuda = e__; return GM_ERR_CUDA; } \
   } while (0)
 
+constexpr size_t GM_GUARD_BYTES = 256;
+constexpr int GM_GUARD_PATTERN = 0xA5;
+
 template <typename T>
 int dev_alloc(gm_ctx *c, T **p, size_t n, bool zero = true) {
   void *q = nullptr;
-  GM_CUDA(c, cudaMalloc(&q, n * sizeof(T) > 0 ? n * sizeof(T) : 16));
+  const size_t bytes = ((n * sizeof(T) > 0 ? n * sizeof(T) : 16) + 255) & ~static_cast<size_t>(255);
+  GM_CUDA(c, cudaMalloc(&q, bytes + GM_GUARD_BYTES));
   c->allocs.push_back(q);
+  unsigned char *guard = static_cast<unsigned char *>(q) + bytes;
+  GM_CUDA(c, cudaMemsetAsync(guard, GM_GUARD_PATTERN, GM_GUARD_BYTES, c->stream));
+  c->guards.push_back(guard);
   if (zero) GM_CUDA(c, cudaMemsetAsync(q, 0, n * sizeof(T), c->stream));
   *p = static_cast<T *>(q);
   return GM_OK;

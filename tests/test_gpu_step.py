@@ -348,3 +348,30 @@ def test_graph_replayed_cycle_equals_host_launched_cycle():
     np.testing.assert_array_equal(h0[1], h1[1])
     assert torch.equal(h0[2], h1[2]) and torch.equal(h0[3], h1[3])
     assert h1[4] == h0[4] + 12                                     # the same kernels + one step-index store per replay
+
+
+def test_guard_words_behind_the_workspaces_stay_intact(monkeypatch):
+    """With GM_CANARY set the library checks the 256 guard bytes behind each of its workspaces whenever the status is
+    read: prefill, cycles at the largest depth, top-p, record and rollout bookkeeping leave all of them untouched."""
+    import paper_2609_16648_b200 as gmb
+    monkeypatch.setenv("GM_CANARY", "1")
+    cfg = get_config("tiny").with_(k=7, prompt_len=30)
+    K, B = cfg.k, cfg.batch
+    w, ost, ctx, gst = tiny_setup(cfg, cap_tokens=30 + 8 * (K + 1) + 8)
+    assert gmb.gm_last_status(ctx) == 0
+    prompts = np.array([s.tokens[:30] for s in ost.seqs], np.int32)
+    gmb.gm_prefill(ctx, gst, torch.from_numpy(prompts).cuda(), torch.full((B,), 30, dtype=torch.int32, device="cuda"), 30, 1.0,
+                   None, 5)
+    assert gmb.gm_last_status(ctx) == 0
+    gmb.gm_set_top_p(ctx, 0.8)
+    rec = gmb.Record(B, K, cfg.d_model)
+    a = torch.zeros(B, dtype=torch.int32, device="cuda")
+    t = torch.zeros(B, dtype=torch.int32, device="cuda")
+    d = torch.zeros((B, K), dtype=torch.int32, device="cuda")
+    for it in range(3):
+        gmb.gm_spec_step_rec(ctx, gst, K, 1.0, 5, 1 + it, a, t, d, rec)
+    ro = gmb.Rollout(B, 12, -1)
+    gmb.gm_rollout_begin(ctx, gst, ro)
+    gmb.gm_rollout_run(ctx, gst, ro, K, 1.0, 5, 10, 3, 1)
+    assert gmb.gm_last_status(ctx) == 0
+    ctx.close()
