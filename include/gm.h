@@ -202,8 +202,9 @@ int gm_rollout_run(gm_ctx *ctx, gm_state *st, const gm_rollout *ro, int k, float
  *                     gm_last_status;
  *   gm_pages_release  rows with finished[b] != 0 hand their pages back;
  *   gm_pages_free_count  free pages per pool (host outputs; synchronises the stream).
- * One thread walks the rows in order, so page assignment is the same on every run.  A context serves one
- * state at a time while the allocator is on.                                                            */
+ * Rows take their slices of the stack in row order (a prefix sum over the rows), so the page assignment
+ * is the same on every run.  Batches of at most 1024 rows.  A context serves one state at a time while
+ * the allocator is on.                                                                                  */
 int gm_pages_reset(gm_ctx *ctx, gm_state *st);
 int gm_pages_reserve(gm_ctx *ctx, gm_state *st, const int32_t *length, int extra, const int32_t *finished);
 int gm_pages_release(gm_ctx *ctx, gm_state *st, const int32_t *finished);

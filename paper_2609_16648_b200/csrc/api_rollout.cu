@@ -41,24 +41,24 @@ int gm_pages_reset(gm_ctx *c, gm_state *st) {
 int gm_pages_reserve(gm_ctx *c, gm_state *st, const int32_t *length, int extra, const int32_t *finished) {
   if (!c || !st || extra < 0) return GM_ERR_INVALID_ARG;
   if (!c->alloc_on) return GM_ERR_INVALID_ARG;
+  PageAllocArgs P[2];
   for (int pool = 0; pool < 2; ++pool) {
-    PageAllocArgs P;
-    fill_alloc(c, st, pool, P);
-    P.length = length ? length : st->kv_len; P.extra = extra; P.finished = finished;
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_page_reserve(P, c->stream));
+    fill_alloc(c, st, pool, P[pool]);
+    P[pool].length = length ? length : st->kv_len; P[pool].extra = extra; P[pool].finished = finished;
   }
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_page_reserve(P[0], P[1], c->stream));
   return GM_OK;
 }
 
 int gm_pages_release(gm_ctx *c, gm_state *st, const int32_t *finished) {
   if (!c || !st || !finished) return GM_ERR_INVALID_ARG;
   if (!c->alloc_on) return GM_ERR_INVALID_ARG;
+  PageAllocArgs P[2];
   for (int pool = 0; pool < 2; ++pool) {
-    PageAllocArgs P;
-    fill_alloc(c, st, pool, P);
-    P.finished = finished;
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_page_release(P, c->stream));
+    fill_alloc(c, st, pool, P[pool]);
+    P[pool].finished = finished;
   }
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_page_release(P[0], P[1], c->stream));
   return GM_OK;
 }
 

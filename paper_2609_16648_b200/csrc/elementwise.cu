@@ -147,43 +147,76 @@ __global__ void page_reset_kernel(const PageAllocArgs A) {
 cudaError_t launch_page_reset(const PageAllocArgs &A, cudaStream_t stream) {
   return launch_k(page_reset_kernel, dim3(64), dim3(256), 0, stream, 1, A);
 }
-__global__ void page_reserve_kernel(const PageAllocArgs A) {
+// Reserve / release for both pools in one launch (block p = pool p), one thread per row.  A block-wide exclusive prefix
+// sum of the rows' page counts gives every row its slice of the free stack, which is exactly the slice the rows would
+// get one after the other: the assignment does not depend on thread scheduling.
+__device__ __forceinline__ int block_exclusive_scan_1024(int v, int *total) {
+  __shared__ int warp_tot[32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+  for (int o = 1; o < 32; o <<= 1) {
+    const int up = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += up;
+  }
+  __syncthreads();                                   // warp_tot may still be read from a previous call
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  int before = 0, all = 0;
+  for (int w = 0; w < static_cast<int>(blockDim.x >> 5); ++w) {
+    const int t = warp_tot[w];
+    if (w < warp) before += t;
+    all += t;
+  }
+  *total = all;
+  return before + incl - v;
+}
+__global__ void __launch_bounds__(1024) page_reserve_kernel(const PageAllocArgs A0, const PageAllocArgs A1) {
+  const PageAllocArgs &A = blockIdx.x == 0 ? A0 : A1;
   pdl_prologue();
-  if (threadIdx.x != 0) return;
-  int top = *A.free_top;
-  for (int b = 0; b < A.batch; ++b) {
-    if (A.finished && A.finished[b]) continue;
+  const int b = threadIdx.x;
+  int have = 0, want = 0;
+  if (b < A.batch && !(A.finished && A.finished[b])) {
     const int need = (A.length[b] + A.extra + 15) >> 4;
-    int have = A.held[b];
-    if (need > A.max_pages_per_seq) { set_status(A.status, ST_KV_CAPACITY); continue; }
-    while (have < need) {
-      if (top <= 0) { set_status(A.status, ST_KV_CAPACITY); break; }
-      A.page_table[static_cast<size_t>(b) * A.max_pages_per_seq + have++] = A.free_list[--top];
-    }
-    A.held[b] = have;
+    have = A.held[b];
+    if (need > A.max_pages_per_seq) set_status(A.status, ST_KV_CAPACITY);
+    else want = max(need - have, 0);
   }
-  *A.free_top = top;
+  int total = 0;
+  const int off = block_exclusive_scan_1024(want, &total);
+  const int top = *A.free_top;
+  const int grant = min(want, max(top - off, 0));
+  if (grant < want) set_status(A.status, ST_KV_CAPACITY);      // the stack ran out
+  for (int i = 0; i < grant; ++i)
+    A.page_table[static_cast<size_t>(b) * A.max_pages_per_seq + have + i] = A.free_list[top - 1 - (off + i)];
+  if (b < A.batch && grant > 0) A.held[b] = have + grant;
+  __syncthreads();                                   // every thread has read free_top
+  if (threadIdx.x == 0) *A.free_top = top - min(total, top);
 }
-cudaError_t launch_page_reserve(const PageAllocArgs &A, cudaStream_t stream) {
-  return launch_k(page_reserve_kernel, dim3(1), dim3(32), 0, stream, 1, A);
+cudaError_t launch_page_reserve(const PageAllocArgs &A0, const PageAllocArgs &A1, cudaStream_t stream) {
+  if (A0.batch > 1024 || A1.batch > 1024) return cudaErrorInvalidValue;
+  return launch_k(page_reserve_kernel, dim3(2), dim3(1024), 0, stream, 1, A0, A1);
 }
-__global__ void page_release_kernel(const PageAllocArgs A) {
+__global__ void __launch_bounds__(1024) page_release_kernel(const PageAllocArgs A0, const PageAllocArgs A1) {
+  const PageAllocArgs &A = blockIdx.x == 0 ? A0 : A1;
   pdl_prologue();
-  if (threadIdx.x != 0) return;
-  int top = *A.free_top;
-  for (int b = 0; b < A.batch; ++b) {
-    if (!A.finished[b]) continue;
-    int32_t *row = A.page_table + static_cast<size_t>(b) * A.max_pages_per_seq;
-    for (int i = A.held[b] - 1; i >= 0; --i) {
-      if (top < A.num_pages) A.free_list[top++] = row[i];
-      row[i] = -1;
-    }
-    A.held[b] = 0;
+  const int b = threadIdx.x;
+  const int n = (b < A.batch && A.finished[b]) ? A.held[b] : 0;
+  int total = 0;
+  const int off = block_exclusive_scan_1024(n, &total);
+  const int top = *A.free_top;
+  int32_t *row = A.page_table + static_cast<size_t>(b < A.batch ? b : 0) * A.max_pages_per_seq;
+  for (int k = 0; k < n; ++k) {                       // the row's pages go back last-reserved first
+    const int i = n - 1 - k;
+    if (top + off + k < A.num_pages) A.free_list[top + off + k] = row[i];
+    row[i] = -1;
   }
-  *A.free_top = top;
+  if (n > 0) A.held[b] = 0;
+  __syncthreads();
+  if (threadIdx.x == 0) *A.free_top = min(top + total, A.num_pages);
 }
-cudaError_t launch_page_release(const PageAllocArgs &A, cudaStream_t stream) {
-  return launch_k(page_release_kernel, dim3(1), dim3(32), 0, stream, 1, A);
+cudaError_t launch_page_release(const PageAllocArgs &A0, const PageAllocArgs &A1, cudaStream_t stream) {
+  if (A0.batch > 1024 || A1.batch > 1024) return cudaErrorInvalidValue;
+  return launch_k(page_release_kernel, dim3(2), dim3(1024), 0, stream, 1, A0, A1);
 }
 
 // ---- prompt prefill: chunk bookkeeping ----------------------------------------------------------------------

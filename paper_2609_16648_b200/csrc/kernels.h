@@ -159,7 +159,8 @@ cudaError_t launch_rollout_append(const RolloutArgs &A, bool begin, cudaStream_t
 cudaError_t launch_set_step(uint64_t *dst, uint64_t value, cudaStream_t stream);      // *dst = value
 // Page allocator: a stack of free page ids per pool.  reserve: every running row gets pages until its table covers
 // length[b] + extra positions (ST_KV_CAPACITY when the stack or the table row runs out); release: the pages of
-// finished rows go back on the stack.  One thread walks the rows in order, so the assignment is deterministic.
+// finished rows go back on the stack.  A row's slice of the stack comes from a prefix sum over the rows in order, so the
+// assignment is the one a sequential walk would make and does not depend on scheduling.
 struct PageAllocArgs {
   int batch, max_pages_per_seq, num_pages, extra;
   const int32_t *length, *finished;     // finished may be null
@@ -167,8 +168,8 @@ struct PageAllocArgs {
   uint32_t *status;
 };
 cudaError_t launch_page_reset(const PageAllocArgs &A, cudaStream_t stream);
-cudaError_t launch_page_reserve(const PageAllocArgs &A, cudaStream_t stream);
-cudaError_t launch_page_release(const PageAllocArgs &A, cudaStream_t stream);
+cudaError_t launch_page_reserve(const PageAllocArgs &target, const PageAllocArgs &head, cudaStream_t stream);   // both pools
+cudaError_t launch_page_release(const PageAllocArgs &target, const PageAllocArgs &head, cudaStream_t stream);
 
 // ---- forward pass of the head update on recorded cycles ---------------------------------------------------
 // A chain = a virtual sequence: shared head-cache pages of its sequence before the page of its first entry, two
