@@ -12,6 +12,12 @@ Objective.  alpha_k = sum_d min(p_k(d), q_k(d)) (Eq. 5), estimated from the reco
 log-probabilities plus one residual bin (App. D.2); the chain surrogate -sum_l prod_{i<=l} alpha_i (Eq. 6),
 its logarithmic form (Eq. 7) and the truncation of the chain sum at min(j, K), j the first rejected
 position, K+1 if none (Eq. 9).  The update minimises the mean over cycles.
+
+First step of the backward pass: the gradient of that mean with respect to the reconstructed head logits.
+dL/dalpha_k is Eq. 8 with the chain sums cut at min(j, K) (zero beyond the cut).  alpha_k is piecewise linear
+in q_k: on a retained token the slope is 1 where q < p, and the residual bin, q_res = 1 - (sum of q over the
+retained tokens), contributes -1 on every retained token where q_res < p_res; at a tie the slope is taken as 0.
+The chain rule through q = softmax(logits / T) gives dalpha/dlogit_v = q_v (g_v - sum_d q_d g_d) / T.
 """
 from __future__ import annotations
 
@@ -77,6 +83,53 @@ def dca_position_weights(alphas) -> np.ndarray:
         D = sum(np.prod(a[k + 1:l + 1]) for l in range(k, K))
         out[k] = np.prod(a[:k]) * D / (-tv_chain_loss(a))
     return out
+
+
+def softmax64(logits, temperature: float) -> np.ndarray:
+    x = np.asarray(logits, np.float64) / float(temperature)
+    e = np.exp(x - x.max(axis=-1, keepdims=True))
+    return e / e.sum(axis=-1, keepdims=True)
+
+
+def dca_loss_grad_alpha(alphas, j: int | None = None) -> np.ndarray:
+    """dL/dalpha_k of Eq. 9 for one cycle: -(prod_{i<k} alpha_i) D_k / M with M and D_k cut at L = min(j, K);
+    0 for k > L (Eq. 8 with the verify gate)."""
+    a = np.asarray(alphas, np.float64)
+    K = len(a)
+    L = K if j is None else min(int(j), K)
+    M = np.cumprod(a[:L]).sum()
+    g = np.zeros(K)
+    for k in range(L):
+        D = sum(np.prod(a[k + 1:l + 1]) for l in range(k, L))
+        g[k] = -np.prod(a[:k]) * D / M
+    return g
+
+
+def overlap_grad_logits(p_top_idx, p_top_logprob, logits, temperature: float) -> np.ndarray:
+    """dalpha/dlogits [V] of the sparsified overlap (App. D.2) at q = softmax(logits / T)."""
+    q = softmax64(logits, temperature)
+    keep = np.asarray(p_top_idx) >= 0
+    idx = np.asarray(p_top_idx)[keep]
+    p_kept = np.exp(np.asarray(p_top_logprob, np.float64)[keep])
+    q_kept = q[idx]
+    p_res, q_res = max(1.0 - p_kept.sum(), 0.0), max(1.0 - q_kept.sum(), 0.0)
+    g = np.zeros(len(q))
+    g[idx] = (q_kept < p_kept).astype(np.float64) - (1.0 if q_res < p_res else 0.0)
+    return q * (g - float((q * g).sum())) / temperature
+
+
+def head_update_grad_logits(logits, records, temperature: float = 1.0) -> np.ndarray:
+    """d(mean over cycles of Eq. 9)/d(reconstructed logits): logits [n, K, V]; records = the n record dicts."""
+    logits = np.asarray(logits, np.float64)
+    n, K, V = logits.shape
+    out = np.zeros((n, K, V))
+    for r, rec in enumerate(records):
+        q = softmax64(logits[r], temperature)
+        ga = dca_loss_grad_alpha(chain_alphas(rec, q), rec["accepted"])
+        for k in range(K):
+            if ga[k] != 0.0:
+                out[r, k] = ga[k] * overlap_grad_logits(rec["top_index"][k], rec["top_logprob"][k], logits[r, k], temperature)
+    return out / n
 
 
 def head_update_loss(w, cfg, sequences, records, temperature: float = 1.0, round_interface: bool = True):

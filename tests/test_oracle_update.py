@@ -123,3 +123,61 @@ def test_head_update_loss_is_the_mean_over_cycles():
     assert loss == pytest.approx(np.mean(per))
     # a perfect head (q = p) would give alpha = 1 everywhere and loss -log(min(j, K)) per cycle: the bound
     assert loss >= -np.mean([np.log(min(r["accepted"], 3)) for _, r in recs]) - 1e-9
+
+
+def _toy_records(rng, n, K, V, kept, T):
+    """Records over a small vocabulary: `kept` retained target tokens per position (padded with -1 to 64), the
+    rest of the target mass in the residual bin."""
+    recs = []
+    for _ in range(n):
+        p = update.softmax64(rng.normal(0, 2.0, (K + 1, V)), T)
+        idx = np.full((K + 1, 64), -1, np.int64)
+        lp = np.full((K + 1, 64), -np.inf)
+        for k in range(K + 1):
+            top = np.argsort(-p[k])[:kept]
+            idx[k, :kept], lp[k, :kept] = top, np.log(p[k, top])
+        recs.append({"top_index": idx, "top_logprob": lp, "accepted": int(rng.integers(1, K + 2))})
+    return recs
+
+
+def _mean_loss(logits, recs, T):
+    per = []
+    for r, rec in enumerate(recs):
+        a = update.chain_alphas(rec, update.softmax64(logits[r], T))
+        per.append(update.dca_loss(a, rec["accepted"]))
+    return float(np.mean(per))
+
+
+def test_truncated_alpha_gradient_matches_finite_differences_and_eq8():
+    rng = np.random.default_rng(9)
+    for K in (1, 3, 7):
+        a = rng.uniform(0.05, 0.95, K)
+        np.testing.assert_allclose(update.dca_loss_grad_alpha(a), -update.dca_position_weights(a), rtol=1e-12)
+        for j in range(1, K + 2):
+            g = update.dca_loss_grad_alpha(a, j)
+            for k in range(K):
+                e = np.zeros(K)
+                e[k] = 1e-6
+                fd = (update.dca_loss(a + e, j) - update.dca_loss(a - e, j)) / 2e-6
+                assert g[k] == pytest.approx(fd, rel=1e-5, abs=1e-9)
+            assert (g[min(j, K):] == 0).all() and (g[:min(j, K)] < 0).all()      # larger overlap, smaller loss
+
+
+def test_logit_gradient_matches_finite_differences_of_the_objective():
+    """The whole chain record -> overlap with residual bin -> truncated log-domain loss -> mean, differentiated
+    numerically with respect to every reconstructed logit."""
+    rng = np.random.default_rng(3)
+    n, K, V, T = 4, 3, 14, 0.7
+    for kept in (5, 14):                                     # with a residual bin, and with the whole vocabulary retained
+        recs = _toy_records(rng, n, K, V, kept, T)
+        logits = rng.normal(0, 2.0, (n, K, V))
+        g = update.head_update_grad_logits(logits, recs, T)
+        assert np.abs(g.sum(-1)).max() < 1e-12               # softmax: the gradient of a row sums to zero
+        fd = np.zeros_like(g)
+        for i in np.ndindex(n, K, V):
+            e = np.zeros_like(logits)
+            e[i] = 1e-6
+            fd[i] = (_mean_loss(logits + e, recs, T) - _mean_loss(logits - e, recs, T)) / 2e-6
+        np.testing.assert_allclose(g, fd, rtol=2e-5, atol=1e-9)
+        for r, rec in enumerate(recs):                       # positions after the first rejection get no gradient
+            assert (g[r, min(rec["accepted"], K):] == 0).all() and np.abs(g[r, 0]).max() > 0
