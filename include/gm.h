@@ -316,7 +316,8 @@ int gm_spec_step_rec(gm_ctx *ctx, gm_state *st, int k, float temperature, uint64
 
 /* ---- Forward pass of the draft-head update on recorded cycles (Sec. 3.2 Eq. 4; Sec. 3.3-3.4 Eq. 5-9; App. D.2,
  * D.3).  The recorded inputs: per sequence its committed tokens x[0..L-1] and the rollout-time target hidden
- * states H_0..H_{L-2} (H_i produced x_{i+1}); per cycle a gm_record entry.  Forward only: no gradients.
+ * states H_0..H_{L-2} (H_i produced x_{i+1}); per cycle a gm_record entry.  Forward pass, and the gradient of
+ * the objective with respect to the reconstructed logits; the backward pass through the head is not part of it.
  *
  * gm_head_prefill rebuilds the head cache of every sequence from its recorded pairs (H_{i-1}, x_i),
  *   i = 1..L_b-1, at head positions 0..L_b-2 (the shared prefix every chain attends).
@@ -335,11 +336,21 @@ int gm_spec_step_rec(gm_ctx *ctx, gm_state *st, int k, float temperature, uint64
  *
  * gm_overlap: alpha[r, j] = sum over the record's 64 retained tokens of min(p, q) + min(1 - sum p, 1 - sum q)
  *   (Eq. 5 on the sparsified record, App. D.2), q = softmax(draft_logits / T) over the full vocabulary.
- *   alpha fp32 [n_cycles, k] out.
+ *   alpha fp32 [n_cycles, k] out.  lse fp32 [n_cycles, k] out, or NULL: logsumexp(draft_logits / T) of every
+ *   row, which gm_dca_grad takes back to skip its own statistics pass.
  *
  * gm_dca_loss: loss[r] = -log sum_{l=1..min(accepted[r], k)} prod_{i<=l} alpha[r, i] (Eq. 9; accepted =
  *   accepted drafts + 1 = the first rejected position, k + 1 if none), evaluated in the log domain (Eq. 7);
- *   mean[0] = their mean, added in a fixed order.  A chain whose first overlap is 0 gives +inf.           */
+ *   mean[0] = their mean, added in a fixed order.  A chain whose first overlap is 0 gives +inf.
+ *
+ * gm_dca_grad (first step of the backward pass): grad_logits bf16 [n_cycles, k, V] = d mean / d draft_logits.
+ *   Per row (r, j): dL/dalpha = -(prod_{i<j} alpha_i) D_j / M with the chain sums cut at min(accepted[r], k)
+ *   (Eq. 8 under the gate of Eq. 9), divided by n_cycles; rows at or after the cut, and rows of a chain whose
+ *   first overlap is 0, are written as zeros.  alpha is piecewise linear in q: slope 1 on a retained token
+ *   where q < p, minus 1 on every retained token when the residual bin of q is the smaller one, 0 on all
+ *   other tokens and at ties; the softmax gives d alpha / d logit_v = q_v (slope_v - sum_e q_e slope_e) / T.
+ *   alpha and accepted are the arrays gm_overlap and the record produced; lse is gm_overlap's second output
+ *   for the same logits and temperature, or NULL (recomputed); draft_logits is only read.                */
 /* Rollout-time capture of the target hidden states (App. D.2: every sequence also stores the rollout-time
  * target hidden states of the prompt and of all committed tokens).  While seq_hidden (device bf16
  * [max_batch, stride, d]) is set, gm_prefill writes H_0..H_{L-1} of every prompt and every committing
@@ -353,9 +364,12 @@ int gm_reconstruct(gm_ctx *ctx, gm_state *st, int n_cycles, int k, const int32_t
                    const gm_record *rec, const int32_t *seq_tok, int tok_stride,
                    const int32_t *scratch_pages, void *draft_logits);
 int gm_overlap(gm_ctx *ctx, int n_cycles, int k, float temperature, const void *draft_logits,
-               const gm_record *rec, float *alpha);
+               const gm_record *rec, float *alpha, float *lse);
 int gm_dca_loss(gm_ctx *ctx, int n_cycles, int k, const float *alpha, const int32_t *accepted,
                 float *loss, float *mean);
+int gm_dca_grad(gm_ctx *ctx, int n_cycles, int k, float temperature, const void *draft_logits,
+                const gm_record *rec, const float *alpha, const float *lse, const int32_t *accepted,
+                void *grad_logits);
 
 
 /* Dense projection out[M, N] = x[M, K] w[N, K]^T on the context's stream (bf16 in, fp32

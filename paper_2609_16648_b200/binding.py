@@ -24,7 +24,7 @@ GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER, GM_KC_RECORD = 0,
 
 EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw", "gm_set_top_p", "gm_nucleus", "gm_prefill",
            "gm_rollout_begin", "gm_rollout_step", "gm_rollout_run", "gm_pages_reset", "gm_pages_reserve",
-           "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_overlap", "gm_dca_loss",
+           "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_overlap", "gm_dca_loss", "gm_dca_grad",
            "gm_spec_step_host", "gm_gemm", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
            "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
@@ -94,8 +94,9 @@ def lib() -> C.CDLL:
     L.gm_capture_hidden.argtypes = [vp, vp, i32]
     L.gm_head_prefill.argtypes = [vp, C.POINTER(gm_state), vp, i32, vp, i32, vp, i32]
     L.gm_reconstruct.argtypes = [vp, C.POINTER(gm_state), i32, i32, vp, C.POINTER(gm_record), vp, i32, vp, vp]
-    L.gm_overlap.argtypes = [vp, i32, i32, f32, vp, C.POINTER(gm_record), vp]
+    L.gm_overlap.argtypes = [vp, i32, i32, f32, vp, C.POINTER(gm_record), vp, vp]
     L.gm_dca_loss.argtypes = [vp, i32, i32, vp, vp, vp, vp]
+    L.gm_dca_grad.argtypes = [vp, i32, i32, f32, vp, C.POINTER(gm_record), vp, vp, vp, vp]
     L.gm_pages_reserve.argtypes = [vp, C.POINTER(gm_state), vp, i32, vp]
     L.gm_pages_release.argtypes = [vp, C.POINTER(gm_state), vp]
     L.gm_pages_free_count.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
@@ -387,13 +388,19 @@ def gm_reconstruct(ctx: Context, st: State, n_cycles: int, k: int, cycle_seq, re
                                 _p(seq_tok), seq_tok.shape[1], _p(scratch_pages), _p(draft_logits)), "gm_reconstruct")
 
 
-def gm_overlap(ctx: Context, n_cycles: int, k: int, temperature: float, draft_logits, rec, alpha):
-    _check(lib().gm_overlap(ctx.handle, n_cycles, k, temperature, _p(draft_logits), C.byref(rec.struct()), _p(alpha)),
-           "gm_overlap")
+def gm_overlap(ctx: Context, n_cycles: int, k: int, temperature: float, draft_logits, rec, alpha, lse=None):
+    _check(lib().gm_overlap(ctx.handle, n_cycles, k, temperature, _p(draft_logits), C.byref(rec.struct()), _p(alpha),
+                            _p(lse)), "gm_overlap")
 
 
 def gm_dca_loss(ctx: Context, n_cycles: int, k: int, alpha, accepted, loss, mean):
     _check(lib().gm_dca_loss(ctx.handle, n_cycles, k, _p(alpha), _p(accepted), _p(loss), _p(mean)), "gm_dca_loss")
+
+
+def gm_dca_grad(ctx: Context, n_cycles: int, k: int, temperature: float, draft_logits, rec, alpha, accepted, grad_logits,
+                lse=None):
+    _check(lib().gm_dca_grad(ctx.handle, n_cycles, k, temperature, _p(draft_logits), C.byref(rec.struct()), _p(alpha),
+                             _p(lse), _p(accepted), _p(grad_logits)), "gm_dca_grad")
 
 
 def gm_pages_reset(ctx: Context, st: State):

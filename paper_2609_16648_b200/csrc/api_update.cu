@@ -52,13 +52,13 @@ int gm_reconstruct(gm_ctx *c, gm_state *st, int n_cycles, int k, const int32_t *
 }
 
 int gm_overlap(gm_ctx *c, int n_cycles, int k, float temperature, const void *draft_logits, const gm_record *rec,
-               float *alpha) {
+               float *alpha, float *lse) {
   if (!c || n_cycles < 1 || k < 1 || k > GM_MAX_K || !draft_logits || !rec || !rec->top_index || !rec->top_logprob || !alpha)
     return GM_ERR_INVALID_ARG;
   if (!(temperature > 0.f) || !std::isfinite(temperature)) return GM_ERR_UNSUPPORTED;
   OverlapArgs A;
   A.logits = static_cast<const __nv_bfloat16 *>(draft_logits); A.top_index = rec->top_index;
-  A.top_logprob = static_cast<const __nv_bfloat16 *>(rec->top_logprob); A.alpha = alpha; A.V = c->V;
+  A.top_logprob = static_cast<const __nv_bfloat16 *>(rec->top_logprob); A.alpha = alpha; A.lse = lse; A.V = c->V;
   A.inv_temp = 1.0f / temperature;
   GM_LAUNCH(c, GM_KC_RECORD, launch_overlap(A, n_cycles * k, c->stream));
   return GM_OK;
@@ -67,6 +67,21 @@ int gm_overlap(gm_ctx *c, int n_cycles, int k, float temperature, const void *dr
 int gm_dca_loss(gm_ctx *c, int n_cycles, int k, const float *alpha, const int32_t *accepted, float *loss, float *mean) {
   if (!c || n_cycles < 1 || k < 1 || k > GM_MAX_K || !alpha || !accepted || !loss || !mean) return GM_ERR_INVALID_ARG;
   GM_LAUNCH(c, GM_KC_RECORD, launch_dca_loss(alpha, accepted, n_cycles, k, loss, mean, c->stream));
+  return GM_OK;
+}
+
+int gm_dca_grad(gm_ctx *c, int n_cycles, int k, float temperature, const void *draft_logits, const gm_record *rec,
+                const float *alpha, const float *lse, const int32_t *accepted, void *grad_logits) {
+  if (!c || n_cycles < 1 || k < 1 || k > GM_MAX_K || !draft_logits || !rec || !rec->top_index || !rec->top_logprob ||
+      !alpha || !accepted || !grad_logits)
+    return GM_ERR_INVALID_ARG;
+  if (!(temperature > 0.f) || !std::isfinite(temperature)) return GM_ERR_UNSUPPORTED;
+  DcaGradArgs A;
+  A.logits = static_cast<const __nv_bfloat16 *>(draft_logits); A.top_index = rec->top_index;
+  A.top_logprob = static_cast<const __nv_bfloat16 *>(rec->top_logprob); A.alpha = alpha; A.lse = lse; A.accepted = accepted;
+  A.grad = static_cast<__nv_bfloat16 *>(grad_logits); A.V = c->V; A.K = k; A.n = n_cycles;
+  A.inv_temp = 1.0f / temperature;
+  GM_LAUNCH(c, GM_KC_RECORD, launch_dca_grad(A, c->stream));
   return GM_OK;
 }
 

@@ -195,10 +195,23 @@ struct OverlapArgs {
   const int32_t *top_index;                        // [rows, 64]
   const __nv_bfloat16 *top_logprob;                // [rows, 64]
   float *alpha;                                    // [rows]
+  float *lse;                                      // [rows] logsumexp(logits / T) out, or null
   int V;
   float inv_temp;
 };
 cudaError_t launch_overlap(const OverlapArgs &A, int rows, cudaStream_t stream);
+struct DcaGradArgs {
+  const __nv_bfloat16 *logits;                     // [n, K, V] head logits of the reconstructed chains
+  const int32_t *top_index;                        // [n, K, 64]
+  const __nv_bfloat16 *top_logprob;
+  const float *alpha;                              // [n, K]
+  const int32_t *accepted;                         // [n]
+  const float *lse;                                // [n, K] from the overlap pass, or null: recomputed
+  __nv_bfloat16 *grad;                             // [n, K, V] out
+  int V, K, n;
+  float inv_temp;
+};
+cudaError_t launch_dca_grad(const DcaGradArgs &A, cudaStream_t stream);
 // Rollout-time capture of the target hidden states of committed positions (App. D.2: "each sequence additionally
 // stores the rollout-time target hidden states"): dst[b][pos] = the hidden state computed at position pos.
 //   chunk form (prefill): rows j < row_n[v] of src [rows, QT, d] go to positions row_base[v] + j of sequence v / vr;

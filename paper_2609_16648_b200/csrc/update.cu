@@ -66,44 +66,56 @@ gather_chunk_hidden_kernel(const __nv_bfloat16 *seq_hidden, int hid_stride, cons
   for (int i = threadIdx.x; i < d / 8; i += blockDim.x) o[i] = s[i];
 }
 
+// Softmax statistics of one row in a single pass: running maximum with the sum rescaled when it moves.  Returns
+// logsumexp(x / T) to every thread of the CTA.  NT threads, NT / 32 <= 32.
+template <int NT>
+__device__ __forceinline__ float row_lse(const uint4 *xv, int nvec, float inv_temp, float *red_m, float *red_z, float *out) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float m = -INFINITY, z = 0.f;
+  auto take = [&](const uint4 &v) {
+    const uint32_t wds[4] = {v.x, v.y, v.z, v.w};
+    const float cm = fmaxf(fmaxf(fmaxf(bf16_lo(v.x), bf16_hi(v.x)), fmaxf(bf16_lo(v.y), bf16_hi(v.y))),
+                           fmaxf(fmaxf(bf16_lo(v.z), bf16_hi(v.z)), fmaxf(bf16_lo(v.w), bf16_hi(v.w))));
+    if (cm > m) { z *= __expf((m - cm) * inv_temp); m = cm; }
+#pragma unroll
+    for (int t = 0; t < 4; ++t) z += __expf((bf16_lo(wds[t]) - m) * inv_temp) + __expf((bf16_hi(wds[t]) - m) * inv_temp);
+  };
+  int i = tid;
+  for (; i + 3 * NT < nvec; i += 4 * NT) {                // four loads in flight per thread
+    const uint4 v0 = xv[i], v1 = xv[i + NT], v2 = xv[i + 2 * NT], v3 = xv[i + 3 * NT];
+    take(v0); take(v1); take(v2); take(v3);
+  }
+  for (; i < nvec; i += NT) take(xv[i]);
+  for (int o = 16; o; o >>= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, m, o), z2 = __shfl_xor_sync(0xffffffffu, z, o);
+    const float mn = fmaxf(m, m2);
+    z = (m == -INFINITY ? 0.f : z * __expf((m - mn) * inv_temp)) + (m2 == -INFINITY ? 0.f : z2 * __expf((m2 - mn) * inv_temp));
+    m = mn;
+  }
+  if (lane == 0) { red_m[warp] = m; red_z[warp] = z; }
+  __syncthreads();
+  if (tid == 0) {
+    float mm = red_m[0];
+    for (int w = 1; w < NT / 32; ++w) mm = fmaxf(mm, red_m[w]);
+    float t = 0.f;
+    for (int w = 0; w < NT / 32; ++w)
+      if (red_m[w] != -INFINITY) t += red_z[w] * __expf((red_m[w] - mm) * inv_temp);
+    *out = mm * inv_temp + logf(t);
+  }
+  __syncthreads();
+  return *out;
+}
+
 // alpha = sum_i min(p_i, q_i) + min(1 - sum p_i, 1 - sum q_i) over the record's retained entries; one CTA per row.
-constexpr int OV_THREADS = 256;
+constexpr int OV_THREADS = 512;
 __global__ void __launch_bounds__(OV_THREADS) overlap_kernel(const OverlapArgs A) {
-  __shared__ float red[OV_THREADS / 32];
+  __shared__ float red_m[OV_THREADS / 32], red_z[OV_THREADS / 32];
   __shared__ float sh_lse;
   const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const __nv_bfloat16 *x = A.logits + static_cast<size_t>(row) * A.V;
-  const uint4 *xv = reinterpret_cast<const uint4 *>(x);
-  const int nvec = A.V >> 3;
   pdl_prologue();
-  float m = -INFINITY;
-  for (int i = tid; i < nvec; i += OV_THREADS) {
-    const uint4 v = xv[i];
-    m = fmaxf(m, fmaxf(fmaxf(fmaxf(bf16_lo(v.x), bf16_hi(v.x)), fmaxf(bf16_lo(v.y), bf16_hi(v.y))),
-                       fmaxf(fmaxf(bf16_lo(v.z), bf16_hi(v.z)), fmaxf(bf16_lo(v.w), bf16_hi(v.w)))));
-  }
-  for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-  if (lane == 0) red[warp] = m;
-  __syncthreads();
-  m = red[0];
-  for (int w = 1; w < OV_THREADS / 32; ++w) m = fmaxf(m, red[w]);
-  __syncthreads();
-  float z = 0.f;
-  for (int i = tid; i < nvec; i += OV_THREADS) {
-    const uint4 v = xv[i];
-    const uint32_t wds[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int t = 0; t < 4; ++t) z += __expf((bf16_lo(wds[t]) - m) * A.inv_temp) + __expf((bf16_hi(wds[t]) - m) * A.inv_temp);
-  }
-  for (int o = 16; o; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
-  if (lane == 0) red[warp] = z;
-  __syncthreads();
-  if (tid == 0) {
-    float t = 0.f;
-    for (int w = 0; w < OV_THREADS / 32; ++w) t += red[w];
-    sh_lse = m * A.inv_temp + logf(t);
-  }
-  __syncthreads();
+  row_lse<OV_THREADS>(reinterpret_cast<const uint4 *>(x), A.V >> 3, A.inv_temp, red_m, red_z, &sh_lse);
+  if (tid == 0 && A.lse) A.lse[row] = sh_lse;
   if (warp < 2) {                                          // 64 retained entries: two warps
     const int e = tid;
     const int idx = A.top_index[static_cast<size_t>(row) * 64 + e];
@@ -125,6 +137,93 @@ __global__ void __launch_bounds__(OV_THREADS) overlap_kernel(const OverlapArgs A
       const float mins = part[0][0] + part[1][0], psum = part[0][1] + part[1][1], qsum = part[0][2] + part[1][2];
       A.alpha[row] = mins + fminf(fmaxf(1.f - psum, 0.f), fmaxf(1.f - qsum, 0.f));
     }
+  }
+}
+
+// Gradient of the mean objective with respect to the reconstructed head logits (first step of the backward pass).
+// Row (cycle c, position k): dL/dalpha = -(prod_{i<k} alpha_i) D_k / M with the chain sums cut at L = min(j, K)
+// (Eq. 8 with the gate of Eq. 9), 0 for k >= L and for a dead chain (M = 0).  alpha is piecewise linear in q: slope
+// g_e = 1[q_e < p_e] - 1[q_res < p_res] on the retained tokens, 0 elsewhere (ties: slope 0);
+// dalpha/dlogit_v = q_v (g_v - G) / T with G = sum_e q_e g_e.  One CTA per row: one pass for the softmax statistics
+// (running maximum and rescaled sum), the 64 retained entries, then one pass that writes the whole row.
+constexpr int DG_THREADS = 512;
+__global__ void __launch_bounds__(DG_THREADS) dca_grad_kernel(const DcaGradArgs A) {
+  __shared__ float red_m[DG_THREADS / 32], red_z[DG_THREADS / 32];
+  __shared__ float sh_lse, sh_G;
+  __shared__ float part[2][3];
+  __shared__ int sh_res;
+  const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int c = row / A.K, kk = row % A.K;
+  const __nv_bfloat16 *x = A.logits + static_cast<size_t>(row) * A.V;
+  const uint4 *xv = reinterpret_cast<const uint4 *>(x);
+  uint4 *ov = reinterpret_cast<uint4 *>(A.grad + static_cast<size_t>(row) * A.V);
+  const int nvec = A.V >> 3;
+  pdl_prologue();
+  float coef = 0.f;
+  {
+    const int L = min(max(A.accepted[c], 1), A.K);
+    if (kk < L) {
+      float a[GM_MAX_K_];
+      for (int i = 0; i < L; ++i) a[i] = A.alpha[static_cast<size_t>(c) * A.K + i];
+      float M = 0.f, run = 1.f, pre = 1.f;
+      for (int l = 0; l < L; ++l) { if (l == kk) pre = run; run *= a[l]; M += run; }
+      float D = 0.f, t = 1.f;
+      for (int l = kk; l < L; ++l) { if (l > kk) t *= a[l]; D += t; }
+      if (M > 0.f) coef = -(pre * D / M) / static_cast<float>(A.n);
+    }
+  }
+  if (coef == 0.f) {
+    for (int i = tid; i < nvec; i += DG_THREADS) ov[i] = make_uint4(0u, 0u, 0u, 0u);
+    return;
+  }
+  float lse;
+  if (A.lse) lse = A.lse[row];
+  else lse = row_lse<DG_THREADS>(xv, nvec, A.inv_temp, red_m, red_z, &sh_lse);
+  int idx = -1;
+  float qe = 0.f, ge = 0.f;
+  if (warp < 2) {                                          // the 64 retained entries: two warps
+    idx = A.top_index[static_cast<size_t>(row) * 64 + tid];
+    float p = 0.f;
+    if (idx >= 0 && idx < A.V) {
+      p = expf(bf16_to_float(A.top_logprob[static_cast<size_t>(row) * 64 + tid]));
+      qe = expf(bf16_to_float(x[idx]) * A.inv_temp - lse);
+    } else {
+      idx = -1;
+    }
+    ge = (idx >= 0 && qe < p) ? 1.f : 0.f;
+    float ps = p, qs = qe, gq = qe * ge;
+    for (int o = 16; o; o >>= 1) {
+      ps += __shfl_xor_sync(0xffffffffu, ps, o);
+      qs += __shfl_xor_sync(0xffffffffu, qs, o);
+      gq += __shfl_xor_sync(0xffffffffu, gq, o);
+    }
+    if (lane == 0) { part[warp][0] = ps; part[warp][1] = qs; part[warp][2] = gq; }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    const float psum = part[0][0] + part[1][0], qsum = part[0][1] + part[1][1];
+    const int res = fmaxf(1.f - qsum, 0.f) < fmaxf(1.f - psum, 0.f);
+    sh_res = res;
+    sh_G = part[0][2] + part[1][2] - (res ? qsum : 0.f);
+  }
+  __syncthreads();
+  const float G = sh_G, scale = coef * A.inv_temp;
+  const float base = -G * scale;                           // every token outside the retained set: q_v * base
+  for (int i = tid; i < nvec; i += DG_THREADS) {
+    const uint4 v = xv[i];
+    const uint32_t wds[4] = {v.x, v.y, v.z, v.w};
+    uint32_t o4[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const float q0 = __expf(bf16_lo(wds[t]) * A.inv_temp - lse), q1 = __expf(bf16_hi(wds[t]) * A.inv_temp - lse);
+      o4[t] = pack_bf16(q0 * base, q1 * base);
+    }
+    ov[i] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+  }
+  __syncthreads();                                         // the retained entries are rewritten after the row pass
+  if (warp < 2 && idx >= 0) {
+    if (sh_res) ge -= 1.f;
+    A.grad[static_cast<size_t>(row) * A.V + idx] = __float2bfloat16_rn(qe * (ge - G) * scale);
   }
 }
 
@@ -212,6 +311,9 @@ cudaError_t launch_gather_chunk_hidden(const __nv_bfloat16 *seq_hidden, int hid_
 }
 cudaError_t launch_overlap(const OverlapArgs &A, int rows, cudaStream_t stream) {
   return launch_k(overlap_kernel, dim3(rows), dim3(OV_THREADS), 0, stream, 1, A);
+}
+cudaError_t launch_dca_grad(const DcaGradArgs &A, cudaStream_t stream) {
+  return launch_k(dca_grad_kernel, dim3(A.n * A.K), dim3(DG_THREADS), 0, stream, 1, A);
 }
 cudaError_t launch_dca_loss(const float *alpha, const int32_t *accepted, int n, int K, float *loss, float *mean,
                             cudaStream_t stream) {

@@ -113,6 +113,87 @@ def test_head_update_forward_matches_the_oracle():
     assert float(mean[0]) == pytest.approx(want.mean(), rel=1e-5)
     ref_loss, _ = oupdate.head_update_loss(w, cfg, seqs, cycles, T)
     assert abs(float(mean[0]) - ref_loss) < 3e-2
+
+    # first step of the backward pass: d mean / d logits, against the oracle on the device's logits
+    grad = torch.full((n, K, V), 7.0, dtype=torch.bfloat16, device="cuda")
+    gmb.gm_dca_grad(ctx, n, K, T, logits, rec, alpha, rec.accepted, grad)
+    _check_grad(grad.float().cpu().numpy(), lg, [r for _, r in cycles], T)
+    # with the row statistics handed over from the overlap pass: the same numbers
+    lse = torch.zeros((n, K), dtype=torch.float32, device="cuda")
+    alpha2 = torch.zeros_like(alpha)
+    gmb.gm_overlap(ctx, n, K, T, logits, rec, alpha2, lse)
+    assert torch.equal(alpha2, alpha)
+    y = lg / T
+    np.testing.assert_allclose(lse.cpu().numpy(), np.log(np.exp(y - y.max(-1, keepdims=True)).sum(-1)) + y.max(-1), rtol=0, atol=2e-5 * np.abs(y).max())
+    grad2 = torch.full_like(grad, 7.0)
+    gmb.gm_dca_grad(ctx, n, K, T, logits, rec, alpha, rec.accepted, grad2, lse)
+    assert torch.equal(grad2, grad)
+    ctx.close()
+
+
+def _check_grad(got, lg, recs, T):
+    """Element-wise against the oracle's gradient.  A retained token whose q and p agree to fp32 rounding may take
+    either slope (the objective has a kink there): such rows are left out, and must be rare."""
+    n, K, V = got.shape
+    want = oupdate.head_update_grad_logits(lg, recs, T)
+    q = oupdate.softmax64(lg, T)
+    skipped = 0
+    for r, rec in enumerate(recs):
+        L = min(rec["accepted"], K)
+        assert (got[r, L:] == 0).all()                       # the verify gate: nothing after the first rejection
+        for k in range(L):
+            keep = rec["top_index"][k] >= 0
+            pk = np.exp(rec["top_logprob"][k][keep].astype(np.float64))
+            qk = q[r, k][rec["top_index"][k][keep]]
+            near = np.abs(pk - qk) <= 1e-5 * np.maximum(pk, qk)
+            res_near = abs(max(1 - pk.sum(), 0) - max(1 - qk.sum(), 0)) <= 1e-5
+            if near.any() or res_near:
+                skipped += 1
+                continue
+            scale = np.abs(want[r, k]).max()
+            assert scale > 0
+            # bf16 output: 2^-8 relative per element, on top of fp32 exponentials
+            np.testing.assert_allclose(got[r, k], want[r, k], rtol=1.2e-2, atol=1e-3 * scale)
+            assert abs(got[r, k].sum()) < 2e-2 * np.abs(got[r, k]).sum()
+    assert skipped <= max(2, n * K // 20), skipped
+    return skipped
+
+
+def test_gradient_kernel_full_vocabulary_and_edge_cases():
+    """gm_dca_grad alone at the 4B vocabulary (ragged tail of the vector loop: 151936 = 8 * 18992): synthetic head
+    logits and records built by the oracle from synthetic target logits; dead chains, gated rows, K = 7."""
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny").with_(vocab=151936)
+    n, K, V = 8, 7, cfg.vocab
+    ctx = gmb.Context(cfg, gmb.random_packed_weights(cfg, "cuda"), 4, K, 4, 8, 8)
+    rng = np.random.default_rng(11)
+    Tg = 0.8
+    head = omodel.round_bf16(rng.normal(0, 2.5, (n, K, V))).astype(np.float64)
+    recs = []
+    for r in range(n):
+        tgt = omodel.round_bf16(head[r] + rng.normal(0, 1.0, (K, V)))
+        full = orecord.cycle_record(np.zeros(cfg.d_model), np.zeros(K, np.int64),
+                                    np.concatenate([tgt, tgt[:1]]), int(r % (K + 1)), 5, Tg)
+        recs.append({"top_index": full["top_index"][:K], "top_logprob": full["top_logprob"][:K], "accepted": full["accepted"]})
+    rec = gmb.Record(n, K, cfg.d_model)
+    rec.top_index.copy_(torch.from_numpy(np.stack([r["top_index"] for r in recs]).astype(np.int32)))
+    rec.top_logprob.copy_(torch.from_numpy(np.stack([r["top_logprob"] for r in recs])).to(torch.bfloat16))
+    rec.accepted.copy_(torch.tensor([r["accepted"] for r in recs], dtype=torch.int32))
+    logits = torch.from_numpy(head).to(device="cuda", dtype=torch.bfloat16)
+    alpha = torch.zeros((n, K), dtype=torch.float32, device="cuda")
+    lse = torch.zeros((n, K), dtype=torch.float32, device="cuda")
+    gmb.gm_overlap(ctx, n, K, Tg, logits, rec, alpha, lse)
+    grad = torch.full((n, K, V), 7.0, dtype=torch.bfloat16, device="cuda")
+    gmb.gm_dca_grad(ctx, n, K, Tg, logits, rec, alpha, rec.accepted, grad, lse)
+    assert gmb.gm_last_status(ctx) == 0
+    got = grad.float().cpu().numpy()
+    _check_grad(got, head, recs, Tg)
+    assert any(r["accepted"] == 1 for r in recs) and any(r["accepted"] == K + 1 for r in recs)
+    # a dead chain (first overlap 0) has no finite objective: its rows are written as zeros
+    alpha[2, 0] = 0.0
+    gmb.gm_dca_grad(ctx, n, K, Tg, logits, rec, alpha, rec.accepted, grad)
+    g2 = grad.float().cpu().numpy()
+    assert (g2[2] == 0).all() and np.array_equal(g2[[0, 1, 3, 4, 5, 6, 7]], got[[0, 1, 3, 4, 5, 6, 7]])
     ctx.close()
 
 
