@@ -377,6 +377,10 @@ int gm_dca_grad(gm_ctx *ctx, int n_cycles, int k, float temperature, const void 
  *   out_fp32 != 0: out is fp32 [M, N]; else bf16 [M, N].  K % 64 == 0, N % 8 == 0, M >= 1.   */
 int gm_gemm(gm_ctx *ctx, const void *x, const void *w, void *out, int M, int N, int K,
             int out_fp32);
+/* The gate/up projection as the step runs it: y = x w^T with gate and up rows interleaved in w (row 2f = gate
+ * feature f, row 2f + 1 = up feature f; the decoder's SwiGLU feed-forward, App. B.1), out bf16 [M, N / 2] = silu(y[:, 2f]) * y[:, 2f + 1],
+ * fused into the projection's epilogue.  Same constraints as gm_gemm; N % 16 == 0 (else GM_ERR_UNSUPPORTED).                        */
+int gm_gemm_swiglu(gm_ctx *ctx, const void *x, const void *w, void *out, int M, int N, int K);
 
 /* Multi-query paged decode attention as a stand-alone call: the kernel both phases run once per layer
  * (Sec. 2.2: the target verifies all K candidates in a single forward pass; App. B.1: the head keeps a KV

@@ -25,7 +25,7 @@ GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER, GM_KC_RECORD = 0,
 EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw", "gm_set_top_p", "gm_nucleus", "gm_prefill",
            "gm_rollout_begin", "gm_rollout_step", "gm_rollout_run", "gm_pages_reset", "gm_pages_reserve",
            "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_overlap", "gm_dca_loss", "gm_dca_grad",
-           "gm_spec_step_host", "gm_gemm", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
+           "gm_spec_step_host", "gm_gemm", "gm_gemm_swiglu", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
            "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
 
@@ -103,6 +103,7 @@ def lib() -> C.CDLL:
     L.gm_prefill.argtypes = [vp, C.POINTER(gm_state), vp, vp, i32, i32, f32, vp, u64, vp, vp]
     L.gm_nucleus.argtypes = [vp, vp, i32, f32, f32, vp, vp]
     L.gm_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
+    L.gm_gemm_swiglu.argtypes = [vp, vp, vp, vp, i32, i32, i32]
     L.gm_attention.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, i32, i32, vp]
     L.gm_attention_noalloc.argtypes = [i32, i32, i32, i32, vp, vp, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp]
     L.gm_record_begin.argtypes = [vp, C.POINTER(gm_state), C.POINTER(gm_record)]
@@ -427,6 +428,10 @@ def gm_set_top_p(ctx: Context, top_p: float):
 
 def gm_nucleus(ctx: Context, logits, rows: int, temperature: float, top_p: float, out, dbg_weight=None):
     _check(lib().gm_nucleus(ctx.handle, _p(logits), rows, temperature, top_p, _p(out), _p(dbg_weight)), "gm_nucleus")
+
+
+def gm_gemm_swiglu(ctx: Context, x, w, out, M: int, N: int, K: int):
+    _check(lib().gm_gemm_swiglu(ctx.handle, _p(x), _p(w), _p(out), M, N, K), "gm_gemm_swiglu")
 
 
 def gm_gemm(ctx: Context, x, w, out, M: int, N: int, K: int, out_fp32: bool):

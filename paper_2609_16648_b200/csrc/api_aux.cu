@@ -71,7 +71,7 @@ int gm_spec_step_rec(gm_ctx *c, gm_state *st, int k, float temperature, uint64_t
   return gm_record_end(c, st->batch, k, temperature, c->ws_target_logits, dt, accept_len, rec);
 }
 
-int gm_gemm(gm_ctx *c, const void *x, const void *w, void *out, int M, int N, int K, int out_fp32) {
+static int gemm_entry(gm_ctx *c, const void *x, const void *w, void *out, int M, int N, int K, int epi, size_t ldo) {
   if (!c || !x || !w || !out || M < 1 || N < 1 || K < 1) return GM_ERR_INVALID_ARG;
   if ((K % 64) || (N % 8)) return GM_ERR_UNSUPPORTED;
   CUtensorMap wm;
@@ -87,7 +87,16 @@ int gm_gemm(gm_ctx *c, const void *x, const void *w, void *out, int M, int N, in
     wm = it->second;
   }
   return run_gemm(c, static_cast<const __nv_bfloat16 *>(x), M, &wm, static_cast<const __nv_bfloat16 *>(w), M, N, K, out,
-                  out_fp32 ? EPI_STORE_F32 : EPI_STORE_BF16, N);
+                  epi, ldo);
+}
+
+int gm_gemm(gm_ctx *c, const void *x, const void *w, void *out, int M, int N, int K, int out_fp32) {
+  return gemm_entry(c, x, w, out, M, N, K, out_fp32 ? EPI_STORE_F32 : EPI_STORE_BF16, static_cast<size_t>(N));
+}
+
+int gm_gemm_swiglu(gm_ctx *c, const void *x, const void *w, void *out, int M, int N, int K) {
+  if (c && N > 0 && (N % 16)) return GM_ERR_UNSUPPORTED;
+  return gemm_entry(c, x, w, out, M, N, K, EPI_SWIGLU_BF16, static_cast<size_t>(N / 2));
 }
 
 int gm_attention(gm_ctx *c, const void *q, const void *kv_pool, int pool_layers, int num_pages, int layer,

@@ -50,6 +50,8 @@ def test_error_strings_and_null_handling_need_no_gpu():
     assert L.gm_overlap(None, 1, 3, 1.0, None, None, None, None) == inv
     assert L.gm_dca_loss(None, 1, 3, None, None, None, None) == inv
     assert L.gm_dca_grad(None, 1, 3, 1.0, None, None, None, None, None, None) == inv
+    assert L.gm_gemm(None, None, None, None, 1, 8, 64, 0) == inv
+    assert L.gm_gemm_swiglu(None, None, None, None, 1, 16, 64) == inv
     assert L.gm_rollout_begin(None, None, None) == inv
     assert L.gm_rollout_step(None, None, None, 3, 1.0, 0, 0) == inv
     assert L.gm_rollout_run(None, None, None, 3, 1.0, 0, 0, 1, 1, None, None) == inv

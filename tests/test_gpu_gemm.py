@@ -67,3 +67,24 @@ def test_full_size_projections_on_sampled_outputs(M, N, K):
     got = out[:, cols].float().cpu().numpy()
     assert np.abs(got - ref).max() <= 5e-3 * np.abs(ref).max()
     ctx.close()
+
+
+@pytest.mark.parametrize("M", [256, 64, 300, 37])
+def test_gate_up_projection_with_fused_swiglu_full_matrix(M):
+    """The 4B gate/up projection (152 feature tiles: a full wave plus a split tail launch) over the whole output,
+    plain stores and the fused SwiGLU epilogue on interleaved gate/up rows, against fp64."""
+    N, K = 19456, 2560
+    gmb, ctx = _ctx()
+    g = torch.Generator(device="cuda").manual_seed(M)
+    x = torch.randn((M, K), device="cuda", generator=g).to(torch.bfloat16)
+    w = (torch.randn((N, K), device="cuda", generator=g) * 0.02).to(torch.bfloat16)
+    ref = (x.double() @ w.double().T).cpu().numpy()
+    act_ref = ref[:, 0::2] / (1 + np.exp(-ref[:, 0::2])) * ref[:, 1::2]
+    o32 = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    act = torch.full((M, N // 2), float("nan"), dtype=torch.bfloat16, device="cuda")
+    gmb.gm_gemm(ctx, x, w, o32, M, N, K, True)
+    gmb.gm_gemm_swiglu(ctx, x, w, act, M, N, K)
+    assert gmb.gm_last_status(ctx) == 0
+    assert np.abs(o32.cpu().numpy() - ref).max() <= 3e-5 * np.abs(ref).max()
+    assert np.abs(act.float().cpu().numpy() - act_ref).max() <= 6e-3 * np.abs(act_ref).max()
+    ctx.close()
