@@ -20,6 +20,9 @@
 // SwiGLU on interleaved gate/up rows.  Every wait is bounded; on expiry the kernel records
 // ST_TIMEOUT, still meets every barrier and frees its tensor memory.
 //
+// gemm_pair_kernel: the same projection on pairs of CTAs (tcgen05 cta_group::2) for full waves of one-slice tiles;
+// described at the kernel.
+//
 // gemm_simple_kernel: a plain warp-level mma.sync version with the same epilogues, kept as an
 // independent on-device cross-check and for shapes the tcgen05 kernel does not take.
 #include <cooperative_groups.h>
@@ -218,6 +221,125 @@ gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
   if (warp == 1) tc_dealloc(tmem, ncols);
 }
 
+// ---- CTA-pair variant --------------------------------------------------------------------------------------------------
+// Projections with one K slice per tile are bound by filling shared memory from L2: every CTA re-reads the whole
+// activation tile for its 128 features.  Here two CTAs on neighbouring feature tiles form a pair (a cluster of
+// two): each stages its own 128 x 64 weight box and only HALF of the activation box per K block, and one
+// tcgen05.mma of the pair (M = 256 features, N = T tokens) reads both halves, so a CTA moves 2/3 of the bytes per K
+// block (at T = 256) and its ring holds more K blocks.  The accumulator rows of a CTA's own 128 features land in its
+// own tensor memory, so the epilogue is the single-CTA one.
+//   even CTA (leader): producer + the MMA issuer for the pair.  Its `full` barriers count the bytes of both CTAs.
+//   odd CTA: producer only; its loads complete on the leader's barriers.  The leader's tcgen05.commit arrives on
+//   the `empty` / accumulator barriers of both CTAs (relaying those arrivals through the leader's waiting threads
+//   instead made every stage refill ~3 us longer and the main loop 0.93 us per K block instead of 0.50).
+__global__ void __launch_bounds__(GT_THREADS, 1)
+gemm_pair_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
+  extern __shared__ unsigned char gt_smem_raw[];
+  unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(gt_smem_raw) + 1023) & ~uintptr_t(1023));
+  const int T = A.block_t, H = T / 2;
+  const int a_bytes = GT_BN * 128, b_bytes = H * 128, stage_b = a_bytes + b_bytes;
+  size_t pipe_b = static_cast<size_t>(nstages) * stage_b;
+  if (static_cast<size_t>(T) * GT_BN * 4 > pipe_b) pipe_b = static_cast<size_t>(T) * GT_BN * 4;
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem + pipe_b);
+  uint64_t *empty = full + 8;
+  uint64_t *acc_full = empty + 8;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  float *park = reinterpret_cast<float *>(smem);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();            // 0: leader, 1: peer
+  const bool leader = rank == 0;
+  const int n0 = A.n_base + blockIdx.x * GT_BN, m0 = blockIdx.y * T;     // the pair = two neighbouring feature tiles
+  const int KB = A.K / GT_BK;
+  const uint32_t ncols = T <= 32 ? 32u : T <= 64 ? 64u : T <= 128 ? 128u : 256u;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < nstages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    tc2_alloc(tmem_slot, ncols);
+    tc2_relinquish();
+  }
+  if (warp == 0 && lane == 0) {
+    tma_prefetch_desc(&A.w_map);
+    tma_prefetch_desc(&A.x_half_map);
+  }
+  tc_fence_before();
+  cg::cluster_group cluster = cg::this_cluster();
+  cluster.sync();                                  // both CTAs' barriers exist before anything arrives on them
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  pdl_prologue();
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int kb = 0; kb < KB; ++kb) {
+        const int s = kb % nstages;
+        if (!mbar_wait(&empty[s], ((kb / nstages) & 1) ^ 1)) { set_status(A.status, ST_TIMEOUT); break; }
+        if (leader) {
+          mbar_expect_tx(&full[s], 2 * stage_b);
+        }
+        const uint32_t bar = cluster_addr(&full[s], 0);
+        unsigned char *dst = smem + static_cast<size_t>(s) * stage_b;
+        tma2_load_2d(dst, &A.w_map, kb * GT_BK, n0, bar);
+        tma2_load_2d(dst + a_bytes, &A.x_half_map, kb * GT_BK, m0 + static_cast<int>(rank) * H, bar);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && leader) {
+      const uint32_t idesc = tc_idesc_bf16(2 * GT_BN, T);
+      bool ok = true;
+      for (int kb = 0; kb < KB; ++kb) {
+        const int s = kb % nstages;
+        if (!mbar_wait(&full[s], (kb / nstages) & 1)) { set_status(A.status, ST_TIMEOUT); ok = false; break; }
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(smem + static_cast<size_t>(s) * stage_b);
+        const uint64_t adesc = tc_smem_desc_sw128(a_addr), bdesc = tc_smem_desc_sw128(a_addr + a_bytes);
+#pragma unroll
+        for (int k = 0; k < GT_BK / 16; ++k)
+          tc2_mma_bf16(tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+        tc2_commit_mc(&empty[s], 3);                // the stage is free in both CTAs
+      }
+      if (ok) tc2_commit_mc(acc_full, 3);
+    }
+  }
+  bool acc_ok = KB > 0;
+  const bool reader = warp >= 2 && warp < 10;
+  if (reader) {
+    if (acc_ok && !mbar_wait(acc_full, 0)) { set_status(A.status, ST_TIMEOUT); acc_ok = false; }
+    tc_fence_after();
+  }
+  __syncthreads();                                 // the pipeline stages are done with (both CTAs' MMAs have completed)
+  if (reader) {
+    const int quad = warp & 3;
+    const int r = quad * 32 + lane;
+    for (int c0 = ((warp - 2) >> 2) * 16; c0 < T; c0 += 32) {
+      uint32_t v[16];
+      if (acc_ok) {
+        tc_ld_32x16(tmem + (static_cast<uint32_t>(quad * 32) << 16) + c0, v);
+        tc_wait_ld();
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = 0u;
+      }
+#pragma unroll
+      for (int j = 0; j < 16; ++j) park[(c0 + j) * GT_BN + r] = __uint_as_float(v[j]);
+    }
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < T * (GT_BN / 4); idx += GT_THREADS) {
+    const int c = idx / (GT_BN / 4), r4 = (idx % (GT_BN / 4)) * 4;
+    const int m = m0 + c, n = n0 + r4;
+    if (m >= A.M || n >= A.N) continue;
+    epilogue4(A, m, n, *reinterpret_cast<const float4 *>(park + c * GT_BN + r4));
+  }
+  tc_fence_before();
+  cluster.sync();                                  // neither CTA frees tensor memory while the other still reads its own
+  if (warp == 1) tc2_dealloc(tmem, ncols);
+}
+
 // The kernel may use the whole opt-in shared memory of an SM (227 KB); set once per process.
 static cudaError_t gt_configure() {
   static bool done = false;
@@ -245,6 +367,29 @@ cudaError_t gemm_tc_max_clusters(int block_t, int nsplit, int *out) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaOccupancyMaxActiveClusters(out, gemm_tc_kernel, &cfg);
+}
+
+static int pair_stages(int T) {
+  int s = GT_SMEM_BUDGET / (GT_BN * 128 + (T / 2) * 128);
+  return s > 8 ? 8 : s;
+}
+cudaError_t launch_gemm_pair(const GemmArgs &A, cudaStream_t stream) {
+  const int T = A.block_t;
+  if (T < 32 || T > 256 || (T & 31) || (A.K % GT_BK) || A.nsplit != 1 || A.wtiles != 1 || A.n_tiles < 2 ||
+      (A.n_tiles & 1) || A.n_base < 0)
+    return cudaErrorInvalidValue;
+  static bool done = false;
+  if (!done) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    done = true;
+  }
+  const int st = pair_stages(T);
+  size_t pipe = static_cast<size_t>(st) * (GT_BN * 128 + (T / 2) * 128);
+  const size_t park = static_cast<size_t>(T) * GT_BN * 4;
+  if (park > pipe) pipe = park;
+  const dim3 grid(A.n_tiles, (A.M + T - 1) / T, 1);
+  return launch_kc(gemm_pair_kernel, grid, dim3(GT_THREADS), pipe + 1024 + 256, stream, dim3(2, 1, 1), A, st);
 }
 
 cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream) {

@@ -107,7 +107,13 @@ int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *w
   const int rem = (units * mblocks) % c->sm_count;
   if (A.nsplit == 1 && mblocks == 1 && units > c->sm_count && rem != 0 && rem * 4 <= c->sm_count) {
     A.n_tiles = units - rem;
-    GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(A, c->stream));
+    if (c->pair_gemm && A.wtiles == 1 && (T % 32) == 0 && (A.n_tiles % 2) == 0) {
+      rc = x_map(c, x, x_rows, K, T / 2, &A.x_half_map);
+      if (rc != GM_OK) return rc;
+      GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_pair(A, c->stream));
+    } else {
+      GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(A, c->stream));
+    }
     GemmArgs Tl = A;
     Tl.n_base = A.n_tiles * 128 * A.wtiles;
     Tl.wtiles = 1;
@@ -283,6 +289,7 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
   c->w.layers = c->layers.data();
   c->stream = static_cast<cudaStream_t>(cuda_stream);
   c->check_guards = std::getenv("GM_CANARY") != nullptr;
+  c->pair_gemm = std::getenv("GM_NO_PAIR_GEMM") == nullptr;
   cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev);
   c->d = cfg->d_model; c->q_dim = cfg->n_q_heads * cfg->head_dim; c->kv_dim = cfg->n_kv_heads * cfg->head_dim;
   c->n_qkv = c->q_dim + 2 * c->kv_dim; c->F = cfg->d_ffn; c->V = cfg->vocab; c->group = group;

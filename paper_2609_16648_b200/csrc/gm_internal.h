@@ -52,6 +52,7 @@ struct gm_ctx {
   // workspaces (device)
   float *x = nullptr, *g = nullptr, *part_o = nullptr, *part_ml = nullptr;
   __nv_bfloat16 *xn = nullptr, *zin = nullptr, *qkv = nullptr, *qbuf = nullptr, *attn_out = nullptr, *act = nullptr, *gn = nullptr;
+  bool pair_gemm = true;              // CTA-pair kernel for the full wave of wide projections (GM_NO_PAIR_GEMM: off)
   int max_clusters[17][9];            // resident clusters of the GEMM kernel by (block_t / 16, cluster size); -1 = not asked yet
   __nv_bfloat16 *ws_draft_logits = nullptr, *ws_target_logits = nullptr, *ws_target_hidden = nullptr;
   int32_t *ws_draft_tok = nullptr, *ws_accept_len = nullptr, *ws_next_token = nullptr;

@@ -6,14 +6,16 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 namespace gm {
 
 // Launch with programmatic stream serialisation (the kernel calls pdl_prologue() first) and, if cluster_z > 1, a
-// thread-block cluster along z.  GM_NO_PDL=1 in the environment turns the attribute off (plain serialisation).
+// thread-block cluster (launch_k: along z; launch_kc: any shape).  GM_NO_PDL=1 in the environment turns the attribute off (plain serialisation).
 bool pdl_enabled();
 template <typename... KArgs, typename... Args>
-cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, int cluster_z,
-                     Args &&...args) {
+cudaError_t launch_kc(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, dim3 cluster,
+                      Args &&...args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -26,14 +28,19 @@ cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sme
     attr[n].val.programmaticStreamSerializationAllowed = 1;
     ++n;
   }
-  if (cluster_z > 1) {
+  if (cluster.x * cluster.y * cluster.z > 1) {
     attr[n].id = cudaLaunchAttributeClusterDimension;
-    attr[n].val.clusterDim.x = 1; attr[n].val.clusterDim.y = 1; attr[n].val.clusterDim.z = cluster_z;
+    attr[n].val.clusterDim.x = cluster.x; attr[n].val.clusterDim.y = cluster.y; attr[n].val.clusterDim.z = cluster.z;
     ++n;
   }
   cfg.attrs = attr;
   cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, int cluster_z,
+                     Args &&...args) {
+  return launch_kc(kernel, grid, block, smem, stream, dim3(1, 1, cluster_z > 1 ? cluster_z : 1), std::forward<Args>(args)...);
 }
 
 constexpr int GM_MAX_K_ = 7;
@@ -301,6 +308,7 @@ enum GemmEpilogue {
 };
 struct GemmArgs {
   CUtensorMap w_map, x_map;             // tcgen05 path only
+  CUtensorMap x_half_map;               // CTA-pair kernel only: activation boxes of block_t / 2 rows
   const __nv_bfloat16 *x, *w;
   void *out; int epi;
   int M, N, K;
@@ -313,6 +321,8 @@ struct GemmArgs {
   uint32_t *status;
 };
 cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream);
+// CTA-pair form (one K slice per tile, an even number of feature tiles, block_t a multiple of 32).
+cudaError_t launch_gemm_pair(const GemmArgs &A, cudaStream_t stream);
 cudaError_t launch_gemm_simple(const GemmArgs &A, cudaStream_t stream);
 // How many clusters of `nsplit` CTAs of the tcgen05 kernel can be resident at once (GPC packing).
 cudaError_t gemm_tc_max_clusters(int block_t, int nsplit, int *out);

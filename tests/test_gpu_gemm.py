@@ -88,3 +88,29 @@ def test_gate_up_projection_with_fused_swiglu_full_matrix(M):
     assert np.abs(o32.cpu().numpy() - ref).max() <= 3e-5 * np.abs(ref).max()
     assert np.abs(act.float().cpu().numpy() - act_ref).max() <= 6e-3 * np.abs(act_ref).max()
     ctx.close()
+
+
+@pytest.mark.parametrize("M", [256, 64, 96])
+def test_cta_pair_kernel_equals_single_cta_kernel(M, monkeypatch):
+    """The full wave of a wide projection runs on CTA pairs (one MMA over two SMs, each CTA staging half of the
+    activation box).  Same K order and the same accumulation per output as the single-CTA kernel: bit-identical."""
+    N, K = 19456, 2560
+    g = torch.Generator(device="cuda").manual_seed(100 + M)
+    x = torch.randn((M, K), device="cuda", generator=g).to(torch.bfloat16)
+    w = (torch.randn((N, K), device="cuda", generator=g) * 0.02).to(torch.bfloat16)
+    outs = []
+    for pair in (True, False):
+        if not pair:
+            monkeypatch.setenv("GM_NO_PAIR_GEMM", "1")
+        gmb, ctx = _ctx()
+        o32 = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        act = torch.full((M, N // 2), float("nan"), dtype=torch.bfloat16, device="cuda")
+        for rep in range(2):
+            gmb.gm_gemm(ctx, x, w, o32, M, N, K, True)
+            gmb.gm_gemm_swiglu(ctx, x, w, act, M, N, K)
+        assert gmb.gm_last_status(ctx) == 0
+        outs.append((o32.clone(), act.clone()))
+        ctx.close()
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    ref = (x.double() @ w.double().T).cpu().numpy()
+    assert np.abs(outs[0][0].cpu().numpy() - ref).max() <= 3e-5 * np.abs(ref).max()
