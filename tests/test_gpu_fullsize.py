@@ -1,0 +1,115 @@
+"""One whole cycle at the 4B dimensions (d 2560, 32/8 heads of 128, FFN 9728, vocabulary 151936), one decoder layer,
+64 sequences with 1.2k-7.9k cached positions in fragmented pages: the launch configuration the benchmark times
+(256-token GEMM tiles, cluster split-K, CTA pairs, the 148-CTA attention partition, CTA-per-sequence sampler).
+The oracle replays sampled sequences one by one from a snapshot of their pages."""
+import os
+import sys
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import philox, sampler as osampler, step as ostep
+from oracle.model import PagedKV
+
+from helpers import rel_err
+
+pytestmark = pytest.mark.gpu
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+TOL = 2e-2
+
+
+def _unpack_layer(lw, cfg):
+    f = lambda t: t.double().cpu().numpy()
+    q, kv = cfg.q_dim, cfg.kv_dim
+    wqkv, gu = f(lw["wqkv"]), f(lw["w_gate_up"])
+    return {"ln1": f(lw["ln1"]), "ln2": f(lw["ln2"]), "wq": wqkv[:q], "wk": wqkv[q:q + kv], "wv": wqkv[q + kv:],
+            "wo": f(lw["wo"]), "wg": gu[0::2], "wu": gu[1::2], "wd": f(lw["w_down"])}
+
+
+def _unpack_weights(packed, cfg):
+    """The library's fused bf16 layout -> the oracle's per-projection matrices, as float64."""
+    f = lambda t: t.double().cpu().numpy()
+    h = packed["head"]
+    return {"embed": f(packed["embed"]), "lm_head": f(packed["lm_head"]), "final_norm": f(packed["final_norm"]),
+            "layers": [_unpack_layer(lw, cfg) for lw in packed["layers"]],
+            "head": {"enorm": f(h["enorm"]), "hnorm": f(h["hnorm"]), "proj": f(h["proj"]),
+                     "final_norm": f(h["final_norm"]), "layer": _unpack_layer(h["layer"], cfg)}}
+
+
+def _snapshot(gst, cfg, b, K):
+    """The pages, lengths and pending pair of sequence b, as a one-sequence oracle state."""
+    L1 = int(gst.kv_len[b])
+    n_pages = (L1 + K + 1 + cfg.page_size - 1) // cfg.page_size
+    caches = []
+    for pool, table, layers in ((gst.kv_pool, gst.page_table, cfg.n_layers), (gst.head_kv_pool, gst.head_page_table, 1)):
+        phys = table[b, :n_pages].long()
+        kv = PagedKV(layers, cfg.n_kv_heads, cfg.head_dim, np.arange(n_pages)[None, :], n_pages, cfg.page_size)
+        kv.pool = pool[:, :, phys].double().cpu().numpy()
+        caches.append(kv)
+    n = int(gst.pending_n[b])
+    ptok = [int(t) for t in gst.pending_tok[b, :n].cpu()]
+    phid = gst.pending_hidden[b, :n].double().cpu().numpy()
+    seq = ostep.SeqState([0] * L1 + [ptok[-1]], phid, ptok)
+    return ostep.BatchState([seq], caches[0], caches[1], step=1)
+
+
+@pytest.mark.parametrize("name,K", [("4b", 3), ("7b", 3), ("4b", 5)])
+def test_full_dimension_cycle_on_sampled_sequences(name, K):
+    """4B: 16 query rows per KV head at K = 3, 24 at K = 5 (the transposed attention kernel); 7B dimensions
+    (d 3584, 28/4 heads, FFN 18944): 28 rows per KV head, two token blocks in the LM head."""
+    sys.path.insert(0, ROOT)
+    import bench
+    import paper_2609_16648_b200 as gmb
+    seed, step = 11, 1
+    cfg, ctx, gst, lens = bench.build_workload(name, 0, 2, K, "cuda", layers=1, batch=64)
+    B, V, d = cfg.batch, cfg.vocab, cfg.d_model
+    assert B == 64 and (name != "4b" or (V, d) == (151936, 2560))
+    g = torch.Generator(device="cuda").manual_seed(3)
+    norms = [ctx.packed["final_norm"]] + [ctx.packed["head"][n] for n in ("enorm", "hnorm", "final_norm")]
+    for lw in ctx.packed["layers"] + [ctx.packed["head"]["layer"]]:
+        norms += [lw["ln1"], lw["ln2"]]
+    for t in norms:                                           # a forgotten norm weight must show
+        t.copy_((1 + (torch.rand(t.shape, device="cuda", generator=g) - 0.5) * 0.5).to(torch.bfloat16))
+    sample = sorted({0, 21, 42, 63, int(np.argmax(lens)), int(np.argmin(lens))})
+    snaps = {b: _snapshot(gst, cfg, b, K) for b in sample}
+
+    z = lambda shape, dt: torch.zeros(shape, dtype=dt, device="cuda")
+    dtok, dl = z((B, K), torch.int32), z((B, K, V), torch.bfloat16)
+    tl, th = z((B, K + 1, V), torch.bfloat16), z((B, K + 1, d), torch.bfloat16)
+    q1, q2, p = z((B, K, V), torch.float32), z((B, K, V), torch.float32), z((B, K + 1, V), torch.float32)
+    a, t = z((B,), torch.int32), z((B,), torch.int32)
+    gmb.gm_draft(ctx, gst, K, 1.0, None, seed, step, dtok, dl, q1)
+    gmb.gm_verify(ctx, gst, K, dtok, tl, th)
+    gmb.gm_accept(ctx, gst, B, K, 1.0, tl, dl, dtok, None, seed, step, a, t, p, q2, th, commit_state=False)
+    assert gmb.gm_last_status(ctx) == 0
+    assert torch.equal(q1, q2)
+
+    # (1) every row: the device's draws and decisions are the oracle's decision function on the device's own p, q
+    ud, ua = philox.u24_draft(seed, step, B, K), philox.u24_accept(seed, step, B, K)
+    g_dtok, ga, gt = dtok.cpu().numpy(), a.cpu().numpy(), t.cpu().numpy()
+    qn, pn = q1.cpu().numpy(), p.cpu().numpy()
+    for b in range(B):
+        for k in range(K):
+            assert g_dtok[b, k] == osampler.draw_token(qn[b, k], ud[b, k])[0]
+        ea, et, _ = osampler.decide(pn[b], qn[b], g_dtok[b], ua[b])
+        assert (ea, et) == (int(ga[b]), int(gt[b]))
+
+    # (2) sampled sequences: the oracle's own forward passes along the device's drafts
+    w = _unpack_weights(ctx.packed, cfg)
+    worst, agree, total = 0.0, 0, 0
+    for b in sample:
+        ref = ostep.spec_step(w, cfg, snaps[b], K, 1.0, seed=seed, do_commit=False, u24_draft=ud[b:b + 1],
+                              u24_accept=ua[b:b + 1], forced_draft=g_dtok[b:b + 1])
+        for got, want in ((dl[b], ref["draft_logits"][0]), (tl[b], ref["target_logits"][0]), (th[b], ref["target_hidden"][0])):
+            worst = max(worst, rel_err(got.float().cpu().numpy(), want))
+        for j in range(K + 1):
+            worst = max(worst, rel_err(tl[b, j].float().cpu().numpy(), ref["target_logits"][0][j]))
+        both = min(int(ga[b]), int(ref["accept_len"][0]))
+        total += min(both + 1, K)
+        agree += both + (1 if (both < K and ga[b] == ref["accept_len"][0]) else 0)
+    print(f"sampled sequences {sample} (kv_len {[int(lens[b]) for b in sample]}): worst rel err {worst:.3e}, accept bits {agree}/{total}")
+    assert worst < TOL, worst
+    assert agree >= total - 1, (agree, total)
+    ctx.close()
