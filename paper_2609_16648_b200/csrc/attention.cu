@@ -57,8 +57,10 @@ __device__ __forceinline__ int cta_of_page(long long x, long long P, long long G
   return static_cast<int>(((x + 1) * G - 1) / P);
 }
 
-template <int HD, int MT>
-__global__ void __launch_bounds__((ATT_MAX_HPC + 1) * 32, 1)
+// RT > 1 (with MT = 1): RT warps per KV head, each owning one 16-row query tile (rows rt*16 ..) and consuming every page
+// of its head - more warps to hide latency where two tiles in one warp are bound by instruction issue.
+template <int HD, int MT, int RT = 1>
+__global__ void __launch_bounds__((ATT_MAX_HPC * RT + 1) * 32, 1)
 attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int nstages) {
   using C = AttCfg<HD>;
   constexpr int NSUB = C::NSUB;
@@ -78,7 +80,7 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
   const int B = A.batch;
   // barrier set-up touches shared memory only: it runs before the wait for the previous kernel
   if (threadIdx.x == 0) {
-    for (int s = 0; s < nstages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], hpc); }
+    for (int s = 0; s < nstages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], hpc * RT); }
     mbar_fence_init();
   }
   __syncthreads();
@@ -100,7 +102,7 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
     b0 = l;
   }
 
-  if (warp == hpc) {
+  if (warp == hpc * RT) {
     // ---- producer ------------------------------------------------------------------------------------------
     if (lane == 0) {
       tma_prefetch_desc(&A.kv_map);
@@ -125,10 +127,12 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
     }
     return;
   }
-  if (warp > hpc) return;
+  if (warp > hpc * RT) return;
 
   // ---- compute warp: KV head = hg*hpc + warp -------------------------------------------------------------------
-  const int head = hg * hpc + warp;
+  const int hw = warp % hpc, rt = warp / hpc;     // head within the CTA, row tile
+  const int head = hg * hpc + hw;
+  const int row0 = rt * 16;
   const int t4 = lane & 3, r8 = lane >> 2;
   const float c = A.scale_log2e;
   const uint32_t smem_base = smem_u32(smem);
@@ -136,7 +140,7 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
   const int mi = lane >> 3;
   const int k_tok = (mi >> 1) * 8 + (lane & 7), k_chunk = mi & 1;        // K: non-transposed
   const int v_tok = (mi & 1) * 8 + (lane & 7), v_chunk = mi >> 1;        // V: transposed
-  const uint32_t k_row_off = (warp * 16 + k_tok) * 128, v_row_off = (warp * 16 + v_tok) * 128;
+  const uint32_t k_row_off = (hw * 16 + k_tok) * 128, v_row_off = (hw * 16 + v_tok) * 128;
   const int k_sw = k_tok & 7, v_sw = v_tok & 7;
 
   int it = 0;
@@ -150,14 +154,16 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
 
     // query fragments: in registers for one 16-row tile; staged in shared memory (128-byte rows, XOR swizzle)
     // for two tiles and fetched per page
-    constexpr int QREG = MT == 1 ? KSTEPS : 1;
+    constexpr bool QSM = MT > 1 || RT > 1;        // Q staged in shared memory (register pressure)
+    constexpr int QROWS = MT * 16;                // rows this warp stages
+    constexpr int QREG = QSM ? 1 : KSTEPS;
     uint32_t qf[MT][QREG][4];
     const __nv_bfloat16 *qp = A.qbuf + (static_cast<size_t>(b) * A.n_kv + head) * A.qrows * HD;
-    const uint32_t q_smem = smem_u32(qsm) + warp * (32 * HD * 2);
-    if constexpr (MT == 1) {
+    const uint32_t q_smem = smem_u32(qsm) + warp * (QROWS * HD * 2);
+    if constexpr (!QSM) {
 #pragma unroll
       for (int ks = 0; ks < KSTEPS; ++ks) {
-        const __nv_bfloat16 *r0 = qp + r8 * HD + ks * 16 + 2 * t4;
+        const __nv_bfloat16 *r0 = qp + (row0 + r8) * HD + ks * 16 + 2 * t4;
         qf[0][ks][0] = *reinterpret_cast<const uint32_t *>(r0);
         qf[0][ks][1] = *reinterpret_cast<const uint32_t *>(r0 + 8 * HD);
         qf[0][ks][2] = *reinterpret_cast<const uint32_t *>(r0 + 8);
@@ -166,10 +172,10 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
     } else {
       __syncwarp();                               // the previous segment's fragment reads are done
       constexpr int CPR = HD / 8;                 // 16-byte chunks per row
-      for (int idx = lane; idx < 32 * CPR; idx += 32) {
+      for (int idx = lane; idx < QROWS * CPR; idx += 32) {
         const int row = idx / CPR, ch = idx % CPR;
-        const uint4 v = *reinterpret_cast<const uint4 *>(qp + row * HD + ch * 8);
-        unsigned char *dst = qsm + warp * (32 * HD * 2) + (ch >> 3) * (32 * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4);
+        const uint4 v = *reinterpret_cast<const uint4 *>(qp + (row0 + row) * HD + ch * 8);
+        unsigned char *dst = qsm + warp * (QROWS * HD * 2) + (ch >> 3) * (QROWS * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4);
         *reinterpret_cast<uint4 *>(dst) = v;
       }
       __syncwarp();
@@ -202,12 +208,12 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
         ldmatrix_x4(kf, kbase + (ks >> 2) * tile_b + k_row_off + ((chunk ^ k_sw) << 4));
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-          if constexpr (MT == 1) {
+          if constexpr (!QSM) {
             mma_16816(sc[mt][0], qf[mt][ks], kf[0], kf[1]);
             mma_16816(sc[mt][1], qf[mt][ks], kf[2], kf[3]);
           } else {
             const int row = mt * 16 + q_row;
-            ldmatrix_x4(qf[mt][0], q_smem + (ks >> 2) * (32 * 128) + row * 128 + ((((ks & 3) * 2 + q_chunk) ^ (row & 7)) << 4));
+            ldmatrix_x4(qf[mt][0], q_smem + (ks >> 2) * (QROWS * 128) + row * 128 + ((((ks & 3) * 2 + q_chunk) ^ (row & 7)) << 4));
             mma_16816(sc[mt][0], qf[mt][0], kf[0], kf[1]);
             mma_16816(sc[mt][1], qf[mt][0], kf[2], kf[3]);
           }
@@ -223,7 +229,7 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
         if (need_mask) {
 #pragma unroll
           for (int hrow = 0; hrow < 2; ++hrow) {
-            const int j = (mt * 16 + r8 + hrow * 8) / A.group;
+            const int j = (row0 + mt * 16 + r8 + hrow * 8) / A.group;
             const int lim = j < qn ? qbase + j : -1;
 #pragma unroll
             for (int n = 0; n < 2; ++n)
@@ -295,7 +301,7 @@ attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int ns
         float l = lrow[mt][hrow];
         l += __shfl_xor_sync(0xffffffffu, l, 1);
         l += __shfl_xor_sync(0xffffffffu, l, 2);
-        const int row = mt * 16 + r8 + hrow * 8;
+        const int row = row0 + mt * 16 + r8 + hrow * 8;
         if (row < rows_valid) {
           if (t4 == 0) {
             pml[row * 2 + 0] = mrow[mt][hrow] == -INFINITY ? -INFINITY : mrow[mt][hrow] * c;
@@ -565,19 +571,20 @@ static cudaError_t launch_att_t(const AttnArgs &A, cudaStream_t stream) {
   return launch_k(attention_t_kernel<HD, NR>, grid, dim3((hpc + 1) * 32), smem, stream, 1, A, hpc, nst);
 }
 
-template <int HD, int MT>
+template <int HD, int MT, int RT = 1>
 static cudaError_t launch_att(const AttnArgs &A, cudaStream_t stream) {
-  const int hpc = att_hpc(A.n_kv), nst = att_stages(A.n_kv, HD, MT);
-  const size_t smem = attention_smem_bytes(A.n_kv, HD, MT);
+  // the variants that stage Q in shared memory share one layout: 32 rows x head_dim per KV head
+  const int hpc = att_hpc(A.n_kv), nst = att_stages(A.n_kv, HD, MT * RT);
+  const size_t smem = attention_smem_bytes(A.n_kv, HD, MT * RT);
   static size_t configured = 0;
   if (smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(attention_kernel<HD, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(attention_kernel<HD, MT, RT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(smem));
     if (e != cudaSuccess) return e;
     configured = smem;
   }
   dim3 grid(A.n_ctas, A.n_kv / hpc);
-  return launch_k(attention_kernel<HD, MT>, grid, dim3((hpc + 1) * 32), smem, stream, 1, A, hpc, nst);
+  return launch_k(attention_kernel<HD, MT, RT>, grid, dim3((hpc * RT + 1) * 32), smem, stream, 1, A, hpc, nst);
 }
 
 cudaError_t launch_attention(const AttnArgs &A, cudaStream_t stream) {
@@ -587,6 +594,9 @@ cudaError_t launch_attention(const AttnArgs &A, cudaStream_t stream) {
   static const bool no_t = std::getenv("GM_NO_ATT_T") != nullptr;
   if (!no_t && A.hd == 128 && mt == 2 && A.rows_used > 16 && A.rows_used <= 24) return launch_att_t<128, 3>(A, stream);
   if (A.hd == 128 && mt == 1) return launch_att<128, 1>(A, stream);
+  // 25..32 query rows: two warps per KV head, one 16-row tile each (GM_NO_ATT_RT2: one warp with two tiles)
+  static const bool no_rt2 = std::getenv("GM_NO_ATT_RT2") != nullptr;
+  if (!no_rt2 && A.hd == 128 && mt == 2) return launch_att<128, 1, 2>(A, stream);
   if (A.hd == 128 && mt == 2) return launch_att<128, 2>(A, stream);
   if (A.hd == 64 && mt == 1) return launch_att<64, 1>(A, stream);
   if (A.hd == 64 && mt == 2) return launch_att<64, 2>(A, stream);
