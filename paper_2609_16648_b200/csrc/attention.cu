@@ -58,7 +58,8 @@ __device__ __forceinline__ int cta_of_page(long long x, long long P, long long G
 }
 
 // RT > 1 (with MT = 1): RT warps per KV head, each owning one 16-row query tile (rows rt*16 ..) and consuming every page
-// of its head - more warps to hide latency where two tiles in one warp are bound by instruction issue.
+// of its head - more warps to hide latency where two tiles in one warp are bound by instruction issue.  17 warps are
+// allocated as 20 (granularity 4), which leaves 96 registers per thread: a few spills; 112 or 120 do not launch.
 template <int HD, int MT, int RT = 1>
 __global__ void __launch_bounds__((ATT_MAX_HPC * RT + 1) * 32, 1)
 attention_kernel(const __grid_constant__ AttnArgs A, const int hpc, const int nstages) {
