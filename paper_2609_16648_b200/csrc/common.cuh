@@ -162,7 +162,8 @@ __device__ __forceinline__ void tc2_mma_bf16(uint32_t d_tmem, uint64_t a_desc, u
       : "memory");
 }
 // Arrives, once every pair MMA issued so far has completed in both CTAs, on the mbarrier at this offset in every CTA
-// of the cluster whose bit is set in `cta_mask`.
+// of the cluster whose bit is set in `cta_mask`.  (A barrier arrival only: no data is copied.  Two separate commits,
+// one per CTA's barrier address, also work and cost about 1 us more per launch.)
 __device__ __forceinline__ void tc2_commit_mc(uint64_t *bar, uint16_t cta_mask) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                ::"r"(smem_u32(bar)), "h"(cta_mask)
