@@ -2,6 +2,36 @@
 // Host code only; the helpers it calls are declared in gm_internal.h.
 #include "gm_internal.h"
 
+// Virtual rows per sequence for a prefill pass (at most the count the workspaces were sized for).  A pass of m
+// 256-token blocks runs every projection as ceil(tiles * m / SMs) waves, and with a few hundred tokens more or less
+// a projection can need a whole extra wave (20 feature tiles x 8 blocks = 160 CTAs on 148 SMs); the cost per token of
+// each candidate is estimated from the wave counts with the same tiling rules the projections use, and the cheapest
+// wins.  GM_PREFILL_VR forces a value.
+static int pick_prefill_vr(const gm_ctx *c, int B, int QT) {
+  const int vr_max = c->pf_vr;
+  if (const char *ov = std::getenv("GM_PREFILL_VR")) {
+    const int v = std::atoi(ov);
+    if (v >= 1 && v <= vr_max) return v;
+  }
+  const int sms = c->sm_count;
+  const int shape[4][2] = {{c->n_qkv, c->d}, {c->d, c->q_dim}, {2 * c->F, c->d}, {c->d, c->F}};   // (N, K) per projection
+  int best = vr_max;
+  double best_cost = 0.0;
+  for (int vr = vr_max; vr >= 1; --vr) {
+    const int rows = B * vr * QT, m = (rows + 255) / 256;
+    double cost = 0.0;
+    for (const auto &g : shape) {
+      const int tiles = (g[0] + 127) / 128, kb = g[1] / 64;
+      const int wt = tiles * m >= 2 * sms ? 2 : 1;
+      const int ctas = ((tiles + wt - 1) / wt) * m;
+      cost += static_cast<double>((ctas + sms - 1) / sms) * kb * wt + 24.0;            // + fixed cost of a launch
+    }
+    cost /= rows;
+    if (vr == vr_max || cost < best_cost * 0.97) { best = vr; best_cost = cost; }
+  }
+  return best;
+}
+
 extern "C" {
 
 int gm_prefill(gm_ctx *c, gm_state *st, const int32_t *prompt_tok, const int32_t *prompt_len, int prompt_stride,
@@ -18,7 +48,7 @@ int gm_prefill(gm_ctx *c, gm_state *st, const int32_t *prompt_tok, const int32_t
   // Every pass gives each prompt VR consecutive chunks of QT positions: VR "virtual rows" per sequence, which the
   // planner, the rotary/append kernel and attention treat as independent sequences sharing the prompt's page table
   // (all keys of the pass are appended before attention runs, and each row attends only positions up to its own).
-  const int B = st->batch, QT = cf.max_k + 1, VR = c->pf_vr, R = B * VR;
+  const int B = st->batch, QT = cf.max_k + 1, VR = pick_prefill_vr(c, B, QT), R = B * VR;
   PhaseShape ph;
   ph.B = R; ph.QT = QT; ph.M = R * QT; ph.qrows = round16(QT * c->group);
   CUtensorMap kvm, hkvm;
