@@ -35,6 +35,24 @@ def test_gemm_matches_fp64_matmul(M, N, K, out_fp32):
     ctx.close()
 
 
+def test_gemm_argument_checks():
+    gmb, ctx = _ctx()
+    x = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros((24, 64), dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros((4, 24), dtype=torch.bfloat16, device="cuda")
+    for call, code in ((lambda: gmb.gm_gemm(ctx, x, w, out, 4, 24, 48, False), gmb.GM_ERR_UNSUPPORTED),      # K % 64
+                       (lambda: gmb.gm_gemm(ctx, x, w, out, 4, 20, 64, False), gmb.GM_ERR_UNSUPPORTED),      # N % 8
+                       (lambda: gmb.gm_gemm_swiglu(ctx, x, w, out, 4, 24, 64), gmb.GM_ERR_UNSUPPORTED),      # N % 16
+                       (lambda: gmb.gm_gemm(ctx, x, w, out, 0, 24, 64, False), gmb.GM_ERR_INVALID_ARG),
+                       (lambda: gmb.gm_gemm(ctx, x, None, out, 4, 24, 64, False), gmb.GM_ERR_INVALID_ARG)):
+        with pytest.raises(gmb.GmError) as e:
+            call()
+        assert e.value.code == code
+    gmb.gm_gemm(ctx, x, w, out, 4, 24, 64, False)
+    assert gmb.gm_last_status(ctx) == 0
+    ctx.close()
+
+
 def test_simple_kernel_agrees():
     gmb, ctx = _ctx(flags=1)
     M, N, K = 70, 200, 192

@@ -189,6 +189,19 @@ def test_gradient_kernel_full_vocabulary_and_edge_cases():
     got = grad.float().cpu().numpy()
     _check_grad(got, head, recs, Tg)
     assert any(r["accepted"] == 1 for r in recs) and any(r["accepted"] == K + 1 for r in recs)
+    # argument checks of the update entry points: nothing is launched
+    for bad in (dict(temperature=0.0), dict(temperature=float("nan")), dict(k=8), dict(n=0)):
+        with pytest.raises(gmb.GmError) as e:
+            gmb.gm_dca_grad(ctx, bad.get("n", n), bad.get("k", K), bad.get("temperature", Tg), logits, rec, alpha,
+                            rec.accepted, grad, lse)
+        assert e.value.code == (gmb.GM_ERR_UNSUPPORTED if "temperature" in bad else gmb.GM_ERR_INVALID_ARG)
+    with pytest.raises(gmb.GmError) as e:
+        gmb.gm_overlap(ctx, n, K, -1.0, logits, rec, alpha)
+    assert e.value.code == gmb.GM_ERR_UNSUPPORTED
+    with pytest.raises(gmb.GmError) as e:
+        gmb.gm_dca_grad(ctx, n, K, Tg, logits, rec, None, rec.accepted, grad)
+    assert e.value.code == gmb.GM_ERR_INVALID_ARG
+    assert gmb.gm_last_status(ctx) == 0
     # a dead chain (first overlap 0) has no finite objective: its rows are written as zeros
     alpha[2, 0] = 0.0
     gmb.gm_dca_grad(ctx, n, K, Tg, logits, rec, alpha, rec.accepted, grad)
