@@ -54,10 +54,10 @@ static size_t gt_smem(int block_t, int wt) {
 __device__ __forceinline__ void epilogue4(const GemmArgs &A, int m, int n, float4 v) {
   if (A.epi == EPI_SWIGLU_BF16) {           // (gate, up, gate, up) -> two outputs
     if (n + 1 >= A.N) return;
-    const float a0 = v.x / (1.f + __expf(-v.x)) * v.y;
+    const float a0 = __fdividef(v.x, 1.f + __expf(-v.x)) * v.y;        // fast reciprocal: the result is rounded to bf16
     __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(A.out) + static_cast<size_t>(m) * A.ldo + (n >> 1);
     if (n + 3 < A.N) {
-      const float a1 = v.z / (1.f + __expf(-v.z)) * v.w;
+      const float a1 = __fdividef(v.z, 1.f + __expf(-v.z)) * v.w;
       *reinterpret_cast<uint32_t *>(out) = pack_bf16(a0, a1);
     } else {
       out[0] = __float2bfloat16(a0);
