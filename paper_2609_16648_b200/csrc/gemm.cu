@@ -27,6 +27,7 @@
 // independent on-device cross-check and for shapes the tcgen05 kernel does not take.
 #include <cooperative_groups.h>
 
+#include <cstdlib>
 #include "common.cuh"
 #include "kernels.h"
 
@@ -90,7 +91,8 @@ __device__ __forceinline__ void epilogue4(const GemmArgs &A, int m, int n, float
   }
 }
 
-__global__ void __launch_bounds__(GT_THREADS, 1)
+template <int MINB>
+__global__ void __launch_bounds__(GT_THREADS, MINB)
 gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
   extern __shared__ unsigned char gt_smem_raw[];
   unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(gt_smem_raw) + 1023) & ~uintptr_t(1023));
@@ -344,7 +346,7 @@ gemm_pair_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
 static cudaError_t gt_configure() {
   static bool done = false;
   if (done) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess) done = true;
   return e;
 }
@@ -354,7 +356,7 @@ cudaError_t gemm_tc_max_clusters(int block_t, int nsplit, int *out) {
   cudaError_t e = gt_configure();
   if (e != cudaSuccess) return e;
   if (nsplit > 8) {
-    e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    e = cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
   }
   cudaLaunchConfig_t cfg = {};
@@ -366,7 +368,7 @@ cudaError_t gemm_tc_max_clusters(int block_t, int nsplit, int *out) {
   attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = nsplit;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaOccupancyMaxActiveClusters(out, gemm_tc_kernel, &cfg);
+  return cudaOccupancyMaxActiveClusters(out, gemm_tc_kernel<1>, &cfg);
 }
 
 static int pair_stages(int T) {
@@ -401,7 +403,27 @@ cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream) {
   cudaError_t ec = gt_configure();
   if (ec != cudaSuccess) return ec;
   const dim3 grid((A.M + T - 1) / T, A.n_tiles, A.nsplit);
-  return launch_k(gemm_tc_kernel, grid, dim3(GT_THREADS), smem, stream, A.nsplit, A, gt_stages(T, A.wtiles));
+  // Few tokens, many tiles per SM (the draft phase's LM head): two CTAs per SM with half the ring each, so that one
+  // CTA's epilogue and its successor's first fill run under the other's main loop.
+  static const bool no_two = std::getenv("GM_NO_GEMM_2CTA") != nullptr;
+  if (!no_two && A.nsplit == 1 && T <= 64 && static_cast<long long>(grid.x) * grid.y >= 4LL * 148) {
+    const int stage = A.wtiles * GT_BN * 128 + T * 128;
+    int st = (100 * 1024) / stage;
+    if (st >= 2) {
+      if (st > 8) st = 8;
+      size_t pipe = static_cast<size_t>(st) * stage;
+      const size_t park = static_cast<size_t>(T) * GT_BN * 4;
+      if (park > pipe) pipe = park;
+      static bool done2 = false;
+      if (!done2) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024);
+        if (e != cudaSuccess) return e;
+        done2 = true;
+      }
+      return launch_k(gemm_tc_kernel<2>, grid, dim3(GT_THREADS), pipe + 1024 + 256, stream, 1, A, st);
+    }
+  }
+  return launch_k(gemm_tc_kernel<1>, grid, dim3(GT_THREADS), smem, stream, A.nsplit, A, gt_stages(T, A.wtiles));
 }
 
 // ---- plain mma.sync GEMM ----------------------------------------------------------------------------------------------
