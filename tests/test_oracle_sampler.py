@@ -363,3 +363,21 @@ def test_cycle_with_truncated_target_follows_the_truncated_law():
     obs = np.bincount(first, minlength=v)[support]
     chi = stats.chisquare(obs, pf[0][support].astype(np.float64) / pf[0][support].sum(dtype=np.float64) * n)
     assert chi.pvalue > 1e-4, chi
+
+
+def test_overlap_is_one_lipschitz_in_the_target_and_the_chain_bound_follows():
+    """App. F: when the target moves from p to p' the overlap with a fixed head moves by at most TV(p, p'), and the
+    expected accepted length of a depth-K chain by at most K(K+1)/2 times the largest such move."""
+    rng = np.random.default_rng(21)
+    for trial in range(200):
+        K = int(rng.integers(1, 8))
+        q = [_dist(rng) for _ in range(K)]
+        p0 = [_dist(rng) for _ in range(K)]
+        mix = rng.uniform(0, 0.3)
+        p1 = [((1 - mix) * p0[k] + mix * _dist(rng)).astype(np.float32) for k in range(K)]
+        a0 = np.array([sampler.acceptance_probability(p0[k], q[k]) for k in range(K)])
+        a1 = np.array([sampler.acceptance_probability(p1[k], q[k]) for k in range(K)])
+        tv = np.array([0.5 * np.abs(p0[k].astype(np.float64) - p1[k].astype(np.float64)).sum() for k in range(K)])
+        assert (np.abs(a1 - a0) <= tv + 1e-6).all()
+        gap = abs(sampler.expected_accepted_length(a1) - sampler.expected_accepted_length(a0))
+        assert gap <= K * (K + 1) / 2 * tv.max() + 1e-6
