@@ -442,6 +442,16 @@ int gm_attention_noalloc(int n_q_heads, int n_kv_heads, int head_dim, int max_pa
 int gm_profile(gm_ctx *ctx, int class_mask);
 int gm_profile_read(gm_ctx *ctx, int kernel_class, double *total_ms, int64_t *launches);
 
+/* Timeline of the persistent projection-chain kernel (the launch that runs a layer's output projection,
+ * feed-forward block and the next layer's QKV projection back to back; a design choice of this library, the
+ * paper describes no kernel).  gm_chain_trace(ctx, 1) makes later chain launches write nanosecond stamps of
+ * their CTAs' phase transitions into a buffer the context allocates on the first call; gm_chain_trace(ctx, 0)
+ * stops it.  gm_chain_trace_read waits for the stream and copies the stamps of the LAST traced launch to
+ * `out` (host memory, `capacity` 64-bit words): 64 words per CTA (slot meaning: see csrc/chain.cu); returns
+ * the number of words written (2 x CTA pairs x 64), or a negative GM_ERR_*.                               */
+int gm_chain_trace(gm_ctx *ctx, int enable);
+int gm_chain_trace_read(gm_ctx *ctx, uint64_t *out, int capacity);
+
 /* Number of kernels this library launched since gm_init (all calls).                        */
 int64_t gm_launch_count(gm_ctx *ctx);
 

@@ -26,7 +26,7 @@ EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_sp
            "gm_rollout_begin", "gm_rollout_step", "gm_rollout_run", "gm_pages_reset", "gm_pages_reserve",
            "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_overlap", "gm_dca_loss", "gm_dca_grad",
            "gm_spec_step_host", "gm_gemm", "gm_gemm_swiglu", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
-           "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_launch_count",
+           "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_chain_trace", "gm_chain_trace_read", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
 
 
@@ -111,6 +111,8 @@ def lib() -> C.CDLL:
     L.gm_spec_step_rec.argtypes = [vp, C.POINTER(gm_state), i32, f32, u64, u64, vp, vp, vp, C.POINTER(gm_record)]
     L.gm_profile.argtypes = [vp, i32]
     L.gm_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    L.gm_chain_trace.argtypes = [vp, i32]
+    L.gm_chain_trace_read.argtypes = [vp, vp, i32]
     L.gm_launch_count.argtypes = [vp]
     L.gm_launch_count.restype = C.c_int64
     L.gm_last_status.argtypes = [vp]
@@ -498,6 +500,20 @@ def gm_profile_read(ctx: Context, kernel_class: int):
     ms, n = C.c_double(), C.c_int64()
     _check(lib().gm_profile_read(ctx.handle, kernel_class, C.byref(ms), C.byref(n)), "gm_profile_read")
     return ms.value, n.value
+
+
+def gm_chain_trace(ctx: Context, enable: bool):
+    _check(lib().gm_chain_trace(ctx.handle, 1 if enable else 0), "gm_chain_trace")
+
+
+def gm_chain_trace_read(ctx: Context):
+    """Stamps of the last traced chain launch as an int64 array [CTAs, 64] (nanoseconds; 0 = slot not reached)."""
+    import numpy as np
+    buf = np.zeros(1024 * 64, dtype=np.uint64)
+    n = lib().gm_chain_trace_read(ctx.handle, buf.ctypes.data_as(C.c_void_p), buf.size)
+    if n < 0:
+        raise GmError(n, "gm_chain_trace_read")
+    return buf[:n].astype(np.int64).reshape(-1, 64)
 
 
 def gm_launch_count(ctx: Context) -> int:

@@ -129,4 +129,26 @@ int gm_attention(gm_ctx *c, const void *q, const void *kv_pool, int pool_layers,
   return GM_OK;
 }
 
+int gm_chain_trace(gm_ctx *c, int enable) {
+  if (!c) return GM_ERR_INVALID_ARG;
+  if (!c->chain_on) return GM_ERR_UNSUPPORTED;
+  if (enable && !c->chain_trace) {
+    int rc = dev_alloc(c, &c->chain_trace, static_cast<size_t>(c->chain_pairs) * 2 * 64);
+    if (rc != GM_OK) return rc;
+  }
+  c->chain_trace_on = enable != 0;
+  return GM_OK;
+}
+
+int gm_chain_trace_read(gm_ctx *c, uint64_t *out, int capacity) {
+  if (!c || !out || capacity < 0) return GM_ERR_INVALID_ARG;
+  if (!c->chain_trace) return GM_ERR_UNSUPPORTED;
+  const int words = c->chain_pairs * 2 * 64;
+  if (capacity < words) return GM_ERR_INVALID_ARG;
+  GM_CUDA(c, cudaStreamSynchronize(c->stream));
+  GM_CUDA(c, cudaMemcpy(out, c->chain_trace, static_cast<size_t>(words) * sizeof(uint64_t), cudaMemcpyDeviceToHost));
+  return words;
+}
+
+
 }  // extern "C"

@@ -73,7 +73,8 @@ int gm_prefill(gm_ctx *c, gm_state *st, const int32_t *prompt_tok, const int32_t
       const bool last = l + 1 == cf.n_layers;
       rc = run_layer(c, c->layers[l], c->lmaps[l], ph, kvm, static_cast<__nv_bfloat16 *>(st->kv_pool), l, cf.num_pages,
                      c->pf_vtable[0], last ? nullptr : static_cast<const __nv_bfloat16 *>(c->layers[l + 1].ln1),
-                     last ? c->pf_hidden : nullptr);
+                     last ? c->pf_hidden : nullptr, last ? nullptr : &c->layers[l + 1], last ? nullptr : &c->lmaps[l + 1],
+                     l > 0);
       if (rc) return rc;
     }
     if (c->capture)

@@ -132,18 +132,56 @@ int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *w
   return GM_OK;
 }
 
+bool chain_usable(const gm_ctx *c, int M) { return c->chain_on && M <= c->chain_max_m; }
+
+// A chain of dependent projections as one persistent launch.
+int run_chain(gm_ctx *c, const ChainSpec *specs, int n, int M) {
+  ChainArgs A;
+  std::memset(&A, 0, sizeof(A));
+  A.n_phases = n; A.M = M; A.mblocks = (M + 255) / 256; A.P = c->chain_pairs; A.m_pad = c->Mmax;
+  A.eps = c->cfg.rms_eps; A.partial = c->chain_partial; A.sync = c->chain_sync; A.status = c->status;
+  A.timeline = c->chain_trace_on ? c->chain_trace : nullptr;
+  A.npw = c->chain_npw; A.npa = c->chain_npa;
+  A.trace_phase = std::getenv("GM_CHAIN_TRACE_PHASE") ? std::atoi(std::getenv("GM_CHAIN_TRACE_PHASE")) : 1;
+  for (int p = 0; p < n; ++p) {
+    const ChainSpec &s = specs[p];
+    ChainPhase &ph = A.ph[p];
+    ph.w_map = *s.wmap;
+    // rows beyond M are out of the map's bounds: the copy engine fills them with zeros and fetches nothing
+    int rc = x_map(c, s.x, M < s.x_rows ? M : s.x_rows, s.K, 128, &ph.x_map);
+    if (rc != GM_OK) return rc;
+    ph.out = s.out; ph.xg = s.xg; ph.gamma = s.gamma; ph.sq_out = s.sq_out; ph.sq_in = s.sq_in;
+    ph.sq_groups = s.sq_in ? (s.norm_dim + 63) / 64 : 0;
+    ph.inv_dim = s.sq_in ? 1.0f / static_cast<float>(s.norm_dim) : 0.f;
+    ph.epi = s.epi; ph.N = s.N; ph.K = s.K; ph.ldo = s.ldo;
+    chain_schedule(ph, A.mblocks, A.P);
+  }
+  GM_LAUNCH(c, GM_KC_GEMM, launch_chain(A, c->stream));
+  return GM_OK;
+}
+
 // One decoder layer on rows x/xn [M, d] (xn = normed input).  `next_norm` is the RMSNorm weight applied to
 // the layer's output for whatever consumes it next (null: none); `hidden_out` optionally receives the
 // bf16 residual stream.
 int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const PhaseShape &ph, const CUtensorMap &kvm,
               __nv_bfloat16 *pool, int layer, int num_pages, const int32_t *page_table,
-              const __nv_bfloat16 *next_norm, __nv_bfloat16 *hidden_out) {
+              const __nv_bfloat16 *next_norm, __nv_bfloat16 *hidden_out, const gm_layer_weights *next_lw,
+              const LayerMaps *next_lm, bool qkv_done) {
   const gm_config &cf = c->cfg;
+  const bool chain = chain_usable(c, ph.M);
   int rc;
   // QKV projection (bf16) -> rotary + KV append + Q rearrangement
-  rc = run_gemm(c, c->xn, c->Mmax, &lm.wqkv, static_cast<const __nv_bfloat16 *>(lw.wqkv), ph.M, c->n_qkv, c->d,
-                c->qkv, EPI_STORE_BF16, c->n_qkv);
-  if (rc) return rc;
+  if (!(chain && qkv_done)) {
+    if (chain) {
+      const ChainSpec q = {&lm.wqkv, c->xn, c->Mmax, c->n_qkv, c->d, c->qkv, EPI_STORE_BF16, c->n_qkv,
+                           nullptr, nullptr, nullptr, nullptr, 0};
+      rc = run_chain(c, &q, 1, ph.M);
+    } else {
+      rc = run_gemm(c, c->xn, c->Mmax, &lm.wqkv, static_cast<const __nv_bfloat16 *>(lw.wqkv), ph.M, c->n_qkv, c->d,
+                    c->qkv, EPI_STORE_BF16, c->n_qkv);
+    }
+    if (rc) return rc;
+  }
   RopeAppendArgs R;
   R.qkv = c->qkv;
   R.batch = ph.B; R.QT = ph.QT; R.n_q = cf.n_q_heads; R.n_kv = cf.n_kv_heads; R.hd = cf.head_dim; R.layer = layer;
@@ -167,6 +205,27 @@ int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const 
   Cb.n_kv = cf.n_kv_heads; Cb.group = c->group; Cb.hd = cf.head_dim; Cb.qrows = ph.qrows; Cb.QT = ph.QT;
   Cb.n_ctas = c->sm_count; Cb.out = c->attn_out;
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_attention_combine(Cb, c->stream));
+  if (chain) {
+    // output projection (+ residual), gate/up (+ SwiGLU), down (+ residual) and the next layer's QKV in one launch;
+    // the two norms in between are folded around the projections (see chain.cu)
+    const bool fuse_next = next_lw && next_lm && next_norm;
+    ChainSpec sp[4];
+    sp[0] = {&lm.wo, c->attn_out, c->Mmax, c->d, c->q_dim, c->x, EPI_ADD_F32, c->d,
+             c->xn, static_cast<const __nv_bfloat16 *>(lw.ln2), c->chain_sq[0], nullptr, 0};
+    sp[1] = {&lm.wgu, c->xn, c->Mmax, 2 * c->F, c->d, c->act, EPI_SWIGLU_BF16, c->F,
+             nullptr, nullptr, nullptr, c->chain_sq[0], c->d};
+    sp[2] = {&lm.wdown, c->act, c->Mmax, c->d, c->F, c->x, EPI_ADD_F32, c->d,
+             fuse_next ? c->xn : nullptr, fuse_next ? next_norm : nullptr, fuse_next ? c->chain_sq[1] : nullptr, nullptr, 0};
+    if (fuse_next)
+      sp[3] = {&next_lm->wqkv, c->xn, c->Mmax, c->n_qkv, c->d, c->qkv, EPI_STORE_BF16, c->n_qkv,
+               nullptr, nullptr, nullptr, c->chain_sq[1], c->d};
+    if ((rc = run_chain(c, sp, fuse_next ? 4 : 3, ph.M)) != GM_OK) return rc;
+    if (!fuse_next && (next_norm || hidden_out))
+      GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+                launch_rmsnorm(c->x, next_norm, next_norm ? c->xn : nullptr, hidden_out, ph.M, c->d, cf.rms_eps,
+                               c->stream));
+    return GM_OK;
+  }
   // output projection added into the residual stream, then the post-attention norm
   rc = run_gemm(c, c->attn_out, c->Mmax, &lm.wo, static_cast<const __nv_bfloat16 *>(lw.wo), ph.M, c->d, c->q_dim,
                 c->x, EPI_ADD_F32, c->d);
@@ -372,6 +431,24 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
   A_(dev_alloc(c, &c->pf_hidden, M * c->d));
   A_(dev_alloc(c, &c->pf_xlast, B1 * c->d));
   A_(dev_alloc(c, &c->status, 1));
+  // persistent chain of a layer's projections: every CTA pair must be resident at once
+  if (std::getenv("GM_NO_CHAIN") == nullptr && !(cfg->flags & GM_FLAG_SIMPLE_GEMM) && (c->q_dim % 64) == 0) {
+    int pairs = 0;
+    if (chain_max_pairs(&pairs) != cudaSuccess) { pairs = 0; (void)cudaGetLastError(); }
+    if (pairs > c->sm_count / 2) pairs = c->sm_count / 2;
+    if (const char *ov = std::getenv("GM_CHAIN_PAIRS")) { const int v = std::atoi(ov); if (v >= 1 && v < pairs) pairs = v; }
+    if (const char *ov = std::getenv("GM_CHAIN_NPW")) c->chain_npw = std::atoi(ov) == 1 ? 1 : 2;
+    if (const char *ov = std::getenv("GM_CHAIN_NPA")) c->chain_npa = std::atoi(ov) == 1 ? 1 : 2;
+    if (const char *ov = std::getenv("GM_CHAIN_MAX_M")) { const int v = std::atoi(ov); if (v >= 1) c->chain_max_m = v; }
+    if (pairs >= 1) {
+      c->chain_pairs = pairs;
+      A_(dev_alloc(c, &c->chain_partial, static_cast<size_t>(pairs) * 2 * 256 * 128));
+      A_(dev_alloc(c, &c->chain_sq[0], static_cast<size_t>((c->d + 31) / 32) * M));
+      A_(dev_alloc(c, &c->chain_sq[1], static_cast<size_t>((c->d + 31) / 32) * M));
+      A_(dev_alloc(c, &c->chain_sync, 4 + static_cast<size_t>(pairs) * 4));
+      c->chain_on = true;
+    }
+  }
   // rotary table: cos/sin of pos * base^(-2i/hd), computed in double precision on the host
   {
     const int half = cfg->head_dim / 2;
@@ -487,7 +564,8 @@ int gm_verify(gm_ctx *c, const gm_state *st, int k, const int32_t *draft_tok, vo
     const __nv_bfloat16 *next_norm =
         static_cast<const __nv_bfloat16 *>(last ? c->w.final_norm : c->layers[l + 1].ln1);
     rc = run_layer(c, c->layers[l], c->lmaps[l], ph, kvm, static_cast<__nv_bfloat16 *>(st->kv_pool), l, cf.num_pages,
-                   st->page_table, next_norm, last ? static_cast<__nv_bfloat16 *>(target_hidden) : nullptr);
+                   st->page_table, next_norm, last ? static_cast<__nv_bfloat16 *>(target_hidden) : nullptr,
+                   last ? nullptr : &c->layers[l + 1], last ? nullptr : &c->lmaps[l + 1], l > 0);
     if (rc) return rc;
   }
   return run_gemm(c, c->xn, c->Mmax, &c->lm_head_map, static_cast<const __nv_bfloat16 *>(c->w.lm_head), ph.M, c->V, c->d,
@@ -647,7 +725,10 @@ int gm_last_status(gm_ctx *c) {
   GM_CUDA(c, cudaStreamSynchronize(c->stream));
   GM_CUDA(c, cudaMemcpy(&s, c->status, sizeof(s), cudaMemcpyDeviceToHost));
   GM_CUDA(c, cudaMemset(c->status, 0, sizeof(s)));
-  if (s & ST_TIMEOUT) return GM_ERR_DEVICE_TIMEOUT;
+  if (s & ST_TIMEOUT) {                 // a chain launch that gave up may have left its barrier words mid-count
+    if (c->chain_sync) GM_CUDA(c, cudaMemset(c->chain_sync, 0, (4 + static_cast<size_t>(c->chain_pairs) * 4) * sizeof(uint32_t)));
+    return GM_ERR_DEVICE_TIMEOUT;
+  }
   if (s & ST_KV_CAPACITY) return GM_ERR_KV_CAPACITY;
   if (s & (ST_BAD_PAGE | ST_BAD_TOKEN)) return GM_ERR_BAD_PAGE;
   if (c->check_guards) {

@@ -53,6 +53,16 @@ struct gm_ctx {
   float *x = nullptr, *g = nullptr, *part_o = nullptr, *part_ml = nullptr;
   __nv_bfloat16 *xn = nullptr, *zin = nullptr, *qkv = nullptr, *qbuf = nullptr, *attn_out = nullptr, *act = nullptr, *gn = nullptr;
   bool pair_gemm = true;              // CTA-pair kernel for the full wave of wide projections (GM_NO_PAIR_GEMM: off)
+  // persistent chain of a layer's projections (chain.cu); GM_NO_CHAIN: off
+  bool chain_on = false;
+  int chain_pairs = 0;                // CTA pairs resident at once
+  int chain_npw = 2, chain_npa = 2;   // producer threads per CTA for weight / activation boxes
+  int chain_max_m = 512;              // phases with more rows than this run as separate launches
+  float *chain_partial = nullptr;     // K-slice partial sums, [pairs][2][256][128]
+  float *chain_sq[2] = {nullptr, nullptr};   // sums of squares per 32 features and row, after the O / down projection
+  uint32_t *chain_sync = nullptr;     // barrier words
+  unsigned long long *chain_trace = nullptr;   // gm_chain_trace: [2 pairs][32] stamps
+  bool chain_trace_on = false;
   int max_clusters[17][9];            // resident clusters of the GEMM kernel by (block_t / 16, cluster size); -1 = not asked yet
   __nv_bfloat16 *ws_draft_logits = nullptr, *ws_target_logits = nullptr, *ws_target_hidden = nullptr;
   int32_t *ws_draft_tok = nullptr, *ws_accept_len = nullptr, *ws_next_token = nullptr;
@@ -175,9 +185,19 @@ int round16(int v);
 int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *wmap, const __nv_bfloat16 *w, int M,
              int N, int K, void *out, int epi, size_t ldo);
 struct PhaseShape { int B, QT, M, qrows; };
+// next_lw / next_lm: the layer whose QKV projection is appended to this layer's chain of projections (its input norm
+// is next_norm); qkv_done: this layer's own QKV projection was produced that way by the layer before.
 int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const PhaseShape &ph, const CUtensorMap &kvm,
               __nv_bfloat16 *pool, int layer, int num_pages, const int32_t *page_table,
-              const __nv_bfloat16 *next_norm, __nv_bfloat16 *hidden_out);
+              const __nv_bfloat16 *next_norm, __nv_bfloat16 *hidden_out, const gm_layer_weights *next_lw = nullptr,
+              const LayerMaps *next_lm = nullptr, bool qkv_done = false);
+bool chain_usable(const gm_ctx *c, int M);
+// One projection of a chain (see ChainPhase); the input is x [x_rows, K] bf16.
+struct ChainSpec {
+  const CUtensorMap *wmap; const __nv_bfloat16 *x; int x_rows, N, K; void *out; int epi, ldo;
+  __nv_bfloat16 *xg; const __nv_bfloat16 *gamma; float *sq_out; const float *sq_in; int norm_dim;
+};
+int run_chain(gm_ctx *c, const ChainSpec *specs, int n, int M);
 int run_plan(gm_ctx *c, const gm_state *st, int mode, int k_or_j);
 int run_plan_chunk(gm_ctx *c, int batch, const int32_t *row_n, const int32_t *row_base, int QT);
 int check_state(const gm_ctx *c, const gm_state *st, int k);
