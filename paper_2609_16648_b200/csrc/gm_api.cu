@@ -77,6 +77,7 @@ int pick_split(gm_ctx *c, int M, int N, int K, int T) {
 }
 
 // out = epilogue(x[M, K] w[N, K]^T) on the tcgen05 kernel (or the plain one under GM_FLAG_SIMPLE_GEMM).
+int run_chain(gm_ctx *c, const ChainSpec *specs, int n, int M);
 int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *wmap, const __nv_bfloat16 *w, int M,
              int N, int K, void *out, int epi, size_t ldo) {
   GemmArgs A;
@@ -87,9 +88,17 @@ int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *w
   A.block_t = T;
   A.nsplit = 1;
   A.wtiles = 1;
-  if ((c->cfg.flags & GM_FLAG_SIMPLE_GEMM) != 0 || (K % 64) != 0) {
+  if ((c->cfg.flags & GM_FLAG_SIMPLE_GEMM) != 0) {
     GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_simple(A, c->stream));
     return GM_OK;
+  }
+  if ((K % 64) != 0) return GM_ERR_UNSUPPORTED;      // the tensor-core kernels stage K in blocks of 64
+  // A SwiGLU projection wide enough for one tile per CTA pair (gate/up): one wave of the persistent-pair kernel - tiles
+  // of 256 / 288 features sized so that the wave is exact - instead of a full wave plus a short tail launch.
+  if (c->chain_on && c->chain_mode >= 1 && epi == EPI_SWIGLU_BF16 && M <= c->chain_max_m && N >= c->chain_pairs * 128 &&
+      N <= c->chain_pairs * 288 && (N % 32) == 0 && (ldo % 8) == 0) {
+    const ChainSpec g = {w, x, x_rows, N, K, out, epi, static_cast<int>(ldo), nullptr, nullptr, nullptr, nullptr, 0, 0};
+    return run_chain(c, &g, 1, M);
   }
   int rc = x_map(c, x, x_rows, K, T, &A.x_map);
   if (rc != GM_OK) return rc;
@@ -132,7 +141,7 @@ int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *w
   return GM_OK;
 }
 
-bool chain_usable(const gm_ctx *c, int M) { return c->chain_on && M <= c->chain_max_m; }
+bool chain_usable(const gm_ctx *c, int M) { return c->chain_on && c->chain_mode == 2 && M <= c->chain_max_m; }
 
 // A chain of dependent projections as one persistent launch.
 int run_chain(gm_ctx *c, const ChainSpec *specs, int n, int M) {
@@ -146,15 +155,22 @@ int run_chain(gm_ctx *c, const ChainSpec *specs, int n, int M) {
   for (int p = 0; p < n; ++p) {
     const ChainSpec &s = specs[p];
     ChainPhase &ph = A.ph[p];
-    ph.w_map = *s.wmap;
+    ph.out = s.out; ph.xg = s.xg; ph.gamma = s.gamma; ph.sq_out = s.sq_out; ph.sq_in = s.sq_in;
+    ph.inv_dim = s.sq_in ? 1.0f / static_cast<float>(s.norm_dim) : 0.f;
+    ph.epi = s.epi; ph.N = s.N; ph.K = s.K; ph.ldo = s.ldo;
+    chain_schedule(ph, A.mblocks, A.P, n >= 3 ? c->chain_force_ns[p] : 0);
+    ph.sq_groups = s.sq_in ? A.ph[s.sq_from].tiles : 0;
+    auto key = std::make_tuple(s.w, s.N, s.K, ph.wbox);
+    auto it = c->chain_w_maps.find(key);
+    if (it == c->chain_w_maps.end()) {
+      CUtensorMap m;
+      if (make_map(c, &m, s.w, s.N, s.K, ph.wbox) != GM_OK) return GM_ERR_CUDA;
+      it = c->chain_w_maps.emplace(key, m).first;
+    }
+    ph.w_map = it->second;
     // rows beyond M are out of the map's bounds: the copy engine fills them with zeros and fetches nothing
     int rc = x_map(c, s.x, M < s.x_rows ? M : s.x_rows, s.K, 128, &ph.x_map);
     if (rc != GM_OK) return rc;
-    ph.out = s.out; ph.xg = s.xg; ph.gamma = s.gamma; ph.sq_out = s.sq_out; ph.sq_in = s.sq_in;
-    ph.sq_groups = s.sq_in ? (s.norm_dim + 63) / 64 : 0;
-    ph.inv_dim = s.sq_in ? 1.0f / static_cast<float>(s.norm_dim) : 0.f;
-    ph.epi = s.epi; ph.N = s.N; ph.K = s.K; ph.ldo = s.ldo;
-    chain_schedule(ph, A.mblocks, A.P);
   }
   GM_LAUNCH(c, GM_KC_GEMM, launch_chain(A, c->stream));
   return GM_OK;
@@ -173,8 +189,8 @@ int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const 
   // QKV projection (bf16) -> rotary + KV append + Q rearrangement
   if (!(chain && qkv_done)) {
     if (chain) {
-      const ChainSpec q = {&lm.wqkv, c->xn, c->Mmax, c->n_qkv, c->d, c->qkv, EPI_STORE_BF16, c->n_qkv,
-                           nullptr, nullptr, nullptr, nullptr, 0};
+      const ChainSpec q = {lw.wqkv, c->xn, c->Mmax, c->n_qkv, c->d, c->qkv, EPI_STORE_BF16, c->n_qkv,
+                           nullptr, nullptr, nullptr, nullptr, 0, 0};
       rc = run_chain(c, &q, 1, ph.M);
     } else {
       rc = run_gemm(c, c->xn, c->Mmax, &lm.wqkv, static_cast<const __nv_bfloat16 *>(lw.wqkv), ph.M, c->n_qkv, c->d,
@@ -210,15 +226,15 @@ int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const 
     // the two norms in between are folded around the projections (see chain.cu)
     const bool fuse_next = next_lw && next_lm && next_norm;
     ChainSpec sp[4];
-    sp[0] = {&lm.wo, c->attn_out, c->Mmax, c->d, c->q_dim, c->x, EPI_ADD_F32, c->d,
-             c->xn, static_cast<const __nv_bfloat16 *>(lw.ln2), c->chain_sq[0], nullptr, 0};
-    sp[1] = {&lm.wgu, c->xn, c->Mmax, 2 * c->F, c->d, c->act, EPI_SWIGLU_BF16, c->F,
-             nullptr, nullptr, nullptr, c->chain_sq[0], c->d};
-    sp[2] = {&lm.wdown, c->act, c->Mmax, c->d, c->F, c->x, EPI_ADD_F32, c->d,
-             fuse_next ? c->xn : nullptr, fuse_next ? next_norm : nullptr, fuse_next ? c->chain_sq[1] : nullptr, nullptr, 0};
+    sp[0] = {lw.wo, c->attn_out, c->Mmax, c->d, c->q_dim, c->x, EPI_ADD_F32, c->d,
+             c->xn, static_cast<const __nv_bfloat16 *>(lw.ln2), c->chain_sq[0], nullptr, 0, 0};
+    sp[1] = {lw.w_gate_up, c->xn, c->Mmax, 2 * c->F, c->d, c->act, EPI_SWIGLU_BF16, c->F,
+             nullptr, nullptr, nullptr, c->chain_sq[0], 0, c->d};
+    sp[2] = {lw.w_down, c->act, c->Mmax, c->d, c->F, c->x, EPI_ADD_F32, c->d,
+             fuse_next ? c->xn : nullptr, fuse_next ? next_norm : nullptr, fuse_next ? c->chain_sq[1] : nullptr, nullptr, 0, 0};
     if (fuse_next)
-      sp[3] = {&next_lm->wqkv, c->xn, c->Mmax, c->n_qkv, c->d, c->qkv, EPI_STORE_BF16, c->n_qkv,
-               nullptr, nullptr, nullptr, c->chain_sq[1], c->d};
+      sp[3] = {next_lw->wqkv, c->xn, c->Mmax, c->n_qkv, c->d, c->qkv, EPI_STORE_BF16, c->n_qkv,
+               nullptr, nullptr, nullptr, c->chain_sq[1], 2, c->d};
     if ((rc = run_chain(c, sp, fuse_next ? 4 : 3, ph.M)) != GM_OK) return rc;
     if (!fuse_next && (next_norm || hidden_out))
       GM_LAUNCH(c, GM_KC_ELEMENTWISE,
@@ -432,20 +448,23 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
   A_(dev_alloc(c, &c->pf_xlast, B1 * c->d));
   A_(dev_alloc(c, &c->status, 1));
   // persistent chain of a layer's projections: every CTA pair must be resident at once
-  if (std::getenv("GM_NO_CHAIN") == nullptr && !(cfg->flags & GM_FLAG_SIMPLE_GEMM) && (c->q_dim % 64) == 0) {
+  if (!(cfg->flags & GM_FLAG_SIMPLE_GEMM) && (c->q_dim % 64) == 0) {
     int pairs = 0;
     if (chain_max_pairs(&pairs) != cudaSuccess) { pairs = 0; (void)cudaGetLastError(); }
     if (pairs > c->sm_count / 2) pairs = c->sm_count / 2;
     if (const char *ov = std::getenv("GM_CHAIN_PAIRS")) { const int v = std::atoi(ov); if (v >= 1 && v < pairs) pairs = v; }
-    if (const char *ov = std::getenv("GM_CHAIN_NPW")) c->chain_npw = std::atoi(ov) == 1 ? 1 : 2;
+    if (const char *ov = std::getenv("GM_CHAIN_NPW")) { const int v = std::atoi(ov); if (v >= 1 && v <= 4) c->chain_npw = v; }
     if (const char *ov = std::getenv("GM_CHAIN_NPA")) c->chain_npa = std::atoi(ov) == 1 ? 1 : 2;
+    if (const char *ov = std::getenv("GM_CHAIN_MODE")) { const int v = std::atoi(ov); if (v >= 0 && v <= 2) c->chain_mode = v; }
     if (const char *ov = std::getenv("GM_CHAIN_MAX_M")) { const int v = std::atoi(ov); if (v >= 1) c->chain_max_m = v; }
     if (pairs >= 1) {
       c->chain_pairs = pairs;
-      A_(dev_alloc(c, &c->chain_partial, static_cast<size_t>(pairs) * 2 * 256 * 128));
-      A_(dev_alloc(c, &c->chain_sq[0], static_cast<size_t>((c->d + 31) / 32) * M));
+      A_(dev_alloc(c, &c->chain_partial, chain_partial_floats(pairs)));
+      A_(dev_alloc(c, &c->chain_sq[0], static_cast<size_t>((c->d + 31) / 32) * M));     // one row per feature tile (at most per 32 features)
       A_(dev_alloc(c, &c->chain_sq[1], static_cast<size_t>((c->d + 31) / 32) * M));
-      A_(dev_alloc(c, &c->chain_sync, 4 + static_cast<size_t>(pairs) * 4));
+      A_(dev_alloc(c, &c->chain_sync, 1 + static_cast<size_t>(pairs) * 2));
+      if (const char *ov = std::getenv("GM_CHAIN_NS"))
+        std::sscanf(ov, "%d,%d,%d,%d", &c->chain_force_ns[0], &c->chain_force_ns[1], &c->chain_force_ns[2], &c->chain_force_ns[3]);
       c->chain_on = true;
     }
   }
@@ -726,7 +745,7 @@ int gm_last_status(gm_ctx *c) {
   GM_CUDA(c, cudaMemcpy(&s, c->status, sizeof(s), cudaMemcpyDeviceToHost));
   GM_CUDA(c, cudaMemset(c->status, 0, sizeof(s)));
   if (s & ST_TIMEOUT) {                 // a chain launch that gave up may have left its barrier words mid-count
-    if (c->chain_sync) GM_CUDA(c, cudaMemset(c->chain_sync, 0, (4 + static_cast<size_t>(c->chain_pairs) * 4) * sizeof(uint32_t)));
+    if (c->chain_sync) GM_CUDA(c, cudaMemset(c->chain_sync, 0, (1 + static_cast<size_t>(c->chain_pairs) * 2) * sizeof(unsigned long long)));
     return GM_ERR_DEVICE_TIMEOUT;
   }
   if (s & ST_KV_CAPACITY) return GM_ERR_KV_CAPACITY;

@@ -56,11 +56,14 @@ struct gm_ctx {
   // persistent chain of a layer's projections (chain.cu); GM_NO_CHAIN: off
   bool chain_on = false;
   int chain_pairs = 0;                // CTA pairs resident at once
-  int chain_npw = 2, chain_npa = 2;   // producer threads per CTA for weight / activation boxes
+  int chain_npw = 4, chain_npa = 2;   // producer threads per CTA for weight / activation boxes
+  int chain_mode = 1;                 // 1: only the wide gate/up projection, as a one-phase launch; 2: the whole chain; 0: off
   int chain_max_m = 512;              // phases with more rows than this run as separate launches
-  float *chain_partial = nullptr;     // K-slice partial sums, [pairs][2][256][128]
-  float *chain_sq[2] = {nullptr, nullptr};   // sums of squares per 32 features and row, after the O / down projection
-  uint32_t *chain_sync = nullptr;     // barrier words
+  float *chain_partial = nullptr;     // K-slice partial sums, one slot per CTA
+  float *chain_sq[2] = {nullptr, nullptr};   // sums of squares per feature tile and row, after the O / down projection
+  unsigned long long *chain_sync = nullptr;  // barrier counters
+  std::map<std::tuple<const void *, int, int, int>, CUtensorMap> chain_w_maps;   // (weights, N, K, box rows)
+  int chain_force_ns[4] = {0, 0, 0, 0};      // GM_CHAIN_NS: K slices per phase position (tuning aid)
   unsigned long long *chain_trace = nullptr;   // gm_chain_trace: [2 pairs][32] stamps
   bool chain_trace_on = false;
   int max_clusters[17][9];            // resident clusters of the GEMM kernel by (block_t / 16, cluster size); -1 = not asked yet
@@ -194,8 +197,9 @@ int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const 
 bool chain_usable(const gm_ctx *c, int M);
 // One projection of a chain (see ChainPhase); the input is x [x_rows, K] bf16.
 struct ChainSpec {
-  const CUtensorMap *wmap; const __nv_bfloat16 *x; int x_rows, N, K; void *out; int epi, ldo;
-  __nv_bfloat16 *xg; const __nv_bfloat16 *gamma; float *sq_out; const float *sq_in; int norm_dim;
+  const void *w; const __nv_bfloat16 *x; int x_rows, N, K; void *out; int epi, ldo;
+  __nv_bfloat16 *xg; const __nv_bfloat16 *gamma; float *sq_out;
+  const float *sq_in; int sq_from, norm_dim;     // sq_from: the phase of this chain that writes sq_in
 };
 int run_chain(gm_ctx *c, const ChainSpec *specs, int n, int M);
 int run_plan(gm_ctx *c, const gm_state *st, int mode, int k_or_j);

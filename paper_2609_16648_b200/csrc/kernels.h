@@ -330,12 +330,12 @@ cudaError_t gemm_tc_max_clusters(int block_t, int nsplit, int *out);
 // ---- a chain of dependent projections in one persistent launch (chain.cu) -------------------------------------------
 // Phase p computes epilogue_p(x_p[M, K_p] * w_p[N_p, K_p]^T); phase p + 1 may read what phase p wrote.
 struct ChainPhase {
-  CUtensorMap w_map;                    // weights [N, K] bf16, box 64 x 128
+  CUtensorMap w_map;                    // weights [N, K] bf16, box 64 x wbox
   CUtensorMap x_map;                    // input rows [M, K] bf16, box 64 x 128
   void *out;                            // EPI_STORE_BF16 / EPI_SWIGLU_BF16: bf16 [M, ldo]; EPI_STORE_F32 / EPI_ADD_F32: fp32 [M, ldo]
   __nv_bfloat16 *xg;                    // fp32 epilogues: also bf16(result * gamma) [M, N], the next norm's input; or null
   const __nv_bfloat16 *gamma;           // [N] norm weight for xg
-  float *sq_out;                        // fp32 epilogues: [ceil(N / 64)][m_pad] sums of squares of the result rows per 64 features; or null
+  float *sq_out;                        // fp32 epilogues: [tiles][m_pad] sums of squares of the result rows per feature tile; or null
   const float *sq_in;                   // [sq_groups][m_pad] sums of squares of this phase's input rows before the norm
                                         // weight was applied: the accumulator rows are scaled by rsqrt(sum * inv_dim + eps); or null
   int sq_groups;
@@ -343,23 +343,25 @@ struct ChainPhase {
   int epi;
   int N, K;
   int ldo;
-  int full, rem, ns;                    // schedule (chain_schedule): whole tiles per pair, leftover tiles, K slices of a leftover tile
+  int G, tiles, ns, wbox;               // schedule (chain_schedule): groups of 32 features, feature tiles, K slices per
+                                        // tile, weight rows a CTA stages per K block (half of the widest tile)
 };
 struct ChainArgs {
   ChainPhase ph[4];
   int n_phases;
   int M, mblocks;                       // token rows, blocks of 256 token rows
   int P;                                // CTA pairs of the launch (all resident at once)
-  int npw, npa;                         // producer threads for weight / activation boxes (1 or 2 each)
+  int npw, npa;                         // producer threads for weight / activation boxes
   int m_pad;                            // row stride of the sums of squares
   float eps;
-  float *partial;                       // [P][2][128][256] fp32 scratch of the K slices
-  uint32_t *sync;                       // {count, generation} of the grid barrier, then one such pair per (pair, CTA rank) from word 4
+  float *partial;                       // [P][2][128][288] fp32 scratch of the K slices
+  unsigned long long *sync;             // monotonic barrier counters: [0] the grid's, [1 + 2 pair + CTA rank] the K-slice groups'
   uint32_t *status;
   unsigned long long *timeline;         // optional trace, [2 P][64] nanosecond stamps (see chain.cu); or null
-  int trace_phase;                      // phase whose per-warp epilogue stamps go to slots 32.. / 48..
+  int trace_phase;                      // phase whose epilogue detail stamps go to slots 32.. / 48..
 };
-void chain_schedule(ChainPhase &ph, int mblocks, int P);
+void chain_schedule(ChainPhase &ph, int mblocks, int P, int force_ns);
+size_t chain_partial_floats(int pairs);
 cudaError_t chain_max_pairs(int *out);
 cudaError_t launch_chain(const ChainArgs &A, cudaStream_t stream);
 

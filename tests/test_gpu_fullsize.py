@@ -55,10 +55,13 @@ def _snapshot(gst, cfg, b, K):
     return ostep.BatchState([seq], caches[0], caches[1], step=1)
 
 
-@pytest.mark.parametrize("name,K", [("4b", 3), ("7b", 3), ("4b", 5)])
-def test_full_dimension_cycle_on_sampled_sequences(name, K):
+@pytest.mark.parametrize("name,K,chain", [("4b", 3, "1"), ("7b", 3, "1"), ("4b", 5, "1"), ("4b", 3, "2")],
+                         ids=["4b-3", "7b-3", "4b-5", "4b-3-whole_chain"])
+def test_full_dimension_cycle_on_sampled_sequences(name, K, chain, monkeypatch):
     """4B: 16 query rows per KV head at K = 3, 24 at K = 5 (the transposed attention kernel); 7B dimensions
-    (d 3584, 28/4 heads, FFN 18944): 28 rows per KV head, two token blocks in the LM head."""
+    (d 4096, 32/8 heads of 128, FFN 11008, vocabulary 151680): 512 token rows at K = 3, two token blocks in every
+    projection.  The last case runs a layer's projections as one persistent launch (GM_CHAIN_MODE=2)."""
+    monkeypatch.setenv("GM_CHAIN_MODE", chain)
     sys.path.insert(0, ROOT)
     import bench
     import paper_2609_16648_b200 as gmb
@@ -72,7 +75,9 @@ def test_full_dimension_cycle_on_sampled_sequences(name, K):
         norms += [lw["ln1"], lw["ln2"]]
     for t in norms:                                           # a forgotten norm weight must show
         t.copy_((1 + (torch.rand(t.shape, device="cuda", generator=g) - 0.5) * 0.5).to(torch.bfloat16))
-    sample = sorted({0, 21, 42, 63, int(np.argmax(lens)), int(np.argmin(lens))})
+    # a seeded third of the batch, always with the shortest and the longest sequence
+    sample = sorted(set(np.random.default_rng(17).choice(B, 20, replace=False).tolist()) |
+                    {int(np.argmax(lens)), int(np.argmin(lens))})
     snaps = {b: _snapshot(gst, cfg, b, K) for b in sample}
 
     z = lambda shape, dt: torch.zeros(shape, dtype=dt, device="cuda")
@@ -111,5 +116,5 @@ def test_full_dimension_cycle_on_sampled_sequences(name, K):
         agree += both + (1 if (both < K and ga[b] == ref["accept_len"][0]) else 0)
     print(f"sampled sequences {sample} (kv_len {[int(lens[b]) for b in sample]}): worst rel err {worst:.3e}, accept bits {agree}/{total}")
     assert worst < TOL, worst
-    assert agree >= total - 1, (agree, total)
+    assert agree >= total - 1, (agree, total)          # ~30 evaluated positions: one threshold case allowed (<= 99.5 % needs 200)
     ctx.close()

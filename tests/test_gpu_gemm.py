@@ -88,10 +88,14 @@ def test_full_size_projections_on_sampled_outputs(M, N, K):
 
 
 @pytest.mark.parametrize("M", [256, 64, 300, 37])
-def test_gate_up_projection_with_fused_swiglu_full_matrix(M):
-    """The 4B gate/up projection (152 feature tiles: a full wave plus a split tail launch) over the whole output,
-    plain stores and the fused SwiGLU epilogue on interleaved gate/up rows, against fp64."""
+@pytest.mark.parametrize("chain", ["1", "0"], ids=["pair_wave_kernel", "full_wave_plus_tail"])
+def test_gate_up_projection_with_fused_swiglu_full_matrix(M, chain, monkeypatch):
+    """The 4B gate/up projection over the whole output, plain stores and the fused SwiGLU epilogue on interleaved
+    gate/up rows, against fp64.  The SwiGLU form runs as one exact wave of the persistent-pair kernel (74 tiles of 256 or
+    288 features; two token blocks at M = 300) or, with GM_CHAIN_MODE=0, as 152 feature tiles: a full wave plus a
+    split tail launch."""
     N, K = 19456, 2560
+    monkeypatch.setenv("GM_CHAIN_MODE", chain)
     gmb, ctx = _ctx()
     g = torch.Generator(device="cuda").manual_seed(M)
     x = torch.randn((M, K), device="cuda", generator=g).to(torch.bfloat16)
@@ -113,6 +117,7 @@ def test_cta_pair_kernel_equals_single_cta_kernel(M, monkeypatch):
     """The full wave of a wide projection runs on CTA pairs (one MMA over two SMs, each CTA staging half of the
     activation box).  Same K order and the same accumulation per output as the single-CTA kernel: bit-identical."""
     N, K = 19456, 2560
+    monkeypatch.setenv("GM_CHAIN_MODE", "0")                  # both runs on the tile kernels this test compares
     g = torch.Generator(device="cuda").manual_seed(100 + M)
     x = torch.randn((M, K), device="cuda", generator=g).to(torch.bfloat16)
     w = (torch.randn((N, K), device="cuda", generator=g) * 0.02).to(torch.bfloat16)

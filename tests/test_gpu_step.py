@@ -82,8 +82,9 @@ def _parity_from_common_state(cfg, flags, n_steps, concat=None, top_p=1.0):
     return worst, (bit_agree, bit_total), (tok_same, tok_total), (fin_same, fin_total)
 
 
-@pytest.mark.parametrize("flags", [1, 0], ids=["mma_sync_gemm", "tcgen05_gemm"])
-def test_tiny_step_parity_from_common_state(flags):
+@pytest.mark.parametrize("flags,chain", [(1, None), (0, "0"), (0, "1"), (0, "2")],
+                         ids=["mma_sync_gemm", "tcgen05_gemm_separate_launches", "tcgen05_gemm", "tcgen05_gemm_whole_chain"])
+def test_tiny_step_parity_from_common_state(flags, chain, monkeypatch):
     """Every step starts from the oracle's state.
     (1) the device's draft draws and accept/resample decisions equal the oracle's decision function on the
         device's own probabilities, bit for bit;
@@ -92,7 +93,12 @@ def test_tiny_step_parity_from_common_state(flags):
         sides evaluate;
     (3) free-running (each side sampling its own drafts from the same uniforms) the sampled tokens agree on
         most positions - a looser bar, because an inverse-CDF draw turns a relative logit error e into a
-        disagreement probability of order e * sqrt(V)."""
+        disagreement probability of order e * sqrt(V).
+    The tcgen05 path is run three ways (GM_CHAIN_MODE, read when the context is created): every projection a launch of
+    its own; the default (the wide gate/up projection on the persistent-pair kernel); and a layer's output projection,
+    gate/up, down and the next QKV projection as one persistent launch with the norms folded in."""
+    if chain is not None:
+        monkeypatch.setenv("GM_CHAIN_MODE", chain)
     cfg = get_config("tiny").with_(prompt_len=40)
     worst, bits, toks, fins = _parity_from_common_state(cfg, flags, n_steps=24)
     assert worst < TOL, worst
