@@ -413,8 +413,11 @@ int gm_attention(gm_ctx *ctx, const void *q, const void *kv_pool, int pool_layer
  *   that device current; make that first call before any stream capture begins.
  *   Sharing: every call uses the same array, which keeps the previous call's contents; the call clears what
  *   must start at zero itself.  Two calls that overlap on the GPU (different streams, or two host threads)
- *   race on it - serialise them.  Device-seen conditions are not reported: a sequence that does not fit its
- *   page-table row is skipped (its output rows stay untouched) and an out-of-range page id reads page 0.
+ *   race on it - serialise them.  Device-seen conditions are not reported (there is no context whose status a
+ *   later call could read): a sequence that does not fit its page-table row is skipped (its output rows stay
+ *   untouched), an out-of-range page id reads page 0, and should one of the kernels' bounded waits ever run out
+ *   the call still returns GM_OK with the rows of the affected segment incomplete - use gm_attention with a
+ *   context where such conditions must be seen.
  *   cuda_stream: a cudaStream_t (NULL = the default stream) of the current device.                        */
 #define GM_NOALLOC_SCRATCH_BYTES (16u << 20)
 #define GM_NOALLOC_MAX_BATCH 256
@@ -454,6 +457,13 @@ int gm_chain_trace_read(gm_ctx *ctx, uint64_t *out, int capacity);
 
 /* Number of kernels this library launched since gm_init (all calls).                        */
 int64_t gm_launch_count(gm_ctx *ctx);
+
+/* Self-test of the failure path (the paper has no counterpart): every device-side wait of the library is a
+ * bounded poll that records GM_ERR_DEVICE_TIMEOUT and returns instead of hanging.  This call launches one tiny
+ * kernel whose only thread waits, with a limit of 1024 polls, on a barrier nothing ever arrives on; the wait runs
+ * out, the status word is set, the kernel exits normally.  The next gm_last_status returns
+ * GM_ERR_DEVICE_TIMEOUT and clears it; the context stays usable.  No GPU fault, trap or unbounded loop is involved. */
+int gm_selftest_wait_expiry(gm_ctx *ctx);
 
 /* Waits for the stream and returns 0 or the GM_ERR_* of the first sticky device condition;
  * clears the status word.                                                                   */

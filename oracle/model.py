@@ -5,12 +5,11 @@ attention, SwiGLU feed-forward).  The decoder-layer families the paper names (Ap
 differ in the attention projections only: one adds a bias to the query/key/value
 projections (keys "bq", "bk", "bv" of a layer), one normalises every query and key head
 with an RMSNorm over the head dimension before the rotary embedding (keys "qnorm",
-"knorm").  A layer without those keys has neither.  Draft head (App. B.1, "MTP
-Architecture"): ONE such decoder layer.  For each position it drafts, it consumes the
-hidden state and the token embedding of the position before it: the two are
-normalised by separate RMSNorms, concatenated, projected back to the model width by a
-bias-free linear layer and passed through the layer; it keeps a KV cache of its own
-and borrows the embedding and the output head from the backbone.
+"knorm").  A layer without those keys has neither.  Draft head (App. B.1): ONE such
+decoder layer with its own KV cache; embedding table and output head are the backbone's.
+Its input at position i is z_i = W_proj [RMSNorm_e(E[x_i]) ; RMSNorm_h(h_{i-1})] with a
+bias-free W_proj of shape [d, 2d]: x_i the token at that position, h_{i-1} the backbone
+state that produced it.
 
 Conventions the paper leaves open (see the package docstring): the concatenation is
 [norm(embedding) ; norm(hidden)]; the hidden state is the backbone's residual stream

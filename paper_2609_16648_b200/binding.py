@@ -26,7 +26,7 @@ EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_sp
            "gm_rollout_begin", "gm_rollout_step", "gm_rollout_run", "gm_pages_reset", "gm_pages_reserve",
            "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_overlap", "gm_dca_loss", "gm_dca_grad",
            "gm_spec_step_host", "gm_gemm", "gm_gemm_swiglu", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
-           "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_chain_trace", "gm_chain_trace_read", "gm_launch_count",
+           "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_chain_trace", "gm_chain_trace_read", "gm_selftest_wait_expiry", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
 
 
@@ -113,6 +113,7 @@ def lib() -> C.CDLL:
     L.gm_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     L.gm_chain_trace.argtypes = [vp, i32]
     L.gm_chain_trace_read.argtypes = [vp, vp, i32]
+    L.gm_selftest_wait_expiry.argtypes = [vp]
     L.gm_launch_count.argtypes = [vp]
     L.gm_launch_count.restype = C.c_int64
     L.gm_last_status.argtypes = [vp]
@@ -514,6 +515,10 @@ def gm_chain_trace_read(ctx: Context):
     if n < 0:
         raise GmError(n, "gm_chain_trace_read")
     return buf[:n].astype(np.int64).reshape(-1, 64)
+
+
+def gm_selftest_wait_expiry(ctx: Context):
+    _check(lib().gm_selftest_wait_expiry(ctx.handle), "gm_selftest_wait_expiry")
 
 
 def gm_launch_count(ctx: Context) -> int:

@@ -14,6 +14,20 @@ int gmh::run_nucleus(gm_ctx *c, const void *logits, int rows, float temperature,
   return GM_OK;
 }
 
+namespace gm {
+// Self-test of the bounded-wait path: one warp waits on an mbarrier nobody will ever arrive on, gives up after
+// `limit` polls, records ST_TIMEOUT like every other wait of the library, and returns.  Nothing spins without a limit.
+__global__ void wait_expiry_kernel(uint32_t *status, uint32_t limit) {
+  __shared__ uint64_t bar;
+  pdl_prologue();
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    mbar_fence_init();
+    if (!mbar_wait(&bar, 0, limit)) set_status(status, ST_TIMEOUT);
+  }
+}
+}  // namespace gm
+
 extern "C" {
 
 int gm_nucleus(gm_ctx *c, const void *logits, int rows, float temperature, float top_p, void *out, float *dbg_weight) {
@@ -150,5 +164,11 @@ int gm_chain_trace_read(gm_ctx *c, uint64_t *out, int capacity) {
   return words;
 }
 
+
+int gm_selftest_wait_expiry(gm_ctx *c) {
+  if (!c) return GM_ERR_INVALID_ARG;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_k(wait_expiry_kernel, dim3(1), dim3(32), 0, c->stream, 1, c->status, 1024u));
+  return GM_OK;
+}
 
 }  // extern "C"

@@ -561,13 +561,8 @@ static cudaError_t launch_att_t(const AttnArgs &A, cudaStream_t stream) {
   // bound by instruction issue, not by the depth of the ring.)
   const int hpc = att_hpc(A.n_kv), nst = att_stages(A.n_kv, HD, 2);
   const size_t smem = attention_smem_bytes(A.n_kv, HD, 2);
-  static size_t configured = 0;
-  if (smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(attention_t_kernel<HD, NR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    configured = smem;
-  }
+  static SmemConfigured configured;
+  if (cudaError_t e = ensure_dyn_smem(attention_t_kernel<HD, NR>, smem, configured); e != cudaSuccess) return e;
   dim3 grid(A.n_ctas, A.n_kv / hpc);
   return launch_k(attention_t_kernel<HD, NR>, grid, dim3((hpc + 1) * 32), smem, stream, 1, A, hpc, nst);
 }
@@ -577,13 +572,8 @@ static cudaError_t launch_att(const AttnArgs &A, cudaStream_t stream) {
   // the variants that stage Q in shared memory share one layout: 32 rows x head_dim per KV head
   const int hpc = att_hpc(A.n_kv), nst = att_stages(A.n_kv, HD, MT * RT);
   const size_t smem = attention_smem_bytes(A.n_kv, HD, MT * RT);
-  static size_t configured = 0;
-  if (smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(attention_kernel<HD, MT, RT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    configured = smem;
-  }
+  static SmemConfigured configured;
+  if (cudaError_t e = ensure_dyn_smem(attention_kernel<HD, MT, RT>, smem, configured); e != cudaSuccess) return e;
   dim3 grid(A.n_ctas, A.n_kv / hpc);
   return launch_k(attention_kernel<HD, MT, RT>, grid, dim3((hpc * RT + 1) * 32), smem, stream, 1, A, hpc, nst);
 }

@@ -616,14 +616,8 @@ chain_kernel(const __grid_constant__ ChainArgs A) {
 // ---- host side --------------------------------------------------------------------------------------------------------------
 static size_t chain_smem() { return static_cast<size_t>(CH_STAGES) * CH_STAGE_BYTES + 4096 + 1024; }
 static cudaError_t chain_configure() {
-  static bool done[64] = {};
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
-  e = cudaFuncSetAttribute(chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-  if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
-  return e;
+  static SmemConfigured configured;
+  return ensure_dyn_smem(chain_kernel, 227 * 1024, configured);
 }
 
 cudaError_t chain_max_pairs(int *out) {

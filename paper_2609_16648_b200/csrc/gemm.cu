@@ -342,13 +342,10 @@ gemm_pair_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
   if (warp == 1) tc2_dealloc(tmem, ncols);
 }
 
-// The kernel may use the whole opt-in shared memory of an SM (227 KB); set once per process.
+// The kernel may use the whole opt-in shared memory of an SM (227 KB); set once per device.
 static cudaError_t gt_configure() {
-  static bool done = false;
-  if (done) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-  if (e == cudaSuccess) done = true;
-  return e;
+  static SmemConfigured configured;
+  return ensure_dyn_smem(gemm_tc_kernel<1>, 227 * 1024, configured);
 }
 
 cudaError_t gemm_tc_max_clusters(int block_t, int nsplit, int *out) {
@@ -380,12 +377,8 @@ cudaError_t launch_gemm_pair(const GemmArgs &A, cudaStream_t stream) {
   if (T < 32 || T > 256 || (T & 31) || (A.K % GT_BK) || A.nsplit != 1 || A.wtiles != 1 || A.n_tiles < 2 ||
       (A.n_tiles & 1) || A.n_base < 0)
     return cudaErrorInvalidValue;
-  static bool done = false;
-  if (!done) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e != cudaSuccess) return e;
-    done = true;
-  }
+  static SmemConfigured configured;
+  if (cudaError_t e = ensure_dyn_smem(gemm_pair_kernel, 227 * 1024, configured); e != cudaSuccess) return e;
   const int st = pair_stages(T);
   size_t pipe = static_cast<size_t>(st) * (GT_BN * 128 + (T / 2) * 128);
   const size_t park = static_cast<size_t>(T) * GT_BN * 4;
@@ -414,12 +407,8 @@ cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream) {
       size_t pipe = static_cast<size_t>(st) * stage;
       const size_t park = static_cast<size_t>(T) * GT_BN * 4;
       if (park > pipe) pipe = park;
-      static bool done2 = false;
-      if (!done2) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024);
-        if (e != cudaSuccess) return e;
-        done2 = true;
-      }
+      static SmemConfigured configured2;
+      if (cudaError_t e = ensure_dyn_smem(gemm_tc_kernel<2>, 112 * 1024, configured2); e != cudaSuccess) return e;
       return launch_k(gemm_tc_kernel<2>, grid, dim3(GT_THREADS), pipe + 1024 + 256, stream, 1, A, st);
     }
   }

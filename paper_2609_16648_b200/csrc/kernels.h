@@ -43,6 +43,21 @@ cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sme
   return launch_kc(kernel, grid, block, smem, stream, dim3(1, 1, cluster_z > 1 ? cluster_z : 1), std::forward<Args>(args)...);
 }
 
+// The opt-in dynamic shared memory size is an attribute per kernel AND per device: `slot` is a function-local static
+// table (one entry per device ordinal) that remembers the largest size already set on each device.
+struct SmemConfigured { size_t bytes[64] = {}; };
+template <typename K>
+cudaError_t ensure_dyn_smem(K kernel, size_t bytes, SmemConfigured &slot) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool tracked = dev >= 0 && dev < 64;
+  if (tracked && bytes <= slot.bytes[dev]) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+  if (e == cudaSuccess && tracked) slot.bytes[dev] = bytes;
+  return e;
+}
+
 constexpr int GM_MAX_K_ = 7;
 constexpr int SAMP_THREADS = 512;
 constexpr int SAMP_CLUSTER = 8;

@@ -258,12 +258,8 @@ cudaError_t launch_record_topk(const RecordTopkArgs &A, int batch, cudaStream_t 
   const int vpc = ((A.V >> 3) + REC_CLUSTER - 1) / REC_CLUSTER;
   const size_t dyn = (static_cast<size_t>(vpc) * 16 + 127) & ~size_t(127);
   if (dyn > 160 * 1024) return cudaErrorInvalidValue;
-  static size_t configured = 0;
-  if (dyn > configured) {
-    cudaError_t e = cudaFuncSetAttribute(record_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(dyn));
-    if (e != cudaSuccess) return e;
-    configured = dyn;
-  }
+  static SmemConfigured configured;
+  if (cudaError_t e = ensure_dyn_smem(record_topk_kernel, dyn, configured); e != cudaSuccess) return e;
   return launch_k(record_topk_kernel, dim3(batch * A.K * REC_CLUSTER), dim3(REC_THREADS), dyn, stream, 1, A);
 }
 

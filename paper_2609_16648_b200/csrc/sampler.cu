@@ -350,12 +350,8 @@ cudaError_t launch_sampler(const SamplerArgs &A, int batch, cudaStream_t stream)
   const size_t stage_b = (static_cast<size_t>(vpc) * 16 + 127) & ~size_t(127);
   const size_t dyn = 2 * stage_b + static_cast<size_t>(vpc) * sizeof(unsigned long long);
   if (dyn > 227 * 1024 - 4096) return cudaErrorInvalidValue;      // vocabulary too large for the shared-memory ring
-  static size_t configured = 0;
-  if (dyn > configured) {
-    cudaError_t e = cudaFuncSetAttribute(sampler_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(dyn));
-    if (e != cudaSuccess) return e;
-    configured = dyn;
-  }
+  static SmemConfigured configured;
+  if (cudaError_t e = ensure_dyn_smem(sampler_kernel, dyn, configured); e != cudaSuccess) return e;
   return launch_k(sampler_kernel, dim3(batch * SAMP_CLUSTER), dim3(SAMP_THREADS), dyn, stream, 1, A);
 }
 

@@ -413,12 +413,8 @@ bool sampler_stream_supported(int V) { return ((V >> 3) + SS_CH - 1) / SS_CH <= 
 
 cudaError_t launch_sampler_stream(const SamplerArgs &A, int batch, cudaStream_t stream) {
   const size_t dyn = static_cast<size_t>(SS_NST) * SS_CH * 16 + static_cast<size_t>(SS_CH) * sizeof(unsigned long long);
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(sampler_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(dyn));
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static SmemConfigured configured;
+  if (cudaError_t e = ensure_dyn_smem(sampler_stream_kernel, dyn, configured); e != cudaSuccess) return e;
   return launch_k(sampler_stream_kernel, dim3(batch), dim3(SS_THREADS), dyn, stream, 1, A);
 }
 

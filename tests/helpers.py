@@ -49,3 +49,38 @@ def push_state(ost, gst, ctx):
     gst.pending_tok.copy_(torch.from_numpy(ptok))
     gst.pending_hidden.copy_(torch.from_numpy(phid).to(torch.bfloat16))
     torch.cuda.synchronize()
+
+
+# ---- "a disagreement is a threshold case": what rounding may explain, and nothing more -----------------------------------
+# Both sides run the same rule (checked bit for bit on the device's own probabilities elsewhere); they may still decide
+# differently because their logits differ by rounding.  A logit row that is off by at most eps (absolute, after the
+# temperature) moves every probability by a factor within exp(+-2 eps) - numerator and normaliser - so the
+# distribution moves by at most E(eps) = exp(2 eps) - 1 in total variation mass.  The helpers below accept a
+# disagreement only if the oracle's own numbers are within that band of the decision boundary.
+
+def band(eps: float) -> float:
+    return float(np.expm1(2.0 * eps))
+
+
+def softmax64(logits, temperature=1.0):
+    x = np.asarray(logits, np.float64) / temperature
+    e = np.exp(x - x.max())
+    return e / e.sum()
+
+
+def draw_is_threshold_case(weights_or, u24: int, tok_dev: int, tok_or: int, delta: float) -> bool:
+    """The oracle drew tok_or at quantile u from its (unnormalised) weights, the device drew tok_dev != tok_or at the
+    same u from its own: explained by rounding iff u lies within `delta` (in normalised CDF mass, the bound on the two
+    CDFs' distance) of the oracle's boundary on the device token's side."""
+    w = np.asarray(weights_or, np.float64)
+    cdf = np.cumsum(w) / w.sum()
+    u = u24 / 2.0 ** 24
+    dist = cdf[tok_dev - 1] - u if tok_dev > tok_or else u - cdf[tok_dev]
+    return dist <= delta + 2.0 ** -20          # + the 24-bit quantile and the 44-bit weight quantisation
+
+
+def accept_bit_is_threshold_case(p_or: float, q_or: float, u24: int, eps_p: float, eps_q: float) -> bool:
+    """Opposite accept bits for the same draft: the margins p - u q have opposite signs on the two sides, so the
+    oracle's margin is at most the two sides' difference, which the logit errors bound."""
+    u = u24 / 2.0 ** 24
+    return abs(p_or - u * q_or) <= band(eps_p) * p_or + band(eps_q) * u * q_or + 1e-12

@@ -69,7 +69,15 @@ def test_accept_decisions_bit_exact_on_dumped_probabilities(B, K, V, sigma, temp
     np.testing.assert_allclose(p.sum(-1), 1.0, atol=2e-5)
     # end to end (oracle softmax in fp64 instead of the device's): decisions agree on almost every row
     ea, et, _ = osampler.accept_batch(tgt, drf, dtok, u24, temp)
-    assert (ea == a.cpu().numpy()).mean() >= 0.8 or B < 5
+    ga = a.cpu().numpy()
+    print(f"accepted lengths equal to the fp64 softmax path on {(ea == ga).sum()} of {B} rows")
+    for b in np.nonzero(ea != ga)[0]:
+        # same logits on both sides, so only the softmax arithmetic differs (<= 5e-6 relative, asserted above): a
+        # different accept bit must sit that close to its threshold u q = p
+        k = int(min(ea[b], ga[b]))
+        pk, qk = ref_p[b, k, dtok[b, k]], ref_q[b, k, dtok[b, k]]
+        u = float(u24[b, k]) / 2.0 ** 24
+        assert abs(pk - u * qk) <= 1e-5 * (pk + u * qk) + 1e-12, ("accept bit differs away from its threshold", b, k)
     # without the dump buffers the result is the same
     a2, t2 = torch.zeros_like(a), torch.zeros_like(t)
     gmb.gm_accept(ctx, None, B, K, temp, _bf16(tgt), _bf16(drf), torch.from_numpy(dtok).cuda(),

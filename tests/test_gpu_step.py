@@ -6,7 +6,8 @@ import torch
 from oracle import philox, sampler as osampler, step as ostep
 from synth_inputs import get_config
 
-from helpers import push_state, rel_err, tiny_setup
+from helpers import (accept_bit_is_threshold_case, band, draw_is_threshold_case, push_state, rel_err, softmax64,
+                     tiny_setup)
 
 pytestmark = pytest.mark.gpu
 
@@ -38,7 +39,7 @@ def _parity_from_common_state(cfg, flags, n_steps, concat=None, top_p=1.0):
     gmb.gm_set_top_p(ctx, top_p)
     bufs = _bufs(B, K, V, d)
     seed = 5
-    bit_agree = bit_total = tok_same = tok_total = fin_same = fin_total = 0
+    bit_agree = bit_total = tok_same = tok_total = fin_same = fin_total = explained = 0
     worst = 0.0
     for it in range(n_steps):
         push_state(ost, gst, ctx)
@@ -64,21 +65,55 @@ def _parity_from_common_state(cfg, flags, n_steps, concat=None, top_p=1.0):
                     rel_err(bufs["tgt_hidden"].float().cpu().numpy(), ref["target_hidden"]))
         for j in range(K + 1):
             worst = max(worst, rel_err(bufs["tgt_logits"][:, j].float().cpu().numpy(), ref["target_logits"][:, j]))
+        dev_dl = bufs["draft_logits"].float().cpu().numpy().astype(np.float64)
+        dev_tl = bufs["tgt_logits"].float().cpu().numpy().astype(np.float64)
         for b in range(B):
             both = min(ga[b], ref["accept_len"][b])                 # positions 0..both-1 accepted by both
             n_eval = min(both + 1, K)                                # ... and the next one is evaluated by both
             bit_total += n_eval
             bit_agree += both + (1 if (both < K and ga[b] == ref["accept_len"][b]) else 0)
+            if ga[b] != ref["accept_len"][b] and top_p >= 1.0:
+                # the first position where the bits differ: the oracle's margin must lie inside the band its logit
+                # rows' measured errors allow
+                k = int(both)
+                eps_p = np.abs(dev_tl[b, k] - ref["target_logits"][b, k]).max()
+                eps_q = np.abs(dev_dl[b, k] - ref["draft_logits"][b, k]).max()
+                d = int(g_dtok[b, k])
+                assert accept_bit_is_threshold_case(softmax64(ref["target_logits"][b, k])[d],
+                                                    softmax64(ref["draft_logits"][b, k])[d], int(ua[b, k]), eps_p, eps_q), \
+                    ("accept bit differs outside the rounding band", it, b, k)
+                explained += 1
             if ga[b] == ref["accept_len"][b]:
                 fin_total += 1
                 fin_same += int(gt[b] == ref["next_token"][b])
+                if gt[b] != ref["next_token"][b] and top_p >= 1.0:
+                    a_ = int(ga[b])
+                    p_or = softmax64(ref["target_logits"][b, a_])
+                    eps_p = np.abs(dev_tl[b, a_] - ref["target_logits"][b, a_]).max()
+                    if a_ < K:                               # residual max(0, p - q), normalised by its own mass
+                        q_or = softmax64(ref["draft_logits"][b, a_])
+                        eps_q = np.abs(dev_dl[b, a_] - ref["draft_logits"][b, a_]).max()
+                        w_or = np.maximum(p_or - q_or, 0.0)
+                        delta = 2.0 * (band(eps_p) + band(eps_q)) / w_or.sum()
+                    else:                                    # all drafts accepted: the extra token comes from p
+                        w_or, delta = p_or, band(eps_p)
+                    assert draw_is_threshold_case(w_or, int(ua[b, K]), int(gt[b]), int(ref["next_token"][b]), delta), \
+                        ("final token differs outside the rounding band", it, b, a_)
+                    explained += 1
         # (3) free-running oracle from the same state and uniforms
         free = ostep.spec_step(w, cfg, ost, K, 1.0, seed=seed, do_commit=True, top_p=top_p)
         tok_total += B
         tok_same += int((g_dtok[:, 0] == free["draft_tok"][:, 0]).sum())
+        for b in range(B):
+            if g_dtok[b, 0] != free["draft_tok"][b, 0]:       # same state, same uniform, different first draft
+                eps_q = np.abs(dev_dl[b, 0] - free["draft_logits"][b, 0]).max()
+                assert draw_is_threshold_case(softmax64(free["draft_logits"][b, 0]), int(ud[b, 0]), int(g_dtok[b, 0]),
+                                              int(free["draft_tok"][b, 0]), band(eps_q)), \
+                    ("first draft token differs outside the rounding band", it, b)
+                explained += 1
     ctx.close()
     print(f"worst rel err {worst:.3e}; accept bits {bit_agree}/{bit_total}; first draft token {tok_same}/{tok_total}; "
-          f"final token {fin_same}/{fin_total}")
+          f"final token {fin_same}/{fin_total}; disagreements shown to be threshold cases: {explained}")
     return worst, (bit_agree, bit_total), (tok_same, tok_total), (fin_same, fin_total)
 
 
@@ -92,8 +127,10 @@ def test_tiny_step_parity_from_common_state(flags, chain, monkeypatch):
         and hidden state agrees within 2e-2 and the accept bits agree on >= 99.5 % of the positions both
         sides evaluate;
     (3) free-running (each side sampling its own drafts from the same uniforms) the sampled tokens agree on
-        most positions - a looser bar, because an inverse-CDF draw turns a relative logit error e into a
-        disagreement probability of order e * sqrt(V).
+        most positions (an inverse-CDF draw turns a relative logit error e into a disagreement probability of
+        order e * sqrt(V)), and EVERY disagreement - a first draft token, an accept bit, a final token - must be a
+        threshold case: the oracle's own quantile / margin lies within the band that the measured error of that
+        logit row allows (helpers.band).  A wrong index or a swapped row does not fit that band; rounding does.
     The tcgen05 path is run three ways (GM_CHAIN_MODE, read when the context is created): every projection a launch of
     its own; the default (the wide gate/up projection on the persistent-pair kernel); and a layer's output projection,
     gate/up, down and the next QKV projection as one persistent launch with the norms folded in."""
@@ -225,6 +262,33 @@ def test_free_running_rollout_keeps_caches_consistent():
         for x, y in zip(dev_h.gather(0, b, m), hkv.gather(0, b, m)):
             assert rel_err(x, y) < TOL
     ctx.close()
+
+
+def test_an_expired_device_side_wait_is_reported_and_the_context_stays_usable():
+    """Failure detection without a GPU fault: a bounded wait that runs out (a barrier nothing arrives on, 1024 polls)
+    sets the status word, the kernel returns normally, the host reads GM_ERR_DEVICE_TIMEOUT once, and the next cycle
+    on the same context is clean and equals the cycle of a context that never saw the timeout."""
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny").with_(prompt_len=24)
+    K, B = cfg.k, cfg.batch
+    outs = []
+    for inject in (True, False):
+        w, ost, ctx, gst = tiny_setup(cfg, cap_tokens=64)
+        push_state(ost, gst, ctx)
+        a = torch.zeros(B, dtype=torch.int32, device="cuda")
+        t = torch.zeros(B, dtype=torch.int32, device="cuda")
+        d = torch.zeros((B, K), dtype=torch.int32, device="cuda")
+        if inject:
+            gmb.gm_selftest_wait_expiry(ctx)
+            assert gmb.gm_last_status(ctx) == gmb.GM_ERR_DEVICE_TIMEOUT
+            assert gmb.gm_strerror(gmb.GM_ERR_DEVICE_TIMEOUT) == "a bounded device-side wait expired"
+            assert gmb.gm_last_status(ctx) == 0                      # sticky until read, then cleared
+        gmb.gm_spec_step(ctx, gst, K, 1.0, 7, 0, a, t, d)
+        assert gmb.gm_last_status(ctx) == 0
+        outs.append((a.clone(), t.clone(), d.clone(), gst.kv_len.clone()))
+        ctx.close()
+    for x, y in zip(*outs):
+        assert torch.equal(x, y)
 
 
 def test_device_seen_errors_and_host_validation():

@@ -58,6 +58,21 @@ def test_reference_arm_prints_one_line_on_rank0_only():
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
 
 
+def test_gpus_flag_starts_the_ranks_itself():
+    """`python bench.py --gpus 2` with no launcher around it re-executes under torch.distributed.run with two ranks
+    (gloo here: no GPU); the line counts both replicas."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run"], capture_output=True,
+                       text=True, env=env, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and lines[0]["n_gpus"] == 2 and lines[0]["sequences_all_ranks"] == 128
+    # a rank count that contradicts the launcher is refused instead of silently measuring fewer GPUs
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "3", "--dry-run"], capture_output=True,
+                       text=True, env=dict(env, RANK="0", WORLD_SIZE="1"), timeout=120)
+    assert r.returncode != 0
+
+
 def test_workload_recipes():
     sys.path.insert(0, ROOT)
     from synth_inputs import get_config, kv_lengths_lognormal, kv_lengths_uniform, make_page_tables
