@@ -7,10 +7,10 @@
 // CTA pairs (one pair per two SMs, all resident at once) that walks the projections ("phases") in order:
 //
 //   * a pair's tile is 256 token rows (128 per CTA, on the lanes of tensor memory) x W output features, W a multiple of
-//     32 up to 288, computed by tcgen05.mma cta_group::2 (M = 256, N = W as one or two instructions per K step).  Per
+//     16 up to 288, computed by tcgen05.mma cta_group::2 (M = 256, N = W as one or two instructions per K step).  Per
 //     K block of 64 a CTA stages its own 128 x 64 activation box and W / 2 weight rows.  The features of a phase are
 //     dealt out in near-equal tiles, as many as there are pairs, so every phase is one wave: wide projections get
-//     W = 256 / 288, narrow ones thin tiles (W = 32 ... 96) instead of a deep split along K - a thin tile re-reads the
+//     W = 256 / 272, narrow ones thin tiles (W = 32 ... 96) instead of a deep split along K - a thin tile re-reads the
 //     activations from L2 more often, but leaves nothing to reduce across SMs.  Only a projection with a long K and few
 //     features (down) is cut along K as well, over ns = 2 ... 8 consecutive pairs: the K slices leave fp32 partial sums
 //     in an L2-resident scratch slot per CTA, meet at a counter of their own, and each slice owner reduces one slice of
@@ -139,7 +139,7 @@ __device__ __forceinline__ bool chain_item(const ChainPhase &ph, int mblocks, in
   it.mb = unit % mblocks; it.tile = unit / mblocks;              // token blocks vary fastest: neighbours share a weight tile
   const int g_lo = static_cast<int>(static_cast<long long>(it.tile) * ph.G / ph.tiles);
   const int g_hi = static_cast<int>(static_cast<long long>(it.tile + 1) * ph.G / ph.tiles);
-  it.f0 = g_lo * 32; it.W = (g_hi - g_lo) * 32;
+  it.f0 = g_lo * 16; it.W = (g_hi - g_lo) * 16;
   const int KB = ph.K / CH_BK;
   it.kb_lo = static_cast<int>(static_cast<long long>(it.split) * KB / ph.ns);
   it.kb_hi = static_cast<int>(static_cast<long long>(it.split + 1) * KB / ph.ns);
@@ -166,13 +166,14 @@ struct SlotIter {
     if (++kb >= it.kb_hi) { ++idx; seek(A, pair); }
   }
 };
-// Feature (relative to the tile's first) held by accumulator column `col` (a multiple of 4; 16-column blocks stay
-// contiguous).  One MMA (W <= 256): the even CTA's weight rows are columns [0, W/2), the odd CTA's [W/2, W): identity.
-// Two MMAs (W > 256) of n1 and W - n1 columns: the first takes the first n1 / 2 weight rows of both CTAs' boxes, the
-// second the rows behind.
+// Feature (relative to the tile's first) held by accumulator column `col` (a multiple of 4; runs of 8 columns stay
+// contiguous).  One MMA (W <= 256): the even CTA's W / 2 weight rows are columns [0, W/2), the odd CTA's [W/2, W):
+// identity.  Two MMAs (W > 256) of n1 and W - n1 columns: the first takes the first n1 / 2 weight rows of both CTAs'
+// boxes, the second the rows behind.
+__device__ __forceinline__ int chain_n1(int W) { return W <= 256 ? W : 16 * ((W + 31) / 32); }
 __device__ __forceinline__ int chain_col_feature(int col, int W) {
   if (W <= 256) return col;
-  const int hw = W >> 1, n1 = (hw + 31) & ~31, h1 = n1 >> 1;   // first MMA: n1 columns, h1 weight rows of each CTA
+  const int hw = W >> 1, n1 = chain_n1(W), h1 = n1 >> 1;      // first MMA: n1 columns, h1 weight rows of each CTA
   if (col < n1) return (col / h1) * hw + col % h1;
   const int h2 = (W - n1) >> 1, c2 = col - n1;
   return (c2 / h2) * hw + h1 + c2 % h2;
@@ -273,7 +274,7 @@ chain_kernel(const __grid_constant__ ChainArgs A) {
       int q = 0, last_q = -1;
       bool ok = true;
       unsigned long long t_wait = 0, t_issue = 0;
-      const bool timed = A.timeline != nullptr && pi == 0;
+      const bool timed = A.timeline != nullptr && A.trace_phase >= 100 && pi == 0;   // interval sums perturb the loop: on request only
       for (; it.valid && ok; it.next(A, pair), ++q) {
         if (q % np != pi) continue;
         const int s = q % nstages;
@@ -323,7 +324,7 @@ chain_kernel(const __grid_constant__ ChainArgs A) {
       int q = 0, item_no = 0;
       bool ok = true;
       unsigned long long t_wait = 0, t_issue = 0, pw[4] = {0, 0, 0, 0}, pi_[4] = {0, 0, 0, 0};
-      const bool timed = A.timeline != nullptr;
+      const bool timed = A.timeline != nullptr && A.trace_phase >= 100;
       const uint32_t smem0 = smem_u32(smem);
       for (int p = 0; p < A.n_phases && ok; ++p) {
         ChainItem it;
@@ -333,7 +334,7 @@ chain_kernel(const __grid_constant__ ChainArgs A) {
           tc_fence_after();
           // one MMA per K step for tiles up to 256 features; wider tiles as two of about half the width each (an
           // instruction of this shape takes at least ~85 cycles however narrow, and N / 2 cycles beyond N = 170)
-          const int W = it.W, n1 = W <= 256 ? W : (((W >> 1) + 31) & ~31), n2 = W - n1;
+          const int W = it.W, n1 = chain_n1(W), n2 = W - n1;
           const uint32_t idesc1 = tc_idesc_bf16(2 * CH_TOK, n1), idesc2 = n2 ? tc_idesc_bf16(2 * CH_TOK, n2) : 0u;
           const uint32_t b2_off = static_cast<uint32_t>(n1 >> 1) * 128u;
           for (int kb = it.kb_lo; kb < it.kb_hi; ++kb, ++q) {
@@ -346,14 +347,20 @@ chain_kernel(const __grid_constant__ ChainArgs A) {
             const uint32_t a_addr = smem0 + static_cast<uint32_t>(s) * stage_b;
             const uint64_t adesc = tc_smem_desc_sw128(a_addr), bdesc = tc_smem_desc_sw128(a_addr + CH_A_BYTES);
             const uint32_t acc = kb > it.kb_lo ? 1u : 0u;
-            tc2_mma_bf16(tmem, adesc, bdesc, idesc1, acc);
+            if (n2 == 0) {
+              tc2_mma_bf16(tmem, adesc, bdesc, idesc1, acc);
 #pragma unroll
-            for (int k = 1; k < CH_BK / 16; ++k) tc2_mma_bf16(tmem, adesc + 2 * k, bdesc + 2 * k, idesc1, 1u);
-            if (n2 > 0) {                            // the weight rows behind the first n1 / 2 of both CTAs' boxes
+              for (int k = 1; k < CH_BK / 16; ++k) tc2_mma_bf16(tmem, adesc + 2 * k, bdesc + 2 * k, idesc1, 1u);
+            } else {
+              // Two column ranges (the second from the weight rows behind the first n1 / 2 of both CTAs' boxes), issued
+              // alternately: consecutive MMAs into the SAME accumulator wait for one another (about 85 cycles each,
+              // measured), MMAs into different column ranges overlap.
               const uint64_t bdesc2 = tc_smem_desc_sw128(a_addr + CH_A_BYTES + b2_off);
-              tc2_mma_bf16(tmem + n1, adesc, bdesc2, idesc2, acc);
 #pragma unroll
-              for (int k = 1; k < CH_BK / 16; ++k) tc2_mma_bf16(tmem + n1, adesc + 2 * k, bdesc2 + 2 * k, idesc2, 1u);
+              for (int k = 0; k < CH_BK / 16; ++k) {
+                tc2_mma_bf16(tmem, adesc + 2 * k, bdesc + 2 * k, idesc1, k > 0 ? 1u : acc);
+                tc2_mma_bf16(tmem + n1, adesc + 2 * k, bdesc2 + 2 * k, idesc2, k > 0 ? 1u : acc);
+              }
             }
             tc2_commit_mc(&empty[s], 3);             // the stage is free in both CTAs once these MMAs have read it
             if (timed) {
@@ -439,7 +446,7 @@ chain_kernel(const __grid_constant__ ChainArgs A) {
         float ssq = 0.f;                                         // sum of squares of this thread's results
 #pragma unroll 1
         for (int b = chunk; b < nblk; b += 4) {
-          const int col = b << 4, n = it.f0 + chain_col_feature(col, W);   // 16 feature columns
+          const int col = b << 4;                    // 16 accumulator columns
           uint32_t v[16];
           if (acc_ok) {
             tc_ld_32x16(tmem + (static_cast<uint32_t>(quad * 32) << 16) + col, v);
@@ -455,45 +462,42 @@ chain_kernel(const __grid_constant__ ChainArgs A) {
             continue;
           }
           if (!row_live) continue;
-          if (ph.epi == EPI_SWIGLU_BF16) {           // columns (2 i, 2 i + 1) = (gate_i, up_i)
-            uint32_t o[4];
+          // two runs of 8 columns, each 8 consecutive features (the runs of a block need not be neighbours in a tile of two MMAs)
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              o[j] = pack_bf16(silu_mul(__uint_as_float(v[4 * j]) * rs, __uint_as_float(v[4 * j + 1]) * rs),
-                               silu_mul(__uint_as_float(v[4 * j + 2]) * rs, __uint_as_float(v[4 * j + 3]) * rs));
-            *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(ph.out) + static_cast<size_t>(m) * ph.ldo + (n >> 1)) =
-                make_uint4(o[0], o[1], o[2], o[3]);
-          } else if (ph.epi == EPI_STORE_BF16) {
-            uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(ph.out) + static_cast<size_t>(m) * ph.ldo + n);
-#pragma unroll
-            for (int j = 0; j < 2; ++j)
-              dst[j] = make_uint4(pack_bf16(__uint_as_float(v[8 * j]) * rs, __uint_as_float(v[8 * j + 1]) * rs),
-                                  pack_bf16(__uint_as_float(v[8 * j + 2]) * rs, __uint_as_float(v[8 * j + 3]) * rs),
-                                  pack_bf16(__uint_as_float(v[8 * j + 4]) * rs, __uint_as_float(v[8 * j + 5]) * rs),
-                                  pack_bf16(__uint_as_float(v[8 * j + 6]) * rs, __uint_as_float(v[8 * j + 7]) * rs));
-          } else {                                   // residual-stream update (EPI_ADD_F32) or plain fp32 store
-            float4 *o4 = reinterpret_cast<float4 *>(reinterpret_cast<float *>(ph.out) + static_cast<size_t>(m) * ph.ldo + n);
-            float x[16];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
-              if (ph.epi == EPI_ADD_F32) r = o4[j];
-              x[4 * j] = __uint_as_float(v[4 * j]) * rs + r.x; x[4 * j + 1] = __uint_as_float(v[4 * j + 1]) * rs + r.y;
-              x[4 * j + 2] = __uint_as_float(v[4 * j + 2]) * rs + r.z; x[4 * j + 3] = __uint_as_float(v[4 * j + 3]) * rs + r.w;
-              o4[j] = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
-            }
-#pragma unroll
-            for (int j = 0; j < 16; ++j) ssq += x[j] * x[j];
-            if (ph.xg) {
-              const uint4 *gw = reinterpret_cast<const uint4 *>(ph.gamma + n);
-              uint4 *dst = reinterpret_cast<uint4 *>(ph.xg + static_cast<size_t>(m) * ph.N + n);
+          for (int h8 = 0; h8 < 2; ++h8) {
+            const int n = it.f0 + chain_col_feature(col + 8 * h8, W);
+            const uint32_t *u = v + 8 * h8;
+            if (ph.epi == EPI_SWIGLU_BF16) {         // columns (2 i, 2 i + 1) = (gate_i, up_i)
+              uint2 o;
+              o.x = pack_bf16(silu_mul(__uint_as_float(u[0]) * rs, __uint_as_float(u[1]) * rs),
+                              silu_mul(__uint_as_float(u[2]) * rs, __uint_as_float(u[3]) * rs));
+              o.y = pack_bf16(silu_mul(__uint_as_float(u[4]) * rs, __uint_as_float(u[5]) * rs),
+                              silu_mul(__uint_as_float(u[6]) * rs, __uint_as_float(u[7]) * rs));
+              *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(ph.out) + static_cast<size_t>(m) * ph.ldo + (n >> 1)) = o;
+            } else if (ph.epi == EPI_STORE_BF16) {
+              *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(ph.out) + static_cast<size_t>(m) * ph.ldo + n) =
+                  make_uint4(pack_bf16(__uint_as_float(u[0]) * rs, __uint_as_float(u[1]) * rs),
+                             pack_bf16(__uint_as_float(u[2]) * rs, __uint_as_float(u[3]) * rs),
+                             pack_bf16(__uint_as_float(u[4]) * rs, __uint_as_float(u[5]) * rs),
+                             pack_bf16(__uint_as_float(u[6]) * rs, __uint_as_float(u[7]) * rs));
+            } else {                                 // residual-stream update (EPI_ADD_F32) or plain fp32 store
+              float4 *o4 = reinterpret_cast<float4 *>(reinterpret_cast<float *>(ph.out) + static_cast<size_t>(m) * ph.ldo + n);
+              float x[8];
 #pragma unroll
               for (int j = 0; j < 2; ++j) {
-                const uint4 g = gw[j];
-                dst[j] = make_uint4(pack_bf16(x[8 * j] * bf16_lo(g.x), x[8 * j + 1] * bf16_hi(g.x)),
-                                    pack_bf16(x[8 * j + 2] * bf16_lo(g.y), x[8 * j + 3] * bf16_hi(g.y)),
-                                    pack_bf16(x[8 * j + 4] * bf16_lo(g.z), x[8 * j + 5] * bf16_hi(g.z)),
-                                    pack_bf16(x[8 * j + 6] * bf16_lo(g.w), x[8 * j + 7] * bf16_hi(g.w)));
+                float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (ph.epi == EPI_ADD_F32) r = o4[j];
+                x[4 * j] = __uint_as_float(u[4 * j]) * rs + r.x; x[4 * j + 1] = __uint_as_float(u[4 * j + 1]) * rs + r.y;
+                x[4 * j + 2] = __uint_as_float(u[4 * j + 2]) * rs + r.z; x[4 * j + 3] = __uint_as_float(u[4 * j + 3]) * rs + r.w;
+                o4[j] = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
+              }
+#pragma unroll
+              for (int j = 0; j < 8; ++j) ssq += x[j] * x[j];
+              if (ph.xg) {
+                const uint4 g = *reinterpret_cast<const uint4 *>(ph.gamma + n);
+                *reinterpret_cast<uint4 *>(ph.xg + static_cast<size_t>(m) * ph.N + n) =
+                    make_uint4(pack_bf16(x[0] * bf16_lo(g.x), x[1] * bf16_hi(g.x)), pack_bf16(x[2] * bf16_lo(g.y), x[3] * bf16_hi(g.y)),
+                               pack_bf16(x[4] * bf16_lo(g.z), x[5] * bf16_hi(g.z)), pack_bf16(x[6] * bf16_lo(g.w), x[7] * bf16_hi(g.w)));
               }
             }
           }
@@ -637,14 +641,14 @@ cudaError_t chain_max_pairs(int *out) {
 
 size_t chain_partial_floats(int pairs) { return static_cast<size_t>(pairs) * 2 * CH_TOK * CH_WMAX; }
 
-// Tiling of one phase: `tiles` near-equal feature tiles (multiples of 32 features, at most 288) and ns K slices per
+// Tiling of one phase: `tiles` near-equal feature tiles (multiples of 16 features, at most 288) and ns K slices per
 // tile, chosen from a cost estimate per pair - K blocks x the slower of the tensor time and the time to fill shared
 // memory (activation box + weight rows), per wave, plus what the slices' partial sums cost - over ns = 1 ... 8.  A
 // deterministic function of (N, K, mblocks, P): the arithmetic of a token row does not depend on the batch it is in.
 void chain_schedule(ChainPhase &ph, int mblocks, int P, int force_ns) {
-  const int G = ph.N / 32, KB = ph.K / CH_BK;
+  const int G = ph.N / 16, KB = ph.K / CH_BK;        // groups of 16 features
   ph.G = G;
-  const int min_tiles = (G + CH_WMAX / 32 - 1) / (CH_WMAX / 32);
+  const int min_tiles = (G + CH_WMAX / 16 - 1) / (CH_WMAX / 16);
   double best = 1e30;
   int best_ns = 1, best_tiles = min_tiles;
   for (int ns = 1; ns <= 8 && ns <= KB; ++ns) {
@@ -654,8 +658,8 @@ void chain_schedule(ChainPhase &ph, int mblocks, int P, int force_ns) {
     if (tiles < min_tiles) { if (ns > 1) continue; tiles = min_tiles; }   // several waves: no K slices
     const int Pp = P - P % ns;
     const int waves = (tiles * mblocks * ns + Pp - 1) / Pp;
-    const int gw = (G + tiles - 1) / tiles;          // widest tile in groups of 32 features
-    const int w = 32 * gw, n1 = w <= 256 ? w : (((w >> 1) + 31) & ~31), n2 = w - n1;
+    const int gw = (G + tiles - 1) / tiles;          // widest tile in groups of 16 features
+    const int w = 16 * gw, n1 = w <= 256 ? w : 16 * ((w + 31) / 32), n2 = w - n1;
     // measured on B200: one MMA of this shape per K step of 16 takes max(85, N / 2) cycles at 1.965 GHz; a K block costs
     // about 0.1 us of barrier round trips on top; a CTA fills shared memory at roughly 140 KB per us
     const double cyc = (n1 / 2 > 85 ? n1 / 2 : 85) + (n2 ? (n2 / 2 > 85 ? n2 / 2 : 85) : 0);
@@ -669,7 +673,7 @@ void chain_schedule(ChainPhase &ph, int mblocks, int P, int force_ns) {
   }
   ph.ns = best_ns;
   ph.tiles = best_tiles;
-  ph.wbox = ((G + best_tiles - 1) / best_tiles) * 16;           // weight rows per CTA of the widest tile
+  ph.wbox = ((G + best_tiles - 1) / best_tiles) * 8;            // weight rows per CTA of the widest tile
 }
 
 cudaError_t launch_chain(const ChainArgs &A, cudaStream_t stream) {
@@ -678,8 +682,8 @@ cudaError_t launch_chain(const ChainArgs &A, cudaStream_t stream) {
     return cudaErrorInvalidValue;
   for (int p = 0; p < A.n_phases; ++p) {
     const ChainPhase &ph = A.ph[p];
-    if ((ph.K % CH_BK) || (ph.N % 32) || ph.K < CH_BK || (ph.ldo % 8) || ph.ns < 1 || ph.ns > 8 || ph.tiles < 1 ||
-        ph.G != ph.N / 32 || ph.wbox < 16 || ph.wbox > CH_WMAX / 2 || (ph.G + ph.tiles - 1) / ph.tiles * 16 > ph.wbox ||
+    if ((ph.K % CH_BK) || (ph.N % 16) || ph.K < CH_BK || (ph.ldo % 8) || ph.ns < 1 || ph.ns > 8 || ph.tiles < 1 ||
+        ph.G != ph.N / 16 || ph.wbox < 8 || ph.wbox > CH_WMAX / 2 || (ph.G + ph.tiles - 1) / ph.tiles * 8 > ph.wbox ||
         (ph.ns > 1 && ph.tiles * A.mblocks * ph.ns > A.P) || (ph.sq_in && ph.sq_out))
       return cudaErrorInvalidValue;
   }

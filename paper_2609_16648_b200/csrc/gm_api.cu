@@ -96,7 +96,7 @@ int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *w
   // A SwiGLU projection wide enough for one tile per CTA pair (gate/up): one wave of the persistent-pair kernel - tiles
   // of 256 / 288 features sized so that the wave is exact - instead of a full wave plus a short tail launch.
   if (c->chain_on && c->chain_mode >= 1 && epi == EPI_SWIGLU_BF16 && M <= c->chain_max_m && N >= c->chain_pairs * 128 &&
-      N <= c->chain_pairs * 288 && (N % 32) == 0 && (ldo % 8) == 0) {
+      N <= c->chain_pairs * 288 && (N % 16) == 0 && (ldo % 8) == 0) {
     const ChainSpec g = {w, x, x_rows, N, K, out, epi, static_cast<int>(ldo), nullptr, nullptr, nullptr, nullptr, 0, 0};
     return run_chain(c, &g, 1, M);
   }
@@ -460,8 +460,8 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
     if (pairs >= 1) {
       c->chain_pairs = pairs;
       A_(dev_alloc(c, &c->chain_partial, chain_partial_floats(pairs)));
-      A_(dev_alloc(c, &c->chain_sq[0], static_cast<size_t>((c->d + 31) / 32) * M));     // one row per feature tile (at most per 32 features)
-      A_(dev_alloc(c, &c->chain_sq[1], static_cast<size_t>((c->d + 31) / 32) * M));
+      A_(dev_alloc(c, &c->chain_sq[0], static_cast<size_t>((c->d + 15) / 16) * M));     // one row per feature tile (at most per 16 features)
+      A_(dev_alloc(c, &c->chain_sq[1], static_cast<size_t>((c->d + 15) / 16) * M));
       A_(dev_alloc(c, &c->chain_sync, 1 + static_cast<size_t>(pairs) * 2));
       if (const char *ov = std::getenv("GM_CHAIN_NS"))
         std::sscanf(ov, "%d,%d,%d,%d", &c->chain_force_ns[0], &c->chain_force_ns[1], &c->chain_force_ns[2], &c->chain_force_ns[3]);

@@ -358,7 +358,7 @@ struct ChainPhase {
   int epi;
   int N, K;
   int ldo;
-  int G, tiles, ns, wbox;               // schedule (chain_schedule): groups of 32 features, feature tiles, K slices per
+  int G, tiles, ns, wbox;               // schedule (chain_schedule): groups of 16 features, feature tiles, K slices per
                                         // tile, weight rows a CTA stages per K block (half of the widest tile)
 };
 struct ChainArgs {
