@@ -18,13 +18,18 @@ dL/dalpha_k is Eq. 8 with the chain sums cut at min(j, K) (zero beyond the cut).
 in q_k: on a retained token the slope is 1 where q < p, and the residual bin, q_res = 1 - (sum of q over the
 retained tokens), contributes -1 on every retained token where q_res < p_res; at a tie the slope is taken as 0.
 The chain rule through q = softmax(logits / T) gives dalpha/dlogit_v = q_v (g_v - sum_d q_d g_d) / T.
+
+Second step (Alg. 1, "update phi"): from the logits back to the head state g_k that produced them.  The head's logits
+are LMhead(RMSNorm_hf(g_k)) with the backbone's LM head (App. B.1), so dL/dy = (dL/dlogits) W_lm for the normed state y
+and dL/dg follows from the derivative of the RMSNorm.  This is the partial derivative through the logits of position
+k alone; the recurrence g_k -> g_{k+1} (Eq. 4) adds further terms in a later step of the backward pass.
 """
 from __future__ import annotations
 
 import numpy as np
 
 from . import record, sampler
-from .model import PagedKV, head_forward, head_logits, round_bf16
+from .model import PagedKV, f64, head_forward, head_logits, round_bf16
 
 
 def reconstruct_chain(w, cfg, seq_hidden, seq_tokens, start_len: int, drafts, temperature: float = 1.0,
@@ -143,3 +148,29 @@ def head_update_loss(w, cfg, sequences, records, temperature: float = 1.0, round
         alphas.append(a)
         losses.append(dca_loss(a, rec["accepted"]))
     return float(np.mean(losses)), np.array(alphas)
+
+
+def lm_head_input_grad(grad_logits, w_lm) -> np.ndarray:
+    """logits = y W_lm^T  =>  dL/dy = (dL/dlogits) W_lm.   grad_logits [..., V], w_lm [V, d]  ->  [..., d]."""
+    return np.asarray(grad_logits, np.float64) @ f64(w_lm)
+
+
+def rmsnorm_grad(dy, x, weight, eps: float) -> np.ndarray:
+    """Derivative of y = x r w, r = (mean(x^2) + eps)^(-1/2), with respect to x:
+    dL/dx = r (w dy) - x r^3 mean(x w dy)   (the second term is the derivative of r)."""
+    x, dy, w = f64(x), f64(dy), f64(weight)
+    r = 1.0 / np.sqrt((x * x).mean(axis=-1, keepdims=True) + eps)
+    wdy = w * dy
+    return r * wdy - x * r ** 3 * (x * wdy).mean(axis=-1, keepdims=True)
+
+
+def head_update_grad_state(w, cfg, states, records, temperature: float = 1.0):
+    """d(mean over cycles of Eq. 9)/d(head states), through the head's final norm and the shared LM head only.
+    states [n, K, d] = g_k of every recorded cycle (what the reconstruction computes); records = the n record dicts.
+    Returns (grad_state [n, K, d], grad_normed [n, K, d], logits [n, K, V])."""
+    states = np.asarray(states, np.float64)
+    n, K, d = states.shape
+    logits = head_logits(w, states.reshape(n * K, d), cfg).reshape(n, K, -1)
+    gl = head_update_grad_logits(logits, records, temperature)
+    gy = lm_head_input_grad(gl, w["lm_head"])
+    return rmsnorm_grad(gy, states, w["head"]["final_norm"], cfg.rms_eps), gy, logits

@@ -181,3 +181,44 @@ def test_logit_gradient_matches_finite_differences_of_the_objective():
         np.testing.assert_allclose(g, fd, rtol=2e-5, atol=1e-9)
         for r, rec in enumerate(recs):                       # positions after the first rejection get no gradient
             assert (g[r, min(rec["accepted"], K):] == 0).all() and np.abs(g[r, 0]).max() > 0
+
+
+def test_rmsnorm_gradient_matches_finite_differences():
+    rng = np.random.default_rng(11)
+    x, w, dy = rng.normal(0, 1.5, (3, 12)), rng.uniform(0.5, 1.5, 12), rng.normal(0, 1, (3, 12))
+    eps = 1e-3                                                 # large enough to matter
+    f = lambda xx: float((model.rmsnorm(xx, w, eps) * dy).sum())
+    g = update.rmsnorm_grad(dy, x, w, eps)
+    for i in np.ndindex(*x.shape):
+        e = np.zeros_like(x)
+        e[i] = 1e-6
+        assert g[i] == pytest.approx((f(x + e) - f(x - e)) / 2e-6, rel=1e-6, abs=1e-9)
+    # a row scaled by c has the same normed output (eps aside): the gradient is orthogonal to x when eps = 0
+    g0 = update.rmsnorm_grad(dy, x, w, 0.0)
+    assert np.abs((g0 * x).sum(-1)).max() < 1e-12
+
+
+def test_head_state_gradient_matches_finite_differences_of_the_objective():
+    """state -> head norm -> shared LM head -> softmax -> overlap with residual bin -> truncated loss -> mean,
+    differentiated numerically with respect to every coordinate of every head state."""
+    rng = np.random.default_rng(5)
+    n, K, V, d, T = 3, 3, 14, 6, 0.8
+    cfg = CFG.with_(d_model=d, vocab=V, rms_eps=1e-4)
+    w = {"lm_head": rng.normal(0, 0.8, (V, d)), "head": {"final_norm": rng.uniform(0.6, 1.4, d)}}
+    for kept in (5, 14):
+        recs = _toy_records(rng, n, K, V, kept, T)
+        states = rng.normal(0, 1.0, (n, K, d))
+        g, gy, logits = update.head_update_grad_state(w, cfg, states, recs, T)
+        np.testing.assert_allclose(logits, model.head_logits(w, states.reshape(-1, d), cfg).reshape(n, K, V))
+        loss = lambda st: _mean_loss(model.head_logits(w, st.reshape(-1, d), cfg).reshape(n, K, V), recs, T)
+        fd = np.zeros_like(g)
+        for i in np.ndindex(n, K, d):
+            e = np.zeros_like(states)
+            e[i] = 1e-6
+            fd[i] = (loss(states + e) - loss(states - e)) / 2e-6
+        np.testing.assert_allclose(g, fd, rtol=5e-5, atol=1e-9)
+        # the LM-head step alone: a matrix product with the untransposed weight (row of logits gradient times W_lm)
+        gl = update.head_update_grad_logits(logits, recs, T)
+        np.testing.assert_allclose(gy, np.einsum("nkv,vd->nkd", gl, w["lm_head"]), rtol=1e-12)
+        for r, rec in enumerate(recs):                       # positions after the first rejection get no gradient
+            assert (g[r, min(rec["accepted"], K):] == 0).all()
