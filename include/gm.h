@@ -363,6 +363,12 @@ int gm_head_prefill(gm_ctx *ctx, gm_state *st, const void *seq_hidden, int hid_s
 int gm_reconstruct(gm_ctx *ctx, gm_state *st, int n_cycles, int k, const int32_t *cycle_seq,
                    const gm_record *rec, const int32_t *seq_tok, int tok_stride,
                    const int32_t *scratch_pages, void *draft_logits);
+/* gm_reconstruct that also returns the head states: head_states fp32 [n_cycles, k, d] out (or NULL) receives
+ * g_j of every chain and depth, the state the head's final norm and the LM head turn into draft_logits[r, j]
+ * (Eq. 4) - the point the backward pass re-enters the head at.                                             */
+int gm_reconstruct_states(gm_ctx *ctx, gm_state *st, int n_cycles, int k, const int32_t *cycle_seq,
+                          const gm_record *rec, const int32_t *seq_tok, int tok_stride,
+                          const int32_t *scratch_pages, void *draft_logits, float *head_states);
 int gm_overlap(gm_ctx *ctx, int n_cycles, int k, float temperature, const void *draft_logits,
                const gm_record *rec, float *alpha, float *lse);
 int gm_dca_loss(gm_ctx *ctx, int n_cycles, int k, const float *alpha, const int32_t *accepted,
@@ -370,6 +376,21 @@ int gm_dca_loss(gm_ctx *ctx, int n_cycles, int k, const float *alpha, const int3
 int gm_dca_grad(gm_ctx *ctx, int n_cycles, int k, float temperature, const void *draft_logits,
                 const gm_record *rec, const float *alpha, const float *lse, const int32_t *accepted,
                 void *grad_logits);
+/* Second step of the backward pass (Alg. 1, "update phi"): from the logits back to the head states.  The head's
+ * logits are LMhead(RMSNorm(g; head final norm)) with the backbone's LM head (App. B.1), which the head update
+ * leaves fixed, so no weight gradient is formed here.
+ *   grad_logits  device bf16 [rows, V], rows = n_cycles * k: gm_dca_grad's output
+ *   grad_normed  device fp32 [rows, d] out: dL/dy = grad_logits x W_lm for the normed state y (one projection with
+ *                the vocabulary as its contraction dimension, fp32 accumulation)
+ *   head_states  device fp32 [rows, d] in, grad_states device fp32 [rows, d] out: dL/dg through the norm,
+ *                r (w dy) - g r^3 mean(g w dy) with r = (mean(g^2) + eps)^(-1/2); both NULL = skip this step.
+ *                This is the derivative through the logits of the state's own position; the terms that reach
+ *                g_j through g_{j+1} (Eq. 4) belong to the backward pass of the head layer, which is not built.
+ * The projection reads a transposed copy [d, V] of the LM head that the context makes on the first call (d * V
+ * bf16 of device memory, kept until gm_free); refresh_weights != 0 remakes it, for a caller that has rewritten the
+ * LM head's weights in place since.  V % 64 != 0 returns GM_ERR_UNSUPPORTED.                                   */
+int gm_head_state_grad(gm_ctx *ctx, int rows, const void *grad_logits, const float *head_states,
+                       float *grad_normed, float *grad_states, int refresh_weights);
 
 
 /* Dense projection out[M, N] = x[M, K] w[N, K]^T on the context's stream (bf16 in, fp32

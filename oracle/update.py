@@ -32,22 +32,30 @@ from . import record, sampler
 from .model import PagedKV, f64, head_forward, head_logits, round_bf16
 
 
-def reconstruct_chain(w, cfg, seq_hidden, seq_tokens, start_len: int, drafts, temperature: float = 1.0,
-                      round_interface: bool = True):
-    """Eq. 4 for one cycle.  seq_hidden[i] = H_i, the target hidden state that produced token x_{i+1};
-    seq_tokens = the sequence's committed tokens; start_len = Len >= 2 (a prompt token and the first
-    response token at least).
-    Returns (q[K, V] fp32, logits[K, V])."""
+def reconstruct_states(w, cfg, seq_hidden, seq_tokens, start_len: int, drafts) -> np.ndarray:
+    """The recurrence of Eq. 4 for one cycle: g_1 from the committed prefix, g_k from (g_{k-1}, d_{k-1}).
+    seq_hidden[i] = H_i, the target hidden state that produced token x_{i+1}; seq_tokens = the sequence's
+    committed tokens; start_len = Len >= 2 (a prompt token and the first response token at least).  Returns g [K, d]."""
     Len, K = int(start_len), len(drafts)
     assert Len >= 2 and len(seq_tokens) >= Len and len(seq_hidden) >= Len - 1
     pages = (Len + K + cfg.page_size) // cfg.page_size + 1
     hkv = PagedKV(1, cfg.n_kv_heads, cfg.head_dim, np.arange(pages)[None, :], pages, cfg.page_size)
     g = head_forward(w, np.asarray(seq_hidden)[:Len - 1], list(seq_tokens[1:Len]), np.arange(Len - 1), hkv, 0, cfg)[-1:]
-    qs, lgs = [], []
+    gs = []
     for k in range(1, K + 1):
         if k > 1:
             g = head_forward(w, g, [int(drafts[k - 2])], np.array([Len + k - 3]), hkv, 0, cfg)
-        lg = head_logits(w, g, cfg)[0]
+        gs.append(g[0])
+    return np.array(gs)
+
+
+def reconstruct_chain(w, cfg, seq_hidden, seq_tokens, start_len: int, drafts, temperature: float = 1.0,
+                      round_interface: bool = True):
+    """Eq. 4 for one cycle: q_k = softmax(LMhead(norm(g_k)) / T) from the states above.
+    Returns (q[K, V] fp32, logits[K, V])."""
+    qs, lgs = [], []
+    for g in reconstruct_states(w, cfg, seq_hidden, seq_tokens, start_len, drafts):
+        lg = head_logits(w, g[None, :], cfg)[0]
         if round_interface:
             lg = round_bf16(lg).astype(np.float64)
         lgs.append(lg)

@@ -24,7 +24,7 @@ GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER, GM_KC_RECORD = 0,
 
 EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw", "gm_set_top_p", "gm_nucleus", "gm_prefill",
            "gm_rollout_begin", "gm_rollout_step", "gm_rollout_run", "gm_pages_reset", "gm_pages_reserve",
-           "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_overlap", "gm_dca_loss", "gm_dca_grad",
+           "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_reconstruct_states", "gm_head_state_grad", "gm_overlap", "gm_dca_loss", "gm_dca_grad",
            "gm_spec_step_host", "gm_gemm", "gm_gemm_swiglu", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
            "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_chain_trace", "gm_chain_trace_read", "gm_selftest_wait_expiry", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
@@ -94,6 +94,8 @@ def lib() -> C.CDLL:
     L.gm_capture_hidden.argtypes = [vp, vp, i32]
     L.gm_head_prefill.argtypes = [vp, C.POINTER(gm_state), vp, i32, vp, i32, vp, i32]
     L.gm_reconstruct.argtypes = [vp, C.POINTER(gm_state), i32, i32, vp, C.POINTER(gm_record), vp, i32, vp, vp]
+    L.gm_reconstruct_states.argtypes = [vp, C.POINTER(gm_state), i32, i32, vp, C.POINTER(gm_record), vp, i32, vp, vp, vp]
+    L.gm_head_state_grad.argtypes = [vp, i32, vp, vp, vp, vp, i32]
     L.gm_overlap.argtypes = [vp, i32, i32, f32, vp, C.POINTER(gm_record), vp, vp]
     L.gm_dca_loss.argtypes = [vp, i32, i32, vp, vp, vp, vp]
     L.gm_dca_grad.argtypes = [vp, i32, i32, f32, vp, C.POINTER(gm_record), vp, vp, vp, vp]
@@ -387,9 +389,22 @@ def gm_head_prefill(ctx: Context, st: State, seq_hidden, seq_tok, seq_len, max_l
                                  seq_tok.shape[1], _p(seq_len), max_len), "gm_head_prefill")
 
 
-def gm_reconstruct(ctx: Context, st: State, n_cycles: int, k: int, cycle_seq, rec, seq_tok, scratch_pages, draft_logits):
-    _check(lib().gm_reconstruct(ctx.handle, C.byref(st.struct()), n_cycles, k, _p(cycle_seq), C.byref(rec.struct()),
-                                _p(seq_tok), seq_tok.shape[1], _p(scratch_pages), _p(draft_logits)), "gm_reconstruct")
+def gm_reconstruct(ctx: Context, st: State, n_cycles: int, k: int, cycle_seq, rec, seq_tok, scratch_pages, draft_logits,
+                   head_states=None):
+    """head_states (fp32 [n_cycles, k, d]) given: gm_reconstruct_states, which also returns g_j of every chain."""
+    if head_states is None:
+        _check(lib().gm_reconstruct(ctx.handle, C.byref(st.struct()), n_cycles, k, _p(cycle_seq), C.byref(rec.struct()),
+                                    _p(seq_tok), seq_tok.shape[1], _p(scratch_pages), _p(draft_logits)), "gm_reconstruct")
+    else:
+        _check(lib().gm_reconstruct_states(ctx.handle, C.byref(st.struct()), n_cycles, k, _p(cycle_seq), C.byref(rec.struct()),
+                                           _p(seq_tok), seq_tok.shape[1], _p(scratch_pages), _p(draft_logits),
+                                           _p(head_states)), "gm_reconstruct_states")
+
+
+def gm_head_state_grad(ctx: Context, rows: int, grad_logits, grad_normed, head_states=None, grad_states=None,
+                       refresh_weights: bool = False):
+    _check(lib().gm_head_state_grad(ctx.handle, rows, _p(grad_logits), _p(head_states), _p(grad_normed), _p(grad_states),
+                                    int(refresh_weights)), "gm_head_state_grad")
 
 
 def gm_overlap(ctx: Context, n_cycles: int, k: int, temperature: float, draft_logits, rec, alpha, lse=None):

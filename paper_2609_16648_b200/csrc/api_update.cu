@@ -1,4 +1,5 @@
-// C ABI of libgm: forward pass of the head update on recorded cycles (Sec. 3.2-3.4, App. D.2-D.3).
+// C ABI of libgm: forward pass of the head update on recorded cycles (Sec. 3.2-3.4, App. D.2-D.3) and the first two
+// steps of its backward pass (Alg. 1: objective -> head logits -> head states).
 // Host code only; the helpers it calls are declared in gm_internal.h.
 #include "gm_internal.h"
 
@@ -13,6 +14,12 @@ int gm_capture_hidden(gm_ctx *c, void *seq_hidden, int stride) {
 
 int gm_reconstruct(gm_ctx *c, gm_state *st, int n_cycles, int k, const int32_t *cycle_seq, const gm_record *rec,
                    const int32_t *seq_tok, int tok_stride, const int32_t *scratch_pages, void *draft_logits) {
+  return gm_reconstruct_states(c, st, n_cycles, k, cycle_seq, rec, seq_tok, tok_stride, scratch_pages, draft_logits, nullptr);
+}
+
+int gm_reconstruct_states(gm_ctx *c, gm_state *st, int n_cycles, int k, const int32_t *cycle_seq, const gm_record *rec,
+                          const int32_t *seq_tok, int tok_stride, const int32_t *scratch_pages, void *draft_logits,
+                          float *head_states) {
   NvtxRange nvtx_range("gm_reconstruct");
   int rc = check_state(c, st, k);
   if (rc) return rc;
@@ -44,8 +51,10 @@ int gm_reconstruct(gm_ctx *c, gm_state *st, int n_cycles, int k, const int32_t *
     gm_state vs = *st;
     vs.batch = m; vs.kv_len = c->v_kv_len; vs.head_page_table = c->v_table; vs.pending_n = c->v_pending_n;
     vs.pending_tok = c->v_pending_tok; vs.pending_hidden = c->v_pending_hidden;
+    c->state_out = head_states ? head_states + static_cast<size_t>(off) * k * c->d : nullptr;
     rc = draft_impl(c, &vs, k, 1.0f, nullptr, 0, 0, rec->drafts + static_cast<size_t>(off) * k,
                     static_cast<__nv_bfloat16 *>(draft_logits) + static_cast<size_t>(off) * k * c->V, nullptr, true);
+    c->state_out = nullptr;
     if (rc) return rc;
   }
   return GM_OK;
@@ -82,6 +91,33 @@ int gm_dca_grad(gm_ctx *c, int n_cycles, int k, float temperature, const void *d
   A.grad = static_cast<__nv_bfloat16 *>(grad_logits); A.V = c->V; A.K = k; A.n = n_cycles;
   A.inv_temp = 1.0f / temperature;
   GM_LAUNCH(c, GM_KC_RECORD, launch_dca_grad(A, c->stream));
+  return GM_OK;
+}
+
+int gm_head_state_grad(gm_ctx *c, int rows, const void *grad_logits, const float *head_states, float *grad_normed,
+                       float *grad_states, int refresh_weights) {
+  if (!c || rows < 1 || !grad_logits || !grad_normed || (grad_states != nullptr) != (head_states != nullptr))
+    return GM_ERR_INVALID_ARG;
+  if ((c->V % 64) != 0 || (c->d % 8) != 0) return GM_ERR_UNSUPPORTED;
+  int rc;
+  const bool simple = (c->cfg.flags & GM_FLAG_SIMPLE_GEMM) != 0;
+  if (!c->lm_head_t) {
+    if ((rc = dev_alloc(c, &c->lm_head_t, static_cast<size_t>(c->d) * c->V, false)) != GM_OK) return rc;
+    std::memset(&c->lm_head_t_map, 0, sizeof(c->lm_head_t_map));
+    if (!simple && make_map(c, &c->lm_head_t_map, c->lm_head_t, c->d, c->V, 128) != GM_OK) return GM_ERR_CUDA;
+    refresh_weights = 1;
+  }
+  if (refresh_weights)
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+              launch_transpose_bf16(static_cast<const __nv_bfloat16 *>(c->w.lm_head), c->V, c->d, c->lm_head_t, c->stream));
+  // dL/dy [rows, d] = grad_logits [rows, V] x W_lm [V, d]: the projection kernel with the vocabulary as its K
+  rc = run_gemm(c, static_cast<const __nv_bfloat16 *>(grad_logits), rows, &c->lm_head_t_map, c->lm_head_t, rows, c->d, c->V,
+                grad_normed, EPI_STORE_F32, static_cast<size_t>(c->d));
+  if (rc) return rc;
+  if (grad_states)
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+              launch_rmsnorm_grad(grad_normed, head_states, static_cast<const __nv_bfloat16 *>(c->w.head_final_norm),
+                                  grad_states, rows, c->d, c->cfg.rms_eps, c->stream));
   return GM_OK;
 }
 

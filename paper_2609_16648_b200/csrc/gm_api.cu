@@ -545,6 +545,9 @@ int gmh::draft_impl(gm_ctx *c, const gm_state *st, int k, float temperature, con
     GM_LAUNCH(c, GM_KC_ELEMENTWISE,
               launch_head_out(c->x, c->qn, ph.B, ph.QT, c->d, static_cast<const __nv_bfloat16 *>(c->w.head_final_norm),
                               cf.rms_eps, c->g, c->gn, c->stream));
+    if (c->state_out)                      // the update's backward pass wants g_j of every chain (row stride k*d)
+      GM_CUDA(c, cudaMemcpy2DAsync(c->state_out + static_cast<size_t>(j - 1) * c->d, sizeof(float) * k * c->d, c->g,
+                                   sizeof(float) * c->d, sizeof(float) * c->d, ph.B, cudaMemcpyDeviceToDevice, c->stream));
     // shared LM head -> row j-1 of every sequence's draft logits (row stride k*V)
     rc = run_gemm(c, c->gn, cf.max_batch, &c->lm_head_map, static_cast<const __nv_bfloat16 *>(c->w.lm_head), ph.B, c->V,
                   c->d, dl + static_cast<size_t>(j - 1) * c->V, EPI_STORE_BF16, static_cast<size_t>(k) * c->V);

@@ -99,6 +99,9 @@ struct gm_ctx {
   __nv_bfloat16 *v_pending_hidden = nullptr;
   __nv_bfloat16 *capture = nullptr;         // gm_capture_hidden: [max_batch, capture_stride, d] or null
   int capture_stride = 0;
+  float *state_out = nullptr;               // set by the reconstruction while it runs: g_j of chain r -> state_out[(r*k + j-1)*d]
+  __nv_bfloat16 *lm_head_t = nullptr;       // [d, V]: the LM head transposed, the weight operand of the gradient GEMM
+  CUtensorMap lm_head_t_map;
   float top_p = 1.f;                    // nucleus of the target distributions (1 = none)
   __nv_bfloat16 *ws_nucleus = nullptr;  // [max_batch (max_k + 1)][V] filtered target rows, allocated by gm_set_top_p
   std::vector<void *> allocs;

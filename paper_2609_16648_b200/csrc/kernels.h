@@ -246,6 +246,11 @@ cudaError_t launch_capture_cycle(const __nv_bfloat16 *src, const int32_t *accept
                                  cudaStream_t stream);
 cudaError_t launch_dca_loss(const float *alpha, const int32_t *accepted, int n, int K, float *loss, float *mean,
                             cudaStream_t stream);
+// Backward through an RMSNorm y = x r w (fp32 rows of d values, bf16 weight): gx = r (w gy) - x r^3 mean(x w gy).
+cudaError_t launch_rmsnorm_grad(const float *gy, const float *x, const __nv_bfloat16 *w, float *gx, int rows, int d, float eps,
+                                cudaStream_t stream);
+// dst [cols, rows] = transpose of src [rows, cols] (bf16, both row-major).
+cudaError_t launch_transpose_bf16(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst, cudaStream_t stream);
 
 // ---- element-wise --------------------------------------------------------------------------------------
 // x[m] = embed[token(m)] (fp32), xn[m] = RMSNorm(x[m]; w) (bf16); rows m = b*QT + j of the verify phase.

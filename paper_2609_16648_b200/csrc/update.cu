@@ -287,6 +287,46 @@ capture_cycle_kernel(const __nv_bfloat16 *src, const int32_t *accept_len, const 
   for (int i = threadIdx.x; i < d / 8; i += blockDim.x) o[i] = s[i];
 }
 
+// ---- backward through the head's final norm (Alg. 1, "update phi"; the norm of App. B.1) -----------------------------------
+// y = x r w with r = (mean(x^2) + eps)^(-1/2):  dL/dx = r (w gy) - x r^3 mean(x w gy).  One CTA per row, fp32.
+constexpr int NG_THREADS = 256;
+__global__ void __launch_bounds__(NG_THREADS)
+rmsnorm_grad_kernel(const float *gy, const float *x, const __nv_bfloat16 *w, float *gx, int d, float eps) {
+  __shared__ float red[2][NG_THREADS / 32];
+  const size_t row = static_cast<size_t>(blockIdx.x) * d;
+  const int tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
+  pdl_prologue();
+  float sq = 0.f, dot = 0.f;
+  for (int i = tid; i < d; i += NG_THREADS) {
+    const float xv = x[row + i];
+    sq = fmaf(xv, xv, sq);
+    dot = fmaf(xv, bf16_to_float(w[i]) * gy[row + i], dot);
+  }
+  sq = warp_sum(sq); dot = warp_sum(dot);
+  if (lane == 0) { red[0][wp] = sq; red[1][wp] = dot; }
+  __syncthreads();
+  sq = 0.f; dot = 0.f;
+#pragma unroll
+  for (int i = 0; i < NG_THREADS / 32; ++i) { sq += red[0][i]; dot += red[1][i]; }   // same order in every thread
+  const float inv_d = 1.0f / static_cast<float>(d);
+  const float r = rsqrtf(sq * inv_d + eps);
+  const float c = r * r * r * dot * inv_d;
+  for (int i = tid; i < d; i += NG_THREADS)
+    gx[row + i] = r * bf16_to_float(w[i]) * gy[row + i] - x[row + i] * c;
+}
+
+// dst[c][r] = src[r][c] for a row-major bf16 matrix [rows, cols]; 64 x 64 tiles through shared memory.
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst) {
+  __shared__ __nv_bfloat16 tile[64][66];
+  const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+  for (int i = ty; i < 64; i += 4)
+    if (r0 + i < rows && c0 + tx < cols) tile[i][tx] = src[static_cast<size_t>(r0 + i) * cols + c0 + tx];
+  __syncthreads();
+  for (int i = ty; i < 64; i += 4)
+    if (c0 + i < cols && r0 + tx < rows) dst[static_cast<size_t>(c0 + i) * rows + r0 + tx] = tile[tx][i];
+}
+
 }  // namespace
 
 cudaError_t launch_capture_chunk(const __nv_bfloat16 *src, const int32_t *row_n, const int32_t *row_base, int rows, int vr,
@@ -318,6 +358,14 @@ cudaError_t launch_dca_grad(const DcaGradArgs &A, cudaStream_t stream) {
 cudaError_t launch_dca_loss(const float *alpha, const int32_t *accepted, int n, int K, float *loss, float *mean,
                             cudaStream_t stream) {
   return launch_k(dca_loss_kernel, dim3(1), dim3(DL_THREADS), 0, stream, 1, alpha, accepted, n, K, loss, mean);
+}
+cudaError_t launch_rmsnorm_grad(const float *gy, const float *x, const __nv_bfloat16 *w, float *gx, int rows, int d, float eps,
+                                cudaStream_t stream) {
+  return launch_k(rmsnorm_grad_kernel, dim3(rows), dim3(NG_THREADS), 0, stream, 1, gy, x, w, gx, d, eps);
+}
+cudaError_t launch_transpose_bf16(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst, cudaStream_t stream) {
+  transpose_bf16_kernel<<<dim3((cols + 63) / 64, (rows + 63) / 64), 256, 0, stream>>>(src, rows, cols, dst);
+  return cudaGetLastError();
 }
 
 }  // namespace gm

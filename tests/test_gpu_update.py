@@ -83,8 +83,12 @@ def test_head_update_forward_matches_the_oracle():
     logits = torch.zeros((n, K, V), dtype=torch.bfloat16, device="cuda")
     shared = torch.as_tensor(hpt[hpt >= 0], device="cuda", dtype=torch.long)
     before = gst.head_kv_pool[:, :, shared].clone()
-    gmb.gm_reconstruct(ctx, gst, n, K, cycle_seq, rec, tok_d, scratch, logits)        # 20 chains, 4 per pass
+    states = torch.full((n, K, d), 7.0, dtype=torch.float32, device="cuda")
+    gmb.gm_reconstruct(ctx, gst, n, K, cycle_seq, rec, tok_d, scratch, logits, head_states=states)   # 20 chains, 4 per pass
     assert gmb.gm_last_status(ctx) == 0
+    logits_plain = torch.zeros_like(logits)
+    gmb.gm_reconstruct(ctx, gst, n, K, cycle_seq, rec, tok_d, scratch, logits_plain)    # the call without the states: same logits
+    assert torch.equal(logits_plain, logits)
     assert torch.equal(gst.head_kv_pool[:, :, shared], before)                         # chains wrote to their own pages only
 
     lg = logits.float().cpu().numpy()
@@ -128,6 +132,37 @@ def test_head_update_forward_matches_the_oracle():
     grad2 = torch.full_like(grad, 7.0)
     gmb.gm_dca_grad(ctx, n, K, T, logits, rec, alpha, rec.accepted, grad2, lse)
     assert torch.equal(grad2, grad)
+
+    # second step: through the shared LM head and the head's final norm, back to the head states
+    st_np = states.cpu().numpy().astype(np.float64)
+    # the states the reconstruction returned are the ones its logits came from (up to the bf16 normed state and logits)
+    relg = rel_err(omodel.head_logits(w, st_np.reshape(n * K, d), cfg).reshape(n, K, V), lg)
+    assert relg < TOL, relg
+    gy = torch.full((n * K, d), 7.0, dtype=torch.float32, device="cuda")
+    gs = torch.full((n * K, d), 7.0, dtype=torch.float32, device="cuda")
+    gmb.gm_head_state_grad(ctx, n * K, grad, gy, states, gs)
+    assert gmb.gm_last_status(ctx) == 0
+    g_in = grad.float().cpu().numpy().astype(np.float64)                      # the device's own bf16 gradient rows
+    want_gy = oupdate.lm_head_input_grad(g_in, omodel.round_bf16(w["lm_head"])).reshape(n * K, d)
+    want_gs = oupdate.rmsnorm_grad(want_gy, st_np.reshape(n * K, d), omodel.round_bf16(w["head"]["final_norm"]), cfg.rms_eps)
+    assert np.abs(want_gy).max() > 0
+    assert rel_err(gy.cpu().numpy(), want_gy) < 2e-4                          # bf16 products, fp32 sums over 4096 terms
+    assert rel_err(gs.cpu().numpy(), want_gs) < 2e-4
+    live = np.array([[j < min(r["accepted"], K) for j in range(K)] for _, r in cycles]).reshape(-1)
+    assert (gs.cpu().numpy()[~live] == 0).all() and (np.abs(gs.cpu().numpy()[live]).max(-1) > 0).all()
+    # end to end against the oracle's own chain (its logits, its states): the direction of the update agrees
+    ref_states = np.stack([oupdate.reconstruct_states(w, cfg, seqs[b][0], seqs[b][1], r["start_pos"], r["drafts"])
+                           for b, r in cycles])
+    assert rel_err(st_np, ref_states) < TOL
+    ref_gs, _, _ = oupdate.head_update_grad_state(w, cfg, ref_states, [r for _, r in cycles], T)
+    cos = (ref_gs.reshape(-1) * gs.cpu().numpy().reshape(-1)).sum() / (np.linalg.norm(ref_gs) * np.linalg.norm(gs.cpu().numpy()))
+    assert cos > 0.98, cos
+    # the projection alone, and a refreshed weight copy: the same numbers
+    gy2 = torch.zeros_like(gy)
+    gmb.gm_head_state_grad(ctx, n * K, grad, gy2, refresh_weights=True)
+    assert torch.equal(gy2, gy)
+    with pytest.raises(gmb.GmError):
+        gmb.gm_head_state_grad(ctx, n * K, grad, gy, states, None)
     ctx.close()
 
 
@@ -207,6 +242,49 @@ def test_gradient_kernel_full_vocabulary_and_edge_cases():
     gmb.gm_dca_grad(ctx, n, K, Tg, logits, rec, alpha, rec.accepted, grad)
     g2 = grad.float().cpu().numpy()
     assert (g2[2] == 0).all() and np.array_equal(g2[[0, 1, 3, 4, 5, 6, 7]], got[[0, 1, 3, 4, 5, 6, 7]])
+    ctx.close()
+
+
+@pytest.mark.parametrize("rows", [192, 448], ids=["64x3", "two_token_blocks_ragged"])
+def test_head_state_gradient_at_the_4b_dimensions(rows):
+    """gm_head_state_grad alone at d = 2560, V = 151936: the projection contracts over 2374 K blocks (split along K over
+    clusters at 192 rows; two token blocks, the second ragged, at 448).  Synthetic gradient rows with the structure
+    gm_dca_grad writes: dense small values, a third of the rows exactly zero.  The oracle computes sampled rows."""
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny").with_(vocab=151936, d_model=2560)
+    V, d = cfg.vocab, cfg.d_model
+    ctx = gmb.Context(cfg, gmb.random_packed_weights(cfg, "cuda"), 4, 3, 4, 8, 8)
+    g = torch.Generator(device="cuda").manual_seed(9)
+    ctx.packed["head"]["final_norm"].copy_((1 + (torch.rand(d, device="cuda", generator=g) - 0.5) * 0.5).to(torch.bfloat16))
+    grad = (torch.randn((rows, V), device="cuda", generator=g) * 1e-3).to(torch.bfloat16)
+    grad[2::3] = 0
+    states = torch.randn((rows, d), device="cuda", generator=g) * 3.0
+    gy = torch.full((rows, d), 7.0, dtype=torch.float32, device="cuda")
+    gs = torch.full((rows, d), 7.0, dtype=torch.float32, device="cuda")
+    gmb.gm_head_state_grad(ctx, rows, grad, gy, states, gs)
+    assert gmb.gm_last_status(ctx) == 0
+    sample = sorted(set(np.random.default_rng(3).choice(rows, 24, replace=False).tolist()) | {0, 2, 255 % rows, rows - 1})
+    w_lm = ctx.packed["lm_head"].double().cpu().numpy()
+    want_gy = oupdate.lm_head_input_grad(grad[sample].double().cpu().numpy(), w_lm)
+    want_gs = oupdate.rmsnorm_grad(want_gy, states[sample].double().cpu().numpy(),
+                                   ctx.packed["head"]["final_norm"].double().cpu().numpy(), cfg.rms_eps)
+    got_gy, got_gs = gy[sample].cpu().numpy(), gs[sample].cpu().numpy()
+    assert rel_err(got_gy, want_gy) < 2e-4 and rel_err(got_gs, want_gs) < 2e-4     # fp32 sums over 151936 exact bf16 products
+    zero = [i for i, r in enumerate(sample) if r % 3 == 2]
+    assert zero and (got_gy[zero] == 0).all() and (got_gs[zero] == 0).all()
+    assert not torch.isnan(gs).any() and float(gs[0::3].abs().max()) > 0
+    # timing of the two launches (weights already transposed)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    for _ in range(3):
+        gmb.gm_head_state_grad(ctx, rows, grad, gy, states, gs)
+    ev[0].record()
+    for _ in range(10):
+        gmb.gm_head_state_grad(ctx, rows, grad, gy, states, gs)
+    ev[1].record()
+    torch.cuda.synchronize()
+    ms = ev[0].elapsed_time(ev[1]) / 10
+    print(f"gm_head_state_grad rows {rows}: {ms:.3f} ms per call, {(d * V * 2 + rows * V * 2) / ms / 1e6:.0f} GB/s of the "
+          f"operands, {2.0 * rows * d * V / ms / 1e9:.0f} TFLOP/s")
     ctx.close()
 
 
