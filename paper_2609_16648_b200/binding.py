@@ -19,7 +19,7 @@ GM_ERR_INVALID_ARG, GM_ERR_UNSUPPORTED, GM_ERR_KV_CAPACITY, GM_ERR_CUDA = -1, -2
 GM_ERR_DEVICE_TIMEOUT, GM_ERR_BAD_PAGE, GM_ERR_NO_EXTENSION, GM_ERR_SCRATCH_LIMIT, GM_ERR_OVERRUN = -5, -6, -7, -8, -9
 GM_NOALLOC_SCRATCH_BYTES, GM_NOALLOC_MAX_BATCH = 16 << 20, 256
 GM_MAX_K, GM_PAGE = 7, 16
-GM_FLAG_SIMPLE_GEMM, GM_FLAG_SAMPLER_CLUSTER, GM_FLAG_SAMPLER_STREAM, GM_FLAG_GRAPH = 1, 2, 4, 8
+GM_FLAG_SIMPLE_GEMM, GM_FLAG_SAMPLER_CLUSTER, GM_FLAG_SAMPLER_STREAM, GM_FLAG_GRAPH, GM_FLAG_SAMPLER_FLOW = 1, 2, 4, 8, 16
 GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER, GM_KC_RECORD = 0, 1, 2, 3, 4
 
 EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw", "gm_set_top_p", "gm_nucleus", "gm_prefill",

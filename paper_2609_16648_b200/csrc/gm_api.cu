@@ -294,10 +294,23 @@ int check_state(const gm_ctx *c, const gm_state *st, int k) {
 // Mapping of the sampler: a cluster per sequence while sequences are few, one CTA per sequence once there are enough
 // of them to fill the SMs (the flags force one or the other).
 cudaError_t run_sampler(gm_ctx *c, const SamplerArgs &S, int batch) {
-  bool stream_variant = batch * 3 >= c->sm_count * 2;
-  if (c->cfg.flags & GM_FLAG_SAMPLER_CLUSTER) stream_variant = false;
-  if (c->cfg.flags & GM_FLAG_SAMPLER_STREAM) stream_variant = true;
-  if (stream_variant && sampler_stream_supported(S.V)) return launch_sampler_stream(S, batch, c->stream);
+  int mode = c->sampler_mode;
+  if (c->cfg.flags & GM_FLAG_SAMPLER_CLUSTER) mode = 1;
+  if (c->cfg.flags & GM_FLAG_SAMPLER_STREAM) mode = 2;
+  if (c->cfg.flags & GM_FLAG_SAMPLER_FLOW) mode = 3;
+  if (mode == 0) mode = batch * 3 >= c->sm_count * 2 ? 2 : 1;
+  if (mode == 3 && sampler_flow_supported(S.V, batch, S.K, c->sm_count)) {
+    if (batch > c->flow_cap) {                         // a batch above max_batch (stand-alone gm_accept): grow, outside any capture
+      const size_t need = sampler_flow_ws_bytes(batch, S.V, c->sm_count);
+      void *q = nullptr;
+      if (cudaError_t e = cudaMalloc(&q, need); e != cudaSuccess) return e;
+      c->allocs.push_back(q);
+      if (cudaError_t e = cudaMemsetAsync(q, 0, need, c->stream); e != cudaSuccess) return e;
+      c->flow_ws = q; c->flow_ws_bytes = need; c->flow_cap = batch;
+    }
+    return launch_sampler_flow(S, batch, c->flow_ws, c->flow_cap, c->sm_count, c->stream);
+  }
+  if (mode == 2 && sampler_stream_supported(S.V)) return launch_sampler_stream(S, batch, c->stream);
   return launch_sampler(S, batch, c->stream);
 }
 
@@ -447,6 +460,16 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
   A_(dev_alloc(c, &c->pf_hidden, M * c->d));
   A_(dev_alloc(c, &c->pf_xlast, B1 * c->d));
   A_(dev_alloc(c, &c->status, 1));
+  if (sampler_flow_supported(c->V, static_cast<int>(B), cfg->max_k, c->sm_count)) {
+    unsigned char *ws = nullptr;
+    c->flow_ws_bytes = sampler_flow_ws_bytes(static_cast<int>(B), c->V, c->sm_count);
+    c->flow_cap = static_cast<int>(B);
+    A_(dev_alloc(c, &ws, c->flow_ws_bytes));
+    c->flow_ws = ws;
+  }
+  if (const char *ov = std::getenv("GM_SAMPLER")) {     // tuning aid: cluster | stream | flow for every sampler launch
+    c->sampler_mode = !std::strcmp(ov, "cluster") ? 1 : !std::strcmp(ov, "stream") ? 2 : !std::strcmp(ov, "flow") ? 3 : 0;
+  }
   // persistent chain of a layer's projections: every CTA pair must be resident at once
   if (!(cfg->flags & GM_FLAG_SIMPLE_GEMM) && (c->q_dim % 64) == 0) {
     int pairs = 0;
@@ -748,6 +771,7 @@ int gm_last_status(gm_ctx *c) {
   GM_CUDA(c, cudaMemcpy(&s, c->status, sizeof(s), cudaMemcpyDeviceToHost));
   GM_CUDA(c, cudaMemset(c->status, 0, sizeof(s)));
   if (s & ST_TIMEOUT) {                 // a chain launch that gave up may have left its barrier words mid-count
+    if (c->flow_ws) GM_CUDA(c, cudaMemset(c->flow_ws, 0, c->flow_ws_bytes));      // likewise the sampler's work queue
     if (c->chain_sync) GM_CUDA(c, cudaMemset(c->chain_sync, 0, (1 + static_cast<size_t>(c->chain_pairs) * 2) * sizeof(unsigned long long)));
     return GM_ERR_DEVICE_TIMEOUT;
   }

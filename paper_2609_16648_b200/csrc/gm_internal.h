@@ -99,6 +99,10 @@ struct gm_ctx {
   __nv_bfloat16 *v_pending_hidden = nullptr;
   __nv_bfloat16 *capture = nullptr;         // gm_capture_hidden: [max_batch, capture_stride, d] or null
   int capture_stride = 0;
+  void *flow_ws = nullptr;                  // work-queue sampler: counters, per-sequence state, slice partials, queue slots
+  size_t flow_ws_bytes = 0;
+  int flow_cap = 0;                         // batch the workspace was sized for
+  int sampler_mode = 0;                     // 0 = by batch size; 1 cluster, 2 stream, 3 work queue (GM_SAMPLER in the environment)
   float *state_out = nullptr;               // set by the reconstruction while it runs: g_j of chain r -> state_out[(r*k + j-1)*d]
   __nv_bfloat16 *lm_head_t = nullptr;       // [d, V]: the LM head transposed, the weight operand of the gradient GEMM
   CUtensorMap lm_head_t_map;

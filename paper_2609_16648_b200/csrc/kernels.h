@@ -91,6 +91,11 @@ struct SamplerArgs {
 cudaError_t launch_sampler(const SamplerArgs &A, int batch, cudaStream_t stream);          // cluster of 8 CTAs per sequence
 cudaError_t launch_sampler_stream(const SamplerArgs &A, int batch, cudaStream_t stream);   // one CTA per sequence
 bool sampler_stream_supported(int V);
+// Vocabulary-sliced mapping: every CTA (one per SM) owns the same slice of every row of every sequence; `ws` is device memory
+// of sampler_flow_ws_bytes(...) bytes, zeroed once before its first use (the kernel leaves it ready for the next launch).
+bool sampler_flow_supported(int V, int batch, int K, int sm_count);
+size_t sampler_flow_ws_bytes(int cap_batch, int V, int sm_count);
+cudaError_t launch_sampler_flow(const SamplerArgs &A, int batch, void *ws, int cap_batch, int sm_count, cudaStream_t stream);
 
 // ---- cycle record (top-64 target log-probabilities and the other recorded items) ---------------------------------
 struct RecordTopkArgs {

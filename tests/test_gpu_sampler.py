@@ -13,9 +13,9 @@ pytestmark = pytest.mark.gpu
 MAPPING = {"flags": 0}
 
 
-@pytest.fixture(autouse=True, params=[2, 4], ids=["cluster_per_sequence", "cta_per_sequence"])
+@pytest.fixture(autouse=True, params=[2, 4, 16], ids=["cluster_per_sequence", "cta_per_sequence", "work_queue"])
 def _mapping(request):
-    """Every test of this file runs with both mappings of the sampler kernel."""
+    """Every test of this file runs with all three mappings of the sampler kernel."""
     MAPPING["flags"] = request.param
     yield
 
