@@ -61,7 +61,7 @@ extern "C" {
 #define GM_FLAG_SIMPLE_GEMM 1       /* debug: route every GEMM through the plain mma.sync kernel */
 #define GM_FLAG_SAMPLER_CLUSTER 2   /* always map the sampler as one 8-CTA cluster per sequence  */
 #define GM_FLAG_SAMPLER_STREAM 4    /* always map the sampler as one CTA per sequence            */
-#define GM_FLAG_SAMPLER_FLOW 16     /* always map the sampler as slice-sized items on a device work queue */
+#define GM_FLAG_SAMPLER_FLOW 16     /* always map the sampler as one vocabulary slice of every row per CTA */
 #define GM_FLAG_GRAPH 8             /* gm_spec_step, gm_spec_step_host and gm_rollout_run replay a
                                        captured CUDA graph of one cycle (needs a context created on a
                                        stream of its own: on a default stream the flag has no effect) */

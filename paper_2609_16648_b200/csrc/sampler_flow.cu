@@ -164,15 +164,6 @@ __device__ __forceinline__ MZ sf_merge_slices(F ld, int NA, int lane, float s) {
   return MZ{-st.m * s, __frcp_rn(st.z)};
 }
 
-#ifdef SF_TRACE
-__device__ unsigned long long sf_trace[148 * 32];
-__device__ __forceinline__ unsigned long long sf_now() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory"); return t; }
-#define SF_T(slot, val) do { if (lane == 0) sf_trace[blockIdx.x * 32 + (slot)] = (val); } while (0)
-#define SF_TADD(var, expr) do { const unsigned long long _t0 = sf_now(); expr; var += sf_now() - _t0; } while (0)
-#else
-#define SF_T(slot, val) do {} while (0)
-#define SF_TADD(var, expr) do { expr; } while (0)
-#endif
 constexpr int SF_MAX_B = 2048;
 constexpr int SF_ROUNDS = GM_MAX_K_ + 4;              // stride of the per-sequence stage arrays (STAT x (K+1), RES, RES again, SEARCH)
 
@@ -266,10 +257,6 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
   if (warp == SF_PRODUCER) {
     uint32_t n = 0;                                   // ring items posted so far (same value in every lane)
     bool alive = true;
-#ifdef SF_TRACE
-    unsigned long long t_poll = 0, t_post = 0;
-    SF_T(0, sf_now());
-#endif
     // every lane that holds an item takes the next free ring slots in lane order and starts its own copies
     auto post = [&](bool has, uint32_t desc, const uint4 *prow, const uint4 *qrow) {
       const uint32_t m = __ballot_sync(0xffffffffu, has);
@@ -294,7 +281,6 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
     };
     for (int r = 0; r < rounds && alive; ++r) {
       bool any = false;
-      SF_T(1 + r, sf_now());
       for (int blk = 0; blk < nblk && alive; ++blk) {
         const int b = blk * 32 + lane;
         bool act = b < B && !((sh.done_mask[blk] >> lane) & 1u);
@@ -313,9 +299,6 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
           const unsigned long long *wp = W.stage + static_cast<size_t>(b < B ? b : 0) * SF_ROUNDS + r;
           unsigned long long w = 0;
           bool ready = !act;
-#ifdef SF_TRACE
-          const unsigned long long tp0 = sf_now();
-#endif
           for (uint32_t i = 0; i < SF_SPIN_LIMIT; ++i) {
             if (!ready) {
               w = ld_acquire_u64(wp);
@@ -325,9 +308,6 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
             if (sh.dead) break;
             __nanosleep(64);
           }
-#ifdef SF_TRACE
-          t_poll += sf_now() - tp0;
-#endif
           if (!__all_sync(0xffffffffu, ready)) {
             if (lane == 0 && !sh.dead) { sh.dead = 1; set_status(A.status, ST_TIMEOUT); }
             alive = false;
@@ -341,9 +321,6 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
         const int prow_r = k, qrow_r = K + 1 + k;     // STAT k and RES at position a = k read the rows (p_k, q_k)
         const bool has_q = type == SF_STAT ? k < K : use_q != 0;
         // the slice every CTA holds
-#ifdef SF_TRACE
-        const unsigned long long tq0 = sf_now();
-#endif
         post(bulk && vps > 0, sf_desc(type, use_q, k, 0, r, b), bulk ? sf_row(A, b, prow_r) : nullptr,
              bulk && has_q ? sf_row(A, b, qrow_r) : nullptr);
         // what only one CTA does: the vectors after the last slice, the token search, the fallback
@@ -354,15 +331,9 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
              nullptr, nullptr);
         if (fin) atomicOr(&sh.done_mask[blk], 1u << lane);
         __syncwarp();
-#ifdef SF_TRACE
-        t_post += sf_now() - tq0;
-#endif
       }
       if (!any) break;                                // every walk has ended
     }
-#ifdef SF_TRACE
-    SF_T(12, t_poll); SF_T(13, t_post); SF_T(14, sf_now()); SF_T(15, n);
-#endif
     // one quit marker per compute warp
     post(lane < SF_CWARPS && !sh.dead, static_cast<uint32_t>(SF_QUIT), nullptr, nullptr);
     if (lane == 0) {                                  // the last CTA to leave opens the next epoch
@@ -400,9 +371,6 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
     };
     prefetch_decision();
     uint32_t spins = 0;
-#ifdef SF_TRACE
-    unsigned long long t_merge = 0, n_merge = 0;
-#endif
     while (__any_sync(0xffffffffu, active)) {
       bool ready = false;
       if (active) ready = ld_acquire_u32(&W.cnt[static_cast<size_t>(my_b) * SF_ROUNDS + r]) == static_cast<uint32_t>(NA);
@@ -417,9 +385,6 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
       }
       spins = 0;
       while (m != 0u) {
-#ifdef SF_TRACE
-        const unsigned long long tm0 = sf_now();
-#endif
         const int src = __ffs(m) - 1;
         m &= m - 1u;
         const int b = __shfl_sync(0xffffffffu, my_b, src), rr = __shfl_sync(0xffffffffu, r, src);
@@ -560,31 +525,15 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
           if (n_type == SF_SEARCH || n_type == SF_ARGMAX || r >= rounds) active = false;
           prefetch_decision();
         }
-#ifdef SF_TRACE
-        t_merge += sf_now() - tm0; ++n_merge;
-        SF_T(20, n_merge); SF_T(21, t_merge); SF_T(22, sf_now());
-#endif
       }
     }
     return;
   }
 
   // ==================================================== compute warps ====================================================
-#ifdef SF_TRACE
-  unsigned long long t_full = 0, t_work = 0, tw0 = 0;
-#endif
   for (uint32_t n = warp;; n += SF_CWARPS) {
     const int slot = n % R;
-#ifdef SF_TRACE
-    const unsigned long long tf0 = sf_now();
-    if (n >= SF_CWARPS) t_work += tf0 - tw0;
-#endif
     if (!wait_bar(&sh.full[slot], (n / R) & 1u)) return;
-#ifdef SF_TRACE
-    tw0 = sf_now();
-    t_full += tw0 - tf0;
-    if (warp == 0) { SF_T(16, t_full); SF_T(17, n); SF_T(18, tw0); SF_T(19, t_work); }
-#endif
     const uint32_t desc = sh.desc[slot];
     const int type = desc & 7u, use_q = (desc >> 3) & 1u, k = (desc >> 4) & 15u, is_tail = (desc >> 8) & 1u, r = (desc >> 9) & 15u;
     const int b = desc >> 16;
@@ -801,11 +750,5 @@ cudaError_t launch_sampler_flow(const SamplerArgs &A, int batch, void *ws, int c
   return launch_k(sampler_flow_kernel, dim3(g.G), dim3(SF_THREADS), dyn, stream, 1, A, W, batch);
 }
 
-#ifdef SF_TRACE
-cudaError_t sampler_flow_trace_read(unsigned long long *out) { return cudaMemcpyFromSymbol(out, sf_trace, sizeof(unsigned long long) * 148 * 32); }
-#endif
 
 }  // namespace gm
-#ifdef SF_TRACE
-extern "C" int gm_debug_sf_trace(unsigned long long *out) { return static_cast<int>(gm::sampler_flow_trace_read(out)); }
-#endif

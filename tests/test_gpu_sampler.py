@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 MAPPING = {"flags": 0}
 
 
-@pytest.fixture(autouse=True, params=[2, 4, 16], ids=["cluster_per_sequence", "cta_per_sequence", "work_queue"])
+@pytest.fixture(autouse=True, params=[2, 4, 16], ids=["cluster_per_sequence", "cta_per_sequence", "slice_per_cta"])
 def _mapping(request):
     """Every test of this file runs with all three mappings of the sampler kernel."""
     MAPPING["flags"] = request.param
