@@ -2,26 +2,25 @@
 // positions the target's top-64 log-probabilities (bf16, full-vocabulary normalisation) with their token ids,
 // plus the cycle's start hidden state, start position, drafts and accepted length.
 //
-// top-64 of a 150k-entry bf16 row.  One cluster of 8 CTAs per row, each CTA one eighth of the vocabulary, copied
-// once into shared memory (bulk asynchronous copy).  Every global top-64 entry is in its CTA's local top-64, so a
-// CTA selects its local 64 exactly with two 256-bin histogram passes over the 16-bit order-preserving key of the
-// bf16 logit (high byte, then low byte inside the boundary bin), collects the entries above the cut in any order
-// and the ties at the cut in token order (block-wide scan), and the cluster's first CTA merges the 8 x 64
-// candidates with a bitonic sort on (key descending, token id ascending).  Log-probabilities use the row's
-// (max, sum exp) reduced over the cluster in fixed order.
-#include <cooperative_groups.h>
-
+// top-64 of a 150k-entry bf16 row: one CTA per row, the row streamed from global memory twice (it is L2-resident: the
+// LM head has just written it, the sampler has just read it).  The selection works on the 16-bit order-preserving key
+// of the bf16 logit.  Pass 1: (max, sum exp) with a running maximum, and every thread's own largest key; the 64th
+// largest of the 512 thread maxima is a lower bound L of the row's 64th largest entry (they are 64 different entries).
+// Pass 2 keeps aside every entry with key >= L - typically 70 to 100 of 150k, so the shared-memory atomics are rare -
+// and the 64 places are the entries' ranks by (key descending, token id ascending) inside that list.  Rows with more
+// than 1024 entries at or above L (long runs of equal values) take the general path instead: 256-bin histograms of the
+// key (high byte, then low byte inside the boundary bin) fix the cut, a third pass collects the entries above it in
+// any order and the ties at the cut in token order (block-wide scan, early exit), a bitonic sort orders the 64.
 #include "common.cuh"
 #include "kernels.h"
-
-namespace cg = cooperative_groups;
 
 namespace gm {
 
 constexpr int REC_THREADS = 512;
 constexpr int REC_WARPS = REC_THREADS / 32;
-constexpr int REC_CLUSTER = 8;
 constexpr int REC_TOP = 64;
+constexpr int REC_UNROLL = 8;                         // row vectors a thread has in flight in the streaming passes
+constexpr int REC_LIST = 1024;                        // entries kept aside in pass 2 (more than that: the general path)
 
 __device__ __forceinline__ float rec_ex2(float x) {
   float y;
@@ -41,226 +40,263 @@ __device__ __forceinline__ void rec_keys8(const uint4 &v, uint32_t (&k)[8]) {
   k[0] = rec_key(v.x & 0xFFFFu); k[1] = rec_key(v.x >> 16); k[2] = rec_key(v.y & 0xFFFFu); k[3] = rec_key(v.y >> 16);
   k[4] = rec_key(v.z & 0xFFFFu); k[5] = rec_key(v.z >> 16); k[6] = rec_key(v.w & 0xFFFFu); k[7] = rec_key(v.w >> 16);
 }
+__device__ __forceinline__ uint4 rec_ldg(const uint4 *p) {
+  uint4 v;
+  asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint32_t rec_bmax2(uint32_t a, uint32_t b) {      // packed bf16x2 maximum
+  __nv_bfloat162 r = __hmax2(*reinterpret_cast<__nv_bfloat162 *>(&a), *reinterpret_cast<__nv_bfloat162 *>(&b));
+  return *reinterpret_cast<uint32_t *>(&r);
+}
+
+__device__ __forceinline__ uint32_t rec_ge2(uint32_t a, uint32_t b) {       // per half: 0xFFFF where a >= b
+  return __hge2_mask(*reinterpret_cast<__nv_bfloat162 *>(&a), *reinterpret_cast<__nv_bfloat162 *>(&b));
+}
 
 struct RecMZ { float m, z; };
 
-__global__ void __cluster_dims__(REC_CLUSTER, 1, 1) __launch_bounds__(REC_THREADS)
-record_topk_kernel(const RecordTopkArgs A) {
-  cg::cluster_group cluster = cg::this_cluster();
-  const int rank = static_cast<int>(cluster.block_rank());
-  const int row_id = blockIdx.x / REC_CLUSTER, b = row_id / A.K, k = row_id % A.K;
+__global__ void __launch_bounds__(REC_THREADS, 2) record_topk_kernel(const RecordTopkArgs A) {
+  const int b = blockIdx.x / A.K, k = blockIdx.x % A.K;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int V = A.V;
+  const int V = A.V, nvec = V >> 3;
   const float s = A.inv_temp * 1.4426950408889634f;
 
-  const int nvec_total = V >> 3;
-  const int vpc = (nvec_total + REC_CLUSTER - 1) / REC_CLUSTER;
-  const int v_lo = min(rank * vpc, nvec_total);
-  const int n = min(v_lo + vpc, nvec_total) - v_lo;
-
-  extern __shared__ __align__(128) unsigned char rec_smem[];
-  const uint4 *buf = reinterpret_cast<const uint4 *>(rec_smem);                           // [vpc] the row slice
   __shared__ uint32_t hist[REC_WARPS][256];
   __shared__ uint32_t hsum[256];
-  __shared__ unsigned long long cand[REC_TOP];            // this CTA's candidates (read by the first CTA)
-  __shared__ unsigned long long merge[REC_CLUSTER * REC_TOP];
+  __shared__ unsigned long long cand[REC_TOP];
   __shared__ RecMZ warp_mz[REC_WARPS];
-  __shared__ RecMZ local_mz;                              // read by the first CTA
-  __shared__ uint64_t full_bar;
-  __shared__ int sh_cut, sh_above, sh_take, sh_cnt, sh_alive;
+  __shared__ int sh_cut, sh_above, sh_cnt, sh_nlist;
+  __shared__ unsigned long long wlist[REC_LIST];          // pass 2: every entry at or above the lower bound
   __shared__ int warp_tot[REC_WARPS];
+  __shared__ uint32_t tkeys[REC_THREADS];
+  __shared__ uint32_t sh_low;
 
   pdl_prologue();
-  if (tid == 0) {
-    mbar_init(&full_bar, 1);
-    mbar_fence_init();
-    sh_alive = 1;
-    sh_cnt = 0;
-  }
+  const uint4 *row = reinterpret_cast<const uint4 *>(A.target_logits + static_cast<size_t>(b) * A.bstride + static_cast<size_t>(k) * V);
   if (tid < REC_TOP) cand[tid] = 0ull;
-  __syncthreads();
-  const uint4 *src = reinterpret_cast<const uint4 *>(A.target_logits + static_cast<size_t>(b) * A.bstride +
-                                                      static_cast<size_t>(k) * V) + v_lo;
-  if (tid == 0 && n > 0) {
-    mbar_expect_tx(&full_bar, static_cast<uint32_t>(n) * 16u);
-    bulk_load(const_cast<uint4 *>(buf), src, static_cast<uint32_t>(n) * 16u, &full_bar);
-    if (!mbar_wait(&full_bar, 0)) { sh_alive = 0; set_status(A.status, ST_TIMEOUT); }
-  }
-  __syncthreads();
-  const bool alive = sh_alive != 0;
-  const int n_use = alive ? n : 0;
+  if (tid == 0) { sh_cnt = 0; sh_nlist = 0; }
 
-  // ---- (max, sum 2^((x - max) s)) of the slice ----------------------------------------------------------------------
+  // ---- pass 1: (max, sum 2^((x - max) s)) with a running maximum; the largest key ---------------------------------------
+  RecMZ st{-INFINITY, 0.f};
+  uint32_t tm2 = 0xff80ff80u;                          // packed maximum of this thread's entries
+  for (int i0 = tid; i0 < nvec; i0 += REC_UNROLL * REC_THREADS) {
+    uint4 v[REC_UNROLL];
+    uint32_t m2 = 0xff80ff80u;
+#pragma unroll
+    for (int t = 0; t < REC_UNROLL; ++t) {
+      const int i = i0 + t * REC_THREADS;
+      v[t] = i < nvec ? rec_ldg(row + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+      m2 = rec_bmax2(rec_bmax2(m2, rec_bmax2(v[t].x, v[t].y)), rec_bmax2(v[t].z, v[t].w));
+    }
+    tm2 = rec_bmax2(tm2, m2);
+    const float mx = fmaxf(bf16_lo(m2), bf16_hi(m2));
+    if (mx > st.m) { st.z *= rec_ex2((st.m - mx) * s); st.m = mx; }           // 0 * 2^-inf = 0 on the first block
+    if (st.m != -INFINITY) {
+      const float c = -st.m * s;
+      float acc = 0.f;
+#pragma unroll
+      for (int t = 0; t < REC_UNROLL; ++t)
+        acc += rec_ex2(fmaf(bf16_lo(v[t].x), s, c)) + rec_ex2(fmaf(bf16_hi(v[t].x), s, c)) + rec_ex2(fmaf(bf16_lo(v[t].y), s, c)) +
+               rec_ex2(fmaf(bf16_hi(v[t].y), s, c)) + rec_ex2(fmaf(bf16_lo(v[t].z), s, c)) + rec_ex2(fmaf(bf16_hi(v[t].z), s, c)) +
+               rec_ex2(fmaf(bf16_lo(v[t].w), s, c)) + rec_ex2(fmaf(bf16_hi(v[t].w), s, c));
+      st.z += acc;
+    }
+  }
   {
-    float mx = -INFINITY;
-    for (int i = tid; i < n_use; i += REC_THREADS) {
-      const uint4 v = buf[i];
-      mx = fmaxf(mx, fmaxf(fmaxf(fmaxf(bf16_lo(v.x), bf16_hi(v.x)), fmaxf(bf16_lo(v.y), bf16_hi(v.y))),
-                           fmaxf(fmaxf(bf16_lo(v.z), bf16_hi(v.z)), fmaxf(bf16_lo(v.w), bf16_hi(v.w)))));
-    }
-    mx = warp_max(mx);
-    if (lane == 0) warp_mz[warp].m = mx;
-    __syncthreads();
-    float m = -INFINITY;
-    for (int w = 0; w < REC_WARPS; ++w) m = fmaxf(m, warp_mz[w].m);
-    const float c = -m * s;
-    float z = 0.f;
-    for (int i = tid; i < n_use; i += REC_THREADS) {
-      const uint4 v = buf[i];
-      z += rec_ex2(fmaf(bf16_lo(v.x), s, c)) + rec_ex2(fmaf(bf16_hi(v.x), s, c)) + rec_ex2(fmaf(bf16_lo(v.y), s, c)) +
-           rec_ex2(fmaf(bf16_hi(v.y), s, c)) + rec_ex2(fmaf(bf16_lo(v.z), s, c)) + rec_ex2(fmaf(bf16_hi(v.z), s, c)) +
-           rec_ex2(fmaf(bf16_lo(v.w), s, c)) + rec_ex2(fmaf(bf16_hi(v.w), s, c));
-    }
+    const float wm = warp_max(st.m);
+    float z = (wm == -INFINITY || st.m == -INFINITY) ? 0.f : st.z * rec_ex2((st.m - wm) * s);
     z = warp_sum(z);
-    if (lane == 0) warp_mz[warp].z = z;
-    __syncthreads();
-    if (tid == 0) {
-      float zt = 0.f;
-      for (int w = 0; w < REC_WARPS; ++w) zt += warp_mz[w].z;
-      local_mz = RecMZ{m, n_use > 0 ? zt : 0.f};
-    }
+    if (lane == 0) warp_mz[warp] = RecMZ{wm, z};
+    // a thread without entries counts as the lowest key
+    tkeys[tid] = tid < nvec ? rec_key(__float_as_uint(fmaxf(bf16_lo(tm2), bf16_hi(tm2))) >> 16) : 0u;
   }
+  __syncthreads();
+  RecMZ rowst{-INFINITY, 0.f};
+  for (int w = 0; w < REC_WARPS; ++w) rowst.m = fmaxf(rowst.m, warp_mz[w].m);
+  for (int w = 0; w < REC_WARPS; ++w)
+    if (warp_mz[w].z > 0.f) rowst.z += warp_mz[w].z * rec_ex2((warp_mz[w].m - rowst.m) * s);   // same order in every thread
+  const uint32_t kmax = rec_key(__float_as_uint(rowst.m) >> 16);
 
-  // ---- local top-64: two histogram levels on the 16-bit key ---------------------------------------------------------
-  const int want = min(REC_TOP, n_use * 8);
-  int hi_bin = -1;                                           // level 1 boundary bin; level 2 runs inside it
-  for (int level = 0; level < 2; ++level) {
-    for (int i = tid; i < REC_WARPS * 256; i += REC_THREADS) (&hist[0][0])[i] = 0u;
-    __syncthreads();
-    for (int i = tid; i < n_use; i += REC_THREADS) {
-      uint32_t key[8];
-      rec_keys8(buf[i], key);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        if (level == 0) atomicAdd(&hist[warp][key[j] >> 8], 1u);
-        else if (static_cast<int>(key[j] >> 8) == hi_bin) atomicAdd(&hist[warp][key[j] & 0xFFu], 1u);
-      }
+  // ---- lower bound of the 64th largest entry, the entries at or above it, their ranks ---------------------------------------
+  const int want = min(REC_TOP, V);
+  {
+    const uint32_t mine = tkeys[tid];
+    int rnk = 0;
+    for (int j = 0; j < REC_THREADS; ++j) {
+      const uint32_t o = tkeys[j];
+      rnk += (o > mine) || (o == mine && j < tid);
     }
-    __syncthreads();
-    if (tid < 256) {
-      uint32_t t = 0;
-      for (int w = 0; w < REC_WARPS; ++w) t += hist[w][tid];
-      hsum[tid] = t;
-    }
-    __syncthreads();
-    if (tid == 0) {
-      // walk down from the largest bin until `need` entries are covered
-      int need = level == 0 ? want : want - sh_above;
-      int above = 0, bin = 255;
-      for (; bin > 0; --bin) {
-        if (above + static_cast<int>(hsum[bin]) >= need) break;
-        above += static_cast<int>(hsum[bin]);
-      }
-      if (level == 0) { sh_cut = bin; sh_above = above; }
-      else { sh_cut = (hi_bin << 8) | bin; sh_above += above; sh_take = want - sh_above; }
-    }
-    __syncthreads();
-    if (level == 0) hi_bin = sh_cut;
+    if (rnk == REC_TOP - 1) sh_low = mine;
   }
-  const uint32_t cut = static_cast<uint32_t>(sh_cut);       // entries with key > cut are in; `take` of the ties at the cut
-  const int above = sh_above, take = sh_take;
-
-  // entries above the cut, any order
-  for (int i = tid; i < n_use; i += REC_THREADS) {
-    uint32_t key[8];
-    rec_keys8(buf[i], key);
+  __syncthreads();
+  const uint32_t low = max(sh_low, 0x007Fu);            // not below the key of -inf (threads without entries hold key 0)
+  const uint32_t low_bits = __float_as_uint(rec_value(low)) >> 16, low2 = (low_bits << 16) | low_bits;
+  for (int i0 = tid; i0 < nvec; i0 += REC_UNROLL * REC_THREADS) {
+    uint4 v[REC_UNROLL];
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
-      if (key[j] > cut) {
-        const int pos = atomicAdd(&sh_cnt, 1);
-        if (pos < REC_TOP)
-          cand[pos] = (static_cast<unsigned long long>(key[j]) << 32) |
-                      (0xFFFFFFFFull - static_cast<unsigned long long>((v_lo + i) * 8 + j));
+    for (int t = 0; t < REC_UNROLL; ++t) {
+      const int i = i0 + t * REC_THREADS;
+      v[t] = i < nvec ? rec_ldg(row + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+    }
+#pragma unroll
+    for (int t = 0; t < REC_UNROLL; ++t) {
+      // numeric packed comparison first (-0 equals +0 there as in the key): almost no vector holds an entry at or above the bound
+      if (i0 + t * REC_THREADS < nvec && (rec_ge2(v[t].x, low2) | rec_ge2(v[t].y, low2) | rec_ge2(v[t].z, low2) | rec_ge2(v[t].w, low2)) != 0u) {
+        uint32_t key[8];
+        rec_keys8(v[t], key);
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (key[j] >= low) {
+            const int pos = atomicAdd(&sh_nlist, 1);
+            if (pos < REC_LIST)
+              wlist[pos] = (static_cast<unsigned long long>(key[j]) << 32) |
+                           (0xFFFFFFFFull - static_cast<unsigned long long>((i0 + t * REC_THREADS) * 8 + j));
+          }
       }
+    }
   }
-  // ties at the cut, in token order: block-wide exclusive scan of the per-vector tie counts
-  int tie_base = 0;
-  for (int i0 = 0; i0 < n_use && tie_base < take; i0 += REC_THREADS) {
-    const int i = i0 + tid;
-    uint32_t key[8];
-    int mine = 0;
-    if (i < n_use) {
-      rec_keys8(buf[i], key);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) mine += key[j] == cut;
+  __syncthreads();
+  const bool from_list = sh_nlist <= REC_LIST;
+  if (from_list) {
+    const int nl = sh_nlist;
+    for (int i = tid; i < nl; i += REC_THREADS) {
+      const unsigned long long e = wlist[i];
+      int rnk = 0;
+      for (int j = 0; j < nl; ++j) rnk += wlist[j] > e;        // larger composite: larger key, then lower token id
+      if (rnk < REC_TOP) cand[rnk] = e;
     }
-    int incl = mine;
+  } else {
+    // ---- the general path.  The cut: 256-bin histograms of the key, high byte first, then the low byte inside the boundary bin
+    if (tid == 0) sh_cnt = 0;
+    uint32_t base = 0u;
+    int shift = 8;
+    for (int level = 0; level < 2; ++level) {
+      for (int i = tid; i < REC_WARPS * 256; i += REC_THREADS) (&hist[0][0])[i] = 0u;
+      __syncthreads();
+      for (int i0 = tid; i0 < nvec; i0 += 4 * REC_THREADS) {
+        uint4 v[4];
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int up = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += up;
-    }
-    __syncthreads();                                        // warp_tot of the previous iteration has been read
-    if (lane == 31) warp_tot[warp] = incl;
-    __syncthreads();
-    int base = tie_base;
-    for (int w = 0; w < warp; ++w) base += warp_tot[w];
-    int total = 0;
-    for (int w = 0; w < REC_WARPS; ++w) total += warp_tot[w];
-    int rnk = base + incl - mine;
-    if (i < n_use && mine > 0) {
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        if (key[j] == cut) {
-          if (rnk < take)
-            cand[above + rnk] = (static_cast<unsigned long long>(cut) << 32) |
-                                (0xFFFFFFFFull - static_cast<unsigned long long>((v_lo + i) * 8 + j));
-          ++rnk;
+        for (int t = 0; t < 4; ++t) {
+          const int i = i0 + t * REC_THREADS;
+          v[t] = i < nvec ? rec_ldg(row + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
         }
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          if (i0 + t * REC_THREADS < nvec) {
+            uint32_t key[8];
+            rec_keys8(v[t], key);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const uint32_t rel = (key[j] - base) >> shift;
+              if (key[j] >= base && rel < 256u) atomicAdd(&hist[warp][rel], 1u);
+            }
+          }
+        }
+      }
+      __syncthreads();
+      if (tid < 256) {
+        uint32_t t = 0;
+        for (int w = 0; w < REC_WARPS; ++w) t += hist[w][tid];
+        hsum[tid] = t;
+      }
+      __syncthreads();
+      if (tid == 0) {
+        // walk down from the largest bin until `need` entries are covered
+        const int need = level == 1 ? want - sh_above : want;
+        int above = 0, bin = 255;
+        for (; bin > 0; --bin) {
+          if (above + static_cast<int>(hsum[bin]) >= need) break;
+          above += static_cast<int>(hsum[bin]);
+        }
+        sh_cut = level == 0 ? bin : bin + static_cast<int>(base);     // the boundary bin, then the cut key
+        if (level == 1) sh_above += above; else sh_above = above;
+      }
+      __syncthreads();
+      base = static_cast<uint32_t>(sh_cut) << 8; shift = 0;
+      __syncthreads();                                // sh_* have been read before the next level rewrites them
     }
-    tie_base += total;
-  }
-  cluster.sync();
+    const uint32_t cut = static_cast<uint32_t>(sh_cut);     // entries with key > cut are in; `take` of the ties at the cut
+    const int above = sh_above, take = want - above;
 
-  // ---- merge in the first CTA -------------------------------------------------------------------------------------------
-  if (rank == 0) {
-    merge[tid] = *(cluster.map_shared_rank(&cand[0], tid / REC_TOP) + (tid % REC_TOP));     // 8 x 64 = 512 = REC_THREADS
-    __shared__ RecMZ row;
-    if (tid == 0) {
-      float m = -INFINITY;
-      RecMZ parts[REC_CLUSTER];
-      for (int c2 = 0; c2 < REC_CLUSTER; ++c2) { parts[c2] = *cluster.map_shared_rank(&local_mz, c2); m = fmaxf(m, parts[c2].m); }
-      float z = 0.f;
-      for (int c2 = 0; c2 < REC_CLUSTER; ++c2)
-        if (parts[c2].z > 0.f) z += parts[c2].z * rec_ex2((parts[c2].m - m) * s);
-      row = RecMZ{m, z};
+    // ---- pass 3: entries above the cut in any order; ties at the cut in token order --------------------------------------
+    int tie_base = 0;
+    for (int i0 = 0; i0 < nvec; i0 += REC_THREADS) {
+      const int i = i0 + tid;
+      uint32_t key[8];
+      int mine = 0;
+      if (i < nvec) {
+        rec_keys8(rec_ldg(row + i), key);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          mine += key[j] == cut;
+          if (key[j] > cut) {
+            const int pos = atomicAdd(&sh_cnt, 1);
+            if (pos < REC_TOP)
+              cand[pos] = (static_cast<unsigned long long>(key[j]) << 32) | (0xFFFFFFFFull - static_cast<unsigned long long>(i * 8 + j));
+          }
+        }
+      }
+      if (tie_base < take) {                                // uniform: tie_base is the same in every thread
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int up = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += up;
+        }
+        __syncthreads();                                    // warp_tot of the previous iteration has been read
+        if (lane == 31) warp_tot[warp] = incl;
+        __syncthreads();
+        int basep = tie_base, total = 0;
+        for (int w = 0; w < REC_WARPS; ++w) { if (w < warp) basep += warp_tot[w]; total += warp_tot[w]; }
+        int rnk = basep + incl - mine;
+        if (i < nvec && mine > 0) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (key[j] == cut) {
+              if (rnk < take)
+                cand[above + rnk] = (static_cast<unsigned long long>(cut) << 32) | (0xFFFFFFFFull - static_cast<unsigned long long>(i * 8 + j));
+              ++rnk;
+            }
+        }
+        tie_base += total;
+      }
     }
     __syncthreads();
-    // bitonic sort, descending, 512 composites (key, then lower token id first)
-    for (int size = 2; size <= REC_CLUSTER * REC_TOP; size <<= 1)
+    // order the 64 candidates (key descending, then lower token id first)
+    for (int size = 2; size <= REC_TOP; size <<= 1)
       for (int stride = size >> 1; stride > 0; stride >>= 1) {
-        const int partner = tid ^ stride;
-        if (partner > tid) {
-          const unsigned long long a = merge[tid], c2 = merge[partner];
-          const bool desc = (tid & size) == 0;
-          if (desc ? a < c2 : a > c2) { merge[tid] = c2; merge[partner] = a; }
+        if (tid < REC_TOP) {
+          const int partner = tid ^ stride;
+          if (partner > tid) {
+            const unsigned long long a2 = cand[tid], c2 = cand[partner];
+            const bool desc = (tid & size) == 0;
+            if (desc ? a2 < c2 : a2 > c2) { cand[tid] = c2; cand[partner] = a2; }
+          }
         }
         __syncthreads();
       }
-    if (tid < REC_TOP) {
-      const unsigned long long e = merge[tid];
-      const size_t o = (static_cast<size_t>(b) * A.K + k) * REC_TOP + tid;
-      if (e == 0ull) {
-        A.top_index[o] = -1;
-        A.top_logprob[o] = __float2bfloat16(-INFINITY);
-      } else {
-        const float x = rec_value(static_cast<uint32_t>(e >> 32));
-        A.top_index[o] = static_cast<int32_t>(0xFFFFFFFFull - (e & 0xFFFFFFFFull));
-        // ln p = ((x - max) s - log2 Z) ln 2
-        A.top_logprob[o] = __float2bfloat16(((x - row.m) * s - log2f(row.z)) * 0.6931471805599453f);
-      }
+  }
+  __syncthreads();
+
+  // ---- the record ----------------------------------------------------------------------------------------------------------
+  if (tid < REC_TOP) {
+    const unsigned long long e = cand[tid];
+    const size_t o = (static_cast<size_t>(b) * A.K + k) * REC_TOP + tid;
+    if (e == 0ull) {
+      A.top_index[o] = -1;
+      A.top_logprob[o] = __float2bfloat16(-INFINITY);
+    } else {
+      const float x = rec_value(static_cast<uint32_t>(e >> 32));
+      A.top_index[o] = static_cast<int32_t>(0xFFFFFFFFull - (e & 0xFFFFFFFFull));
+      // ln p = ((x - max) s - log2 Z) ln 2
+      A.top_logprob[o] = __float2bfloat16(((x - rowst.m) * s - log2f(rowst.z)) * 0.6931471805599453f);
     }
   }
-  cluster.sync();                                           // the peers' shared memory stays alive until it has been read
 }
 
 cudaError_t launch_record_topk(const RecordTopkArgs &A, int batch, cudaStream_t stream) {
-  const int vpc = ((A.V >> 3) + REC_CLUSTER - 1) / REC_CLUSTER;
-  const size_t dyn = (static_cast<size_t>(vpc) * 16 + 127) & ~size_t(127);
-  if (dyn > 160 * 1024) return cudaErrorInvalidValue;
-  static SmemConfigured configured;
-  if (cudaError_t e = ensure_dyn_smem(record_topk_kernel, dyn, configured); e != cudaSuccess) return e;
-  return launch_k(record_topk_kernel, dim3(batch * A.K * REC_CLUSTER), dim3(REC_THREADS), dyn, stream, 1, A);
+  return launch_k(record_topk_kernel, dim3(batch * A.K), dim3(REC_THREADS), 0, stream, 1, A);
 }
 
 // ---- the other items of the record -----------------------------------------------------------------------------------------

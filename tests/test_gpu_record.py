@@ -67,6 +67,17 @@ def test_ties_and_short_rows():
     idx, lp = _run_end(gmb, ctx, tgt, K)
     _check(tgt, K, idx, lp)
     ctx.close()
+    # peaked rows: fewer than 64 entries within 256 key steps of the maximum (the selection's full-range levels)
+    gmb, ctx = _ctx(4096, 2)
+    tgt = np.full((2, 3, 4096), -30.0, np.float32)
+    tgt[0, 0, 77] = 30.0                               # one-hot-like: the other 63 places are ties far below
+    tgt[0, 1, 5:25] = bf16_round(np.linspace(8, 20, 20).astype(np.float32))
+    tgt[1, 0] = bf16_round(np.random.default_rng(4).normal(0, 1, 4096).astype(np.float32))
+    tgt[1, 0, 1000:1040] = 500.0                       # 40 large ties, then the bulk of the row far below
+    tgt[1, 1] = bf16_round((np.arange(4096) % 97).astype(np.float32) * -0.5)
+    idx, lp = _run_end(gmb, ctx, tgt, 2)
+    _check(tgt, 2, idx, lp)
+    ctx.close()
     gmb, ctx = _ctx(40, 2)
     tgt, _ = sampler_only_logits(2, 1, 40, seed=9)
     idx, lp = _run_end(gmb, ctx, tgt, 1)
