@@ -101,7 +101,7 @@ static int gemm_entry(gm_ctx *c, const void *x, const void *w, void *out, int M,
     wm = it->second;
   }
   return run_gemm(c, static_cast<const __nv_bfloat16 *>(x), M, &wm, static_cast<const __nv_bfloat16 *>(w), M, N, K, out,
-                  epi, ldo);
+                  epi, ldo, false);        // a caller's matrix may have been written by the kernel before
 }
 
 int gm_gemm(gm_ctx *c, const void *x, const void *w, void *out, int M, int N, int K, int out_fp32) {

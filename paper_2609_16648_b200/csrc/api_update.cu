@@ -112,7 +112,7 @@ int gm_head_state_grad(gm_ctx *c, int rows, const void *grad_logits, const float
               launch_transpose_bf16(static_cast<const __nv_bfloat16 *>(c->w.lm_head), c->V, c->d, c->lm_head_t, c->stream));
   // dL/dy [rows, d] = grad_logits [rows, V] x W_lm [V, d]: the projection kernel with the vocabulary as its K
   rc = run_gemm(c, static_cast<const __nv_bfloat16 *>(grad_logits), rows, &c->lm_head_t_map, c->lm_head_t, rows, c->d, c->V,
-                grad_normed, EPI_STORE_F32, static_cast<size_t>(c->d));
+                grad_normed, EPI_STORE_F32, static_cast<size_t>(c->d), false);
   if (rc) return rc;
   if (grad_states)
     GM_LAUNCH(c, GM_KC_ELEMENTWISE,

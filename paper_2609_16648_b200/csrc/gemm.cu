@@ -132,7 +132,15 @@ gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  pdl_prologue();                                  // everything above touches no global data: it overlaps the previous kernel
+  // The weights are never written by a kernel of the stream, so the first ring of weight boxes may be requested before
+  // the previous kernel has finished (their bytes are counted on the stage barrier before its expect-tx arrives, which
+  // the barrier allows: the phase cannot complete until that arrival).  The activations wait for the dependency.
+  const int pre = A.early_weights ? min(nstages, kb_hi - kb_lo) : 0;
+  if (warp == 0 && lane == 0)
+    for (int it = 0; it < pre; ++it)
+      for (int a = 0; a < wt; ++a)
+        tma_load_2d(smem + static_cast<size_t>(it) * stage_b + a * GT_BN * 128, &A.w_map, (kb_lo + it) * GT_BK, n0 + a * GT_BN, &full[it]);
+  pdl_prologue();                                  // everything above touches no data a kernel writes: it overlaps the previous kernel
 
   if (warp == 0) {
     if (lane == 0) {
@@ -141,7 +149,8 @@ gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
         if (!mbar_wait(&empty[s], ((it / nstages) & 1) ^ 1)) { set_status(A.status, ST_TIMEOUT); break; }
         mbar_expect_tx(&full[s], stage_b);
         unsigned char *dst = smem + static_cast<size_t>(s) * stage_b;
-        for (int a = 0; a < wt; ++a) tma_load_2d(dst + a * GT_BN * 128, &A.w_map, kb * GT_BK, n0 + a * GT_BN, &full[s]);
+        if (it >= pre)
+          for (int a = 0; a < wt; ++a) tma_load_2d(dst + a * GT_BN * 128, &A.w_map, kb * GT_BK, n0 + a * GT_BN, &full[s]);
         tma_load_2d(dst + a_bytes, &A.x_map, kb * GT_BK, m0, &full[s]);
       }
     }

@@ -79,11 +79,12 @@ int pick_split(gm_ctx *c, int M, int N, int K, int T) {
 // out = epilogue(x[M, K] w[N, K]^T) on the tcgen05 kernel (or the plain one under GM_FLAG_SIMPLE_GEMM).
 int run_chain(gm_ctx *c, const ChainSpec *specs, int n, int M);
 int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *wmap, const __nv_bfloat16 *w, int M,
-             int N, int K, void *out, int epi, size_t ldo) {
+             int N, int K, void *out, int epi, size_t ldo, bool const_w) {
   GemmArgs A;
   std::memset(&A, 0, sizeof(A));
   A.x = x; A.w = w; A.M = M; A.N = N; A.K = K; A.status = c->status;
   A.out = out; A.epi = epi; A.ldo = ldo;
+  A.early_weights = (const_w && c->early_weights) ? 1 : 0;
   const int T = M >= 256 ? 256 : round16(M);
   A.block_t = T;
   A.nsplit = 1;
@@ -470,6 +471,7 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
     A_(dev_alloc(c, &ws, c->flow_ws_bytes));
     c->flow_ws = ws;
   }
+  if (std::getenv("GM_NO_EARLY_W")) c->early_weights = false;
   if (const char *ov = std::getenv("GM_SAMPLER")) {     // tuning aid: cluster | stream | flow for every sampler launch
     c->sampler_mode = !std::strcmp(ov, "cluster") ? 1 : !std::strcmp(ov, "stream") ? 2 : !std::strcmp(ov, "flow") ? 3 : 0;
   }

@@ -343,6 +343,7 @@ struct GemmArgs {
   int block_t;                          // tokens per CTA (multiple of 16, <= 256)
   int wtiles;                           // 128-feature sub-tiles per CTA sharing one activation tile (1 or 2)
   size_t ldo;                           // output row stride in elements
+  int early_weights;                    // w is written by no kernel of the stream: its first boxes may be fetched before the dependency wait
   uint32_t *status;
 };
 cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream);
