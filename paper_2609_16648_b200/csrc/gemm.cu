@@ -91,6 +91,74 @@ __device__ __forceinline__ void epilogue4(const GemmArgs &A, int m, int n, float
   }
 }
 
+// EPI_QKV_ROPE: one warp holds the 128 features [n0, n0 + 128) of token row m (lane l: features 4l .. 4l + 3), i.e. one
+// head of 128 or two heads of 64.  The value is rounded to bf16 first, exactly as the stand-alone projection stores it;
+// then bias, the head's RMSNorm, the rotary embedding (the partner half of a head sits hd/8 lanes away), and the
+// destination: the attention kernel's query layout, or the sequence's key / value page.
+__device__ __forceinline__ void rope_epilogue(const GemmArgs &G, int m, int n0, int lane, float4 acc) {
+  const RopeAppendArgs &A = G.rope;
+  const int hd = A.hd, half = hd >> 1, lph = hd >> 2;              // lanes per head
+  const int b = m / A.QT, j = m % A.QT;
+  const int n = n0 + 4 * lane, h = n / hd, fh = n % hd;
+  const int group = A.n_q / A.n_kv;
+  const int qn = A.qn[b];
+  float x[4] = {__bfloat162float(__float2bfloat16(acc.x)), __bfloat162float(__float2bfloat16(acc.y)),
+                __bfloat162float(__float2bfloat16(acc.z)), __bfloat162float(__float2bfloat16(acc.w))};
+  if (j >= qn) {                           // padding row: zero its query rows, append nothing
+    if (h < A.n_q)
+      *reinterpret_cast<uint2 *>(A.qbuf + ((static_cast<size_t>(b) * A.n_kv + h / group) * A.qrows + j * group + h % group) * hd + fh) =
+          make_uint2(0u, 0u);
+    return;
+  }
+  const int pos = A.qbase[b] + j;
+  if (A.bias) {
+    const uint2 bv = *reinterpret_cast<const uint2 *>(A.bias + n);
+    x[0] += bf16_lo(bv.x); x[1] += bf16_hi(bv.x); x[2] += bf16_lo(bv.y); x[3] += bf16_hi(bv.y);
+  }
+  const bool is_v = h >= A.n_q + A.n_kv;
+  {
+    // RMSNorm over the head dimension, before the rotation (the reduction runs in every lane: a warp may hold two heads)
+    float ss = x[0] * x[0] + x[1] * x[1] + x[2] * x[2] + x[3] * x[3];
+    for (int off = lph >> 1; off >= 1; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+    const __nv_bfloat16 *nw = is_v ? nullptr : (h < A.n_q ? A.qnorm : A.knorm);
+    if (nw) {
+      const float inv = rsqrtf(ss / static_cast<float>(hd) + A.eps);
+      const uint2 wv = *reinterpret_cast<const uint2 *>(nw + fh);
+      x[0] = x[0] * inv * bf16_lo(wv.x); x[1] = x[1] * inv * bf16_hi(wv.x);
+      x[2] = x[2] * inv * bf16_lo(wv.y); x[3] = x[3] * inv * bf16_hi(wv.y);
+    }
+  }
+  // the other half of the head (every lane takes part in the exchange, value heads too)
+  float xp[4];
+#pragma unroll
+  for (int t = 0; t < 4; ++t) xp[t] = __shfl_xor_sync(0xffffffffu, x[t], lph >> 1);
+  float y[4] = {x[0], x[1], x[2], x[3]};
+  if (!is_v) {
+    const bool lower = fh < half;
+    const float2 *cs = A.rope + static_cast<size_t>(pos) * half + (lower ? fh : fh - half);
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const float2 c = cs[t];
+      y[t] = lower ? x[t] * c.x - xp[t] * c.y : x[t] * c.x + xp[t] * c.y;
+    }
+  }
+  const uint2 o = make_uint2(pack_bf16(y[0], y[1]), pack_bf16(y[2], y[3]));
+  if (h < A.n_q) {
+    *reinterpret_cast<uint2 *>(A.qbuf + ((static_cast<size_t>(b) * A.n_kv + h / group) * A.qrows + j * group + h % group) * hd + fh) = o;
+    return;
+  }
+  const int page = A.page_table[static_cast<size_t>(b) * A.max_pages_per_seq + (pos >> 4)];
+  if (page < 0 || page >= A.num_pages) {
+    if (lane == 0) set_status(A.status, ST_BAD_PAGE);
+    return;
+  }
+  const int kvh = is_v ? h - A.n_q - A.n_kv : h - A.n_q;
+  const size_t page_elems = static_cast<size_t>(A.n_kv) * 16 * hd;
+  __nv_bfloat16 *dst = A.pool + ((static_cast<size_t>(A.layer) * 2 + (is_v ? 1 : 0)) * A.num_pages + page) * page_elems +
+                       (static_cast<size_t>(kvh) * 16 + (pos & 15)) * hd + fh;
+  *reinterpret_cast<uint2 *>(dst) = o;
+}
+
 template <int MINB>
 __global__ void __launch_bounds__(GT_THREADS, MINB)
 gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
@@ -223,7 +291,8 @@ gemm_tc_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
 #pragma unroll
         for (int p = 1; p < 8; ++p) { acc.x += v[p].x; acc.y += v[p].y; acc.z += v[p].z; acc.w += v[p].w; }
       }
-      epilogue4(A, m, n, acc);
+      if (A.epi == EPI_QKV_ROPE) rope_epilogue(A, m, n0 + a * GT_BN, lane, acc);
+      else epilogue4(A, m, n, acc);
     }
     if (ns > 1) cluster.sync();                    // peers may still be reading this CTA's parked tile
   }

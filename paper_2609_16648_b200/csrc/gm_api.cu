@@ -79,12 +79,13 @@ int pick_split(gm_ctx *c, int M, int N, int K, int T) {
 // out = epilogue(x[M, K] w[N, K]^T) on the tcgen05 kernel (or the plain one under GM_FLAG_SIMPLE_GEMM).
 int run_chain(gm_ctx *c, const ChainSpec *specs, int n, int M);
 int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *wmap, const __nv_bfloat16 *w, int M,
-             int N, int K, void *out, int epi, size_t ldo, bool const_w) {
+             int N, int K, void *out, int epi, size_t ldo, bool const_w, const RopeAppendArgs *rope) {
   GemmArgs A;
   std::memset(&A, 0, sizeof(A));
   A.x = x; A.w = w; A.M = M; A.N = N; A.K = K; A.status = c->status;
   A.out = out; A.epi = epi; A.ldo = ldo;
   A.early_weights = (const_w && c->early_weights) ? 1 : 0;
+  if (rope) A.rope = *rope;
   const int T = M >= 256 ? 256 : round16(M);
   A.block_t = T;
   A.nsplit = 1;
@@ -187,18 +188,8 @@ int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const 
   const gm_config &cf = c->cfg;
   const bool chain = chain_usable(c, ph.M);
   int rc;
-  // QKV projection (bf16) -> rotary + KV append + Q rearrangement
-  if (!(chain && qkv_done)) {
-    if (chain) {
-      const ChainSpec q = {lw.wqkv, c->xn, c->Mmax, c->n_qkv, c->d, c->qkv, EPI_STORE_BF16, c->n_qkv,
-                           nullptr, nullptr, nullptr, nullptr, 0, 0};
-      rc = run_chain(c, &q, 1, ph.M);
-    } else {
-      rc = run_gemm(c, c->xn, c->Mmax, &lm.wqkv, static_cast<const __nv_bfloat16 *>(lw.wqkv), ph.M, c->n_qkv, c->d,
-                    c->qkv, EPI_STORE_BF16, c->n_qkv);
-    }
-    if (rc) return rc;
-  }
+  // QKV projection (bf16) -> rotary + KV append + Q rearrangement: in the projection's epilogue where the tensor-core
+  // kernel runs it and a 128-feature tile holds whole heads, else as a kernel of its own
   RopeAppendArgs R;
   R.qkv = c->qkv;
   R.batch = ph.B; R.QT = ph.QT; R.n_q = cf.n_q_heads; R.n_kv = cf.n_kv_heads; R.hd = cf.head_dim; R.layer = layer;
@@ -208,7 +199,20 @@ int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const 
   R.bias = static_cast<const __nv_bfloat16 *>(lw.b_qkv);
   R.qnorm = static_cast<const __nv_bfloat16 *>(lw.q_norm); R.knorm = static_cast<const __nv_bfloat16 *>(lw.k_norm);
   R.eps = cf.rms_eps;
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rope_append(R, c->stream));
+  const bool fuse_rope = c->fuse_rope && !chain && !(cf.flags & GM_FLAG_SIMPLE_GEMM) && (cf.head_dim == 64 || cf.head_dim == 128) &&
+                         (c->d % 64) == 0;
+  if (!(chain && qkv_done)) {
+    if (chain) {
+      const ChainSpec q = {lw.wqkv, c->xn, c->Mmax, c->n_qkv, c->d, c->qkv, EPI_STORE_BF16, c->n_qkv,
+                           nullptr, nullptr, nullptr, nullptr, 0, 0};
+      rc = run_chain(c, &q, 1, ph.M);
+    } else {
+      rc = run_gemm(c, c->xn, c->Mmax, &lm.wqkv, static_cast<const __nv_bfloat16 *>(lw.wqkv), ph.M, c->n_qkv, c->d,
+                    c->qkv, fuse_rope ? EPI_QKV_ROPE : EPI_STORE_BF16, c->n_qkv, true, fuse_rope ? &R : nullptr);
+    }
+    if (rc) return rc;
+  }
+  if (!fuse_rope) GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rope_append(R, c->stream));
   // attention over the pages + merge of the segments
   AttnArgs T;
   T.kv_map = kvm; T.qbuf = c->qbuf; T.qn = c->qn; T.qbase = c->qbase; T.page_start = c->page_start;
@@ -472,6 +476,7 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
     c->flow_ws = ws;
   }
   if (std::getenv("GM_NO_EARLY_W")) c->early_weights = false;
+  if (std::getenv("GM_FUSED_ROPE")) c->fuse_rope = true;
   if (const char *ov = std::getenv("GM_SAMPLER")) {     // tuning aid: cluster | stream | flow for every sampler launch
     c->sampler_mode = !std::strcmp(ov, "cluster") ? 1 : !std::strcmp(ov, "stream") ? 2 : !std::strcmp(ov, "flow") ? 3 : 0;
   }

@@ -102,6 +102,7 @@ struct gm_ctx {
   void *flow_ws = nullptr;                  // work-queue sampler: counters, per-sequence state, slice partials, queue slots
   size_t flow_ws_bytes = 0;
   int flow_cap = 0;                         // batch the workspace was sized for
+  bool fuse_rope = false;                   // GM_FUSED_ROPE: rotary embedding + KV append in the QKV projection's epilogue (measured slower: off)
   bool early_weights = true;                // projections fetch their first weight boxes before the dependency wait (GM_NO_EARLY_W switches it off)
   int sampler_mode = 0;                     // 0 = by batch size; 1 cluster, 2 stream, 3 work queue (GM_SAMPLER in the environment)
   float *state_out = nullptr;               // set by the reconstruction while it runs: g_j of chain r -> state_out[(r*k + j-1)*d]
@@ -194,7 +195,8 @@ int x_map(gm_ctx *c, const void *ptr, int rows, int K, int box_rows, CUtensorMap
 int kv_map(gm_ctx *c, const void *pool, int layers, int num_pages, CUtensorMap *out);
 int round16(int v);
 int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *wmap, const __nv_bfloat16 *w, int M,
-             int N, int K, void *out, int epi, size_t ldo, bool const_w = true);   // const_w: w is a model weight (written by no kernel of the stream)
+             int N, int K, void *out, int epi, size_t ldo, bool const_w = true,
+             const RopeAppendArgs *rope = nullptr);   // const_w: w is a model weight (written by no kernel of the stream)
 struct PhaseShape { int B, QT, M, qrows; };
 // next_lw / next_lm: the layer whose QKV projection is appended to this layer's chain of projections (its input norm
 // is next_norm); qkv_done: this layer's own QKV projection was produced that way by the layer before.

@@ -330,6 +330,8 @@ enum GemmEpilogue {
   EPI_STORE_F32 = 1,     // out fp32 [M, ldo]
   EPI_ADD_F32 = 2,       // out fp32 [M, ldo] += result   (residual stream update)
   EPI_SWIGLU_BF16 = 3,   // rows of w interleaved (gate_i, up_i): out bf16 [M, ldo], column i = silu(gate_i) * up_i
+  EPI_QKV_ROPE = 4,      // the QKV projection: rounded to bf16, then bias, head norms, rotary embedding, query rows to qbuf and
+                         // keys / values appended to their pages (GemmArgs::rope; `out` unused); head_dim 64 or 128
 };
 struct GemmArgs {
   CUtensorMap w_map, x_map;             // tcgen05 path only
@@ -343,6 +345,7 @@ struct GemmArgs {
   int block_t;                          // tokens per CTA (multiple of 16, <= 256)
   int wtiles;                           // 128-feature sub-tiles per CTA sharing one activation tile (1 or 2)
   size_t ldo;                           // output row stride in elements
+  RopeAppendArgs rope;                  // EPI_QKV_ROPE only (qkv unused)
   int early_weights;                    // w is written by no kernel of the stream: its first boxes may be fetched before the dependency wait
   uint32_t *status;
 };

@@ -149,16 +149,21 @@ def test_tiny_step_parity_from_common_state(flags, chain, monkeypatch):
                                     dict(qkv_bias=True, qk_norm=True, n_q_heads=2, n_kv_heads=1, head_dim=128),
                                     dict(k=7), dict(k=1), dict(top_p=0.7),
                                     dict(k=5, n_q_heads=8, n_kv_heads=2, head_dim=128),
-                                    dict(k=7, n_q_heads=8, n_kv_heads=2, head_dim=128)],
+                                    dict(k=7, n_q_heads=8, n_kv_heads=2, head_dim=128),
+                                    dict(qkv_bias=True, qk_norm=True, fused_rope=True),
+                                    dict(qkv_bias=True, qk_norm=True, n_q_heads=2, n_kv_heads=1, head_dim=128, fused_rope=True)],
                          ids=["qkv_bias", "qk_norm", "bias_norm_hidden_first", "bias_norm_head128", "depth7", "depth1",
-                              "top_p_0.7", "depth5_group4_24_rows", "depth7_group4_32_rows"])
-def test_tiny_step_parity_variants(extras):
+                              "top_p_0.7", "depth5_group4_24_rows", "depth7_group4_32_rows", "fused_rope_head64",
+                              "fused_rope_head128"])
+def test_tiny_step_parity_variants(extras, monkeypatch):
     """The same bars for the other operating points of the cycle: the decoder-layer families of App. B.1
     (projection bias; query/key head norms), a head that concatenates [hidden ; embedding], and the
-    smallest and largest drafting depth, and the evaluation's nucleus sampling of the target."""
+    smallest and largest drafting depth, the evaluation's nucleus sampling of the target, and the fused QKV epilogue."""
     extras = dict(extras)
     concat = extras.pop("concat", None)
     top_p = extras.pop("top_p", 1.0)
+    if extras.pop("fused_rope", False):       # the option that runs the rotary embedding and the KV append in the QKV epilogue
+        monkeypatch.setenv("GM_FUSED_ROPE", "1")
     cfg = get_config("tiny").with_(prompt_len=40, **extras)
     worst, bits, toks, fins = _parity_from_common_state(cfg, 0, n_steps=10, concat=concat, top_p=top_p)
     assert worst < TOL, worst
