@@ -239,8 +239,8 @@ struct DcaGradArgs {
   float inv_temp;
 };
 cudaError_t launch_dca_grad(const DcaGradArgs &A, cudaStream_t stream);
-// Rollout-time capture of the target hidden states of committed positions (App. D.2: "each sequence additionally
-// stores the rollout-time target hidden states"): dst[b][pos] = the hidden state computed at position pos.
+// Rollout-time capture of the target hidden states of committed positions (App. D.2: the record keeps, per sequence,
+// the hidden states the target computed during the rollout): dst[b][pos] = the hidden state computed at position pos.
 //   chunk form (prefill): rows j < row_n[v] of src [rows, QT, d] go to positions row_base[v] + j of sequence v / vr;
 //   cycle form: rows l <= accept_len[b] of src [B, k+1, d] go to positions kv_len[b] - (accept_len[b] + 1) + l, with
 //   kv_len already advanced by the commit; rows of finished sequences are skipped.

@@ -1,4 +1,4 @@
-// The per-cycle record of a speculative rollout (App. D.2 "Recording in Rollout"): for each of the K verification
+// The per-cycle record of a speculative rollout (App. D.2, what is recorded during the rollout): for each of the K verification
 // positions the target's top-64 log-probabilities (bf16, full-vocabulary normalisation) with their token ids,
 // plus the cycle's start hidden state, start position, drafts and accepted length.
 //
