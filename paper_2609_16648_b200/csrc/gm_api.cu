@@ -303,9 +303,9 @@ cudaError_t run_sampler(gm_ctx *c, const SamplerArgs &S, int batch) {
   if (c->cfg.flags & GM_FLAG_SAMPLER_CLUSTER) mode = 1;
   if (c->cfg.flags & GM_FLAG_SAMPLER_STREAM) mode = 2;
   if (c->cfg.flags & GM_FLAG_SAMPLER_FLOW) mode = 3;
-  // by batch size (measured at K = 3, V = 151936): a cluster per sequence while sequences are few, the sliced mapping
-  // up to about 1.5 sequences per SM, one CTA per sequence beyond
-  if (mode == 0) mode = batch * 3 < c->sm_count * 2 ? 1 : (batch * 2 <= c->sm_count * 3 ? 3 : 2);
+  // by batch size (measured at K = 3, V = 151936): a cluster per sequence while sequences are few, the sliced mapping up
+  // to two sequences per SM, one CTA per sequence beyond
+  if (mode == 0) mode = batch * 3 < c->sm_count * 2 ? 1 : (batch <= c->sm_count * 2 ? 3 : 2);
   if (mode == 3 && !sampler_flow_supported(S.V, batch, S.K, c->sm_count)) mode = 2;
   if (mode == 3) {
     if (batch > c->flow_cap) {                         // a batch above max_batch (stand-alone gm_accept): grow, outside any capture

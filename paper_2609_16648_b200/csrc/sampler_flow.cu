@@ -51,7 +51,7 @@ struct SFWs {
   uint32_t *cnt;                                      // [B][rounds] arrivals
   unsigned long long *ent;                            // [B][4][NA] deliveries: tag << 32 | 32 payload bits (p max, p sum, q max, q sum;
                                                       // or the low and high half of a slice's residual weight)
-  int G, vps, tail, NA, rounds, R, nmain;                    // CTAs, vectors per slice, vectors after the last slice, deliveries per stage
+  int G, vps, tail, NA, rounds, R, nmain, wide;                    // CTAs, vectors per slice, vectors after the last slice, deliveries per stage
 };
 
 __device__ __forceinline__ unsigned long long sf_word(uint32_t epoch, int type, int k, int slice) {
@@ -170,6 +170,7 @@ constexpr int SF_ROUNDS = GM_MAX_K_ + 4;              // stride of the per-seque
 struct SFShared {
   uint64_t full[SF_MAX_R], empty[SF_MAX_R];
   uint32_t desc[SF_MAX_R];                            // type | use_q << 3 | k << 4 | tail << 8 | round << 9 | b << 16
+  volatile uint32_t use[SF_MAX_R];                    // 1 + the use count a slot is armed for (0: never)
   uint32_t done_mask[SF_MAX_B / 32];                  // producer: sequences whose walk has ended
   volatile int dead;
 };
@@ -231,7 +232,11 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
   const int c = blockIdx.x, G = W.G, vps = W.vps, NA = W.NA, R = W.R, rounds = W.rounds;
   const int K = A.K, V = A.V;
   const float s = A.inv_temp * 1.4426950408889634f;
-  const int nblk = (B + 31) / 32;
+  // `wide` neighbouring CTAs share a slice index and split the sequences among them (b mod wide): wider slices, fewer items
+  const int wide = W.wide, Gs = G / wide, grp = c % wide, sidx = c / wide;
+  const int nseq = B > grp ? (B - grp + wide - 1) / wide : 0;
+  const int nblk = (nseq + 31) / 32;
+  auto owner_of = [=](int b) { return wide == 1 ? b % G : ((b / wide) % Gs) * wide + (b % wide); };
 
   if (tid == 0) {
     for (int i = 0; i < R; ++i) { mbar_init(&sh.full[i], 1); mbar_init(&sh.empty[i], 1); }
@@ -239,6 +244,7 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
     sh.dead = 0;
   }
   for (int i = tid; i < SF_MAX_B / 32; i += SF_THREADS) sh.done_mask[i] = 0u;
+  for (int i = tid; i < SF_MAX_R; i += SF_THREADS) sh.use[i] = 0u;
   __syncthreads();
   pdl_prologue();
   const uint32_t epoch = ld_acquire_u32(&W.ctrl[SF_EPOCH]);
@@ -258,36 +264,41 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
     uint32_t n = 0;                                   // ring items posted so far (same value in every lane)
     bool alive = true;
     // every lane that holds an item takes the next free ring slots in lane order and starts its own copies
-    auto post = [&](bool has, uint32_t desc, const uint4 *prow, const uint4 *qrow) {
-      const uint32_t m = __ballot_sync(0xffffffffu, has);
-      if (has) {
-        const uint32_t mine = n + __popc(m & ((1u << lane) - 1u));
-        const int slot = mine % R;
-        if (wait_bar(&sh.empty[slot], ((mine / R) & 1u) ^ 1u)) {
-          sh.desc[slot] = desc;
-          if (prow != nullptr) {
-            const uint32_t bytes = static_cast<uint32_t>(vps) * 16u;
-            mbar_expect_tx(&sh.full[slot], qrow ? 2u * bytes : bytes);
-            fence_proxy_async();
-            bulk_load(ring + static_cast<size_t>(slot) * 2 * vps, prow + static_cast<size_t>(c) * vps, bytes, &sh.full[slot]);
-            if (qrow) bulk_load(ring + (static_cast<size_t>(slot) * 2 + 1) * vps, qrow + static_cast<size_t>(c) * vps, bytes, &sh.full[slot]);
-          } else {
-            mbar_arrive(&sh.full[slot]);
+    auto post = [&](bool has_all, uint32_t desc, const uint4 *prow, const uint4 *qrow) {
+      const int npass = R >= 32 ? 1 : 2;              // a small ring takes sixteen lanes at a time: never more items than slots
+      for (int pass = 0; pass < npass; ++pass) {
+        const bool has = has_all && (npass == 1 || (lane >> 4) == pass);
+        const uint32_t m = __ballot_sync(0xffffffffu, has);
+        if (has) {
+          const uint32_t mine = n + __popc(m & ((1u << lane) - 1u));
+          const int slot = mine % R;
+          if (wait_bar(&sh.empty[slot], ((mine / R) & 1u) ^ 1u)) {
+            sh.desc[slot] = desc;
+            if (R < 2 * SF_CWARPS + 2) sh.use[slot] = mine / R + 1u;   // armed for this use (before the barrier operations below)
+            if (prow != nullptr) {
+              const uint32_t bytes = static_cast<uint32_t>(vps) * 16u;
+              mbar_expect_tx(&sh.full[slot], qrow ? 2u * bytes : bytes);
+              fence_proxy_async();
+              bulk_load(ring + static_cast<size_t>(slot) * 2 * vps, prow + static_cast<size_t>(sidx) * vps, bytes, &sh.full[slot]);
+              if (qrow) bulk_load(ring + (static_cast<size_t>(slot) * 2 + 1) * vps, qrow + static_cast<size_t>(sidx) * vps, bytes, &sh.full[slot]);
+            } else {
+              mbar_arrive(&sh.full[slot]);
+            }
           }
         }
+        n += __popc(m);
+        __syncwarp();
       }
-      n += __popc(m);
-      __syncwarp();
     };
     for (int r = 0; r < rounds && alive; ++r) {
       bool any = false;
       for (int blk = 0; blk < nblk && alive; ++blk) {
-        const int b = blk * 32 + lane;
+        const int b = grp + wide * (blk * 32 + lane);
         bool act = b < B && !((sh.done_mask[blk] >> lane) & 1u);
         int type = SF_NONE, k = 0, use_q = 0, slice = 0;
         if (r == 0) {
           if (act && A.finished && A.finished[b]) {   // the row sits out: its owner writes the outputs
-            if (b % G == c) {
+            if (owner_of(b) == c) {
               if (A.accept_len) A.accept_len[b] = 0;
               A.next_token[static_cast<size_t>(b) * A.tok_out_stride] = A.accept_len ? -1 : 0;
             }
@@ -324,10 +335,10 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
         post(bulk && vps > 0, sf_desc(type, use_q, k, 0, r, b), bulk ? sf_row(A, b, prow_r) : nullptr,
              bulk && has_q ? sf_row(A, b, qrow_r) : nullptr);
         // what only one CTA does: the vectors after the last slice, the token search, the fallback
-        const bool own = act && b % G == c;
+        const bool own = act && owner_of(b) == c;
         post(bulk && own && W.tail > 0, sf_desc(type, use_q, k, 1, r, b), nullptr, nullptr);
         const bool fin = act && (type == SF_SEARCH || type == SF_ARGMAX);
-        post(fin && (type == SF_ARGMAX ? own : (slice == W.nmain ? own : slice == c)), sf_desc(type, use_q, k, slice == W.nmain ? 1 : 0, r, b),
+        post(fin && (type == SF_ARGMAX ? own : (slice == W.nmain ? own : slice == sidx)), sf_desc(type, use_q, k, slice == W.nmain ? 1 : 0, r, b),
              nullptr, nullptr);
         if (fin) atomicOr(&sh.done_mask[blk], 1u << lane);
         __syncwarp();
@@ -350,7 +361,7 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
   // ======================================================== merger ========================================================
   // Lane i watches the arrival counter of the i-th sequence this CTA owns; a completed stage is merged by the whole warp.
   if (warp == SF_MERGER) {
-    const int my_b = c + lane * G;
+    const int my_b = grp + wide * (sidx + Gs * lane);         // the sequences with owner_of(b) == c
     bool active = lane < SF_MAX_OWN && my_b < B && !(A.finished && A.finished[my_b]);
     int r = 0, type = SF_STAT, k = 0, use_q = 0;      // the stage in flight of lane i's sequence
     // what the accept decision of that stage will need, requested when the stage starts
@@ -533,13 +544,27 @@ __global__ void __launch_bounds__(SF_THREADS, 1) sampler_flow_kernel(const Sampl
   // ==================================================== compute warps ====================================================
   for (uint32_t n = warp;; n += SF_CWARPS) {
     const int slot = n % R;
+    // A ring shorter than two rounds of warps lets a warp get here before the slot's PREVIOUS use has even landed, and a
+    // parity wait cannot tell "not yet" from "already": wait until the producer has armed the slot for THIS use first.
+    if (R < 2 * SF_CWARPS + 2) {
+      const uint32_t want_use = n / R + 1u;
+      bool ok = false;
+      for (uint32_t i = 0; i < SF_SPIN_LIMIT; ++i) {
+        if (sh.use[slot] == want_use) { ok = true; break; }
+        if ((i & 63u) == 63u && sh.dead) break;
+      }
+      if (!ok) {
+        if (!sh.dead) { sh.dead = 1; set_status(A.status, ST_TIMEOUT); }
+        return;
+      }
+    }
     if (!wait_bar(&sh.full[slot], (n / R) & 1u)) return;
     const uint32_t desc = sh.desc[slot];
     const int type = desc & 7u, use_q = (desc >> 3) & 1u, k = (desc >> 4) & 15u, is_tail = (desc >> 8) & 1u, r = (desc >> 9) & 15u;
     const int b = desc >> 16;
     if (type == SF_QUIT) return;
-    const int idx = is_tail ? W.nmain : c;                  // which delivery of the stage this is
-    const int v_lo = is_tail ? W.nmain * vps : c * vps, nv = is_tail ? W.tail : vps;
+    const int idx = is_tail ? W.nmain : sidx;                  // which delivery of the stage this is
+    const int v_lo = is_tail ? W.nmain * vps : sidx * vps, nv = is_tail ? W.tail : vps;
     const uint4 *sp = ring + static_cast<size_t>(slot) * 2 * vps, *sq_ = sp + vps;
     bool released = false;                            // the ring slot has already been given back
     if (type == SF_STAT) {
@@ -695,14 +720,20 @@ __global__ void __launch_bounds__(SF_DUMP_THREADS) sampler_flow_dump_kernel(cons
   }
 }
 
-struct SFGeom { int G, vps, tail, NA, R, nmain; };
-SFGeom sf_geometry(int V, int sm_count) {
+struct SFGeom { int G, vps, tail, NA, R, nmain, wide; };
+// batch = 0: the widest geometry (one slice per CTA), which sizes the workspace
+SFGeom sf_geometry(int V, int sm_count, int batch) {
   SFGeom g;
   const int nvec = V >> 3;
   g.G = std::max(1, std::min(sm_count, nvec / 32));
-  g.vps = 32 * (nvec / (32 * g.G));
-  g.tail = nvec - g.G * g.vps;
-  g.nmain = g.vps > 0 ? g.G : 0;                      // slices that every CTA holds one of
+  // Large batches: pairs of CTAs share a slice index and take every other sequence each - slices twice as wide, half the
+  // items, copies and deliveries per stage (the per-item costs of the producer and of the compute warps are what binds).
+  g.wide = (batch >= 160 && g.G % 2 == 0 && nvec / (32 * (g.G / 2)) <= SF_UMAX) ? 2 : 1;
+  if (const char *ov = std::getenv("GM_SF_WIDE")) { const int v = std::atoi(ov); if ((v == 1 || v == 2 || v == 4) && g.G % v == 0) g.wide = v; }
+  const int gs = g.G / g.wide;
+  g.vps = 32 * (nvec / (32 * gs));
+  g.tail = nvec - gs * g.vps;
+  g.nmain = g.vps > 0 ? gs : 0;                       // slices that a CTA holds one of
   g.NA = g.nmain + (g.tail > 0 ? 1 : 0);
   g.R = g.vps > 0 ? std::min(SF_MAX_R, SF_RING_BYTES / (2 * g.vps * 16)) : SF_MAX_R;
   return g;
@@ -713,26 +744,26 @@ size_t sf_align(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
 bool sampler_flow_supported(int V, int batch, int K, int sm_count) {
   if ((V % 8) != 0 || V < 8 || batch < 1 || batch > SF_MAX_B || batch > 65535 || K > GM_MAX_K_) return false;
-  const SFGeom g = sf_geometry(V, sm_count);
-  return g.vps <= 32 * SF_UMAX && g.NA <= 32 * SF_EPL && batch <= SF_MAX_OWN * g.G && g.R >= 2 * SF_CWARPS + 2 && g.G <= 65535;
+  const SFGeom g = sf_geometry(V, sm_count, batch);
+  return g.vps <= 32 * SF_UMAX && g.NA <= 32 * SF_EPL && batch <= SF_MAX_OWN * g.G && g.R >= 16 && g.G <= 65535;
 }
 
 // Workspace: control words, per-sequence state, stage words, arrival counters, slice partials (zero-initialised once;
 // the kernel leaves the counters clean and tags the stage words with its epoch).  Its layout depends only on the
 // capacity it was sized for, so launches of any smaller batch and any depth share it.  The tail is scratch of the dump.
 size_t sampler_flow_ws_bytes(int cap_batch, int V, int sm_count) {
-  const SFGeom g = sf_geometry(V, sm_count);
+  const SFGeom g = sf_geometry(V, sm_count, 0);
   const size_t B = static_cast<size_t>(cap_batch), NA = static_cast<size_t>(g.NA);
   return sf_align(SF_CTRL_WORDS * 4) + sf_align(B * sizeof(SFSeq)) + sf_align(B * SF_ROUNDS * 8) + sf_align(B * SF_ROUNDS * 4) +
          sf_align(B * 4 * NA * 8) + sf_align(B * (2 * GM_MAX_K_ + 1) * NA * sizeof(MZ));
 }
 
 cudaError_t launch_sampler_flow(const SamplerArgs &A, int batch, void *ws, int cap_batch, int sm_count, cudaStream_t stream) {
-  const SFGeom g = sf_geometry(A.V, sm_count);
-  const size_t B = static_cast<size_t>(cap_batch), NA = static_cast<size_t>(g.NA);
+  const SFGeom g = sf_geometry(A.V, sm_count, batch);
+  const size_t B = static_cast<size_t>(cap_batch), NA = static_cast<size_t>(sf_geometry(A.V, sm_count, 0).NA);   // the layout's capacity
   if (batch > cap_batch) return cudaErrorInvalidValue;
   SFWs W;
-  W.G = g.G; W.vps = g.vps; W.tail = g.tail; W.NA = g.NA; W.R = g.R; W.rounds = A.K + 4; W.nmain = g.nmain;
+  W.G = g.G; W.vps = g.vps; W.tail = g.tail; W.NA = g.NA; W.R = g.R; W.rounds = A.K + 4; W.nmain = g.nmain; W.wide = g.wide;
   unsigned char *p = static_cast<unsigned char *>(ws);
   W.ctrl = reinterpret_cast<uint32_t *>(p); p += sf_align(SF_CTRL_WORDS * 4);
   W.seq = reinterpret_cast<SFSeq *>(p); p += sf_align(B * sizeof(SFSeq));
@@ -741,7 +772,7 @@ cudaError_t launch_sampler_flow(const SamplerArgs &A, int batch, void *ws, int c
   W.ent = reinterpret_cast<unsigned long long *>(p); p += sf_align(B * 4 * NA * 8);
   MZ *dump_scratch = reinterpret_cast<MZ *>(p);
   if (A.dbg_p != nullptr || A.dbg_q != nullptr) {
-    sampler_flow_dump_kernel<<<batch * (2 * A.K + 1), SF_DUMP_THREADS, 0, stream>>>(A, g.G, g.vps, g.tail, dump_scratch);
+    sampler_flow_dump_kernel<<<batch * (2 * A.K + 1), SF_DUMP_THREADS, 0, stream>>>(A, g.G / g.wide, g.vps, g.tail, dump_scratch);
     if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
   }
   const size_t dyn = static_cast<size_t>(g.R) * 2 * std::max(g.vps, 1) * 16;
