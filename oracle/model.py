@@ -140,6 +140,14 @@ def project_qkv(lw, h, cfg):
     return q, k, v
 
 
+def ffn_block(lw, x, cfg) -> np.ndarray:
+    """The feed-forward half of a pre-norm decoder layer (App. B.1): x + W_d (silu(W_g u) * (W_u u)), u = RMSNorm(x; ln2)."""
+    x = f64(x)
+    h2 = rmsnorm(x, lw["ln2"], cfg.rms_eps)
+    act = silu(h2 @ f64(lw["wg"]).T) * (h2 @ f64(lw["wu"]).T)
+    return x + act @ f64(lw["wd"]).T
+
+
 def decoder_layer(lw, x, pos, kv: PagedKV, layer: int, b: int, cfg) -> np.ndarray:
     """One pre-norm decoder layer over new rows x [T, d] at positions pos, against the cache.
 
@@ -158,9 +166,7 @@ def decoder_layer(lw, x, pos, kv: PagedKV, layer: int, b: int, cfg) -> np.ndarra
     kc, vc = kv.gather(layer, b, n)
     o = attention(q, kc, vc, pos, np.arange(n)).reshape(T, cfg.q_dim)
     x = x + o @ f64(lw["wo"]).T
-    h2 = rmsnorm(x, lw["ln2"], cfg.rms_eps)
-    act = silu(h2 @ f64(lw["wg"]).T) * (h2 @ f64(lw["wu"]).T)
-    return x + act @ f64(lw["wd"]).T
+    return ffn_block(lw, x, cfg)
 
 
 def target_forward(w, tokens, pos, kv: PagedKV, b: int, cfg) -> np.ndarray:

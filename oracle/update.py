@@ -23,6 +23,11 @@ Second step (Alg. 1, "update phi"): from the logits back to the head state g_k t
 are LMhead(RMSNorm_hf(g_k)) with the backbone's LM head (App. B.1), so dL/dy = (dL/dlogits) W_lm for the normed state y
 and dL/dg follows from the derivative of the RMSNorm.  This is the partial derivative through the logits of position
 k alone; the recurrence g_k -> g_{k+1} (Eq. 4) adds further terms in a later step of the backward pass.
+
+Third step: through the feed-forward half of the head's decoder layer (App. B.1: the head is one more layer of the
+backbone's shape), g = x + W_d (silu(W_g u) * (W_u u)) with u = RMSNorm(x; ln2).  Given dL/dg it returns dL/dx (the
+residual path plus the path through the block) and the gradients of the block's four parameter tensors, which are the
+first of the head's own weights the update step touches (Alg. 1, "update phi").
 """
 from __future__ import annotations
 
@@ -182,3 +187,26 @@ def head_update_grad_state(w, cfg, states, records, temperature: float = 1.0):
     gl = head_update_grad_logits(logits, records, temperature)
     gy = lm_head_input_grad(gl, w["lm_head"])
     return rmsnorm_grad(gy, states, w["head"]["final_norm"], cfg.rms_eps), gy, logits
+
+
+def ffn_block_grad(dg, x, lw, eps: float) -> dict:
+    """Backward of model.ffn_block.  dg [T, d] = dL/d(output), x [T, d] = the block's input (residual stream after
+    attention), lw = the layer's weights (ln2 [d], wg / wu [F, d], wd [d, F]).
+    Returns {"dx", "dln2", "dwg", "dwu", "dwd"} in float64."""
+    dg, x = f64(dg), f64(x)
+    w2, wg, wu, wd = f64(lw["ln2"]), f64(lw["wg"]), f64(lw["wu"]), f64(lw["wd"])
+    r = 1.0 / np.sqrt((x * x).mean(axis=-1, keepdims=True) + eps)
+    u = x * r * w2
+    a, b = u @ wg.T, u @ wu.T
+    sig = 1.0 / (1.0 + np.exp(-a))
+    act = a * sig
+    h = act * b
+    dh = dg @ wd                                              # y = h W_d^T
+    dwd = dg.T @ h
+    db = dh * act
+    da = dh * b * sig * (1.0 + a * (1.0 - sig))               # d silu(a) / da = sig (1 + a (1 - sig))
+    dwg, dwu = da.T @ u, db.T @ u
+    du = da @ wg + db @ wu
+    dx = dg + rmsnorm_grad(du, x, w2, eps)
+    dln2 = (du * x * r).sum(axis=0)
+    return {"dx": dx, "dln2": dln2, "dwg": dwg, "dwu": dwu, "dwd": dwd}

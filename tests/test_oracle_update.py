@@ -222,3 +222,39 @@ def test_head_state_gradient_matches_finite_differences_of_the_objective():
         np.testing.assert_allclose(gy, np.einsum("nkv,vd->nkd", gl, w["lm_head"]), rtol=1e-12)
         for r, rec in enumerate(recs):                       # positions after the first rejection get no gradient
             assert (g[r, min(rec["accepted"], K):] == 0).all()
+
+
+def test_ffn_block_gradient_matches_finite_differences():
+    """L = sum(C * ffn_block(x)) for a random C: every input coordinate and every entry of the four parameter tensors,
+    against central differences of the forward function the decoder layer itself calls."""
+    rng = np.random.default_rng(21)
+    T_, d, F = 3, 6, 5
+    cfg = CFG.with_(d_model=d, d_ffn=F, rms_eps=1e-3)
+    lw = {"ln2": rng.uniform(0.6, 1.4, d), "wg": rng.normal(0, 0.7, (F, d)), "wu": rng.normal(0, 0.7, (F, d)),
+          "wd": rng.normal(0, 0.7, (d, F))}
+    x, C = rng.normal(0, 1.2, (T_, d)), rng.normal(0, 1, (T_, d))
+    g = update.ffn_block_grad(C, x, lw, cfg.rms_eps)
+
+    def fd(get, put, shape):
+        out = np.zeros(shape)
+        for i in np.ndindex(*shape):
+            v = get()[i]
+            put(i, v + 1e-6); hi = float((model.ffn_block(lw, x, cfg) * C).sum())
+            put(i, v - 1e-6); lo = float((model.ffn_block(lw, x, cfg) * C).sum())
+            put(i, v)
+            out[i] = (hi - lo) / 2e-6
+        return out
+
+    def setter(arr):
+        def put(i, v):
+            arr[i] = v
+        return put
+
+    np.testing.assert_allclose(g["dx"], fd(lambda: x, setter(x), x.shape), rtol=2e-6, atol=1e-8)
+    for name, key in (("dln2", "ln2"), ("dwg", "wg"), ("dwu", "wu"), ("dwd", "wd")):
+        np.testing.assert_allclose(g[name], fd(lambda: lw[key], setter(lw[key]), lw[key].shape), rtol=2e-6, atol=1e-8)
+    # the residual path alone: with a zero down projection the block is the identity and so is its backward
+    lw0 = dict(lw, wd=np.zeros((d, F)))
+    g0 = update.ffn_block_grad(C, x, lw0, cfg.rms_eps)
+    np.testing.assert_array_equal(g0["dx"], C)
+    assert np.abs(g0["dwg"]).max() == 0 and np.abs(g0["dln2"]).max() == 0 and np.abs(g0["dwd"]).max() > 0
