@@ -392,6 +392,22 @@ int gm_dca_grad(gm_ctx *ctx, int n_cycles, int k, float temperature, const void 
  * LM head's weights in place since.  V % 64 != 0 returns GM_ERR_UNSUPPORTED.                                   */
 int gm_head_state_grad(gm_ctx *ctx, int rows, const void *grad_logits, const float *head_states,
                        float *grad_normed, float *grad_states, int refresh_weights);
+/* Third step of the backward pass: through the feed-forward half of the head's decoder layer (App. B.1: the head is one
+ * more layer of the backbone's shape),  g = x + W_d (silu(W_g u) * (W_u u)),  u = RMSNorm(x; ln2).
+ *   x    device fp32 [rows, d]: the block's input (the residual stream after the head layer's attention)
+ *   dg   device fp32 [rows, d]: dL/dg (for the rows' own logits: gm_head_state_grad's grad_states)
+ *   dx   device fp32 [rows, d] out: dL/dx = dg + the path through the block
+ *   dw_gate_up  device fp32 [2 F, d] out, rows interleaved like the packed weight (2f = gate feature f, 2f + 1 = up f);
+ *   dw_down     device fp32 [d, F] out;  dln2  device fp32 [d] out: the gradients of the block's parameters, summed
+ *               over the rows (the first of the head's own weights the update touches; Alg. 1, "update phi")
+ * The forward values it needs (u and the gate / up pre-activations) are recomputed from x in bf16 as the forward pass
+ * computes them; products run on the projection kernel (fp32 accumulation, bf16 operands: dg, the activation
+ * gradients and the recomputed activations are rounded to bf16 before they enter a product).  Transposed copies of the
+ * two weight matrices (3 d F bf16) and scratch for `rows` rounded up to 64 are allocated on first use and kept until
+ * gm_free; refresh_weights != 0 remakes the copies after the weights have been rewritten in place.
+ * d % 64 != 0, F % 64 != 0 or GM_FLAG_SIMPLE_GEMM: GM_ERR_UNSUPPORTED.                                         */
+int gm_head_ffn_backward(gm_ctx *ctx, int rows, const float *x, const float *dg, float *dx, float *dw_gate_up,
+                         float *dw_down, float *dln2, int refresh_weights);
 
 
 /* Dense projection out[M, N] = x[M, K] w[N, K]^T on the context's stream (bf16 in, fp32

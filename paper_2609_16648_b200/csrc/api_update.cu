@@ -121,4 +121,74 @@ int gm_head_state_grad(gm_ctx *c, int rows, const void *grad_logits, const float
   return GM_OK;
 }
 
+int gm_head_ffn_backward(gm_ctx *c, int rows, const float *x, const float *dg, float *dx, float *dw_gate_up, float *dw_down,
+                         float *dln2, int refresh_weights) {
+  if (!c || rows < 1 || !x || !dg || !dx || !dw_gate_up || !dw_down || !dln2) return GM_ERR_INVALID_ARG;
+  const int d = c->d, F = c->F;
+  if ((c->cfg.flags & GM_FLAG_SIMPLE_GEMM) || (d % 64) || (F % 64)) return GM_ERR_UNSUPPORTED;
+  const gm_layer_weights &lw = c->w.head_layer;
+  const __nv_bfloat16 *w_gu = static_cast<const __nv_bfloat16 *>(lw.w_gate_up), *w_d = static_cast<const __nv_bfloat16 *>(lw.w_down);
+  const __nv_bfloat16 *ln2 = static_cast<const __nv_bfloat16 *>(lw.ln2);
+  int rc;
+  if (!c->ffn_wd_t) {
+    if ((rc = dev_alloc(c, &c->ffn_wd_t, static_cast<size_t>(F) * d, false)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->ffn_wgu_t, static_cast<size_t>(d) * 2 * F, false)) != GM_OK) return rc;
+    if (make_map(c, &c->ffn_wd_t_map, c->ffn_wd_t, F, d, 128) != GM_OK) return GM_ERR_CUDA;
+    if (make_map(c, &c->ffn_wgu_t_map, c->ffn_wgu_t, d, 2 * F, 128) != GM_OK) return GM_ERR_CUDA;
+    refresh_weights = 1;
+  }
+  if (refresh_weights) {
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(w_d, d, F, c->ffn_wd_t, c->stream));             // [d, F] -> [F, d]
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(w_gu, 2 * F, d, c->ffn_wgu_t, c->stream));       // [2F, d] -> [d, 2F]
+  }
+  const int Mp = (rows + 63) / 64 * 64;              // the weight-gradient products contract over the rows: blocks of 64
+  if (Mp > c->ffn_rows_cap) {
+    const size_t M = static_cast<size_t>(Mp);
+    if ((rc = dev_alloc(c, &c->ffn_u, M * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->ffn_ab, M * 2 * F)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->ffn_dy, M * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->ffn_dab, M * 2 * F)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->ffn_h, M * F)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->ffn_ut, M * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->ffn_dyt, M * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->ffn_dabt, M * 2 * F)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->ffn_ht, M * F)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->ffn_dh, M * F)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->ffn_du, M * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->ffn_t, M * d)) != GM_OK) return rc;
+    c->ffn_rows_cap = Mp;
+  }
+  // forward values the backward needs, recomputed: u = RMSNorm(x; ln2), (a, b) = u W_gu^T (interleaved, bf16)
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rmsnorm(x, ln2, c->ffn_u, nullptr, rows, d, c->cfg.rms_eps, c->stream));
+  if ((rc = run_gemm(c, c->ffn_u, rows, &c->head_maps.wgu, w_gu, rows, 2 * F, d, c->ffn_ab, EPI_STORE_BF16, 2 * static_cast<size_t>(F))) != GM_OK)
+    return rc;
+  // dh = dg W_d   (the block's output is x + h W_d^T)
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_cast_bf16(dg, c->ffn_dy, static_cast<size_t>(rows) * d, c->stream));
+  if ((rc = run_gemm(c, c->ffn_dy, rows, &c->ffn_wd_t_map, c->ffn_wd_t, rows, F, d, c->ffn_dh, EPI_STORE_F32, static_cast<size_t>(F), false)) != GM_OK)
+    return rc;
+  // through the activation: (da, db) interleaved, and h for the down projection's weight gradient
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_swiglu_grad(c->ffn_ab, c->ffn_dh, c->ffn_dab, c->ffn_h, rows, F, c->stream));
+  // du = (da, db) W_gu;  dx = dg + d RMSNorm;  dln2 = sum over rows of du x r
+  if ((rc = run_gemm(c, c->ffn_dab, rows, &c->ffn_wgu_t_map, c->ffn_wgu_t, rows, d, 2 * F, c->ffn_du, EPI_STORE_F32, static_cast<size_t>(d), false)) != GM_OK)
+    return rc;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rmsnorm_grad(c->ffn_du, x, ln2, dx, rows, d, c->cfg.rms_eps, c->stream, dg, c->ffn_t));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->ffn_t, rows, d, dln2, c->stream));
+  // weight gradients contract over the rows: both operands transposed to [features, rows] (rows padded with zeros to Mp)
+  GM_CUDA(c, cudaMemsetAsync(c->ffn_ut, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
+  GM_CUDA(c, cudaMemsetAsync(c->ffn_dyt, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
+  GM_CUDA(c, cudaMemsetAsync(c->ffn_dabt, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * 2 * F, c->stream));
+  GM_CUDA(c, cudaMemsetAsync(c->ffn_ht, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * F, c->stream));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->ffn_u, rows, d, c->ffn_ut, c->stream, Mp));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->ffn_dy, rows, d, c->ffn_dyt, c->stream, Mp));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->ffn_dab, rows, 2 * F, c->ffn_dabt, c->stream, Mp));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->ffn_h, rows, F, c->ffn_ht, c->stream, Mp));
+  CUtensorMap wm;
+  // dW_d [d, F] = dg^T h
+  if (make_map(c, &wm, c->ffn_ht, F, Mp, 128) != GM_OK) return GM_ERR_CUDA;
+  if ((rc = run_gemm(c, c->ffn_dyt, d, &wm, c->ffn_ht, d, F, Mp, dw_down, EPI_STORE_F32, static_cast<size_t>(F), false)) != GM_OK) return rc;
+  // dW_gu [2F, d] = (da, db)^T u   (rows interleaved like the packed weight)
+  if (make_map(c, &wm, c->ffn_ut, d, Mp, 128) != GM_OK) return GM_ERR_CUDA;
+  return run_gemm(c, c->ffn_dabt, 2 * F, &wm, c->ffn_ut, 2 * F, d, Mp, dw_gate_up, EPI_STORE_F32, static_cast<size_t>(d), false);
+}
+
 }  // extern "C"

@@ -106,6 +106,13 @@ struct gm_ctx {
   bool early_weights = true;                // projections fetch their first weight boxes before the dependency wait (GM_NO_EARLY_W switches it off)
   int sampler_mode = 0;                     // 0 = by batch size; 1 cluster, 2 stream, 3 work queue (GM_SAMPLER in the environment)
   float *state_out = nullptr;               // set by the reconstruction while it runs: g_j of chain r -> state_out[(r*k + j-1)*d]
+  // head-update backward through the feed-forward block: transposed weight copies and scratch, made on first use
+  __nv_bfloat16 *ffn_wd_t = nullptr, *ffn_wgu_t = nullptr;   // [F, d], [d, 2F]
+  CUtensorMap ffn_wd_t_map, ffn_wgu_t_map;
+  int ffn_rows_cap = 0;
+  __nv_bfloat16 *ffn_u = nullptr, *ffn_ab = nullptr, *ffn_dy = nullptr, *ffn_dab = nullptr, *ffn_h = nullptr;
+  __nv_bfloat16 *ffn_ut = nullptr, *ffn_dyt = nullptr, *ffn_dabt = nullptr, *ffn_ht = nullptr;
+  float *ffn_dh = nullptr, *ffn_du = nullptr, *ffn_t = nullptr;
   __nv_bfloat16 *lm_head_t = nullptr;       // [d, V]: the LM head transposed, the weight operand of the gradient GEMM
   CUtensorMap lm_head_t_map;
   float top_p = 1.f;                    // nucleus of the target distributions (1 = none)

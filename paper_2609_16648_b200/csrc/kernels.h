@@ -252,10 +252,18 @@ cudaError_t launch_capture_cycle(const __nv_bfloat16 *src, const int32_t *accept
 cudaError_t launch_dca_loss(const float *alpha, const int32_t *accepted, int n, int K, float *loss, float *mean,
                             cudaStream_t stream);
 // Backward through an RMSNorm y = x r w (fp32 rows of d values, bf16 weight): gx = r (w gy) - x r^3 mean(x w gy).
+//   res (or null): added to gx (the gradient that reaches x past the norm, e.g. along a residual connection);
+//   wterm (or null): fp32 [rows, d], gy x r per row - the rows' terms of dL/dw.
 cudaError_t launch_rmsnorm_grad(const float *gy, const float *x, const __nv_bfloat16 *w, float *gx, int rows, int d, float eps,
-                                cudaStream_t stream);
-// dst [cols, rows] = transpose of src [rows, cols] (bf16, both row-major).
-cudaError_t launch_transpose_bf16(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst, cudaStream_t stream);
+                                cudaStream_t stream, const float *res = nullptr, float *wterm = nullptr);
+// dst [cols, dst_ld] = transpose of src [rows, cols] (bf16, both row-major; dst_ld >= rows, 0 = rows; padding untouched).
+cudaError_t launch_transpose_bf16(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst, cudaStream_t stream, int dst_ld = 0);
+// out[j] = sum over rows of t[row][j] (fp32, row order).
+cudaError_t launch_colsum(const float *t, int rows, int d, float *out, cudaStream_t stream);
+cudaError_t launch_cast_bf16(const float *src, __nv_bfloat16 *dst, size_t n, cudaStream_t stream);       // n % 4 == 0
+// Backward of h = silu(a) * b on interleaved (a, b) columns: dab bf16 [rows, 2F] (da, db interleaved), h bf16 [rows, F].
+cudaError_t launch_swiglu_grad(const __nv_bfloat16 *ab, const float *dh, __nv_bfloat16 *dab, __nv_bfloat16 *h, int rows, int F,
+                               cudaStream_t stream);
 
 // ---- element-wise --------------------------------------------------------------------------------------
 // x[m] = embed[token(m)] (fp32), xn[m] = RMSNorm(x[m]; w) (bf16); rows m = b*QT + j of the verify phase.

@@ -291,7 +291,8 @@ capture_cycle_kernel(const __nv_bfloat16 *src, const int32_t *accept_len, const 
 // y = x r w with r = (mean(x^2) + eps)^(-1/2):  dL/dx = r (w gy) - x r^3 mean(x w gy).  One CTA per row, fp32.
 constexpr int NG_THREADS = 256;
 __global__ void __launch_bounds__(NG_THREADS)
-rmsnorm_grad_kernel(const float *gy, const float *x, const __nv_bfloat16 *w, float *gx, int d, float eps) {
+rmsnorm_grad_kernel(const float *gy, const float *x, const __nv_bfloat16 *w, float *gx, int d, float eps, const float *res,
+                    float *wterm) {
   __shared__ float red[2][NG_THREADS / 32];
   const size_t row = static_cast<size_t>(blockIdx.x) * d;
   const int tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
@@ -311,12 +312,46 @@ rmsnorm_grad_kernel(const float *gy, const float *x, const __nv_bfloat16 *w, flo
   const float inv_d = 1.0f / static_cast<float>(d);
   const float r = rsqrtf(sq * inv_d + eps);
   const float c = r * r * r * dot * inv_d;
-  for (int i = tid; i < d; i += NG_THREADS)
-    gx[row + i] = r * bf16_to_float(w[i]) * gy[row + i] - x[row + i] * c;
+  for (int i = tid; i < d; i += NG_THREADS) {
+    const float g = gy[row + i], xv = x[row + i];
+    gx[row + i] = (res ? res[row + i] : 0.f) + (r * bf16_to_float(w[i]) * g - xv * c);     // res: the residual path's gradient
+    if (wterm) wterm[row + i] = g * xv * r;                    // this row's term of dL/dw (summed over the rows afterwards)
+  }
 }
 
+// out[j] = sum over the rows of t[row][j], added in row order (fp32).
+__global__ void __launch_bounds__(256) colsum_kernel(const float *t, int rows, int d, float *out) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= d) return;
+  float acc = 0.f;
+  for (int r = 0; r < rows; ++r) acc += t[static_cast<size_t>(r) * d + j];
+  out[j] = acc;
+}
+
+// fp32 -> bf16, n elements (n % 4 == 0)
+__global__ void __launch_bounds__(256) cast_bf16_kernel(const float *src, __nv_bfloat16 *dst, size_t n4) {
+  const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= n4) return;
+  const float4 v = reinterpret_cast<const float4 *>(src)[i];
+  reinterpret_cast<uint2 *>(dst)[i] = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
+}
+
+// Backward of the SwiGLU activation h = silu(a) * b on interleaved rows (a_f at column 2f, b_f at 2f + 1):
+//   dab[2f] = dh_f b_f sig (1 + a_f (1 - sig)),  dab[2f + 1] = dh_f silu(a_f),  h_f recomputed for the down projection's
+//   weight gradient.  One thread per (row, f) pair.
+__global__ void __launch_bounds__(256)
+swiglu_grad_kernel(const __nv_bfloat16 *ab, const float *dh, __nv_bfloat16 *dab, __nv_bfloat16 *h, size_t n, int F) {
+  const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const uint32_t w = reinterpret_cast<const uint32_t *>(ab)[i];
+  const float a = bf16_lo(w), b = bf16_hi(w), g = dh[i];
+  const float sig = 1.0f / (1.0f + __expf(-a)), act = a * sig;
+  reinterpret_cast<uint32_t *>(dab)[i] = pack_bf16(g * b * sig * (1.0f + a * (1.0f - sig)), g * act);
+  h[i] = __float2bfloat16(act * b);
+  }
+
 // dst[c][r] = src[r][c] for a row-major bf16 matrix [rows, cols]; 64 x 64 tiles through shared memory.
-__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst) {
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst, int dst_ld) {
   __shared__ __nv_bfloat16 tile[64][66];
   const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
   const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
@@ -324,7 +359,7 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16
     if (r0 + i < rows && c0 + tx < cols) tile[i][tx] = src[static_cast<size_t>(r0 + i) * cols + c0 + tx];
   __syncthreads();
   for (int i = ty; i < 64; i += 4)
-    if (c0 + i < cols && r0 + tx < rows) dst[static_cast<size_t>(c0 + i) * rows + r0 + tx] = tile[tx][i];
+    if (c0 + i < cols && r0 + tx < rows) dst[static_cast<size_t>(c0 + i) * dst_ld + r0 + tx] = tile[tx][i];
 }
 
 }  // namespace
@@ -360,11 +395,25 @@ cudaError_t launch_dca_loss(const float *alpha, const int32_t *accepted, int n, 
   return launch_k(dca_loss_kernel, dim3(1), dim3(DL_THREADS), 0, stream, 1, alpha, accepted, n, K, loss, mean);
 }
 cudaError_t launch_rmsnorm_grad(const float *gy, const float *x, const __nv_bfloat16 *w, float *gx, int rows, int d, float eps,
-                                cudaStream_t stream) {
-  return launch_k(rmsnorm_grad_kernel, dim3(rows), dim3(NG_THREADS), 0, stream, 1, gy, x, w, gx, d, eps);
+                                cudaStream_t stream, const float *res, float *wterm) {
+  return launch_k(rmsnorm_grad_kernel, dim3(rows), dim3(NG_THREADS), 0, stream, 1, gy, x, w, gx, d, eps, res, wterm);
 }
-cudaError_t launch_transpose_bf16(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst, cudaStream_t stream) {
-  transpose_bf16_kernel<<<dim3((cols + 63) / 64, (rows + 63) / 64), 256, 0, stream>>>(src, rows, cols, dst);
+cudaError_t launch_transpose_bf16(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst, cudaStream_t stream, int dst_ld) {
+  transpose_bf16_kernel<<<dim3((cols + 63) / 64, (rows + 63) / 64), 256, 0, stream>>>(src, rows, cols, dst, dst_ld > 0 ? dst_ld : rows);
+  return cudaGetLastError();
+}
+cudaError_t launch_colsum(const float *t, int rows, int d, float *out, cudaStream_t stream) {
+  colsum_kernel<<<(d + 255) / 256, 256, 0, stream>>>(t, rows, d, out);
+  return cudaGetLastError();
+}
+cudaError_t launch_cast_bf16(const float *src, __nv_bfloat16 *dst, size_t n, cudaStream_t stream) {
+  cast_bf16_kernel<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, stream>>>(src, dst, n / 4);
+  return cudaGetLastError();
+}
+cudaError_t launch_swiglu_grad(const __nv_bfloat16 *ab, const float *dh, __nv_bfloat16 *dab, __nv_bfloat16 *h, int rows, int F,
+                               cudaStream_t stream) {
+  const size_t n = static_cast<size_t>(rows) * F;
+  swiglu_grad_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(ab, dh, dab, h, n, F);
   return cudaGetLastError();
 }
 

@@ -288,6 +288,64 @@ def test_head_state_gradient_at_the_4b_dimensions(rows):
     ctx.close()
 
 
+@pytest.mark.parametrize("name,rows", [("tiny", 24), ("tiny", 100), ("4b", 192)], ids=["tiny-24", "tiny-100_ragged", "4b-192"])
+def test_head_ffn_backward_matches_the_oracle(name, rows):
+    """gm_head_ffn_backward on the head layer's feed-forward block against the oracle's fp64 backward of the same block
+    (same bf16 weights, same fp32 inputs).  The device rounds the recomputed activations and the activation gradients
+    to bf16 before each product, so tensors are compared by their largest entry; at the 4B dimensions (d 2560, F 9728)
+    the weight gradients are compared on sampled rows."""
+    import paper_2609_16648_b200 as gmb
+    base = get_config("tiny")
+    cfg = base if name == "tiny" else base.with_(d_model=2560, d_ffn=9728, vocab=4096)
+    d, F = cfg.d_model, cfg.d_ffn
+    ctx = gmb.Context(cfg, gmb.random_packed_weights(cfg, "cuda"), 4, 3, 4, 8, 8)
+    g = torch.Generator(device="cuda").manual_seed(5)
+    hl = ctx.packed["head"]["layer"]
+    hl["ln2"].copy_((1 + (torch.rand(d, device="cuda", generator=g) - 0.5) * 0.5).to(torch.bfloat16))
+    for key in ("w_gate_up", "w_down"):                       # larger than the init scale, so that the block's path matters
+        hl[key].copy_((torch.randn(hl[key].shape, device="cuda", generator=g) * (2.0 / np.sqrt(hl[key].shape[1]))).to(torch.bfloat16))
+    x = torch.randn((rows, d), device="cuda", generator=g) * 1.5
+    dg = torch.randn((rows, d), device="cuda", generator=g) * 0.1
+    dg[1::4] = 0                                               # rows without a gradient (after the first rejection)
+    z = lambda *shape: torch.full(shape, 7.0, dtype=torch.float32, device="cuda")
+    dx, dwgu, dwd, dln2 = z(rows, d), z(2 * F, d), z(d, F), z(d)
+    gmb.gm_head_ffn_backward(ctx, rows, x, dg, dx, dwgu, dwd, dln2)
+    assert gmb.gm_last_status(ctx) == 0
+    f = lambda t: t.double().cpu().numpy()
+    wgu = f(hl["w_gate_up"])
+    lw = {"ln2": f(hl["ln2"]), "wg": wgu[0::2], "wu": wgu[1::2], "wd": f(hl["w_down"])}
+    want = oupdate.ffn_block_grad(f(dg), f(x), lw, cfg.rms_eps)
+    tol = 2.5e-2
+    assert rel_err(f(dx), want["dx"]) < tol
+    assert rel_err(f(dx) - f(dg), want["dx"] - f(dg)) < tol          # the block's own path, not hidden behind the residual one
+    assert (f(dx)[1::4] == 0).all()                                    # no gradient in, none out
+    assert rel_err(f(dln2), want["dln2"]) < tol
+    rs = np.random.default_rng(2).choice(F, min(F, 64), replace=False)
+    assert rel_err(f(dwgu)[0::2][rs], want["dwg"][rs]) < tol and rel_err(f(dwgu)[1::2][rs], want["dwu"][rs]) < tol
+    cs = np.random.default_rng(3).choice(d, min(d, 64), replace=False)
+    assert rel_err(f(dwd)[cs], want["dwd"][cs]) < tol
+    assert np.abs(want["dwd"]).max() > 0 and np.abs(want["dwg"]).max() > 0
+    # a second call with fewer rows reuses the scratch: same numbers as a fresh computation of that prefix
+    r2 = rows // 2
+    dx2, dwgu2, dwd2, dln22 = z(r2, d), z(2 * F, d), z(d, F), z(d)
+    gmb.gm_head_ffn_backward(ctx, r2, x[:r2].contiguous(), dg[:r2].contiguous(), dx2, dwgu2, dwd2, dln22, refresh_weights=True)
+    want2 = oupdate.ffn_block_grad(f(dg)[:r2], f(x)[:r2], lw, cfg.rms_eps)
+    assert torch.equal(dx2, dx[:r2])
+    assert rel_err(f(dwd2)[cs], want2["dwd"][cs]) < tol and rel_err(f(dln22), want2["dln2"]) < tol
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    for _ in range(2):
+        gmb.gm_head_ffn_backward(ctx, rows, x, dg, dx, dwgu, dwd, dln2)
+    ev[0].record()
+    for _ in range(5):
+        gmb.gm_head_ffn_backward(ctx, rows, x, dg, dx, dwgu, dwd, dln2)
+    ev[1].record()
+    torch.cuda.synchronize()
+    ms = ev[0].elapsed_time(ev[1]) / 5
+    print(f"gm_head_ffn_backward {name} rows {rows}: {ms:.3f} ms per call, {16.0 * rows * d * F / ms / 1e9:.0f} TFLOP/s "
+          f"over its five products (the recomputed gate/up forward, two input gradients, two weight gradients)")
+    ctx.close()
+
+
 def test_loss_kernel_edge_cases():
     import paper_2609_16648_b200 as gmb
     cfg = get_config("tiny")
