@@ -379,10 +379,12 @@ def test_rerun_is_bit_identical_and_resume_equals_uninterrupted():
     ctx.close()
 
 
-def test_graph_replayed_cycle_equals_host_launched_cycle():
+@pytest.mark.parametrize("sampler_flag", [0, 16], ids=["sampler_by_batch", "sampler_slice_per_cta"])
+def test_graph_replayed_cycle_equals_host_launched_cycle(sampler_flag):
     """GM_FLAG_GRAPH on a stream of its own: gm_spec_step and gm_spec_step_host replay a captured cycle; accept
     lengths, tokens, drafts and the final state are bit-identical to the host-launched cycle, across re-captures
-    (other output buffers) and with the step index changing every call."""
+    (other output buffers) and with the step index changing every call.  With the sliced sampler the replayed launches
+    find their epoch and their clean counters in device memory, not in captured arguments."""
     import paper_2609_16648_b200 as gmb
     cfg = get_config("tiny").with_(prompt_len=33)
     K, B = cfg.k, cfg.batch
@@ -390,7 +392,7 @@ def test_graph_replayed_cycle_equals_host_launched_cycle():
     side = torch.cuda.Stream()
     for flags in (0, gmb.GM_FLAG_GRAPH):
         with torch.cuda.stream(side):
-            w, ost, ctx, gst = tiny_setup(cfg, cap_tokens=160, flags=flags)
+            w, ost, ctx, gst = tiny_setup(cfg, cap_tokens=160, flags=flags | sampler_flag)
             push_state(ost, gst, ctx)
             z = lambda *shape: torch.zeros(shape, dtype=torch.int32, device="cuda")
             a, t, d, a2, t2 = z(B), z(B), z(B, K), z(B), z(B)
