@@ -31,11 +31,15 @@ def _free_running_streams(gmb, ctx, gst, K, seed, n_steps):
     return streams, per_step
 
 
-def test_rollout_equals_plain_cycles_cut_by_the_stopping_rules():
+@pytest.mark.parametrize("sampler", [None, "flow"], ids=["sampler_by_batch", "sampler_slice_per_cta"])
+def test_rollout_equals_plain_cycles_cut_by_the_stopping_rules(sampler, monkeypatch):
     """The rollout driver's responses are the streams of plain cycles cut by the oracle's stopping rule; rows
     that have ended sit out and leave the others unchanged (here every attention segment is a single page, so
-    the running rows' arithmetic does not depend on who else is running)."""
+    the running rows' arithmetic does not depend on who else is running).  Both with the sampler mapping the batch
+    size selects and with the sliced mapping forced (rows that sit out, state commit)."""
     import paper_2609_16648_b200 as gmb
+    if sampler:
+        monkeypatch.setenv("GM_SAMPLER", sampler)
     cfg = get_config("tiny").with_(prompt_len=20)
     K, B = cfg.k, cfg.batch
     n_steps, cap = 10, 13
