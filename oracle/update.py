@@ -28,6 +28,11 @@ Third step: through the feed-forward half of the head's decoder layer (App. B.1:
 backbone's shape), g = x + W_d (silu(W_g u) * (W_u u)) with u = RMSNorm(x; ln2).  Given dL/dg it returns dL/dx (the
 residual path plus the path through the block) and the gradients of the block's four parameter tensors, which are the
 first of the head's own weights the update step touches (Alg. 1, "update phi").
+
+The update itself: AdamW on the head's parameter group, with the head's learning-rate schedule (App. B, optimizer and
+learning rate: linear warm-up over 10 steps, then a cosine decay to a tenth of the peak).  The paper names the
+optimizer and the rates only; the moment coefficients, the stabilising constant and the weight decay are the defaults
+of the optimizer it names (0.9, 0.999, 1e-8, 0.01), with the decay applied to the parameter directly (decoupled).
 """
 from __future__ import annotations
 
@@ -210,3 +215,26 @@ def ffn_block_grad(dg, x, lw, eps: float) -> dict:
     dx = dg + rmsnorm_grad(du, x, w2, eps)
     dln2 = (du * x * r).sum(axis=0)
     return {"dx": dx, "dln2": dln2, "dwg": dwg, "dwu": dwu, "dwd": dwd}
+
+
+def adamw_step(p, g, m, v, step: int, lr: float, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
+               weight_decay: float = 0.01):
+    """One AdamW update (decoupled weight decay); `step` counts from 1.  Returns (p, m, v), float64.
+        m <- b1 m + (1 - b1) g,  v <- b2 v + (1 - b2) g^2,
+        p <- p (1 - lr wd) - lr (m / (1 - b1^t)) / (sqrt(v / (1 - b2^t)) + eps)."""
+    p, g, m, v = f64(p), f64(g), f64(m), f64(v)
+    m = beta1 * m + (1.0 - beta1) * g
+    v = beta2 * v + (1.0 - beta2) * g * g
+    m_hat = m / (1.0 - beta1 ** step)
+    v_hat = v / (1.0 - beta2 ** step)
+    p = p * (1.0 - lr * weight_decay) - lr * m_hat / (np.sqrt(v_hat) + eps)
+    return p, m, v
+
+
+def head_lr(step: int, peak: float, total_steps: int, warmup: int = 10, floor: float = 0.1) -> float:
+    """Learning rate of the head's parameter group at update `step` (from 0): linear warm-up to `peak` over `warmup`
+    steps, then half a cosine from `peak` down to `floor * peak` at `total_steps`."""
+    if step < warmup:
+        return peak * (step + 1) / warmup
+    t = min(1.0, (step - warmup) / max(1, total_steps - warmup))
+    return peak * (floor + (1.0 - floor) * 0.5 * (1.0 + np.cos(np.pi * t)))

@@ -258,3 +258,45 @@ def test_ffn_block_gradient_matches_finite_differences():
     g0 = update.ffn_block_grad(C, x, lw0, cfg.rms_eps)
     np.testing.assert_array_equal(g0["dx"], C)
     assert np.abs(g0["dwg"]).max() == 0 and np.abs(g0["dln2"]).max() == 0 and np.abs(g0["dwd"]).max() > 0
+
+
+def test_adamw_step_matches_the_library_optimizer_and_its_closed_forms():
+    import torch
+    rng = np.random.default_rng(8)
+    p0 = rng.normal(0, 1, 37)
+    grads = [rng.normal(0, 0.3, 37) for _ in range(6)]
+    lr, wd = 3e-4, 0.01
+    tp = torch.nn.Parameter(torch.tensor(p0, dtype=torch.float64))
+    opt = torch.optim.AdamW([tp], lr=lr, betas=(0.9, 0.999), eps=1e-8, weight_decay=wd)
+    p, m, v = p0.copy(), np.zeros(37), np.zeros(37)
+    for t, g in enumerate(grads, start=1):
+        tp.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        p, m, v = update.adamw_step(p, g, m, v, t, lr, weight_decay=wd)
+        np.testing.assert_allclose(p, tp.detach().numpy(), rtol=1e-13, atol=1e-15)
+    # first step from zero moments: the bias corrections give m_hat = g, v_hat = g^2, so the move is lr g / (|g| + eps)
+    g = grads[0]
+    p1, _, _ = update.adamw_step(p0, g, np.zeros(37), np.zeros(37), 1, lr, weight_decay=0.0)
+    np.testing.assert_allclose(p0 - p1, lr * g / (np.abs(g) + 1e-8), rtol=1e-12)
+    # weight decay alone (zero gradient, zero moments): a plain shrink of the parameter
+    p2, m2, v2 = update.adamw_step(p0, np.zeros(37), np.zeros(37), np.zeros(37), 1, lr, weight_decay=wd)
+    np.testing.assert_allclose(p2, p0 * (1 - lr * wd), rtol=1e-15)
+    assert not m2.any() and not v2.any()
+    # a common positive factor on the whole gradient history leaves the step unchanged up to eps (App. on SGD vs Adam)
+    pa, ma, va = p0.copy(), np.zeros(37), np.zeros(37)
+    pb, mb, vb = p0.copy(), np.zeros(37), np.zeros(37)
+    for t, g in enumerate(grads, start=1):
+        pa, ma, va = update.adamw_step(pa, g, ma, va, t, lr, eps=0.0, weight_decay=0.0)
+        pb, mb, vb = update.adamw_step(pb, 7.5 * g, mb, vb, t, lr, eps=0.0, weight_decay=0.0)
+    np.testing.assert_allclose(pa, pb, rtol=1e-12)
+
+
+def test_head_learning_rate_schedule():
+    peak, total = 3e-4, 200
+    lrs = np.array([update.head_lr(s, peak, total) for s in range(total + 5)])
+    assert lrs[0] == pytest.approx(peak / 10) and lrs[9] == pytest.approx(peak)          # warm-up over 10 steps
+    assert np.all(np.diff(lrs[:10]) > 0) and np.allclose(np.diff(lrs[:10]), peak / 10)
+    assert lrs[10] == pytest.approx(peak) and np.all(np.diff(lrs[10:total + 1]) <= 1e-18)  # then it only decays
+    assert lrs[total] == pytest.approx(peak / 10) and lrs[total + 4] == pytest.approx(peak / 10)   # to a tenth of the peak
+    mid = (10 + total) // 2
+    assert lrs[mid] == pytest.approx(peak * 0.55, rel=1e-9)                               # half-way down the cosine
