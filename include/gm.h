@@ -408,6 +408,18 @@ int gm_head_state_grad(gm_ctx *ctx, int rows, const void *grad_logits, const flo
  * d % 64 != 0, F % 64 != 0 or GM_FLAG_SIMPLE_GEMM: GM_ERR_UNSUPPORTED.                                         */
 int gm_head_ffn_backward(gm_ctx *ctx, int rows, const float *x, const float *dg, float *dx, float *dw_gate_up,
                          float *dw_down, float *dln2, int refresh_weights);
+/* The update of a parameter tensor of the head (Alg. 1, "update phi"; App. B, optimizer and learning rate: AdamW on the
+ * head's own parameter group).  All arrays on the device, n elements:
+ *   master fp32 in/out (the parameters), param_bf16 out or NULL (the bf16 copy the forward pass reads, rewritten from
+ *   the new master values), grad fp32 in, m / v fp32 in/out (first and second moments; zeros before step 1).
+ *   m <- b1 m + (1 - b1) g,  v <- b2 v + (1 - b2) g^2,  p <- p (1 - lr wd) - lr (m / (1 - b1^t)) / (sqrt(v / (1 - b2^t)) + eps)
+ *   with g = grad_scale * grad (1 for no clipping) and t = step >= 1.  The schedule of lr (warm-up over 10 updates,
+ *   cosine decay to a tenth of the peak) is the caller's; the paper gives no moment coefficients, eps or weight decay
+ *   for the head: the optimizer's usual defaults are 0.9, 0.999, 1e-8, 0.01.
+ * One streaming pass (16 bytes read, 12 + 2 written per element).  beta outside [0, 1), negative lr or eps,
+ * non-finite lr or grad_scale: GM_ERR_UNSUPPORTED.                                                             */
+int gm_adamw_step(gm_ctx *ctx, int64_t n, float *master, void *param_bf16, const float *grad, float *m, float *v,
+                  int step, float lr, float beta1, float beta2, float eps, float weight_decay, float grad_scale);
 
 
 /* Dense projection out[M, N] = x[M, K] w[N, K]^T on the context's stream (bf16 in, fp32

@@ -191,4 +191,20 @@ int gm_head_ffn_backward(gm_ctx *c, int rows, const float *x, const float *dg, f
   return run_gemm(c, c->ffn_dabt, 2 * F, &wm, c->ffn_ut, 2 * F, d, Mp, dw_gate_up, EPI_STORE_F32, static_cast<size_t>(d), false);
 }
 
+int gm_adamw_step(gm_ctx *c, int64_t n, float *master, void *param_bf16, const float *grad, float *m, float *v, int step, float lr,
+                  float beta1, float beta2, float eps, float weight_decay, float grad_scale) {
+  if (!c || n < 1 || !master || !grad || !m || !v || step < 1) return GM_ERR_INVALID_ARG;
+  if (!(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(lr >= 0.f) || !(eps >= 0.f) || !std::isfinite(lr) ||
+      !std::isfinite(grad_scale))
+    return GM_ERR_UNSUPPORTED;
+  const double c1 = 1.0 / (1.0 - std::pow(static_cast<double>(beta1), step));
+  const double c2 = 1.0 / (1.0 - std::pow(static_cast<double>(beta2), step));
+  const double decay = 1.0 - static_cast<double>(lr) * static_cast<double>(weight_decay);
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+            launch_adamw(master, static_cast<__nv_bfloat16 *>(param_bf16), grad, m, v, static_cast<size_t>(n), lr, beta1, beta2, eps,
+                         static_cast<float>(decay), static_cast<float>(c1), static_cast<float>(c2), grad_scale, c->sm_count,
+                         c->stream));
+  return GM_OK;
+}
+
 }  // extern "C"

@@ -260,6 +260,10 @@ cudaError_t launch_rmsnorm_grad(const float *gy, const float *x, const __nv_bflo
 cudaError_t launch_transpose_bf16(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst, cudaStream_t stream, int dst_ld = 0);
 // out[j] = sum over rows of t[row][j] (fp32, row order).
 cudaError_t launch_colsum(const float *t, int rows, int d, float *out, cudaStream_t stream);
+// AdamW on n fp32 master parameters with fp32 moments; param (bf16 copy the forward pass reads) or null.  decay = 1 - lr wd,
+// c1 / c2 = the bias corrections 1 / (1 - b^t), gscale multiplies the gradient (clipping).
+cudaError_t launch_adamw(float *master, __nv_bfloat16 *param, const float *grad, float *m, float *v, size_t n, float lr, float b1,
+                         float b2, float eps, float decay, float c1, float c2, float gscale, int sm_count, cudaStream_t stream);
 cudaError_t launch_cast_bf16(const float *src, __nv_bfloat16 *dst, size_t n, cudaStream_t stream);       // n % 4 == 0
 // Backward of h = silu(a) * b on interleaved (a, b) columns: dab bf16 [rows, 2F] (da, db interleaved), h bf16 [rows, F].
 cudaError_t launch_swiglu_grad(const __nv_bfloat16 *ab, const float *dh, __nv_bfloat16 *dab, __nv_bfloat16 *h, int rows, int F,

@@ -362,6 +362,44 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16
     if (c0 + i < cols && r0 + tx < rows) dst[static_cast<size_t>(c0 + i) * dst_ld + r0 + tx] = tile[tx][i];
 }
 
+// ---- AdamW on the head's parameters (Alg. 1, "update phi"; App. B: optimizer and learning rate) ------------------------------
+// Per element: m <- b1 m + (1 - b1) g,  v <- b2 v + (1 - b2) g^2,  p <- p (1 - lr wd) - lr (m c1) / (sqrt(v c2) + eps), with the
+// bias corrections c1 = 1 / (1 - b1^t), c2 = 1 / (1 - b2^t) formed on the host in double.  fp32 master parameters and
+// moments; the bf16 copy the forward pass reads is rewritten in the same pass.  Pure streaming: 16 bytes in, 14 out per element.
+struct AdamwArgs {
+  float *master, *m, *v;
+  const float *grad;
+  __nv_bfloat16 *param;                            // or null
+  size_t n;
+  float lr, b1, b2, eps, decay, c1, c2, gscale;
+};
+__device__ __forceinline__ float adamw_one(float p, float g, float &m, float &v, const AdamwArgs &A) {
+  g *= A.gscale;
+  m = fmaf(A.b1, m, (1.0f - A.b1) * g);
+  v = fmaf(A.b2, v, (1.0f - A.b2) * g * g);
+  return p * A.decay - A.lr * (m * A.c1) / (sqrtf(v * A.c2) + A.eps);
+}
+__global__ void __launch_bounds__(256) adamw_kernel(const AdamwArgs A) {
+  const size_t n4 = A.n >> 2, stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    float4 p = reinterpret_cast<float4 *>(A.master)[i], m = reinterpret_cast<float4 *>(A.m)[i], v = reinterpret_cast<float4 *>(A.v)[i];
+    const float4 g = reinterpret_cast<const float4 *>(A.grad)[i];
+    p.x = adamw_one(p.x, g.x, m.x, v.x, A); p.y = adamw_one(p.y, g.y, m.y, v.y, A);
+    p.z = adamw_one(p.z, g.z, m.z, v.z, A); p.w = adamw_one(p.w, g.w, m.w, v.w, A);
+    reinterpret_cast<float4 *>(A.master)[i] = p;
+    reinterpret_cast<float4 *>(A.m)[i] = m;
+    reinterpret_cast<float4 *>(A.v)[i] = v;
+    if (A.param) reinterpret_cast<uint2 *>(A.param)[i] = make_uint2(pack_bf16(p.x, p.y), pack_bf16(p.z, p.w));
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (A.n & 3)) {                        // the last one to three elements
+    const size_t i = (n4 << 2) + threadIdx.x;
+    float m = A.m[i], v = A.v[i];
+    const float p = adamw_one(A.master[i], A.grad[i], m, v, A);
+    A.master[i] = p; A.m[i] = m; A.v[i] = v;
+    if (A.param) A.param[i] = __float2bfloat16(p);
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_capture_chunk(const __nv_bfloat16 *src, const int32_t *row_n, const int32_t *row_base, int rows, int vr,
@@ -414,6 +452,14 @@ cudaError_t launch_swiglu_grad(const __nv_bfloat16 *ab, const float *dh, __nv_bf
                                cudaStream_t stream) {
   const size_t n = static_cast<size_t>(rows) * F;
   swiglu_grad_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(ab, dh, dab, h, n, F);
+  return cudaGetLastError();
+}
+cudaError_t launch_adamw(float *master, __nv_bfloat16 *param, const float *grad, float *m, float *v, size_t n, float lr, float b1,
+                         float b2, float eps, float decay, float c1, float c2, float gscale, int sm_count, cudaStream_t stream) {
+  AdamwArgs A{master, m, v, grad, param, n, lr, b1, b2, eps, decay, c1, c2, gscale};
+  const size_t want = ((n >> 2) + 255) / 256;
+  const unsigned grid = static_cast<unsigned>(std::max<size_t>(1, std::min<size_t>(want, static_cast<size_t>(sm_count) * 8)));
+  adamw_kernel<<<grid, 256, 0, stream>>>(A);
   return cudaGetLastError();
 }
 

@@ -346,6 +346,57 @@ def test_head_ffn_backward_matches_the_oracle(name, rows):
     ctx.close()
 
 
+@pytest.mark.parametrize("n", [1003, 49_807_360], ids=["ragged_1003", "gate_up_of_the_4b_head"])
+def test_adamw_step_matches_the_oracle(n):
+    """gm_adamw_step over several updates with the head's schedule against the oracle's fp64 AdamW (sampled entries at the
+    size of the 4B head's gate/up matrix, 19456 x 2560), the rewritten bf16 copy, argument checks, and the pass's bandwidth."""
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny")
+    ctx = gmb.Context(cfg, gmb.random_packed_weights(cfg, "cuda"), 4, 3, 4, 8, 8)
+    g = torch.Generator(device="cuda").manual_seed(12)
+    p = torch.randn(n, device="cuda", generator=g) * 0.05
+    m, v = torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
+    pb = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    idx = torch.from_numpy(np.unique(np.concatenate([np.random.default_rng(1).integers(0, n, 4000), [0, n - 1, n - 2, n - 3]]))).cuda()
+    po, mo, vo = (t[idx].double().cpu().numpy() for t in (p, m, v))
+    steps, peak = 4, 3e-4
+    f32 = lambda x: float(np.float32(x))                               # the C ABI takes the coefficients as floats: same values on both sides
+    b1, b2, eps, wd = f32(0.9), f32(0.999), f32(1e-8), f32(0.01)
+    for t in range(1, steps + 1):
+        grad = torch.randn(n, device="cuda", generator=g) * (0.02 * t)
+        grad[::7] = 0                                                  # entries without a gradient still decay
+        lr = f32(oupdate.head_lr(t - 1, peak, 100))
+        scale = 0.5 if t == 3 else 1.0                                 # a clipped update
+        gmb.gm_adamw_step(ctx, p, grad, m, v, t, lr, param_bf16=pb, beta1=b1, beta2=b2, eps=eps, weight_decay=wd, grad_scale=scale)
+        po, mo, vo = oupdate.adamw_step(po, scale * grad[idx].double().cpu().numpy(), mo, vo, t, lr, b1, b2, eps, wd)
+    assert gmb.gm_last_status(ctx) == 0
+    got = p[idx].double().cpu().numpy()
+    # fp32 arithmetic: the parameter to an ulp or two, the accumulated movement (about steps * lr) to 1e-5 of itself
+    np.testing.assert_allclose(got, po, rtol=3e-7, atol=steps * peak * 1e-5)
+    np.testing.assert_allclose(m[idx].double().cpu().numpy(), mo, rtol=1e-5, atol=3e-8)      # gradients of both signs cancel in m
+    np.testing.assert_allclose(v[idx].double().cpu().numpy(), vo, rtol=1e-5, atol=1e-12)
+    assert torch.equal(pb, p.to(torch.bfloat16))
+    for bad in (dict(beta1=1.0), dict(beta2=-0.1), dict(eps=-1.0), dict(lr=float("nan"))):
+        with pytest.raises(gmb.GmError) as e:
+            gmb.gm_adamw_step(ctx, p, grad, m, v, 1, bad.pop("lr", 1e-4), **bad)
+        assert e.value.code == gmb.GM_ERR_UNSUPPORTED
+    with pytest.raises(gmb.GmError) as e:
+        gmb.gm_adamw_step(ctx, p, grad, m, v, 0, 1e-4)
+    assert e.value.code == gmb.GM_ERR_INVALID_ARG
+    if n > 1 << 20:
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        for _ in range(3):
+            gmb.gm_adamw_step(ctx, p, grad, m, v, 5, 1e-4, param_bf16=pb)
+        ev[0].record()
+        for _ in range(10):
+            gmb.gm_adamw_step(ctx, p, grad, m, v, 5, 1e-4, param_bf16=pb)
+        ev[1].record()
+        torch.cuda.synchronize()
+        ms = ev[0].elapsed_time(ev[1]) / 10
+        print(f"gm_adamw_step n {n}: {ms:.3f} ms per call, {30.0 * n / ms / 1e6:.0f} GB/s (16 bytes read, 14 written per element)")
+    ctx.close()
+
+
 def test_loss_kernel_edge_cases():
     import paper_2609_16648_b200 as gmb
     cfg = get_config("tiny")
