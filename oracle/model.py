@@ -183,9 +183,9 @@ def target_logits(w, hidden, cfg) -> np.ndarray:
     return rmsnorm(hidden, w["final_norm"], cfg.rms_eps) @ f64(w["lm_head"]).T
 
 
-def head_forward(w, hidden, tokens, pos, hkv: PagedKV, b: int, cfg) -> np.ndarray:
-    """Draft head over pairs (hidden_i, token_i) at positions pos; returns g [T, d], the
-    head layer's residual output (its recurrent state).
+def head_input(w, hidden, tokens, cfg) -> np.ndarray:
+    """Input of the head's layer for pairs (hidden_i, token_i) (App. B.1): the token embedding and the hidden state, each
+    through its own RMSNorm, concatenated and projected from 2d to d by a bias-free matrix.
 
     The two normalised inputs are concatenated [embedding ; hidden]; a head whose
     "concat" entry is "hidden_first" takes them in the opposite order (App. B.1: one
@@ -196,8 +196,13 @@ def head_forward(w, hidden, tokens, pos, hkv: PagedKV, b: int, cfg) -> np.ndarra
     if hw.get("concat", "embedding_first") == "hidden_first":
         parts.reverse()
     z = np.concatenate(parts, axis=-1)
-    z = z @ f64(hw["proj"]).T
-    return decoder_layer(hw["layer"], z, pos, hkv, 0, b, cfg)
+    return z @ f64(hw["proj"]).T
+
+
+def head_forward(w, hidden, tokens, pos, hkv: PagedKV, b: int, cfg) -> np.ndarray:
+    """Draft head over pairs (hidden_i, token_i) at positions pos; returns g [T, d], the
+    head layer's residual output (its recurrent state)."""
+    return decoder_layer(w["head"]["layer"], head_input(w, hidden, tokens, cfg), pos, hkv, 0, b, cfg)
 
 
 def head_logits(w, g, cfg) -> np.ndarray:

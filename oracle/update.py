@@ -29,6 +29,10 @@ backbone's shape), g = x + W_d (silu(W_g u) * (W_u u)) with u = RMSNorm(x; ln2).
 residual path plus the path through the block) and the gradients of the block's four parameter tensors, which are the
 first of the head's own weights the update step touches (Alg. 1, "update phi").
 
+Fourth step: through the head's input (App. B.1), z = W_p [RMSNorm_e(E[token]) ; RMSNorm_h(hidden)].  Given dL/dz it returns
+the gradients of the projection and of the two norm weights (the embedding table is the backbone's: no gradient), and
+dL/d(hidden) - which, for a draft application k >= 2, is a further term of dL/dg_{k-1}: the recurrence of Eq. 4.
+
 The update itself: AdamW on the head's parameter group, with the head's learning-rate schedule (App. B, optimizer and
 learning rate: linear warm-up over 10 steps, then a cosine decay to a tenth of the peak).  The paper names the
 optimizer and the rates only; the moment coefficients, the stabilising constant and the weight decay are the defaults
@@ -39,7 +43,7 @@ from __future__ import annotations
 import numpy as np
 
 from . import record, sampler
-from .model import PagedKV, f64, head_forward, head_logits, round_bf16
+from .model import PagedKV, f64, head_forward, head_logits, rmsnorm, round_bf16
 
 
 def reconstruct_states(w, cfg, seq_hidden, seq_tokens, start_len: int, drafts) -> np.ndarray:
@@ -215,6 +219,25 @@ def ffn_block_grad(dg, x, lw, eps: float) -> dict:
     dx = dg + rmsnorm_grad(du, x, w2, eps)
     dln2 = (du * x * r).sum(axis=0)
     return {"dx": dx, "dln2": dln2, "dwg": dwg, "dwu": dwu, "dwd": dwd}
+
+
+def head_input_grad(dz, w, hidden, tokens, cfg) -> dict:
+    """Backward of model.head_input.  dz [T, d] = dL/dz; hidden [T, d], tokens [T] = the pairs that entered.
+    Returns {"dhidden" [T, d], "dproj" [d, 2d] (columns in the order the head concatenates), "denorm" [d], "dhnorm" [d]}."""
+    hw = w["head"]
+    dz, hidden = f64(dz), f64(hidden)
+    d = hidden.shape[-1]
+    e = f64(w["embed"])[np.asarray(tokens)]
+    en, hn = rmsnorm(e, hw["enorm"], cfg.rms_eps), rmsnorm(hidden, hw["hnorm"], cfg.rms_eps)
+    hidden_first = hw.get("concat", "embedding_first") == "hidden_first"
+    zin = np.concatenate([hn, en] if hidden_first else [en, hn], axis=-1)
+    dzin = dz @ f64(hw["proj"])
+    dproj = dz.T @ zin
+    dhn, den = (dzin[:, :d], dzin[:, d:]) if hidden_first else (dzin[:, d:], dzin[:, :d])
+    r_e = 1.0 / np.sqrt((e * e).mean(axis=-1, keepdims=True) + cfg.rms_eps)
+    r_h = 1.0 / np.sqrt((hidden * hidden).mean(axis=-1, keepdims=True) + cfg.rms_eps)
+    return {"dhidden": rmsnorm_grad(dhn, hidden, hw["hnorm"], cfg.rms_eps), "dproj": dproj,
+            "denorm": (den * e * r_e).sum(axis=0), "dhnorm": (dhn * hidden * r_h).sum(axis=0)}
 
 
 def adamw_step(p, g, m, v, step: int, lr: float, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,

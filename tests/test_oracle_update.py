@@ -300,3 +300,38 @@ def test_head_learning_rate_schedule():
     assert lrs[total] == pytest.approx(peak / 10) and lrs[total + 4] == pytest.approx(peak / 10)   # to a tenth of the peak
     mid = (10 + total) // 2
     assert lrs[mid] == pytest.approx(peak * 0.55, rel=1e-9)                               # half-way down the cosine
+
+
+@pytest.mark.parametrize("concat", ["embedding_first", "hidden_first"])
+def test_head_input_gradient_matches_finite_differences(concat):
+    """L = sum(C * head_input(hidden, tokens)): every coordinate of the hidden states, every entry of the projection and of
+    the two norm weights, against central differences of the function head_forward itself calls; both concatenation orders."""
+    rng = np.random.default_rng(31)
+    T_, d, V = 4, 5, 9
+    cfg = CFG.with_(d_model=d, vocab=V, rms_eps=1e-3)
+    w = {"embed": rng.normal(0, 1, (V, d)),
+         "head": {"enorm": rng.uniform(0.6, 1.4, d), "hnorm": rng.uniform(0.6, 1.4, d), "proj": rng.normal(0, 0.6, (d, 2 * d)),
+                  "concat": concat}}
+    hidden, tokens, C = rng.normal(0, 1.3, (T_, d)), np.array([3, 0, 8, 3]), rng.normal(0, 1, (T_, d))
+    g = update.head_input_grad(C, w, hidden, tokens, cfg)
+    L = lambda: float((model.head_input(w, hidden, tokens, cfg) * C).sum())
+
+    def fd(arr):
+        out = np.zeros(arr.shape)
+        for i in np.ndindex(*arr.shape):
+            v = arr[i]
+            arr[i] = v + 1e-6; hi = L()
+            arr[i] = v - 1e-6; lo = L()
+            arr[i] = v
+            out[i] = (hi - lo) / 2e-6
+        return out
+
+    np.testing.assert_allclose(g["dhidden"], fd(hidden), rtol=2e-6, atol=1e-8)
+    np.testing.assert_allclose(g["dproj"], fd(w["head"]["proj"]), rtol=2e-6, atol=1e-8)
+    np.testing.assert_allclose(g["denorm"], fd(w["head"]["enorm"]), rtol=2e-6, atol=1e-8)
+    np.testing.assert_allclose(g["dhnorm"], fd(w["head"]["hnorm"]), rtol=2e-6, atol=1e-8)
+    # the embedding half of the projection sees the token, the hidden half does not: swapping two tokens' rows of C and of
+    # the embedding-side inputs only permutes contributions - checked through the column halves of dproj
+    half = slice(d, 2 * d) if concat == "hidden_first" else slice(0, d)
+    e_n = model.rmsnorm(w["embed"][tokens], w["head"]["enorm"], cfg.rms_eps)
+    np.testing.assert_allclose(g["dproj"][:, half], C.T @ e_n, rtol=1e-12)
