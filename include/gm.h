@@ -408,6 +408,20 @@ int gm_head_state_grad(gm_ctx *ctx, int rows, const void *grad_logits, const flo
  * d % 64 != 0, F % 64 != 0 or GM_FLAG_SIMPLE_GEMM: GM_ERR_UNSUPPORTED.                                         */
 int gm_head_ffn_backward(gm_ctx *ctx, int rows, const float *x, const float *dg, float *dx, float *dw_gate_up,
                          float *dw_down, float *dln2, int refresh_weights);
+/* Fourth step of the backward pass: through the head's input (App. B.1),
+ *   z = W_p [RMSNorm(E[token]; enorm) ; RMSNorm(hidden; hnorm)]   (the order the packed projection uses).
+ *   tokens int32 [rows], hidden fp32 [rows, d]: the pairs that entered;  dz fp32 [rows, d] = dL/dz (device)
+ *   dhidden fp32 [rows, d] out: dL/d hidden - for a draft application k >= 2 the hidden state is the head's own previous
+ *            output g_{k-1} (Eq. 4), so this is a further term of dL/dg_{k-1}; for the first application it is the
+ *            target's hidden state and is dropped
+ *   dproj fp32 [d, 2 d], denorm fp32 [d], dhnorm fp32 [d] out: the gradients of the projection and of the two norm
+ *            weights, summed over the rows (the embedding table is the backbone's: no gradient)
+ * Same conventions as gm_head_ffn_backward: the input rows are recomputed in bf16 as the forward pass computes them, the
+ * two products run on the projection kernel over a transposed copy of W_p and transposed operands, scratch is
+ * allocated on first use.  d % 64 != 0 or GM_FLAG_SIMPLE_GEMM: GM_ERR_UNSUPPORTED; a token id outside the vocabulary
+ * is reported by gm_last_status as GM_ERR_BAD_PAGE (like every out-of-range id) and is treated as token 0.      */
+int gm_head_input_backward(gm_ctx *ctx, int rows, const int32_t *tokens, const float *hidden, const float *dz,
+                           float *dhidden, float *dproj, float *denorm, float *dhnorm, int refresh_weights);
 /* The update of a parameter tensor of the head (Alg. 1, "update phi"; App. B, optimizer and learning rate: AdamW on the
  * head's own parameter group).  All arrays on the device, n elements:
  *   master fp32 in/out (the parameters), param_bf16 out or NULL (the bf16 copy the forward pass reads, rewritten from

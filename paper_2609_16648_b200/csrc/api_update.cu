@@ -207,4 +207,57 @@ int gm_adamw_step(gm_ctx *c, int64_t n, float *master, void *param_bf16, const f
   return GM_OK;
 }
 
+int gm_head_input_backward(gm_ctx *c, int rows, const int32_t *tokens, const float *hidden, const float *dz, float *dhidden,
+                           float *dproj, float *denorm, float *dhnorm, int refresh_weights) {
+  if (!c || rows < 1 || !tokens || !hidden || !dz || !dhidden || !dproj || !denorm || !dhnorm) return GM_ERR_INVALID_ARG;
+  const int d = c->d;
+  if ((c->cfg.flags & GM_FLAG_SIMPLE_GEMM) || (d % 64)) return GM_ERR_UNSUPPORTED;
+  const __nv_bfloat16 *proj = static_cast<const __nv_bfloat16 *>(c->w.head_proj);
+  const __nv_bfloat16 *we = static_cast<const __nv_bfloat16 *>(c->w.head_enorm), *wh = static_cast<const __nv_bfloat16 *>(c->w.head_hnorm);
+  int rc;
+  if (!c->hin_proj_t) {
+    if ((rc = dev_alloc(c, &c->hin_proj_t, static_cast<size_t>(2) * d * d, false)) != GM_OK) return rc;
+    if (make_map(c, &c->hin_proj_t_map, c->hin_proj_t, 2 * d, d, 128) != GM_OK) return GM_ERR_CUDA;
+    refresh_weights = 1;
+  }
+  if (refresh_weights)
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(proj, d, 2 * d, c->hin_proj_t, c->stream));     // [d, 2d] -> [2d, d]
+  const int Mp = (rows + 63) / 64 * 64;
+  if (Mp > c->hin_rows_cap) {
+    const size_t M = static_cast<size_t>(Mp);
+    if ((rc = dev_alloc(c, &c->hin_zin, M * 2 * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hin_dz, M * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hin_zint, M * 2 * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hin_dzt, M * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hin_e, M * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hin_dzin, M * 2 * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hin_t, M * d)) != GM_OK) return rc;
+    c->hin_rows_cap = Mp;
+  }
+  // the forward's input rows, recomputed: [RMSNorm(E[token]) ; RMSNorm(hidden)] in bf16, and the embedding rows in fp32
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+            launch_head_input_rows(static_cast<const __nv_bfloat16 *>(c->w.embed), tokens, hidden, we, wh, rows, d, c->V, c->cfg.rms_eps,
+                                   c->hin_zin, c->hin_e, c->status, c->stream));
+  // d zin = dz W_p
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_cast_bf16(dz, c->hin_dz, static_cast<size_t>(rows) * d, c->stream));
+  if ((rc = run_gemm(c, c->hin_dz, rows, &c->hin_proj_t_map, c->hin_proj_t, rows, 2 * d, d, c->hin_dzin, EPI_STORE_F32, 2 * static_cast<size_t>(d),
+                     false)) != GM_OK)
+    return rc;
+  // through the two norms: the hidden half gives dL/d hidden and dL/d hnorm, the embedding half only dL/d enorm
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+            launch_rmsnorm_grad(c->hin_dzin + d, hidden, wh, dhidden, rows, d, c->cfg.rms_eps, c->stream, nullptr, c->hin_t, 2 * d));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hin_t, rows, d, dhnorm, c->stream));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+            launch_rmsnorm_grad(c->hin_dzin, c->hin_e, we, nullptr, rows, d, c->cfg.rms_eps, c->stream, nullptr, c->hin_t, 2 * d));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hin_t, rows, d, denorm, c->stream));
+  // dW_p [d, 2d] = dz^T zin: both operands transposed to [features, rows] (rows padded with zeros to Mp)
+  GM_CUDA(c, cudaMemsetAsync(c->hin_dzt, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
+  GM_CUDA(c, cudaMemsetAsync(c->hin_zint, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * 2 * d, c->stream));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->hin_dz, rows, d, c->hin_dzt, c->stream, Mp));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->hin_zin, rows, 2 * d, c->hin_zint, c->stream, Mp));
+  CUtensorMap wm;
+  if (make_map(c, &wm, c->hin_zint, 2 * d, Mp, 128) != GM_OK) return GM_ERR_CUDA;
+  return run_gemm(c, c->hin_dzt, d, &wm, c->hin_zint, d, 2 * d, Mp, dproj, EPI_STORE_F32, 2 * static_cast<size_t>(d), false);
+}
+
 }  // extern "C"

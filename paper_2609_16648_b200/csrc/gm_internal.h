@@ -113,6 +113,12 @@ struct gm_ctx {
   __nv_bfloat16 *ffn_u = nullptr, *ffn_ab = nullptr, *ffn_dy = nullptr, *ffn_dab = nullptr, *ffn_h = nullptr;
   __nv_bfloat16 *ffn_ut = nullptr, *ffn_dyt = nullptr, *ffn_dabt = nullptr, *ffn_ht = nullptr;
   float *ffn_dh = nullptr, *ffn_du = nullptr, *ffn_t = nullptr;
+  // ... and through the head's input projection
+  __nv_bfloat16 *hin_proj_t = nullptr;      // [2d, d]
+  CUtensorMap hin_proj_t_map;
+  int hin_rows_cap = 0;
+  __nv_bfloat16 *hin_zin = nullptr, *hin_dz = nullptr, *hin_zint = nullptr, *hin_dzt = nullptr;
+  float *hin_e = nullptr, *hin_dzin = nullptr, *hin_t = nullptr;
   __nv_bfloat16 *lm_head_t = nullptr;       // [d, V]: the LM head transposed, the weight operand of the gradient GEMM
   CUtensorMap lm_head_t_map;
   float top_p = 1.f;                    // nucleus of the target distributions (1 = none)

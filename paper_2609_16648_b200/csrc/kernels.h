@@ -255,7 +255,12 @@ cudaError_t launch_dca_loss(const float *alpha, const int32_t *accepted, int n, 
 //   res (or null): added to gx (the gradient that reaches x past the norm, e.g. along a residual connection);
 //   wterm (or null): fp32 [rows, d], gy x r per row - the rows' terms of dL/dw.
 cudaError_t launch_rmsnorm_grad(const float *gy, const float *x, const __nv_bfloat16 *w, float *gx, int rows, int d, float eps,
-                                cudaStream_t stream, const float *res = nullptr, float *wterm = nullptr);
+                                cudaStream_t stream, const float *res = nullptr, float *wterm = nullptr, int gy_ld = 0);
+// (gx may be null when only wterm is wanted; gy_ld: row stride of gy when it is a column block of a wider matrix, 0 = d)
+// zin bf16 [rows, 2d] = [RMSNorm(embed[tokens]; we) ; RMSNorm(hidden; wh)], e_out fp32 [rows, d] = the embedding rows.
+cudaError_t launch_head_input_rows(const __nv_bfloat16 *embed, const int32_t *tokens, const float *hidden, const __nv_bfloat16 *we,
+                                   const __nv_bfloat16 *wh, int rows, int d, int vocab, float eps, __nv_bfloat16 *zin, float *e_out,
+                                   uint32_t *status, cudaStream_t stream);
 // dst [cols, dst_ld] = transpose of src [rows, cols] (bf16, both row-major; dst_ld >= rows, 0 = rows; padding untouched).
 cudaError_t launch_transpose_bf16(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst, cudaStream_t stream, int dst_ld = 0);
 // out[j] = sum over rows of t[row][j] (fp32, row order).

@@ -292,9 +292,10 @@ capture_cycle_kernel(const __nv_bfloat16 *src, const int32_t *accept_len, const 
 constexpr int NG_THREADS = 256;
 __global__ void __launch_bounds__(NG_THREADS)
 rmsnorm_grad_kernel(const float *gy, const float *x, const __nv_bfloat16 *w, float *gx, int d, float eps, const float *res,
-                    float *wterm) {
+                    float *wterm, int gy_ld) {
   __shared__ float red[2][NG_THREADS / 32];
   const size_t row = static_cast<size_t>(blockIdx.x) * d;
+  gy += static_cast<size_t>(blockIdx.x) * gy_ld - row;        // gy rows may be wider than d (a column block of a larger matrix)
   const int tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
   pdl_prologue();
   float sq = 0.f, dot = 0.f;
@@ -314,7 +315,7 @@ rmsnorm_grad_kernel(const float *gy, const float *x, const __nv_bfloat16 *w, flo
   const float c = r * r * r * dot * inv_d;
   for (int i = tid; i < d; i += NG_THREADS) {
     const float g = gy[row + i], xv = x[row + i];
-    gx[row + i] = (res ? res[row + i] : 0.f) + (r * bf16_to_float(w[i]) * g - xv * c);     // res: the residual path's gradient
+    if (gx) gx[row + i] = (res ? res[row + i] : 0.f) + (r * bf16_to_float(w[i]) * g - xv * c);     // res: the residual path's gradient
     if (wterm) wterm[row + i] = g * xv * r;                    // this row's term of dL/dw (summed over the rows afterwards)
   }
 }
@@ -400,6 +401,38 @@ __global__ void __launch_bounds__(256) adamw_kernel(const AdamwArgs A) {
   }
 }
 
+// The head's input rows for given (token, hidden) pairs (App. B.1): zin[row] = [RMSNorm(E[token]; we) ; RMSNorm(hidden; wh)]
+// in bf16, and the embedding row itself in fp32 (the norm's backward needs it).  One CTA per row.
+__global__ void __launch_bounds__(NG_THREADS)
+head_input_rows_kernel(const __nv_bfloat16 *embed, const int32_t *tokens, const float *hidden, const __nv_bfloat16 *we,
+                       const __nv_bfloat16 *wh, int d, int vocab, float eps, __nv_bfloat16 *zin, float *e_out, uint32_t *status) {
+  __shared__ float red[2][NG_THREADS / 32];
+  const int m = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
+  pdl_prologue();
+  int tok = tokens[m];
+  if (tok < 0 || tok >= vocab) { if (tid == 0) set_status(status, ST_BAD_TOKEN); tok = 0; }
+  const __nv_bfloat16 *er = embed + static_cast<size_t>(tok) * d;
+  const float *hr = hidden + static_cast<size_t>(m) * d;
+  float se = 0.f, sh = 0.f;
+  for (int i = tid; i < d; i += NG_THREADS) {
+    const float e = bf16_to_float(er[i]), h = hr[i];
+    e_out[static_cast<size_t>(m) * d + i] = e;
+    se = fmaf(e, e, se); sh = fmaf(h, h, sh);
+  }
+  se = warp_sum(se); sh = warp_sum(sh);
+  if (lane == 0) { red[0][wp] = se; red[1][wp] = sh; }
+  __syncthreads();
+  se = 0.f; sh = 0.f;
+#pragma unroll
+  for (int i = 0; i < NG_THREADS / 32; ++i) { se += red[0][i]; sh += red[1][i]; }
+  const float re = rsqrtf(se / static_cast<float>(d) + eps), rh = rsqrtf(sh / static_cast<float>(d) + eps);
+  __nv_bfloat16 *out = zin + static_cast<size_t>(m) * 2 * d;
+  for (int i = tid; i < d; i += NG_THREADS) {
+    out[i] = __float2bfloat16(bf16_to_float(er[i]) * re * bf16_to_float(we[i]));
+    out[d + i] = __float2bfloat16(hr[i] * rh * bf16_to_float(wh[i]));
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_capture_chunk(const __nv_bfloat16 *src, const int32_t *row_n, const int32_t *row_base, int rows, int vr,
@@ -433,12 +466,19 @@ cudaError_t launch_dca_loss(const float *alpha, const int32_t *accepted, int n, 
   return launch_k(dca_loss_kernel, dim3(1), dim3(DL_THREADS), 0, stream, 1, alpha, accepted, n, K, loss, mean);
 }
 cudaError_t launch_rmsnorm_grad(const float *gy, const float *x, const __nv_bfloat16 *w, float *gx, int rows, int d, float eps,
-                                cudaStream_t stream, const float *res, float *wterm) {
-  return launch_k(rmsnorm_grad_kernel, dim3(rows), dim3(NG_THREADS), 0, stream, 1, gy, x, w, gx, d, eps, res, wterm);
+                                cudaStream_t stream, const float *res, float *wterm, int gy_ld) {
+  return launch_k(rmsnorm_grad_kernel, dim3(rows), dim3(NG_THREADS), 0, stream, 1, gy, x, w, gx, d, eps, res, wterm,
+                  gy_ld > 0 ? gy_ld : d);
 }
 cudaError_t launch_transpose_bf16(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst, cudaStream_t stream, int dst_ld) {
   transpose_bf16_kernel<<<dim3((cols + 63) / 64, (rows + 63) / 64), 256, 0, stream>>>(src, rows, cols, dst, dst_ld > 0 ? dst_ld : rows);
   return cudaGetLastError();
+}
+cudaError_t launch_head_input_rows(const __nv_bfloat16 *embed, const int32_t *tokens, const float *hidden, const __nv_bfloat16 *we,
+                                   const __nv_bfloat16 *wh, int rows, int d, int vocab, float eps, __nv_bfloat16 *zin, float *e_out,
+                                   uint32_t *status, cudaStream_t stream) {
+  return launch_k(head_input_rows_kernel, dim3(rows), dim3(NG_THREADS), 0, stream, 1, embed, tokens, hidden, we, wh, d, vocab, eps, zin,
+                  e_out, status);
 }
 cudaError_t launch_colsum(const float *t, int rows, int d, float *out, cudaStream_t stream) {
   colsum_kernel<<<(d + 255) / 256, 256, 0, stream>>>(t, rows, d, out);

@@ -346,6 +346,53 @@ def test_head_ffn_backward_matches_the_oracle(name, rows):
     ctx.close()
 
 
+@pytest.mark.parametrize("name,rows,concat", [("tiny", 40, None), ("tiny", 40, "hidden_first"), ("4b", 192, None)],
+                         ids=["tiny-40", "tiny-40-hidden_first", "4b-192"])
+def test_head_input_backward_matches_the_oracle(name, rows, concat):
+    """gm_head_input_backward against the oracle's fp64 backward of the head's input on the same bf16 weights: the hidden
+    states' gradient (the recurrence term), the projection's and the two norm weights' gradients; both concatenation
+    orders (the packed projection always takes [embedding ; hidden], so dproj comes back with its column halves swapped)."""
+    import paper_2609_16648_b200 as gmb
+    base = get_config("tiny")
+    cfg = base if name == "tiny" else base.with_(d_model=2560, vocab=4096)
+    d, V = cfg.d_model, cfg.vocab
+    w = perturb_norm_weights(make_weights(cfg, 3))
+    w["head"]["proj"] = np.random.default_rng(4).normal(0, 1.0 / np.sqrt(2 * d), (d, 2 * d)).astype(np.float32)
+    if concat:
+        w["head"]["concat"] = concat
+    packed = gmb.pack_weights(w)
+    ctx = gmb.Context(cfg, packed, 4, 3, 4, 8, 8)
+    rng = np.random.default_rng(6)
+    tokens = rng.integers(0, V, rows).astype(np.int32)
+    hidden = rng.normal(0, 1.5, (rows, d)).astype(np.float32)
+    dz = rng.normal(0, 0.1, (rows, d)).astype(np.float32)
+    dz[2::5] = 0
+    z = lambda *shape: torch.full(shape, 7.0, dtype=torch.float32, device="cuda")
+    dh, dp, de, dhn = z(rows, d), z(d, 2 * d), z(d), z(d)
+    cu = lambda a: torch.from_numpy(a).cuda()
+    gmb.gm_head_input_backward(ctx, rows, cu(tokens), cu(hidden), cu(dz), dh, dp, de, dhn)
+    assert gmb.gm_last_status(ctx) == 0
+    r16 = lambda a: omodel.round_bf16(a).astype(np.float64)           # the oracle on the weights the device holds
+    wo = {"embed": r16(w["embed"]), "head": {"enorm": r16(w["head"]["enorm"]), "hnorm": r16(w["head"]["hnorm"]),
+                                             "proj": r16(w["head"]["proj"]), "concat": concat or "embedding_first"}}
+    want = oupdate.head_input_grad(dz, wo, hidden, tokens, cfg)
+    f = lambda t: t.double().cpu().numpy()
+    tol = 2.5e-2
+    assert rel_err(f(dh), want["dhidden"]) < tol and (f(dh)[2::5] == 0).all()
+    want_dp = want["dproj"]
+    if concat == "hidden_first":                                        # packed order is always [embedding ; hidden]
+        want_dp = np.concatenate([want_dp[:, d:], want_dp[:, :d]], axis=1)
+    assert rel_err(f(dp), want_dp) < tol
+    assert rel_err(f(de), want["denorm"]) < tol and rel_err(f(dhn), want["dhnorm"]) < tol
+    assert np.abs(want["denorm"]).max() > 0 and np.abs(want["dproj"]).max() > 0
+    # a token id outside the vocabulary is reported, not dereferenced
+    bad = cu(tokens.copy())
+    bad[1] = V + 5
+    gmb.gm_head_input_backward(ctx, rows, bad, cu(hidden), cu(dz), dh, dp, de, dhn)
+    assert gmb.gm_last_status(ctx) == gmb.GM_ERR_BAD_PAGE
+    ctx.close()
+
+
 @pytest.mark.parametrize("n", [1003, 49_807_360], ids=["ragged_1003", "gate_up_of_the_4b_head"])
 def test_adamw_step_matches_the_oracle(n):
     """gm_adamw_step over several updates with the head's schedule against the oracle's fp64 AdamW (sampled entries at the
