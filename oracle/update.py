@@ -29,6 +29,10 @@ backbone's shape), g = x + W_d (silu(W_g u) * (W_u u)) with u = RMSNorm(x; ln2).
 residual path plus the path through the block) and the gradients of the block's four parameter tensors, which are the
 first of the head's own weights the update step touches (Alg. 1, "update phi").
 
+The attention core of the head's layer (scores, softmax, weighted values) has its backward as an operator of its own:
+gradients with respect to the queries and to every cached key and value, whichever pass wrote them (the committed
+prefix is shared by all chains of a sequence, so its entries collect terms from all of them).
+
 Fourth step: through the head's input (App. B.1), z = W_p [RMSNorm_e(E[token]) ; RMSNorm_h(hidden)].  Given dL/dz it returns
 the gradients of the projection and of the two norm weights (the embedding table is the backbone's: no gradient), and
 dL/d(hidden) - which, for a draft application k >= 2, is a further term of dL/dg_{k-1}: the recurrence of Eq. 4.
@@ -219,6 +223,30 @@ def ffn_block_grad(dg, x, lw, eps: float) -> dict:
     dx = dg + rmsnorm_grad(du, x, w2, eps)
     dln2 = (du * x * r).sum(axis=0)
     return {"dx": dx, "dln2": dln2, "dwg": dwg, "dwu": dwu, "dwd": dwd}
+
+
+def attention_grad(dout, q, k, v, q_pos, k_pos):
+    """Backward of model.attention (causal grouped-query attention with an explicit softmax).  dout, q [T, n_q, hd];
+    k, v [S, n_kv, hd].  Per head, with P = softmax(S), S = q k^T / sqrt(hd) on the visible keys:
+        dP = dout v^T,  dS = P * (dP - rowsum(dP * P)),  dq = dS k / sqrt(hd),  dk += dS^T q / sqrt(hd),  dv += P^T dout
+    (keys and values of a KV head collect the terms of every query head of their group).  Returns (dq, dk, dv), float64."""
+    dout, q, k, v = f64(dout), f64(q), f64(k), f64(v)
+    T, n_q, hd = q.shape
+    g = n_q // k.shape[1]
+    visible = np.asarray(k_pos)[None, :] <= np.asarray(q_pos)[:, None]
+    dq, dk, dv = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v)
+    scale = 1.0 / np.sqrt(hd)
+    for h in range(n_q):
+        kh, vh = k[:, h // g, :], v[:, h // g, :]
+        sc = np.where(visible, q[:, h, :] @ kh.T * scale, -np.inf)
+        e = np.exp(sc - sc.max(axis=1, keepdims=True))
+        pr = e / e.sum(axis=1, keepdims=True)
+        dpr = dout[:, h, :] @ vh.T
+        ds = pr * (dpr - (dpr * pr).sum(axis=1, keepdims=True))
+        dq[:, h, :] = ds @ kh * scale
+        dk[:, h // g, :] += ds.T @ q[:, h, :] * scale
+        dv[:, h // g, :] += pr.T @ dout[:, h, :]
+    return dq, dk, dv
 
 
 def head_input_grad(dz, w, hidden, tokens, cfg) -> dict:

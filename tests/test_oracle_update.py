@@ -335,3 +335,35 @@ def test_head_input_gradient_matches_finite_differences(concat):
     half = slice(d, 2 * d) if concat == "hidden_first" else slice(0, d)
     e_n = model.rmsnorm(w["embed"][tokens], w["head"]["enorm"], cfg.rms_eps)
     np.testing.assert_allclose(g["dproj"][:, half], C.T @ e_n, rtol=1e-12)
+
+
+def test_attention_gradient_matches_finite_differences():
+    """L = sum(C * attention(q, k, v)) with a ragged causal mask (queries in the middle of the key range, a key nobody sees):
+    every coordinate of q, k and v against central differences of the forward the decoder layer calls."""
+    rng = np.random.default_rng(41)
+    T_, S, n_q, n_kv, hd = 3, 7, 4, 2, 6
+    q, k, v = rng.normal(0, 1, (T_, n_q, hd)), rng.normal(0, 1, (S, n_kv, hd)), rng.normal(0, 1, (S, n_kv, hd))
+    q_pos, k_pos = np.array([2, 4, 5]), np.array([0, 1, 2, 3, 4, 5, 9])          # key 6 (position 9) is visible to nobody
+    C = rng.normal(0, 1, (T_, n_q, hd))
+    dq, dk, dv = update.attention_grad(C, q, k, v, q_pos, k_pos)
+    L = lambda: float((model.attention(q, k, v, q_pos, k_pos) * C).sum())
+
+    def fd(arr):
+        out = np.zeros(arr.shape)
+        for i in np.ndindex(*arr.shape):
+            x = arr[i]
+            arr[i] = x + 1e-6; hi = L()
+            arr[i] = x - 1e-6; lo = L()
+            arr[i] = x
+            out[i] = (hi - lo) / 2e-6
+        return out
+
+    np.testing.assert_allclose(dq, fd(q), rtol=2e-6, atol=1e-8)
+    np.testing.assert_allclose(dk, fd(k), rtol=2e-6, atol=1e-8)
+    np.testing.assert_allclose(dv, fd(v), rtol=2e-6, atol=1e-8)
+    assert not dk[6].any() and not dv[6].any()                       # the invisible key gets nothing
+    # a row's score gradients sum to zero over its keys (softmax ignores a common shift), and dk_j = dS_j q / sqrt(hd):
+    # the key gradients of a KV head sum to zero over the keys
+    assert np.abs(dk.sum(axis=0)).max() < 1e-12
+    # values enter linearly: dv is the attention-weighted sum of the output gradients, so it sums to the sum of dout per group
+    np.testing.assert_allclose(dv.sum(axis=0), C.reshape(T_, n_kv, n_q // n_kv, hd).sum(axis=(0, 2)), rtol=1e-12)
