@@ -408,6 +408,23 @@ int gm_head_state_grad(gm_ctx *ctx, int rows, const void *grad_logits, const flo
  * d % 64 != 0, F % 64 != 0 or GM_FLAG_SIMPLE_GEMM: GM_ERR_UNSUPPORTED.                                         */
 int gm_head_ffn_backward(gm_ctx *ctx, int rows, const float *x, const float *dg, float *dx, float *dw_gate_up,
                          float *dw_down, float *dln2, int refresh_weights);
+/* Backward of gm_attention's core (scores, softmax, weighted values) - the operator the attention half of the head's
+ * layer needs in the update (Alg. 1, "update phi").  Same query layout, pool, page tables and row conventions as
+ * gm_attention; for every valid query row (j < q_count[b]) with output gradient dO and P = softmax(q k^T / sqrt(hd)):
+ *   dP_j = dO . v_j,  dS_j = P_j (dP_j - sum_i P_i dP_i),  dq = sum_j dS_j k_j / sqrt(hd),
+ *   dk_j += dS_j q / sqrt(hd),  dv_j += P_j dO      (a KV head collects the terms of every query head of its group)
+ *   dout     device fp32 [batch * q_stride][n_q * head_dim]: gradient of gm_attention's `out` rows
+ *   dq       device fp32 [batch * q_stride][n_q * head_dim] out (rows j >= q_count[b] are zero); with respect to the
+ *            queries as gm_attention receives them (rotary embedding already applied)
+ *   dk_pool, dv_pool  device fp32 [num_pages][n_kv][16][head_dim]: gradient planes laid out like one layer of the pool,
+ *            ACCUMULATED with atomic additions (the caller zeroes them): sequences whose page tables share pages - the
+ *            chains of one sequence share its committed prefix - add into the same entries; with respect to the cached
+ *            keys (after their rotary embedding) and values, whichever pass wrote them
+ * Reads the cache in bf16, computes in fp32; two passes over a row's keys (statistics, then gradients).
+ * q_stride > 8, more than 8 query heads per KV head, head_dim other than 64 / 128: GM_ERR_UNSUPPORTED.           */
+int gm_attention_backward(gm_ctx *ctx, const void *q, const float *dout, const void *kv_pool, int pool_layers,
+                          int num_pages, int layer, const int32_t *page_table, const int32_t *q_count,
+                          const int32_t *q_base, int batch, int q_stride, float *dq, float *dk_pool, float *dv_pool);
 /* Fourth step of the backward pass: through the head's input (App. B.1),
  *   z = W_p [RMSNorm(E[token]; enorm) ; RMSNorm(hidden; hnorm)]   (the order the packed projection uses).
  *   tokens int32 [rows], hidden fp32 [rows, d]: the pairs that entered;  dz fp32 [rows, d] = dL/dz (device)

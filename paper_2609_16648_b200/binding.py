@@ -24,7 +24,7 @@ GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER, GM_KC_RECORD = 0,
 
 EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw", "gm_set_top_p", "gm_nucleus", "gm_prefill",
            "gm_rollout_begin", "gm_rollout_step", "gm_rollout_run", "gm_pages_reset", "gm_pages_reserve",
-           "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_reconstruct_states", "gm_head_state_grad", "gm_head_ffn_backward", "gm_head_input_backward", "gm_adamw_step", "gm_overlap", "gm_dca_loss", "gm_dca_grad",
+           "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_reconstruct_states", "gm_head_state_grad", "gm_head_ffn_backward", "gm_attention_backward", "gm_head_input_backward", "gm_adamw_step", "gm_overlap", "gm_dca_loss", "gm_dca_grad",
            "gm_spec_step_host", "gm_gemm", "gm_gemm_swiglu", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
            "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_chain_trace", "gm_chain_trace_read", "gm_selftest_wait_expiry", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
@@ -97,6 +97,7 @@ def lib() -> C.CDLL:
     L.gm_reconstruct_states.argtypes = [vp, C.POINTER(gm_state), i32, i32, vp, C.POINTER(gm_record), vp, i32, vp, vp, vp]
     L.gm_head_state_grad.argtypes = [vp, i32, vp, vp, vp, vp, i32]
     L.gm_head_ffn_backward.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, i32]
+    L.gm_attention_backward.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp]
     L.gm_head_input_backward.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, i32]
     L.gm_adamw_step.argtypes = [vp, C.c_int64, vp, vp, vp, vp, vp, i32, f32, f32, f32, f32, f32, f32]
     L.gm_overlap.argtypes = [vp, i32, i32, f32, vp, C.POINTER(gm_record), vp, vp]
@@ -413,6 +414,14 @@ def gm_head_state_grad(ctx: Context, rows: int, grad_logits, grad_normed, head_s
 def gm_head_ffn_backward(ctx: Context, rows: int, x, dg, dx, dw_gate_up, dw_down, dln2, refresh_weights: bool = False):
     _check(lib().gm_head_ffn_backward(ctx.handle, rows, _p(x), _p(dg), _p(dx), _p(dw_gate_up), _p(dw_down), _p(dln2),
                                       int(refresh_weights)), "gm_head_ffn_backward")
+
+
+def gm_attention_backward(ctx: Context, q, dout, kv_pool, layer: int, page_table, q_count, q_base, batch: int, q_stride: int,
+                          dq, dk_pool, dv_pool):
+    pool_layers, num_pages = kv_pool.shape[0], kv_pool.shape[2]
+    _check(lib().gm_attention_backward(ctx.handle, _p(q), _p(dout), _p(kv_pool), pool_layers, num_pages, layer, _p(page_table),
+                                       _p(q_count), _p(q_base), batch, q_stride, _p(dq), _p(dk_pool), _p(dv_pool)),
+           "gm_attention_backward")
 
 
 def gm_head_input_backward(ctx: Context, rows: int, tokens, hidden, dz, dhidden, dproj, denorm, dhnorm, refresh_weights: bool = False):

@@ -260,4 +260,29 @@ int gm_head_input_backward(gm_ctx *c, int rows, const int32_t *tokens, const flo
   return run_gemm(c, c->hin_dzt, d, &wm, c->hin_zint, d, 2 * d, Mp, dproj, EPI_STORE_F32, 2 * static_cast<size_t>(d), false);
 }
 
+int gm_attention_backward(gm_ctx *c, const void *q, const float *dout, const void *kv_pool, int pool_layers, int num_pages, int layer,
+                          const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch, int q_stride,
+                          float *dq, float *dk_pool, float *dv_pool) {
+  if (!c || !q || !dout || !kv_pool || !page_table || !q_count || !q_base || !dq || !dk_pool || !dv_pool) return GM_ERR_INVALID_ARG;
+  if (batch < 1 || q_stride < 1 || pool_layers < 1 || layer < 0 || layer >= pool_layers || num_pages < 1) return GM_ERR_INVALID_ARG;
+  const gm_config &cf = c->cfg;
+  if (q_stride > 8 || c->group > 8 || (cf.head_dim != 64 && cf.head_dim != 128)) return GM_ERR_UNSUPPORTED;
+  const size_t need = static_cast<size_t>(batch) * q_stride * cf.n_q_heads * 3;
+  if (need > c->ab_stats_cap) {
+    int rc = dev_alloc(c, &c->ab_stats, need);
+    if (rc != GM_OK) return rc;
+    c->ab_stats_cap = need;
+  }
+  AttnBwdArgs A;
+  A.q = static_cast<const __nv_bfloat16 *>(q); A.dout = dout; A.pool = static_cast<const __nv_bfloat16 *>(kv_pool);
+  A.qn = q_count; A.qbase = q_base; A.page_table = page_table;
+  A.batch = batch; A.QT = q_stride; A.n_kv = cf.n_kv_heads; A.group = c->group; A.hd = cf.head_dim;
+  A.qrows = round16(q_stride * c->group); A.layer = layer; A.num_pages = num_pages; A.max_pages_per_seq = cf.max_pages_per_seq;
+  A.scale = static_cast<float>(1.0 / std::sqrt(static_cast<double>(cf.head_dim)));
+  A.stats = c->ab_stats; A.dq = dq; A.dk_pool = dk_pool; A.dv_pool = dv_pool; A.status = c->status;
+  GM_CUDA(c, cudaMemsetAsync(dq, 0, sizeof(float) * static_cast<size_t>(batch) * q_stride * cf.n_q_heads * cf.head_dim, c->stream));
+  GM_LAUNCH(c, GM_KC_ATTENTION, launch_attention_backward(A, c->stream));
+  return GM_OK;
+}
+
 }  // extern "C"

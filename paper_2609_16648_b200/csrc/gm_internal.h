@@ -119,6 +119,8 @@ struct gm_ctx {
   int hin_rows_cap = 0;
   __nv_bfloat16 *hin_zin = nullptr, *hin_dz = nullptr, *hin_zint = nullptr, *hin_dzt = nullptr;
   float *hin_e = nullptr, *hin_dzin = nullptr, *hin_t = nullptr;
+  float *ab_stats = nullptr;                // attention backward: (max, 1 / sum, D) per (row, query head)
+  size_t ab_stats_cap = 0;
   __nv_bfloat16 *lm_head_t = nullptr;       // [d, V]: the LM head transposed, the weight operand of the gradient GEMM
   CUtensorMap lm_head_t_map;
   float top_p = 1.f;                    // nucleus of the target distributions (1 = none)

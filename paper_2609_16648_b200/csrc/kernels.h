@@ -328,6 +328,20 @@ struct AttnArgs {
   int rows_used = 0;                    // query rows a sequence can have (q positions x group); 0 = unknown (qrows is assumed)
 };
 cudaError_t launch_attention(const AttnArgs &A, cudaStream_t stream);
+// Backward of the attention core: dq for every query row, and the key / value gradients accumulated (atomically) into fp32
+// planes laid out like one layer of the pool.  stats: scratch fp32 [batch * QT][n_q][3].
+struct AttnBwdArgs {
+  const __nv_bfloat16 *q;               // [B][n_kv][qrows][hd], row j*group + g (the forward kernel's query layout)
+  const float *dout;                    // [B * QT][n_q * hd]: gradient of the attention output
+  const __nv_bfloat16 *pool;            // [L][2][num_pages][n_kv][16][hd]
+  const int32_t *qn, *qbase, *page_table;
+  int batch, QT, n_kv, group, hd, qrows, layer, num_pages, max_pages_per_seq;
+  float scale;                          // 1 / sqrt(hd)
+  float *stats, *dq;                    // dq [B * QT][n_q * hd]
+  float *dk_pool, *dv_pool;             // [num_pages][n_kv][16][hd], accumulated
+  uint32_t *status;
+};
+cudaError_t launch_attention_backward(const AttnBwdArgs &A, cudaStream_t stream);
 struct AttnCombineArgs {
   const float *part_o, *part_ml;
   const int32_t *qn, *page_start;

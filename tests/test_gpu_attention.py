@@ -124,3 +124,74 @@ def test_4b_shape_batch_on_sampled_sequences(qs):
         ref = omodel.attention(qq, k, v, np.arange(lens[b], S), idx)
         assert np.abs(got[b] - ref).max() / np.abs(ref).max() < 1.5e-2
     ctx.close()
+
+
+@pytest.mark.parametrize("n_q,n_kv,hd,q_stride", [(4, 2, 64, 4), (32, 8, 128, 4), (8, 1, 128, 3), (16, 8, 128, 8)])
+def test_attention_backward_matches_the_oracle(n_q, n_kv, hd, q_stride):
+    """gm_attention_backward against the oracle's attention_grad, sequence by sequence, on ragged lengths in shuffled pages.
+    The last two sequences are chains of one sequence: their page-table rows share the pages of a common prefix and own
+    the pages after it, so the prefix entries must collect the key / value gradients of both."""
+    import paper_2609_16648_b200 as gmb
+    from oracle import update as oupdate
+    lens = [0, 15, 16, 40, 333, 77, 77]
+    B = len(lens)
+    group = n_q // n_kv
+    rng = np.random.default_rng(9 + q_stride)
+    q_counts = np.array([q_stride] + [int(rng.integers(1, q_stride + 1)) for _ in lens[1:]], np.int32)
+    q_counts[-2:] = q_stride
+    lens = np.asarray(lens)
+    total = lens + q_counts
+    layers, layer = 2, 1
+    cfg = ModelConfig("a", layers, 64, n_q, n_kv, hd, 64, 8, batch=B, k=max(q_stride - 1, 1), kv_len_min=0, kv_len_max=0,
+                      length_law="uniform")
+    pt, npg = make_page_tables(total, 16, seed=4, slack_pages=2)
+    shared = lens[-1] // 16                                   # whole pages of the common prefix (77 // 16 = 4)
+    pt[-1, :shared] = pt[-2, :shared]
+    ctx = gmb.Context(cfg, gmb.random_packed_weights(cfg, "cuda"), B, max(q_stride - 1, 1), pt.shape[1], npg, 4)
+    pool = np.zeros((layers, 2, npg, n_kv, 16, hd), np.float32)
+    q_rows = 16 * ((q_stride * group + 15) // 16)
+    qbuf = np.zeros((B, n_kv, q_rows, hd), np.float32)
+    dout = np.zeros((B, q_stride, n_q, hd), np.float32)
+    qs, ks, vs = [], [], []
+    for b in range(B):
+        S, n = int(total[b]), int(q_counts[b])
+        k = bf16_round(rng.standard_normal((S, n_kv, hd)).astype(np.float32))
+        v = bf16_round(rng.standard_normal((S, n_kv, hd)).astype(np.float32))
+        if b == B - 1:                                         # the second chain sees the first one's prefix entries
+            k[:shared * 16], v[:shared * 16] = ks[-1][:shared * 16], vs[-1][:shared * 16]
+        q = bf16_round(rng.standard_normal((n, n_q, hd)).astype(np.float32) * 1.5)
+        idx = np.arange(S)
+        pool[layer, 0, pt[b, idx // 16], :, idx % 16, :] = k
+        pool[layer, 1, pt[b, idx // 16], :, idx % 16, :] = v
+        for j in range(n):
+            for h in range(n_q):
+                qbuf[b, h // group, j * group + h % group] = q[j, h]
+        dout[b, :n] = rng.standard_normal((n, n_q, hd)).astype(np.float32)
+        dout[b, n:] = 5.0                                      # rows beyond q_count must be ignored
+        qs.append(q); ks.append(k); vs.append(v)
+    dev = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(device="cuda", dtype=dt)
+    dq = torch.full((B * q_stride, n_q * hd), 7.0, dtype=torch.float32, device="cuda")
+    dkp = torch.zeros((npg, n_kv, 16, hd), dtype=torch.float32, device="cuda")
+    dvp = torch.zeros_like(dkp)
+    gmb.gm_attention_backward(ctx, dev(qbuf, torch.bfloat16), dev(dout.reshape(B * q_stride, -1), torch.float32),
+                              dev(pool, torch.bfloat16), layer, dev(np.where(pt < 0, 0, pt), torch.int32),
+                              dev(q_counts, torch.int32), dev(lens.astype(np.int32), torch.int32), B, q_stride, dq, dkp, dvp)
+    assert gmb.gm_last_status(ctx) == 0
+    got_dq = dq.cpu().numpy().reshape(B, q_stride, n_q, hd)
+    got_dk, got_dv = dkp.cpu().numpy().astype(np.float64), dvp.cpu().numpy().astype(np.float64)
+    want_dk, want_dv = np.zeros_like(got_dk), np.zeros_like(got_dv)
+    worst = 0.0
+    for b in range(B):
+        S, n = int(total[b]), int(q_counts[b])
+        idx = np.arange(S)
+        rdq, rdk, rdv = oupdate.attention_grad(dout[b, :n], qs[b], ks[b], vs[b], np.arange(lens[b], S), idx)
+        worst = max(worst, np.abs(got_dq[b, :n] - rdq).max() / np.abs(rdq).max())
+        assert np.all(got_dq[b, n:] == 0)
+        np.add.at(want_dk, (pt[b, idx // 16], slice(None), idx % 16), rdk)
+        np.add.at(want_dv, (pt[b, idx // 16], slice(None), idx % 16), rdv)
+    assert worst < 2e-4, worst                                 # fp32 arithmetic on exact bf16 inputs
+    assert np.abs(got_dk - want_dk).max() < 2e-4 * np.abs(want_dk).max()
+    assert np.abs(got_dv - want_dv).max() < 2e-4 * np.abs(want_dv).max()
+    prefix_pages = pt[-2, :shared]
+    assert np.abs(want_dk[prefix_pages]).max() > 0              # the shared pages did collect terms (from both chains)
+    ctx.close()
