@@ -148,12 +148,10 @@ def ffn_block(lw, x, cfg) -> np.ndarray:
     return x + act @ f64(lw["wd"]).T
 
 
-def decoder_layer(lw, x, pos, kv: PagedKV, layer: int, b: int, cfg) -> np.ndarray:
-    """One pre-norm decoder layer over new rows x [T, d] at positions pos, against the cache.
-
-    The rows' keys/values are written to the cache first; each row then attends every
-    cached position <= its own.
-    """
+def attention_block(lw, x, pos, kv: PagedKV, layer: int, b: int, cfg) -> np.ndarray:
+    """The attention half of a pre-norm decoder layer over new rows x [T, d] at positions pos, against the cache:
+    x + W_o attention(...).  The rows' keys/values are written to the cache first; each row then attends every
+    cached position <= its own."""
     x = f64(x)
     T = x.shape[0]
     pos = np.asarray(pos)
@@ -165,8 +163,12 @@ def decoder_layer(lw, x, pos, kv: PagedKV, layer: int, b: int, cfg) -> np.ndarra
     n = int(pos.max()) + 1
     kc, vc = kv.gather(layer, b, n)
     o = attention(q, kc, vc, pos, np.arange(n)).reshape(T, cfg.q_dim)
-    x = x + o @ f64(lw["wo"]).T
-    return ffn_block(lw, x, cfg)
+    return x + o @ f64(lw["wo"]).T
+
+
+def decoder_layer(lw, x, pos, kv: PagedKV, layer: int, b: int, cfg) -> np.ndarray:
+    """One pre-norm decoder layer over new rows x [T, d] at positions pos, against the cache."""
+    return ffn_block(lw, attention_block(lw, x, pos, kv, layer, b, cfg), cfg)
 
 
 def target_forward(w, tokens, pos, kv: PagedKV, b: int, cfg) -> np.ndarray:

@@ -37,6 +37,14 @@ Fourth step: through the head's input (App. B.1), z = W_p [RMSNorm_e(E[token]) ;
 the gradients of the projection and of the two norm weights (the embedding table is the backbone's: no gradient), and
 dL/d(hidden) - which, for a draft application k >= 2, is a further term of dL/dg_{k-1}: the recurrence of Eq. 4.
 
+The attention half of the head's layer around that core: the output projection, the rotary embedding (its backward is
+the rotation by the opposite angle), the optional per-head norms and projection biases, the query / key / value
+projections and the first norm.  With it the pieces chain into the gradient of the whole objective with respect to
+every parameter of the head (`head_update_grad`): applications are walked from the last draft back to the pass over
+the committed prefix, a state's gradient collecting the term through its own logits and the term through the next
+application's input (Eq. 4), a cache entry's gradient collecting the terms of every later row that attended to it
+before the application that wrote it is walked.
+
 The update itself: AdamW on the head's parameter group, with the head's learning-rate schedule (App. B, optimizer and
 learning rate: linear warm-up over 10 steps, then a cosine decay to a tenth of the peak).  The paper names the
 optimizer and the rates only; the moment coefficients, the stabilising constant and the weight decay are the defaults
@@ -47,7 +55,8 @@ from __future__ import annotations
 import numpy as np
 
 from . import record, sampler
-from .model import PagedKV, f64, head_forward, head_logits, rmsnorm, round_bf16
+from .model import (PagedKV, attention, attention_block, f64, ffn_block, head_forward, head_input, head_logits, project_qkv,
+                    rmsnorm, rope, round_bf16)
 
 
 def reconstruct_states(w, cfg, seq_hidden, seq_tokens, start_len: int, drafts) -> np.ndarray:
@@ -266,6 +275,117 @@ def head_input_grad(dz, w, hidden, tokens, cfg) -> dict:
     r_h = 1.0 / np.sqrt((hidden * hidden).mean(axis=-1, keepdims=True) + cfg.rms_eps)
     return {"dhidden": rmsnorm_grad(dhn, hidden, hw["hnorm"], cfg.rms_eps), "dproj": dproj,
             "denorm": (den * e * r_e).sum(axis=0), "dhnorm": (dhn * hidden * r_h).sum(axis=0)}
+
+
+def rope_grad(dy, pos, base: float) -> np.ndarray:
+    """Backward of model.rope: a rotation is linear and orthogonal, so the gradient turns by the opposite angle.
+    dy [T, H, hd], pos [T]."""
+    return rope(dy, -f64(pos), base)
+
+
+def _rms_weight_grad(dy, x, eps: float) -> np.ndarray:
+    """dL/dw of y = x r w summed over every leading axis: sum dy x r."""
+    x, dy = f64(x), f64(dy)
+    r = 1.0 / np.sqrt((x * x).mean(axis=-1, keepdims=True) + eps)
+    return (dy * x * r).reshape(-1, x.shape[-1]).sum(axis=0)
+
+
+def attention_block_grad(dxmid, x, lw, pos, kc, vc, dkc, dvc, cfg) -> dict:
+    """Backward of model.attention_block for rows x [T, d] at positions pos.  dxmid [T, d] = dL/d(output).
+    kc, vc [n, n_kv, hd] = cache entries 0..n-1 as the rows saw them (their own included, n = max(pos) + 1).
+    dkc, dvc [>= n, n_kv, hd] = gradient already collected on the cache entries from rows of later applications;
+    the terms of these rows are added IN PLACE, after which the rows' own entries are complete and are taken back
+    through the rotary embedding, the optional head norms and the projections.
+    Returns {"dx", "dln1", "dwq", "dwk", "dwv", "dwo"} plus {"dbq", "dbk", "dbv"} / {"dqnorm", "dknorm"} where the
+    layer has them."""
+    dxmid, x = f64(dxmid), f64(x)
+    T = x.shape[0]
+    pos = np.asarray(pos)
+    n = int(pos.max()) + 1
+    eps = cfg.rms_eps
+    h = rmsnorm(x, lw["ln1"], eps)
+    raw = {k: v for k, v in lw.items() if k not in ("qnorm", "knorm")}
+    q0, k0, _ = project_qkv(raw, h, cfg)                       # heads before the optional norm
+    qn, _, _ = project_qkv(lw, h, cfg)
+    q = rope(qn, pos, cfg.rope_base)
+    o = attention(q, kc[:n], vc[:n], pos, np.arange(n)).reshape(T, cfg.q_dim)
+    out = {"dwo": dxmid.T @ o}
+    do = (dxmid @ f64(lw["wo"])).reshape(T, cfg.n_q_heads, cfg.head_dim)
+    dq, dk_all, dv_all = attention_grad(do, q, kc[:n], vc[:n], pos, np.arange(n))
+    dkc[:n] += dk_all
+    dvc[:n] += dv_all
+    dq = rope_grad(dq, pos, cfg.rope_base)
+    dk = rope_grad(dkc[pos], pos, cfg.rope_base)
+    dv = f64(dvc[pos])
+    if "qnorm" in lw:
+        out["dqnorm"], out["dknorm"] = _rms_weight_grad(dq, q0, eps), _rms_weight_grad(dk, k0, eps)
+        dq, dk = rmsnorm_grad(dq, q0, lw["qnorm"], eps), rmsnorm_grad(dk, k0, lw["knorm"], eps)
+    dq, dk, dv = dq.reshape(T, -1), dk.reshape(T, -1), dv.reshape(T, -1)
+    if "bq" in lw:
+        out["dbq"], out["dbk"], out["dbv"] = dq.sum(axis=0), dk.sum(axis=0), dv.sum(axis=0)
+    out["dwq"], out["dwk"], out["dwv"] = dq.T @ h, dk.T @ h, dv.T @ h
+    dh = dq @ f64(lw["wq"]) + dk @ f64(lw["wk"]) + dv @ f64(lw["wv"])
+    out["dx"] = dxmid + rmsnorm_grad(dh, x, lw["ln1"], eps)
+    out["dln1"] = _rms_weight_grad(dh, x, eps)
+    return out
+
+
+def _accumulate(total: dict, part: dict, names) -> None:
+    for name in names:
+        if name in part:
+            total[name] = total.get(name, 0.0) + part[name]
+
+
+def head_update_grad(w, cfg, sequences, records, temperature: float = 1.0) -> dict:
+    """Gradient of head_update_loss (no rounding at the logits interface) with respect to every parameter of the head.
+    Same arguments as head_update_loss.  Returns {"proj", "enorm", "hnorm", "final_norm", "layer": {"ln1", "wq", "wk",
+    "wv", "wo", "ln2", "wg", "wu", "wd" [, "bq", "bk", "bv"] [, "qnorm", "knorm"]}} in float64; the embedding table
+    and the LM head are the backbone's and get none."""
+    hw, lw = w["head"], w["head"]["layer"]
+    top, lay = {}, {}
+    n_rec = len(records)
+    for s, rec in records:
+        hid, toks = sequences[s]
+        Len, drafts = int(rec["start_pos"]), rec["drafts"]
+        K = len(drafts)
+        # forward, keeping each application's input pairs and positions (application 1 = the pass over the prefix)
+        pages = (Len + K + cfg.page_size) // cfg.page_size + 1
+        hkv = PagedKV(1, cfg.n_kv_heads, cfg.head_dim, np.arange(pages)[None, :], pages, cfg.page_size)
+        apps = [(f64(np.asarray(hid)[:Len - 1]), list(toks[1:Len]), np.arange(Len - 1))]
+        g = head_forward(w, *apps[0], hkv, 0, cfg)[-1:]
+        states = [g[0]]
+        for k in range(2, K + 1):
+            apps.append((g, [int(drafts[k - 2])], np.array([Len + k - 3])))
+            g = head_forward(w, *apps[-1], hkv, 0, cfg)
+            states.append(g[0])
+        states = np.array(states)
+        kc, vc = hkv.gather(0, 0, Len + K - 2)
+        # the term of every state through its own logits
+        dstate, gy, _ = head_update_grad_state(w, cfg, states[None], [rec], temperature)
+        dstate, gy = dstate[0] / n_rec, gy[0] / n_rec
+        top["final_norm"] = top.get("final_norm", 0.0) + _rms_weight_grad(gy, states, cfg.rms_eps)
+        # backward, last application first
+        dkc, dvc = np.zeros_like(kc), np.zeros_like(vc)
+        for a in range(K - 1, -1, -1):
+            hidden, tokens, pos = apps[a]
+            z = head_input(w, hidden, tokens, cfg)
+            akv = PagedKV(1, cfg.n_kv_heads, cfg.head_dim, np.arange(pages)[None, :], pages, cfg.page_size)
+            akv.pool[:] = hkv.pool                            # entries beyond these rows' positions are never read
+            xmid = attention_block(lw, z, pos, akv, 0, 0, cfg)
+            dg = np.zeros_like(xmid)
+            dg[-1] = dstate[a]                                # only the last row's state is used (all of them: 1 row, a >= 1)
+            f = ffn_block_grad(dg, xmid, lw, cfg.rms_eps)
+            n = int(pos.max()) + 1
+            at = attention_block_grad(f["dx"], z, lw, pos, kc[:n], vc[:n], dkc, dvc, cfg)
+            hi = head_input_grad(at["dx"], w, hidden, tokens, cfg)
+            if a >= 1:
+                dstate[a - 1] += hi["dhidden"][0]             # Eq. 4: this application consumed g_{a}
+            _accumulate(lay, {k[1:]: v for k, v in f.items()}, ("ln2", "wg", "wu", "wd"))
+            _accumulate(lay, {k[1:]: v for k, v in at.items()},
+                        ("ln1", "wq", "wk", "wv", "wo", "bq", "bk", "bv", "qnorm", "knorm"))
+            _accumulate(top, {k[1:]: v for k, v in hi.items()}, ("proj", "enorm", "hnorm"))
+    top["layer"] = lay
+    return top
 
 
 def adamw_step(p, g, m, v, step: int, lr: float, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,

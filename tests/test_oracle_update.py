@@ -367,3 +367,92 @@ def test_attention_gradient_matches_finite_differences():
     assert np.abs(dk.sum(axis=0)).max() < 1e-12
     # values enter linearly: dv is the attention-weighted sum of the output gradients, so it sums to the sum of dout per group
     np.testing.assert_allclose(dv.sum(axis=0), C.reshape(T_, n_kv, n_q // n_kv, hd).sum(axis=(0, 2)), rtol=1e-12)
+
+
+def test_rope_gradient_is_the_inverse_rotation():
+    rng = np.random.default_rng(43)
+    x, C = rng.normal(0, 1, (3, 2, 8)), rng.normal(0, 1, (3, 2, 8))
+    pos = np.array([0, 5, 17])
+    g = update.rope_grad(C, pos, 1.0e4)
+    for i in [(0, 0, 1), (1, 1, 2), (2, 0, 6), (1, 0, 7)]:
+        e = np.zeros(x.shape)
+        e[i] = 1e-6
+        fd = ((model.rope(x + e, pos, 1.0e4) - model.rope(x - e, pos, 1.0e4)) * C).sum() / 2e-6
+        assert g[i] == pytest.approx(fd, rel=1e-7, abs=1e-10)
+    np.testing.assert_allclose(update.rope_grad(model.rope(x, pos, 1.0e4), pos, 1.0e4), x, atol=1e-12)   # orthogonal
+    np.testing.assert_allclose(g[0], C[0], atol=1e-15)                                                    # position 0: identity
+
+
+def _flat_params(w):
+    """(name, array) of every head parameter, views into w (float64 copies installed in place)."""
+    hw = w["head"]
+    out = []
+    for name in ("proj", "enorm", "hnorm", "final_norm"):
+        hw[name] = np.array(hw[name], np.float64)
+        out.append((name, hw[name]))
+    for name in sorted(hw["layer"]):
+        hw["layer"][name] = np.array(hw["layer"][name], np.float64)
+        out.append(("layer." + name, hw["layer"][name]))
+    return out
+
+
+@pytest.mark.parametrize("family", ["plain", "qkv_bias", "qk_norm"])
+def test_head_update_gradient_matches_finite_differences_of_the_objective(family):
+    """Every parameter tensor of the head: sampled coordinates and one random direction over all of them against
+    central differences of head_update_loss - which goes through the prefix pass, the recurrence over the drafts, the
+    shared cache entries, the logits and Eq. 9; any missing path (a state's second term, a cache entry's later readers,
+    a norm's weight) changes these numbers."""
+    import dataclasses
+    global CFG
+    keep = CFG
+    CFG = dataclasses.replace(CFG, qkv_bias=family == "qkv_bias", qk_norm=family == "qk_norm")
+    try:
+        w, st, cycles = _rollout_with_records(rounding=False, n_steps=2)
+        seqs = _sequence_features(w, st, rounding=False)
+        cfg = CFG
+    finally:
+        CFG = keep
+    recs = [(b, dict(rec, accepted=i % 4 + 1)) for i, (b, rec, _, _) in enumerate(cycles)]   # every cut of Eq. 9: j = 1 .. K + 1
+    params = _flat_params(w)
+    grad = update.head_update_grad(w, cfg, seqs, recs, T)
+
+    def loss():
+        """head_update_loss without the fp32 rounding of q (which would drown a 1e-6 step): same states, same logits,
+        same objective, every step in float64."""
+        per = []
+        for s_, rec in recs:
+            g = update.reconstruct_states(w, cfg, seqs[s_][0], seqs[s_][1], rec["start_pos"], rec["drafts"])
+            q = update.softmax64(model.head_logits(w, g, cfg), T)
+            per.append(update.dca_loss(update.chain_alphas(rec, q), rec["accepted"]))
+        return float(np.mean(per))
+
+    assert loss() == pytest.approx(update.head_update_loss(w, cfg, seqs, recs, T, round_interface=False)[0], rel=1e-5)
+    names = {n for n, _ in params}
+    assert {"layer." + n for n in grad["layer"]} | (set(grad) - {"layer"}) == names
+    rng = np.random.default_rng(47)
+    for name, arr in params:
+        g = grad["layer"][name[6:]] if name.startswith("layer.") else grad[name]
+        assert g.shape == arr.shape
+        scale = np.abs(g).max()
+        assert scale > 0
+        for _ in range(3):
+            i = tuple(rng.integers(0, n) for n in arr.shape)
+            x = arr[i]
+            h = 1e-4 * max(1.0, abs(x))                 # the loss carries ~1e-12 of rounding noise: not smaller
+            arr[i] = x + h; hi = loss()
+            arr[i] = x - h; lo = loss()
+            arr[i] = x
+            assert g[i] == pytest.approx((hi - lo) / (2 * h), rel=5e-4, abs=1e-5 * scale), (name, i)
+    # one random direction over all parameters at once
+    dirs = [rng.normal(0, 1, a.shape) * np.abs(a).mean() for _, a in params]
+    expect = sum(float(((grad["layer"][n[6:]] if n.startswith("layer.") else grad[n]) * d).sum()) for (n, _), d in zip(params, dirs))
+    h = 1e-6
+    for (_, a), d in zip(params, dirs):
+        a += h * d
+    hi = loss()
+    for (_, a), d in zip(params, dirs):
+        a -= 2 * h * d
+    lo = loss()
+    for (_, a), d in zip(params, dirs):
+        a += h * d
+    assert expect == pytest.approx((hi - lo) / (2 * h), rel=2e-4)
