@@ -425,6 +425,33 @@ int gm_head_ffn_backward(gm_ctx *ctx, int rows, const float *x, const float *dg,
 int gm_attention_backward(gm_ctx *ctx, const void *q, const float *dout, const void *kv_pool, int pool_layers,
                           int num_pages, int layer, const int32_t *page_table, const int32_t *q_count,
                           const int32_t *q_base, int batch, int q_stride, float *dq, float *dk_pool, float *dv_pool);
+/* The attention half of the head's decoder layer, backward (App. B.1; Alg. 1, "update phi"):
+ *   xmid = x + W_o attention(rope(norm_q(q)), cache),  (q, k, v) = W_qkv RMSNorm(x; ln1) (+ bias),  the rows' own
+ *   rope(norm_k(k)), v being the cache entries at their positions.
+ * A pass is `batch` sequences of up to q_stride rows, row j of sequence b at position q_base[b] + j, j < q_count[b]
+ * (the conventions of gm_attention); passes that share cache entries are walked from the last one written to the first.
+ *   x        device fp32 [batch * q_stride, d]: the layer's input rows (the head's projected input z)
+ *   dxmid    device fp32 [batch * q_stride, d]: dL/d xmid (gm_head_ffn_backward's dx); zero in rows j >= q_count[b]
+ *   kv_pool  device bf16 [1][2][num_pages][n_kv][16][head_dim]: the head's cache as the forward pass left it (read only)
+ *   dk_pool, dv_pool  device fp32 [num_pages][n_kv][16][head_dim], IN and OUT: on entry the gradient the rows of LATER
+ *            passes left on the cache entries (zero before the first call); these rows' terms are added
+ *            (gm_attention_backward), after which the rows' own entries are complete and are read back
+ *   dx       device fp32 [batch * q_stride, d] out: dL/dx = dxmid + the path through the attention half
+ *   dw_qkv   device fp32 [(n_q + 2 n_kv) head_dim, d] out;  dw_o  device fp32 [d, n_q head_dim] out;  dln1  fp32 [d] out
+ *   db_qkv   device fp32 [(n_q + 2 n_kv) head_dim] out - required iff the layer has projection biases, else NULL
+ *   dqk_norm device fp32 [2 head_dim] out (query norm, then key norm) - required iff the layer has head norms, else NULL
+ * The parameter gradients are this pass's sums over its rows (the caller adds passes up).  Forward values (the normed
+ * rows, the projection, the rotated queries, the attention output) are recomputed in bf16 as the forward pass computes
+ * them, in the context's own workspaces - not to be interleaved with a cycle in flight on the same context; products run
+ * on the projection kernel with bf16 operands and fp32 accumulation.  Transposed copies of W_o and W_qkv and scratch for
+ * the rows rounded up to 64 are allocated on first use and kept until gm_free; refresh_weights != 0 remakes the copies.
+ * GM_ERR_UNSUPPORTED: GM_FLAG_SIMPLE_GEMM, d, n_q head_dim or (n_q + 2 n_kv) head_dim not a multiple of 64, head_dim
+ * other than 64 / 128, more than 8 query heads per KV head, q_stride > min(8, max_k + 1), or more rows than a prefill
+ * pass of the context holds.  A page outside the pool: the status word reports GM_ERR_BAD_PAGE and the row gets zeros. */
+int gm_head_attn_backward(gm_ctx *ctx, const float *x, const float *dxmid, const void *kv_pool, int num_pages,
+                          const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch, int q_stride,
+                          float *dk_pool, float *dv_pool, float *dx, float *dw_qkv, float *dw_o, float *dln1, float *db_qkv,
+                          float *dqk_norm, int refresh_weights);
 /* Fourth step of the backward pass: through the head's input (App. B.1),
  *   z = W_p [RMSNorm(E[token]; enorm) ; RMSNorm(hidden; hnorm)]   (the order the packed projection uses).
  *   tokens int32 [rows], hidden fp32 [rows, d]: the pairs that entered;  dz fp32 [rows, d] = dL/dz (device)

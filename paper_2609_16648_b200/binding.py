@@ -24,7 +24,7 @@ GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER, GM_KC_RECORD = 0,
 
 EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw", "gm_set_top_p", "gm_nucleus", "gm_prefill",
            "gm_rollout_begin", "gm_rollout_step", "gm_rollout_run", "gm_pages_reset", "gm_pages_reserve",
-           "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_reconstruct_states", "gm_head_state_grad", "gm_head_ffn_backward", "gm_attention_backward", "gm_head_input_backward", "gm_adamw_step", "gm_overlap", "gm_dca_loss", "gm_dca_grad",
+           "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_reconstruct_states", "gm_head_state_grad", "gm_head_ffn_backward", "gm_attention_backward", "gm_head_attn_backward", "gm_head_input_backward", "gm_adamw_step", "gm_overlap", "gm_dca_loss", "gm_dca_grad",
            "gm_spec_step_host", "gm_gemm", "gm_gemm_swiglu", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
            "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_chain_trace", "gm_chain_trace_read", "gm_selftest_wait_expiry", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
@@ -98,6 +98,7 @@ def lib() -> C.CDLL:
     L.gm_head_state_grad.argtypes = [vp, i32, vp, vp, vp, vp, i32]
     L.gm_head_ffn_backward.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, i32]
     L.gm_attention_backward.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp]
+    L.gm_head_attn_backward.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32]
     L.gm_head_input_backward.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, i32]
     L.gm_adamw_step.argtypes = [vp, C.c_int64, vp, vp, vp, vp, vp, i32, f32, f32, f32, f32, f32, f32]
     L.gm_overlap.argtypes = [vp, i32, i32, f32, vp, C.POINTER(gm_record), vp, vp]
@@ -422,6 +423,13 @@ def gm_attention_backward(ctx: Context, q, dout, kv_pool, layer: int, page_table
     _check(lib().gm_attention_backward(ctx.handle, _p(q), _p(dout), _p(kv_pool), pool_layers, num_pages, layer, _p(page_table),
                                        _p(q_count), _p(q_base), batch, q_stride, _p(dq), _p(dk_pool), _p(dv_pool)),
            "gm_attention_backward")
+
+
+def gm_head_attn_backward(ctx: Context, x, dxmid, kv_pool, page_table, q_count, q_base, batch: int, q_stride: int, dk_pool, dv_pool,
+                          dx, dw_qkv, dw_o, dln1, db_qkv=None, dqk_norm=None, refresh_weights: bool = False):
+    _check(lib().gm_head_attn_backward(ctx.handle, _p(x), _p(dxmid), _p(kv_pool), kv_pool.shape[2], _p(page_table), _p(q_count),
+                                       _p(q_base), batch, q_stride, _p(dk_pool), _p(dv_pool), _p(dx), _p(dw_qkv), _p(dw_o),
+                                       _p(dln1), _p(db_qkv), _p(dqk_norm), int(refresh_weights)), "gm_head_attn_backward")
 
 
 def gm_head_input_backward(ctx: Context, rows: int, tokens, hidden, dz, dhidden, dproj, denorm, dhnorm, refresh_weights: bool = False):

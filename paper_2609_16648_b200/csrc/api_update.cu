@@ -285,4 +285,120 @@ int gm_attention_backward(gm_ctx *c, const void *q, const float *dout, const voi
   return GM_OK;
 }
 
+int gm_head_attn_backward(gm_ctx *c, const float *x, const float *dxmid, const void *kv_pool, int num_pages,
+                          const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch, int q_stride,
+                          float *dk_pool, float *dv_pool, float *dx, float *dw_qkv, float *dw_o, float *dln1, float *db_qkv,
+                          float *dqk_norm, int refresh_weights) {
+  if (!c || !x || !dxmid || !kv_pool || !page_table || !q_count || !q_base || !dk_pool || !dv_pool || !dx || !dw_qkv || !dw_o ||
+      !dln1 || batch < 1 || q_stride < 1 || num_pages < 1)
+    return GM_ERR_INVALID_ARG;
+  const gm_config &cf = c->cfg;
+  const gm_layer_weights &lw = c->w.head_layer;
+  const int d = c->d, hd = cf.head_dim, NQ = c->q_dim, NQKV = c->n_qkv, rows = batch * q_stride;
+  if ((db_qkv != nullptr) != (lw.b_qkv != nullptr) || (dqk_norm != nullptr) != (lw.q_norm != nullptr)) return GM_ERR_INVALID_ARG;
+  if ((cf.flags & GM_FLAG_SIMPLE_GEMM) || (d % 64) || (NQ % 64) || (NQKV % 64) || (hd != 64 && hd != 128) || c->group > 8 ||
+      q_stride > cf.max_k + 1 || q_stride > 8 || batch > cf.max_batch * c->pf_vr || rows > c->Mmax)
+    return GM_ERR_UNSUPPORTED;
+  const __nv_bfloat16 *wqkv = static_cast<const __nv_bfloat16 *>(lw.wqkv), *wo = static_cast<const __nv_bfloat16 *>(lw.wo);
+  const __nv_bfloat16 *ln1 = static_cast<const __nv_bfloat16 *>(lw.ln1);
+  int rc;
+  if (!c->hat_wo_t) {
+    if ((rc = dev_alloc(c, &c->hat_wo_t, static_cast<size_t>(NQ) * d, false)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hat_wqkv_t, static_cast<size_t>(d) * NQKV, false)) != GM_OK) return rc;
+    if (make_map(c, &c->hat_wo_t_map, c->hat_wo_t, NQ, d, 128) != GM_OK) return GM_ERR_CUDA;
+    if (make_map(c, &c->hat_wqkv_t_map, c->hat_wqkv_t, d, NQKV, 128) != GM_OK) return GM_ERR_CUDA;
+    refresh_weights = 1;
+  }
+  if (refresh_weights) {
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(wo, d, NQ, c->hat_wo_t, c->stream));             // [d, q_dim] -> [q_dim, d]
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(wqkv, NQKV, d, c->hat_wqkv_t, c->stream));       // [n_qkv, d] -> [d, n_qkv]
+  }
+  const int Mp = (rows + 63) / 64 * 64;
+  if (Mp > c->hat_rows_cap) {
+    const size_t M = static_cast<size_t>(Mp);
+    if ((rc = dev_alloc(c, &c->hat_dy, M * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hat_dqkv_bf, M * NQKV)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hat_dyt, M * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hat_ot, M * NQ)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hat_dqkvt, M * NQKV)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hat_ht, M * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hat_do, M * NQ)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hat_dq, M * NQ)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hat_dqkv, M * NQKV)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hat_dh, M * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hat_t, M * d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hat_tq, M * NQ)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hat_tk, M * (NQKV - NQ) / 2)) != GM_OK) return rc;
+    c->hat_rows_cap = Mp;
+  }
+  // ---- the forward's values, recomputed: h = RMSNorm(x; ln1), the projection, the rotated queries, the attention output ----
+  if ((rc = run_plan_chunk(c, batch, q_count, q_base, q_stride)) != GM_OK) return rc;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rmsnorm(x, ln1, c->xn, nullptr, rows, d, cf.rms_eps, c->stream));
+  if ((rc = run_gemm(c, c->xn, c->Mmax, &c->head_maps.wqkv, wqkv, rows, NQKV, d, c->qkv, EPI_STORE_BF16, NQKV)) != GM_OK) return rc;
+  const int qrows = round16(q_stride * c->group);
+  RopeAppendArgs R;
+  R.qkv = c->qkv; R.batch = batch; R.QT = q_stride; R.n_q = cf.n_q_heads; R.n_kv = cf.n_kv_heads; R.hd = hd; R.layer = 0;
+  R.num_pages = num_pages; R.max_pages_per_seq = cf.max_pages_per_seq; R.qrows = qrows; R.qn = c->qn; R.qbase = c->qbase;
+  R.page_table = page_table; R.rope = c->rope; R.qbuf = c->qbuf; R.pool = nullptr; R.status = c->status;   // the cache is read, not rewritten
+  R.bias = static_cast<const __nv_bfloat16 *>(lw.b_qkv);
+  R.qnorm = static_cast<const __nv_bfloat16 *>(lw.q_norm); R.knorm = static_cast<const __nv_bfloat16 *>(lw.k_norm);
+  R.eps = cf.rms_eps;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rope_append(R, c->stream));
+  CUtensorMap kvm;
+  if ((rc = kv_map(c, kv_pool, 1, num_pages, &kvm)) != GM_OK) return rc;
+  AttnArgs T;
+  T.kv_map = kvm; T.qbuf = c->qbuf; T.qn = c->qn; T.qbase = c->qbase; T.page_start = c->page_start; T.page_table = page_table;
+  T.batch = batch; T.n_kv = cf.n_kv_heads; T.group = c->group; T.hd = hd; T.qrows = qrows; T.layer = 0; T.num_pages = num_pages;
+  T.max_pages_per_seq = cf.max_pages_per_seq; T.n_ctas = c->sm_count;
+  T.scale_log2e = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(hd)));
+  T.part_o = c->part_o; T.part_ml = c->part_ml; T.status = c->status; T.rows_used = q_stride * c->group;
+  GM_LAUNCH(c, GM_KC_ATTENTION, launch_attention(T, c->stream));
+  AttnCombineArgs Cb;
+  Cb.part_o = c->part_o; Cb.part_ml = c->part_ml; Cb.qn = c->qn; Cb.page_start = c->page_start; Cb.batch = batch;
+  Cb.n_kv = cf.n_kv_heads; Cb.group = c->group; Cb.hd = hd; Cb.qrows = qrows; Cb.QT = q_stride; Cb.n_ctas = c->sm_count;
+  Cb.out = c->attn_out;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_attention_combine(Cb, c->stream));
+  // ---- d(attention output) = dxmid W_o, then the attention core ----
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_cast_bf16(dxmid, c->hat_dy, static_cast<size_t>(rows) * d, c->stream));
+  if ((rc = run_gemm(c, c->hat_dy, rows, &c->hat_wo_t_map, c->hat_wo_t, rows, NQ, d, c->hat_do, EPI_STORE_F32, static_cast<size_t>(NQ), false)) != GM_OK)
+    return rc;
+  if ((rc = gm_attention_backward(c, c->qbuf, c->hat_do, kv_pool, 1, num_pages, 0, page_table, c->qn, c->qbase, batch, q_stride,
+                                  c->hat_dq, dk_pool, dv_pool)) != GM_OK)
+    return rc;
+  // ---- the rows' own entries are complete now: back through the rotation and the head norms, packed like the projection ----
+  QkvGradArgs Q;
+  Q.qkv = c->qkv; Q.bias = R.bias; Q.qnorm = R.qnorm; Q.knorm = R.knorm; Q.dq = c->hat_dq; Q.dk_pool = dk_pool; Q.dv_pool = dv_pool;
+  Q.qn = c->qn; Q.qbase = c->qbase; Q.page_table = page_table; Q.rope = c->rope; Q.batch = batch; Q.QT = q_stride;
+  Q.n_q = cf.n_q_heads; Q.n_kv = cf.n_kv_heads; Q.hd = hd; Q.num_pages = num_pages; Q.max_pages_per_seq = cf.max_pages_per_seq;
+  Q.eps = cf.rms_eps; Q.dqkv = c->hat_dqkv; Q.dqkv_bf = c->hat_dqkv_bf; Q.status = c->status;
+  if (dqk_norm) { Q.tq = c->hat_tq; Q.tk = c->hat_tk; }
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_qkv_grad_rows(Q, c->stream));
+  if (dqk_norm) {
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_tq, rows * cf.n_q_heads, hd, dqk_norm, c->stream));
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_tk, rows * cf.n_kv_heads, hd, dqk_norm + hd, c->stream));
+  }
+  if (db_qkv) GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_dqkv, rows, NQKV, db_qkv, c->stream));
+  // ---- dh = dqkv W_qkv;  dx = dxmid + d RMSNorm;  dln1 ----
+  if ((rc = run_gemm(c, c->hat_dqkv_bf, rows, &c->hat_wqkv_t_map, c->hat_wqkv_t, rows, d, NQKV, c->hat_dh, EPI_STORE_F32, static_cast<size_t>(d), false)) != GM_OK)
+    return rc;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rmsnorm_grad(c->hat_dh, x, ln1, dx, rows, d, cf.rms_eps, c->stream, dxmid, c->hat_t));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_t, rows, d, dln1, c->stream));
+  // ---- weight gradients contract over the rows: operands transposed to [features, rows] (rows padded with zeros to Mp) ----
+  GM_CUDA(c, cudaMemsetAsync(c->hat_dyt, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
+  GM_CUDA(c, cudaMemsetAsync(c->hat_ot, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * NQ, c->stream));
+  GM_CUDA(c, cudaMemsetAsync(c->hat_dqkvt, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * NQKV, c->stream));
+  GM_CUDA(c, cudaMemsetAsync(c->hat_ht, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->hat_dy, rows, d, c->hat_dyt, c->stream, Mp));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->attn_out, rows, NQ, c->hat_ot, c->stream, Mp));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->hat_dqkv_bf, rows, NQKV, c->hat_dqkvt, c->stream, Mp));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->xn, rows, d, c->hat_ht, c->stream, Mp));
+  CUtensorMap wm;
+  // dW_o [d, q_dim] = dxmid^T o
+  if (make_map(c, &wm, c->hat_ot, NQ, Mp, 128) != GM_OK) return GM_ERR_CUDA;
+  if ((rc = run_gemm(c, c->hat_dyt, d, &wm, c->hat_ot, d, NQ, Mp, dw_o, EPI_STORE_F32, static_cast<size_t>(NQ), false)) != GM_OK) return rc;
+  // dW_qkv [n_qkv, d] = dqkv^T h
+  if (make_map(c, &wm, c->hat_ht, d, Mp, 128) != GM_OK) return GM_ERR_CUDA;
+  return run_gemm(c, c->hat_dqkvt, NQKV, &wm, c->hat_ht, NQKV, d, Mp, dw_qkv, EPI_STORE_F32, static_cast<size_t>(d), false);
+}
+
 }  // extern "C"

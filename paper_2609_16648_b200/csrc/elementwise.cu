@@ -459,8 +459,9 @@ __global__ void __launch_bounds__(EW_THREADS) rope_append_kernel(const RopeAppen
   }
   const int pos = qb + j;
   const int page = A.page_table[static_cast<size_t>(b) * A.max_pages_per_seq + (pos >> 4)];
-  const bool page_ok = page >= 0 && page < A.num_pages;
-  if (!page_ok && threadIdx.x == 0) set_status(A.status, ST_BAD_PAGE);
+  const bool in_pool = page >= 0 && page < A.num_pages;
+  if (!in_pool && threadIdx.x == 0) set_status(A.status, ST_BAD_PAGE);
+  const bool page_ok = in_pool && A.pool != nullptr;              // no pool: queries only, nothing is appended
   const float2 *cs = A.rope + static_cast<size_t>(pos) * half;
   const size_t page_elems = static_cast<size_t>(A.n_kv) * 16 * hd;
   __nv_bfloat16 *kdst = A.pool + ((static_cast<size_t>(A.layer) * 2 + 0) * A.num_pages + (page_ok ? page : 0)) * page_elems;

@@ -121,6 +121,12 @@ struct gm_ctx {
   float *hin_e = nullptr, *hin_dzin = nullptr, *hin_t = nullptr;
   float *ab_stats = nullptr;                // attention backward: (max, 1 / sum, D) per (row, query head)
   size_t ab_stats_cap = 0;
+  // attention half of the head's layer, backward: transposed weight copies and per-call scratch
+  __nv_bfloat16 *hat_wo_t = nullptr, *hat_wqkv_t = nullptr;      // [q_dim, d], [d, n_qkv]
+  CUtensorMap hat_wo_t_map, hat_wqkv_t_map;
+  int hat_rows_cap = 0;
+  __nv_bfloat16 *hat_dy = nullptr, *hat_dqkv_bf = nullptr, *hat_dyt = nullptr, *hat_ot = nullptr, *hat_dqkvt = nullptr, *hat_ht = nullptr;
+  float *hat_do = nullptr, *hat_dq = nullptr, *hat_dqkv = nullptr, *hat_dh = nullptr, *hat_t = nullptr, *hat_tq = nullptr, *hat_tk = nullptr;
   __nv_bfloat16 *lm_head_t = nullptr;       // [d, V]: the LM head transposed, the weight operand of the gradient GEMM
   CUtensorMap lm_head_t_map;
   float top_p = 1.f;                    // nucleus of the target distributions (1 = none)

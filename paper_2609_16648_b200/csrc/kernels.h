@@ -271,6 +271,24 @@ cudaError_t launch_adamw(float *master, __nv_bfloat16 *param, const float *grad,
                          float b2, float eps, float decay, float c1, float c2, float gscale, int sm_count, cudaStream_t stream);
 cudaError_t launch_cast_bf16(const float *src, __nv_bfloat16 *dst, size_t n, cudaStream_t stream);       // n % 4 == 0
 // Backward of h = silu(a) * b on interleaved (a, b) columns: dab bf16 [rows, 2F] (da, db interleaved), h bf16 [rows, F].
+// Backward of what lies between the QKV projection and the attention core, for the rows of one pass (App. B.1): takes the
+// rows' query gradients and their own cache entries' key / value gradients back through the rotary embedding (the
+// rotation by the opposite angle) and the optional per-head RMSNorm, into the packed order of the projection's output.
+struct QkvGradArgs {
+  const __nv_bfloat16 *qkv;                             // [M][(n_q + 2 n_kv) hd] projection output of the forward, before bias
+  const __nv_bfloat16 *bias = nullptr, *qnorm = nullptr, *knorm = nullptr;
+  const float *dq;                                      // [M][n_q][hd] gradient of the rotated queries
+  const float *dk_pool, *dv_pool;                       // [num_pages][n_kv][16][hd] gradient planes of the cache
+  const int32_t *qn, *qbase, *page_table;
+  const float2 *rope;
+  int batch, QT, n_q, n_kv, hd, num_pages, max_pages_per_seq;
+  float eps = 0.f;
+  float *dqkv;                                          // [M][(n_q + 2 n_kv) hd]; rows beyond a sequence's count are zero
+  __nv_bfloat16 *dqkv_bf;                               // the same in bf16 (operand of the projections' backward)
+  float *tq = nullptr, *tk = nullptr;                   // per-head terms of the norm weights' gradients [M n_q][hd], [M n_kv][hd]
+  uint32_t *status;
+};
+cudaError_t launch_qkv_grad_rows(const QkvGradArgs &A, cudaStream_t stream);
 cudaError_t launch_swiglu_grad(const __nv_bfloat16 *ab, const float *dh, __nv_bfloat16 *dab, __nv_bfloat16 *h, int rows, int F,
                                cudaStream_t stream);
 
@@ -307,7 +325,7 @@ struct RopeAppendArgs {
   const __nv_bfloat16 *qnorm = nullptr, *knorm = nullptr;  // [hd] RMSNorm weights of the query / key heads, or null
   float eps = 0.f;
   __nv_bfloat16 *qbuf;                                  // [B][n_kv][qrows][hd], row = j*group + g
-  __nv_bfloat16 *pool;                                  // [L][2][num_pages][n_kv][16][hd]
+  __nv_bfloat16 *pool;                                  // [L][2][num_pages][n_kv][16][hd]; null: queries only, nothing appended
   uint32_t *status;
 };
 cudaError_t launch_rope_append(const RopeAppendArgs &A, cudaStream_t stream);

@@ -351,6 +351,91 @@ swiglu_grad_kernel(const __nv_bfloat16 *ab, const float *dh, __nv_bfloat16 *dab,
   h[i] = __float2bfloat16(act * b);
   }
 
+// ---- between the QKV projection and the attention core, backward (App. B.1) -------------------------------------------------
+// One CTA per token row, a warp per head.  Lane l holds elements l*EH .. l*EH + EH - 1 of the head's first half and their
+// rotation partners in the second half (EH = hd / 64).
+template <int EH>
+__global__ void __launch_bounds__(256) qkv_grad_rows_kernel(const QkvGradArgs A) {
+  constexpr int HD = 64 * EH, HALF = 32 * EH;
+  const int m = blockIdx.x, b = m / A.QT, j = m % A.QT;
+  const int lane = threadIdx.x & 31, wp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const int ncols = (A.n_q + 2 * A.n_kv) * HD;
+  pdl_prologue();
+  const int qn = A.qn[b], pos = A.qbase[b] + j;
+  float *out = A.dqkv + static_cast<size_t>(m) * ncols;
+  __nv_bfloat16 *outb = A.dqkv_bf + static_cast<size_t>(m) * ncols;
+  int page = -1;
+  if (j < qn) {
+    page = A.page_table[static_cast<size_t>(b) * A.max_pages_per_seq + (pos >> 4)];
+    if (page < 0 || page >= A.num_pages) { if (threadIdx.x == 0) set_status(A.status, ST_BAD_PAGE); page = -1; }
+  }
+  const size_t page_elems = static_cast<size_t>(A.n_kv) * 16 * HD;
+  for (int h = wp; h < A.n_q + 2 * A.n_kv; h += nw) {
+    const bool is_q = h < A.n_q, is_k = !is_q && h < A.n_q + A.n_kv;
+    const int kvh = is_q ? 0 : (is_k ? h - A.n_q : h - A.n_q - A.n_kv);
+    float *tn = is_q ? (A.tq ? A.tq + (static_cast<size_t>(m) * A.n_q + h) * HD : nullptr)
+                     : (is_k && A.tk ? A.tk + (static_cast<size_t>(m) * A.n_kv + kvh) * HD : nullptr);
+    float g1[EH], g2[EH];
+    if (page < 0) {                                    // padding row (or a page outside the pool): no gradient
+#pragma unroll
+      for (int t = 0; t < EH; ++t) {
+        const int i = lane * EH + t;
+        out[h * HD + i] = 0.f; out[h * HD + HALF + i] = 0.f;
+        outb[h * HD + i] = __float2bfloat16(0.f); outb[h * HD + HALF + i] = __float2bfloat16(0.f);
+        if (tn) { tn[i] = 0.f; tn[HALF + i] = 0.f; }
+      }
+      continue;
+    }
+    const float *src = is_q ? A.dq + (static_cast<size_t>(m) * A.n_q + h) * HD
+                            : (is_k ? A.dk_pool : A.dv_pool) + static_cast<size_t>(page) * page_elems +
+                                  (static_cast<size_t>(kvh) * 16 + (pos & 15)) * HD;
+#pragma unroll
+    for (int t = 0; t < EH; ++t) { g1[t] = src[lane * EH + t]; g2[t] = src[HALF + lane * EH + t]; }
+    if (is_q || is_k) {
+      // the rotation's transpose: turn back by the position's angle
+      const float2 *cs = A.rope + static_cast<size_t>(pos) * HALF;
+#pragma unroll
+      for (int t = 0; t < EH; ++t) {
+        const float2 c = cs[lane * EH + t];
+        const float y1 = g1[t], y2 = g2[t];
+        g1[t] = y1 * c.x + y2 * c.y;
+        g2[t] = y2 * c.x - y1 * c.y;
+      }
+      const __nv_bfloat16 *wn = is_q ? A.qnorm : A.knorm;
+      if (wn) {                                        // y = x0 r w over the head: dx0 = r (w g) - x0 r^3 mean(x0 w g)
+        float x1[EH], x2[EH], w1[EH], w2[EH];
+        float ss = 0.f, dot = 0.f;
+#pragma unroll
+        for (int t = 0; t < EH; ++t) {
+          const int i = lane * EH + t;
+          x1[t] = bf16_to_float(A.qkv[static_cast<size_t>(m) * ncols + h * HD + i]);
+          x2[t] = bf16_to_float(A.qkv[static_cast<size_t>(m) * ncols + h * HD + HALF + i]);
+          if (A.bias) { x1[t] += bf16_to_float(A.bias[h * HD + i]); x2[t] += bf16_to_float(A.bias[h * HD + HALF + i]); }
+          w1[t] = bf16_to_float(wn[i]); w2[t] = bf16_to_float(wn[HALF + i]);
+          ss += x1[t] * x1[t] + x2[t] * x2[t];
+          dot += x1[t] * w1[t] * g1[t] + x2[t] * w2[t] * g2[t];
+        }
+        ss = warp_sum(ss); dot = warp_sum(dot);
+        const float r = rsqrtf(ss / static_cast<float>(HD) + A.eps);
+        const float c3 = r * r * r * dot / static_cast<float>(HD);
+#pragma unroll
+        for (int t = 0; t < EH; ++t) {
+          const int i = lane * EH + t;
+          if (tn) { tn[i] = g1[t] * x1[t] * r; tn[HALF + i] = g2[t] * x2[t] * r; }
+          g1[t] = r * w1[t] * g1[t] - x1[t] * c3;
+          g2[t] = r * w2[t] * g2[t] - x2[t] * c3;
+        }
+      }
+    }
+#pragma unroll
+    for (int t = 0; t < EH; ++t) {
+      const int i = lane * EH + t;
+      out[h * HD + i] = g1[t]; out[h * HD + HALF + i] = g2[t];
+      outb[h * HD + i] = __float2bfloat16(g1[t]); outb[h * HD + HALF + i] = __float2bfloat16(g2[t]);
+    }
+  }
+}
+
 // dst[c][r] = src[r][c] for a row-major bf16 matrix [rows, cols]; 64 x 64 tiles through shared memory.
 __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst, int dst_ld) {
   __shared__ __nv_bfloat16 tile[64][66];
@@ -487,6 +572,11 @@ cudaError_t launch_colsum(const float *t, int rows, int d, float *out, cudaStrea
 cudaError_t launch_cast_bf16(const float *src, __nv_bfloat16 *dst, size_t n, cudaStream_t stream) {
   cast_bf16_kernel<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, stream>>>(src, dst, n / 4);
   return cudaGetLastError();
+}
+cudaError_t launch_qkv_grad_rows(const QkvGradArgs &A, cudaStream_t stream) {
+  if (A.hd == 128) return launch_k(qkv_grad_rows_kernel<2>, dim3(A.batch * A.QT), dim3(256), 0, stream, 1, A);
+  if (A.hd == 64) return launch_k(qkv_grad_rows_kernel<1>, dim3(A.batch * A.QT), dim3(256), 0, stream, 1, A);
+  return cudaErrorInvalidValue;
 }
 cudaError_t launch_swiglu_grad(const __nv_bfloat16 *ab, const float *dh, __nv_bfloat16 *dab, __nv_bfloat16 *h, int rows, int F,
                                cudaStream_t stream) {

@@ -393,6 +393,118 @@ def test_head_input_backward_matches_the_oracle(name, rows, concat):
     ctx.close()
 
 
+@pytest.mark.parametrize("name,family", [("tiny", "plain"), ("tiny", "qkv_bias"), ("tiny", "qk_norm"), ("4b", "qk_norm")],
+                         ids=["tiny-plain", "tiny-qkv_bias", "tiny-qk_norm", "4b_heads-qk_norm"])
+def test_head_attn_backward_matches_the_oracle(name, family):
+    """gm_head_attn_backward against the oracle's backward of the attention half, sequence by sequence: ragged row counts
+    at ragged prefix lengths in shuffled pages, gradient already sitting on every cache entry (the rows of later passes),
+    and two chains of one sequence whose page tables share the prefix pages.  The rows' own cache entries are the oracle's
+    keys / values of those rows rounded to bf16, on both sides."""
+    import paper_2609_16648_b200 as gmb
+    base = get_config("tiny").with_(n_layers=1, qkv_bias=family == "qkv_bias", qk_norm=family == "qk_norm")
+    cfg = base if name == "tiny" else base.with_(d_model=2560, n_q_heads=32, n_kv_heads=8, head_dim=128)
+    d, hd, n_q, n_kv, NQ, NKV = cfg.d_model, cfg.head_dim, cfg.n_q_heads, cfg.n_kv_heads, cfg.q_dim, cfg.kv_dim
+    QT = 4
+    lens = np.array([0, 15, 40, 333, 77, 77])
+    B = len(lens)
+    rng = np.random.default_rng(17)
+    counts = np.array([QT, 1, 3, 2, QT, QT], np.int32)
+    total = lens + counts
+    pt, npg = make_page_tables(total, 16, seed=4, slack_pages=2)
+    shared = lens[-1] // 16
+    pt[-1, :shared] = pt[-2, :shared]
+    ctx = gmb.Context(cfg, gmb.random_packed_weights(cfg, "cuda"), B, QT - 1, pt.shape[1], 8, npg)
+    g = torch.Generator(device="cuda").manual_seed(5)
+    hl = ctx.packed["head"]["layer"]
+    pert = lambda n: (1 + (torch.rand(n, device="cuda", generator=g) - 0.5) * 0.5).to(torch.bfloat16)
+    hl["ln1"].copy_(pert(d))
+    for key in ("wqkv", "wo"):                                   # larger than the init scale, so that the block's path matters
+        hl[key].copy_((torch.randn(hl[key].shape, device="cuda", generator=g) * (1.5 / np.sqrt(hl[key].shape[1]))).to(torch.bfloat16))
+    if cfg.qkv_bias:
+        hl["b_qkv"].copy_((torch.randn(NQ + 2 * NKV, device="cuda", generator=g) * 0.3).to(torch.bfloat16))
+    if cfg.qk_norm:
+        hl["q_norm"].copy_(pert(hd)); hl["k_norm"].copy_(pert(hd))
+    f = lambda t: t.double().cpu().numpy()
+    wqkv = f(hl["wqkv"])
+    lw = {"ln1": f(hl["ln1"]), "wq": wqkv[:NQ], "wk": wqkv[NQ:NQ + NKV], "wv": wqkv[NQ + NKV:], "wo": f(hl["wo"])}
+    if cfg.qkv_bias:
+        bq = f(hl["b_qkv"])
+        lw.update(bq=bq[:NQ], bk=bq[NQ:NQ + NKV], bv=bq[NQ + NKV:])
+    if cfg.qk_norm:
+        lw.update(qnorm=f(hl["q_norm"]), knorm=f(hl["k_norm"]))
+    x = rng.normal(0, 1.5, (B, QT, d)).astype(np.float32)
+    dxmid = rng.normal(0, 0.1, (B, QT, d)).astype(np.float32)
+    pool = np.zeros((1, 2, npg, n_kv, 16, hd), np.float32)
+    dk0 = np.zeros((npg, n_kv, 16, hd), np.float32)
+    dv0 = np.zeros_like(dk0)
+    kcs, vcs = [], []
+    for b in range(B):
+        S, n = int(total[b]), int(counts[b])
+        dxmid[b, n:] = 0
+        pos = lens[b] + np.arange(n)
+        kc = omodel.round_bf16(rng.standard_normal((S, n_kv, hd))).astype(np.float64)
+        vc = omodel.round_bf16(rng.standard_normal((S, n_kv, hd))).astype(np.float64)
+        if b == B - 1:
+            kc[:shared * 16], vc[:shared * 16] = kcs[-1][:shared * 16], vcs[-1][:shared * 16]
+        _, k_own, v_own = omodel.project_qkv(lw, omodel.rmsnorm(x[b, :n], lw["ln1"], cfg.rms_eps), cfg)
+        kc[pos] = omodel.round_bf16(omodel.rope(k_own, pos, cfg.rope_base))
+        vc[pos] = omodel.round_bf16(v_own)
+        idx = np.arange(S)
+        pool[0, 0, pt[b, idx // 16], :, idx % 16, :] = kc
+        pool[0, 1, pt[b, idx // 16], :, idx % 16, :] = vc
+        dk0[pt[b, idx // 16], :, idx % 16, :] = rng.normal(0, 0.02, (S, n_kv, hd))
+        dv0[pt[b, idx // 16], :, idx % 16, :] = rng.normal(0, 0.02, (S, n_kv, hd))
+        kcs.append(kc); vcs.append(vc)
+    dev = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(device="cuda", dtype=dt)
+    z = lambda *shape: torch.full(shape, 7.0, dtype=torch.float32, device="cuda")
+    dkp, dvp = dev(dk0, torch.float32), dev(dv0, torch.float32)
+    dx, dwqkv, dwo, dln1 = z(B * QT, d), z(NQ + 2 * NKV, d), z(d, NQ), z(d)
+    dbias = z(NQ + 2 * NKV) if cfg.qkv_bias else None
+    dqkn = z(2 * hd) if cfg.qk_norm else None
+    args = (ctx, dev(x.reshape(B * QT, d), torch.float32), dev(dxmid.reshape(B * QT, d), torch.float32), dev(pool, torch.bfloat16),
+            dev(np.where(pt < 0, 0, pt), torch.int32), dev(counts, torch.int32), dev(lens.astype(np.int32), torch.int32), B, QT)
+    pool_before = args[3].clone()
+    gmb.gm_head_attn_backward(*args, dkp, dvp, dx, dwqkv, dwo, dln1, dbias, dqkn)
+    assert gmb.gm_last_status(ctx) == 0
+    assert torch.equal(args[3], pool_before)                                # the cache is read, not rewritten
+    want = {}
+    want_dk, want_dv = dk0.astype(np.float64), dv0.astype(np.float64)
+    got_dx = f(dx).reshape(B, QT, d)
+    tol = 2.5e-2
+    for b in range(B):
+        S, n = int(total[b]), int(counts[b])
+        idx = np.arange(S)
+        pg, sl = pt[b, idx // 16], idx % 16
+        dkc, dvc = dk0[pg, :, sl, :].astype(np.float64), dv0[pg, :, sl, :].astype(np.float64)
+        before_k, before_v = dkc.copy(), dvc.copy()
+        out = oupdate.attention_block_grad(dxmid[b, :n], x[b, :n], lw, lens[b] + np.arange(n), kcs[b], vcs[b], dkc, dvc, cfg)
+        np.add.at(want_dk, (pg, slice(None), sl), dkc - before_k)
+        np.add.at(want_dv, (pg, slice(None), sl), dvc - before_v)
+        assert rel_err(got_dx[b, :n], out["dx"]) < tol, b
+        assert rel_err(got_dx[b, :n] - dxmid[b, :n], out["dx"] - dxmid[b, :n]) < tol, b       # the attention half's own path
+        assert (got_dx[b, n:] == 0).all()
+        for key, val in out.items():
+            if key != "dx":
+                want[key] = want.get(key, 0.0) + val
+    # what this pass added to the planes (the device rounds the queries, the attention output's gradient enters in fp32)
+    assert rel_err(f(dkp) - dk0, want_dk - dk0) < tol and rel_err(f(dvp) - dv0, want_dv - dv0) < tol
+    assert np.abs((want_dk - dk0)[pt[-2, :shared]]).max() > 0                      # the shared prefix pages collected terms
+    got_w = f(dwqkv)
+    assert rel_err(got_w[:NQ], want["dwq"]) < tol and rel_err(got_w[NQ:NQ + NKV], want["dwk"]) < tol
+    assert rel_err(got_w[NQ + NKV:], want["dwv"]) < tol
+    assert rel_err(f(dwo), want["dwo"]) < tol and rel_err(f(dln1), want["dln1"]) < tol
+    if cfg.qkv_bias:
+        assert rel_err(f(dbias), np.concatenate([want["dbq"], want["dbk"], want["dbv"]])) < tol
+    if cfg.qk_norm:
+        assert rel_err(f(dqkn)[:hd], want["dqnorm"]) < tol and rel_err(f(dqkn)[hd:], want["dknorm"]) < tol
+    for key in ("dwq", "dwk", "dwv", "dwo", "dln1"):
+        assert np.abs(want[key]).max() > 0
+    # a layer's optional outputs must be asked for exactly when the layer has them
+    with pytest.raises(RuntimeError):
+        gmb.gm_head_attn_backward(*args, dkp, dvp, dx, dwqkv, dwo, dln1, None if cfg.qkv_bias else z(NQ + 2 * NKV), dqkn)
+    ctx.close()
+
+
 @pytest.mark.parametrize("n", [1003, 49_807_360], ids=["ragged_1003", "gate_up_of_the_4b_head"])
 def test_adamw_step_matches_the_oracle(n):
     """gm_adamw_step over several updates with the head's schedule against the oracle's fp64 AdamW (sampled entries at the
