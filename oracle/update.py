@@ -336,15 +336,18 @@ def _accumulate(total: dict, part: dict, names) -> None:
             total[name] = total.get(name, 0.0) + part[name]
 
 
-def head_update_grad(w, cfg, sequences, records, temperature: float = 1.0) -> dict:
+def head_update_grad(w, cfg, sequences, records, temperature: float = 1.0, grad_logits=None) -> dict:
     """Gradient of head_update_loss (no rounding at the logits interface) with respect to every parameter of the head.
-    Same arguments as head_update_loss.  Returns {"proj", "enorm", "hnorm", "final_norm", "layer": {"ln1", "wq", "wk",
+    Same arguments as head_update_loss.  grad_logits [n_records, K, V], if given, replaces the objective's own
+    d(mean loss)/d(logits) (first step of the backward pass) and everything downstream of it is computed as usual - for
+    checking a pipeline whose reconstructed logits differ from these in rounding, where the piecewise-linear overlap
+    would pick other branches.  Returns {"proj", "enorm", "hnorm", "final_norm", "layer": {"ln1", "wq", "wk",
     "wv", "wo", "ln2", "wg", "wu", "wd" [, "bq", "bk", "bv"] [, "qnorm", "knorm"]}} in float64; the embedding table
     and the LM head are the backbone's and get none."""
     hw, lw = w["head"], w["head"]["layer"]
     top, lay = {}, {}
     n_rec = len(records)
-    for s, rec in records:
+    for r_i, (s, rec) in enumerate(records):
         hid, toks = sequences[s]
         Len, drafts = int(rec["start_pos"]), rec["drafts"]
         K = len(drafts)
@@ -361,8 +364,12 @@ def head_update_grad(w, cfg, sequences, records, temperature: float = 1.0) -> di
         states = np.array(states)
         kc, vc = hkv.gather(0, 0, Len + K - 2)
         # the term of every state through its own logits
-        dstate, gy, _ = head_update_grad_state(w, cfg, states[None], [rec], temperature)
-        dstate, gy = dstate[0] / n_rec, gy[0] / n_rec
+        if grad_logits is None:
+            dstate, gy, _ = head_update_grad_state(w, cfg, states[None], [rec], temperature)
+            dstate, gy = dstate[0] / n_rec, gy[0] / n_rec
+        else:
+            gy = lm_head_input_grad(grad_logits[r_i], w["lm_head"])
+            dstate = rmsnorm_grad(gy, states, hw["final_norm"], cfg.rms_eps)
         top["final_norm"] = top.get("final_norm", 0.0) + _rms_weight_grad(gy, states, cfg.rms_eps)
         # backward, last application first
         dkc, dvc = np.zeros_like(kc), np.zeros_like(vc)

@@ -456,3 +456,20 @@ def test_head_update_gradient_matches_finite_differences_of_the_objective(family
     for (_, a), d in zip(params, dirs):
         a += h * d
     assert expect == pytest.approx((hi - lo) / (2 * h), rel=2e-4)
+
+
+def test_head_update_gradient_with_given_logit_gradients_is_the_same_chain():
+    """Handing head_update_grad the objective's own logit gradients reproduces the default; the result is linear in them."""
+    w, st, cycles = _rollout_with_records(rounding=False, n_steps=2)
+    seqs = _sequence_features(w, st, rounding=False)
+    recs = [(b, dict(rec, accepted=i % 4 + 1)) for i, (b, rec, _, _) in enumerate(cycles)]
+    base = update.head_update_grad(w, CFG, seqs, recs, T)
+    lgs = np.array([update.reconstruct_chain(w, CFG, seqs[b][0], seqs[b][1], r["start_pos"], r["drafts"], T, False)[1] for b, r in recs])
+    gl = update.head_update_grad_logits(lgs, [r for _, r in recs], T)
+    same = update.head_update_grad(w, CFG, seqs, recs, T, grad_logits=gl)
+    twice = update.head_update_grad(w, CFG, seqs, recs, T, grad_logits=2 * gl)
+    for name in ("proj", "final_norm"):
+        np.testing.assert_allclose(same[name], base[name], rtol=1e-9, atol=1e-14)
+        np.testing.assert_allclose(twice[name], 2 * base[name], rtol=1e-9, atol=1e-14)
+    for name in base["layer"]:
+        np.testing.assert_allclose(same["layer"][name], base["layer"][name], rtol=1e-9, atol=1e-14)
