@@ -452,6 +452,41 @@ int gm_head_attn_backward(gm_ctx *ctx, const float *x, const float *dxmid, const
                           const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch, int q_stride,
                           float *dk_pool, float *dv_pool, float *dx, float *dw_qkv, float *dw_o, float *dln1, float *db_qkv,
                           float *dqk_norm, int refresh_weights);
+/* The whole backward pass of the head update over recorded cycles (Alg. 1, "update phi"; Eq. 4-9): the gradient of the
+ * mean objective with respect to every parameter of the head, given its gradient with respect to the reconstructed
+ * logits.  Call order: gm_head_prefill and gm_reconstruct / gm_reconstruct_states (the head's cache over the committed
+ * prefixes, the chains' logits), gm_overlap + gm_dca_grad (grad_logits), then this call with the SAME state, cycles,
+ * record, tokens and scratch pages.  It replays the chains a chunk of max_batch at a time (the states they produce are
+ * the forward pass's, the kernels being deterministic), takes every application from the last draft back to the
+ * first through gm_head_state_grad, gm_head_ffn_backward, gm_head_attn_backward and gm_head_input_backward - a state's
+ * gradient collecting the term through its own logits and the term through the next application's input, a cache
+ * entry's gradient collecting the terms of every later row that read it - moves what the chains left on the copied
+ * part of their private boundary pages to the shared originals, and finishes with the pass over the committed prefixes,
+ * whose rows receive gradient only through their cache entries.
+ *   grad_logits       device bf16 [n_cycles, k, vocab] (gm_dca_grad)
+ *   seq_hidden, hid_stride, seq_len, max_len, seq_tok, tok_stride   as in gm_head_prefill / gm_reconstruct
+ *   dk_pool, dv_pool  device fp32 [head_num_pages][n_kv][16][head_dim] scratch (zeroed here; on return the gradient of
+ *                     every head-cache entry, shared prefix pages and private chain pages alike)
+ *   out               device fp32 buffers, overwritten with the sums over all cycles
+ * Uses the context's cycle workspaces (not to be interleaved with a cycle in flight); scratch for the passes and
+ * transposed copies of the head's matrices are allocated on first use and kept until gm_free.
+ * Limits: those of the four operators (d, q_dim, n_qkv, F multiples of 64; head_dim 64 / 128; group <= 8; no
+ * GM_FLAG_SIMPLE_GEMM): GM_ERR_UNSUPPORTED.  An optional output (b_qkv, qk_norm) must be given iff the layer has it.   */
+typedef struct {
+  float *proj;                      /* [d, 2 d]   packed order [embedding ; hidden]                                     */
+  float *enorm, *hnorm, *final_norm;/* [d] each                                                                          */
+  float *ln1, *ln2;                 /* [d] each                                                                          */
+  float *wqkv;                      /* [(n_q + 2 n_kv) head_dim, d]                                                       */
+  float *wo;                        /* [d, n_q head_dim]                                                                  */
+  float *w_gate_up;                 /* [2 F, d]   rows interleaved like the packed weight                                 */
+  float *w_down;                    /* [d, F]                                                                             */
+  float *b_qkv;                     /* [(n_q + 2 n_kv) head_dim] or NULL                                                  */
+  float *qk_norm;                   /* [2 head_dim] (query norm, key norm) or NULL                                        */
+} gm_head_grads;
+int gm_head_update_backward(gm_ctx *ctx, gm_state *st, int n_cycles, int k, const int32_t *cycle_seq, const gm_record *rec,
+                            const int32_t *seq_tok, int tok_stride, const int32_t *scratch_pages, const void *grad_logits,
+                            const void *seq_hidden, int hid_stride, const int32_t *seq_len, int max_len, float *dk_pool,
+                            float *dv_pool, const gm_head_grads *out);
 /* Fourth step of the backward pass: through the head's input (App. B.1),
  *   z = W_p [RMSNorm(E[token]; enorm) ; RMSNorm(hidden; hnorm)]   (the order the packed projection uses).
  *   tokens int32 [rows], hidden fp32 [rows, d]: the pairs that entered;  dz fp32 [rows, d] = dL/dz (device)

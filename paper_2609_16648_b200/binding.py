@@ -24,7 +24,7 @@ GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER, GM_KC_RECORD = 0,
 
 EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw", "gm_set_top_p", "gm_nucleus", "gm_prefill",
            "gm_rollout_begin", "gm_rollout_step", "gm_rollout_run", "gm_pages_reset", "gm_pages_reserve",
-           "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_reconstruct_states", "gm_head_state_grad", "gm_head_ffn_backward", "gm_attention_backward", "gm_head_attn_backward", "gm_head_input_backward", "gm_adamw_step", "gm_overlap", "gm_dca_loss", "gm_dca_grad",
+           "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_reconstruct_states", "gm_head_state_grad", "gm_head_ffn_backward", "gm_attention_backward", "gm_head_attn_backward", "gm_head_update_backward", "gm_head_input_backward", "gm_adamw_step", "gm_overlap", "gm_dca_loss", "gm_dca_grad",
            "gm_spec_step_host", "gm_gemm", "gm_gemm_swiglu", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
            "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_chain_trace", "gm_chain_trace_read", "gm_selftest_wait_expiry", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
@@ -63,6 +63,13 @@ class gm_record(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("start_hidden", "start_pos", "drafts", "top_logprob", "top_index", "accepted")]
 
 
+HEAD_GRAD_FIELDS = ("proj", "enorm", "hnorm", "final_norm", "ln1", "ln2", "wqkv", "wo", "w_gate_up", "w_down", "b_qkv", "qk_norm")
+
+
+class gm_head_grads(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in HEAD_GRAD_FIELDS]
+
+
 _lib = None
 
 
@@ -99,6 +106,8 @@ def lib() -> C.CDLL:
     L.gm_head_ffn_backward.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, i32]
     L.gm_attention_backward.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp]
     L.gm_head_attn_backward.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32]
+    L.gm_head_update_backward.argtypes = [vp, C.POINTER(gm_state), i32, i32, vp, C.POINTER(gm_record), vp, i32, vp, vp, vp, i32, vp, i32, vp,
+                                          vp, C.POINTER(gm_head_grads)]
     L.gm_head_input_backward.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, i32]
     L.gm_adamw_step.argtypes = [vp, C.c_int64, vp, vp, vp, vp, vp, i32, f32, f32, f32, f32, f32, f32]
     L.gm_overlap.argtypes = [vp, i32, i32, f32, vp, C.POINTER(gm_record), vp, vp]
@@ -430,6 +439,29 @@ def gm_head_attn_backward(ctx: Context, x, dxmid, kv_pool, page_table, q_count, 
     _check(lib().gm_head_attn_backward(ctx.handle, _p(x), _p(dxmid), _p(kv_pool), kv_pool.shape[2], _p(page_table), _p(q_count),
                                        _p(q_base), batch, q_stride, _p(dk_pool), _p(dv_pool), _p(dx), _p(dw_qkv), _p(dw_o),
                                        _p(dln1), _p(db_qkv), _p(dqk_norm), int(refresh_weights)), "gm_head_attn_backward")
+
+
+def head_grad_buffers(cfg, device="cuda") -> dict:
+    """fp32 device buffers for every parameter of the head, in the shapes gm_head_update_backward fills."""
+    d, f, nqkv = cfg.d_model, cfg.d_ffn, cfg.q_dim + 2 * cfg.kv_dim
+    z = lambda *shape: torch.zeros(shape, dtype=torch.float32, device=device)
+    g = {"proj": z(d, 2 * d), "enorm": z(d), "hnorm": z(d), "final_norm": z(d), "ln1": z(d), "ln2": z(d), "wqkv": z(nqkv, d),
+         "wo": z(d, cfg.q_dim), "w_gate_up": z(2 * f, d), "w_down": z(d, f)}
+    if getattr(cfg, "qkv_bias", False):
+        g["b_qkv"] = z(nqkv)
+    if getattr(cfg, "qk_norm", False):
+        g["qk_norm"] = z(2 * cfg.head_dim)
+    return g
+
+
+def gm_head_update_backward(ctx: Context, st: State, n_cycles: int, k: int, cycle_seq, rec, seq_tok, scratch_pages, grad_logits,
+                            seq_hidden, seq_len, max_len: int, dk_pool, dv_pool, grads: dict):
+    """grads: head_grad_buffers(cfg); overwritten with the gradient of the mean objective."""
+    gs = gm_head_grads(*[_p(grads.get(n)) for n in HEAD_GRAD_FIELDS])
+    _check(lib().gm_head_update_backward(ctx.handle, C.byref(st.struct()), n_cycles, k, _p(cycle_seq), C.byref(rec.struct()),
+                                         _p(seq_tok), seq_tok.shape[1], _p(scratch_pages), _p(grad_logits), _p(seq_hidden),
+                                         seq_hidden.shape[1], _p(seq_len), max_len, _p(dk_pool), _p(dv_pool), C.byref(gs)),
+           "gm_head_update_backward")
 
 
 def gm_head_input_backward(ctx: Context, rows: int, tokens, hidden, dz, dhidden, dproj, denorm, dhnorm, refresh_weights: bool = False):

@@ -121,9 +121,11 @@ int gm_head_state_grad(gm_ctx *c, int rows, const void *grad_logits, const float
   return GM_OK;
 }
 
-int gm_head_ffn_backward(gm_ctx *c, int rows, const float *x, const float *dg, float *dx, float *dw_gate_up, float *dw_down,
-                         float *dln2, int refresh_weights) {
+// accum: the parameter gradients are added to what the output buffers hold (a pass among several) instead of stored
+static int head_ffn_backward_impl(gm_ctx *c, int rows, const float *x, const float *dg, float *dx, float *dw_gate_up, float *dw_down,
+                                  float *dln2, int refresh_weights, bool accum) {
   if (!c || rows < 1 || !x || !dg || !dx || !dw_gate_up || !dw_down || !dln2) return GM_ERR_INVALID_ARG;
+  const int wepi = accum ? EPI_ADD_F32 : EPI_STORE_F32;
   const int d = c->d, F = c->F;
   if ((c->cfg.flags & GM_FLAG_SIMPLE_GEMM) || (d % 64) || (F % 64)) return GM_ERR_UNSUPPORTED;
   const gm_layer_weights &lw = c->w.head_layer;
@@ -172,7 +174,7 @@ int gm_head_ffn_backward(gm_ctx *c, int rows, const float *x, const float *dg, f
   if ((rc = run_gemm(c, c->ffn_dab, rows, &c->ffn_wgu_t_map, c->ffn_wgu_t, rows, d, 2 * F, c->ffn_du, EPI_STORE_F32, static_cast<size_t>(d), false)) != GM_OK)
     return rc;
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rmsnorm_grad(c->ffn_du, x, ln2, dx, rows, d, c->cfg.rms_eps, c->stream, dg, c->ffn_t));
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->ffn_t, rows, d, dln2, c->stream));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->ffn_t, rows, d, dln2, c->stream, accum));
   // weight gradients contract over the rows: both operands transposed to [features, rows] (rows padded with zeros to Mp)
   GM_CUDA(c, cudaMemsetAsync(c->ffn_ut, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
   GM_CUDA(c, cudaMemsetAsync(c->ffn_dyt, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
@@ -185,10 +187,14 @@ int gm_head_ffn_backward(gm_ctx *c, int rows, const float *x, const float *dg, f
   CUtensorMap wm;
   // dW_d [d, F] = dg^T h
   if (make_map(c, &wm, c->ffn_ht, F, Mp, 128) != GM_OK) return GM_ERR_CUDA;
-  if ((rc = run_gemm(c, c->ffn_dyt, d, &wm, c->ffn_ht, d, F, Mp, dw_down, EPI_STORE_F32, static_cast<size_t>(F), false)) != GM_OK) return rc;
+  if ((rc = run_gemm(c, c->ffn_dyt, d, &wm, c->ffn_ht, d, F, Mp, dw_down, wepi, static_cast<size_t>(F), false)) != GM_OK) return rc;
   // dW_gu [2F, d] = (da, db)^T u   (rows interleaved like the packed weight)
   if (make_map(c, &wm, c->ffn_ut, d, Mp, 128) != GM_OK) return GM_ERR_CUDA;
-  return run_gemm(c, c->ffn_dabt, 2 * F, &wm, c->ffn_ut, 2 * F, d, Mp, dw_gate_up, EPI_STORE_F32, static_cast<size_t>(d), false);
+  return run_gemm(c, c->ffn_dabt, 2 * F, &wm, c->ffn_ut, 2 * F, d, Mp, dw_gate_up, wepi, static_cast<size_t>(d), false);
+}
+int gm_head_ffn_backward(gm_ctx *c, int rows, const float *x, const float *dg, float *dx, float *dw_gate_up, float *dw_down,
+                         float *dln2, int refresh_weights) {
+  return head_ffn_backward_impl(c, rows, x, dg, dx, dw_gate_up, dw_down, dln2, refresh_weights, false);
 }
 
 int gm_adamw_step(gm_ctx *c, int64_t n, float *master, void *param_bf16, const float *grad, float *m, float *v, int step, float lr,
@@ -207,9 +213,10 @@ int gm_adamw_step(gm_ctx *c, int64_t n, float *master, void *param_bf16, const f
   return GM_OK;
 }
 
-int gm_head_input_backward(gm_ctx *c, int rows, const int32_t *tokens, const float *hidden, const float *dz, float *dhidden,
-                           float *dproj, float *denorm, float *dhnorm, int refresh_weights) {
-  if (!c || rows < 1 || !tokens || !hidden || !dz || !dhidden || !dproj || !denorm || !dhnorm) return GM_ERR_INVALID_ARG;
+// dhidden may be null here (rows whose hidden state is a recorded input, not a head state)
+static int head_input_backward_impl(gm_ctx *c, int rows, const int32_t *tokens, const float *hidden, const float *dz, float *dhidden,
+                                    float *dproj, float *denorm, float *dhnorm, int refresh_weights, bool accum) {
+  if (!c || rows < 1 || !tokens || !hidden || !dz || !dproj || !denorm || !dhnorm) return GM_ERR_INVALID_ARG;
   const int d = c->d;
   if ((c->cfg.flags & GM_FLAG_SIMPLE_GEMM) || (d % 64)) return GM_ERR_UNSUPPORTED;
   const __nv_bfloat16 *proj = static_cast<const __nv_bfloat16 *>(c->w.head_proj);
@@ -246,10 +253,10 @@ int gm_head_input_backward(gm_ctx *c, int rows, const int32_t *tokens, const flo
   // through the two norms: the hidden half gives dL/d hidden and dL/d hnorm, the embedding half only dL/d enorm
   GM_LAUNCH(c, GM_KC_ELEMENTWISE,
             launch_rmsnorm_grad(c->hin_dzin + d, hidden, wh, dhidden, rows, d, c->cfg.rms_eps, c->stream, nullptr, c->hin_t, 2 * d));
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hin_t, rows, d, dhnorm, c->stream));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hin_t, rows, d, dhnorm, c->stream, accum));
   GM_LAUNCH(c, GM_KC_ELEMENTWISE,
             launch_rmsnorm_grad(c->hin_dzin, c->hin_e, we, nullptr, rows, d, c->cfg.rms_eps, c->stream, nullptr, c->hin_t, 2 * d));
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hin_t, rows, d, denorm, c->stream));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hin_t, rows, d, denorm, c->stream, accum));
   // dW_p [d, 2d] = dz^T zin: both operands transposed to [features, rows] (rows padded with zeros to Mp)
   GM_CUDA(c, cudaMemsetAsync(c->hin_dzt, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
   GM_CUDA(c, cudaMemsetAsync(c->hin_zint, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * 2 * d, c->stream));
@@ -257,7 +264,12 @@ int gm_head_input_backward(gm_ctx *c, int rows, const int32_t *tokens, const flo
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->hin_zin, rows, 2 * d, c->hin_zint, c->stream, Mp));
   CUtensorMap wm;
   if (make_map(c, &wm, c->hin_zint, 2 * d, Mp, 128) != GM_OK) return GM_ERR_CUDA;
-  return run_gemm(c, c->hin_dzt, d, &wm, c->hin_zint, d, 2 * d, Mp, dproj, EPI_STORE_F32, 2 * static_cast<size_t>(d), false);
+  return run_gemm(c, c->hin_dzt, d, &wm, c->hin_zint, d, 2 * d, Mp, dproj, accum ? EPI_ADD_F32 : EPI_STORE_F32, 2 * static_cast<size_t>(d), false);
+}
+int gm_head_input_backward(gm_ctx *c, int rows, const int32_t *tokens, const float *hidden, const float *dz, float *dhidden,
+                           float *dproj, float *denorm, float *dhnorm, int refresh_weights) {
+  if (!dhidden) return GM_ERR_INVALID_ARG;
+  return head_input_backward_impl(c, rows, tokens, hidden, dz, dhidden, dproj, denorm, dhnorm, refresh_weights, false);
 }
 
 int gm_attention_backward(gm_ctx *c, const void *q, const float *dout, const void *kv_pool, int pool_layers, int num_pages, int layer,
@@ -285,11 +297,56 @@ int gm_attention_backward(gm_ctx *c, const void *q, const float *dout, const voi
   return GM_OK;
 }
 
-int gm_head_attn_backward(gm_ctx *c, const float *x, const float *dxmid, const void *kv_pool, int num_pages,
-                          const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch, int q_stride,
-                          float *dk_pool, float *dv_pool, float *dx, float *dw_qkv, float *dw_o, float *dln1, float *db_qkv,
-                          float *dqk_norm, int refresh_weights) {
-  if (!c || !x || !dxmid || !kv_pool || !page_table || !q_count || !q_base || !dk_pool || !dv_pool || !dx || !dw_qkv || !dw_o ||
+// The attention half's forward values for one pass of rows x [batch * q_stride, d], with the forward pass's own kernels:
+// c->xn = RMSNorm(x; ln1), c->qkv = the projection, and - with_attention - c->qbuf = the rotated (normed, biased) queries,
+// c->attn_out = the attention output over the given cache, which is only read.  Leaves the plan (c->qn, c->qbase) in place.
+static int head_attn_forward(gm_ctx *c, const float *x, const void *kv_pool, int num_pages, const int32_t *page_table,
+                             const int32_t *q_count, const int32_t *q_base, int batch, int q_stride, bool with_attention) {
+  const gm_config &cf = c->cfg;
+  const gm_layer_weights &lw = c->w.head_layer;
+  const int d = c->d, hd = cf.head_dim, NQKV = c->n_qkv, rows = batch * q_stride;
+  int rc;
+  if ((rc = run_plan_chunk(c, batch, q_count, q_base, q_stride)) != GM_OK) return rc;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+            launch_rmsnorm(x, static_cast<const __nv_bfloat16 *>(lw.ln1), c->xn, nullptr, rows, d, cf.rms_eps, c->stream));
+  if ((rc = run_gemm(c, c->xn, c->Mmax, &c->head_maps.wqkv, static_cast<const __nv_bfloat16 *>(lw.wqkv), rows, NQKV, d, c->qkv,
+                     EPI_STORE_BF16, NQKV)) != GM_OK)
+    return rc;
+  if (!with_attention) return GM_OK;
+  const int qrows = round16(q_stride * c->group);
+  RopeAppendArgs R;
+  R.qkv = c->qkv; R.batch = batch; R.QT = q_stride; R.n_q = cf.n_q_heads; R.n_kv = cf.n_kv_heads; R.hd = hd; R.layer = 0;
+  R.num_pages = num_pages; R.max_pages_per_seq = cf.max_pages_per_seq; R.qrows = qrows; R.qn = c->qn; R.qbase = c->qbase;
+  R.page_table = page_table; R.rope = c->rope; R.qbuf = c->qbuf; R.pool = nullptr; R.status = c->status;   // the cache is read, not rewritten
+  R.bias = static_cast<const __nv_bfloat16 *>(lw.b_qkv);
+  R.qnorm = static_cast<const __nv_bfloat16 *>(lw.q_norm); R.knorm = static_cast<const __nv_bfloat16 *>(lw.k_norm);
+  R.eps = cf.rms_eps;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rope_append(R, c->stream));
+  CUtensorMap kvm;
+  if ((rc = kv_map(c, kv_pool, 1, num_pages, &kvm)) != GM_OK) return rc;
+  AttnArgs T;
+  T.kv_map = kvm; T.qbuf = c->qbuf; T.qn = c->qn; T.qbase = c->qbase; T.page_start = c->page_start; T.page_table = page_table;
+  T.batch = batch; T.n_kv = cf.n_kv_heads; T.group = c->group; T.hd = hd; T.qrows = qrows; T.layer = 0; T.num_pages = num_pages;
+  T.max_pages_per_seq = cf.max_pages_per_seq; T.n_ctas = c->sm_count;
+  T.scale_log2e = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(hd)));
+  T.part_o = c->part_o; T.part_ml = c->part_ml; T.status = c->status; T.rows_used = q_stride * c->group;
+  GM_LAUNCH(c, GM_KC_ATTENTION, launch_attention(T, c->stream));
+  AttnCombineArgs Cb;
+  Cb.part_o = c->part_o; Cb.part_ml = c->part_ml; Cb.qn = c->qn; Cb.page_start = c->page_start; Cb.batch = batch;
+  Cb.n_kv = cf.n_kv_heads; Cb.group = c->group; Cb.hd = hd; Cb.qrows = qrows; Cb.QT = q_stride; Cb.n_ctas = c->sm_count;
+  Cb.out = c->attn_out;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_attention_combine(Cb, c->stream));
+  return GM_OK;
+}
+
+// dxmid may be null here: rows whose outputs nothing consumed (the pass over the committed prefix) - only what later rows
+// left on their cache entries flows back, the attention core and W_o are skipped and dw_o is left as it is
+static int head_attn_backward_impl(gm_ctx *c, const float *x, const float *dxmid, const void *kv_pool, int num_pages,
+                                   const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch, int q_stride,
+                                   float *dk_pool, float *dv_pool, float *dx, float *dw_qkv, float *dw_o, float *dln1, float *db_qkv,
+                                   float *dqk_norm, int refresh_weights, bool accum, bool forward_done = false) {
+  const int wepi = accum ? EPI_ADD_F32 : EPI_STORE_F32;
+  if (!c || !x || !kv_pool || !page_table || !q_count || !q_base || !dk_pool || !dv_pool || !dx || !dw_qkv || !dw_o ||
       !dln1 || batch < 1 || q_stride < 1 || num_pages < 1)
     return GM_ERR_INVALID_ARG;
   const gm_config &cf = c->cfg;
@@ -332,32 +389,12 @@ int gm_head_attn_backward(gm_ctx *c, const float *x, const float *dxmid, const v
     c->hat_rows_cap = Mp;
   }
   // ---- the forward's values, recomputed: h = RMSNorm(x; ln1), the projection, the rotated queries, the attention output ----
-  if ((rc = run_plan_chunk(c, batch, q_count, q_base, q_stride)) != GM_OK) return rc;
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rmsnorm(x, ln1, c->xn, nullptr, rows, d, cf.rms_eps, c->stream));
-  if ((rc = run_gemm(c, c->xn, c->Mmax, &c->head_maps.wqkv, wqkv, rows, NQKV, d, c->qkv, EPI_STORE_BF16, NQKV)) != GM_OK) return rc;
-  const int qrows = round16(q_stride * c->group);
-  RopeAppendArgs R;
-  R.qkv = c->qkv; R.batch = batch; R.QT = q_stride; R.n_q = cf.n_q_heads; R.n_kv = cf.n_kv_heads; R.hd = hd; R.layer = 0;
-  R.num_pages = num_pages; R.max_pages_per_seq = cf.max_pages_per_seq; R.qrows = qrows; R.qn = c->qn; R.qbase = c->qbase;
-  R.page_table = page_table; R.rope = c->rope; R.qbuf = c->qbuf; R.pool = nullptr; R.status = c->status;   // the cache is read, not rewritten
-  R.bias = static_cast<const __nv_bfloat16 *>(lw.b_qkv);
-  R.qnorm = static_cast<const __nv_bfloat16 *>(lw.q_norm); R.knorm = static_cast<const __nv_bfloat16 *>(lw.k_norm);
-  R.eps = cf.rms_eps;
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rope_append(R, c->stream));
-  CUtensorMap kvm;
-  if ((rc = kv_map(c, kv_pool, 1, num_pages, &kvm)) != GM_OK) return rc;
-  AttnArgs T;
-  T.kv_map = kvm; T.qbuf = c->qbuf; T.qn = c->qn; T.qbase = c->qbase; T.page_start = c->page_start; T.page_table = page_table;
-  T.batch = batch; T.n_kv = cf.n_kv_heads; T.group = c->group; T.hd = hd; T.qrows = qrows; T.layer = 0; T.num_pages = num_pages;
-  T.max_pages_per_seq = cf.max_pages_per_seq; T.n_ctas = c->sm_count;
-  T.scale_log2e = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(hd)));
-  T.part_o = c->part_o; T.part_ml = c->part_ml; T.status = c->status; T.rows_used = q_stride * c->group;
-  GM_LAUNCH(c, GM_KC_ATTENTION, launch_attention(T, c->stream));
-  AttnCombineArgs Cb;
-  Cb.part_o = c->part_o; Cb.part_ml = c->part_ml; Cb.qn = c->qn; Cb.page_start = c->page_start; Cb.batch = batch;
-  Cb.n_kv = cf.n_kv_heads; Cb.group = c->group; Cb.hd = hd; Cb.qrows = qrows; Cb.QT = q_stride; Cb.n_ctas = c->sm_count;
-  Cb.out = c->attn_out;
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_attention_combine(Cb, c->stream));
+  if (!forward_done &&
+      (rc = head_attn_forward(c, x, kv_pool, num_pages, page_table, q_count, q_base, batch, q_stride, dxmid != nullptr)) != GM_OK)
+    return rc;
+  const __nv_bfloat16 *bias = static_cast<const __nv_bfloat16 *>(lw.b_qkv);
+  const __nv_bfloat16 *qnorm = static_cast<const __nv_bfloat16 *>(lw.q_norm), *knorm = static_cast<const __nv_bfloat16 *>(lw.k_norm);
+  if (dxmid) {
   // ---- d(attention output) = dxmid W_o, then the attention core ----
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_cast_bf16(dxmid, c->hat_dy, static_cast<size_t>(rows) * d, c->stream));
   if ((rc = run_gemm(c, c->hat_dy, rows, &c->hat_wo_t_map, c->hat_wo_t, rows, NQ, d, c->hat_do, EPI_STORE_F32, static_cast<size_t>(NQ), false)) != GM_OK)
@@ -365,40 +402,197 @@ int gm_head_attn_backward(gm_ctx *c, const float *x, const float *dxmid, const v
   if ((rc = gm_attention_backward(c, c->qbuf, c->hat_do, kv_pool, 1, num_pages, 0, page_table, c->qn, c->qbase, batch, q_stride,
                                   c->hat_dq, dk_pool, dv_pool)) != GM_OK)
     return rc;
+  } else {
+    GM_CUDA(c, cudaMemsetAsync(c->hat_dq, 0, sizeof(float) * static_cast<size_t>(rows) * NQ, c->stream));
+  }
   // ---- the rows' own entries are complete now: back through the rotation and the head norms, packed like the projection ----
   QkvGradArgs Q;
-  Q.qkv = c->qkv; Q.bias = R.bias; Q.qnorm = R.qnorm; Q.knorm = R.knorm; Q.dq = c->hat_dq; Q.dk_pool = dk_pool; Q.dv_pool = dv_pool;
+  Q.qkv = c->qkv; Q.bias = bias; Q.qnorm = qnorm; Q.knorm = knorm; Q.dq = c->hat_dq; Q.dk_pool = dk_pool; Q.dv_pool = dv_pool;
   Q.qn = c->qn; Q.qbase = c->qbase; Q.page_table = page_table; Q.rope = c->rope; Q.batch = batch; Q.QT = q_stride;
   Q.n_q = cf.n_q_heads; Q.n_kv = cf.n_kv_heads; Q.hd = hd; Q.num_pages = num_pages; Q.max_pages_per_seq = cf.max_pages_per_seq;
   Q.eps = cf.rms_eps; Q.dqkv = c->hat_dqkv; Q.dqkv_bf = c->hat_dqkv_bf; Q.status = c->status;
   if (dqk_norm) { Q.tq = c->hat_tq; Q.tk = c->hat_tk; }
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_qkv_grad_rows(Q, c->stream));
   if (dqk_norm) {
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_tq, rows * cf.n_q_heads, hd, dqk_norm, c->stream));
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_tk, rows * cf.n_kv_heads, hd, dqk_norm + hd, c->stream));
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_tq, rows * cf.n_q_heads, hd, dqk_norm, c->stream, accum));
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_tk, rows * cf.n_kv_heads, hd, dqk_norm + hd, c->stream, accum));
   }
-  if (db_qkv) GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_dqkv, rows, NQKV, db_qkv, c->stream));
+  if (db_qkv) GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_dqkv, rows, NQKV, db_qkv, c->stream, accum));
   // ---- dh = dqkv W_qkv;  dx = dxmid + d RMSNorm;  dln1 ----
   if ((rc = run_gemm(c, c->hat_dqkv_bf, rows, &c->hat_wqkv_t_map, c->hat_wqkv_t, rows, d, NQKV, c->hat_dh, EPI_STORE_F32, static_cast<size_t>(d), false)) != GM_OK)
     return rc;
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rmsnorm_grad(c->hat_dh, x, ln1, dx, rows, d, cf.rms_eps, c->stream, dxmid, c->hat_t));
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_t, rows, d, dln1, c->stream));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_t, rows, d, dln1, c->stream, accum));
   // ---- weight gradients contract over the rows: operands transposed to [features, rows] (rows padded with zeros to Mp) ----
-  GM_CUDA(c, cudaMemsetAsync(c->hat_dyt, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
-  GM_CUDA(c, cudaMemsetAsync(c->hat_ot, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * NQ, c->stream));
   GM_CUDA(c, cudaMemsetAsync(c->hat_dqkvt, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * NQKV, c->stream));
   GM_CUDA(c, cudaMemsetAsync(c->hat_ht, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->hat_dy, rows, d, c->hat_dyt, c->stream, Mp));
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->attn_out, rows, NQ, c->hat_ot, c->stream, Mp));
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->hat_dqkv_bf, rows, NQKV, c->hat_dqkvt, c->stream, Mp));
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->xn, rows, d, c->hat_ht, c->stream, Mp));
   CUtensorMap wm;
-  // dW_o [d, q_dim] = dxmid^T o
-  if (make_map(c, &wm, c->hat_ot, NQ, Mp, 128) != GM_OK) return GM_ERR_CUDA;
-  if ((rc = run_gemm(c, c->hat_dyt, d, &wm, c->hat_ot, d, NQ, Mp, dw_o, EPI_STORE_F32, static_cast<size_t>(NQ), false)) != GM_OK) return rc;
+  if (dxmid) {                                       // dW_o [d, q_dim] = dxmid^T o
+    GM_CUDA(c, cudaMemsetAsync(c->hat_dyt, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
+    GM_CUDA(c, cudaMemsetAsync(c->hat_ot, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * NQ, c->stream));
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->hat_dy, rows, d, c->hat_dyt, c->stream, Mp));
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_transpose_bf16(c->attn_out, rows, NQ, c->hat_ot, c->stream, Mp));
+    if (make_map(c, &wm, c->hat_ot, NQ, Mp, 128) != GM_OK) return GM_ERR_CUDA;
+    if ((rc = run_gemm(c, c->hat_dyt, d, &wm, c->hat_ot, d, NQ, Mp, dw_o, wepi, static_cast<size_t>(NQ), false)) != GM_OK) return rc;
+  }
   // dW_qkv [n_qkv, d] = dqkv^T h
   if (make_map(c, &wm, c->hat_ht, d, Mp, 128) != GM_OK) return GM_ERR_CUDA;
-  return run_gemm(c, c->hat_dqkvt, NQKV, &wm, c->hat_ht, NQKV, d, Mp, dw_qkv, EPI_STORE_F32, static_cast<size_t>(d), false);
+  return run_gemm(c, c->hat_dqkvt, NQKV, &wm, c->hat_ht, NQKV, d, Mp, dw_qkv, wepi, static_cast<size_t>(d), false);
+}
+int gm_head_attn_backward(gm_ctx *c, const float *x, const float *dxmid, const void *kv_pool, int num_pages,
+                          const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch, int q_stride,
+                          float *dk_pool, float *dv_pool, float *dx, float *dw_qkv, float *dw_o, float *dln1, float *db_qkv,
+                          float *dqk_norm, int refresh_weights) {
+  if (!dxmid) return GM_ERR_INVALID_ARG;
+  return head_attn_backward_impl(c, x, dxmid, kv_pool, num_pages, page_table, q_count, q_base, batch, q_stride, dk_pool, dv_pool, dx,
+                                 dw_qkv, dw_o, dln1, db_qkv, dqk_norm, refresh_weights, false);
+}
+
+// z = W_p [RMSNorm(E[token]) ; RMSNorm(hidden)] for `rows` pairs, with the forward pass's operand precision
+static int head_z_forward(gm_ctx *c, int rows, const int32_t *tokens, const float *hidden, float *z) {
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+            launch_head_input_rows(static_cast<const __nv_bfloat16 *>(c->w.embed), tokens, hidden,
+                                   static_cast<const __nv_bfloat16 *>(c->w.head_enorm), static_cast<const __nv_bfloat16 *>(c->w.head_hnorm),
+                                   rows, c->d, c->V, c->cfg.rms_eps, c->zin, c->hub_e, c->status, c->stream));
+  return run_gemm(c, c->zin, c->Mmax, &c->head_proj_map, static_cast<const __nv_bfloat16 *>(c->w.head_proj), rows, c->d, 2 * c->d, z,
+                  EPI_STORE_F32, c->d);
+}
+
+int gm_head_update_backward(gm_ctx *c, gm_state *st, int n_cycles, int k, const int32_t *cycle_seq, const gm_record *rec,
+                            const int32_t *seq_tok, int tok_stride, const int32_t *scratch_pages, const void *grad_logits,
+                            const void *seq_hidden, int hid_stride, const int32_t *seq_len, int max_len, float *dk_pool,
+                            float *dv_pool, const gm_head_grads *out) {
+  NvtxRange nvtx_range("gm_head_update_backward");
+  int rc = check_state(c, st, k);
+  if (rc) return rc;
+  if (n_cycles < 1 || !cycle_seq || !rec || !rec->start_hidden || !rec->start_pos || !rec->drafts || !seq_tok || tok_stride < 2 ||
+      !scratch_pages || !grad_logits || !seq_hidden || !seq_len || max_len < 2 || tok_stride < max_len || hid_stride < max_len - 1 ||
+      !dk_pool || !dv_pool || !out)
+    return GM_ERR_INVALID_ARG;
+  const gm_config &cf = c->cfg;
+  const gm_layer_weights &lw = c->w.head_layer;
+  if (!out->proj || !out->enorm || !out->hnorm || !out->final_norm || !out->ln1 || !out->ln2 || !out->wqkv || !out->wo ||
+      !out->w_gate_up || !out->w_down || (out->b_qkv != nullptr) != (lw.b_qkv != nullptr) ||
+      (out->qk_norm != nullptr) != (lw.q_norm != nullptr))
+    return GM_ERR_INVALID_ARG;
+  if (max_len + cf.max_k + 1 > cf.max_pages_per_seq * GM_PAGE) return GM_ERR_KV_CAPACITY;
+  const int d = c->d, F = c->F, MB = cf.max_batch, PS = cf.max_k + 1, hd = cf.head_dim;
+  const int B = st->batch, QT = cf.max_k + 1, VR = c->pf_vr, R = B * VR;
+  if (!c->v_table) return GM_ERR_INVALID_ARG;          // no reconstruction has run on this context
+  const int cap = std::max(MB, R * QT);
+  if (cap > c->hub_rows_cap) {
+    const size_t S = static_cast<size_t>(MB) * cf.max_k * d, M = static_cast<size_t>(cap) * d;
+    if ((rc = dev_alloc(c, &c->hub_states, S)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hub_gn, S)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hub_dstate, S)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hub_t, S)) != GM_OK) return rc;
+    for (float **p : {&c->hub_hidden, &c->hub_z, &c->hub_xmid, &c->hub_dg, &c->hub_dxmid, &c->hub_dz, &c->hub_dhid, &c->hub_e})
+      if ((rc = dev_alloc(c, p, M)) != GM_OK) return rc;
+    for (int32_t **p : {&c->hub_tok, &c->hub_base, &c->hub_cnt})
+      if ((rc = dev_alloc(c, p, static_cast<size_t>(cap))) != GM_OK) return rc;
+    c->hub_rows_cap = cap;
+  }
+  // every output starts at zero; the passes add to them
+  const size_t NQKV = c->n_qkv, NQ = c->q_dim;
+  const size_t plane = static_cast<size_t>(cf.head_num_pages) * cf.n_kv_heads * GM_PAGE * hd;
+  GM_CUDA(c, cudaMemsetAsync(dk_pool, 0, sizeof(float) * plane, c->stream));
+  GM_CUDA(c, cudaMemsetAsync(dv_pool, 0, sizeof(float) * plane, c->stream));
+  struct { float *p; size_t n; } outs[] = {{out->proj, static_cast<size_t>(2) * d * d}, {out->enorm, static_cast<size_t>(d)},
+      {out->hnorm, static_cast<size_t>(d)}, {out->final_norm, static_cast<size_t>(d)}, {out->ln1, static_cast<size_t>(d)},
+      {out->ln2, static_cast<size_t>(d)}, {out->wqkv, NQKV * d}, {out->wo, NQ * d}, {out->w_gate_up, static_cast<size_t>(2) * F * d},
+      {out->w_down, static_cast<size_t>(F) * d}, {out->b_qkv, NQKV}, {out->qk_norm, static_cast<size_t>(2) * hd}};
+  for (const auto &o : outs)
+    if (o.p) GM_CUDA(c, cudaMemsetAsync(o.p, 0, sizeof(float) * o.n, c->stream));
+  const __nv_bfloat16 *fnorm = static_cast<const __nv_bfloat16 *>(c->w.head_final_norm);
+  bool refresh = true;                                   // the transposed weight copies are remade once per call
+
+  // ---- the chains, a chunk of max_batch at a time: replay (Eq. 4), then the applications from the last one back ----
+  for (int off = 0; off < n_cycles; off += MB) {
+    const int m = std::min(MB, n_cycles - off);
+    ChainSetupArgs A;
+    A.cycle_seq = cycle_seq + off; A.start_pos = rec->start_pos + off;
+    A.start_hidden = static_cast<const __nv_bfloat16 *>(rec->start_hidden) + static_cast<size_t>(off) * d;
+    A.seq_tok = seq_tok; A.scratch_pages = scratch_pages + 2 * static_cast<size_t>(off);
+    A.head_page_table = st->head_page_table; A.pool = static_cast<__nv_bfloat16 *>(st->head_kv_pool);
+    A.n_seq = st->batch; A.tok_stride = tok_stride; A.k = k; A.d = d; A.vocab = c->V;
+    A.max_pages_per_seq = cf.max_pages_per_seq; A.num_pages = cf.head_num_pages;
+    A.page_elems = cf.n_kv_heads * GM_PAGE * hd; A.pend_stride = PS;
+    A.v_kv_len = c->v_kv_len; A.v_pending_n = c->v_pending_n; A.v_pending_tok = c->v_pending_tok; A.v_table = c->v_table;
+    A.v_pending_hidden = c->v_pending_hidden; A.status = c->status;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_chain_setup(A, m, c->stream));
+    gm_state vs = *st;
+    vs.batch = m; vs.kv_len = c->v_kv_len; vs.head_page_table = c->v_table; vs.pending_n = c->v_pending_n;
+    vs.pending_tok = c->v_pending_tok; vs.pending_hidden = c->v_pending_hidden;
+    c->state_out = c->hub_states;
+    rc = draft_impl(c, &vs, k, 1.0f, nullptr, 0, 0, rec->drafts + static_cast<size_t>(off) * k, c->ws_draft_logits, nullptr, true);
+    c->state_out = nullptr;
+    if (rc) return rc;
+    // every state's term through its own logits, and the final norm's weight
+    const __nv_bfloat16 *gl = static_cast<const __nv_bfloat16 *>(grad_logits) + static_cast<size_t>(off) * k * c->V;
+    if ((rc = gm_head_state_grad(c, m * k, gl, c->hub_states, c->hub_gn, c->hub_dstate, refresh ? 1 : 0)) != GM_OK) return rc;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+              launch_rmsnorm_grad(c->hub_gn, c->hub_states, fnorm, nullptr, m * k, d, cf.rms_eps, c->stream, nullptr, c->hub_t));
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hub_t, m * k, d, out->final_norm, c->stream, true));
+    for (int j = k; j >= 1; --j) {
+      StepRowsArgs S;
+      S.k = j; S.K = k; S.d = d; S.vocab = c->V; S.start_pos = rec->start_pos + off;
+      S.start_hidden = static_cast<const __nv_bfloat16 *>(rec->start_hidden) + static_cast<size_t>(off) * d;
+      S.first_tok = c->v_pending_tok; S.first_tok_stride = PS; S.drafts = rec->drafts + static_cast<size_t>(off) * k;
+      S.states = c->hub_states; S.dstate = c->hub_dstate; S.hidden = c->hub_hidden; S.dg = c->hub_dg;
+      S.tok = c->hub_tok; S.base = c->hub_base; S.count = c->hub_cnt; S.status = c->status;
+      GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_step_rows(S, m, c->stream));
+      // the application's forward values: z, then xmid = z + W_o attention(...)
+      if ((rc = head_z_forward(c, m, c->hub_tok, c->hub_hidden, c->hub_z)) != GM_OK) return rc;
+      if ((rc = head_attn_forward(c, c->hub_z, st->head_kv_pool, cf.head_num_pages, c->v_table, c->hub_cnt, c->hub_base, m, 1, true)) != GM_OK)
+        return rc;
+      GM_CUDA(c, cudaMemcpyAsync(c->hub_xmid, c->hub_z, sizeof(float) * static_cast<size_t>(m) * d, cudaMemcpyDeviceToDevice, c->stream));
+      if ((rc = run_gemm(c, c->attn_out, c->Mmax, &c->head_maps.wo, static_cast<const __nv_bfloat16 *>(lw.wo), m, d, c->q_dim, c->hub_xmid,
+                         EPI_ADD_F32, d)) != GM_OK)
+        return rc;
+      if ((rc = head_ffn_backward_impl(c, m, c->hub_xmid, c->hub_dg, c->hub_dxmid, out->w_gate_up, out->w_down, out->ln2, refresh, true)) != GM_OK)
+        return rc;
+      if ((rc = head_attn_backward_impl(c, c->hub_z, c->hub_dxmid, st->head_kv_pool, cf.head_num_pages, c->v_table, c->hub_cnt, c->hub_base,
+                                        m, 1, dk_pool, dv_pool, c->hub_dz, out->wqkv, out->wo, out->ln1, out->b_qkv, out->qk_norm, refresh,
+                                        true, true)) != GM_OK)
+        return rc;
+      if ((rc = head_input_backward_impl(c, m, c->hub_tok, c->hub_hidden, c->hub_dz, c->hub_dhid, out->proj, out->enorm, out->hnorm, refresh,
+                                         true)) != GM_OK)
+        return rc;
+      refresh = false;
+      // Eq. 4: application j >= 2 consumed the state of application j - 1
+      if (j >= 2) GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_add_state_grad(c->hub_dstate, c->hub_dhid, m, k, j - 2, d, c->stream));
+    }
+  }
+  // ---- what the chains left on the copied part of their boundary pages belongs to the shared originals ----
+  FoldArgs Fo;
+  Fo.cycle_seq = cycle_seq; Fo.start_pos = rec->start_pos; Fo.scratch_pages = scratch_pages; Fo.head_page_table = st->head_page_table;
+  Fo.n_seq = st->batch; Fo.max_pages_per_seq = cf.max_pages_per_seq; Fo.num_pages = cf.head_num_pages; Fo.n_kv = cf.n_kv_heads; Fo.hd = hd;
+  Fo.dk_pool = dk_pool; Fo.dv_pool = dv_pool;
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_fold_boundary(Fo, n_cycles, c->stream));
+  // ---- the pass over the committed prefixes: nothing consumed these rows' outputs, only their cache entries ----
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_dup_table_rows(st->head_page_table, B, VR, cf.max_pages_per_seq, c->pf_vtable[1], c->stream));
+  for (int base = 0; base + 1 < max_len; base += VR * QT) {
+    ChunkSetupArgs Cs;
+    Cs.prompt_tok = seq_tok; Cs.prompt_len = seq_len; Cs.batch = B; Cs.stride = tok_stride; Cs.base = base; Cs.QT = QT;
+    Cs.max_len = max_len; Cs.pair_stride = QT; Cs.vr = VR; Cs.row_n = c->pf_row_n; Cs.head_n = c->pf_head_n;
+    Cs.pair_tok = c->pf_pair_tok; Cs.row_base = c->pf_row_base; Cs.status = c->status;
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_chunk_setup(Cs, c->stream));
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE,
+              launch_gather_chunk_hidden(static_cast<const __nv_bfloat16 *>(seq_hidden), hid_stride, c->pf_row_base, R, VR, QT, d,
+                                         c->pf_head_n, c->pf_hidden, c->stream));
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rows_to_f32(c->pf_hidden, c->pf_head_n, R * QT, QT, d, c->hub_hidden, c->stream));
+    if ((rc = head_z_forward(c, R * QT, c->pf_pair_tok, c->hub_hidden, c->hub_z)) != GM_OK) return rc;
+    if ((rc = head_attn_backward_impl(c, c->hub_z, nullptr, st->head_kv_pool, cf.head_num_pages, c->pf_vtable[1], c->pf_head_n,
+                                      c->pf_row_base, R, QT, dk_pool, dv_pool, c->hub_dz, out->wqkv, out->wo, out->ln1, out->b_qkv,
+                                      out->qk_norm, 0, true)) != GM_OK)
+      return rc;
+    if ((rc = head_input_backward_impl(c, R * QT, c->pf_pair_tok, c->hub_hidden, c->hub_dz, nullptr, out->proj, out->enorm, out->hnorm, 0,
+                                       true)) != GM_OK)
+      return rc;
+  }
+  return GM_OK;
 }
 
 }  // extern "C"

@@ -121,6 +121,12 @@ struct gm_ctx {
   float *hin_e = nullptr, *hin_dzin = nullptr, *hin_t = nullptr;
   float *ab_stats = nullptr;                // attention backward: (max, 1 / sum, D) per (row, query head)
   size_t ab_stats_cap = 0;
+  // backward pass over a reconstruction: per-chunk states and their gradients, one pass's rows
+  int hub_rows_cap = 0;
+  float *hub_states = nullptr, *hub_gn = nullptr, *hub_dstate = nullptr, *hub_t = nullptr;          // [max_batch, max_k, d]
+  float *hub_hidden = nullptr, *hub_z = nullptr, *hub_xmid = nullptr, *hub_dg = nullptr, *hub_dxmid = nullptr, *hub_dz = nullptr,
+        *hub_dhid = nullptr, *hub_e = nullptr;                                                        // [rows, d]
+  int32_t *hub_tok = nullptr, *hub_base = nullptr, *hub_cnt = nullptr;                               // [rows]
   // attention half of the head's layer, backward: transposed weight copies and per-call scratch
   __nv_bfloat16 *hat_wo_t = nullptr, *hat_wqkv_t = nullptr;      // [q_dim, d], [d, n_qkv]
   CUtensorMap hat_wo_t_map, hat_wqkv_t_map;

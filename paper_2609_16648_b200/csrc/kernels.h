@@ -264,7 +264,28 @@ cudaError_t launch_head_input_rows(const __nv_bfloat16 *embed, const int32_t *to
 // dst [cols, dst_ld] = transpose of src [rows, cols] (bf16, both row-major; dst_ld >= rows, 0 = rows; padding untouched).
 cudaError_t launch_transpose_bf16(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst, cudaStream_t stream, int dst_ld = 0);
 // out[j] = sum over rows of t[row][j] (fp32, row order).
-cudaError_t launch_colsum(const float *t, int rows, int d, float *out, cudaStream_t stream);
+cudaError_t launch_colsum(const float *t, int rows, int d, float *out, cudaStream_t stream, bool add = false);
+// Bookkeeping of the backward pass over a reconstruction (chains of recorded cycles; Eq. 4).
+struct StepRowsArgs {
+  int k, K, d, vocab;                                   // application k (from 1) of K
+  const int32_t *start_pos;                             // [chains]
+  const __nv_bfloat16 *start_hidden;                    // [chains, d] the pair of application 1
+  const int32_t *first_tok; int first_tok_stride;       // token of application 1 at first_tok[c * stride]
+  const int32_t *drafts;                                // [chains, K] recorded drafts: application k >= 2 consumes drafts[k - 2]
+  const float *states, *dstate;                         // [chains, K, d] head states and their gradients
+  float *hidden, *dg;                                   // out [chains, d]
+  int32_t *tok, *base, *count;                          // out [chains]: token, position, 1
+  uint32_t *status;
+};
+cudaError_t launch_step_rows(const StepRowsArgs &A, int chains, cudaStream_t stream);
+cudaError_t launch_add_state_grad(float *dstate, const float *dhidden, int chains, int K, int k, int d, cudaStream_t stream);
+struct FoldArgs {
+  const int32_t *cycle_seq, *start_pos, *scratch_pages, *head_page_table;
+  int n_seq, max_pages_per_seq, num_pages, n_kv, hd;
+  float *dk_pool, *dv_pool;
+};
+cudaError_t launch_fold_boundary(const FoldArgs &A, int chains, cudaStream_t stream);
+cudaError_t launch_rows_to_f32(const __nv_bfloat16 *src, const int32_t *row_n, int rows, int QT, int d, float *dst, cudaStream_t stream);
 // AdamW on n fp32 master parameters with fp32 moments; param (bf16 copy the forward pass reads) or null.  decay = 1 - lr wd,
 // c1 / c2 = the bias corrections 1 / (1 - b^t), gscale multiplies the gradient (clipping).
 cudaError_t launch_adamw(float *master, __nv_bfloat16 *param, const float *grad, float *m, float *v, size_t n, float lr, float b1,

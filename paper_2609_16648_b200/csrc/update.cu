@@ -321,17 +321,73 @@ rmsnorm_grad_kernel(const float *gy, const float *x, const __nv_bfloat16 *w, flo
 }
 
 // out[j] = sum over the rows of t[row][j], added in row order (fp32).
-__global__ void __launch_bounds__(256) colsum_kernel(const float *t, int rows, int d, float *out) {
+__global__ void __launch_bounds__(256) colsum_kernel(const float *t, int rows, int d, float *out, int add) {
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  pdl_prologue();
   if (j >= d) return;
   float acc = 0.f;
   for (int r = 0; r < rows; ++r) acc += t[static_cast<size_t>(r) * d + j];
-  out[j] = acc;
+  out[j] = add ? out[j] + acc : acc;
+}
+
+// ---- bookkeeping of the backward pass over a reconstruction (Alg. 1, "update phi"; Eq. 4) ---------------------------------------
+// Rows of draft application k (from 1) of every chain: the (hidden, token) pair that entered, the gradient of the state
+// it produced, and its position.  One CTA per chain.
+__global__ void __launch_bounds__(128) step_rows_kernel(const StepRowsArgs A) {
+  const int c = blockIdx.x;
+  pdl_prologue();
+  const int k = A.k;
+  if (threadIdx.x == 0) {
+    int tok = k == 1 ? A.first_tok[static_cast<size_t>(c) * A.first_tok_stride] : A.drafts[static_cast<size_t>(c) * A.K + k - 2];
+    if (tok < 0 || tok >= A.vocab) { set_status(A.status, ST_BAD_TOKEN); tok = 0; }
+    A.tok[c] = tok;
+    A.base[c] = A.start_pos[c] + k - 3;
+    A.count[c] = 1;
+  }
+  const size_t row = static_cast<size_t>(c) * A.d;
+  for (int i = threadIdx.x; i < A.d; i += blockDim.x) {
+    A.hidden[row + i] = k == 1 ? bf16_to_float(A.start_hidden[row + i]) : A.states[(static_cast<size_t>(c) * A.K + k - 2) * A.d + i];
+    A.dg[row + i] = A.dstate[(static_cast<size_t>(c) * A.K + k - 1) * A.d + i];
+  }
+}
+// dstate[c][k] += dhidden[c]: the recurrence's term of the previous state's gradient (Eq. 4)
+__global__ void __launch_bounds__(128) add_state_grad_kernel(float *dstate, const float *dhidden, int K, int k, int d) {
+  const int c = blockIdx.x;
+  pdl_prologue();
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dstate[(static_cast<size_t>(c) * K + k) * d + i] += dhidden[static_cast<size_t>(c) * d + i];
+}
+// A chain's private boundary page started as a copy of its sequence's shared page: what the chain's rows left on the
+// copied entries (positions before the chain's first) belongs to the originals.  One CTA per chain, both planes.
+__global__ void __launch_bounds__(128) fold_boundary_kernel(const FoldArgs A) {
+  const int c = blockIdx.x;
+  pdl_prologue();
+  const int seq = A.cycle_seq[c], len = A.start_pos[c];
+  if (seq < 0 || seq >= A.n_seq || len < 2) return;
+  const int pb = (len - 2) >> 4, slots = (len - 2) & 15;
+  const int orig = A.head_page_table[static_cast<size_t>(seq) * A.max_pages_per_seq + pb], p0 = A.scratch_pages[2 * c];
+  if (orig < 0 || orig >= A.num_pages || p0 < 0 || p0 >= A.num_pages || orig == p0) return;
+  const int per_head = 16 * A.hd;
+  for (int i = threadIdx.x; i < A.n_kv * slots * A.hd; i += blockDim.x) {
+    const int h = i / (slots * A.hd), r = i % (slots * A.hd);
+    const size_t o = (static_cast<size_t>(orig) * A.n_kv + h) * per_head + r, s = (static_cast<size_t>(p0) * A.n_kv + h) * per_head + r;
+    const float a = A.dk_pool[s], b = A.dv_pool[s];
+    if (a != 0.f) atomicAdd(A.dk_pool + o, a);
+    if (b != 0.f) atomicAdd(A.dv_pool + o, b);
+  }
+}
+// fp32 copy of bf16 rows; row m = v * QT + j is zero when j >= row_n[v]
+__global__ void __launch_bounds__(128) rows_to_f32_kernel(const __nv_bfloat16 *src, const int32_t *row_n, int QT, int d, float *dst) {
+  const int m = blockIdx.x, v = m / QT, j = m % QT;
+  pdl_prologue();
+  const bool live = j < row_n[v];
+  for (int i = threadIdx.x; i < d; i += blockDim.x)
+    dst[static_cast<size_t>(m) * d + i] = live ? bf16_to_float(src[static_cast<size_t>(m) * d + i]) : 0.f;
 }
 
 // fp32 -> bf16, n elements (n % 4 == 0)
 __global__ void __launch_bounds__(256) cast_bf16_kernel(const float *src, __nv_bfloat16 *dst, size_t n4) {
   const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  pdl_prologue();
   if (i >= n4) return;
   const float4 v = reinterpret_cast<const float4 *>(src)[i];
   reinterpret_cast<uint2 *>(dst)[i] = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
@@ -343,6 +399,7 @@ __global__ void __launch_bounds__(256) cast_bf16_kernel(const float *src, __nv_b
 __global__ void __launch_bounds__(256)
 swiglu_grad_kernel(const __nv_bfloat16 *ab, const float *dh, __nv_bfloat16 *dab, __nv_bfloat16 *h, size_t n, int F) {
   const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  pdl_prologue();
   if (i >= n) return;
   const uint32_t w = reinterpret_cast<const uint32_t *>(ab)[i];
   const float a = bf16_lo(w), b = bf16_hi(w), g = dh[i];
@@ -441,6 +498,7 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16
   __shared__ __nv_bfloat16 tile[64][66];
   const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
   const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+  pdl_prologue();
   for (int i = ty; i < 64; i += 4)
     if (r0 + i < rows && c0 + tx < cols) tile[i][tx] = src[static_cast<size_t>(r0 + i) * cols + c0 + tx];
   __syncthreads();
@@ -467,6 +525,7 @@ __device__ __forceinline__ float adamw_one(float p, float g, float &m, float &v,
 }
 __global__ void __launch_bounds__(256) adamw_kernel(const AdamwArgs A) {
   const size_t n4 = A.n >> 2, stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  pdl_prologue();
   for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n4; i += stride) {
     float4 p = reinterpret_cast<float4 *>(A.master)[i], m = reinterpret_cast<float4 *>(A.m)[i], v = reinterpret_cast<float4 *>(A.v)[i];
     const float4 g = reinterpret_cast<const float4 *>(A.grad)[i];
@@ -565,9 +624,20 @@ cudaError_t launch_head_input_rows(const __nv_bfloat16 *embed, const int32_t *to
   return launch_k(head_input_rows_kernel, dim3(rows), dim3(NG_THREADS), 0, stream, 1, embed, tokens, hidden, we, wh, d, vocab, eps, zin,
                   e_out, status);
 }
-cudaError_t launch_colsum(const float *t, int rows, int d, float *out, cudaStream_t stream) {
-  colsum_kernel<<<(d + 255) / 256, 256, 0, stream>>>(t, rows, d, out);
-  return cudaGetLastError();
+cudaError_t launch_colsum(const float *t, int rows, int d, float *out, cudaStream_t stream, bool add) {
+  return launch_k(colsum_kernel, dim3((d + 255) / 256), dim3(256), 0, stream, 1, t, rows, d, out, add ? 1 : 0);
+}
+cudaError_t launch_step_rows(const StepRowsArgs &A, int chains, cudaStream_t stream) {
+  return launch_k(step_rows_kernel, dim3(chains), dim3(128), 0, stream, 1, A);
+}
+cudaError_t launch_add_state_grad(float *dstate, const float *dhidden, int chains, int K, int k, int d, cudaStream_t stream) {
+  return launch_k(add_state_grad_kernel, dim3(chains), dim3(128), 0, stream, 1, dstate, dhidden, K, k, d);
+}
+cudaError_t launch_fold_boundary(const FoldArgs &A, int chains, cudaStream_t stream) {
+  return launch_k(fold_boundary_kernel, dim3(chains), dim3(128), 0, stream, 1, A);
+}
+cudaError_t launch_rows_to_f32(const __nv_bfloat16 *src, const int32_t *row_n, int rows, int QT, int d, float *dst, cudaStream_t stream) {
+  return launch_k(rows_to_f32_kernel, dim3(rows), dim3(128), 0, stream, 1, src, row_n, QT, d, dst);
 }
 cudaError_t launch_cast_bf16(const float *src, __nv_bfloat16 *dst, size_t n, cudaStream_t stream) {
   cast_bf16_kernel<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, stream>>>(src, dst, n / 4);

@@ -505,6 +505,80 @@ def test_head_attn_backward_matches_the_oracle(name, family):
     ctx.close()
 
 
+@pytest.mark.parametrize("family", ["plain", "qk_norm", "qkv_bias"])
+def test_head_update_backward_matches_the_oracle(family):
+    """gm_head_update_backward - the whole backward pass over recorded cycles, chains replayed three chunks of max_batch
+    at a time - against the oracle's head_update_grad on the weights the device holds, both starting from the device's
+    own logit gradients (the piecewise-linear overlap picks its branches from the logits, which differ in rounding).
+    Every parameter tensor of the head; the oracle's is pinned by finite differences of the objective."""
+    import paper_2609_16648_b200 as gmb
+    cfg = get_config("tiny").with_(prompt_len=12, qk_norm=family == "qk_norm", qkv_bias=family == "qkv_bias")
+    B, K, V, d = cfg.batch, cfg.k, cfg.vocab, cfg.d_model
+    w = perturb_norm_weights(make_weights(cfg, 0))
+    st, cycles, seqs, hpt, hnpg = _oracle_rollout(cfg, w, n_steps=3)
+    n = len(cycles)
+    assert any(r["accepted"] >= 2 for _, r in cycles)                     # some chains reach the recurrence
+    ctx = gmb.Context(cfg, gmb.pack_weights(w), B, K, hpt.shape[1], hnpg, hnpg + 2 * n)
+    gst = gmb.State(ctx, B, hpt, hpt)
+    S = max(len(t) for _, t in seqs)
+    seq_tok, seq_hid, seq_len = np.zeros((B, S), np.int32), np.zeros((B, S, d), np.float32), np.zeros(B, np.int32)
+    for b, (H, toks) in enumerate(seqs):
+        seq_tok[b, :len(toks)] = toks
+        seq_hid[b, :len(toks) - 1] = H
+        seq_len[b] = len(toks)
+    tok_d, len_d = torch.from_numpy(seq_tok).cuda(), torch.from_numpy(seq_len).cuda()
+    hid_d = torch.from_numpy(seq_hid).to(device="cuda", dtype=torch.bfloat16)
+    gmb.gm_head_prefill(ctx, gst, hid_d, tok_d, len_d, int(seq_len.max()))
+    rec = gmb.Record(n, K, d)
+    rec.start_hidden.copy_(torch.from_numpy(np.stack([r["start_hidden"] for _, r in cycles])).to(torch.bfloat16))
+    rec.start_pos.copy_(torch.tensor([r["start_pos"] for _, r in cycles], dtype=torch.int32))
+    rec.drafts.copy_(torch.from_numpy(np.stack([r["drafts"] for _, r in cycles]).astype(np.int32)))
+    rec.top_index.copy_(torch.from_numpy(np.stack([r["top_index"] for _, r in cycles]).astype(np.int32)))
+    rec.top_logprob.copy_(torch.from_numpy(np.stack([r["top_logprob"] for _, r in cycles])).to(torch.bfloat16))
+    rec.accepted.copy_(torch.tensor([r["accepted"] for _, r in cycles], dtype=torch.int32))
+    cycle_seq = torch.tensor([b for b, _ in cycles], dtype=torch.int32, device="cuda")
+    scratch = torch.arange(hnpg, hnpg + 2 * n, dtype=torch.int32, device="cuda").reshape(n, 2)
+    logits = torch.zeros((n, K, V), dtype=torch.bfloat16, device="cuda")
+    gmb.gm_reconstruct(ctx, gst, n, K, cycle_seq, rec, tok_d, scratch, logits)
+    alpha = torch.zeros((n, K), dtype=torch.float32, device="cuda")
+    gmb.gm_overlap(ctx, n, K, T, logits, rec, alpha)
+    grad = torch.zeros((n, K, V), dtype=torch.bfloat16, device="cuda")
+    gmb.gm_dca_grad(ctx, n, K, T, logits, rec, alpha, rec.accepted, grad)
+    npg_h = hnpg + 2 * n
+    dkp = torch.full((npg_h, cfg.n_kv_heads, 16, cfg.head_dim), 7.0, dtype=torch.float32, device="cuda")
+    dvp = torch.full_like(dkp, 7.0)
+    grads = gmb.head_grad_buffers(cfg)
+    for t in grads.values():
+        t.fill_(7.0)                                                       # outputs are overwritten, not added to
+    pool_before = gst.head_kv_pool.clone()
+    gmb.gm_head_update_backward(ctx, gst, n, K, cycle_seq, rec, tok_d, scratch, grad, hid_d, len_d, int(seq_len.max()), dkp, dvp, grads)
+    assert gmb.gm_last_status(ctx) == 0
+    assert torch.equal(gst.head_kv_pool, pool_before)                      # the replay rewrites the chains' pages with the same values
+    # the oracle on the device's weights and the device's logit gradients
+    r16 = lambda a: omodel.round_bf16(a).astype(np.float64)
+    w16 = {"embed": r16(w["embed"]), "lm_head": r16(w["lm_head"]),
+           "head": {k_: (r16(v_) if k_ != "layer" else {n_: r16(a_) for n_, a_ in v_.items()}) for k_, v_ in w["head"].items() if k_ != "concat"}}
+    want = oupdate.head_update_grad(w16, cfg, seqs, cycles, T, grad_logits=grad.double().cpu().numpy())
+    f = lambda t: t.double().cpu().numpy()
+    NQ, NKV = cfg.q_dim, cfg.kv_dim
+    got = {"proj": f(grads["proj"]), "enorm": f(grads["enorm"]), "hnorm": f(grads["hnorm"]), "final_norm": f(grads["final_norm"])}
+    gl = {"ln1": f(grads["ln1"]), "ln2": f(grads["ln2"]), "wq": f(grads["wqkv"])[:NQ], "wk": f(grads["wqkv"])[NQ:NQ + NKV],
+          "wv": f(grads["wqkv"])[NQ + NKV:], "wo": f(grads["wo"]), "wg": f(grads["w_gate_up"])[0::2], "wu": f(grads["w_gate_up"])[1::2],
+          "wd": f(grads["w_down"])}
+    if cfg.qkv_bias:
+        bq = f(grads["b_qkv"])
+        gl.update(bq=bq[:NQ], bk=bq[NQ:NQ + NKV], bv=bq[NQ + NKV:])
+    if cfg.qk_norm:
+        gl.update(qnorm=f(grads["qk_norm"])[:cfg.head_dim], knorm=f(grads["qk_norm"])[cfg.head_dim:])
+    assert set(gl) == set(want["layer"])
+    errs = {k_: rel_err(v_, want[k_]) for k_, v_ in got.items()}
+    errs.update({"layer." + k_: rel_err(v_, want["layer"][k_]) for k_, v_ in gl.items()})
+    print({k_: round(v_, 4) for k_, v_ in errs.items()})
+    for k_, e in errs.items():
+        assert e < 2e-2, (k_, e)
+    ctx.close()
+
+
 @pytest.mark.parametrize("n", [1003, 49_807_360], ids=["ragged_1003", "gate_up_of_the_4b_head"])
 def test_adamw_step_matches_the_oracle(n):
     """gm_adamw_step over several updates with the head's schedule against the oracle's fp64 AdamW (sampled entries at the
