@@ -24,7 +24,7 @@ GM_KC_GEMM, GM_KC_ATTENTION, GM_KC_ELEMENTWISE, GM_KC_SAMPLER, GM_KC_RECORD = 0,
 
 EXPORTS = ["gm_init", "gm_destroy", "gm_draft", "gm_verify", "gm_accept", "gm_spec_step", "gm_draw", "gm_set_top_p", "gm_nucleus", "gm_prefill",
            "gm_rollout_begin", "gm_rollout_step", "gm_rollout_run", "gm_pages_reset", "gm_pages_reserve",
-           "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_reconstruct_states", "gm_head_state_grad", "gm_head_ffn_backward", "gm_attention_backward", "gm_head_attn_backward", "gm_head_update_backward", "gm_head_input_backward", "gm_adamw_step", "gm_overlap", "gm_dca_loss", "gm_dca_grad",
+           "gm_pages_release", "gm_pages_free_count", "gm_capture_hidden", "gm_head_prefill", "gm_reconstruct", "gm_reconstruct_states", "gm_head_state_grad", "gm_head_ffn_backward", "gm_attention_backward", "gm_head_attn_backward", "gm_head_update_backward", "gm_head_update_step", "gm_head_input_backward", "gm_adamw_step", "gm_overlap", "gm_dca_loss", "gm_dca_grad",
            "gm_spec_step_host", "gm_gemm", "gm_gemm_swiglu", "gm_attention", "gm_attention_noalloc", "gm_record_begin", "gm_record_end",
            "gm_spec_step_rec", "gm_profile", "gm_profile_read", "gm_chain_trace", "gm_chain_trace_read", "gm_selftest_wait_expiry", "gm_launch_count",
            "gm_last_status", "gm_strerror"]
@@ -108,6 +108,8 @@ def lib() -> C.CDLL:
     L.gm_head_attn_backward.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32]
     L.gm_head_update_backward.argtypes = [vp, C.POINTER(gm_state), i32, i32, vp, C.POINTER(gm_record), vp, i32, vp, vp, vp, i32, vp, i32, vp,
                                           vp, C.POINTER(gm_head_grads)]
+    L.gm_head_update_step.argtypes = [vp, C.POINTER(gm_state), i32, i32, f32, vp, C.POINTER(gm_record), vp, i32, vp, vp, i32, vp, i32, i32,
+                                      f32, f32, f32, f32, f32, vp]
     L.gm_head_input_backward.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, i32]
     L.gm_adamw_step.argtypes = [vp, C.c_int64, vp, vp, vp, vp, vp, i32, f32, f32, f32, f32, f32, f32]
     L.gm_overlap.argtypes = [vp, i32, i32, f32, vp, C.POINTER(gm_record), vp, vp]
@@ -462,6 +464,15 @@ def gm_head_update_backward(ctx: Context, st: State, n_cycles: int, k: int, cycl
                                          _p(seq_tok), seq_tok.shape[1], _p(scratch_pages), _p(grad_logits), _p(seq_hidden),
                                          seq_hidden.shape[1], _p(seq_len), max_len, _p(dk_pool), _p(dv_pool), C.byref(gs)),
            "gm_head_update_backward")
+
+
+def gm_head_update_step(ctx: Context, st: State, n_cycles: int, k: int, temperature: float, cycle_seq, rec, seq_tok, scratch_pages,
+                        seq_hidden, seq_len, max_len: int, step: int, lr: float, mean_loss, beta1: float = 0.9, beta2: float = 0.999,
+                        eps: float = 1e-8, weight_decay: float = 0.01):
+    _check(lib().gm_head_update_step(ctx.handle, C.byref(st.struct()), n_cycles, k, temperature, _p(cycle_seq), C.byref(rec.struct()),
+                                     _p(seq_tok), seq_tok.shape[1], _p(scratch_pages), _p(seq_hidden), seq_hidden.shape[1],
+                                     _p(seq_len), max_len, step, lr, beta1, beta2, eps, weight_decay, _p(mean_loss)),
+           "gm_head_update_step")
 
 
 def gm_head_input_backward(ctx: Context, rows: int, tokens, hidden, dz, dhidden, dproj, denorm, dhnorm, refresh_weights: bool = False):

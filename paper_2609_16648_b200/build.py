@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgm.so")
-SOURCES = ["gm_api.cu", "api_prefill.cu", "api_aux.cu", "api_update.cu", "api_rollout.cu", "sampler.cu", "sampler_stream.cu", "sampler_flow.cu", "elementwise.cu", "attention.cu", "attention_bwd.cu", "gemm.cu", "chain.cu", "noalloc.cu", "record.cu", "nucleus.cu", "update.cu"]
+SOURCES = ["gm_api.cu", "api_prefill.cu", "api_aux.cu", "api_update.cu", "api_train.cu", "api_rollout.cu", "sampler.cu", "sampler_stream.cu", "sampler_flow.cu", "elementwise.cu", "attention.cu", "attention_bwd.cu", "gemm.cu", "chain.cu", "noalloc.cu", "record.cu", "nucleus.cu", "update.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC"]
 

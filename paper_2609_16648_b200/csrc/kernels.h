@@ -285,6 +285,7 @@ struct FoldArgs {
   float *dk_pool, *dv_pool;
 };
 cudaError_t launch_fold_boundary(const FoldArgs &A, int chains, cudaStream_t stream);
+cudaError_t launch_widen_bf16(const __nv_bfloat16 *src, float *dst, size_t n, cudaStream_t stream);          // dst[i] = src[i]
 cudaError_t launch_rows_to_f32(const __nv_bfloat16 *src, const int32_t *row_n, int rows, int QT, int d, float *dst, cudaStream_t stream);
 // AdamW on n fp32 master parameters with fp32 moments; param (bf16 copy the forward pass reads) or null.  decay = 1 - lr wd,
 // c1 / c2 = the bias corrections 1 / (1 - b^t), gscale multiplies the gradient (clipping).

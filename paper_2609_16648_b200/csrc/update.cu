@@ -375,6 +375,11 @@ __global__ void __launch_bounds__(128) fold_boundary_kernel(const FoldArgs A) {
     if (b != 0.f) atomicAdd(A.dv_pool + o, b);
   }
 }
+__global__ void __launch_bounds__(256) widen_bf16_kernel(const __nv_bfloat16 *src, float *dst, size_t n) {
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  pdl_prologue();
+  for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += stride) dst[i] = bf16_to_float(src[i]);
+}
 // fp32 copy of bf16 rows; row m = v * QT + j is zero when j >= row_n[v]
 __global__ void __launch_bounds__(128) rows_to_f32_kernel(const __nv_bfloat16 *src, const int32_t *row_n, int QT, int d, float *dst) {
   const int m = blockIdx.x, v = m / QT, j = m % QT;
@@ -635,6 +640,10 @@ cudaError_t launch_add_state_grad(float *dstate, const float *dhidden, int chain
 }
 cudaError_t launch_fold_boundary(const FoldArgs &A, int chains, cudaStream_t stream) {
   return launch_k(fold_boundary_kernel, dim3(chains), dim3(128), 0, stream, 1, A);
+}
+cudaError_t launch_widen_bf16(const __nv_bfloat16 *src, float *dst, size_t n, cudaStream_t stream) {
+  const size_t blocks = std::min<size_t>((n + 255) / 256, 148 * 8);
+  return launch_k(widen_bf16_kernel, dim3(static_cast<unsigned>(std::max<size_t>(blocks, 1))), dim3(256), 0, stream, 1, src, dst, n);
 }
 cudaError_t launch_rows_to_f32(const __nv_bfloat16 *src, const int32_t *row_n, int rows, int QT, int d, float *dst, cudaStream_t stream) {
   return launch_k(rows_to_f32_kernel, dim3(rows), dim3(128), 0, stream, 1, src, row_n, QT, d, dst);

@@ -53,6 +53,7 @@ def test_error_strings_and_null_handling_need_no_gpu():
     assert L.gm_attention_backward(None, None, None, None, 1, 1, 0, None, None, None, 1, 1, None, None, None) == inv
     assert L.gm_head_attn_backward(None, None, None, None, 1, None, None, None, 1, 1, None, None, None, None, None, None, None, None, 0) == inv
     assert L.gm_head_update_backward(None, None, 1, 1, None, None, None, 2, None, None, None, 1, None, 2, None, None, None) == inv
+    assert L.gm_head_update_step(None, None, 1, 1, 1.0, None, None, None, 2, None, None, 1, None, 2, 1, 1e-4, 0.9, 0.999, 1e-8, 0.01, None) == inv
     assert L.gm_head_input_backward(None, 1, None, None, None, None, None, None, None, 0) == inv
     assert L.gm_adamw_step(None, 1, None, None, None, None, None, 1, 1e-4, 0.9, 0.999, 1e-8, 0.01, 1.0) == inv
     assert L.gm_overlap(None, 1, 3, 1.0, None, None, None, None) == inv

@@ -505,12 +505,8 @@ def test_head_attn_backward_matches_the_oracle(name, family):
     ctx.close()
 
 
-@pytest.mark.parametrize("family", ["plain", "qk_norm", "qkv_bias"])
-def test_head_update_backward_matches_the_oracle(family):
-    """gm_head_update_backward - the whole backward pass over recorded cycles, chains replayed three chunks of max_batch
-    at a time - against the oracle's head_update_grad on the weights the device holds, both starting from the device's
-    own logit gradients (the piecewise-linear overlap picks its branches from the logits, which differ in rounding).
-    Every parameter tensor of the head; the oracle's is pinned by finite differences of the objective."""
+def _update_setup(family, n_steps=3):
+    """A short oracle rollout with its records, and a device context / state / record holding the same cycles."""
     import paper_2609_16648_b200 as gmb
     cfg = get_config("tiny").with_(prompt_len=12, qk_norm=family == "qk_norm", qkv_bias=family == "qkv_bias")
     B, K, V, d = cfg.batch, cfg.k, cfg.vocab, cfg.d_model
@@ -528,7 +524,6 @@ def test_head_update_backward_matches_the_oracle(family):
         seq_len[b] = len(toks)
     tok_d, len_d = torch.from_numpy(seq_tok).cuda(), torch.from_numpy(seq_len).cuda()
     hid_d = torch.from_numpy(seq_hid).to(device="cuda", dtype=torch.bfloat16)
-    gmb.gm_head_prefill(ctx, gst, hid_d, tok_d, len_d, int(seq_len.max()))
     rec = gmb.Record(n, K, d)
     rec.start_hidden.copy_(torch.from_numpy(np.stack([r["start_hidden"] for _, r in cycles])).to(torch.bfloat16))
     rec.start_pos.copy_(torch.tensor([r["start_pos"] for _, r in cycles], dtype=torch.int32))
@@ -538,6 +533,21 @@ def test_head_update_backward_matches_the_oracle(family):
     rec.accepted.copy_(torch.tensor([r["accepted"] for _, r in cycles], dtype=torch.int32))
     cycle_seq = torch.tensor([b for b, _ in cycles], dtype=torch.int32, device="cuda")
     scratch = torch.arange(hnpg, hnpg + 2 * n, dtype=torch.int32, device="cuda").reshape(n, 2)
+    return dict(gmb=gmb, cfg=cfg, w=w, cycles=cycles, seqs=seqs, n=n, ctx=ctx, gst=gst, tok_d=tok_d, len_d=len_d, hid_d=hid_d,
+                max_len=int(seq_len.max()), rec=rec, cycle_seq=cycle_seq, scratch=scratch, hnpg=hnpg)
+
+
+@pytest.mark.parametrize("family", ["plain", "qk_norm", "qkv_bias"])
+def test_head_update_backward_matches_the_oracle(family):
+    """gm_head_update_backward - the whole backward pass over recorded cycles, chains replayed three chunks of max_batch
+    at a time - against the oracle's head_update_grad on the weights the device holds, both starting from the device's
+    own logit gradients (the piecewise-linear overlap picks its branches from the logits, which differ in rounding).
+    Every parameter tensor of the head; the oracle's is pinned by finite differences of the objective."""
+    u = _update_setup(family)
+    gmb, cfg, w, cycles, seqs, n, ctx, gst = (u[k_] for k_ in ("gmb", "cfg", "w", "cycles", "seqs", "n", "ctx", "gst"))
+    tok_d, len_d, hid_d, rec, cycle_seq, scratch, hnpg = (u[k_] for k_ in ("tok_d", "len_d", "hid_d", "rec", "cycle_seq", "scratch", "hnpg"))
+    B, K, V, d = cfg.batch, cfg.k, cfg.vocab, cfg.d_model
+    gmb.gm_head_prefill(ctx, gst, hid_d, tok_d, len_d, u["max_len"])
     logits = torch.zeros((n, K, V), dtype=torch.bfloat16, device="cuda")
     gmb.gm_reconstruct(ctx, gst, n, K, cycle_seq, rec, tok_d, scratch, logits)
     alpha = torch.zeros((n, K), dtype=torch.float32, device="cuda")
@@ -551,7 +561,7 @@ def test_head_update_backward_matches_the_oracle(family):
     for t in grads.values():
         t.fill_(7.0)                                                       # outputs are overwritten, not added to
     pool_before = gst.head_kv_pool.clone()
-    gmb.gm_head_update_backward(ctx, gst, n, K, cycle_seq, rec, tok_d, scratch, grad, hid_d, len_d, int(seq_len.max()), dkp, dvp, grads)
+    gmb.gm_head_update_backward(ctx, gst, n, K, cycle_seq, rec, tok_d, scratch, grad, hid_d, len_d, u["max_len"], dkp, dvp, grads)
     assert gmb.gm_last_status(ctx) == 0
     assert torch.equal(gst.head_kv_pool, pool_before)                      # the replay rewrites the chains' pages with the same values
     # the oracle on the device's weights and the device's logit gradients
@@ -576,6 +586,89 @@ def test_head_update_backward_matches_the_oracle(family):
     print({k_: round(v_, 4) for k_, v_ in errs.items()})
     for k_, e in errs.items():
         assert e < 2e-2, (k_, e)
+    ctx.close()
+
+
+HEAD_TENSORS = ("proj", "enorm", "hnorm", "final_norm")
+
+
+def _head_params(packed):
+    out = {n_: packed["head"][n_] for n_ in HEAD_TENSORS}
+    out.update({"layer." + n_: t for n_, t in packed["head"]["layer"].items()})
+    return out
+
+
+@pytest.mark.parametrize("family", ["plain", "qk_norm"])
+def test_head_update_steps_lower_the_objective_and_equal_the_calls_made_one_by_one(family):
+    """gm_head_update_step (Alg. 1, "update phi" as one call).  (1) Its first update leaves exactly the parameters that the
+    public calls it is made of leave when made one by one on a second context (cache rebuild, reconstruction, overlap,
+    loss, logit gradients, backward pass, AdamW per tensor from fp32 copies of the bf16 parameters and zero moments).
+    (2) Repeated on the same recorded cycles with the head's schedule, it lowers the objective it reports - the mean of
+    Eq. 9 before each update - i.e. the head's acceptance on those cycles rises; the backbone's tensors never change."""
+    u = _update_setup(family)
+    gmb, cfg, n, ctx, gst = u["gmb"], u["cfg"], u["n"], u["ctx"], u["gst"]
+    K, V, d = cfg.k, cfg.vocab, cfg.d_model
+    common = (u["cycle_seq"], u["rec"], u["tok_d"], u["scratch"])
+    frozen = {k_: ctx.packed[k_].clone() for k_ in ("embed", "lm_head", "final_norm")}
+    frozen["l0.wqkv"] = ctx.packed["layers"][0]["wqkv"].clone()
+    before = {k_: t.clone() for k_, t in _head_params(ctx.packed).items()}
+    mean = torch.zeros(1, dtype=torch.float32, device="cuda")
+    peak, steps = 2e-3, 8
+    f32 = lambda x: float(np.float32(x))
+    lr1 = f32(oupdate.head_lr(0, peak, steps, warmup=2))
+    with pytest.raises(gmb.GmError):                                      # updates are numbered from 1, in order
+        gmb.gm_head_update_step(ctx, gst, n, K, T, *common, u["hid_d"], u["len_d"], u["max_len"], 2, lr1, mean)
+    gmb.gm_head_update_step(ctx, gst, n, K, T, *common, u["hid_d"], u["len_d"], u["max_len"], 1, lr1, mean)
+    assert gmb.gm_last_status(ctx) == 0
+    losses = [float(mean[0])]
+    after1 = {k_: t.clone() for k_, t in _head_params(ctx.packed).items()}
+    # every matrix moved; a norm weight near 1 has a bf16 spacing of 2^-7, which one step of 1e-3 does not cross - the
+    # fp32 master copy carries it
+    assert all(not torch.equal(after1[k_], before[k_]) for k_ in after1 if after1[k_].dim() == 2)
+
+    # (1) the same update, call by call, on a second context with its own copy of the weights
+    u2 = _update_setup(family)
+    c2, g2 = u2["ctx"], u2["gst"]
+    gmb.gm_head_prefill(c2, g2, u2["hid_d"], u2["tok_d"], u2["len_d"], u2["max_len"])
+    logits = torch.zeros((n, K, V), dtype=torch.bfloat16, device="cuda")
+    gmb.gm_reconstruct(c2, g2, n, K, u2["cycle_seq"], u2["rec"], u2["tok_d"], u2["scratch"], logits)
+    alpha, lse = torch.zeros((n, K), device="cuda"), torch.zeros((n, K), device="cuda")
+    gmb.gm_overlap(c2, n, K, T, logits, u2["rec"], alpha, lse)
+    loss, mean2 = torch.zeros(n, device="cuda"), torch.zeros(1, device="cuda")
+    gmb.gm_dca_loss(c2, n, K, alpha, u2["rec"].accepted, loss, mean2)
+    assert float(mean2[0]) == losses[0]
+    grad = torch.zeros((n, K, V), dtype=torch.bfloat16, device="cuda")
+    gmb.gm_dca_grad(c2, n, K, T, logits, u2["rec"], alpha, u2["rec"].accepted, grad, lse)
+    npg_h = u2["hnpg"] + 2 * n
+    dkp = torch.zeros((npg_h, cfg.n_kv_heads, 16, cfg.head_dim), dtype=torch.float32, device="cuda")
+    grads = gmb.head_grad_buffers(cfg)
+    gmb.gm_head_update_backward(c2, g2, n, K, u2["cycle_seq"], u2["rec"], u2["tok_d"], u2["scratch"], grad, u2["hid_d"], u2["len_d"],
+                                u2["max_len"], dkp, torch.zeros_like(dkp), grads)
+    hd = cfg.head_dim
+    gmap = {"proj": grads["proj"], "enorm": grads["enorm"], "hnorm": grads["hnorm"], "final_norm": grads["final_norm"],
+            "layer.ln1": grads["ln1"], "layer.ln2": grads["ln2"], "layer.wqkv": grads["wqkv"], "layer.wo": grads["wo"],
+            "layer.w_gate_up": grads["w_gate_up"], "layer.w_down": grads["w_down"]}
+    if family == "qk_norm":
+        gmap.update({"layer.q_norm": grads["qk_norm"][:hd].contiguous(), "layer.k_norm": grads["qk_norm"][hd:].contiguous()})
+    p2 = _head_params(c2.packed)
+    assert set(p2) == set(gmap)
+    for name, t in p2.items():
+        master = t.float().reshape(-1).contiguous()
+        gmb.gm_adamw_step(c2, master, gmap[name].reshape(-1), torch.zeros_like(master), torch.zeros_like(master), 1, lr1, param_bf16=t)
+        assert torch.equal(t, after1[name]), name
+    c2.close()
+
+    # (2) more updates on the same cycles
+    for s_ in range(1, steps):
+        gmb.gm_head_update_step(ctx, gst, n, K, T, *common, u["hid_d"], u["len_d"], u["max_len"], s_ + 1,
+                                f32(oupdate.head_lr(s_, peak, steps, warmup=2)), mean)
+        losses.append(float(mean[0]))
+    assert gmb.gm_last_status(ctx) == 0
+    print("mean objective before each update:", [round(x, 4) for x in losses])
+    assert all(np.isfinite(losses))
+    assert losses[-1] < losses[0] - 0.02 and min(losses[1:]) < losses[0]
+    assert torch.equal(ctx.packed["lm_head"], frozen["lm_head"]) and torch.equal(ctx.packed["embed"], frozen["embed"])
+    assert torch.equal(ctx.packed["final_norm"], frozen["final_norm"]) and torch.equal(ctx.packed["layers"][0]["wqkv"], frozen["l0.wqkv"])
     ctx.close()
 
 
