@@ -3,6 +3,15 @@
 // Host code only; the helpers it calls are declared in gm_internal.h.
 #include "gm_internal.h"
 
+// scratch for column sums split over several CTAs; null (single-chunk sums) if the allocation fails
+static float *colsum_ws(gm_ctx *c) {
+  if (!c->colsum_ws) {
+    const size_t widest = static_cast<size_t>(std::max(std::max(c->n_qkv, 2 * c->d), static_cast<int>(c->cfg.head_dim)));
+    if (dev_alloc(c, &c->colsum_ws, gm::colsum_scratch_floats(static_cast<int>(widest))) != GM_OK) c->colsum_ws = nullptr;
+  }
+  return c->colsum_ws;
+}
+
 extern "C" {
 
 int gm_capture_hidden(gm_ctx *c, void *seq_hidden, int stride) {
@@ -174,7 +183,7 @@ static int head_ffn_backward_impl(gm_ctx *c, int rows, const float *x, const flo
   if ((rc = run_gemm(c, c->ffn_dab, rows, &c->ffn_wgu_t_map, c->ffn_wgu_t, rows, d, 2 * F, c->ffn_du, EPI_STORE_F32, static_cast<size_t>(d), false)) != GM_OK)
     return rc;
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rmsnorm_grad(c->ffn_du, x, ln2, dx, rows, d, c->cfg.rms_eps, c->stream, dg, c->ffn_t));
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->ffn_t, rows, d, dln2, c->stream, accum));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->ffn_t, rows, d, dln2, c->stream, accum, colsum_ws(c)));
   // weight gradients contract over the rows: both operands transposed to [features, rows] (rows padded with zeros to Mp)
   GM_CUDA(c, cudaMemsetAsync(c->ffn_ut, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
   GM_CUDA(c, cudaMemsetAsync(c->ffn_dyt, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
@@ -253,10 +262,10 @@ static int head_input_backward_impl(gm_ctx *c, int rows, const int32_t *tokens, 
   // through the two norms: the hidden half gives dL/d hidden and dL/d hnorm, the embedding half only dL/d enorm
   GM_LAUNCH(c, GM_KC_ELEMENTWISE,
             launch_rmsnorm_grad(c->hin_dzin + d, hidden, wh, dhidden, rows, d, c->cfg.rms_eps, c->stream, nullptr, c->hin_t, 2 * d));
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hin_t, rows, d, dhnorm, c->stream, accum));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hin_t, rows, d, dhnorm, c->stream, accum, colsum_ws(c)));
   GM_LAUNCH(c, GM_KC_ELEMENTWISE,
             launch_rmsnorm_grad(c->hin_dzin, c->hin_e, we, nullptr, rows, d, c->cfg.rms_eps, c->stream, nullptr, c->hin_t, 2 * d));
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hin_t, rows, d, denorm, c->stream, accum));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hin_t, rows, d, denorm, c->stream, accum, colsum_ws(c)));
   // dW_p [d, 2d] = dz^T zin: both operands transposed to [features, rows] (rows padded with zeros to Mp)
   GM_CUDA(c, cudaMemsetAsync(c->hin_dzt, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
   GM_CUDA(c, cudaMemsetAsync(c->hin_zint, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * 2 * d, c->stream));
@@ -285,7 +294,19 @@ int gm_attention_backward(gm_ctx *c, const void *q, const float *dout, const voi
     if (rc != GM_OK) return rc;
     c->ab_stats_cap = need;
   }
+  const int pairs = q_stride * c->group;
+  const int nseg = (cf.max_pages_per_seq * GM_PAGE + ATTN_BWD_SEG - 1) / ATTN_BWD_SEG;
+  if (pairs <= ATTN_BWD_MAX_PAIRS) {
+    const size_t np = pairs <= 4 ? 4 : (pairs <= 8 ? 8 : 16);
+    const size_t want = static_cast<size_t>(batch) * cf.n_kv_heads * nseg * np * 3;
+    if (want > c->ab_part_cap) {
+      int rc = dev_alloc(c, &c->ab_part, want);
+      if (rc != GM_OK) return rc;
+      c->ab_part_cap = want;
+    }
+  }
   AttnBwdArgs A;
+  if (pairs <= ATTN_BWD_MAX_PAIRS) { A.part = c->ab_part; A.nseg = nseg; }
   A.q = static_cast<const __nv_bfloat16 *>(q); A.dout = dout; A.pool = static_cast<const __nv_bfloat16 *>(kv_pool);
   A.qn = q_count; A.qbase = q_base; A.page_table = page_table;
   A.batch = batch; A.QT = q_stride; A.n_kv = cf.n_kv_heads; A.group = c->group; A.hd = cf.head_dim;
@@ -414,15 +435,15 @@ static int head_attn_backward_impl(gm_ctx *c, const float *x, const float *dxmid
   if (dqk_norm) { Q.tq = c->hat_tq; Q.tk = c->hat_tk; }
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_qkv_grad_rows(Q, c->stream));
   if (dqk_norm) {
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_tq, rows * cf.n_q_heads, hd, dqk_norm, c->stream, accum));
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_tk, rows * cf.n_kv_heads, hd, dqk_norm + hd, c->stream, accum));
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_tq, rows * cf.n_q_heads, hd, dqk_norm, c->stream, accum, colsum_ws(c)));
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_tk, rows * cf.n_kv_heads, hd, dqk_norm + hd, c->stream, accum, colsum_ws(c)));
   }
-  if (db_qkv) GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_dqkv, rows, NQKV, db_qkv, c->stream, accum));
+  if (db_qkv) GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_dqkv, rows, NQKV, db_qkv, c->stream, accum, colsum_ws(c)));
   // ---- dh = dqkv W_qkv;  dx = dxmid + d RMSNorm;  dln1 ----
   if ((rc = run_gemm(c, c->hat_dqkv_bf, rows, &c->hat_wqkv_t_map, c->hat_wqkv_t, rows, d, NQKV, c->hat_dh, EPI_STORE_F32, static_cast<size_t>(d), false)) != GM_OK)
     return rc;
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rmsnorm_grad(c->hat_dh, x, ln1, dx, rows, d, cf.rms_eps, c->stream, dxmid, c->hat_t));
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_t, rows, d, dln1, c->stream, accum));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hat_t, rows, d, dln1, c->stream, accum, colsum_ws(c)));
   // ---- weight gradients contract over the rows: operands transposed to [features, rows] (rows padded with zeros to Mp) ----
   GM_CUDA(c, cudaMemsetAsync(c->hat_dqkvt, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * NQKV, c->stream));
   GM_CUDA(c, cudaMemsetAsync(c->hat_ht, 0, sizeof(__nv_bfloat16) * static_cast<size_t>(Mp) * d, c->stream));
@@ -531,10 +552,10 @@ int gm_head_update_backward(gm_ctx *c, gm_state *st, int n_cycles, int k, const 
     if (rc) return rc;
     // every state's term through its own logits, and the final norm's weight
     const __nv_bfloat16 *gl = static_cast<const __nv_bfloat16 *>(grad_logits) + static_cast<size_t>(off) * k * c->V;
-    if ((rc = gm_head_state_grad(c, m * k, gl, c->hub_states, c->hub_gn, c->hub_dstate, refresh ? 1 : 0)) != GM_OK) return rc;
+    if ((rc = gm_head_state_grad(c, m * k, gl, c->hub_states, c->hub_gn, c->hub_dstate, 0)) != GM_OK) return rc;   // the LM head is the backbone's: its copy stays
     GM_LAUNCH(c, GM_KC_ELEMENTWISE,
               launch_rmsnorm_grad(c->hub_gn, c->hub_states, fnorm, nullptr, m * k, d, cf.rms_eps, c->stream, nullptr, c->hub_t));
-    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hub_t, m * k, d, out->final_norm, c->stream, true));
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_colsum(c->hub_t, m * k, d, out->final_norm, c->stream, true, colsum_ws(c)));
     for (int j = k; j >= 1; --j) {
       StepRowsArgs S;
       S.k = j; S.K = k; S.d = d; S.vocab = c->V; S.start_pos = rec->start_pos + off;

@@ -121,6 +121,8 @@ struct gm_ctx {
   float *hin_e = nullptr, *hin_dzin = nullptr, *hin_t = nullptr;
   float *ab_stats = nullptr;                // attention backward: (max, 1 / sum, D) per (row, query head)
   size_t ab_stats_cap = 0;
+  float *ab_part = nullptr;                 // partial statistics per key segment (the key-split kernels)
+  size_t ab_part_cap = 0;
   // one update of the head (gm_head_update_step): gradients, optimizer state (fp32 master, first and second moments, the
   // tensors one after the other, each padded to 4 elements), per-call buffers
   gm_head_grads hu_grads = {};
@@ -128,6 +130,7 @@ struct gm_ctx {
   __nv_bfloat16 *hu_logits = nullptr, *hu_glogits = nullptr;
   float *hu_alpha = nullptr, *hu_lse = nullptr, *hu_loss = nullptr;
   int hu_cycles_cap = 0, hu_step = 0;
+  float *colsum_ws = nullptr;               // partial column sums (64 chunks x the widest row: n_qkv or 2 d)
   // backward pass over a reconstruction: per-chunk states and their gradients, one pass's rows
   int hub_rows_cap = 0;
   float *hub_states = nullptr, *hub_gn = nullptr, *hub_dstate = nullptr, *hub_t = nullptr;          // [max_batch, max_k, d]

@@ -264,7 +264,9 @@ cudaError_t launch_head_input_rows(const __nv_bfloat16 *embed, const int32_t *to
 // dst [cols, dst_ld] = transpose of src [rows, cols] (bf16, both row-major; dst_ld >= rows, 0 = rows; padding untouched).
 cudaError_t launch_transpose_bf16(const __nv_bfloat16 *src, int rows, int cols, __nv_bfloat16 *dst, cudaStream_t stream, int dst_ld = 0);
 // out[j] = sum over rows of t[row][j] (fp32, row order).
-cudaError_t launch_colsum(const float *t, int rows, int d, float *out, cudaStream_t stream, bool add = false);
+// scratch (colsum_scratch_floats(d) floats, or null): lets many rows be split into chunks summed by separate CTAs
+cudaError_t launch_colsum(const float *t, int rows, int d, float *out, cudaStream_t stream, bool add = false, float *scratch = nullptr);
+size_t colsum_scratch_floats(int d);
 // Bookkeeping of the backward pass over a reconstruction (chains of recorded cycles; Eq. 4).
 struct StepRowsArgs {
   int k, K, d, vocab;                                   // application k (from 1) of K
@@ -377,11 +379,15 @@ struct AttnBwdArgs {
   const int32_t *qn, *qbase, *page_table;
   int batch, QT, n_kv, group, hd, qrows, layer, num_pages, max_pages_per_seq;
   float scale;                          // 1 / sqrt(hd)
-  float *stats, *dq;                    // dq [B * QT][n_q * hd]
+  float *stats, *dq;                    // dq [B * QT][n_q * hd], zero on entry (the key-split kernels add into it)
   float *dk_pool, *dv_pool;             // [num_pages][n_kv][16][hd], accumulated
+  float *part = nullptr;                // [B][n_kv][nseg][pairs][3] partial softmax statistics per key segment, or null
+  int nseg = 0;                         // segments the scratch holds per (sequence, KV head)
   uint32_t *status;
 };
 cudaError_t launch_attention_backward(const AttnBwdArgs &A, cudaStream_t stream);
+constexpr int ATTN_BWD_SEG = 256;       // keys per CTA of the key-split kernels
+constexpr int ATTN_BWD_MAX_PAIRS = 16;  // (row, query head of the group) pairs per (sequence, KV head) they hold in registers
 struct AttnCombineArgs {
   const float *part_o, *part_ml;
   const int32_t *qn, *page_start;

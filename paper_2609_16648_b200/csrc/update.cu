@@ -320,13 +320,35 @@ rmsnorm_grad_kernel(const float *gy, const float *x, const __nv_bfloat16 *w, flo
   }
 }
 
-// out[j] = sum over the rows of t[row][j], added in row order (fp32).
-__global__ void __launch_bounds__(256) colsum_kernel(const float *t, int rows, int d, float *out, int add) {
+// out[j] (+)= sum over the rows of t[row][j] (fp32), in a fixed order whatever the launch: a CTA sums 32 columns of one
+// chunk of rows - 32 row lanes striding the chunk, then the lanes in order - and, when the rows were split into several
+// chunks, a second kernel adds the chunks' partial sums in chunk order.
+constexpr int CS_COLS = 32, CS_LANES = 32, CS_MAX_CHUNKS = 64;
+__global__ void __launch_bounds__(CS_COLS * CS_LANES)
+colsum_kernel(const float *t, int rows, int d, int chunk_rows, float *out, int add) {
+  __shared__ float red[CS_LANES][CS_COLS + 1];
+  const int col = blockIdx.x * CS_COLS + threadIdx.x, ty = threadIdx.y;
+  const int r0 = blockIdx.y * chunk_rows, r1 = min(rows, r0 + chunk_rows);
+  pdl_prologue();
+  float acc = 0.f;
+  if (col < d)
+    for (int r = r0 + ty; r < r1; r += CS_LANES) acc += t[static_cast<size_t>(r) * d + col];
+  red[ty][threadIdx.x] = acc;
+  __syncthreads();
+  if (ty == 0 && col < d) {
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < CS_LANES; ++i) sum += red[i][threadIdx.x];
+    float *dst = out + static_cast<size_t>(blockIdx.y) * d + col;       // gridDim.y > 1: out is the partial-sum scratch
+    *dst = (add && gridDim.y == 1) ? *dst + sum : sum;
+  }
+}
+__global__ void __launch_bounds__(256) colsum_finish_kernel(const float *part, int chunks, int d, float *out, int add) {
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   pdl_prologue();
   if (j >= d) return;
   float acc = 0.f;
-  for (int r = 0; r < rows; ++r) acc += t[static_cast<size_t>(r) * d + j];
+  for (int c = 0; c < chunks; ++c) acc += part[static_cast<size_t>(c) * d + j];
   out[j] = add ? out[j] + acc : acc;
 }
 
@@ -629,8 +651,19 @@ cudaError_t launch_head_input_rows(const __nv_bfloat16 *embed, const int32_t *to
   return launch_k(head_input_rows_kernel, dim3(rows), dim3(NG_THREADS), 0, stream, 1, embed, tokens, hidden, we, wh, d, vocab, eps, zin,
                   e_out, status);
 }
-cudaError_t launch_colsum(const float *t, int rows, int d, float *out, cudaStream_t stream, bool add) {
-  return launch_k(colsum_kernel, dim3((d + 255) / 256), dim3(256), 0, stream, 1, t, rows, d, out, add ? 1 : 0);
+size_t colsum_scratch_floats(int d) { return static_cast<size_t>(CS_MAX_CHUNKS) * d; }
+cudaError_t launch_colsum(const float *t, int rows, int d, float *out, cudaStream_t stream, bool add, float *scratch) {
+  // enough CTAs to fill the device when there are many rows; a single chunk needs no scratch
+  const int col_blocks = (d + CS_COLS - 1) / CS_COLS;
+  int chunks = 1;
+  if (scratch) chunks = std::max(1, std::min(std::min(CS_MAX_CHUNKS, rows / 64), (4 * 148 + col_blocks - 1) / col_blocks));
+  const int chunk_rows = (rows + chunks - 1) / chunks;
+  chunks = (rows + chunk_rows - 1) / chunk_rows;
+  const dim3 grid(col_blocks, chunks), block(CS_COLS, CS_LANES);
+  if (chunks == 1) return launch_k(colsum_kernel, grid, block, 0, stream, 1, t, rows, d, chunk_rows, out, add ? 1 : 0);
+  if (cudaError_t e = launch_k(colsum_kernel, grid, block, 0, stream, 1, t, rows, d, chunk_rows, scratch, 0); e != cudaSuccess) return e;
+  return launch_k(colsum_finish_kernel, dim3((d + 255) / 256), dim3(256), 0, stream, 1, static_cast<const float *>(scratch), chunks, d, out,
+                  add ? 1 : 0);
 }
 cudaError_t launch_step_rows(const StepRowsArgs &A, int chains, cudaStream_t stream) {
   return launch_k(step_rows_kernel, dim3(chains), dim3(128), 0, stream, 1, A);
