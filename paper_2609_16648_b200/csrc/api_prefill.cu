@@ -100,8 +100,9 @@ int gm_prefill(gm_ctx *c, gm_state *st, const int32_t *prompt_tok, const int32_t
       GM_LAUNCH(c, GM_KC_ELEMENTWISE,
                 launch_rmsnorm(c->x, static_cast<const __nv_bfloat16 *>(c->w.head_layer.ln1), c->xn, nullptr, ph.M, c->d,
                                cf.rms_eps, c->stream));
+      // only the pairs' cache entries matter: the head's outputs on prompt rows are read by nothing
       rc = run_layer(c, c->w.head_layer, c->head_maps, ph, hkvm, static_cast<__nv_bfloat16 *>(st->head_kv_pool), 0,
-                     cf.head_num_pages, c->pf_vtable[1], nullptr, nullptr);
+                     cf.head_num_pages, c->pf_vtable[1], nullptr, nullptr, nullptr, nullptr, false, true);
       if (rc) return rc;
     }
   }
@@ -163,7 +164,7 @@ int gm_head_prefill(gm_ctx *c, gm_state *st, const void *seq_hidden, int hid_str
               launch_rmsnorm(c->x, static_cast<const __nv_bfloat16 *>(c->w.head_layer.ln1), c->xn, nullptr, ph.M, c->d,
                              cf.rms_eps, c->stream));
     rc = run_layer(c, c->w.head_layer, c->head_maps, ph, hkvm, static_cast<__nv_bfloat16 *>(st->head_kv_pool), 0,
-                   cf.head_num_pages, c->pf_vtable[1], nullptr, nullptr);
+                   cf.head_num_pages, c->pf_vtable[1], nullptr, nullptr, nullptr, nullptr, false, true);   // cache entries only
     if (rc) return rc;
   }
   return GM_OK;

@@ -178,13 +178,13 @@ int run_chain(gm_ctx *c, const ChainSpec *specs, int n, int M) {
   return GM_OK;
 }
 
-// One decoder layer on rows x/xn [M, d] (xn = normed input).  `next_norm` is the RMSNorm weight applied to
+// One decoder layer on rows x/xn [M, d] (xn = normed input).  kv_only: stop after the rows' keys and values are in the cache.  `next_norm` is the RMSNorm weight applied to
 // the layer's output for whatever consumes it next (null: none); `hidden_out` optionally receives the
 // bf16 residual stream.
 int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const PhaseShape &ph, const CUtensorMap &kvm,
               __nv_bfloat16 *pool, int layer, int num_pages, const int32_t *page_table,
               const __nv_bfloat16 *next_norm, __nv_bfloat16 *hidden_out, const gm_layer_weights *next_lw,
-              const LayerMaps *next_lm, bool qkv_done) {
+              const LayerMaps *next_lm, bool qkv_done, bool kv_only) {
   const gm_config &cf = c->cfg;
   const bool chain = chain_usable(c, ph.M);
   int rc;
@@ -213,6 +213,7 @@ int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const 
     if (rc) return rc;
   }
   if (!fuse_rope) GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rope_append(R, c->stream));
+  if (kv_only) return GM_OK;          // the rows' cache entries are all the caller needs (nothing reads their outputs)
   // attention over the pages + merge of the segments
   AttnArgs T;
   T.kv_map = kvm; T.qbuf = c->qbuf; T.qn = c->qn; T.qbase = c->qbase; T.page_start = c->page_start;

@@ -240,7 +240,7 @@ struct PhaseShape { int B, QT, M, qrows; };
 int run_layer(gm_ctx *c, const gm_layer_weights &lw, const LayerMaps &lm, const PhaseShape &ph, const CUtensorMap &kvm,
               __nv_bfloat16 *pool, int layer, int num_pages, const int32_t *page_table,
               const __nv_bfloat16 *next_norm, __nv_bfloat16 *hidden_out, const gm_layer_weights *next_lw = nullptr,
-              const LayerMaps *next_lm = nullptr, bool qkv_done = false);
+              const LayerMaps *next_lm = nullptr, bool qkv_done = false, bool kv_only = false);
 bool chain_usable(const gm_ctx *c, int M);
 // One projection of a chain (see ChainPhase); the input is x [x_rows, K] bf16.
 struct ChainSpec {

@@ -505,13 +505,19 @@ def test_head_attn_backward_matches_the_oracle(name, family):
     ctx.close()
 
 
-def _update_setup(family, n_steps=3):
+def _update_setup(family, n_steps=3, dims="tiny"):
     """A short oracle rollout with its records, and a device context / state / record holding the same cycles."""
     import paper_2609_16648_b200 as gmb
     cfg = get_config("tiny").with_(prompt_len=12, qk_norm=family == "qk_norm", qkv_bias=family == "qkv_bias")
+    if dims == "4b":                                     # the 4B head's layer (one backbone layer, a small vocabulary)
+        cfg = cfg.with_(n_layers=1, d_model=2560, n_q_heads=32, n_kv_heads=8, head_dim=128, d_ffn=9728)
     B, K, V, d = cfg.batch, cfg.k, cfg.vocab, cfg.d_model
     w = perturb_norm_weights(make_weights(cfg, 0))
-    st, cycles, seqs, hpt, hnpg = _oracle_rollout(cfg, w, n_steps=3)
+    st, cycles, seqs, hpt, hnpg = _oracle_rollout(cfg, w, n_steps=n_steps)
+    if not any(r["accepted"] >= 2 for _, r in cycles):
+        # random weights of this size reject every first draft; the objective is defined for any first rejected position,
+        # so spread it over 1 .. K + 1 for the chains to reach the recurrence
+        cycles = [(b_, dict(r, accepted=i % (K + 1) + 1)) for i, (b_, r) in enumerate(cycles)]
     n = len(cycles)
     assert any(r["accepted"] >= 2 for _, r in cycles)                     # some chains reach the recurrence
     ctx = gmb.Context(cfg, gmb.pack_weights(w), B, K, hpt.shape[1], hnpg, hnpg + 2 * n)
@@ -537,13 +543,14 @@ def _update_setup(family, n_steps=3):
                 max_len=int(seq_len.max()), rec=rec, cycle_seq=cycle_seq, scratch=scratch, hnpg=hnpg)
 
 
-@pytest.mark.parametrize("family", ["plain", "qk_norm", "qkv_bias"])
-def test_head_update_backward_matches_the_oracle(family):
+@pytest.mark.parametrize("family,dims", [("plain", "tiny"), ("qk_norm", "tiny"), ("qkv_bias", "tiny"), ("qk_norm", "4b")],
+                         ids=["plain", "qk_norm", "qkv_bias", "qk_norm-4b_head_dimensions"])
+def test_head_update_backward_matches_the_oracle(family, dims):
     """gm_head_update_backward - the whole backward pass over recorded cycles, chains replayed three chunks of max_batch
     at a time - against the oracle's head_update_grad on the weights the device holds, both starting from the device's
     own logit gradients (the piecewise-linear overlap picks its branches from the logits, which differ in rounding).
     Every parameter tensor of the head; the oracle's is pinned by finite differences of the objective."""
-    u = _update_setup(family)
+    u = _update_setup(family, n_steps=3 if dims == "tiny" else 2, dims=dims)
     gmb, cfg, w, cycles, seqs, n, ctx, gst = (u[k_] for k_ in ("gmb", "cfg", "w", "cycles", "seqs", "n", "ctx", "gst"))
     tok_d, len_d, hid_d, rec, cycle_seq, scratch, hnpg = (u[k_] for k_ in ("tok_d", "len_d", "hid_d", "rec", "cycle_seq", "scratch", "hnpg"))
     B, K, V, d = cfg.batch, cfg.k, cfg.vocab, cfg.d_model
@@ -669,6 +676,59 @@ def test_head_update_steps_lower_the_objective_and_equal_the_calls_made_one_by_o
     assert losses[-1] < losses[0] - 0.02 and min(losses[1:]) < losses[0]
     assert torch.equal(ctx.packed["lm_head"], frozen["lm_head"]) and torch.equal(ctx.packed["embed"], frozen["embed"])
     assert torch.equal(ctx.packed["final_norm"], frozen["final_norm"]) and torch.equal(ctx.packed["layers"][0]["wqkv"], frozen["l0.wqkv"])
+    ctx.close()
+
+
+@pytest.mark.parametrize("n_seq,L,n", [(8, 512, 64), (64, 512, 256)], ids=["8x512_64_cycles", "64x512_256_cycles"])
+def test_head_update_step_at_the_4b_head_dimensions_runs_and_is_timed(n_seq, L, n):
+    """gm_head_update_step on the 4B head (d 2560, 32/8 heads of 128, FFN 9728, head norms, the full 151936 vocabulary) over
+    synthetic records: n cycles spread over n_seq recorded sequences of L positions, k = 3, chains in chunks of 64.  There
+    is no oracle at this size (the 4B-dimension parity case of the backward pass runs on a small vocabulary); this checks
+    that the call runs clean at the full shapes - status, finite objective, every matrix of the head moved, the backbone's
+    tensors untouched - and prints the time per update."""
+    import paper_2609_16648_b200 as gmb
+    K = 3
+    cfg = get_config("4b").with_(n_layers=1, batch=n_seq, qk_norm=True)
+    d, V = cfg.d_model, cfg.vocab
+    hpt, hnpg = make_page_tables(np.full(n_seq, L + 8), 16, seed=8)
+    ctx = gmb.Context(cfg, gmb.random_packed_weights(cfg, "cuda"), 64, K, hpt.shape[1], 8, hnpg + 2 * n)
+    gst = gmb.State(ctx, n_seq, hpt, hpt)
+    g = torch.Generator(device="cuda").manual_seed(1)
+    tok = torch.randint(0, V, (n_seq, L), device="cuda", generator=g, dtype=torch.int32)
+    hid = torch.randn((n_seq, L, d), device="cuda", generator=g).to(torch.bfloat16)
+    slen = torch.full((n_seq,), L, dtype=torch.int32, device="cuda")
+    rng = np.random.default_rng(3)
+    seq = rng.integers(0, n_seq, n).astype(np.int32)
+    start = rng.integers(L // 2, L - K - 1, n).astype(np.int32)
+    rec = gmb.Record(n, K, d)
+    rec.start_pos.copy_(torch.from_numpy(start))
+    rec.start_hidden.copy_(hid[torch.from_numpy(seq).long().cuda(), torch.from_numpy(start - 2).long().cuda()])
+    rec.drafts.copy_(torch.randint(0, V, (n, K), device="cuda", generator=g, dtype=torch.int32))
+    order = torch.rand((n * K, V), device="cuda", generator=g).topk(64, dim=-1).indices            # 64 distinct ids per row
+    rec.top_index.copy_(order.reshape(n, K, 64).to(torch.int32))
+    lp = torch.log_softmax(torch.randn((n, K, 64), device="cuda", generator=g) * 2, -1) - 0.3     # 26 % of the mass in the residual bin
+    rec.top_logprob.copy_(lp.sort(dim=-1, descending=True).values.to(torch.bfloat16))
+    rec.accepted.copy_(torch.randint(1, K + 2, (n,), device="cuda", generator=g, dtype=torch.int32))
+    cyc = torch.from_numpy(seq).cuda()
+    scratch = torch.arange(hnpg, hnpg + 2 * n, dtype=torch.int32, device="cuda").reshape(n, 2)
+    mean = torch.zeros(1, device="cuda")
+    before = {k_: t.clone() for k_, t in _head_params(ctx.packed).items()}
+    lm_head = ctx.packed["lm_head"].clone()
+    losses, ev = [], [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    for s_ in range(1, 6):
+        if s_ == 3:
+            ev[0].record()
+        gmb.gm_head_update_step(ctx, gst, n, K, 1.0, cyc, rec, tok, scratch, hid, slen, L, s_, 1e-4, mean)
+        losses.append(float(mean[0]))
+    ev[1].record()
+    torch.cuda.synchronize()
+    assert gmb.gm_last_status(ctx) == 0
+    assert all(np.isfinite(losses)), losses
+    after = _head_params(ctx.packed)
+    assert all(not torch.equal(after[k_], before[k_]) for k_ in after if after[k_].dim() == 2)
+    assert torch.equal(ctx.packed["lm_head"], lm_head)
+    print(f"gm_head_update_step, 4B head, {n} cycles over {n_seq} x {L} positions: {ev[0].elapsed_time(ev[1]) / 3:.1f} ms per update; "
+          f"objective before each update {[round(x, 4) for x in losses]}")
     ctx.close()
 
 
