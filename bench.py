@@ -9,6 +9,8 @@ seeded synthetic sequences; consecutive steps feed on each other's committed sta
 whole-job committed tokens per second with all inputs resident in HBM; `e2e` is the same metric
 through the host-buffer entry point (uniforms copied from pinned host memory, results copied back,
 every step).  With N > 1 every rank runs an independent replica (no collective on the data path).
+Other workloads, each with its own line: `--workload sampler` (accept / resample alone), `--workload rollout` (prefill +
+cycles with the library's page allocator), `--workload head_update` (one update of the draft head on recorded cycles).
 """
 from __future__ import annotations
 
@@ -855,12 +857,142 @@ def run_dry(args):
         dist.destroy_process_group()
 
 
+def run_head_update(args):
+    """Head-update workload (not the default line): one update of the draft head (Alg. 1, "update phi") per step on synthetic
+    recorded cycles at the 4B head's dimensions - 256 cycles spread over 64 recorded sequences of 512 positions, chains
+    replayed in chunks of 64.  A step is one gm_head_update_step: cache rebuild, reconstruction, objective, backward pass
+    over every head parameter, AdamW.  `e2e` adds the upload of the step's records from pinned host memory and the
+    download of the objective."""
+    import torch
+    import paper_2609_16648_b200 as gmb
+    from paper_2609_16648_b200.build import build
+    from synth_inputs import get_config, make_page_tables
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the product path has no CPU fallback")
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    if rank == 0:
+        build()
+    if world > 1:
+        dist.barrier()
+    K, W, S = args.k, args.warmup, args.steps
+    n_seq, L, n = (args.batch if args.batch > 0 else 64), 512, 256
+    cfg = get_config("4b").with_(n_layers=1, batch=n_seq, k=K, qk_norm=True)
+    d, V, F = cfg.d_model, cfg.vocab, cfg.d_ffn
+    hpt, hnpg = make_page_tables(np.full(n_seq, L + 8), 16, seed=8 + rank)
+    ctx = gmb.Context(cfg, gmb.random_packed_weights(cfg, device, seed=rank), 64, K, hpt.shape[1], 8, hnpg + 2 * n)
+    gst = gmb.State(ctx, n_seq, hpt, hpt, device)
+    g = torch.Generator(device=device).manual_seed(1 + rank)
+    tok = torch.randint(0, V, (n_seq, L), device=device, generator=g, dtype=torch.int32)
+    hid = torch.randn((n_seq, L, d), device=device, generator=g).to(torch.bfloat16)
+    slen = torch.full((n_seq,), L, dtype=torch.int32, device=device)
+    rng = np.random.default_rng(3 + rank)
+    seq = rng.integers(0, n_seq, n).astype(np.int32)
+    start = rng.integers(L // 2, L - K - 1, n).astype(np.int32)
+    rec = gmb.Record(n, K, d, device)
+    rec.start_pos.copy_(torch.from_numpy(start))
+    rec.start_hidden.copy_(hid[torch.from_numpy(seq).long().to(device), torch.from_numpy(start - 2).long().to(device)])
+    rec.drafts.copy_(torch.randint(0, V, (n, K), device=device, generator=g, dtype=torch.int32))
+    rec.top_index.copy_(torch.rand((n * K, V), device=device, generator=g).topk(64, dim=-1).indices.reshape(n, K, 64).to(torch.int32))
+    lp = torch.log_softmax(torch.randn((n, K, 64), device=device, generator=g) * 2, -1) - 0.3
+    rec.top_logprob.copy_(lp.sort(dim=-1, descending=True).values.to(torch.bfloat16))
+    rec.accepted.copy_(torch.randint(1, K + 2, (n,), device=device, generator=g, dtype=torch.int32))
+    cyc = torch.from_numpy(seq).to(device)
+    scratch = torch.arange(hnpg, hnpg + 2 * n, dtype=torch.int32, device=device).reshape(n, 2)
+    mean = torch.zeros(1, device=device)
+    step_no = [0]
+
+    def step():
+        step_no[0] += 1
+        gmb.gm_head_update_step(ctx, gst, n, K, 1.0, cyc, rec, tok, scratch, hid, slen, L, step_no[0], 1e-4, mean)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(W):
+        step()
+    clocks = ClockSampler(local)
+    launches0 = gmb.gm_launch_count(ctx)
+    barrier()
+    clocks.start()
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    e[0].record()
+    for _ in range(S):
+        step()
+    e[1].record()
+    barrier()
+    clk = clocks.stop()
+    ms = e[0].elapsed_time(e[1])
+    launches = gmb.gm_launch_count(ctx) - launches0
+    # end to end: the step's records come from pinned host memory, the objective goes back
+    fields = ("start_hidden", "start_pos", "drafts", "top_logprob", "top_index", "accepted")
+    host = {f: getattr(rec, f).cpu().pin_memory() for f in fields}
+    mean_h = torch.zeros(1).pin_memory()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(S):
+        for f in fields:
+            getattr(rec, f).copy_(host[f], non_blocking=True)
+        step()
+        mean_h.copy_(mean, non_blocking=True)
+        torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) * 1e3
+    h2d = sum(host[f].numel() * host[f].element_size() for f in fields)
+    # device time of the projections, every launch bracketed by events, in a pass of its own
+    gmb.gm_profile(ctx, 1 << 0)
+    step()
+    gemm_ms, gemm_n = gmb.gm_profile_read(ctx, 0)
+    gmb.gm_profile(ctx, 0)
+    status = gmb.gm_last_status(ctx)
+    if status != 0 or not np.isfinite(float(mean[0])):
+        raise RuntimeError(f"head_update workload: status {status}, objective {float(mean[0])}")
+    (ms_max, e2e_max), (launches_all,) = reduce_over_ranks([ms, e2e_ms], [launches], device, world)
+    if rank == 0:
+        _, burst, sustained, which = measured_peaks()
+        nqkv, q = cfg.q_dim + 2 * cfg.kv_dim, cfg.q_dim
+        P, C = n_seq * (L - 1), n * K                     # prefix rows, chain rows (one per application)
+        zf, qf, of, ff, lf = 2.0 * 2 * d * d, 2.0 * nqkv * d, 2.0 * q * d, 2.0 * F * d, 2.0 * V * d
+        # prefix rows: z and QKV in the rebuild and again in the backward pass, then dh, dW_qkv, d zin, dW_p
+        flops = P * (2 * (zf + qf) + 2 * qf + 2 * zf)
+        # chain rows: two replays (z, layer, LM head), LM-head gradient, feed-forward backward (recomputed gate/up + four
+        # products), attention half (z, QKV, W_o forward; d out, dh, two weight gradients), input (d zin, dW_p)
+        flops += C * (2 * (zf + qf + of + 3 * ff + lf) + lf + (2 * ff + ff + 2 * ff + ff + 2 * ff) + (zf + qf + of + of + qf + of + qf) + 2 * zf)
+        tf = flops / (gemm_ms * 1e-3) / 1e12
+        line = {"metric": "head_update_cycles_per_s", "value": n * S * world / (ms_max * 1e-3), "unit": "recorded cycles/s",
+                "n_gpus": world, "steps": S, "warmup": W, "ms_per_step": ms_max / S, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": "head_update", "cycles_per_step": n, "sequences": n_seq, "positions": L, "k": K,
+                           "head": "4B dimensions (d 2560, 32/8 heads of 128 with head norms, FFN 9728, vocabulary 151936)",
+                           "chains_per_chunk": 64, "l2": "the head's matrices and fp32 gradients (0.7 GB) exceed the 126 MB L2: no flush needed",
+                           "peaks": which},
+                "clocks": clk,
+                "e2e": {"value": n * S * world / (e2e_max * 1e-3), "unit": "recorded cycles/s", "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": 4, "ms_per_step": e2e_max / S},
+                "gpu_launches": int(launches_all),
+                "roofline": {"kernel": "gemm_tc_kernel (every product of the update: forward recomputation, input gradients, weight gradients)",
+                             "bound": "tensor", "achieved": tf, "peak": burst, "unit": "TFLOP/s", "frac": tf / burst,
+                             "frac_of_sustained": tf / sustained, "traffic": None, "launches": int(gemm_n), "ms_per_step": gemm_ms,
+                             "flops_per_step": flops, "peak_source": which,
+                             "note": "launches bracketed by events one by one in a separate pass; most products have 64 or 2048 rows"}}
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="4b", choices=["tiny", "4b", "7b", "longtail", "sampler", "rollout"])
+    ap.add_argument("--workload", default="4b", choices=["tiny", "4b", "7b", "longtail", "sampler", "rollout", "head_update"])
     ap.add_argument("--k", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (small profiling cases)")
@@ -885,6 +1017,8 @@ def main():
         run_sampler_only(args)
     elif args.workload == "rollout":
         run_rollout(args)
+    elif args.workload == "head_update":
+        run_head_update(args)
     else:
         run_product(args)
 
