@@ -108,6 +108,19 @@ int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *w
   const int mblocks = (M + T - 1) / T;
   const int tiles128 = (N + 127) / 128;
   A.nsplit = pick_split(c, M, N, K, T);
+  // A split projection whose tiles pair up: two 128-feature sub-tiles per CTA share one activation box, so a CTA moves
+  // 2/3 of the bytes per unit of MMA work (the main loops are bound by filling shared memory), with more K slices to
+  // keep the SMs filled.  Taken when it does not leave more SMs idle than the one-sub-tile form.
+  if (c->wide_split && A.nsplit > 1 && T == 256 && mblocks == 1 && (tiles128 % 2) == 0) {
+    const int units2 = tiles128 / 2, KB = K / 64;
+    int best = 0;
+    for (int ns = 2; ns <= 8 && ns <= KB; ++ns) {
+      int &cap = c->max_clusters[T / 16][ns];
+      if (cap < 0) { int v = 0; if (gemm_tc_max_clusters(T, ns, &v) != cudaSuccess) { v = 0; (void)cudaGetLastError(); } cap = v; }
+      if (cap >= units2) best = ns;
+    }
+    if (best > 0 && units2 * best >= tiles128 * A.nsplit) { A.wtiles = 2; A.nsplit = best; }
+  }
   // very wide projections: two sub-tiles per CTA halve the activation re-reads from L2
   if (A.nsplit == 1 && tiles128 * mblocks >= 2 * c->sm_count) A.wtiles = 2;
   const int units = (tiles128 + A.wtiles - 1) / A.wtiles;          // CTAs along N
@@ -477,6 +490,7 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
     c->flow_ws = ws;
   }
   if (std::getenv("GM_NO_EARLY_W")) c->early_weights = false;
+  if (const char *ws = std::getenv("GM_GEMM_WIDE_SPLIT")) c->wide_split = std::atoi(ws) != 0;
   if (std::getenv("GM_FUSED_ROPE")) c->fuse_rope = true;
   if (const char *ov = std::getenv("GM_SAMPLER")) {     // tuning aid: cluster | stream | flow for every sampler launch
     c->sampler_mode = !std::strcmp(ov, "cluster") ? 1 : !std::strcmp(ov, "stream") ? 2 : !std::strcmp(ov, "flow") ? 3 : 0;
