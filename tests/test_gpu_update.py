@@ -505,10 +505,10 @@ def test_head_attn_backward_matches_the_oracle(name, family):
     ctx.close()
 
 
-def _update_setup(family, n_steps=3, dims="tiny", prompt_len=12):
+def _update_setup(family, n_steps=3, dims="tiny", prompt_len=12, k=3, max_k=None):
     """A short oracle rollout with its records, and a device context / state / record holding the same cycles."""
     import paper_2609_16648_b200 as gmb
-    cfg = get_config("tiny").with_(prompt_len=prompt_len, qk_norm=family == "qk_norm", qkv_bias=family == "qkv_bias")
+    cfg = get_config("tiny").with_(prompt_len=prompt_len, qk_norm=family == "qk_norm", qkv_bias=family == "qkv_bias", k=k)
     if dims == "4b":                                     # the 4B head's layer (one backbone layer, a small vocabulary)
         cfg = cfg.with_(n_layers=1, d_model=2560, n_q_heads=32, n_kv_heads=8, head_dim=128, d_ffn=9728)
     B, K, V, d = cfg.batch, cfg.k, cfg.vocab, cfg.d_model
@@ -520,7 +520,7 @@ def _update_setup(family, n_steps=3, dims="tiny", prompt_len=12):
         cycles = [(b_, dict(r, accepted=i % (K + 1) + 1)) for i, (b_, r) in enumerate(cycles)]
     n = len(cycles)
     assert any(r["accepted"] >= 2 for _, r in cycles)                     # some chains reach the recurrence
-    ctx = gmb.Context(cfg, gmb.pack_weights(w), B, K, hpt.shape[1], hnpg, hnpg + 2 * n)
+    ctx = gmb.Context(cfg, gmb.pack_weights(w), B, max_k or K, hpt.shape[1], hnpg, hnpg + 2 * n)
     gst = gmb.State(ctx, B, hpt, hpt)
     S = max(len(t) for _, t in seqs)
     seq_tok, seq_hid, seq_len = np.zeros((B, S), np.int32), np.zeros((B, S, d), np.float32), np.zeros(B, np.int32)
@@ -543,18 +543,20 @@ def _update_setup(family, n_steps=3, dims="tiny", prompt_len=12):
                 max_len=int(seq_len.max()), rec=rec, cycle_seq=cycle_seq, scratch=scratch, hnpg=hnpg)
 
 
-@pytest.mark.parametrize("family,dims,prompt_len", [("plain", "tiny", 12), ("qk_norm", "tiny", 12), ("qkv_bias", "tiny", 12),
-                                                    ("qk_norm", "4b", 12), ("plain", "tiny", 1), ("qk_norm", "tiny", 15)],
+@pytest.mark.parametrize("family,dims,prompt_len,k,max_k",
+                         [("plain", "tiny", 12, 3, 3), ("qk_norm", "tiny", 12, 3, 3), ("qkv_bias", "tiny", 12, 3, 3),
+                          ("qk_norm", "4b", 12, 3, 3), ("plain", "tiny", 1, 3, 3), ("qk_norm", "tiny", 15, 3, 3),
+                          ("plain", "tiny", 12, 2, 4), ("plain", "tiny", 12, 5, 5)],
                          ids=["plain", "qk_norm", "qkv_bias", "qk_norm-4b_head_dimensions", "plain-one_token_prompts",
-                              "qk_norm-first_chain_entry_on_a_page_boundary"])
-def test_head_update_backward_matches_the_oracle(family, dims, prompt_len):
+                              "qk_norm-first_chain_entry_on_a_page_boundary", "plain-k2_in_a_context_of_max_k4", "plain-k5"])
+def test_head_update_backward_matches_the_oracle(family, dims, prompt_len, k, max_k):
     """gm_head_update_backward - the whole backward pass over recorded cycles, chains replayed three chunks of max_batch
     at a time - against the oracle's head_update_grad on the weights the device holds, both starting from the device's
     own logit gradients (the piecewise-linear overlap picks its branches from the logits, which differ in rounding).
     Every parameter tensor of the head; the oracle's is pinned by finite differences of the objective."""
     # one-token prompts: the first cycle starts at length 2, its chain's first entry is position 0 and its prefix is empty;
     # 15-token prompts: length 16 + 2 at the second cycle or so puts a chain's first entry at slot 0 of a page (nothing to fold)
-    u = _update_setup(family, n_steps=3 if dims == "tiny" else 2, dims=dims, prompt_len=prompt_len)
+    u = _update_setup(family, n_steps=3 if dims == "tiny" else 2, dims=dims, prompt_len=prompt_len, k=k, max_k=max_k)
     gmb, cfg, w, cycles, seqs, n, ctx, gst = (u[k_] for k_ in ("gmb", "cfg", "w", "cycles", "seqs", "n", "ctx", "gst"))
     tok_d, len_d, hid_d, rec, cycle_seq, scratch, hnpg = (u[k_] for k_ in ("tok_d", "len_d", "hid_d", "rec", "cycle_seq", "scratch", "hnpg"))
     B, K, V, d = cfg.batch, cfg.k, cfg.vocab, cfg.d_model
