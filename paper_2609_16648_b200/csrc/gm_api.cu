@@ -152,6 +152,15 @@ int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *w
     GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(Tl, c->stream));
     return GM_OK;
   }
+  // Several token blocks (prefill passes, the head update's prefix passes) on a projection too narrow for two sub-tiles
+  // per CTA: CTA pairs, each CTA staging half of the activation box (2/3 of the bytes into shared memory per K block).
+  if (c->pair_gemm && c->pair_blocks && A.nsplit == 1 && A.wtiles == 1 && mblocks > 1 && T == 256 && (units % 2) == 0 &&
+      epi != EPI_QKV_ROPE) {
+    rc = x_map(c, x, x_rows, K, T / 2, &A.x_half_map);
+    if (rc != GM_OK) return rc;
+    GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_pair(A, c->stream));
+    return GM_OK;
+  }
   GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_tc(A, c->stream));
   return GM_OK;
 }
@@ -491,6 +500,7 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
   }
   if (std::getenv("GM_NO_EARLY_W")) c->early_weights = false;
   if (const char *ws = std::getenv("GM_GEMM_WIDE_SPLIT")) c->wide_split = std::atoi(ws) != 0;
+  if (const char *pb = std::getenv("GM_GEMM_PAIR_BLOCKS")) c->pair_blocks = std::atoi(pb) != 0;
   if (std::getenv("GM_FUSED_ROPE")) c->fuse_rope = true;
   if (const char *ov = std::getenv("GM_SAMPLER")) {     // tuning aid: cluster | stream | flow for every sampler launch
     c->sampler_mode = !std::strcmp(ov, "cluster") ? 1 : !std::strcmp(ov, "stream") ? 2 : !std::strcmp(ov, "flow") ? 3 : 0;
