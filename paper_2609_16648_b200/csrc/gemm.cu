@@ -21,7 +21,7 @@
 // ST_TIMEOUT, still meets every barrier and frees its tensor memory.
 //
 // gemm_pair_kernel: the same projection on pairs of CTAs (tcgen05 cta_group::2) for full waves of one-slice tiles;
-// described at the kernel.
+// gemm_pair_split_kernel: pairs with K slices (cluster 2 x slices) for split projections.  Both described at the kernels.
 //
 // gemm_simple_kernel: a plain warp-level mma.sync version with the same epilogues, kept as an
 // independent on-device cross-check and for shapes the tcgen05 kernel does not take.
@@ -420,6 +420,134 @@ gemm_pair_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
   if (warp == 1) tc2_dealloc(tmem, ncols);
 }
 
+// ---- CTA pairs with K slices ---------------------------------------------------------------------------------------------
+// The pair kernel for projections with few output tiles: cluster (2, 1, ns) = ns pairs on one 256-feature tile, pair z
+// taking K slice z.  Inside a pair everything is as above (the leader is the even rank of the pair; barriers and commits
+// address the pair's two CTAs by their cluster ranks); afterwards every CTA parks its 128-feature accumulator and sums
+// one slice of the tile's tokens over the ns CTAs that hold the same features, in slice order, through distributed
+// shared memory - the reduction of gemm_tc_kernel.
+__global__ void __launch_bounds__(GT_THREADS, 1)
+gemm_pair_split_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
+  extern __shared__ unsigned char gt_smem_raw[];
+  unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(gt_smem_raw) + 1023) & ~uintptr_t(1023));
+  const int T = A.block_t, H = T / 2;
+  const int a_bytes = GT_BN * 128, b_bytes = H * 128, stage_b = a_bytes + b_bytes;
+  size_t pipe_b = static_cast<size_t>(nstages) * stage_b;
+  if (static_cast<size_t>(T) * GT_BN * 4 > pipe_b) pipe_b = static_cast<size_t>(T) * GT_BN * 4;
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem + pipe_b);
+  uint64_t *empty = full + 8;
+  uint64_t *acc_full = empty + 8;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  float *park = reinterpret_cast<float *>(smem);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();            // x + 2 z within the cluster
+  const uint32_t half = rank & 1u, lead_rank = rank & ~1u;
+  const bool leader = half == 0;
+  const int ns = A.nsplit, split = blockIdx.z;
+  const int n0 = A.n_base + blockIdx.x * GT_BN, m0 = blockIdx.y * T;
+  const int KB = A.K / GT_BK;
+  const int kb_lo = static_cast<int>(static_cast<long long>(split) * KB / ns);
+  const int kb_hi = static_cast<int>(static_cast<long long>(split + 1) * KB / ns);
+  const uint32_t ncols = T <= 32 ? 32u : T <= 64 ? 64u : T <= 128 ? 128u : 256u;
+  const uint16_t pair_mask = static_cast<uint16_t>(3u << lead_rank);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < nstages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    tc2_alloc(tmem_slot, ncols);
+    tc2_relinquish();
+  }
+  if (warp == 0 && lane == 0) {
+    tma_prefetch_desc(&A.w_map);
+    tma_prefetch_desc(&A.x_half_map);
+  }
+  tc_fence_before();
+  cg::cluster_group cluster = cg::this_cluster();
+  cluster.sync();                                  // every CTA's barriers exist before anything arrives on them
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  pdl_prologue();
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int kb = kb_lo, it = 0; kb < kb_hi; ++kb, ++it) {
+        const int s = it % nstages;
+        if (!mbar_wait(&empty[s], ((it / nstages) & 1) ^ 1)) { set_status(A.status, ST_TIMEOUT); break; }
+        if (leader) mbar_expect_tx(&full[s], 2 * stage_b);
+        const uint32_t bar = cluster_addr(&full[s], lead_rank);
+        unsigned char *dst = smem + static_cast<size_t>(s) * stage_b;
+        tma2_load_2d(dst, &A.w_map, kb * GT_BK, n0, bar);
+        tma2_load_2d(dst + a_bytes, &A.x_half_map, kb * GT_BK, m0 + static_cast<int>(half) * H, bar);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && leader) {
+      const uint32_t idesc = tc_idesc_bf16(2 * GT_BN, T);
+      bool ok = true;
+      for (int kb = kb_lo, it = 0; kb < kb_hi; ++kb, ++it) {
+        const int s = it % nstages;
+        if (!mbar_wait(&full[s], (it / nstages) & 1)) { set_status(A.status, ST_TIMEOUT); ok = false; break; }
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(smem + static_cast<size_t>(s) * stage_b);
+        const uint64_t adesc = tc_smem_desc_sw128(a_addr), bdesc = tc_smem_desc_sw128(a_addr + a_bytes);
+#pragma unroll
+        for (int k = 0; k < GT_BK / 16; ++k)
+          tc2_mma_bf16(tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+        tc2_commit_mc(&empty[s], pair_mask);        // the stage is free in both CTAs of the pair
+      }
+      if (ok) tc2_commit_mc(acc_full, pair_mask);
+    }
+  }
+  bool acc_ok = kb_hi > kb_lo;
+  const bool reader = warp >= 2 && warp < 10;
+  if (reader) {
+    if (acc_ok && !mbar_wait(acc_full, 0)) { set_status(A.status, ST_TIMEOUT); acc_ok = false; }
+    tc_fence_after();
+  }
+  __syncthreads();                                 // the pipeline stages are done with (the pair's MMAs have completed)
+  if (reader) {
+    const int quad = warp & 3;
+    const int r = quad * 32 + lane;
+    for (int c0 = ((warp - 2) >> 2) * 16; c0 < T; c0 += 32) {
+      uint32_t v[16];
+      if (acc_ok) {
+        tc_ld_32x16(tmem + (static_cast<uint32_t>(quad * 32) << 16) + c0, v);
+        tc_wait_ld();
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = 0u;
+      }
+#pragma unroll
+      for (int j = 0; j < 16; ++j) park[(c0 + j) * GT_BN + r] = __uint_as_float(v[j]);
+    }
+  }
+  __syncthreads();
+  cluster.sync();                                  // every slice's accumulator is parked
+  const int per = (T + ns - 1) / ns;               // this CTA reduces tokens [c_lo, c_hi) of its 128 features
+  const int c_lo = split * per, c_hi = min(T, c_lo + per);
+  for (int idx = threadIdx.x; idx < (c_hi - c_lo) * (GT_BN / 4); idx += GT_THREADS) {
+    const int c = c_lo + idx / (GT_BN / 4), r4 = (idx % (GT_BN / 4)) * 4;
+    const int m = m0 + c, n = n0 + r4;
+    if (m >= A.M || n >= A.N) continue;
+    float4 v[4];
+#pragma unroll
+    for (int p = 0; p < 4; ++p)
+      v[p] = p < ns ? *reinterpret_cast<const float4 *>(cluster.map_shared_rank(park, half + 2u * p) + c * GT_BN + r4)
+                    : make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 acc = v[0];
+#pragma unroll
+    for (int p = 1; p < 4; ++p) { acc.x += v[p].x; acc.y += v[p].y; acc.z += v[p].z; acc.w += v[p].w; }
+    epilogue4(A, m, n, acc);
+  }
+  tc_fence_before();
+  cluster.sync();                                  // peers may still be reading this CTA's parked tile / tensor memory in use
+  if (warp == 1) tc2_dealloc(tmem, ncols);
+}
+
 // The kernel may use the whole opt-in shared memory of an SM (227 KB); set once per device.
 static cudaError_t gt_configure() {
   static SmemConfigured configured;
@@ -463,6 +591,39 @@ cudaError_t launch_gemm_pair(const GemmArgs &A, cudaStream_t stream) {
   if (park > pipe) pipe = park;
   const dim3 grid(A.n_tiles, (A.M + T - 1) / T, 1);
   return launch_kc(gemm_pair_kernel, grid, dim3(GT_THREADS), pipe + 1024 + 256, stream, dim3(2, 1, 1), A, st);
+}
+
+cudaError_t launch_gemm_pair_split(const GemmArgs &A, cudaStream_t stream) {
+  const int T = A.block_t;
+  if (T < 32 || T > 256 || (T & 31) || (A.K % GT_BK) || A.nsplit < 2 || A.nsplit > 4 || A.nsplit > A.K / GT_BK || A.wtiles != 1 ||
+      A.n_tiles < 2 || (A.n_tiles & 1) || A.n_base < 0)
+    return cudaErrorInvalidValue;
+  static SmemConfigured configured;
+  if (cudaError_t e = ensure_dyn_smem(gemm_pair_split_kernel, 227 * 1024, configured); e != cudaSuccess) return e;
+  const int st = pair_stages(T);
+  size_t pipe = static_cast<size_t>(st) * (GT_BN * 128 + (T / 2) * 128);
+  const size_t park = static_cast<size_t>(T) * GT_BN * 4;
+  if (park > pipe) pipe = park;
+  const dim3 grid(A.n_tiles, (A.M + T - 1) / T, A.nsplit);
+  return launch_kc(gemm_pair_split_kernel, grid, dim3(GT_THREADS), pipe + 1024 + 256, stream, dim3(2, 1, A.nsplit), A, st);
+}
+cudaError_t gemm_pair_split_max_clusters(int block_t, int nsplit, int *out) {
+  static SmemConfigured configured;
+  if (cudaError_t e = ensure_dyn_smem(gemm_pair_split_kernel, 227 * 1024, configured); e != cudaSuccess) return e;
+  const int st = pair_stages(block_t);
+  size_t pipe = static_cast<size_t>(st) * (GT_BN * 128 + (block_t / 2) * 128);
+  const size_t park = static_cast<size_t>(block_t) * GT_BN * 4;
+  if (park > pipe) pipe = park;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2, 1, nsplit);
+  cfg.blockDim = dim3(GT_THREADS);
+  cfg.dynamicSmemBytes = pipe + 1024 + 256;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = nsplit;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaOccupancyMaxActiveClusters(out, gemm_pair_split_kernel, &cfg);
 }
 
 cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream) {

@@ -121,6 +121,26 @@ int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *w
     }
     if (best > 0 && units2 * best >= tiles128 * A.nsplit) { A.wtiles = 2; A.nsplit = best; }
   }
+  // CTA pairs with K slices: each CTA stages half of the activation box; taken when all clusters of 2 x slices are
+  // resident at once and (unless forced) about as many CTAs run as in the one-CTA form - at 256 rows that is the QKV
+  // projection (24 pair tiles x 2 slices); O and down would run on 80 CTAs instead of 120 and gain nothing
+  if (c->pair_split && A.nsplit > 1 && A.wtiles == 1 && T == 256 && mblocks == 1 && (tiles128 % 2) == 0 && epi != EPI_QKV_ROPE) {
+    const int KB = K / 64;
+    int best = 0;
+    for (int ns = 2; ns <= 4 && ns <= KB; ++ns) {
+      int &cap = c->pair_split_clusters[ns];
+      if (cap < 0) { int v = 0; if (gemm_pair_split_max_clusters(T, ns, &v) != cudaSuccess) { v = 0; (void)cudaGetLastError(); } cap = v; }
+      if (cap >= tiles128 / 2) best = ns;
+    }
+    if (best > 0 && (c->pair_split >= 2 || (tiles128 / 2) * 2 * best >= tiles128 * A.nsplit * 3 / 4)) {
+      A.nsplit = best; A.n_base = 0; A.n_tiles = tiles128;
+      if (std::getenv("GM_DEBUG")) std::fprintf(stderr, "[gm] pair split: N=%d K=%d slices=%d\n", N, K, best);
+      rc = x_map(c, x, x_rows, K, T / 2, &A.x_half_map);
+      if (rc != GM_OK) return rc;
+      GM_LAUNCH(c, GM_KC_GEMM, launch_gemm_pair_split(A, c->stream));
+      return GM_OK;
+    }
+  }
   // very wide projections: two sub-tiles per CTA halve the activation re-reads from L2
   if (A.nsplit == 1 && tiles128 * mblocks >= 2 * c->sm_count) A.wtiles = 2;
   const int units = (tiles128 + A.wtiles - 1) / A.wtiles;          // CTAs along N
@@ -501,6 +521,7 @@ int gm_init(gm_ctx **out, const gm_config *cfg, const gm_weights *w, void *cuda_
   if (std::getenv("GM_NO_EARLY_W")) c->early_weights = false;
   if (const char *ws = std::getenv("GM_GEMM_WIDE_SPLIT")) c->wide_split = std::atoi(ws) != 0;
   if (const char *pb = std::getenv("GM_GEMM_PAIR_BLOCKS")) c->pair_blocks = std::atoi(pb) != 0;
+  if (const char *ps = std::getenv("GM_GEMM_PAIR_SPLIT")) c->pair_split = std::atoi(ps);
   if (std::getenv("GM_FUSED_ROPE")) c->fuse_rope = true;
   if (const char *ov = std::getenv("GM_SAMPLER")) {     // tuning aid: cluster | stream | flow for every sampler launch
     c->sampler_mode = !std::strcmp(ov, "cluster") ? 1 : !std::strcmp(ov, "stream") ? 2 : !std::strcmp(ov, "flow") ? 3 : 0;
