@@ -533,14 +533,14 @@ gemm_pair_split_kernel(const __grid_constant__ GemmArgs A, const int nstages) {
     const int c = c_lo + idx / (GT_BN / 4), r4 = (idx % (GT_BN / 4)) * 4;
     const int m = m0 + c, n = n0 + r4;
     if (m >= A.M || n >= A.N) continue;
-    float4 v[4];
+    float4 v[8];
 #pragma unroll
-    for (int p = 0; p < 4; ++p)
+    for (int p = 0; p < 8; ++p)
       v[p] = p < ns ? *reinterpret_cast<const float4 *>(cluster.map_shared_rank(park, half + 2u * p) + c * GT_BN + r4)
                     : make_float4(0.f, 0.f, 0.f, 0.f);
     float4 acc = v[0];
 #pragma unroll
-    for (int p = 1; p < 4; ++p) { acc.x += v[p].x; acc.y += v[p].y; acc.z += v[p].z; acc.w += v[p].w; }
+    for (int p = 1; p < 8; ++p) { acc.x += v[p].x; acc.y += v[p].y; acc.z += v[p].z; acc.w += v[p].w; }
     epilogue4(A, m, n, acc);
   }
   tc_fence_before();
@@ -595,11 +595,13 @@ cudaError_t launch_gemm_pair(const GemmArgs &A, cudaStream_t stream) {
 
 cudaError_t launch_gemm_pair_split(const GemmArgs &A, cudaStream_t stream) {
   const int T = A.block_t;
-  if (T < 32 || T > 256 || (T & 31) || (A.K % GT_BK) || A.nsplit < 2 || A.nsplit > 4 || A.nsplit > A.K / GT_BK || A.wtiles != 1 ||
+  if (T < 32 || T > 256 || (T & 31) || (A.K % GT_BK) || A.nsplit < 2 || A.nsplit > 8 || A.nsplit > A.K / GT_BK || A.wtiles != 1 ||
       A.n_tiles < 2 || (A.n_tiles & 1) || A.n_base < 0)
     return cudaErrorInvalidValue;
   static SmemConfigured configured;
   if (cudaError_t e = ensure_dyn_smem(gemm_pair_split_kernel, 227 * 1024, configured); e != cudaSuccess) return e;
+  if (A.nsplit > 4)                                  // clusters of more than 8 CTAs are an opt-in
+    if (cudaError_t e = cudaFuncSetAttribute(gemm_pair_split_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1); e != cudaSuccess) return e;
   const int st = pair_stages(T);
   size_t pipe = static_cast<size_t>(st) * (GT_BN * 128 + (T / 2) * 128);
   const size_t park = static_cast<size_t>(T) * GT_BN * 4;
@@ -610,6 +612,8 @@ cudaError_t launch_gemm_pair_split(const GemmArgs &A, cudaStream_t stream) {
 cudaError_t gemm_pair_split_max_clusters(int block_t, int nsplit, int *out) {
   static SmemConfigured configured;
   if (cudaError_t e = ensure_dyn_smem(gemm_pair_split_kernel, 227 * 1024, configured); e != cudaSuccess) return e;
+  if (nsplit > 4)
+    if (cudaError_t e = cudaFuncSetAttribute(gemm_pair_split_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1); e != cudaSuccess) return e;
   const int st = pair_stages(block_t);
   size_t pipe = static_cast<size_t>(st) * (GT_BN * 128 + (block_t / 2) * 128);
   const size_t park = static_cast<size_t>(block_t) * GT_BN * 4;

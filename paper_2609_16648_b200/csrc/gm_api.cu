@@ -127,9 +127,14 @@ int run_gemm(gm_ctx *c, const __nv_bfloat16 *x, int x_rows, const CUtensorMap *w
   if (c->pair_split && A.nsplit > 1 && A.wtiles == 1 && T == 256 && mblocks == 1 && (tiles128 % 2) == 0 && epi != EPI_QKV_ROPE) {
     const int KB = K / 64;
     int best = 0;
-    for (int ns = 2; ns <= 4 && ns <= KB; ++ns) {
+    for (int ns = 2; ns <= (c->pair_split >= 3 ? 8 : 4) && ns <= KB; ++ns) {
       int &cap = c->pair_split_clusters[ns];
-      if (cap < 0) { int v = 0; if (gemm_pair_split_max_clusters(T, ns, &v) != cudaSuccess) { v = 0; (void)cudaGetLastError(); } cap = v; }
+      if (cap < 0) {
+        int v = 0;
+        if (gemm_pair_split_max_clusters(T, ns, &v) != cudaSuccess) { v = 0; (void)cudaGetLastError(); }
+        if (std::getenv("GM_DEBUG")) std::fprintf(stderr, "[gm] resident pair clusters T=%d slices=%d: %d\n", T, ns, v);
+        cap = v;
+      }
       if (cap >= tiles128 / 2) best = ns;
     }
     if (best > 0 && (c->pair_split >= 2 || (tiles128 / 2) * 2 * best >= tiles128 * A.nsplit * 3 / 4)) {

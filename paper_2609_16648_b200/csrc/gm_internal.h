@@ -103,8 +103,8 @@ struct gm_ctx {
   size_t flow_ws_bytes = 0;
   int flow_cap = 0;                         // batch the workspace was sized for
   bool fuse_rope = false;                   // GM_FUSED_ROPE: rotary embedding + KV append in the QKV projection's epilogue (measured slower: off)
-  int pair_split = 1;                        // CTA pairs with K slices for split projections (GM_GEMM_PAIR_SPLIT: 0 off, 1 when no fewer CTAs run, 2 whenever the clusters fit)
-  int pair_split_clusters[5] = {-1, -1, -1, -1, -1};   // resident clusters of 2 x ns CTAs, by ns
+  int pair_split = 1;                        // CTA pairs with K slices for split projections (GM_GEMM_PAIR_SPLIT: 0 off, 1 when no fewer CTAs run, 2 whenever clusters of <= 8 fit, 3 also larger clusters)
+  int pair_split_clusters[9] = {-1, -1, -1, -1, -1, -1, -1, -1, -1};   // resident clusters of 2 x ns CTAs, by ns
   bool pair_blocks = true;                   // CTA pairs for narrow projections over several token blocks (GM_GEMM_PAIR_BLOCKS=0: off)
   bool wide_split = false;                   // split projections with two 128-feature sub-tiles per CTA (GM_GEMM_WIDE_SPLIT=1)
   bool early_weights = true;                // projections fetch their first weight boxes before the dependency wait (GM_NO_EARLY_W switches it off)

@@ -429,7 +429,8 @@ struct GemmArgs {
 cudaError_t launch_gemm_tc(const GemmArgs &A, cudaStream_t stream);
 // CTA-pair form (one K slice per tile, an even number of feature tiles, block_t a multiple of 32).
 cudaError_t launch_gemm_pair(const GemmArgs &A, cudaStream_t stream);
-// CTA pairs with K slices: cluster (2, 1, nsplit), nsplit = 2..4; n_tiles even, one sub-tile per CTA.
+// CTA pairs with K slices: cluster (2, 1, nsplit), nsplit = 2..8 (above 4: clusters of more than 8 CTAs, an opt-in); n_tiles even,
+// one sub-tile per CTA.
 cudaError_t launch_gemm_pair_split(const GemmArgs &A, cudaStream_t stream);
 cudaError_t gemm_pair_split_max_clusters(int block_t, int nsplit, int *out);
 cudaError_t launch_gemm_simple(const GemmArgs &A, cudaStream_t stream);
