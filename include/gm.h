@@ -468,6 +468,8 @@ int gm_head_attn_backward(gm_ctx *ctx, const float *x, const float *dxmid, const
  *   dk_pool, dv_pool  device fp32 [head_num_pages][n_kv][16][head_dim] scratch (zeroed here; on return the gradient of
  *                     every head-cache entry, shared prefix pages and private chain pages alike)
  *   out               device fp32 buffers, overwritten with the sums over all cycles
+ * The result does not depend on thread scheduling: the cache entries' gradients are accumulated in 64-bit fixed point
+ * (units of 2^-40) inside the call and converted into dk_pool / dv_pool at its end; every other sum runs in a fixed order.
  * Uses the context's cycle workspaces (not to be interleaved with a cycle in flight); scratch for the passes and
  * transposed copies of the head's matrices are allocated on first use and kept until gm_free.
  * Limits: those of the four operators (d, q_dim, n_qkv, F multiples of 64; head_dim 64 / 128; group <= 8; no

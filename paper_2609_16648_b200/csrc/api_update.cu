@@ -281,10 +281,14 @@ int gm_head_input_backward(gm_ctx *c, int rows, const int32_t *tokens, const flo
   return head_input_backward_impl(c, rows, tokens, hidden, dz, dhidden, dproj, denorm, dhnorm, refresh_weights, false);
 }
 
-int gm_attention_backward(gm_ctx *c, const void *q, const float *dout, const void *kv_pool, int pool_layers, int num_pages, int layer,
-                          const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch, int q_stride,
-                          float *dq, float *dk_pool, float *dv_pool) {
-  if (!c || !q || !dout || !kv_pool || !page_table || !q_count || !q_base || !dq || !dk_pool || !dv_pool) return GM_ERR_INVALID_ARG;
+// dk_fix / dv_fix / dq_fix given: the gradients are accumulated there in fixed point (order-independent sums) and the float
+// outputs are not touched
+static int attention_backward_impl(gm_ctx *c, const void *q, const float *dout, const void *kv_pool, int pool_layers, int num_pages, int layer,
+                                   const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch, int q_stride,
+                                   float *dq, float *dk_pool, float *dv_pool, long long *dq_fix, long long *dk_fix, long long *dv_fix) {
+  const bool fix = dk_fix != nullptr;
+  if (!c || !q || !dout || !kv_pool || !page_table || !q_count || !q_base) return GM_ERR_INVALID_ARG;
+  if (fix ? (!dq_fix || !dv_fix) : (!dq || !dk_pool || !dv_pool)) return GM_ERR_INVALID_ARG;
   if (batch < 1 || q_stride < 1 || pool_layers < 1 || layer < 0 || layer >= pool_layers || num_pages < 1) return GM_ERR_INVALID_ARG;
   const gm_config &cf = c->cfg;
   if (q_stride > 8 || c->group > 8 || (cf.head_dim != 64 && cf.head_dim != 128)) return GM_ERR_UNSUPPORTED;
@@ -313,9 +317,18 @@ int gm_attention_backward(gm_ctx *c, const void *q, const float *dout, const voi
   A.qrows = round16(q_stride * c->group); A.layer = layer; A.num_pages = num_pages; A.max_pages_per_seq = cf.max_pages_per_seq;
   A.scale = static_cast<float>(1.0 / std::sqrt(static_cast<double>(cf.head_dim)));
   A.stats = c->ab_stats; A.dq = dq; A.dk_pool = dk_pool; A.dv_pool = dv_pool; A.status = c->status;
-  GM_CUDA(c, cudaMemsetAsync(dq, 0, sizeof(float) * static_cast<size_t>(batch) * q_stride * cf.n_q_heads * cf.head_dim, c->stream));
+  A.dq_fix = dq_fix; A.dk_fix = dk_fix; A.dv_fix = dv_fix;
+  const size_t nq = static_cast<size_t>(batch) * q_stride * cf.n_q_heads * cf.head_dim;
+  if (fix) GM_CUDA(c, cudaMemsetAsync(dq_fix, 0, sizeof(long long) * nq, c->stream));
+  else GM_CUDA(c, cudaMemsetAsync(dq, 0, sizeof(float) * nq, c->stream));
   GM_LAUNCH(c, GM_KC_ATTENTION, launch_attention_backward(A, c->stream));
   return GM_OK;
+}
+int gm_attention_backward(gm_ctx *c, const void *q, const float *dout, const void *kv_pool, int pool_layers, int num_pages, int layer,
+                          const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch, int q_stride,
+                          float *dq, float *dk_pool, float *dv_pool) {
+  return attention_backward_impl(c, q, dout, kv_pool, pool_layers, num_pages, layer, page_table, q_count, q_base, batch, q_stride, dq,
+                                 dk_pool, dv_pool, nullptr, nullptr, nullptr);
 }
 
 // The attention half's forward values for one pass of rows x [batch * q_stride, d], with the forward pass's own kernels:
@@ -365,10 +378,12 @@ static int head_attn_forward(gm_ctx *c, const float *x, const void *kv_pool, int
 static int head_attn_backward_impl(gm_ctx *c, const float *x, const float *dxmid, const void *kv_pool, int num_pages,
                                    const int32_t *page_table, const int32_t *q_count, const int32_t *q_base, int batch, int q_stride,
                                    float *dk_pool, float *dv_pool, float *dx, float *dw_qkv, float *dw_o, float *dln1, float *db_qkv,
-                                   float *dqk_norm, int refresh_weights, bool accum, bool forward_done = false) {
+                                   float *dqk_norm, int refresh_weights, bool accum, bool forward_done = false,
+                                   long long *dk_fix = nullptr, long long *dv_fix = nullptr) {
   const int wepi = accum ? EPI_ADD_F32 : EPI_STORE_F32;
-  if (!c || !x || !kv_pool || !page_table || !q_count || !q_base || !dk_pool || !dv_pool || !dx || !dw_qkv || !dw_o ||
-      !dln1 || batch < 1 || q_stride < 1 || num_pages < 1)
+  const bool fix = dk_fix != nullptr;                  // key / value gradients in the fixed-point planes instead of dk_pool / dv_pool
+  if (!c || !x || !kv_pool || !page_table || !q_count || !q_base || !dx || !dw_qkv || !dw_o || !dln1 || batch < 1 || q_stride < 1 ||
+      num_pages < 1 || (fix ? !dv_fix : (!dk_pool || !dv_pool)))
     return GM_ERR_INVALID_ARG;
   const gm_config &cf = c->cfg;
   const gm_layer_weights &lw = c->w.head_layer;
@@ -409,6 +424,10 @@ static int head_attn_backward_impl(gm_ctx *c, const float *x, const float *dxmid
     if ((rc = dev_alloc(c, &c->hat_tk, M * (NQKV - NQ) / 2)) != GM_OK) return rc;
     c->hat_rows_cap = Mp;
   }
+  if (fix && static_cast<size_t>(Mp) * NQ > c->hat_dq_fix_cap) {
+    if ((rc = dev_alloc(c, &c->hat_dq_fix, static_cast<size_t>(Mp) * NQ)) != GM_OK) return rc;
+    c->hat_dq_fix_cap = static_cast<size_t>(Mp) * NQ;
+  }
   // ---- the forward's values, recomputed: h = RMSNorm(x; ln1), the projection, the rotated queries, the attention output ----
   if (!forward_done &&
       (rc = head_attn_forward(c, x, kv_pool, num_pages, page_table, q_count, q_base, batch, q_stride, dxmid != nullptr)) != GM_OK)
@@ -420,15 +439,18 @@ static int head_attn_backward_impl(gm_ctx *c, const float *x, const float *dxmid
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_cast_bf16(dxmid, c->hat_dy, static_cast<size_t>(rows) * d, c->stream));
   if ((rc = run_gemm(c, c->hat_dy, rows, &c->hat_wo_t_map, c->hat_wo_t, rows, NQ, d, c->hat_do, EPI_STORE_F32, static_cast<size_t>(NQ), false)) != GM_OK)
     return rc;
-  if ((rc = gm_attention_backward(c, c->qbuf, c->hat_do, kv_pool, 1, num_pages, 0, page_table, c->qn, c->qbase, batch, q_stride,
-                                  c->hat_dq, dk_pool, dv_pool)) != GM_OK)
+  if ((rc = attention_backward_impl(c, c->qbuf, c->hat_do, kv_pool, 1, num_pages, 0, page_table, c->qn, c->qbase, batch, q_stride,
+                                    c->hat_dq, dk_pool, dv_pool, fix ? c->hat_dq_fix : nullptr, dk_fix, dv_fix)) != GM_OK)
     return rc;
+  } else if (fix) {
+    GM_CUDA(c, cudaMemsetAsync(c->hat_dq_fix, 0, sizeof(long long) * static_cast<size_t>(rows) * NQ, c->stream));
   } else {
     GM_CUDA(c, cudaMemsetAsync(c->hat_dq, 0, sizeof(float) * static_cast<size_t>(rows) * NQ, c->stream));
   }
   // ---- the rows' own entries are complete now: back through the rotation and the head norms, packed like the projection ----
   QkvGradArgs Q;
   Q.qkv = c->qkv; Q.bias = bias; Q.qnorm = qnorm; Q.knorm = knorm; Q.dq = c->hat_dq; Q.dk_pool = dk_pool; Q.dv_pool = dv_pool;
+  if (fix) { Q.dq_fix = c->hat_dq_fix; Q.dk_fix = dk_fix; Q.dv_fix = dv_fix; }
   Q.qn = c->qn; Q.qbase = c->qbase; Q.page_table = page_table; Q.rope = c->rope; Q.batch = batch; Q.QT = q_stride;
   Q.n_q = cf.n_q_heads; Q.n_kv = cf.n_kv_heads; Q.hd = hd; Q.num_pages = num_pages; Q.max_pages_per_seq = cf.max_pages_per_seq;
   Q.eps = cf.rms_eps; Q.dqkv = c->hat_dqkv; Q.dqkv_bf = c->hat_dqkv_bf; Q.status = c->status;
@@ -515,11 +537,17 @@ int gm_head_update_backward(gm_ctx *c, gm_state *st, int n_cycles, int k, const 
       if ((rc = dev_alloc(c, p, static_cast<size_t>(cap))) != GM_OK) return rc;
     c->hub_rows_cap = cap;
   }
-  // every output starts at zero; the passes add to them
+  // every output starts at zero; the passes add to them.  The cache entries' gradients are accumulated in fixed point
+  // (64-bit integer additions), so that the update does not depend on the order in which the chains' CTAs arrive.
   const size_t NQKV = c->n_qkv, NQ = c->q_dim;
   const size_t plane = static_cast<size_t>(cf.head_num_pages) * cf.n_kv_heads * GM_PAGE * hd;
-  GM_CUDA(c, cudaMemsetAsync(dk_pool, 0, sizeof(float) * plane, c->stream));
-  GM_CUDA(c, cudaMemsetAsync(dv_pool, 0, sizeof(float) * plane, c->stream));
+  if (plane > c->hub_fix_cap) {
+    if ((rc = dev_alloc(c, &c->hub_dk_fix, plane, false)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->hub_dv_fix, plane, false)) != GM_OK) return rc;
+    c->hub_fix_cap = plane;
+  }
+  GM_CUDA(c, cudaMemsetAsync(c->hub_dk_fix, 0, sizeof(long long) * plane, c->stream));
+  GM_CUDA(c, cudaMemsetAsync(c->hub_dv_fix, 0, sizeof(long long) * plane, c->stream));
   struct { float *p; size_t n; } outs[] = {{out->proj, static_cast<size_t>(2) * d * d}, {out->enorm, static_cast<size_t>(d)},
       {out->hnorm, static_cast<size_t>(d)}, {out->final_norm, static_cast<size_t>(d)}, {out->ln1, static_cast<size_t>(d)},
       {out->ln2, static_cast<size_t>(d)}, {out->wqkv, NQKV * d}, {out->wo, NQ * d}, {out->w_gate_up, static_cast<size_t>(2) * F * d},
@@ -575,8 +603,8 @@ int gm_head_update_backward(gm_ctx *c, gm_state *st, int n_cycles, int k, const 
       if ((rc = head_ffn_backward_impl(c, m, c->hub_xmid, c->hub_dg, c->hub_dxmid, out->w_gate_up, out->w_down, out->ln2, refresh, true)) != GM_OK)
         return rc;
       if ((rc = head_attn_backward_impl(c, c->hub_z, c->hub_dxmid, st->head_kv_pool, cf.head_num_pages, c->v_table, c->hub_cnt, c->hub_base,
-                                        m, 1, dk_pool, dv_pool, c->hub_dz, out->wqkv, out->wo, out->ln1, out->b_qkv, out->qk_norm, refresh,
-                                        true, true)) != GM_OK)
+                                        m, 1, nullptr, nullptr, c->hub_dz, out->wqkv, out->wo, out->ln1, out->b_qkv, out->qk_norm, refresh,
+                                        true, true, c->hub_dk_fix, c->hub_dv_fix)) != GM_OK)
         return rc;
       if ((rc = head_input_backward_impl(c, m, c->hub_tok, c->hub_hidden, c->hub_dz, c->hub_dhid, out->proj, out->enorm, out->hnorm, refresh,
                                          true)) != GM_OK)
@@ -590,7 +618,7 @@ int gm_head_update_backward(gm_ctx *c, gm_state *st, int n_cycles, int k, const 
   FoldArgs Fo;
   Fo.cycle_seq = cycle_seq; Fo.start_pos = rec->start_pos; Fo.scratch_pages = scratch_pages; Fo.head_page_table = st->head_page_table;
   Fo.n_seq = st->batch; Fo.max_pages_per_seq = cf.max_pages_per_seq; Fo.num_pages = cf.head_num_pages; Fo.n_kv = cf.n_kv_heads; Fo.hd = hd;
-  Fo.dk_pool = dk_pool; Fo.dv_pool = dv_pool;
+  Fo.dk_pool = nullptr; Fo.dv_pool = nullptr; Fo.dk_fix = c->hub_dk_fix; Fo.dv_fix = c->hub_dv_fix;
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_fold_boundary(Fo, n_cycles, c->stream));
   // ---- the pass over the committed prefixes: nothing consumed these rows' outputs, only their cache entries ----
   GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_dup_table_rows(st->head_page_table, B, VR, cf.max_pages_per_seq, c->pf_vtable[1], c->stream));
@@ -606,13 +634,16 @@ int gm_head_update_backward(gm_ctx *c, gm_state *st, int n_cycles, int k, const 
     GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_rows_to_f32(c->pf_hidden, c->pf_head_n, R * QT, QT, d, c->hub_hidden, c->stream));
     if ((rc = head_z_forward(c, R * QT, c->pf_pair_tok, c->hub_hidden, c->hub_z)) != GM_OK) return rc;
     if ((rc = head_attn_backward_impl(c, c->hub_z, nullptr, st->head_kv_pool, cf.head_num_pages, c->pf_vtable[1], c->pf_head_n,
-                                      c->pf_row_base, R, QT, dk_pool, dv_pool, c->hub_dz, out->wqkv, out->wo, out->ln1, out->b_qkv,
-                                      out->qk_norm, 0, true)) != GM_OK)
+                                      c->pf_row_base, R, QT, nullptr, nullptr, c->hub_dz, out->wqkv, out->wo, out->ln1, out->b_qkv,
+                                      out->qk_norm, 0, true, false, c->hub_dk_fix, c->hub_dv_fix)) != GM_OK)
       return rc;
     if ((rc = head_input_backward_impl(c, R * QT, c->pf_pair_tok, c->hub_hidden, c->hub_dz, nullptr, out->proj, out->enorm, out->hnorm, 0,
                                        true)) != GM_OK)
       return rc;
   }
+  // the cache entries' gradients, for the caller
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_fix_to_float(c->hub_dk_fix, dk_pool, plane, c->stream));
+  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_fix_to_float(c->hub_dv_fix, dv_pool, plane, c->stream));
   return GM_OK;
 }
 

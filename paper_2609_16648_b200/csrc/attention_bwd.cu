@@ -155,7 +155,8 @@ __global__ void __launch_bounds__(AB_MAX_GROUP * 32) attn_bwd_grad_kernel(const 
       const int which = i / HD, c = i % HD;
       float acc = 0.f;
       for (int gg = 0; gg < G; ++gg) acc += red[(which * G + gg) * HD + c];
-      if (acc != 0.f) atomicAdd((which ? A.dv_pool : A.dk_pool) + off + c, acc);
+      if (A.dk_fix) fix_add((which ? A.dv_fix : A.dk_fix) + off + c, acc);
+      else if (acc != 0.f) atomicAdd((which ? A.dv_pool : A.dk_pool) + off + c, acc);
     }
     __syncthreads();
   }
@@ -165,7 +166,11 @@ __global__ void __launch_bounds__(AB_MAX_GROUP * 32) attn_bwd_grad_kernel(const 
       if (j < qn) {
         const int m = b * A.QT + j;
 #pragma unroll
-        for (int e = 0; e < E; ++e) A.dq[(static_cast<size_t>(m) * A.n_kv * A.group + h) * HD + lane * E + e] = dq[j][e];
+        for (int e = 0; e < E; ++e) {
+          const size_t o = (static_cast<size_t>(m) * A.n_kv * A.group + h) * HD + lane * E + e;
+          if (A.dq_fix) fix_add(A.dq_fix + o, dq[j][e]);
+          else A.dq[o] = dq[j][e];
+        }
       }
   }
 }
@@ -318,20 +323,31 @@ __global__ void __launch_bounds__(AB_WARPS * 32) attn_bwd_grad_split_kernel(cons
     }
 #pragma unroll
     for (int e = 0; e < E; ++e) {                          // every visible pair's term of this key, from this warp alone
-      atomicAdd(A.dk_pool + off + lane * E + e, dk[e]);
-      atomicAdd(A.dv_pool + off + lane * E + e, dv[e]);
+      if (A.dk_fix) {
+        fix_add(A.dk_fix + off + lane * E + e, dk[e]);
+        fix_add(A.dv_fix + off + lane * E + e, dv[e]);
+      } else {
+        atomicAdd(A.dk_pool + off + lane * E + e, dk[e]);
+        atomicAdd(A.dv_pool + off + lane * E + e, dv[e]);
+      }
     }
   }
+  for (int w = 0; w < AB_WARPS; ++w) {                 // the warps' partial dq, added in warp order
+    if (wp == w) {
 #pragma unroll
-  for (int i = 0; i < NP; ++i)
-    if (i < np) {
+      for (int i = 0; i < NP; ++i)
+        if (i < np) {
 #pragma unroll
-      for (int e = 0; e < E; ++e) atomicAdd(&sdq[i][lane * E + e], dq[i][e]);
+          for (int e = 0; e < E; ++e) sdq[i][lane * E + e] += dq[i][e];
+        }
     }
-  __syncthreads();
+    __syncthreads();
+  }
   for (int t = threadIdx.x; t < np * HD; t += blockDim.x) {
     const int i = t / HD, c = t % HD, j = i / G, g = i % G, m = b * A.QT + j, h = kvh * G + g;
-    atomicAdd(A.dq + (static_cast<size_t>(m) * A.n_kv * G + h) * HD + c, sdq[i][c]);
+    const size_t o = (static_cast<size_t>(m) * A.n_kv * G + h) * HD + c;
+    if (A.dq_fix) fix_add(A.dq_fix + o, sdq[i][c]);
+    else atomicAdd(A.dq + o, sdq[i][c]);
   }
 }
 

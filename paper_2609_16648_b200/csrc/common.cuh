@@ -30,6 +30,12 @@ __device__ __forceinline__ void pdl_prologue() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// ---- order-independent accumulation: 64-bit fixed point (2^-40) --------------------------------------------
+__device__ __forceinline__ void fix_add(long long *p, float x) {
+  if (x != 0.f) atomicAdd(reinterpret_cast<unsigned long long *>(p), static_cast<unsigned long long>(__float2ll_rn(x * 1099511627776.0f)));
+}
+__device__ __forceinline__ float fix_get(const long long *p) { return static_cast<float>(static_cast<double>(*p) * (1.0 / 1099511627776.0)); }
+
 // ---- small math -----------------------------------------------------------------------------------
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }

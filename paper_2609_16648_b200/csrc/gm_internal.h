@@ -134,6 +134,8 @@ struct gm_ctx {
   __nv_bfloat16 *hu_logits = nullptr, *hu_glogits = nullptr;
   float *hu_alpha = nullptr, *hu_lse = nullptr, *hu_loss = nullptr;
   int hu_cycles_cap = 0, hu_step = 0;
+  long long *hub_dk_fix = nullptr, *hub_dv_fix = nullptr, *hat_dq_fix = nullptr;   // fixed-point gradient accumulators of the driver
+  size_t hub_fix_cap = 0, hat_dq_fix_cap = 0;
   float *colsum_ws = nullptr;               // partial column sums (64 chunks x the widest row: n_qkv or 2 d)
   // backward pass over a reconstruction: per-chunk states and their gradients, one pass's rows
   int hub_rows_cap = 0;

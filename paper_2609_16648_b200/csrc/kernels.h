@@ -285,8 +285,12 @@ struct FoldArgs {
   const int32_t *cycle_seq, *start_pos, *scratch_pages, *head_page_table;
   int n_seq, max_pages_per_seq, num_pages, n_kv, hd;
   float *dk_pool, *dv_pool;
+  long long *dk_fix = nullptr, *dv_fix = nullptr;       // fixed-point planes replacing the two above
 };
 cudaError_t launch_fold_boundary(const FoldArgs &A, int chains, cudaStream_t stream);
+// Fixed point of the gradient accumulators: value * 2^40 rounded to a 64-bit integer.
+constexpr float GM_FIX_SCALE = 1099511627776.0f, GM_FIX_INV = 1.0f / 1099511627776.0f;
+cudaError_t launch_fix_to_float(const long long *src, float *dst, size_t n, cudaStream_t stream);
 cudaError_t launch_widen_bf16(const __nv_bfloat16 *src, float *dst, size_t n, cudaStream_t stream);          // dst[i] = src[i]
 cudaError_t launch_rows_to_f32(const __nv_bfloat16 *src, const int32_t *row_n, int rows, int QT, int d, float *dst, cudaStream_t stream);
 // AdamW on n fp32 master parameters with fp32 moments; param (bf16 copy the forward pass reads) or null.  decay = 1 - lr wd,
@@ -303,6 +307,7 @@ struct QkvGradArgs {
   const __nv_bfloat16 *bias = nullptr, *qnorm = nullptr, *knorm = nullptr;
   const float *dq;                                      // [M][n_q][hd] gradient of the rotated queries
   const float *dk_pool, *dv_pool;                       // [num_pages][n_kv][16][hd] gradient planes of the cache
+  const long long *dk_fix = nullptr, *dv_fix = nullptr, *dq_fix = nullptr;   // fixed-point sources (2^-40) replacing the three above
   const int32_t *qn, *qbase, *page_table;
   const float2 *rope;
   int batch, QT, n_q, n_kv, hd, num_pages, max_pages_per_seq;
@@ -381,6 +386,9 @@ struct AttnBwdArgs {
   float scale;                          // 1 / sqrt(hd)
   float *stats, *dq;                    // dq [B * QT][n_q * hd], zero on entry (the key-split kernels add into it)
   float *dk_pool, *dv_pool;             // [num_pages][n_kv][16][hd], accumulated
+  // Fixed-point accumulators (units of 2^-40, 64-bit integer additions: the sums do not depend on the order in which CTAs
+  // arrive).  Given, they replace dk_pool / dv_pool / dq, which are then not touched.
+  long long *dk_fix = nullptr, *dv_fix = nullptr, *dq_fix = nullptr;
   float *part = nullptr;                // [B][n_kv][nseg][pairs][3] partial softmax statistics per key segment, or null
   int nseg = 0;                         // segments the scratch holds per (sequence, KV head)
   uint32_t *status;

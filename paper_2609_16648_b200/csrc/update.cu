@@ -392,10 +392,21 @@ __global__ void __launch_bounds__(128) fold_boundary_kernel(const FoldArgs A) {
   for (int i = threadIdx.x; i < A.n_kv * slots * A.hd; i += blockDim.x) {
     const int h = i / (slots * A.hd), r = i % (slots * A.hd);
     const size_t o = (static_cast<size_t>(orig) * A.n_kv + h) * per_head + r, s = (static_cast<size_t>(p0) * A.n_kv + h) * per_head + r;
+    if (A.dk_fix) {                                     // integer additions: the same sum in any order
+      const long long a = A.dk_fix[s], b = A.dv_fix[s];
+      if (a) atomicAdd(reinterpret_cast<unsigned long long *>(A.dk_fix + o), static_cast<unsigned long long>(a));
+      if (b) atomicAdd(reinterpret_cast<unsigned long long *>(A.dv_fix + o), static_cast<unsigned long long>(b));
+      continue;
+    }
     const float a = A.dk_pool[s], b = A.dv_pool[s];
     if (a != 0.f) atomicAdd(A.dk_pool + o, a);
     if (b != 0.f) atomicAdd(A.dv_pool + o, b);
   }
+}
+__global__ void __launch_bounds__(256) fix_to_float_kernel(const long long *src, float *dst, size_t n) {
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  pdl_prologue();
+  for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += stride) dst[i] = fix_get(src + i);
 }
 __global__ void __launch_bounds__(256) widen_bf16_kernel(const __nv_bfloat16 *src, float *dst, size_t n) {
   const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
@@ -470,11 +481,17 @@ __global__ void __launch_bounds__(256) qkv_grad_rows_kernel(const QkvGradArgs A)
       }
       continue;
     }
-    const float *src = is_q ? A.dq + (static_cast<size_t>(m) * A.n_q + h) * HD
-                            : (is_k ? A.dk_pool : A.dv_pool) + static_cast<size_t>(page) * page_elems +
-                                  (static_cast<size_t>(kvh) * 16 + (pos & 15)) * HD;
+    const size_t so = is_q ? (static_cast<size_t>(m) * A.n_q + h) * HD
+                           : static_cast<size_t>(page) * page_elems + (static_cast<size_t>(kvh) * 16 + (pos & 15)) * HD;
+    if (A.dk_fix) {
+      const long long *src = (is_q ? A.dq_fix : (is_k ? A.dk_fix : A.dv_fix)) + so;
 #pragma unroll
-    for (int t = 0; t < EH; ++t) { g1[t] = src[lane * EH + t]; g2[t] = src[HALF + lane * EH + t]; }
+      for (int t = 0; t < EH; ++t) { g1[t] = fix_get(src + lane * EH + t); g2[t] = fix_get(src + HALF + lane * EH + t); }
+    } else {
+      const float *src = (is_q ? A.dq : (is_k ? A.dk_pool : A.dv_pool)) + so;
+#pragma unroll
+      for (int t = 0; t < EH; ++t) { g1[t] = src[lane * EH + t]; g2[t] = src[HALF + lane * EH + t]; }
+    }
     if (is_q || is_k) {
       // the rotation's transpose: turn back by the position's angle
       const float2 *cs = A.rope + static_cast<size_t>(pos) * HALF;
@@ -673,6 +690,10 @@ cudaError_t launch_add_state_grad(float *dstate, const float *dhidden, int chain
 }
 cudaError_t launch_fold_boundary(const FoldArgs &A, int chains, cudaStream_t stream) {
   return launch_k(fold_boundary_kernel, dim3(chains), dim3(128), 0, stream, 1, A);
+}
+cudaError_t launch_fix_to_float(const long long *src, float *dst, size_t n, cudaStream_t stream) {
+  const size_t blocks = std::min<size_t>((n + 255) / 256, 148 * 8);
+  return launch_k(fix_to_float_kernel, dim3(static_cast<unsigned>(std::max<size_t>(blocks, 1))), dim3(256), 0, stream, 1, src, dst, n);
 }
 cudaError_t launch_widen_bf16(const __nv_bfloat16 *src, float *dst, size_t n, cudaStream_t stream) {
   const size_t blocks = std::min<size_t>((n + 255) / 256, 148 * 8);
