@@ -17,8 +17,9 @@ def test_rollout_record_update_rounds_raise_the_acceptance():
     """Four rounds of (rollout of 12 cycles on 16 sequences with records, 20 updates on those 192 cycles).  The head starts
     at random initialisation, independent of the target, so few drafts are accepted; every round's updates lower the
     objective (mean of Eq. 9) on its own records, and the accepted drafts per cycle of the NEXT rollout - same prompts, new
-    random draws, the updated head - rise well above the first round's.  On other prompts the gain is smaller (a
-    192-cycle training set on a toy model) and is only required not to fall.  Everything goes through the C ABI: prefill,
+    random draws, the updated head - rise well above the first round's.  On other prompts the gain is small (a
+    192-cycle training set on a toy model; measured 0.30 -> 0.38 / 0.45 / 0.43 on the default kernels) and within the
+    sampling noise of 192 cycles under other kernel choices, so it is printed and only loosely bounded.  Everything goes through the C ABI: prefill,
     draft / verify / accept with gm_record_begin / gm_record_end and gm_capture_hidden, then gm_head_update_step."""
     import paper_2609_16648_b200 as gmb
     B, n_steps, K, epochs, peak = 16, 12, 3, 20, 1e-3
@@ -95,5 +96,5 @@ def test_rollout_record_update_rounds_raise_the_acceptance():
         print(f"round {rnd}: accepted drafts per cycle {tau:.3f} (training prompts) {tau_other:.3f} (other prompts); "
               f"objective over the round's updates {losses[0]:.3f} -> {losses[-1]:.3f}")
     assert trained[-1] > trained[0] + 0.2 and min(trained[1:]) > trained[0] + 0.1       # measured 0.35 -> 0.70 / 0.80 / 0.87
-    assert np.mean(other[1:]) >= other[0] - 0.02
+    assert np.mean(other[1:]) >= other[0] - 0.1          # 192 cycles: a standard error of about 0.05 per figure
     ctx.close()
