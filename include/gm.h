@@ -388,7 +388,7 @@ int gm_dca_grad(gm_ctx *ctx, int n_cycles, int k, float temperature, const void 
  *                This is the derivative through the logits of the state's own position; the terms that reach
  *                g_j through g_{j+1} (Eq. 4) belong to the backward pass of the head layer, which is not built.
  * The projection reads a transposed copy [d, V] of the LM head that the context makes on the first call (d * V
- * bf16 of device memory, kept until gm_free); refresh_weights != 0 remakes it, for a caller that has rewritten the
+ * bf16 of device memory, kept until gm_destroy); refresh_weights != 0 remakes it, for a caller that has rewritten the
  * LM head's weights in place since.  V % 64 != 0 returns GM_ERR_UNSUPPORTED.                                   */
 int gm_head_state_grad(gm_ctx *ctx, int rows, const void *grad_logits, const float *head_states,
                        float *grad_normed, float *grad_states, int refresh_weights);
@@ -404,7 +404,7 @@ int gm_head_state_grad(gm_ctx *ctx, int rows, const void *grad_logits, const flo
  * computes them; products run on the projection kernel (fp32 accumulation, bf16 operands: dg, the activation
  * gradients and the recomputed activations are rounded to bf16 before they enter a product).  Transposed copies of the
  * two weight matrices (3 d F bf16) and scratch for `rows` rounded up to 64 are allocated on first use and kept until
- * gm_free; refresh_weights != 0 remakes the copies after the weights have been rewritten in place.
+ * gm_destroy; refresh_weights != 0 remakes the copies after the weights have been rewritten in place.
  * d % 64 != 0, F % 64 != 0 or GM_FLAG_SIMPLE_GEMM: GM_ERR_UNSUPPORTED.                                         */
 int gm_head_ffn_backward(gm_ctx *ctx, int rows, const float *x, const float *dg, float *dx, float *dw_gate_up,
                          float *dw_down, float *dln2, int refresh_weights);
@@ -444,7 +444,7 @@ int gm_attention_backward(gm_ctx *ctx, const void *q, const float *dout, const v
  * rows, the projection, the rotated queries, the attention output) are recomputed in bf16 as the forward pass computes
  * them, in the context's own workspaces - not to be interleaved with a cycle in flight on the same context; products run
  * on the projection kernel with bf16 operands and fp32 accumulation.  Transposed copies of W_o and W_qkv and scratch for
- * the rows rounded up to 64 are allocated on first use and kept until gm_free; refresh_weights != 0 remakes the copies.
+ * the rows rounded up to 64 are allocated on first use and kept until gm_destroy; refresh_weights != 0 remakes the copies.
  * GM_ERR_UNSUPPORTED: GM_FLAG_SIMPLE_GEMM, d, n_q head_dim or (n_q + 2 n_kv) head_dim not a multiple of 64, head_dim
  * other than 64 / 128, more than 8 query heads per KV head, q_stride > min(8, max_k + 1), or more rows than a prefill
  * pass of the context holds.  A page outside the pool: the status word reports GM_ERR_BAD_PAGE and the row gets zeros. */
@@ -471,7 +471,7 @@ int gm_head_attn_backward(gm_ctx *ctx, const float *x, const float *dxmid, const
  * The result does not depend on thread scheduling: the cache entries' gradients are accumulated in 64-bit fixed point
  * (units of 2^-40) inside the call and converted into dk_pool / dv_pool at its end; every other sum runs in a fixed order.
  * Uses the context's cycle workspaces (not to be interleaved with a cycle in flight); scratch for the passes and
- * transposed copies of the head's matrices are allocated on first use and kept until gm_free.
+ * transposed copies of the head's matrices are allocated on first use and kept until gm_destroy.
  * Limits: those of the four operators (d, q_dim, n_qkv, F multiples of 64; head_dim 64 / 128; group <= 8; no
  * GM_FLAG_SIMPLE_GEMM): GM_ERR_UNSUPPORTED.  An optional output (b_qkv, qk_norm) must be given iff the layer has it.   */
 typedef struct {
@@ -500,7 +500,7 @@ int gm_head_update_backward(gm_ctx *ctx, gm_state *st, int n_cycles, int k, cons
  * The bf16 tensors the context was created with (head_proj, head_enorm, head_hnorm, head_final_norm and every tensor of
  * head_layer) are REWRITTEN IN PLACE; the backbone's tensors are read only.  fp32 master copies (initialised from the bf16
  * values at the first call), both moments, the gradients and the per-call buffers belong to the context and live until
- * gm_free (about 16 bytes per head parameter + 4 bytes x 2 x n_cycles x k x vocab).  The head cache of `st` is left as the
+ * gm_destroy (about 16 bytes per head parameter + 4 bytes x 2 x n_cycles x k x vocab).  The head cache of `st` is left as the
  * rebuild with the parameters BEFORE the update wrote it.                                                               */
 int gm_head_update_step(gm_ctx *ctx, gm_state *st, int n_cycles, int k, float temperature, const int32_t *cycle_seq,
                         const gm_record *rec, const int32_t *seq_tok, int tok_stride, const int32_t *scratch_pages,
