@@ -465,8 +465,8 @@ int gm_head_attn_backward(gm_ctx *ctx, const float *x, const float *dxmid, const
  * whose rows receive gradient only through their cache entries.
  *   grad_logits       device bf16 [n_cycles, k, vocab] (gm_dca_grad)
  *   seq_hidden, hid_stride, seq_len, max_len, seq_tok, tok_stride   as in gm_head_prefill / gm_reconstruct
- *   dk_pool, dv_pool  device fp32 [head_num_pages][n_kv][16][head_dim] scratch (zeroed here; on return the gradient of
- *                     every head-cache entry, shared prefix pages and private chain pages alike)
+ *   dk_pool, dv_pool  device fp32 [head_num_pages][n_kv][16][head_dim] out, or both NULL: the gradient of every head-cache
+ *                     entry, shared prefix pages and private chain pages alike (a by-product; the update does not need it)
  *   out               device fp32 buffers, overwritten with the sums over all cycles
  * The result does not depend on thread scheduling: the cache entries' gradients are accumulated in 64-bit fixed point
  * (units of 2^-40) inside the call and converted into dk_pool / dv_pool at its end; every other sum runs in a fixed order.

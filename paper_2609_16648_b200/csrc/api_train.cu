@@ -61,9 +61,6 @@ int gm_head_update_step(gm_ctx *c, gm_state *st, int n_cycles, int k, float temp
     if ((rc = dev_alloc(c, &g.w_down, F * d)) != GM_OK) return rc;
     if (c->w.head_layer.b_qkv && (rc = dev_alloc(c, &g.b_qkv, NQKV)) != GM_OK) return rc;
     if (c->w.head_layer.q_norm && (rc = dev_alloc(c, &g.qk_norm, 2 * hd)) != GM_OK) return rc;
-    const size_t plane = static_cast<size_t>(cf.head_num_pages) * cf.n_kv_heads * GM_PAGE * hd;
-    if ((rc = dev_alloc(c, &c->hu_dk, plane)) != GM_OK) return rc;
-    if ((rc = dev_alloc(c, &c->hu_dv, plane)) != GM_OK) return rc;
     ParamRef ps[13];
     const int np = collect_params(c, g, ps);
     size_t total = 0;
@@ -97,7 +94,7 @@ int gm_head_update_step(gm_ctx *c, gm_state *st, int n_cycles, int k, float temp
   if ((rc = gm_dca_grad(c, n_cycles, k, temperature, c->hu_logits, rec, c->hu_alpha, c->hu_lse, rec->accepted, c->hu_glogits)) != GM_OK)
     return rc;
   if ((rc = gm_head_update_backward(c, st, n_cycles, k, cycle_seq, rec, seq_tok, tok_stride, scratch_pages, c->hu_glogits, seq_hidden,
-                                    hid_stride, seq_len, max_len, c->hu_dk, c->hu_dv, &c->hu_grads)) != GM_OK)
+                                    hid_stride, seq_len, max_len, nullptr, nullptr, &c->hu_grads)) != GM_OK)
     return rc;
   // ---- AdamW on every tensor of the group; the bf16 copies the forward pass reads are rewritten in place ----
   ParamRef ps[13];

@@ -512,7 +512,7 @@ int gm_head_update_backward(gm_ctx *c, gm_state *st, int n_cycles, int k, const 
   if (rc) return rc;
   if (n_cycles < 1 || !cycle_seq || !rec || !rec->start_hidden || !rec->start_pos || !rec->drafts || !seq_tok || tok_stride < 2 ||
       !scratch_pages || !grad_logits || !seq_hidden || !seq_len || max_len < 2 || tok_stride < max_len || hid_stride < max_len - 1 ||
-      !dk_pool || !dv_pool || !out)
+      (dk_pool != nullptr) != (dv_pool != nullptr) || !out)
     return GM_ERR_INVALID_ARG;
   const gm_config &cf = c->cfg;
   const gm_layer_weights &lw = c->w.head_layer;
@@ -641,9 +641,10 @@ int gm_head_update_backward(gm_ctx *c, gm_state *st, int n_cycles, int k, const 
                                        true)) != GM_OK)
       return rc;
   }
-  // the cache entries' gradients, for the caller
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_fix_to_float(c->hub_dk_fix, dk_pool, plane, c->stream));
-  GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_fix_to_float(c->hub_dv_fix, dv_pool, plane, c->stream));
+  if (dk_pool) {                                       // the cache entries' gradients, for a caller that wants them
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_fix_to_float(c->hub_dk_fix, dk_pool, plane, c->stream));
+    GM_LAUNCH(c, GM_KC_ELEMENTWISE, launch_fix_to_float(c->hub_dv_fix, dv_pool, plane, c->stream));
+  }
   return GM_OK;
 }
 

@@ -130,7 +130,7 @@ struct gm_ctx {
   // one update of the head (gm_head_update_step): gradients, optimizer state (fp32 master, first and second moments, the
   // tensors one after the other, each padded to 4 elements), per-call buffers
   gm_head_grads hu_grads = {};
-  float *hu_dk = nullptr, *hu_dv = nullptr, *hu_master = nullptr, *hu_m = nullptr, *hu_v = nullptr;
+  float *hu_master = nullptr, *hu_m = nullptr, *hu_v = nullptr;
   __nv_bfloat16 *hu_logits = nullptr, *hu_glogits = nullptr;
   float *hu_alpha = nullptr, *hu_lse = nullptr, *hu_loss = nullptr;
   int hu_cycles_cap = 0, hu_step = 0;
