@@ -962,9 +962,9 @@ def run_head_update(args):
         zf, qf, of, ff, lf = 2.0 * 2 * d * d, 2.0 * nqkv * d, 2.0 * q * d, 2.0 * F * d, 2.0 * V * d
         # prefix rows: z and QKV in the rebuild and again in the backward pass, then dh, dW_qkv, d zin, dW_p
         flops = P * (2 * (zf + qf) + 2 * qf + 2 * zf)
-        # chain rows: two replays (z, layer, LM head), LM-head gradient, feed-forward backward (recomputed gate/up + four
+        # chain rows: one replay (z, layer, LM head; the call-by-call sequence makes two), LM-head gradient, feed-forward backward (recomputed gate/up + four
         # products), attention half (z, QKV, W_o forward; d out, dh, two weight gradients), input (d zin, dW_p)
-        flops += C * (2 * (zf + qf + of + 3 * ff + lf) + lf + (2 * ff + ff + 2 * ff + ff + 2 * ff) + (zf + qf + of + of + qf + of + qf) + 2 * zf)
+        flops += C * ((zf + qf + of + 3 * ff + lf) + lf + (2 * ff + ff + 2 * ff + ff + 2 * ff) + (zf + qf + of + of + qf + of + qf) + 2 * zf)
         tf = flops / (gemm_ms * 1e-3) / 1e12
         line = {"metric": "head_update_cycles_per_s", "value": n * S * world / (ms_max * 1e-3), "unit": "recorded cycles/s",
                 "n_gpus": world, "steps": S, "warmup": W, "ms_per_step": ms_max / S, "higher_is_better": True, "scaling": "weak",

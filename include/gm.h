@@ -493,14 +493,16 @@ int gm_head_update_backward(gm_ctx *ctx, gm_state *st, int n_cycles, int k, cons
  * the committed prefixes and replays the chains with the parameters as they are now (gm_head_prefill, gm_reconstruct),
  * evaluates the objective (gm_overlap, gm_dca_loss: Eq. 5-9), takes its gradient with respect to every parameter of the
  * head (gm_dca_grad, gm_head_update_backward) and applies AdamW to every tensor of the head's group (gm_adamw_step;
- * App. B).  Arguments as in those calls.
+ * App. B).  Arguments as in those calls, and the same numbers as those calls made one after the other - except that each
+ * chunk of max_batch chains is replayed once, its overlaps, logit gradients and backward pass following directly, so no
+ * [n_cycles, k, vocab] buffer exists.
  *   step         1, 2, 3, ... - the number of this update; must follow the context's previous one (GM_ERR_INVALID_ARG)
  *   lr           this update's learning rate (the caller applies the schedule: warm-up, cosine decay)
  *   mean_loss    device fp32 [1] out: the mean objective over the cycles BEFORE this update
  * The bf16 tensors the context was created with (head_proj, head_enorm, head_hnorm, head_final_norm and every tensor of
  * head_layer) are REWRITTEN IN PLACE; the backbone's tensors are read only.  fp32 master copies (initialised from the bf16
  * values at the first call), both moments, the gradients and the per-call buffers belong to the context and live until
- * gm_destroy (about 16 bytes per head parameter + 4 bytes x 2 x n_cycles x k x vocab).  The head cache of `st` is left as the
+ * gm_destroy (about 16 bytes per head parameter + 2 bytes x max_batch x max_k x vocab).  The head cache of `st` is left as the
  * rebuild with the parameters BEFORE the update wrote it.                                                               */
 int gm_head_update_step(gm_ctx *ctx, gm_state *st, int n_cycles, int k, float temperature, const int32_t *cycle_seq,
                         const gm_record *rec, const int32_t *seq_tok, int tok_stride, const int32_t *scratch_pages,

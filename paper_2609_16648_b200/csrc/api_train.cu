@@ -1,7 +1,8 @@
 // C ABI of libgm: one update of the draft head on recorded cycles (Alg. 1, "update phi"): cache rebuild and draft-path
 // reconstruction with the current parameters (Eq. 4), the objective (Eq. 5-9), its gradient with respect to every
 // parameter of the head, and AdamW on the head's parameter group (App. B).  Host code only: every step is one of the
-// library's own entry points; this file owns the optimizer state and the order of the calls.
+// library's own entry points or the driver behind gm_head_update_backward (which replays each chunk of chains once, for
+// the objective and for the backward pass alike); this file owns the optimizer state and the order of the calls.
 #include "gm_internal.h"
 
 namespace gm {
@@ -78,24 +79,19 @@ int gm_head_update_step(gm_ctx *c, gm_state *st, int n_cycles, int k, float temp
   }
   if (n_cycles > c->hu_cycles_cap) {
     const size_t rows = static_cast<size_t>(n_cycles) * k;
-    if ((rc = dev_alloc(c, &c->hu_logits, rows * c->V, false)) != GM_OK) return rc;
-    if ((rc = dev_alloc(c, &c->hu_glogits, rows * c->V, false)) != GM_OK) return rc;
     if ((rc = dev_alloc(c, &c->hu_alpha, rows)) != GM_OK) return rc;
     if ((rc = dev_alloc(c, &c->hu_lse, rows)) != GM_OK) return rc;
     if ((rc = dev_alloc(c, &c->hu_loss, static_cast<size_t>(n_cycles))) != GM_OK) return rc;
     c->hu_cycles_cap = n_cycles;
   }
-  // ---- forward: the head's cache over the committed prefixes and the chains, with the parameters as they are now ----
+  // ---- the head's cache over the committed prefixes, with the parameters as they are now ----
   if ((rc = gm_head_prefill(c, st, seq_hidden, hid_stride, seq_tok, tok_stride, seq_len, max_len)) != GM_OK) return rc;
-  if ((rc = gm_reconstruct(c, st, n_cycles, k, cycle_seq, rec, seq_tok, tok_stride, scratch_pages, c->hu_logits)) != GM_OK) return rc;
-  if ((rc = gm_overlap(c, n_cycles, k, temperature, c->hu_logits, rec, c->hu_alpha, c->hu_lse)) != GM_OK) return rc;
+  // ---- chunk by chunk: the chains replayed (Eq. 4), their overlaps and logit gradients, the backward pass; then the prefixes ----
+  if ((rc = head_update_backward_impl(c, st, n_cycles, k, cycle_seq, rec, seq_tok, tok_stride, scratch_pages, nullptr, seq_hidden,
+                                      hid_stride, seq_len, max_len, nullptr, nullptr, &c->hu_grads, temperature, c->hu_alpha,
+                                      c->hu_lse)) != GM_OK)
+    return rc;
   if ((rc = gm_dca_loss(c, n_cycles, k, c->hu_alpha, rec->accepted, c->hu_loss, mean_loss)) != GM_OK) return rc;
-  // ---- backward ----
-  if ((rc = gm_dca_grad(c, n_cycles, k, temperature, c->hu_logits, rec, c->hu_alpha, c->hu_lse, rec->accepted, c->hu_glogits)) != GM_OK)
-    return rc;
-  if ((rc = gm_head_update_backward(c, st, n_cycles, k, cycle_seq, rec, seq_tok, tok_stride, scratch_pages, c->hu_glogits, seq_hidden,
-                                    hid_stride, seq_len, max_len, nullptr, nullptr, &c->hu_grads)) != GM_OK)
-    return rc;
   // ---- AdamW on every tensor of the group; the bf16 copies the forward pass reads are rewritten in place ----
   ParamRef ps[13];
   const int np = collect_params(c, c->hu_grads, ps);

@@ -507,13 +507,27 @@ int gm_head_update_backward(gm_ctx *c, gm_state *st, int n_cycles, int k, const 
                             const int32_t *seq_tok, int tok_stride, const int32_t *scratch_pages, const void *grad_logits,
                             const void *seq_hidden, int hid_stride, const int32_t *seq_len, int max_len, float *dk_pool,
                             float *dv_pool, const gm_head_grads *out) {
+  if (!grad_logits) return GM_ERR_INVALID_ARG;
+  return head_update_backward_impl(c, st, n_cycles, k, cycle_seq, rec, seq_tok, tok_stride, scratch_pages, grad_logits, seq_hidden,
+                                   hid_stride, seq_len, max_len, dk_pool, dv_pool, out, 1.0f, nullptr, nullptr);
+}
+
+}  // extern "C"
+
+int gmh::head_update_backward_impl(gm_ctx *c, gm_state *st, int n_cycles, int k, const int32_t *cycle_seq, const gm_record *rec,
+                              const int32_t *seq_tok, int tok_stride, const int32_t *scratch_pages, const void *grad_logits,
+                              const void *seq_hidden, int hid_stride, const int32_t *seq_len, int max_len, float *dk_pool,
+                              float *dv_pool, const gm_head_grads *out, float temperature, float *alpha, float *lse) {
   NvtxRange nvtx_range("gm_head_update_backward");
   int rc = check_state(c, st, k);
   if (rc) return rc;
+  const bool own_grad = grad_logits == nullptr;          // the logit gradients are formed here, chunk by chunk
   if (n_cycles < 1 || !cycle_seq || !rec || !rec->start_hidden || !rec->start_pos || !rec->drafts || !seq_tok || tok_stride < 2 ||
-      !scratch_pages || !grad_logits || !seq_hidden || !seq_len || max_len < 2 || tok_stride < max_len || hid_stride < max_len - 1 ||
+      !scratch_pages || !seq_hidden || !seq_len || max_len < 2 || tok_stride < max_len || hid_stride < max_len - 1 ||
       (dk_pool != nullptr) != (dv_pool != nullptr) || !out)
     return GM_ERR_INVALID_ARG;
+  if (own_grad && (!alpha || !lse || !rec->top_index || !rec->top_logprob || !rec->accepted)) return GM_ERR_INVALID_ARG;
+  if (own_grad && (!(temperature > 0.f) || !std::isfinite(temperature))) return GM_ERR_UNSUPPORTED;
   const gm_config &cf = c->cfg;
   const gm_layer_weights &lw = c->w.head_layer;
   if (!out->proj || !out->enorm || !out->hnorm || !out->final_norm || !out->ln1 || !out->ln2 || !out->wqkv || !out->wo ||
@@ -523,7 +537,14 @@ int gm_head_update_backward(gm_ctx *c, gm_state *st, int n_cycles, int k, const 
   if (max_len + cf.max_k + 1 > cf.max_pages_per_seq * GM_PAGE) return GM_ERR_KV_CAPACITY;
   const int d = c->d, F = c->F, MB = cf.max_batch, PS = cf.max_k + 1, hd = cf.head_dim;
   const int B = st->batch, QT = cf.max_k + 1, VR = c->pf_vr, R = B * VR;
-  if (!c->v_table) return GM_ERR_INVALID_ARG;          // no reconstruction has run on this context
+  if (!c->v_table) {                                   // the chains' virtual state (as gm_reconstruct makes it)
+    const size_t MBs = static_cast<size_t>(MB);
+    if ((rc = dev_alloc(c, &c->v_kv_len, MBs)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->v_pending_n, MBs)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->v_pending_tok, MBs * PS)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->v_pending_hidden, MBs * PS * c->d)) != GM_OK) return rc;
+    if ((rc = dev_alloc(c, &c->v_table, MBs * cf.max_pages_per_seq)) != GM_OK) return rc;
+  }
   const int cap = std::max(MB, R * QT);
   if (cap > c->hub_rows_cap) {
     const size_t S = static_cast<size_t>(MB) * cf.max_k * d, M = static_cast<size_t>(cap) * d;
@@ -580,6 +601,21 @@ int gm_head_update_backward(gm_ctx *c, gm_state *st, int n_cycles, int k, const 
     if (rc) return rc;
     // every state's term through its own logits, and the final norm's weight
     const __nv_bfloat16 *gl = static_cast<const __nv_bfloat16 *>(grad_logits) + static_cast<size_t>(off) * k * c->V;
+    if (own_grad) {                                    // overlaps and objective gradient of this chunk, from the replay's logits
+      if (!c->hub_glogits && (rc = dev_alloc(c, &c->hub_glogits, static_cast<size_t>(MB) * cf.max_k * c->V, false)) != GM_OK) return rc;
+      const size_t ro = static_cast<size_t>(off) * k;
+      OverlapArgs O;
+      O.logits = c->ws_draft_logits; O.top_index = rec->top_index + ro * 64;
+      O.top_logprob = static_cast<const __nv_bfloat16 *>(rec->top_logprob) + ro * 64; O.alpha = alpha + ro; O.lse = lse + ro;
+      O.V = c->V; O.inv_temp = 1.0f / temperature;
+      GM_LAUNCH(c, GM_KC_RECORD, launch_overlap(O, m * k, c->stream));
+      DcaGradArgs G;
+      G.logits = c->ws_draft_logits; G.top_index = O.top_index; G.top_logprob = O.top_logprob; G.alpha = alpha + ro; G.lse = lse + ro;
+      G.accepted = rec->accepted + off; G.grad = c->hub_glogits; G.V = c->V; G.K = k; G.n = m; G.n_total = n_cycles;
+      G.inv_temp = O.inv_temp;
+      GM_LAUNCH(c, GM_KC_RECORD, launch_dca_grad(G, c->stream));
+      gl = c->hub_glogits;
+    }
     if ((rc = gm_head_state_grad(c, m * k, gl, c->hub_states, c->hub_gn, c->hub_dstate, 0)) != GM_OK) return rc;   // the LM head is the backbone's: its copy stays
     GM_LAUNCH(c, GM_KC_ELEMENTWISE,
               launch_rmsnorm_grad(c->hub_gn, c->hub_states, fnorm, nullptr, m * k, d, cf.rms_eps, c->stream, nullptr, c->hub_t));
@@ -647,5 +683,3 @@ int gm_head_update_backward(gm_ctx *c, gm_state *st, int n_cycles, int k, const 
   }
   return GM_OK;
 }
-
-}  // extern "C"

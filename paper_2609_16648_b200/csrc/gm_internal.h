@@ -131,7 +131,6 @@ struct gm_ctx {
   // tensors one after the other, each padded to 4 elements), per-call buffers
   gm_head_grads hu_grads = {};
   float *hu_master = nullptr, *hu_m = nullptr, *hu_v = nullptr;
-  __nv_bfloat16 *hu_logits = nullptr, *hu_glogits = nullptr;
   float *hu_alpha = nullptr, *hu_lse = nullptr, *hu_loss = nullptr;
   int hu_cycles_cap = 0, hu_step = 0;
   long long *hub_dk_fix = nullptr, *hub_dv_fix = nullptr, *hat_dq_fix = nullptr;   // fixed-point gradient accumulators of the driver
@@ -143,6 +142,7 @@ struct gm_ctx {
   float *hub_hidden = nullptr, *hub_z = nullptr, *hub_xmid = nullptr, *hub_dg = nullptr, *hub_dxmid = nullptr, *hub_dz = nullptr,
         *hub_dhid = nullptr, *hub_e = nullptr;                                                        // [rows, d]
   int32_t *hub_tok = nullptr, *hub_base = nullptr, *hub_cnt = nullptr;                               // [rows]
+  __nv_bfloat16 *hub_glogits = nullptr;                                                              // [max_batch, max_k, V] a chunk's logit gradients
   // attention half of the head's layer, backward: transposed weight copies and per-call scratch
   __nv_bfloat16 *hat_wo_t = nullptr, *hat_wqkv_t = nullptr;      // [q_dim, d], [d, n_qkv]
   CUtensorMap hat_wo_t_map, hat_wqkv_t_map;
@@ -261,6 +261,13 @@ int check_state(const gm_ctx *c, const gm_state *st, int k);
 cudaError_t run_sampler(gm_ctx *c, const SamplerArgs &S, int batch);
 int fill_sampler(gm_ctx *c, SamplerArgs &S, float temperature);
 // forced: draft_tok holds recorded drafts that are fed back instead of sampled ones (Eq. 4); nothing is drawn
+// The backward pass over recorded cycles (gm_head_update_backward).  grad_logits null: the logit gradients are formed chunk
+// by chunk from the replay's own logits (overlap and objective gradient at `temperature`, the mean over all n_cycles), and
+// alpha / lse [n_cycles, k] receive the overlaps and row statistics of every cycle.
+int head_update_backward_impl(gm_ctx *c, gm_state *st, int n_cycles, int k, const int32_t *cycle_seq, const gm_record *rec,
+                              const int32_t *seq_tok, int tok_stride, const int32_t *scratch_pages, const void *grad_logits,
+                              const void *seq_hidden, int hid_stride, const int32_t *seq_len, int max_len, float *dk_pool,
+                              float *dv_pool, const gm_head_grads *out, float temperature, float *alpha, float *lse);
 int draft_impl(gm_ctx *c, const gm_state *st, int k, float temperature, const uint32_t *u24_draft, uint64_t seed,
                uint64_t step, int32_t *draft_tok, void *draft_logits, float *dbg_q, bool forced);
 int spec_step_impl(gm_ctx *c, gm_state *st, int k, float temperature, const uint32_t *u24_draft,

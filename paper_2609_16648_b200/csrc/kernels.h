@@ -237,6 +237,7 @@ struct DcaGradArgs {
   __nv_bfloat16 *grad;                             // [n, K, V] out
   int V, K, n;
   float inv_temp;
+  int n_total = 0;                                 // cycles the mean runs over when these n are a part of them (0: n)
 };
 cudaError_t launch_dca_grad(const DcaGradArgs &A, cudaStream_t stream);
 // Rollout-time capture of the target hidden states of committed positions (App. D.2: the record keeps, per sequence,

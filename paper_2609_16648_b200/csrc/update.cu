@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(DG_THREADS) dca_grad_kernel(const DcaGradArgs 
       for (int l = 0; l < L; ++l) { if (l == kk) pre = run; run *= a[l]; M += run; }
       float D = 0.f, t = 1.f;
       for (int l = kk; l < L; ++l) { if (l > kk) t *= a[l]; D += t; }
-      if (M > 0.f) coef = -(pre * D / M) / static_cast<float>(A.n);
+      if (M > 0.f) coef = -(pre * D / M) / static_cast<float>(A.n_total > 0 ? A.n_total : A.n);
     }
   }
   if (coef == 0.f) {
