@@ -13,11 +13,11 @@ pytestmark = pytest.mark.gpu
 T = 0.2          # sharpens the nearly flat random-init distributions so that there is something to learn
 
 
-def test_rollout_record_update_rounds_raise_the_acceptance():
-    """Four rounds of (rollout of 12 cycles on 16 sequences with records, 20 updates on those 192 cycles).  The head starts
-    at random initialisation, independent of the target, so few drafts are accepted; every round's updates lower the
+def test_rollout_record_update_laps_raise_the_acceptance():
+    """Four laps of (rollout of 12 cycles on 16 sequences with records, 20 updates on those 192 cycles).  The head starts
+    at random initialisation, independent of the target, so few drafts are accepted; every lap's updates lower the
     objective (mean of Eq. 9) on its own records, and the accepted drafts per cycle of the NEXT rollout - same prompts, new
-    random draws, the updated head - rise well above the first round's.  On other prompts the gain is small (a
+    random draws, the updated head - rise well above the first lap's.  On other prompts the gain is small (a
     192-cycle training set on a toy model; measured 0.30 -> 0.38 / 0.45 / 0.43 on the default kernels) and within the
     sampling noise of 192 cycles under other kernel choices, so it is printed and only loosely bounded.  Everything goes through the C ABI: prefill,
     draft / verify / accept with gm_record_begin / gm_record_end and gm_capture_hidden, then gm_head_update_step."""
@@ -74,9 +74,9 @@ def test_rollout_record_update_rounds_raise_the_acceptance():
         return big, seq_tok, cur, capture, float(np.mean(np.concatenate(acc)))
 
     step, trained, other = 0, [], []
-    for rnd in range(4):
-        big, seq_tok, cur, capture, tau = rollout(3 + rnd, 5)
-        _, _, _, _, tau_other = rollout(100 + rnd, 77)                       # other prompts, other draws
+    for lap in range(4):
+        big, seq_tok, cur, capture, tau = rollout(3 + lap, 5)
+        _, _, _, _, tau_other = rollout(100 + lap, 77)                       # other prompts, other draws
         trained.append(tau)
         other.append(tau_other)
         st2 = gmb.State(ctx, B, pt, hpt)
@@ -93,8 +93,8 @@ def test_rollout_record_update_rounds_raise_the_acceptance():
             losses.append(float(mean[0]))
         assert gmb.gm_last_status(ctx) == 0
         assert all(np.isfinite(losses)) and losses[-1] < losses[0] - 0.02, losses
-        print(f"round {rnd}: accepted drafts per cycle {tau:.3f} (training prompts) {tau_other:.3f} (other prompts); "
-              f"objective over the round's updates {losses[0]:.3f} -> {losses[-1]:.3f}")
+        print(f"lap {lap}: accepted drafts per cycle {tau:.3f} (training prompts) {tau_other:.3f} (other prompts); "
+              f"objective over the lap's updates {losses[0]:.3f} -> {losses[-1]:.3f}")
     assert trained[-1] > trained[0] + 0.2 and min(trained[1:]) > trained[0] + 0.1       # measured 0.35 -> 0.70 / 0.80 / 0.87
     assert np.mean(other[1:]) >= other[0] - 0.1          # 192 cycles: a standard error of about 0.05 per figure
     ctx.close()
